@@ -1,0 +1,278 @@
+/* KVMem hot path, CPU oracle.  TEST INFRASTRUCTURE, NOT PRODUCT.
+ *
+ * A plain, slow, loop-nest statement of what one recall step computes: Mean-K index,
+ * query-conditioned block scores, selection under the active budget, execution-view
+ * assembly and GQA attention over the view.  Only tests, the smoke check and the
+ * benchmark's CPU-baseline leg may call it.  It shares no code with the CUDA library.
+ *
+ * Precision: bf16 inputs are widened exactly; every reduction accumulates in fp64
+ * (closer to the real-number result than either implementation), with one exception
+ * that is part of the contract: the Mean-K sum is fp32 in ascending token order followed
+ * by a single round-to-nearest-even to bf16, because the stored index is a quantised
+ * code and both sides must take that rounding decision in the same precision.
+ *
+ * Readings taken where the paper is silent (the full list is in the design notes):
+ * candidate set C = every block of the session, reserved blocks included; the selector
+ * alone applies sink/recent reservation; g(h) = h / (H/G); sum over query tokens, mean
+ * over layers and heads; ties broken by lower block id; partial blocks never indexed.
+ *
+ * OpenMP pragmas parallelise independent outer iterations only; no blocking, fusion or
+ * reordering inside a reduction.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef uint16_t bf16_t;
+
+static inline float bf16_to_f32(bf16_t h) {
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+static inline bf16_t f32_to_bf16_rne(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (bf16_t)((u >> 16) | 0x40u); /* NaN */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (bf16_t)(u >> 16);
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Mean-K index (Eq. "mean_k_index", Sec. 4.3):  kbar[l][b][g] = (1/|b|) sum_{i in b} k[l][i][g].
+ * K is token-major [n_blocks*B][L][G][d]; idx is [L][G][idx_stride][d], written at rows
+ * [b_first, b_first + n_blocks).  Only whole blocks exist, so |b| = B.
+ */
+void kvo_mean_k_index(const bf16_t* K, int64_t n_blocks, int B, int L, int G, int d,
+                      bf16_t* idx, int64_t idx_stride, int64_t b_first) {
+    const float inv = 1.0f / (float)B;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t b = 0; b < n_blocks; ++b)
+        for (int l = 0; l < L; ++l)
+            for (int g = 0; g < G; ++g)
+                for (int c = 0; c < d; ++c) {
+                    float acc = 0.0f;
+                    for (int t = 0; t < B; ++t)
+                        acc += bf16_to_f32(K[(((b * B + t) * L + l) * G + g) * (int64_t)d + c]);
+                    float mean = acc * inv;
+                    idx[((l * (int64_t)G + g) * idx_stride + b_first + b) * d + c] = f32_to_bf16_rne(mean);
+                }
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Block relevance (Eq. "kvmem-block-score", Sec. 4.3):
+ *   R_b = sum_m mean_{l,h} softmax_{b' in C}( q[l][m][h] . kbar[l][b'][g(h)] / sqrt(d) )_b
+ * q is [M][L][H][d]; idx is [L][G][idx_stride][d] of which the first NB rows are the
+ * candidate set C.  R is [NB].  R_g (may be NULL) is [G][NB]: the same sum restricted to
+ * the query heads of KV head g and averaged over them and over layers, so that
+ * R_b = (1/G) sum_g R_g[g][b].
+ * Returns 0, or -1 if the logit buffer cannot be allocated.
+ */
+int kvo_block_scores(const bf16_t* q, const bf16_t* idx, int64_t NB, int64_t idx_stride,
+                     int M, int L, int H, int G, int d, float* R, float* R_g) {
+    const int r = H / G;
+    const int64_t rows = (int64_t)L * M * H;
+    double* s = (double*)malloc(sizeof(double) * (size_t)rows * (size_t)NB);
+    double* mx = (double*)malloc(sizeof(double) * (size_t)rows);
+    double* Z = (double*)malloc(sizeof(double) * (size_t)rows);
+    if (!s || !mx || !Z) { free(s); free(mx); free(Z); return -1; }
+    const double inv_sqrt_d = 1.0 / sqrt((double)d);
+
+    /* scaled dot products, then the softmax statistics of each fixed (l, m, h) */
+#pragma omp parallel for schedule(static)
+    for (int64_t row = 0; row < rows; ++row) {
+        const int h = (int)(row % H);
+        const int m = (int)((row / H) % M);
+        const int l = (int)(row / ((int64_t)H * M));
+        const int g = h / r;
+        const bf16_t* qv = q + (((int64_t)m * L + l) * H + h) * d;
+        double* srow = s + row * NB;
+        double best = -INFINITY;
+        for (int64_t b = 0; b < NB; ++b) {
+            const bf16_t* kv = idx + ((l * (int64_t)G + g) * idx_stride + b) * d;
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c) acc += (double)bf16_to_f32(qv[c]) * (double)bf16_to_f32(kv[c]);
+            srow[b] = acc * inv_sqrt_d;
+            if (srow[b] > best) best = srow[b];
+        }
+        double sum = 0.0;
+        for (int64_t b = 0; b < NB; ++b) sum += exp(srow[b] - best);
+        mx[row] = best;
+        Z[row] = sum;
+    }
+
+    /* sum over query tokens, mean over (layer, head) pairs */
+#pragma omp parallel for schedule(static)
+    for (int64_t b = 0; b < NB; ++b) {
+        double total = 0.0;
+        for (int g = 0; g < G; ++g) {
+            double part = 0.0;
+            for (int l = 0; l < L; ++l)
+                for (int m = 0; m < M; ++m)
+                    for (int h = g * r; h < (g + 1) * r; ++h) {
+                        const int64_t row = ((int64_t)l * M + m) * H + h;
+                        part += exp(s[row * NB + b] - mx[row]) / Z[row];
+                    }
+            if (R_g) R_g[(int64_t)g * NB + b] = (float)(part / ((double)L * r));
+            total += part;
+        }
+        R[b] = (float)(total / ((double)L * H));
+    }
+    free(s); free(mx); free(Z);
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Budget (Eq. "active_budget" and Eq. "active_capacity", Sec. 3.1):
+ *   N(Q) + B * |R| <= B_a  =>  k = min(budget_blocks, floor((B_a - N(Q)) / B), NB), never below 0.
+ */
+int64_t kvo_budget_blocks(int64_t NB, int B, int64_t budget_blocks, int64_t max_view_tokens,
+                          int64_t mandatory_tokens) {
+    int64_t room = max_view_tokens - mandatory_tokens;
+    int64_t k = room > 0 ? room / B : 0;
+    if (budget_blocks < k) k = budget_blocks;
+    if (NB < k) k = NB;
+    if (k < 0) k = 0;
+    return k;
+}
+
+typedef struct { float score; int32_t id; } kvo_cand_t;
+
+static int kvo_cand_cmp(const void* a, const void* b) {
+    const kvo_cand_t* x = (const kvo_cand_t*)a;
+    const kvo_cand_t* y = (const kvo_cand_t*)b;
+    if (x->score > y->score) return -1;
+    if (x->score < y->score) return 1;
+    return (x->id > y->id) - (x->id < y->id);           /* equal score: lower id first */
+}
+
+static int kvo_i32_cmp(const void* a, const void* b) {
+    int32_t x = *(const int32_t*)a, y = *(const int32_t*)b;
+    return (x > y) - (x < y);
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Selector (Sec. 4.3, last paragraph of "Query-Conditioned Block Scoring"; Sec. 5.2):
+ * reserve the sink (oldest) and recent (newest) blocks, fill the rest of the budget with
+ * the largest R_b, restore chronological order.  Writes k ascending ids; returns k.
+ */
+int64_t kvo_select(const float* R, int64_t NB, int B, int64_t budget_blocks, int64_t max_view_tokens,
+                   int64_t mandatory_tokens, int64_t n_sink, int64_t n_recent, int32_t* sel) {
+    const int64_t k = kvo_budget_blocks(NB, B, budget_blocks, max_view_tokens, mandatory_tokens);
+    if (k == 0) return 0;
+    char* taken = (char*)calloc((size_t)NB, 1);
+    kvo_cand_t* cand = (kvo_cand_t*)malloc(sizeof(kvo_cand_t) * (size_t)NB);
+    int64_t n = 0;
+    if (n_sink < 0) n_sink = 0;
+    if (n_recent < 0) n_recent = 0;
+    for (int64_t b = 0; b < NB && b < n_sink && n < k; ++b)            /* sinks, oldest first   */
+        if (!taken[b]) { taken[b] = 1; sel[n++] = (int32_t)b; }
+    for (int64_t j = 0; j < n_recent && j < NB && n < k; ++j) {         /* recents, newest first */
+        int64_t b = NB - 1 - j;
+        if (!taken[b]) { taken[b] = 1; sel[n++] = (int32_t)b; }
+    }
+    int64_t nc = 0;
+    for (int64_t b = 0; b < NB; ++b)
+        if (!taken[b]) { cand[nc].score = R[b]; cand[nc].id = (int32_t)b; ++nc; }
+    qsort(cand, (size_t)nc, sizeof(kvo_cand_t), kvo_cand_cmp);          /* total order: no ties left */
+    for (int64_t i = 0; i < nc && n < k; ++i) sel[n++] = cand[i].id;
+    qsort(sel, (size_t)n, sizeof(int32_t), kvo_i32_cmp);                /* chronological order   */
+    free(taken); free(cand);
+    return n;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Repository: physical pages hold B tokens each, token-major inside the page
+ * ([n_pages][B][L][G][d]); logical block b of a session lives in page table[b].
+ */
+void kvo_place_blocks(const bf16_t* K, const bf16_t* V, int64_t n_blocks, int B, int L, int G, int d,
+                      const int32_t* table, bf16_t* pagesK, bf16_t* pagesV) {
+    const size_t page = (size_t)B * L * G * d;
+    for (int64_t b = 0; b < n_blocks; ++b) {
+        memcpy(pagesK + (size_t)table[b] * page, K + (size_t)b * page, page * sizeof(bf16_t));
+        memcpy(pagesV + (size_t)table[b] * page, V + (size_t)b * page, page * sizeof(bf16_t));
+    }
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Execution view (Sec. 4.4, "execution view"; Sec. 5.2): the selected blocks, in
+ * chronological order, at contiguous compact positions: view token j*B + t is token t of
+ * block sel[j], read through the block table.  View layout [L][G][cap_tokens][d].
+ * K is copied unchanged (keys are position-independent on this path).
+ */
+void kvo_gather(const bf16_t* pagesK, const bf16_t* pagesV, const int32_t* table,
+                const int32_t* sel, int64_t n_sel, int B, int L, int G, int d,
+                bf16_t* viewK, bf16_t* viewV, int64_t cap_tokens) {
+    const size_t page = (size_t)B * L * G * d;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n_sel; ++j) {
+        const size_t src = (size_t)table[sel[j]] * page;
+        for (int t = 0; t < B; ++t)
+            for (int l = 0; l < L; ++l)
+                for (int g = 0; g < G; ++g) {
+                    const size_t s = src + (((size_t)t * L + l) * G + g) * d;
+                    const size_t o = (((size_t)l * G + g) * cap_tokens + (size_t)j * B + t) * d;
+                    memcpy(viewK + o, pagesK + s, (size_t)d * sizeof(bf16_t));
+                    memcpy(viewV + o, pagesV + s, (size_t)d * sizeof(bf16_t));
+                }
+    }
+}
+
+/* ---------------------------------------------------------------------------------------
+ * GQA attention over the first T view tokens, no mask (every query token of the step sees
+ * the whole recalled history):  o = softmax(q K^T * scale) V,  lse = ln sum_t exp(s_t).
+ * q [M][L][H][d]; view [L][G][cap_tokens][d]; out [M][L][H][d] fp32; lse [M][L][H] fp32.
+ * T = 0 gives o = 0 and lse = -inf.
+ */
+void kvo_attend(const bf16_t* q, const bf16_t* viewK, const bf16_t* viewV, int64_t T, int64_t cap_tokens,
+                int M, int L, int H, int G, int d, double scale, float* out, float* lse) {
+    const int r = H / G;
+    const int64_t rows = (int64_t)M * L * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t row = 0; row < rows; ++row) {
+        const int h = (int)(row % H);
+        const int l = (int)((row / H) % L);
+        const int g = h / r;
+        const bf16_t* qv = q + row * d;
+        const bf16_t* Kg = viewK + ((size_t)l * G + g) * (size_t)cap_tokens * d;
+        const bf16_t* Vg = viewV + ((size_t)l * G + g) * (size_t)cap_tokens * d;
+        double* s = (double*)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1));
+        double* o = (double*)calloc((size_t)d, sizeof(double));
+        double best = -INFINITY;
+        for (int64_t t = 0; t < T; ++t) {
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c)
+                acc += (double)bf16_to_f32(qv[c]) * (double)bf16_to_f32(Kg[(size_t)t * d + c]);
+            s[t] = acc * scale;
+            if (s[t] > best) best = s[t];
+        }
+        double sum = 0.0;
+        for (int64_t t = 0; t < T; ++t) sum += exp(s[t] - best);
+        for (int64_t t = 0; t < T; ++t) {
+            const double p = exp(s[t] - best) / sum;
+            for (int c = 0; c < d; ++c) o[c] += p * (double)bf16_to_f32(Vg[(size_t)t * d + c]);
+        }
+        for (int c = 0; c < d; ++c) out[row * d + c] = (float)o[c];
+        lse[row] = T > 0 ? (float)(best + log(sum)) : -INFINITY;
+        free(s); free(o);
+    }
+}
+
+/* Threads the parallel loops above will use (reported next to the timed baseline). */
+int kvo_threads(void) {
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp single
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}

@@ -1,0 +1,172 @@
+"""ctypes wrapper of the CPU oracle (``kvmem_oracle.c``).  TEST INFRASTRUCTURE, NOT PRODUCT.
+
+Only ``tests/``, the smoke check and the benchmark's CPU-baseline leg may import this.
+It imports nothing from the CUDA package.  Arrays are NumPy; bf16 tensors travel as
+``uint16`` bit patterns (``torch_tensor.view(torch.int16).numpy().view(np.uint16)``).
+
+Parity pins: every function here is pinned by ``tests/test_oracle_pins.py`` against closed
+forms, invariants of the equations, special cases that reduce to textbook softmax
+attention, and brute force on tiny inputs.  What stays *parity unpinned* is only what the
+paper never prints: the authors' sink/recent sizes, whether their candidate set excludes
+reserved blocks, their index element type, their query-head to KV-head mapping and their
+tie-break.  The readings taken are stated in ``kvmem_oracle.c``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "kvmem_oracle.c")
+_LIB = os.path.join(_HERE, "libkvmem_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        i64, i32, dbl, p = C.c_int64, C.c_int, C.c_double, C.c_void_p
+        L.kvo_mean_k_index.argtypes = [p, i64, i32, i32, i32, i32, p, i64, i64]
+        L.kvo_mean_k_index.restype = None
+        L.kvo_block_scores.argtypes = [p, p, i64, i64, i32, i32, i32, i32, i32, p, p]
+        L.kvo_block_scores.restype = i32
+        L.kvo_budget_blocks.argtypes = [i64, i32, i64, i64, i64]
+        L.kvo_budget_blocks.restype = i64
+        L.kvo_select.argtypes = [p, i64, i32, i64, i64, i64, i64, i64, p]
+        L.kvo_select.restype = i64
+        L.kvo_place_blocks.argtypes = [p, p, i64, i32, i32, i32, i32, p, p, p]
+        L.kvo_place_blocks.restype = None
+        L.kvo_gather.argtypes = [p, p, p, p, i64, i32, i32, i32, i32, p, p, i64]
+        L.kvo_gather.restype = None
+        L.kvo_attend.argtypes = [p, p, p, i64, i64, i32, i32, i32, i32, i32, dbl, p, p]
+        L.kvo_attend.restype = None
+        L.kvo_threads.argtypes = []
+        L.kvo_threads.restype = i32
+        _lib = L
+    return _lib
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _u16(a: np.ndarray) -> np.ndarray:
+    assert a.dtype == np.uint16 and a.flags.c_contiguous, "bf16 bit patterns as contiguous uint16"
+    return a
+
+
+def threads() -> int:
+    return int(lib().kvo_threads())
+
+
+def bf16_bits_to_f32(a: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns (uint16) to fp32 (for use in tests)."""
+    return (a.astype(np.uint32) << 16).view(np.float32)
+
+
+def mean_k_index(K: np.ndarray, B: int, idx: Optional[np.ndarray] = None, b_first: int = 0) -> np.ndarray:
+    """K: uint16 [n_blocks*B][L][G][d]  ->  idx uint16 [L][G][stride][d] (rows b_first.. filled)."""
+    _u16(K)
+    n_tok, L, G, d = K.shape
+    assert n_tok % B == 0, "only whole blocks are indexed"
+    nb = n_tok // B
+    if idx is None:
+        idx = np.zeros((L, G, b_first + nb, d), dtype=np.uint16)
+    _u16(idx)
+    assert idx.shape[0] == L and idx.shape[1] == G and idx.shape[3] == d and idx.shape[2] >= b_first + nb
+    lib().kvo_mean_k_index(_ptr(K), nb, B, L, G, d, _ptr(idx), idx.shape[2], b_first)
+    return idx
+
+
+def block_scores(q: np.ndarray, idx: np.ndarray, NB: int) -> Tuple[np.ndarray, np.ndarray]:
+    """q uint16 [M][L][H][d], idx uint16 [L][G][stride][d]  ->  (R fp32 [NB], R_g fp32 [G][NB])."""
+    _u16(q), _u16(idx)
+    M, L, H, d = q.shape
+    G = idx.shape[1]
+    assert idx.shape[0] == L and idx.shape[3] == d and H % G == 0 and NB <= idx.shape[2]
+    R = np.zeros(NB, dtype=np.float32)
+    Rg = np.zeros((G, NB), dtype=np.float32)
+    rc = lib().kvo_block_scores(_ptr(q), _ptr(idx), NB, idx.shape[2], M, L, H, G, d, _ptr(R), _ptr(Rg))
+    if rc != 0:
+        raise MemoryError("oracle: logit buffer allocation failed")
+    return R, Rg
+
+
+def budget_blocks(NB: int, B: int, budget_blocks: int, max_view_tokens: int, mandatory_tokens: int = 0) -> int:
+    return int(lib().kvo_budget_blocks(NB, B, budget_blocks, max_view_tokens, mandatory_tokens))
+
+
+def select(R: np.ndarray, B: int, budget_blocks: int, max_view_tokens: int, mandatory_tokens: int = 0,
+           n_sink_blocks: int = 0, n_recent_blocks: int = 0) -> np.ndarray:
+    """R fp32 [NB] -> ascending int32 ids of the selected blocks."""
+    assert R.dtype == np.float32 and R.flags.c_contiguous
+    NB = R.shape[0]
+    sel = np.zeros(max(NB, 1), dtype=np.int32)
+    n = lib().kvo_select(_ptr(R), NB, B, budget_blocks, max_view_tokens, mandatory_tokens,
+                         n_sink_blocks, n_recent_blocks, _ptr(sel))
+    return sel[:n].copy()
+
+
+@dataclass
+class Repository:
+    """Physical pages [n_pages][B][L][G][d] (uint16) for K and V."""
+    pagesK: np.ndarray
+    pagesV: np.ndarray
+
+    @classmethod
+    def empty(cls, n_pages: int, B: int, L: int, G: int, d: int) -> "Repository":
+        return cls(np.zeros((n_pages, B, L, G, d), np.uint16), np.zeros((n_pages, B, L, G, d), np.uint16))
+
+    def place(self, K: np.ndarray, V: np.ndarray, table: np.ndarray) -> None:
+        """Copy whole blocks K, V (uint16 [n_blocks*B][L][G][d]) into pages table[0..n_blocks)."""
+        _u16(K), _u16(V)
+        _, B, L, G, d = self.pagesK.shape
+        nb = K.shape[0] // B
+        assert K.shape[0] == nb * B and table.dtype == np.int32 and table.shape[0] >= nb
+        assert int(table[:nb].max(initial=-1)) < self.pagesK.shape[0] and int(table[:nb].min(initial=0)) >= 0
+        lib().kvo_place_blocks(_ptr(K), _ptr(V), nb, B, L, G, d, _ptr(np.ascontiguousarray(table)),
+                               _ptr(self.pagesK), _ptr(self.pagesV))
+
+
+def gather(repo: Repository, table: np.ndarray, sel: np.ndarray, cap_tokens: int,
+           viewK: Optional[np.ndarray] = None, viewV: Optional[np.ndarray] = None
+           ) -> Tuple[np.ndarray, np.ndarray]:
+    """Execution view uint16 [L][G][cap_tokens][d] x2 (tokens beyond len(sel)*B left as they were)."""
+    _, B, L, G, d = repo.pagesK.shape
+    assert table.dtype == np.int32 and sel.dtype == np.int32 and len(sel) * B <= cap_tokens
+    if viewK is None:
+        viewK = np.zeros((L, G, cap_tokens, d), np.uint16)
+        viewV = np.zeros((L, G, cap_tokens, d), np.uint16)
+    lib().kvo_gather(_ptr(repo.pagesK), _ptr(repo.pagesV), _ptr(np.ascontiguousarray(table)),
+                     _ptr(np.ascontiguousarray(sel)), len(sel), B, L, G, d, _ptr(viewK), _ptr(viewV), cap_tokens)
+    return viewK, viewV
+
+
+def attend(q: np.ndarray, viewK: np.ndarray, viewV: np.ndarray, T: int, scale: Optional[float] = None
+           ) -> Tuple[np.ndarray, np.ndarray]:
+    """q uint16 [M][L][H][d]; views uint16 [L][G][cap][d]  ->  (O fp32 [M][L][H][d], LSE fp32 [M][L][H])."""
+    _u16(q), _u16(viewK), _u16(viewV)
+    M, L, H, d = q.shape
+    G, cap = viewK.shape[1], viewK.shape[2]
+    assert viewK.shape == viewV.shape and viewK.shape[0] == L and viewK.shape[3] == d and T <= cap
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    out = np.zeros((M, L, H, d), np.float32)
+    lse = np.zeros((M, L, H), np.float32)
+    lib().kvo_attend(_ptr(q), _ptr(viewK), _ptr(viewV), T, cap, M, L, H, G, d, float(scale), _ptr(out), _ptr(lse))
+    return out, lse
