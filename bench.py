@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the KVMem recall step (select + materialize + attend) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1m] [--impl native|reference]
+
+One "step" is one pass of the whole hot path over one seeded query set: block scoring through
+the Mean-K index, selection under the budget, execution-view assembly, GQA decode attention.
+The history stays resident in HBM; the 16 query sets of the workload are cycled.  Rank 0 prints
+ONE JSON line.  With N > 1 (launched by torch.distributed.run) every rank owns an independent
+session replica on its own GPU (the path shards by session, no collective on the data path);
+the timed region is bracketed by a barrier and the maximum over ranks is reported.
+
+``--impl reference`` times the CPU oracle, as it stands, on the host cores, on a bounded sample
+of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from kvmem_workloads import CONFIGS, kv_blocks, make_queries, page_table, select_params  # noqa: E402
+
+METRIC = "select+materialize+attend steps/s"
+UNIT = "steps/s"
+KERNELS_PER_STEP = 6      # score_logits, score_finish, topk, gather, attend_split, attend_merge
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def algorithmic_bytes(spec, k):
+    """Bytes the method must move per step (per session): index read + view read/write + view read."""
+    view = 2 * k * spec.block_tokens * spec.n_layers * spec.n_kv_heads * spec.head_dim * 2       # K and V, bf16
+    index = spec.n_blocks * spec.n_layers * spec.n_kv_heads * spec.head_dim * 2
+    return {"index": index, "gather": 2 * view, "attend": view if spec.attend else 0,
+            "total": index + 2 * view + (view if spec.attend else 0)}
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+        self.t_start = self.t_stop = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def window(self, t0, t1):
+        self.t_start, self.t_stop = t0, t1
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for t, line in self.rows:
+            if self.t_start is not None and not (self.t_start <= t <= self.t_stop + 0.05):
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- native arm
+
+def fill_pool(spec, device, seed_shift=0):
+    from paper_2609_04852_b200 import Pool
+    spec = spec.with_(seed=spec.seed + seed_shift)
+    pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.block_tokens,
+                spec.n_sessions, spec.n_sessions * spec.n_blocks, spec.n_blocks, device.index)
+    tables = page_table(spec)
+    for s in range(spec.n_sessions):
+        for b0 in range(0, spec.n_blocks, 1024):
+            b1 = min(spec.n_blocks, b0 + 1024)
+            K, V = kv_blocks(spec, s, b0, b1, device)
+            pool.append_blocks(s, K, V, tables[s, b0:b1].tolist())
+        torch.cuda.synchronize(device)
+    return pool, spec
+
+
+def run_native(args):
+    import torch.distributed as dist
+    from paper_2609_04852_b200 import SelectParams
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world and world > 1:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    base = CONFIGS[args.workload]
+    if not base.attend:
+        raise SystemExit(f"workload {base.name} has no attend stage; the benchmark times the whole step")
+    pool, spec = fill_pool(base, device, seed_shift=1000 * rank)     # one independent replica per rank
+    ns, M, B = spec.n_sessions, spec.n_q_tokens, spec.block_tokens
+    prm = SelectParams(**select_params(spec))
+    from paper_2609_04852_b200 import budget_blocks
+    k = budget_blocks(prm, B, spec.n_blocks)
+    cap = k * B
+    qsets = [make_queries(spec, i) for i in range(spec.n_query_sets)]
+    q_dev = [q.to(device) for q in qsets]
+    q_pin = [q.pin_memory() for q in qsets]
+    sel = torch.zeros(ns, k, dtype=torch.int32, device=device)
+    n_sel = torch.zeros(ns, dtype=torch.int32, device=device)
+    view = pool.new_view(ns, cap)
+    out, lse = pool.new_outputs(ns, M)
+    out_pin = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+    lse_pin = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device) if args.flush_l2 else None
+    stream = torch.cuda.current_stream(device)
+
+    def step(i, ev=None):
+        q = q_dev[i % len(q_dev)]
+        pool.select(q, prm, sel, n_sel)
+        if ev is not None:
+            ev[0].record(stream)
+        pool.materialize(sel, n_sel, view)
+        if ev is not None:
+            ev[1].record(stream)
+        if spec.attend:
+            pool.view_attend(q, view, n_sel, out, lse)
+        if ev is not None:
+            ev[2].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize(device)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    assert pool.device_status() == 0, "device status word set during warm-up"
+    assert int(n_sel.min()) == k, "selection did not fill the budget"
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+
+    # ---- timed region: K steps, device-timed, inputs resident in HBM
+    K = args.steps
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    begins = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    e0.record(stream)
+    for i in range(K):
+        if flush is not None:
+            flush.fill_(i & 255)
+        begins[i].record(stream)
+        step(i, marks[i])
+    e1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    total_ms = e0.elapsed_time(e1)
+    step_ms = [begins[i].elapsed_time(marks[i][2]) for i in range(K)]
+    sel_ms = [begins[i].elapsed_time(marks[i][0]) for i in range(K)]
+    gat_ms = [marks[i][0].elapsed_time(marks[i][1]) for i in range(K)]
+    att_ms = [marks[i][1].elapsed_time(marks[i][2]) for i in range(K)]
+    if flush is not None:
+        total_ms = sum(step_ms)          # the flush writes are not part of a step
+    sampler.window(t_wall0, t_wall1)
+    assert pool.device_status() == 0, "device status word set during the timed region"
+
+    # ---- end-to-end: query from pinned host memory, results read back to the host, every step
+    Ke = min(K, 200)
+    barrier()
+    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ee0.record(stream)
+    for i in range(Ke):
+        pool.recall_step_host(q_pin[i % len(q_pin)], prm, sel, n_sel, view, out_pin, lse_pin)
+    ee1.record(stream)
+    barrier()
+    e2e_ms = ee0.elapsed_time(ee1)
+    # keep sampling clocks long enough to see the load even when K is small
+    if rank == 0 and (t_wall1 - t_wall0) < 0.5:
+        t_wall0 = time.time()
+        t_end = t_wall0 + 0.6
+        i = 0
+        while time.time() < t_end:
+            step(i); i += 1
+            if i % 50 == 0:
+                torch.cuda.synchronize(device)
+        torch.cuda.synchronize(device)
+        sampler.window(t_wall0, time.time())
+        clock_note = "timed region shorter than the sampling period: clocks sampled over an identical 0.6 s loop right after it"
+    else:
+        clock_note = "sampled during the timed region"
+
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(times[0]), float(times[1])
+
+    if rank == 0:
+        clocks = sampler.stop()
+        clocks["note"] = clock_note
+        peaks = measured_peaks()
+        ab = algorithmic_bytes(spec, k)
+        med = statistics.median
+        gather_s = (sum(gat_ms) / K) * 1e-3
+        gather_gbs = ns * ab["gather"] / gather_s / 1e9
+        step_gbs = world * K * ns * ab["total"] / (total_ms * 1e-3) / 1e9 / world      # per GPU
+        rows = ns * M * spec.n_layers * spec.n_q_heads
+        line = {
+            "metric": METRIC, "value": world * K / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded; shapes of the paper's agent workspaces)",
+            "config": {"workload": f"{spec.name}: {ns} session(s) x {spec.n_blocks} blocks of {B} tokens "
+                                   f"({spec.tokens} tokens history), {M} query token(s), {spec.n_q_heads}/{spec.n_kv_heads} heads, "
+                                   f"d={spec.head_dim}, budget {k} blocks ({cap} view tokens)",
+                       "history_tokens": spec.tokens, "view_tokens": cap, "query_sets": len(qsets),
+                       "l2": "flushed between steps (256 MiB write)" if flush is not None else
+                             "no flush: every step streams far more than the 126 MB L2",
+                       "parallelism": f"{world} independent session replica(s), one per GPU"},
+            "e2e": {"value": world * Ke / (e2e_ms * 1e-3), "unit": UNIT, "steps": Ke,
+                    "h2d_bytes_per_step": rows * spec.head_dim * 2,
+                    "d2h_bytes_per_step": rows * spec.head_dim * 4 + rows * 4,
+                    "api": "kvmem_recall_step_host (pinned host query in, host O and LSE out, synchronous)"},
+            "gpu_launches": K * KERNELS_PER_STEP,
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "gather_bulk_kernel (kvmem_materialize)",
+                         "achieved": gather_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gather_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+                         "algorithmic_bytes_per_launch": ns * ab["gather"], "avg_launch_ms": gather_s * 1e3,
+                         "traffic": None},
+            "step_hbm": {"algorithmic_bytes_per_step": ns * ab["total"], "achieved_gbs": step_gbs,
+                         "frac_of_peak": step_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+                         "nominal_peak_gbs": 8000.0},
+            "stages_ms": {"select": med(sel_ms), "materialize": med(gat_ms), "attend": med(att_ms),
+                          "step_median": med(step_ms), "step_min": min(step_ms)},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(base, args.cpu_sample_blocks)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- oracle arm / CPU baseline
+
+def _bits(t):
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+class OracleSample:
+    """The oracle on a bounded sample of a workload: scoring and selection over the whole index,
+    view assembly and attention over the first `sample_blocks` selected blocks (cost scaled to k)."""
+
+    def __init__(self, spec, sample_blocks):
+        from oracle import kvmem_oracle as orc
+        self.orc, self.spec = orc, spec
+        gen_dev = torch.device("cuda", 0) if torch.cuda.is_available() else "cpu"
+        nb = spec.n_blocks
+        self.idx = np.zeros((spec.n_layers, spec.n_kv_heads, nb, spec.head_dim), np.uint16)
+        for b0 in range(0, nb, 1024):                                  # setup, untimed: the oracle's own index
+            b1 = min(nb, b0 + 1024)
+            K, _ = kv_blocks(spec, 0, b0, b1, gen_dev)
+            orc.mean_k_index(_bits(K), spec.block_tokens, self.idx, b0)
+        prm = select_params(spec)
+        self.k = orc.budget_blocks(nb, spec.block_tokens, prm["budget_blocks"], prm["max_view_tokens"])
+        self.sample_blocks = min(sample_blocks, self.k)
+        self.prm = prm
+        self.gen_dev = gen_dev
+        self.repo = None
+
+    def _repo_for(self, ids):
+        """Pages of the sampled blocks only (setup, untimed)."""
+        spec, orc = self.spec, self.orc
+        repo = orc.Repository.empty(len(ids), spec.block_tokens, spec.n_layers, spec.n_kv_heads, spec.head_dim)
+        table = np.full(spec.n_blocks, -1, np.int32)
+        for j, b in enumerate(ids):
+            K, V = kv_blocks(spec, 0, int(b), int(b) + 1, self.gen_dev)
+            repo.place(_bits(K), _bits(V), np.array([j], np.int32))
+            table[b] = j
+        return repo, table
+
+    def step(self, qset):
+        """Returns (seconds for a whole step, scaled from the sample)."""
+        spec, orc = self.spec, self.orc
+        qb = _bits(make_queries(spec, qset))[0]
+        t0 = time.perf_counter()
+        R, _ = orc.block_scores(qb, self.idx, spec.n_blocks)
+        sel = orc.select(R, spec.block_tokens, self.prm["budget_blocks"], self.prm["max_view_tokens"])
+        t1 = time.perf_counter()
+        ids = sel[: self.sample_blocks]
+        repo, table = self._repo_for(ids)                               # untimed: materialise the sample's pages
+        t2 = time.perf_counter()
+        cap = len(ids) * spec.block_tokens
+        vK, vV = orc.gather(repo, table, np.ascontiguousarray(ids), cap)
+        if spec.attend:
+            orc.attend(qb, vK, vV, cap)
+        t3 = time.perf_counter()
+        scale = len(sel) / max(len(ids), 1)
+        return (t1 - t0) + (t3 - t2) * scale
+
+
+def cpu_baseline(spec, sample_blocks, steps=1):
+    from oracle import kvmem_oracle as orc
+    smp = OracleSample(spec, sample_blocks)
+    secs = [smp.step(i) for i in range(steps)]
+    t = sum(secs) / len(secs)
+    return {"value": 1.0 / t, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
+            "sample": f"session 0: scoring + selection over all {spec.n_blocks} blocks timed in full; view assembly + "
+                      f"attention timed on the first {smp.sample_blocks} of {smp.k} selected blocks and scaled by "
+                      f"{smp.k / max(smp.sample_blocks, 1):.1f}x; {steps} step(s); oracle seconds per step = {t:.2f}"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import kvmem_oracle as orc
+    spec = CONFIGS[args.workload]
+    smp = OracleSample(spec, args.cpu_sample_blocks)
+    for i in range(min(args.warmup, 1)):
+        smp.step(i)
+    K = max(1, min(args.steps, 3))
+    secs = [smp.step(i) for i in range(K)]
+    t = sum(secs) / K
+    value = 1.0 / t
+    sample = (f"scoring + selection over all {spec.n_blocks} blocks in full; view assembly + attention on the first "
+              f"{smp.sample_blocks} of {smp.k} selected blocks, scaled by {smp.k / max(smp.sample_blocks, 1):.1f}x")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+            "warmup": min(args.warmup, 1), "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64 accumulation on bf16 inputs", "data": "synthetic (seeded)",
+            "config": {"workload": f"{spec.name}: {spec.n_blocks} blocks of {spec.block_tokens} tokens, "
+                                   f"{spec.n_q_tokens} query token(s), budget {smp.k} blocks"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["native", "reference"], default="native")
+    ap.add_argument("--workload", choices=sorted(CONFIGS), default="1m")
+    ap.add_argument("--flush-l2", action="store_true", help="write 256 MiB between steps (for workloads near L2 size)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-blocks", type=int, default=256)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the native arm")
+        run_native(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,208 @@
+/* kvmem.h - C ABI of the KVMem recall step on one NVIDIA B200 (sm_100a).
+ *
+ * One recall step (paper Sec. 4.1, Sec. 5.2): score every historical paged-KV block of a
+ * session against the current query through the Mean-K attention-space index, select the
+ * top blocks under the active-context budget, assemble the query-dependent execution
+ * view from the block table, and run GQA decode attention over that view.
+ *
+ * Conventions
+ *   - Every pointer is marked HOST or DEVICE.  Device buffers, including the pool's backing
+ *     storage, views, outputs and workspaces, are owned by the caller; the library owns only
+ *     the opaque handle and its host-side metadata and never allocates device memory.
+ *   - All device work is enqueued on the given stream (a cudaStream_t passed as void*) and is
+ *     asynchronous unless a call says otherwise.  A pool is not thread-safe.
+ *   - Every call returns a kvmem_status_t.  Argument, state and capacity errors are detected
+ *     on the host before anything is enqueued and leave the pool unchanged; kvmem_last_error()
+ *     then describes the failure.  Anomalies seen on the device (a block id out of range, a
+ *     bounded wait that expired) set a sticky status word read by kvmem_device_status().
+ *   - Element type of K, V, q and the index is bf16 (2 bytes).  Scores, attention outputs
+ *     and log-sum-exp values are fp32.
+ *   - Logical block ids are the append order within a session, i.e. chronological order
+ *     (Sec. 5.2, block records).  Only whole blocks of block_tokens tokens exist: the Mean-K
+ *     index covers completed blocks only (Sec. 5.2).
+ *   - Keys and queries are taken to be position-independent already (Sec. 4.3, "Mean-K
+ *     Retrieval-Index Construction"); K is copied into the view unchanged.
+ *   - Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ */
+#ifndef KVMEM_H_
+#define KVMEM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvmem_pool kvmem_pool_t; /* opaque; created and destroyed by the library */
+
+typedef enum {
+    KVMEM_OK = 0,
+    KVMEM_E_INVALID = -1,     /* bad argument (null, out of range, misaligned, partial block)   */
+    KVMEM_E_CAPACITY = -2,    /* pool, session or caller buffer too small                       */
+    KVMEM_E_STATE = -3,       /* page already in use, session empty, stale handle               */
+    KVMEM_E_CUDA = -4,        /* a CUDA runtime or driver call failed                           */
+    KVMEM_E_TIMEOUT = -5,     /* device status: a bounded wait inside a kernel gave up          */
+    KVMEM_E_UNSUPPORTED = -6, /* shape outside what the kernels were built for                  */
+    KVMEM_E_DEVICE_RANGE = -7 /* device status: a block or page id was out of range and skipped */
+} kvmem_status_t;
+
+/* Geometry of the paged KV repository (Sec. 3.1: logical blocks of B_blk tokens; Sec. 5.2:
+ * blocks aligned with physical pages). */
+typedef struct {
+    int32_t n_layers;               /* scored attention layers L (1 in the benchmark configurations)   */
+    int32_t n_q_heads;              /* H                                                               */
+    int32_t n_kv_heads;             /* G; H % G == 0                                                   */
+    int32_t head_dim;               /* d; 128 is what the kernels are built for                        */
+    int32_t block_tokens;           /* B_blk; a multiple of 16, at most 256                            */
+    int32_t max_sessions;           /* independent workspaces sharing the page pool                    */
+    int32_t max_blocks;             /* physical pages in the pool                                      */
+    int32_t max_blocks_per_session; /* rows of one session's block table and index                     */
+    int32_t device;                 /* CUDA device ordinal                                             */
+} kvmem_pool_config_t;
+
+/* Selection budget (Eq. "active_budget", Eq. "active_capacity" in Sec. 3.1; selector in
+ * Sec. 4.3).  The number of blocks kept is
+ *     k = min(budget_blocks, floor((max_view_tokens - mandatory_tokens) / block_tokens), NB), k >= 0.
+ * The oldest n_sink_blocks and newest n_recent_blocks are kept first (sinks before recents,
+ * truncated to k, overlap counted once); remaining slots go to the largest scores, equal
+ * scores to the lower block id.  Reserved blocks still take part in the softmax. */
+typedef struct {
+    int32_t budget_blocks;    /* requested k                                    */
+    int32_t max_view_tokens;  /* B_a = min(B_model, B_gpu), in tokens           */
+    int32_t mandatory_tokens; /* N(Q_tau): context the view must leave room for */
+    int32_t n_sink_blocks;
+    int32_t n_recent_blocks;
+} kvmem_select_params_t;
+
+/* ---- pure host helpers (no CUDA call) -------------------------------------------------- */
+
+/* Bytes of DEVICE storage kvmem_pool_create needs for this geometry (0 if cfg is invalid).
+ * Holds the K/V pages, the Mean-K index, the block tables and a status word. */
+size_t kvmem_pool_bytes(const kvmem_pool_config_t* cfg /*HOST*/);
+
+/* The budget clamp above for a session of n_blocks blocks; never negative. */
+int32_t kvmem_budget_blocks(const kvmem_select_params_t* params /*HOST*/, int32_t block_tokens, int32_t n_blocks);
+
+/* Bytes of DEVICE workspace kvmem_select needs for n_sessions sessions and n_q_tokens query
+ * tokens per session (0 if the arguments are invalid). */
+size_t kvmem_select_workspace_bytes(const kvmem_pool_config_t* cfg /*HOST*/, int32_t n_sessions, int32_t n_q_tokens);
+
+/* Bytes of DEVICE workspace kvmem_view_attend needs (split-K partial results). */
+size_t kvmem_attend_workspace_bytes(const kvmem_pool_config_t* cfg /*HOST*/, int32_t n_sessions, int32_t n_q_tokens);
+
+/* Description of the calling thread's last failure (static storage, never NULL). */
+const char* kvmem_last_error(void);
+
+/* ---- pool lifetime ---------------------------------------------------------------------- */
+
+/* Create a pool inside caller-owned DEVICE storage of at least kvmem_pool_bytes(cfg) bytes,
+ * 256-byte aligned.  The storage must outlive the pool.  Clears the tables and the status word
+ * (synchronous).  KVMEM_E_UNSUPPORTED if the device is not compute capability 10.x. */
+int kvmem_pool_create(const kvmem_pool_config_t* cfg /*HOST*/, void* storage /*DEVICE*/, size_t bytes,
+                      kvmem_pool_t** out /*HOST*/);
+int kvmem_pool_destroy(kvmem_pool_t* pool);
+
+/* Forget a session's blocks and return its pages to the free list (host-side, immediate). */
+int kvmem_session_reset(kvmem_pool_t* pool, int32_t session);
+
+/* Blocks appended to a session so far, or a negative status. */
+int32_t kvmem_session_blocks(const kvmem_pool_t* pool, int32_t session);
+
+/* ---- repository and index (Sec. 4.3, Eq. "mean_k_index"; Sec. 5.3 "Incremental Indexing") - */
+
+/* Append n_blocks completed blocks to a session: copy their K and V into physical pages,
+ * extend the block table and compute the Mean-K entry of each new block,
+ *     kbar[l][b][g] = (1/B) * sum_{i in b} k[l][i][g]
+ * (fp32 sum in ascending token order, one round-to-nearest-even to bf16).
+ *   k, v       DEVICE bf16 [n_blocks * block_tokens][n_layers][n_kv_heads][head_dim], 16-byte aligned;
+ *              may be released once the stream has run the call
+ *   phys_ids   HOST int32 [n_blocks] page ids to use, or NULL to take free pages in ascending order
+ * Errors: KVMEM_E_CAPACITY (session or pool full), KVMEM_E_STATE (page in use), KVMEM_E_INVALID. */
+int kvmem_append_blocks(kvmem_pool_t* pool, int32_t session, const void* k /*DEVICE*/, const void* v /*DEVICE*/,
+                        int32_t n_blocks, const int32_t* phys_ids /*HOST*/, void* stream);
+
+/* ---- the recall step ----------------------------------------------------------------------- */
+
+/* Score and select (Sec. 4.3, Eq. "kvmem-block-score"; selector; Sec. 5.2 tiled scoring with the
+ * softmax kept global across tiles).  For each session s in [session_first, session_first + n_sessions):
+ *     R_b = sum_m (1/(L*H)) sum_{l,h} softmax_{b' in all blocks of s}( q[m][l][h] . kbar[l][b'][g(h)] / sqrt(d) )_b
+ * then the selector described at kvmem_select_params_t.
+ *   q          DEVICE bf16 [n_sessions][n_q_tokens][n_layers][n_q_heads][head_dim], 16-byte aligned
+ *   sel_ids    DEVICE int32 [n_sessions][sel_stride]: ascending logical ids; entries past n_sel untouched
+ *   sel_stride >= the clamped budget of every session
+ *   n_sel      DEVICE int32 [n_sessions]
+ *   scores     DEVICE fp32 [n_sessions][max_blocks_per_session] receives R (first NB entries), or NULL
+ *   workspace  DEVICE, kvmem_select_workspace_bytes(), 256-byte aligned; contents undefined afterwards
+ * One query chunk gives one score vector and one selection (sum over its tokens). */
+int kvmem_select(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
+                 int32_t n_q_tokens, const kvmem_select_params_t* params /*HOST*/, int32_t* sel_ids /*DEVICE*/,
+                 int32_t sel_stride, int32_t* n_sel /*DEVICE*/, float* scores /*DEVICE*/, void* workspace /*DEVICE*/,
+                 size_t workspace_bytes, void* stream);
+
+/* Assemble the execution view (Sec. 4.4 "execution view"; Sec. 5.2): view tokens
+ * [j*B, (j+1)*B) of session s are block sel_ids[s][j]'s K and V, fetched through the block table.
+ *   view_k, view_v  DEVICE bf16 [n_sessions][n_layers][n_kv_heads][view_cap_tokens][head_dim], 16-byte aligned
+ *   n_sel is read on the device; blocks that would not fit view_cap_tokens are skipped and flagged.
+ * Tokens past n_sel * B are left untouched. */
+int kvmem_materialize(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids /*DEVICE*/,
+                      int32_t sel_stride, const int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/,
+                      void* view_v /*DEVICE*/, int32_t view_cap_tokens, void* stream);
+
+/* GQA decode attention over the view (QW3 attention kernels, Sec. 5.1; decode over the fixed
+ * working set, Sec. 5.2).  For every query token m, layer l and head h, over the first
+ * T = n_sel[s] * B view tokens of KV head g(h), without mask:
+ *     out = softmax(q . K^T * scale) V        lse = ln sum_t exp(q . k_t * scale)
+ * lse lets the caller merge attention over the tokens it appends after the view.
+ *   q        DEVICE bf16 [n_sessions][n_q_tokens][n_layers][n_q_heads][head_dim]
+ *   out      DEVICE fp32 [n_sessions][n_q_tokens][n_layers][n_q_heads][head_dim]
+ *   lse      DEVICE fp32 [n_sessions][n_q_tokens][n_layers][n_q_heads]
+ *   scale    0 selects 1/sqrt(head_dim)
+ *   workspace DEVICE, kvmem_attend_workspace_bytes(), 256-byte aligned
+ * T = 0 gives out = 0 and lse = -inf.  n_q_tokens * (H/G) <= 16 per call. */
+int kvmem_view_attend(kvmem_pool_t* pool, int32_t n_sessions, const void* q /*DEVICE*/, int32_t n_q_tokens,
+                      const void* view_k /*DEVICE*/, const void* view_v /*DEVICE*/, int32_t view_cap_tokens,
+                      const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
+                      void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
+/* The whole recall step for callers whose query and results live in HOST memory: copies q to the
+ * device, runs kvmem_select, kvmem_materialize and kvmem_view_attend, copies out and lse back and
+ * waits for the stream (synchronous).  Same definitions and limits as the three calls above.
+ *   q_host     HOST bf16 [n_sessions][n_q_tokens][L][H][d]   (pinned memory makes the copies asynchronous)
+ *   out_host   HOST fp32 [n_sessions][n_q_tokens][L][H][d];  lse_host HOST fp32 [n_sessions][n_q_tokens][L][H]
+ *   staging    DEVICE, kvmem_step_staging_bytes(), 256-byte aligned: device copies of q, out, lse
+ * sel_ids, n_sel, views and workspaces are DEVICE buffers as in the individual calls and hold the
+ * step's selection and view afterwards. */
+size_t kvmem_step_staging_bytes(const kvmem_pool_config_t* cfg /*HOST*/, int32_t n_sessions, int32_t n_q_tokens);
+int kvmem_recall_step_host(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q_host /*HOST*/,
+                           int32_t n_q_tokens, const kvmem_select_params_t* params /*HOST*/, int32_t* sel_ids /*DEVICE*/,
+                           int32_t sel_stride, int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/, void* view_v /*DEVICE*/,
+                           int32_t view_cap_tokens, float scale, float* out_host /*HOST*/, float* lse_host /*HOST*/,
+                           void* staging /*DEVICE*/, size_t staging_bytes, void* select_workspace /*DEVICE*/,
+                           size_t select_workspace_bytes, void* attend_workspace /*DEVICE*/,
+                           size_t attend_workspace_bytes, void* stream);
+
+/* ---- inspection ------------------------------------------------------------------------------ */
+
+/* Mean-K index of a session: DEVICE bf16 [n_layers][n_kv_heads][max_blocks_per_session][head_dim]
+ * (rows >= *n_blocks undefined).  The pointer aliases pool storage. */
+int kvmem_get_index(kvmem_pool_t* pool, int32_t session, const void** index /*HOST, receives DEVICE ptr*/,
+                    int32_t* n_blocks /*HOST*/);
+
+/* Block table of a session: DEVICE int32 [max_blocks_per_session], logical id -> physical page. */
+int kvmem_get_block_table(kvmem_pool_t* pool, int32_t session, const int32_t** table /*HOST, receives DEVICE ptr*/,
+                          int32_t* n_blocks /*HOST*/);
+
+/* Synchronise the stream and fetch (and clear) the sticky device status word: KVMEM_OK,
+ * KVMEM_E_TIMEOUT or KVMEM_E_DEVICE_RANGE.  Returns KVMEM_OK if the read itself worked. */
+int kvmem_device_status(kvmem_pool_t* pool, int32_t* status /*HOST*/, void* stream);
+
+/* Process-wide implementation switches used to compare kernel variants; they never change results.
+ * (No counterpart in the paper.)  "gather_mode": 1 = bulk asynchronous copies through shared memory
+ * (default), 0 = 128-bit load/store copy. */
+int kvmem_set_option(const char* name /*HOST*/, int32_t value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVMEM_H_ */

@@ -1,0 +1,414 @@
+// C ABI of libkvmem_b200: argument checking, pool and session bookkeeping, launch sequencing.
+// Every step of the recall path runs in the kernels of the sibling files; nothing here computes.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "kvmem_internal.cuh"
+
+namespace kvmem {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+bool config_valid(const kvmem_pool_config_t& c, const char** why) {
+    auto bad = [&](const char* w) { *why = w; return false; };
+    if (c.n_layers < 1 || c.n_layers > 256) return bad("n_layers must be in [1, 256]");
+    if (c.n_kv_heads < 1 || c.n_q_heads < 1 || c.n_q_heads % c.n_kv_heads != 0)
+        return bad("n_q_heads must be a positive multiple of n_kv_heads");
+    if (c.head_dim < 8 || c.head_dim > 512 || c.head_dim % 8 != 0) return bad("head_dim must be a multiple of 8 in [8, 512]");
+    if (c.block_tokens < 16 || c.block_tokens > 256 || c.block_tokens % 16 != 0)
+        return bad("block_tokens must be a multiple of 16 in [16, 256]");
+    if (c.max_sessions < 1 || c.max_sessions > 65535) return bad("max_sessions must be in [1, 65535]");
+    if (c.max_blocks < 1) return bad("max_blocks must be positive");
+    if (c.max_blocks_per_session < 1 || c.max_blocks_per_session > c.max_blocks)
+        return bad("max_blocks_per_session must be in [1, max_blocks]");
+    if (c.device < 0) return bad("device must be a CUDA ordinal");
+    return true;
+}
+
+Layout make_layout(const kvmem_pool_config_t& c) {
+    Layout l{};
+    l.tile_elems = (size_t)c.block_tokens * c.head_dim;
+    l.page_elems = 2 * (size_t)c.n_layers * c.n_kv_heads * l.tile_elems;
+    l.index_elems_per_session = (size_t)c.n_layers * c.n_kv_heads * c.max_blocks_per_session * c.head_dim;
+    size_t off = 0;
+    l.pages_off = off;
+    off = align_up(off + (size_t)c.max_blocks * l.page_elems * 2, 256);
+    l.index_off = off;
+    off = align_up(off + (size_t)c.max_sessions * l.index_elems_per_session * 2, 256);
+    l.tables_off = off;
+    off = align_up(off + (size_t)c.max_sessions * c.max_blocks_per_session * 4, 256);
+    l.nblocks_off = off;
+    off = align_up(off + (size_t)c.max_sessions * 4, 256);
+    l.status_off = off;
+    off = align_up(off + 256, 256);
+    l.total = off;
+    return l;
+}
+
+static bool pool_ok(const kvmem_pool* p) {
+    if (!p || p->magic != kMagic) {
+        set_error("pool handle is null or stale");
+        return false;
+    }
+    return true;
+}
+
+static bool sessions_ok(const kvmem_pool* p, int first, int n) {
+    if (first < 0 || n < 1 || first + n > p->cfg.max_sessions) {
+        set_error("sessions [%d, %d) outside [0, %d)", first, first + n, p->cfg.max_sessions);
+        return false;
+    }
+    return true;
+}
+
+static int cuda_fail(const char* what, cudaError_t e) {
+    set_error("%s: %s", what, cudaGetErrorString(e));
+    return KVMEM_E_CUDA;
+}
+
+static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+}  // namespace kvmem
+
+using namespace kvmem;
+
+extern "C" {
+
+const char* kvmem_last_error(void) { return g_err; }
+
+size_t kvmem_pool_bytes(const kvmem_pool_config_t* cfg) {
+    const char* why = "";
+    if (!cfg || !config_valid(*cfg, &why)) {
+        set_error("invalid pool configuration: %s", cfg ? why : "null");
+        return 0;
+    }
+    return make_layout(*cfg).total;
+}
+
+int32_t kvmem_budget_blocks(const kvmem_select_params_t* prm, int32_t block_tokens, int32_t n_blocks) {
+    if (!prm || block_tokens <= 0) return 0;
+    int64_t room = (int64_t)prm->max_view_tokens - (int64_t)prm->mandatory_tokens;
+    int64_t k = room > 0 ? room / block_tokens : 0;
+    k = std::min<int64_t>(k, prm->budget_blocks);
+    k = std::min<int64_t>(k, n_blocks);
+    return (int32_t)std::max<int64_t>(k, 0);
+}
+
+size_t kvmem_select_workspace_bytes(const kvmem_pool_config_t* cfg, int32_t n_sessions, int32_t n_q_tokens) {
+    const char* why = "";
+    if (!cfg || !config_valid(*cfg, &why) || n_sessions < 1 || n_sessions > cfg->max_sessions || n_q_tokens < 1) {
+        set_error("invalid arguments to kvmem_select_workspace_bytes");
+        return 0;
+    }
+    return plan_score_workspace(*cfg, n_sessions, n_q_tokens, nullptr).total;
+}
+
+size_t kvmem_attend_workspace_bytes(const kvmem_pool_config_t* cfg, int32_t n_sessions, int32_t n_q_tokens) {
+    const char* why = "";
+    if (!cfg || !config_valid(*cfg, &why) || n_sessions < 1 || n_q_tokens < 1) {
+        set_error("invalid arguments to kvmem_attend_workspace_bytes");
+        return 0;
+    }
+    return plan_attend(*cfg, n_sessions, n_q_tokens, kSMs).total;
+}
+
+int kvmem_pool_create(const kvmem_pool_config_t* cfg, void* storage, size_t bytes, kvmem_pool_t** out) {
+    const char* why = "";
+    if (!out) { set_error("out is null"); return KVMEM_E_INVALID; }
+    *out = nullptr;
+    if (!cfg || !config_valid(*cfg, &why)) {
+        set_error("invalid pool configuration: %s", cfg ? why : "null");
+        return KVMEM_E_INVALID;
+    }
+    if (!storage || !aligned(storage, 256)) { set_error("storage must be a 256-byte aligned device pointer"); return KVMEM_E_INVALID; }
+    Layout lay = make_layout(*cfg);
+    if (bytes < lay.total) {
+        set_error("storage holds %zu bytes, the pool needs %zu", bytes, lay.total);
+        return KVMEM_E_CAPACITY;
+    }
+    cudaError_t e = cudaSetDevice(cfg->device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, cfg->device);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDeviceProperties", e);
+    if (prop.major != 10) {
+        set_error("device %d is compute capability %d.%d; this library is built for sm_100a only", cfg->device,
+                  prop.major, prop.minor);
+        return KVMEM_E_UNSUPPORTED;
+    }
+    kvmem_pool* p = new (std::nothrow) kvmem_pool();
+    if (!p) { set_error("host allocation failed"); return KVMEM_E_CAPACITY; }
+    p->magic = kMagic;
+    p->cfg = *cfg;
+    p->geo = Geometry{cfg->n_layers, cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim, cfg->block_tokens,
+                      cfg->n_q_heads / cfg->n_kv_heads, cfg->max_sessions, cfg->max_blocks, cfg->max_blocks_per_session};
+    p->lay = lay;
+    p->base = (char*)storage;
+    p->pages = (__nv_bfloat16*)(p->base + lay.pages_off);
+    p->index = (__nv_bfloat16*)(p->base + lay.index_off);
+    p->tables = (int32_t*)(p->base + lay.tables_off);
+    p->nblocks_dev = (int32_t*)(p->base + lay.nblocks_off);
+    p->status_dev = (int32_t*)(p->base + lay.status_off);
+    p->sess_blocks.assign(cfg->max_sessions, 0);
+    p->sess_pages.assign(cfg->max_sessions, {});
+    p->page_used.assign(cfg->max_blocks, 0);
+    p->free_hint = 0;
+    p->sm_count = prop.multiProcessorCount;
+    e = cudaMemset(p->base + lay.tables_off, 0, lay.total - lay.tables_off);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { delete p; return cuda_fail("clearing pool metadata", e); }
+    *out = p;
+    return KVMEM_OK;
+}
+
+int kvmem_pool_destroy(kvmem_pool_t* pool) {
+    if (!pool_ok(pool)) return KVMEM_E_STATE;
+    pool->magic = 0;
+    delete pool;
+    return KVMEM_OK;
+}
+
+int kvmem_session_reset(kvmem_pool_t* p, int32_t session) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;
+    for (int32_t pg : p->sess_pages[session]) p->page_used[pg] = 0;
+    p->sess_pages[session].clear();
+    p->sess_blocks[session] = 0;
+    p->free_hint = 0;
+    return KVMEM_OK;
+}
+
+int32_t kvmem_session_blocks(const kvmem_pool_t* p, int32_t session) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;
+    return p->sess_blocks[session];
+}
+
+int kvmem_append_blocks(kvmem_pool_t* p, int32_t session, const void* k, const void* v, int32_t n_blocks,
+                        const int32_t* phys_ids, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;
+    if (n_blocks < 0) { set_error("n_blocks is negative"); return KVMEM_E_INVALID; }
+    if (n_blocks == 0) return KVMEM_OK;
+    if (!k || !v || !aligned(k, 16) || !aligned(v, 16)) { set_error("k and v must be 16-byte aligned device pointers"); return KVMEM_E_INVALID; }
+    const int have = p->sess_blocks[session];
+    if ((int64_t)have + n_blocks > p->cfg.max_blocks_per_session) {
+        set_error("session %d holds %d blocks; %d more exceed max_blocks_per_session = %d", session, have, n_blocks,
+                  p->cfg.max_blocks_per_session);
+        return KVMEM_E_CAPACITY;
+    }
+    // choose pages without touching the pool until every id is known to be usable
+    std::vector<int32_t> ids(n_blocks);
+    if (phys_ids) {
+        std::vector<int32_t> sorted(phys_ids, phys_ids + n_blocks);
+        std::sort(sorted.begin(), sorted.end());
+        for (int i = 0; i < n_blocks; ++i) {
+            int32_t pg = phys_ids[i];
+            if (pg < 0 || pg >= p->cfg.max_blocks) { set_error("page id %d outside [0, %d)", pg, p->cfg.max_blocks); return KVMEM_E_INVALID; }
+            if (p->page_used[pg]) { set_error("page %d is already in use", pg); return KVMEM_E_STATE; }
+            if (i > 0 && sorted[i] == sorted[i - 1]) { set_error("page id %d given twice", sorted[i]); return KVMEM_E_INVALID; }
+            ids[i] = pg;
+        }
+    } else {
+        int32_t pg = p->free_hint, got = 0;
+        for (; pg < p->cfg.max_blocks && got < n_blocks; ++pg)
+            if (!p->page_used[pg]) ids[got++] = pg;
+        if (got < n_blocks) { set_error("pool has %d free pages, %d needed", got, n_blocks); return KVMEM_E_CAPACITY; }
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t* table = p->tables + (size_t)session * p->cfg.max_blocks_per_session;
+    cudaError_t e = cudaMemcpyAsync(table + have, ids.data(), (size_t)n_blocks * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail("block table upload", e);
+    const int32_t total = have + n_blocks;
+    e = cudaMemcpyAsync(p->nblocks_dev + session, &total, 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail("block count upload", e);
+    e = launch_append(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st);
+    if (e != cudaSuccess) return cuda_fail("append kernel launch", e);
+    for (int32_t pg : ids) { p->page_used[pg] = 1; p->sess_pages[session].push_back(pg); }
+    if (!phys_ids) p->free_hint = ids.back() + 1;
+    p->sess_blocks[session] = total;
+    return KVMEM_OK;
+}
+
+int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                 const kvmem_select_params_t* prm, int32_t* sel_ids, int32_t sel_stride, int32_t* n_sel, float* scores,
+                 void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!q || !aligned(q, 16) || !prm || !sel_ids || !n_sel || !workspace || !aligned(workspace, 256)) {
+        set_error("kvmem_select: null or misaligned pointer");
+        return KVMEM_E_INVALID;
+    }
+    if (n_q_tokens < 1) { set_error("n_q_tokens must be positive"); return KVMEM_E_INVALID; }
+    if (prm->n_sink_blocks < 0 || prm->n_recent_blocks < 0) { set_error("sink/recent counts must be non-negative"); return KVMEM_E_INVALID; }
+    if (p->cfg.head_dim != 128) { set_error("scoring kernels are built for head_dim 128"); return KVMEM_E_UNSUPPORTED; }
+    int max_k = 0;
+    for (int s = session_first; s < session_first + n_sessions; ++s)
+        max_k = std::max(max_k, kvmem_budget_blocks(prm, p->cfg.block_tokens, p->sess_blocks[s]));
+    if (sel_stride < max_k) { set_error("sel_stride %d is below the clamped budget %d", sel_stride, max_k); return KVMEM_E_CAPACITY; }
+    ScoreWorkspace ws = plan_score_workspace(p->cfg, n_sessions, n_q_tokens, (char*)workspace);
+    if (workspace_bytes < ws.total) { set_error("select workspace holds %zu bytes, %zu needed", workspace_bytes, ws.total); return KVMEM_E_CAPACITY; }
+    cudaStream_t st = (cudaStream_t)stream;
+    float* sc = scores ? scores : ws.scores;
+    cudaError_t e = launch_score_decode(*p, session_first, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, ws, sc,
+                                        p->cfg.max_blocks_per_session, st);
+    if (e != cudaSuccess) return cuda_fail("score kernel launch", e);
+    e = launch_topk(*p, session_first, n_sessions, sc, p->cfg.max_blocks_per_session, *prm, sel_ids, sel_stride, n_sel, st);
+    if (e != cudaSuccess) return cuda_fail("top-k kernel launch", e);
+    return KVMEM_OK;
+}
+
+int kvmem_materialize(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids,
+                      int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v, int32_t view_cap_tokens,
+                      void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!sel_ids || !n_sel || !view_k || !view_v || !aligned(view_k, 16) || !aligned(view_v, 16)) {
+        set_error("kvmem_materialize: null or misaligned pointer");
+        return KVMEM_E_INVALID;
+    }
+    if (sel_stride < 1 || view_cap_tokens < p->cfg.block_tokens || view_cap_tokens % p->cfg.block_tokens != 0) {
+        set_error("view_cap_tokens must be a positive multiple of block_tokens and sel_stride positive");
+        return KVMEM_E_INVALID;
+    }
+    cudaError_t e = launch_gather(*p, session_first, n_sessions, sel_ids, sel_stride, n_sel, (__nv_bfloat16*)view_k,
+                                  (__nv_bfloat16*)view_v, view_cap_tokens, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("gather kernel launch", e);
+    return KVMEM_OK;
+}
+
+int kvmem_view_attend(kvmem_pool_t* p, int32_t n_sessions, const void* q, int32_t n_q_tokens, const void* view_k,
+                      const void* view_v, int32_t view_cap_tokens, const int32_t* n_sel, float scale, float* out,
+                      float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (n_sessions < 1) { set_error("n_sessions must be positive"); return KVMEM_E_INVALID; }
+    if (!q || !view_k || !view_v || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(view_k, 128) ||
+        !aligned(view_v, 128) || !aligned(workspace, 256) || !aligned(out, 16)) {
+        set_error("kvmem_view_attend: null or misaligned pointer (views need 128-byte alignment)");
+        return KVMEM_E_INVALID;
+    }
+    if (n_q_tokens < 1) { set_error("n_q_tokens must be positive"); return KVMEM_E_INVALID; }
+    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
+        set_error("attention kernel is built for head_dim 128 and 64-token blocks");
+        return KVMEM_E_UNSUPPORTED;
+    }
+    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (view_cap_tokens < p->cfg.block_tokens || view_cap_tokens % p->cfg.block_tokens != 0) {
+        set_error("view_cap_tokens must be a positive multiple of block_tokens");
+        return KVMEM_E_INVALID;
+    }
+    if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
+    AttendPlan plan = plan_attend(p->cfg, n_sessions, n_q_tokens, p->sm_count);
+    if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
+    cudaError_t e = launch_attend(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, (const __nv_bfloat16*)view_k,
+                                  (const __nv_bfloat16*)view_v, view_cap_tokens, n_sel, scale, out, lse, workspace,
+                                  (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("attend kernel launch", e);
+    return KVMEM_OK;
+}
+
+static void step_staging(const kvmem_pool_config_t& c, int ns, int M, size_t* q_b, size_t* out_b, size_t* lse_b) {
+    const size_t rows = (size_t)ns * M * c.n_layers * c.n_q_heads;
+    *q_b = align_up(rows * c.head_dim * 2, 256);
+    *out_b = align_up(rows * c.head_dim * 4, 256);
+    *lse_b = align_up(rows * 4, 256);
+}
+
+size_t kvmem_step_staging_bytes(const kvmem_pool_config_t* cfg, int32_t n_sessions, int32_t n_q_tokens) {
+    const char* why = "";
+    if (!cfg || !config_valid(*cfg, &why) || n_sessions < 1 || n_q_tokens < 1) {
+        set_error("invalid arguments to kvmem_step_staging_bytes");
+        return 0;
+    }
+    size_t a, b, c;
+    step_staging(*cfg, n_sessions, n_q_tokens, &a, &b, &c);
+    return a + b + c;
+}
+
+int kvmem_recall_step_host(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q_host,
+                           int32_t n_q_tokens, const kvmem_select_params_t* prm, int32_t* sel_ids, int32_t sel_stride,
+                           int32_t* n_sel, void* view_k, void* view_v, int32_t view_cap_tokens, float scale,
+                           float* out_host, float* lse_host, void* staging, size_t staging_bytes, void* select_ws,
+                           size_t select_ws_bytes, void* attend_ws, size_t attend_ws_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!q_host || !out_host || !lse_host || !staging || !aligned(staging, 256) || n_q_tokens < 1) {
+        set_error("kvmem_recall_step_host: null or misaligned pointer");
+        return KVMEM_E_INVALID;
+    }
+    size_t q_b, out_b, lse_b;
+    step_staging(p->cfg, n_sessions, n_q_tokens, &q_b, &out_b, &lse_b);
+    if (staging_bytes < q_b + out_b + lse_b) { set_error("staging holds %zu bytes, %zu needed", staging_bytes, q_b + out_b + lse_b); return KVMEM_E_CAPACITY; }
+    char* sb = (char*)staging;
+    void* q_dev = sb;
+    float* out_dev = (float*)(sb + q_b);
+    float* lse_dev = (float*)(sb + q_b + out_b);
+    const size_t rows = (size_t)n_sessions * n_q_tokens * p->cfg.n_layers * p->cfg.n_q_heads;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(q_dev, q_host, rows * p->cfg.head_dim * 2, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail("query upload", e);
+    int rc = kvmem_select(p, session_first, n_sessions, q_dev, n_q_tokens, prm, sel_ids, sel_stride, n_sel, nullptr,
+                          select_ws, select_ws_bytes, stream);
+    if (rc != KVMEM_OK) return rc;
+    rc = kvmem_materialize(p, session_first, n_sessions, sel_ids, sel_stride, n_sel, view_k, view_v, view_cap_tokens, stream);
+    if (rc != KVMEM_OK) return rc;
+    rc = kvmem_view_attend(p, n_sessions, q_dev, n_q_tokens, view_k, view_v, view_cap_tokens, n_sel, scale, out_dev,
+                           lse_dev, attend_ws, attend_ws_bytes, stream);
+    if (rc != KVMEM_OK) return rc;
+    e = cudaMemcpyAsync(out_host, out_dev, rows * p->cfg.head_dim * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(lse_host, lse_dev, rows * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail("result download", e);
+    return KVMEM_OK;
+}
+
+int kvmem_set_option(const char* name, int32_t value) {
+    if (!name) { set_error("option name is null"); return KVMEM_E_INVALID; }
+    if (strcmp(name, "gather_mode") == 0 && (value == 0 || value == 1)) { g_gather_mode = value; return KVMEM_OK; }
+    set_error("unknown option or value: %s = %d", name, value);
+    return KVMEM_E_INVALID;
+}
+
+int kvmem_get_index(kvmem_pool_t* p, int32_t session, const void** index, int32_t* n_blocks) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;
+    if (!index || !n_blocks) { set_error("null output pointer"); return KVMEM_E_INVALID; }
+    *index = p->index + (size_t)session * p->lay.index_elems_per_session;
+    *n_blocks = p->sess_blocks[session];
+    return KVMEM_OK;
+}
+
+int kvmem_get_block_table(kvmem_pool_t* p, int32_t session, const int32_t** table, int32_t* n_blocks) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;
+    if (!table || !n_blocks) { set_error("null output pointer"); return KVMEM_E_INVALID; }
+    *table = p->tables + (size_t)session * p->cfg.max_blocks_per_session;
+    *n_blocks = p->sess_blocks[session];
+    return KVMEM_OK;
+}
+
+int kvmem_device_status(kvmem_pool_t* p, int32_t* status, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!status) { set_error("status is null"); return KVMEM_E_INVALID; }
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, p->status_dev, 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->status_dev, 0, 4, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail("reading the device status word", e);
+    *status = word;
+    return KVMEM_OK;
+}
+
+}  // extern "C"

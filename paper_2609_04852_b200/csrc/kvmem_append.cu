@@ -1,0 +1,73 @@
+// Repository append + Mean-K index construction (Eq. "mean_k_index", Sec. 4.3; "Incremental
+// Indexing", Sec. 5.3: the index entry is computed while the block's keys pass through the SM).
+//
+// One CTA per (new block, layer, KV head).  The caller's token-major rows (256 B each at d = 128,
+// strided by L*G*d) are read once with 128-bit loads, written to the page's contiguous [B][d]
+// tile, and the K tile is kept in shared memory so that thread c can walk tokens 0..B-1 of
+// dimension c in order: an fp32 running sum in ascending token order, one multiply by 1/B and one
+// round-to-nearest-even to bf16.  That order is the definition of the stored index value.
+#include "kvmem_internal.cuh"
+
+namespace kvmem {
+
+__global__ void __launch_bounds__(256)
+append_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* __restrict__ v_in,
+              __nv_bfloat16* __restrict__ pages, __nv_bfloat16* __restrict__ index_sess,
+              const int32_t* __restrict__ table_sess, int32_t* __restrict__ status,
+              int b_first, int L, int G, int B, int d, int max_blocks, int max_bps, size_t page_elems) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __nv_bfloat16* tile = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [B][d]
+
+    const int i = blockIdx.x;          // new block index within this call
+    const int lg = blockIdx.y;         // l * G + g
+    const int page = table_sess[b_first + i];
+    if (page < 0 || page >= max_blocks) {
+        if (threadIdx.x == 0) atomicExch(status, (int)KVMEM_E_DEVICE_RANGE);
+        return;
+    }
+    const int chunks_per_row = d / 8;                     // 16-byte chunks
+    const int n_chunks = B * chunks_per_row;
+    const size_t row_stride = (size_t)L * G * d;          // elements between consecutive tokens
+    const __nv_bfloat16* ksrc = k_in + (size_t)i * B * row_stride + (size_t)lg * d;
+    const __nv_bfloat16* vsrc = v_in + (size_t)i * B * row_stride + (size_t)lg * d;
+    const size_t tile_elems = (size_t)B * d;
+    __nv_bfloat16* kdst = pages + (size_t)page * page_elems + (size_t)lg * tile_elems;
+    __nv_bfloat16* vdst = kdst + (size_t)L * G * tile_elems;
+
+    for (int c = threadIdx.x; c < n_chunks; c += blockDim.x) {
+        const int t = c / chunks_per_row, j = c % chunks_per_row;
+        const uint4 kk = *reinterpret_cast<const uint4*>(ksrc + (size_t)t * row_stride + j * 8);
+        const uint4 vv = *reinterpret_cast<const uint4*>(vsrc + (size_t)t * row_stride + j * 8);
+        *reinterpret_cast<uint4*>(tile + (size_t)t * d + j * 8) = kk;
+        *reinterpret_cast<uint4*>(kdst + (size_t)t * d + j * 8) = kk;
+        *reinterpret_cast<uint4*>(vdst + (size_t)t * d + j * 8) = vv;
+    }
+    __syncthreads();
+
+    const float inv = 1.0f / (float)B;
+    __nv_bfloat16* idx_row = index_sess + ((size_t)lg * max_bps + (size_t)(b_first + i)) * d;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        float acc = 0.0f;
+        for (int t = 0; t < B; ++t) acc = __fadd_rn(acc, __bfloat162float(tile[(size_t)t * d + c]));
+        idx_row[c] = __float2bfloat16_rn(__fmul_rn(acc, inv));
+    }
+}
+
+cudaError_t launch_append(const kvmem_pool& p, int session, int b_first, int n_blocks, const __nv_bfloat16* k,
+                          const __nv_bfloat16* v, cudaStream_t st) {
+    const Geometry& g = p.geo;
+    const size_t smem = (size_t)g.B * g.d * sizeof(__nv_bfloat16);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(append_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    const int32_t* table = p.tables + (size_t)session * g.max_bps;
+    __nv_bfloat16* index = p.index + (size_t)session * p.lay.index_elems_per_session;
+    // gridDim.x is limited to 2^31-1 blocks and gridDim.y to 65535: L*G stays far below that
+    dim3 grid((unsigned)n_blocks, (unsigned)(g.L * g.G));
+    append_kernel<<<grid, 256, smem, st>>>(k, v, p.pages, index, table, p.status_dev, b_first, g.L, g.G, g.B, g.d,
+                                           g.max_blocks, g.max_bps, p.lay.page_elems);
+    return cudaGetLastError();
+}
+
+}  // namespace kvmem

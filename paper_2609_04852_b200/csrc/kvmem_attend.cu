@@ -1,0 +1,355 @@
+// GQA decode attention over the execution view (QW3 attention kernels, Sec. 5.1; decode over the
+// fixed working set, Sec. 5.2):  out = softmax(q K^T * scale) V,  lse = ln sum_t exp(s_t), no mask.
+//
+// Split-K flash decoding.  Grid = (split, layer x KV head, session).  A split owns a contiguous
+// range of 64-token view tiles.  Inside a CTA one producer warp streams tiles with TMA
+// (cp.async.bulk.tensor, 128-byte swizzle, mbarrier completion) into a ring of 32 KiB stages
+// (K tile + V tile); two groups of four consumer warps take tiles alternately, each warp 16 tokens.  The M*(H/G) <= 16 query rows of
+// the KV head form one m16 MMA tile: S = Q K^T and O += P V run on bf16 mma.sync with fp32
+// accumulators (at 16 flop per view byte the step would otherwise be ALU-bound instead of
+// HBM-bound), online softmax in fp32 in the exp2 domain.  Each warp carries its own (m, l, O); the
+// CTA merges its warps in shared memory and writes one partial per split; a second kernel merges
+// the splits in split order with the usual log-sum-exp rescale, so the result does not depend on
+// timing.  Every mbarrier wait is bounded and reports KVMEM_E_TIMEOUT through the status word.
+#include <cudaTypedefs.h>
+#include <math.h>
+
+#include "kvmem_internal.cuh"
+#include "kvmem_ptx.cuh"
+
+namespace kvmem {
+
+constexpr int kAttStages = 6;
+constexpr int kAttConsumers = 8;
+constexpr int kAttGroups = 2;                   // consumer groups; kAttStages % kAttGroups == 0
+static_assert(kAttStages % kAttGroups == 0, "each group must own whole stages");
+constexpr int kAttThreads = (kAttConsumers + 1) * 32;
+constexpr int kTile = 64;                       // tokens per tile == block_tokens
+constexpr int kD = 128;
+constexpr int kHalfBytes = kTile * 128;         // one 64-dim half of a tile: 64 rows x 128 B
+constexpr int kStageBytes = 4 * kHalfBytes;     // K lo, K hi, V lo, V hi
+constexpr int kMaxSplits = 64;
+constexpr int kRowsPad = 16;
+constexpr int kMergeStride = 136;               // floats per merged row in shared memory
+constexpr size_t kAttSmem = (size_t)kAttStages * kStageBytes + 1024;
+
+struct AttendArgs {
+    const __nv_bfloat16* q;
+    const int32_t* n_sel;
+    float* part_o;      // [ns*LG][n_splits][16][128]
+    float2* part_ml;    // [ns*LG][n_splits][16]
+    int32_t* status;
+    int M, L, H, G, r, rows, n_splits, cap_tokens;
+    float scale_log2e;
+};
+
+AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, int sm_count) {
+    (void)n_q_tokens; (void)sm_count;
+    AttendPlan p{};
+    p.n_splits = kMaxSplits;
+    p.rows_pad = kRowsPad;
+    const size_t heads = (size_t)n_sessions * c.n_layers * c.n_kv_heads;
+    p.part_o_bytes = align_up(heads * kMaxSplits * kRowsPad * kD * sizeof(float), 256);
+    p.part_ml_bytes = align_up(heads * kMaxSplits * kRowsPad * sizeof(float2), 256);
+    p.total = p.part_o_bytes + p.part_ml_bytes;
+    return p;
+}
+
+// splits per head: fewest waves of CTAs over the SMs, counting a fixed per-CTA cost in tiles
+static int choose_splits(int heads, int max_tiles, int sms) {
+    const int overhead = 6;
+    long long best_cost = -1;
+    int best = 1;
+    for (int s = 1; s <= kMaxSplits && s <= std::max(1, max_tiles); ++s) {
+        const long long waves = ((long long)heads * s + sms - 1) / sms;
+        const long long cost = waves * ((max_tiles + s - 1) / s + overhead);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    }
+    return best;
+}
+
+__global__ void __launch_bounds__(kAttThreads, 1)
+attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, AttendArgs a) {
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages];
+    __shared__ float merge_m[kAttConsumers][kRowsPad], merge_l[kAttConsumers][kRowsPad];
+
+    unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int split = blockIdx.x, lg = blockIdx.y, s = blockIdx.z;
+    const int LG = a.L * a.G;
+    const int z = s * LG + lg;
+    const int l = lg / a.G, g = lg % a.G;
+
+    int n_blk = a.n_sel[s];
+    n_blk = max(0, min(n_blk, a.cap_tokens / kTile));
+    const int t0 = (int)((long long)n_blk * split / a.n_splits);
+    const int t1 = (int)((long long)n_blk * (split + 1) / a.n_splits);
+    const int n_tiles = t1 - t0;
+
+    if (tid == 0) {
+        for (int i = 0; i < kAttStages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kAttConsumers / kAttGroups); }
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+
+    float o[16][4];           // O accumulators: 16 n-tiles of 8 dims
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f; }
+
+    if (warp == kAttConsumers) {
+        // ---------------- producer ----------------
+        if (lane == 0 && n_tiles > 0) {
+            ptx::prefetch_tensormap(&map_k);
+            ptx::prefetch_tensormap(&map_v);
+            for (int it = 0; it < n_tiles; ++it) {
+                const int st = it % kAttStages;
+                if (it >= kAttStages && !ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kAttStages) & 1) ^ 1))) {
+                    atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+                    break;
+                }
+                unsigned char* dst = stages + (size_t)st * kStageBytes;
+                const int y = (t0 + it) * kTile;
+                ptx::mbar_expect_tx(&full_bar[st], kStageBytes);
+                ptx::tma_load_3d(dst, &map_k, 0, y, z, &full_bar[st]);
+                ptx::tma_load_3d(dst + kHalfBytes, &map_k, 64, y, z, &full_bar[st]);
+                ptx::tma_load_3d(dst + 2 * kHalfBytes, &map_v, 0, y, z, &full_bar[st]);
+                ptx::tma_load_3d(dst + 3 * kHalfBytes, &map_v, 64, y, z, &full_bar[st]);
+            }
+        }
+    } else {
+        // ---------------- consumers ----------------
+        // Q fragments (A operand, m16k16 x 8 k-steps).  Row j = m * r + hr  ->  q[s][m][l][g*r + hr].
+        uint32_t qf[8][4];
+        {
+            const int row_a = lane >> 2, row_b = row_a + 8;
+            const __nv_bfloat16* qa = nullptr;
+            const __nv_bfloat16* qb = nullptr;
+            if (row_a < a.rows) qa = a.q + ((((size_t)s * a.M + row_a / a.r) * a.L + l) * a.H + (size_t)g * a.r + row_a % a.r) * kD;
+            if (row_b < a.rows) qb = a.q + ((((size_t)s * a.M + row_b / a.r) * a.L + l) * a.H + (size_t)g * a.r + row_b % a.r) * kD;
+            const int kq = 2 * (lane & 3);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                qf[ks][0] = qa ? *reinterpret_cast<const uint32_t*>(qa + ks * 16 + kq) : 0u;
+                qf[ks][1] = qb ? *reinterpret_cast<const uint32_t*>(qb + ks * 16 + kq) : 0u;
+                qf[ks][2] = qa ? *reinterpret_cast<const uint32_t*>(qa + ks * 16 + kq + 8) : 0u;
+                qf[ks][3] = qb ? *reinterpret_cast<const uint32_t*>(qb + ks * 16 + kq + 8) : 0u;
+            }
+        }
+        const uint32_t stage0 = ptx::smem_u32(stages);
+        const int mj = lane >> 3, mr = lane & 7;        // ldmatrix: matrix index and row within it
+        // Two groups of four warps.  Group grp takes tiles grp, grp + 2, ...; with an even number of
+        // stages it therefore meets the phases of "its" stages strictly in order, which an mbarrier
+        // parity wait requires.  Inside a tile, warp wq owns tokens [16 wq, 16 wq + 16).
+        const int grp = warp >> 2, wq = warp & 3;
+
+        for (int it = grp; it < n_tiles; it += kAttGroups) {
+            const int st = it % kAttStages;
+            const bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kAttStages) & 1));
+            if (!__all_sync(0xffffffffu, arrived)) {          // warp-uniform decision
+                if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+                break;
+            }
+            const uint32_t kbase = stage0 + (uint32_t)st * kStageBytes;
+            const uint32_t vbase = kbase + 2 * kHalfBytes;
+
+            // S = Q K^T for this warp's 16 tokens: 2 n-tiles (8 tokens each) x 8 k-steps
+            float sc[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) { sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.0f; }
+#pragma unroll
+            for (int kp = 0; kp < 4; ++kp) {            // 32 dims = 4 chunks of 16 B = 2 k-steps
+                const int cg = kp * 4 + mj;             // 16-byte chunk along d (0..15)
+                const uint32_t half_off = (uint32_t)(cg >> 3) * kHalfBytes;
+                const int c = cg & 7;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    const int tok = wq * 16 + nt * 8 + mr;
+                    const uint32_t addr = kbase + half_off + (uint32_t)tok * 128u + (uint32_t)((c ^ (tok & 7)) << 4);
+                    uint32_t b0, b1, b2, b3;
+                    ptx::ldmatrix_x4(addr, b0, b1, b2, b3);
+                    ptx::mma_bf16_16816(sc[nt], qf[2 * kp], b0, b1);
+                    ptx::mma_bf16_16816(sc[nt], qf[2 * kp + 1], b2, b3);
+                }
+            }
+            // online softmax (exp2 domain); this thread holds rows lane/4 (c0,c1) and lane/4 + 8 (c2,c3)
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                sc[nt][0] *= a.scale_log2e; sc[nt][1] *= a.scale_log2e; sc[nt][2] *= a.scale_log2e; sc[nt][3] *= a.scale_log2e;
+                mx0 = fmaxf(mx0, fmaxf(sc[nt][0], sc[nt][1]));
+                mx1 = fmaxf(mx1, fmaxf(sc[nt][2], sc[nt][3]));
+            }
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+            const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+            const bool grew = (mn0 != m_run[0]) || (mn1 != m_run[1]);
+            if (__any_sync(0xffffffffu, grew)) {         // a running maximum moved: rescale what is accumulated
+                const float corr0 = exp2f(m_run[0] - mn0), corr1 = exp2f(m_run[1] - mn1);
+                l_run[0] *= corr0; l_run[1] *= corr1;
+#pragma unroll
+                for (int nd = 0; nd < 16; ++nd) { o[nd][0] *= corr0; o[nd][1] *= corr0; o[nd][2] *= corr1; o[nd][3] *= corr1; }
+                m_run[0] = mn0; m_run[1] = mn1;
+            }
+            uint32_t pa[4];
+            {
+                const float p00 = exp2f(sc[0][0] - mn0), p01 = exp2f(sc[0][1] - mn0);
+                const float p02 = exp2f(sc[0][2] - mn1), p03 = exp2f(sc[0][3] - mn1);
+                const float p10 = exp2f(sc[1][0] - mn0), p11 = exp2f(sc[1][1] - mn0);
+                const float p12 = exp2f(sc[1][2] - mn1), p13 = exp2f(sc[1][3] - mn1);
+                l_run[0] += (p00 + p01) + (p10 + p11);
+                l_run[1] += (p02 + p03) + (p12 + p13);
+                pa[0] = ptx::pack_bf16x2(p00, p01); pa[1] = ptx::pack_bf16x2(p02, p03);
+                pa[2] = ptx::pack_bf16x2(p10, p11); pa[3] = ptx::pack_bf16x2(p12, p13);
+            }
+            // O += P V : one k-step (this warp's 16 tokens) x 16 n-tiles (8 dims)
+            {
+                const int tok = wq * 16 + (mj & 1) * 8 + mr;
+#pragma unroll
+                for (int np = 0; np < 8; ++np) {
+                    const int cg = np * 2 + (mj >> 1);
+                    const uint32_t addr = vbase + (uint32_t)(cg >> 3) * kHalfBytes + (uint32_t)tok * 128u +
+                                          (uint32_t)(((cg & 7) ^ (tok & 7)) << 4);
+                    uint32_t b0, b1, b2, b3;
+                    ptx::ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+                    ptx::mma_bf16_16816(o[2 * np], pa, b0, b1);
+                    ptx::mma_bf16_16816(o[2 * np + 1], pa, b2, b3);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&empty_bar[st]);
+        }
+        // row sums live spread over the 4 lanes of a quad
+        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1); l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
+        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1); l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
+    }
+
+    // every issued tile has been consumed (or a wait gave up): the ring can be reused for the merge
+    __syncthreads();
+    float* merge_o = reinterpret_cast<float*>(stages);          // [consumer][16][kMergeStride]
+    if (warp < kAttConsumers) {
+        const int row_a = lane >> 2, row_b = row_a + 8, col = 2 * (lane & 3);
+        float* base = merge_o + (size_t)warp * kRowsPad * kMergeStride;
+#pragma unroll
+        for (int nd = 0; nd < 16; ++nd) {
+            *reinterpret_cast<float2*>(base + row_a * kMergeStride + nd * 8 + col) = make_float2(o[nd][0], o[nd][1]);
+            *reinterpret_cast<float2*>(base + row_b * kMergeStride + nd * 8 + col) = make_float2(o[nd][2], o[nd][3]);
+        }
+        if ((lane & 3) == 0) {
+            merge_m[warp][row_a] = m_run[0]; merge_l[warp][row_a] = l_run[0];
+            merge_m[warp][row_b] = m_run[1]; merge_l[warp][row_b] = l_run[1];
+        }
+    }
+    __syncthreads();
+    if (tid < 256) {
+        const int col = tid & 127, r0 = (tid >> 7) * 8;
+        const size_t pbase = ((size_t)z * a.n_splits + split) * kRowsPad;
+        for (int row = r0; row < r0 + 8; ++row) {
+            float mx = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kAttConsumers; ++w) mx = fmaxf(mx, merge_m[w][row]);
+            float acc = 0.0f, lsum = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kAttConsumers; ++w) {
+                const float mw = merge_m[w][row];
+                if (mw > -INFINITY) {
+                    const float f = exp2f(mw - mx);
+                    acc += f * merge_o[((size_t)w * kRowsPad + row) * kMergeStride + col];
+                    lsum += f * merge_l[w][row];
+                }
+            }
+            a.part_o[(pbase + row) * kD + col] = acc;
+            if (col == 0) a.part_ml[pbase + row] = make_float2(mx, lsum);
+        }
+    }
+}
+
+// Merge the splits of one (session, layer, KV head) in split order; write O and LSE.
+__global__ void __launch_bounds__(128)
+attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, float* __restrict__ out,
+                    float* __restrict__ lse, int M, int L, int H, int G, int r, int rows, int n_splits) {
+    const int z = blockIdx.x, LG = L * G;
+    const int s = z / LG, lg = z % LG, l = lg / G, g = lg % G;
+    const int col = threadIdx.x;
+    for (int row = 0; row < rows; ++row) {
+        float mx = -INFINITY;
+        for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, part_ml[((size_t)z * n_splits + sp) * kRowsPad + row].x);
+        float acc = 0.0f, lsum = 0.0f;
+        for (int sp = 0; sp < n_splits; ++sp) {
+            const size_t pi = ((size_t)z * n_splits + sp) * kRowsPad + row;
+            const float2 ml = part_ml[pi];
+            if (ml.x > -INFINITY) {
+                const float f = exp2f(ml.x - mx);
+                acc += f * part_o[pi * kD + col];
+                lsum += f * ml.y;
+            }
+        }
+        const int m = row / r, hr = row % r;
+        const size_t orow = (((size_t)s * M + m) * L + l) * H + (size_t)g * r + hr;
+        out[orow * kD + col] = lsum > 0.0f ? acc / lsum : 0.0f;
+        if (col == 0) lse[orow] = lsum > 0.0f ? (mx + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
+    }
+}
+
+static PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+    }
+    return fn;
+}
+
+// view [heads][cap_tokens][128] bf16 as a 3-D tensor; box = 64 dims x 64 tokens x 1 head, 128-byte swizzle
+static bool make_view_map(CUtensorMap* map, const __nv_bfloat16* view, int heads, int cap_tokens) {
+    PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)cap_tokens, (cuuint64_t)heads};
+    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)cap_tokens * kD * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)kTile, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(view), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M,
+                          const __nv_bfloat16* view_k, const __nv_bfloat16* view_v, int view_cap_tokens,
+                          const int32_t* n_sel, float scale, float* out, float* lse, void* workspace,
+                          cudaStream_t st) {
+    const Geometry& g = p.geo;
+    const int LG = g.L * g.G, heads = n_sessions * LG;
+    CUtensorMap map_k, map_v;
+    if (!make_view_map(&map_k, view_k, heads, view_cap_tokens) || !make_view_map(&map_v, view_v, heads, view_cap_tokens))
+        return cudaErrorInvalidValue;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(attend_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    AttendPlan plan = plan_attend(p.cfg, n_sessions, M, p.sm_count);
+    AttendArgs a{};
+    a.q = q; a.n_sel = n_sel;
+    a.part_o = reinterpret_cast<float*>(workspace);
+    a.part_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(workspace) + plan.part_o_bytes);
+    a.status = p.status_dev;
+    a.M = M; a.L = g.L; a.H = g.H; a.G = g.G; a.r = g.r; a.rows = M * g.r;
+    a.n_splits = choose_splits(heads, view_cap_tokens / kTile, p.sm_count);
+    a.cap_tokens = view_cap_tokens;
+    const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
+    a.scale_log2e = sc * 1.4426950408889634f;
+    dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
+    attend_split_kernel<<<grid, kAttThreads, kAttSmem, st>>>(map_k, map_v, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    attend_merge_kernel<<<heads, kD, 0, st>>>(a.part_o, a.part_ml, out, lse, M, g.L, g.H, g.G, g.r, a.rows, a.n_splits);
+    return cudaGetLastError();
+}
+
+}  // namespace kvmem

@@ -1,0 +1,108 @@
+// Internal declarations shared by the translation units of libkvmem_b200 (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "kvmem.h"
+
+namespace kvmem {
+
+constexpr int kSMs = 148;                 // B200: 2 dies x 74 SMs
+constexpr uint32_t kSpinLimit = 1u << 24;            // bounded waits: try_wait attempts before a kernel gives up
+constexpr uint64_t kWaitLimitNs = 1000ull * 1000 * 1000;  // ... or about one second of wall time
+
+// ---- device-resident layout inside the caller's storage --------------------------------------
+//   pages   [max_blocks][2 (K|V)][L][G][B][d] bf16   one (block, K|V, l, g) tile is B*d*2 contiguous bytes
+//   index   [max_sessions][L][G][max_blocks_per_session][d] bf16
+//   tables  [max_sessions][max_blocks_per_session] int32 (logical -> physical page)
+//   nblocks [max_sessions] int32
+//   status  int32 (sticky device status word)
+struct Layout {
+    size_t pages_off, index_off, tables_off, nblocks_off, status_off, total;
+    size_t page_elems;  // bf16 elements per page
+    size_t tile_elems;  // B * d
+    size_t index_elems_per_session;
+};
+
+struct Geometry {
+    int L, H, G, d, B, r;
+    int max_sessions, max_blocks, max_bps;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool config_valid(const kvmem_pool_config_t& c, const char** why);
+Layout make_layout(const kvmem_pool_config_t& c);
+
+}  // namespace kvmem
+
+struct kvmem_pool {
+    uint64_t magic;
+    kvmem_pool_config_t cfg;
+    kvmem::Geometry geo;
+    kvmem::Layout lay;
+    char* base;                         // DEVICE storage
+    __nv_bfloat16* pages;
+    __nv_bfloat16* index;
+    int32_t* tables;
+    int32_t* nblocks_dev;
+    int32_t* status_dev;
+    std::vector<int32_t> sess_blocks;               // host mirror of nblocks
+    std::vector<std::vector<int32_t>> sess_pages;   // host mirror of tables
+    std::vector<uint8_t> page_used;
+    int32_t free_hint;
+    int sm_count;
+};
+
+namespace kvmem {
+
+constexpr uint64_t kMagic = 0x4b564d454d423230ull;  // "KVMEMB20"
+
+void set_error(const char* fmt, ...);
+
+// tuning switches (kvmem_set_option)
+extern int g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
+
+// ---- kernel launchers (each defined next to its kernel) ----------------------------------------
+// All return cudaGetLastError() after the launch.
+
+cudaError_t launch_append(const kvmem_pool& p, int session, int b_first, int n_blocks, const __nv_bfloat16* k,
+                          const __nv_bfloat16* v, cudaStream_t st);
+
+struct ScoreWorkspace {
+    float* logits;     // [ns][L][G][rows_pad][nb_pad]
+    float2* partials;  // [ns][L][G][rows_pad][n_chunks]
+    float* scores;     // [ns][max_bps]  (used when the caller passes no score buffer)
+    size_t logits_bytes, partials_bytes, scores_bytes, total;
+    int rows, rows_pad, nb_pad, n_chunks;
+};
+ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, char* base);
+
+cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q,
+                                int M, const ScoreWorkspace& ws, float* scores, int scores_stride, cudaStream_t st);
+
+cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, const float* scores,
+                        int scores_stride, const kvmem_select_params_t& prm, int32_t* sel_ids, int sel_stride,
+                        int32_t* n_sel, cudaStream_t st);
+
+cudaError_t launch_gather(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids,
+                          int sel_stride, const int32_t* n_sel, __nv_bfloat16* view_k, __nv_bfloat16* view_v,
+                          int view_cap_tokens, cudaStream_t st);
+
+struct AttendPlan {
+    int n_splits;
+    int rows_pad;          // 16
+    size_t part_o_bytes, part_ml_bytes, total;
+};
+AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, int sm_count);
+
+cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M,
+                          const __nv_bfloat16* view_k, const __nv_bfloat16* view_v, int view_cap_tokens,
+                          const int32_t* n_sel, float scale, float* out, float* lse, void* workspace,
+                          cudaStream_t st);
+
+}  // namespace kvmem

@@ -1,0 +1,277 @@
+"""ctypes binding of libkvmem_b200.so: argument marshalling only.
+
+Every step of the recall path (index build, scoring, selection, view assembly, attention)
+runs in the library's CUDA kernels; PyTorch supplies device memory and streams.  There is no
+CPU fallback: if the shared library is missing or a call fails, an exception is raised.
+Names mirror the C ABI declared in ``include/kvmem.h``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+from . import _build
+
+OK = 0
+E_INVALID, E_CAPACITY, E_STATE, E_CUDA, E_TIMEOUT, E_UNSUPPORTED, E_DEVICE_RANGE = -1, -2, -3, -4, -5, -6, -7
+
+
+class KvmemError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"kvmem status {status}: {message}")
+        self.status = status
+
+
+class PoolConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "block_tokens",
+                                          "max_sessions", "max_blocks", "max_blocks_per_session", "device")]
+
+
+class SelectParams(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("budget_blocks", "max_view_tokens", "mandatory_tokens",
+                                          "n_sink_blocks", "n_recent_blocks")]
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> C.CDLL:
+    """Load (building first if sources are newer) the CUDA library.  Raises if that is impossible."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    if path is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path) or os.environ.get("KVMEM_REBUILD"):
+            _build.build()
+    if not os.path.exists(path):
+        raise FileNotFoundError(f"{path} is missing: build it with paper_2609_04852_b200._build.build()")
+    L = C.CDLL(path)
+    vp, i32, sz, f32 = C.c_void_p, C.c_int32, C.c_size_t, C.c_float
+    cfgp, prmp = C.POINTER(PoolConfig), C.POINTER(SelectParams)
+    sig = {
+        "kvmem_pool_bytes": (sz, [cfgp]),
+        "kvmem_budget_blocks": (i32, [prmp, i32, i32]),
+        "kvmem_select_workspace_bytes": (sz, [cfgp, i32, i32]),
+        "kvmem_attend_workspace_bytes": (sz, [cfgp, i32, i32]),
+        "kvmem_last_error": (C.c_char_p, []),
+        "kvmem_pool_create": (C.c_int, [cfgp, vp, sz, C.POINTER(vp)]),
+        "kvmem_pool_destroy": (C.c_int, [vp]),
+        "kvmem_session_reset": (C.c_int, [vp, i32]),
+        "kvmem_session_blocks": (i32, [vp, i32]),
+        "kvmem_append_blocks": (C.c_int, [vp, i32, vp, vp, i32, C.POINTER(i32), vp]),
+        "kvmem_select": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, sz, vp]),
+        "kvmem_materialize": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, vp]),
+        "kvmem_view_attend": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
+        "kvmem_get_index": (C.c_int, [vp, i32, C.POINTER(vp), C.POINTER(i32)]),
+        "kvmem_get_block_table": (C.c_int, [vp, i32, C.POINTER(vp), C.POINTER(i32)]),
+        "kvmem_device_status": (C.c_int, [vp, C.POINTER(i32), vp]),
+        "kvmem_set_option": (C.c_int, [C.c_char_p, i32]),
+        "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
+        "kvmem_recall_step_host": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, i32, f32, vp, vp,
+                                             vp, sz, vp, sz, vp, sz, vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(L, name)
+        fn.restype, fn.argtypes = res, args
+    if path == _build.LIB_PATH:
+        _lib = L
+    return L
+
+
+EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_bytes",
+            "kvmem_attend_workspace_bytes", "kvmem_last_error", "kvmem_pool_create", "kvmem_pool_destroy",
+            "kvmem_session_reset", "kvmem_session_blocks", "kvmem_append_blocks", "kvmem_select",
+            "kvmem_materialize", "kvmem_view_attend", "kvmem_get_index", "kvmem_get_block_table",
+            "kvmem_device_status", "kvmem_set_option", "kvmem_step_staging_bytes", "kvmem_recall_step_host")
+
+
+def _check(status: int) -> None:
+    if status != OK:
+        raise KvmemError(status, load_library().kvmem_last_error().decode())
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype=None) -> int:
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def budget_blocks(params: SelectParams, block_tokens: int, n_blocks: int) -> int:
+    return int(load_library().kvmem_budget_blocks(C.byref(params), block_tokens, n_blocks))
+
+
+def set_option(name: str, value: int) -> None:
+    _check(load_library().kvmem_set_option(name.encode(), value))
+
+
+@dataclass
+class View:
+    """Execution view buffers: bf16 [n_sessions][L][G][cap_tokens][d] each."""
+    k: torch.Tensor
+    v: torch.Tensor
+    cap_tokens: int
+
+
+class Pool:
+    """A paged KV repository with its Mean-K index, living in one torch uint8 tensor."""
+
+    def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, block_tokens: int,
+                 max_sessions: int, max_blocks: int, max_blocks_per_session: int, device: int = 0):
+        self.lib = load_library()
+        self.cfg = PoolConfig(n_layers, n_q_heads, n_kv_heads, head_dim, block_tokens, max_sessions, max_blocks,
+                              max_blocks_per_session, device)
+        nbytes = self.lib.kvmem_pool_bytes(C.byref(self.cfg))
+        if nbytes == 0:
+            raise KvmemError(E_INVALID, self.lib.kvmem_last_error().decode())
+        self.device = torch.device("cuda", device)
+        self.storage = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        self.handle = C.c_void_p()
+        _check(self.lib.kvmem_pool_create(C.byref(self.cfg), self.storage.data_ptr(), nbytes, C.byref(self.handle)))
+        self._select_ws: Optional[torch.Tensor] = None
+        self._attend_ws: Optional[torch.Tensor] = None
+        self._staging: Optional[torch.Tensor] = None
+
+    # ---- lifetime
+    def close(self) -> None:
+        if self.handle:
+            self.lib.kvmem_pool_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- repository
+    def session_reset(self, session: int) -> None:
+        _check(self.lib.kvmem_session_reset(self.handle, session))
+
+    def session_blocks(self, session: int) -> int:
+        n = self.lib.kvmem_session_blocks(self.handle, session)
+        if n < 0:
+            _check(n)
+        return n
+
+    def append_blocks(self, session: int, k: torch.Tensor, v: torch.Tensor,
+                      phys_ids: Optional[Sequence[int]] = None) -> None:
+        c = self.cfg
+        per_block = c.block_tokens * c.n_layers * c.n_kv_heads * c.head_dim
+        if k.numel() % per_block or k.shape != v.shape:
+            raise KvmemError(E_INVALID, "k and v must hold whole blocks of identical shape")
+        n = k.numel() // per_block
+        ids = None
+        if phys_ids is not None:
+            if len(phys_ids) != n:
+                raise KvmemError(E_INVALID, "one page id per block")
+            ids = (C.c_int32 * n)(*[int(x) for x in phys_ids])
+        _check(self.lib.kvmem_append_blocks(self.handle, session, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16),
+                                            n, ids, _stream()))
+
+    # ---- the recall step
+    def select_workspace(self, n_sessions: int, n_q_tokens: int) -> torch.Tensor:
+        need = self.lib.kvmem_select_workspace_bytes(C.byref(self.cfg), n_sessions, n_q_tokens)
+        if need == 0:
+            raise KvmemError(E_INVALID, self.lib.kvmem_last_error().decode())
+        if self._select_ws is None or self._select_ws.numel() < need:
+            self._select_ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        return self._select_ws
+
+    def attend_workspace(self, n_sessions: int, n_q_tokens: int) -> torch.Tensor:
+        need = self.lib.kvmem_attend_workspace_bytes(C.byref(self.cfg), n_sessions, n_q_tokens)
+        if need == 0:
+            raise KvmemError(E_INVALID, self.lib.kvmem_last_error().decode())
+        if self._attend_ws is None or self._attend_ws.numel() < need:
+            self._attend_ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        return self._attend_ws
+
+    def select(self, q: torch.Tensor, params: SelectParams, sel_ids: torch.Tensor, n_sel: torch.Tensor,
+               scores: Optional[torch.Tensor] = None, session_first: int = 0) -> None:
+        """q bf16 [n_sessions][M][L][H][d]; sel_ids int32 [n_sessions][stride]; n_sel int32 [n_sessions]."""
+        ns, M = q.shape[0], q.shape[1]
+        ws = self.select_workspace(ns, M)
+        _check(self.lib.kvmem_select(self.handle, session_first, ns, _dev(q, torch.bfloat16), M, C.byref(params),
+                                     _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
+                                     None if scores is None else _dev(scores, torch.float32),
+                                     ws.data_ptr(), ws.numel(), _stream()))
+
+    def materialize(self, sel_ids: torch.Tensor, n_sel: torch.Tensor, view: View, session_first: int = 0) -> None:
+        ns = n_sel.shape[0]
+        _check(self.lib.kvmem_materialize(self.handle, session_first, ns, _dev(sel_ids, torch.int32),
+                                          sel_ids.shape[-1], _dev(n_sel, torch.int32), _dev(view.k, torch.bfloat16),
+                                          _dev(view.v, torch.bfloat16), view.cap_tokens, _stream()))
+
+    def view_attend(self, q: torch.Tensor, view: View, n_sel: torch.Tensor, out: torch.Tensor, lse: torch.Tensor,
+                    scale: float = 0.0) -> None:
+        ns, M = q.shape[0], q.shape[1]
+        ws = self.attend_workspace(ns, M)
+        _check(self.lib.kvmem_view_attend(self.handle, ns, _dev(q, torch.bfloat16), M, _dev(view.k, torch.bfloat16),
+                                          _dev(view.v, torch.bfloat16), view.cap_tokens, _dev(n_sel, torch.int32),
+                                          scale, _dev(out, torch.float32), _dev(lse, torch.float32),
+                                          ws.data_ptr(), ws.numel(), _stream()))
+
+    def recall_step_host(self, q_host: torch.Tensor, params: SelectParams, sel_ids: torch.Tensor,
+                         n_sel: torch.Tensor, view: View, out_host: torch.Tensor, lse_host: torch.Tensor,
+                         scale: float = 0.0, session_first: int = 0) -> None:
+        """Whole step with HOST query and results (the library does the copies and waits for the stream)."""
+        ns, M = q_host.shape[0], q_host.shape[1]
+        for t, dt in ((q_host, torch.bfloat16), (out_host, torch.float32), (lse_host, torch.float32)):
+            if t.is_cuda or not t.is_contiguous() or t.dtype != dt:
+                raise ValueError("expected contiguous CPU tensors (bf16 query, fp32 outputs)")
+        need = self.lib.kvmem_step_staging_bytes(C.byref(self.cfg), ns, M)
+        if self._staging is None or self._staging.numel() < need:
+            self._staging = torch.empty(need, dtype=torch.uint8, device=self.device)
+        sws, aws = self.select_workspace(ns, M), self.attend_workspace(ns, M)
+        _check(self.lib.kvmem_recall_step_host(
+            self.handle, session_first, ns, q_host.data_ptr(), M, C.byref(params), _dev(sel_ids, torch.int32),
+            sel_ids.shape[-1], _dev(n_sel, torch.int32), _dev(view.k, torch.bfloat16), _dev(view.v, torch.bfloat16),
+            view.cap_tokens, scale, out_host.data_ptr(), lse_host.data_ptr(), self._staging.data_ptr(),
+            self._staging.numel(), sws.data_ptr(), sws.numel(), aws.data_ptr(), aws.numel(), _stream()))
+
+    # ---- helpers that only allocate
+    def new_view(self, n_sessions: int, cap_tokens: int) -> View:
+        c = self.cfg
+        shape = (n_sessions, c.n_layers, c.n_kv_heads, cap_tokens, c.head_dim)
+        return View(torch.zeros(shape, dtype=torch.bfloat16, device=self.device),
+                    torch.zeros(shape, dtype=torch.bfloat16, device=self.device), cap_tokens)
+
+    def new_outputs(self, n_sessions: int, n_q_tokens: int) -> Tuple[torch.Tensor, torch.Tensor]:
+        c = self.cfg
+        out = torch.empty(n_sessions, n_q_tokens, c.n_layers, c.n_q_heads, c.head_dim, dtype=torch.float32,
+                          device=self.device)
+        lse = torch.empty(n_sessions, n_q_tokens, c.n_layers, c.n_q_heads, dtype=torch.float32, device=self.device)
+        return out, lse
+
+    # ---- inspection
+    def index(self, session: int) -> torch.Tensor:
+        """Copy of the session's Mean-K index: bf16 [L][G][n_blocks][d]."""
+        ptr, n = C.c_void_p(), C.c_int32()
+        _check(self.lib.kvmem_get_index(self.handle, session, C.byref(ptr), C.byref(n)))
+        c = self.cfg
+        off = (ptr.value - self.storage.data_ptr())
+        elems = c.n_layers * c.n_kv_heads * c.max_blocks_per_session * c.head_dim
+        full = self.storage[off:off + 2 * elems].view(torch.bfloat16).view(c.n_layers, c.n_kv_heads,
+                                                                              c.max_blocks_per_session, c.head_dim)
+        return full[:, :, :n.value, :].clone()
+
+    def block_table(self, session: int) -> torch.Tensor:
+        ptr, n = C.c_void_p(), C.c_int32()
+        _check(self.lib.kvmem_get_block_table(self.handle, session, C.byref(ptr), C.byref(n)))
+        off = ptr.value - self.storage.data_ptr()
+        return self.storage[off:off + 4 * n.value].view(torch.int32).clone()
+
+    def device_status(self) -> int:
+        st = C.c_int32()
+        _check(self.lib.kvmem_device_status(self.handle, C.byref(st), _stream()))
+        return st.value

@@ -1,0 +1,270 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element, on
+the same seeded inputs.  Index, selected ids and gathered views: bit-exact.  Scores: 1e-3
+relative.  Attention outputs and log-sum-exp: 2e-3 max-abs on unit-scale values.
+"""
+import numpy as np
+import pytest
+import torch
+
+from kvmem_harness import (ATTN_ATOL, bits, check_scores, check_selection, fill_oracle, fill_pool, queries)
+from kvmem_workloads import CONFIGS, planted_blocks
+from oracle import kvmem_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+SMALL = CONFIGS["tiny"].with_(name="small", n_blocks=200, n_planted=6, budget_blocks=24)   # ragged: 200 = 128 + 72
+
+
+def _params(**kw):
+    from paper_2609_04852_b200 import SelectParams
+    base = dict(budget_blocks=0, max_view_tokens=1 << 30, mandatory_tokens=0, n_sink_blocks=0, n_recent_blocks=0)
+    base.update(kw)
+    return SelectParams(**base)
+
+
+def _run_step(pool, spec, q_dev, params, cap_blocks, n_sessions=None, attend=True):
+    """select -> materialize -> attend through the C ABI; returns host copies."""
+    ns = spec.n_sessions if n_sessions is None else n_sessions
+    dev = q_dev.device
+    sel = torch.full((ns, max(cap_blocks, 1)), -1, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(ns, dtype=torch.int32, device=dev)
+    scores = torch.zeros(ns, spec.n_blocks, dtype=torch.float32, device=dev)
+    view = pool.new_view(ns, max(cap_blocks, 1) * spec.block_tokens)
+    pool.select(q_dev, params, sel, n_sel, scores)
+    pool.materialize(sel, n_sel, view)
+    out = lse = None
+    if attend:
+        out, lse = pool.new_outputs(ns, spec.n_q_tokens)
+        pool.view_attend(q_dev, view, n_sel, out, lse)
+    assert pool.device_status() == 0
+    return dict(sel=sel.cpu().numpy(), n_sel=n_sel.cpu().numpy(), scores=scores.cpu().numpy(), view=view,
+                out=None if out is None else out.cpu().numpy(), lse=None if lse is None else lse.cpu().numpy())
+
+
+def _oracle_step(spec, osess, qb, s, budget, max_view=1 << 30, mandatory=0, sink=0, recent=0, sel_override=None):
+    R, _ = orc.block_scores(qb[s], osess.idx, osess.n_blocks)
+    sel = orc.select(R, spec.block_tokens, budget, max_view, mandatory, sink, recent)
+    use = sel if sel_override is None else sel_override
+    cap = max(len(use), 1) * spec.block_tokens
+    vK, vV = orc.gather(osess.repo, osess.table, use, cap)
+    out, lse = orc.attend(qb[s], vK, vV, len(use) * spec.block_tokens)
+    return dict(R=R, sel=sel, vK=vK, vV=vV, out=out, lse=lse)
+
+
+def _compare_step(spec, got, s, ref, sink=0, recent=0):
+    n = int(got["n_sel"][s])
+    sel_gpu = got["sel"][s, :n]
+    check_scores(got["scores"][s, :len(ref["R"])], ref["R"], spec.n_q_tokens)
+    how = check_selection(sel_gpu, ref["R"], ref["sel"], sink, recent)
+    return sel_gpu, how
+
+
+def _compare_view_and_attention(spec, got, s, ref_same_ids):
+    n = int(got["n_sel"][s])
+    T = n * spec.block_tokens
+    gk, gv = bits(got["view"].k[s]), bits(got["view"].v[s])
+    assert np.array_equal(gk[:, :, :T], ref_same_ids["vK"][:, :, :T]), "gathered K differs"
+    assert np.array_equal(gv[:, :, :T], ref_same_ids["vV"][:, :, :T]), "gathered V differs"
+    if got["out"] is not None:
+        err_o = np.abs(got["out"][s] - ref_same_ids["out"]).max()
+        if T == 0:                                                   # empty view: lse is -inf on both sides
+            assert np.all(np.isneginf(got["lse"][s])) and np.all(np.isneginf(ref_same_ids["lse"]))
+            assert err_o == 0
+            return
+        err_l = np.abs(got["lse"][s] - ref_same_ids["lse"]).max()
+        assert err_o <= ATTN_ATOL and err_l <= ATTN_ATOL, f"attention error {err_o:.2e} / lse {err_l:.2e}"
+        rel = err_o / max(np.abs(ref_same_ids["out"]).max(), 1e-30)
+        assert rel < 5e-2, f"relative attention error {rel:.2e}"          # the absolute bound must not be vacuous
+
+
+# ------------------------------------------------------------------ index
+
+@pytest.mark.parametrize("spec", [SMALL, SMALL.with_(n_layers=2, n_kv_heads=4, n_q_heads=8, block_tokens=32, n_blocks=37)],
+                         ids=["L1G8B64", "L2G4B32"])
+def test_index_and_block_table_bit_exact(spec):
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    assert np.array_equal(bits(pool.index(0)), osess.idx)
+    assert np.array_equal(pool.block_table(0).cpu().numpy(), osess.table[:spec.n_blocks])
+    assert pool.device_status() == 0
+
+
+# ------------------------------------------------------------------ whole step on small workspaces
+
+@pytest.mark.parametrize("M", [1, 2, 4])
+@pytest.mark.parametrize("gather_mode", [1, 0])
+def test_step_matches_oracle_small(M, gather_mode):
+    from paper_2609_04852_b200 import set_option
+    spec = SMALL.with_(n_q_tokens=M)
+    set_option("gather_mode", gather_mode)
+    try:
+        pool = fill_pool(spec)
+        osess = fill_oracle(spec)[0]
+        for qset in range(2):
+            q, qb = queries(spec, qset)
+            got = _run_step(pool, spec, q.cuda(), _params(budget_blocks=spec.budget_blocks), spec.budget_blocks)
+            ref = _oracle_step(spec, osess, qb, 0, spec.budget_blocks)
+            sel_gpu, _ = _compare_step(spec, got, 0, ref)
+            same = _oracle_step(spec, osess, qb, 0, spec.budget_blocks, sel_override=sel_gpu)
+            _compare_view_and_attention(spec, got, 0, same)
+    finally:
+        set_option("gather_mode", 1)
+
+
+def test_gap_forced_selection_is_identical_and_recovers_planted_blocks():
+    spec = SMALL
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    q, qb = queries(spec)
+    got = _run_step(pool, spec, q.cuda(), _params(budget_blocks=spec.n_planted), spec.n_planted)
+    ref = _oracle_step(spec, osess, qb, 0, spec.n_planted)
+    sel_gpu, how = _compare_step(spec, got, 0, ref)
+    assert how == "exact" and np.array_equal(sel_gpu, ref["sel"])
+    assert set(sel_gpu.tolist()) == set(planted_blocks(spec, 0)[0].tolist())
+    _compare_view_and_attention(spec, got, 0, ref)
+
+
+@pytest.mark.parametrize("budget,max_view,mandatory,sink,recent", [
+    (10 ** 6, 1 << 30, 0, 0, 0),        # k >= NB: the view is the whole history
+    (24, 64 * 10, 1, 0, 0),             # capacity clamp: floor((640 - 1) / 64) = 9 blocks
+    (24, 1 << 30, 0, 3, 5),             # sink + recent reservation
+    (6, 1 << 30, 0, 4, 4),              # reservation larger than the budget
+    (0, 1 << 30, 0, 0, 0),              # empty selection
+    (1, 1 << 30, 0, 0, 0),
+])
+def test_budget_and_reservation_edge_cases(budget, max_view, mandatory, sink, recent):
+    spec = SMALL
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    q, qb = queries(spec, 1)
+    k = orc.budget_blocks(spec.n_blocks, spec.block_tokens, budget, max_view, mandatory)
+    prm = _params(budget_blocks=min(budget, 2 ** 31 - 1), max_view_tokens=max_view, mandatory_tokens=mandatory,
+                  n_sink_blocks=sink, n_recent_blocks=recent)
+    from paper_2609_04852_b200 import budget_blocks
+    assert budget_blocks(prm, spec.block_tokens, spec.n_blocks) == k
+    got = _run_step(pool, spec, q.cuda(), prm, k)
+    ref = _oracle_step(spec, osess, qb, 0, budget, max_view, mandatory, sink, recent)
+    assert int(got["n_sel"][0]) == k == len(ref["sel"])
+    sel_gpu, _ = _compare_step(spec, got, 0, ref, sink, recent)
+    same = _oracle_step(spec, osess, qb, 0, budget, max_view, mandatory, sink, recent, sel_override=sel_gpu)
+    _compare_view_and_attention(spec, got, 0, same)
+    if k == 0:
+        assert not got["out"].any() and np.all(np.isneginf(got["lse"]))
+
+
+def test_selecting_everything_equals_full_attention_over_raw_history():
+    spec = SMALL.with_(n_blocks=70, n_q_tokens=4)
+    pool = fill_pool(spec)
+    q, qb = queries(spec)
+    got = _run_step(pool, spec, q.cuda(), _params(budget_blocks=10 ** 6), spec.n_blocks)
+    assert got["sel"][0].tolist() == list(range(spec.n_blocks))
+    from kvmem_workloads import kv_blocks
+    K, V = kv_blocks(spec, 0, 0, spec.n_blocks)
+    vK = np.ascontiguousarray(np.transpose(bits(K), (1, 2, 0, 3)))
+    vV = np.ascontiguousarray(np.transpose(bits(V), (1, 2, 0, 3)))
+    out, lse = orc.attend(qb[0], vK, vV, spec.tokens)
+    assert np.abs(got["out"][0] - out).max() <= ATTN_ATOL and np.abs(got["lse"][0] - lse).max() <= ATTN_ATOL
+
+
+def test_duplicate_blocks_tie_break_by_lower_id():
+    # identical keys in every block => identical scores: the selection must be the k lowest ids
+    from paper_2609_04852_b200 import Pool
+    spec = SMALL.with_(n_blocks=40)
+    dev = torch.device("cuda", 0)
+    pool = Pool(1, 32, 8, 128, 64, 1, 40, 40, 0)
+    from kvmem_workloads import kv_blocks
+    K, V = kv_blocks(spec, 0, 0, 1, dev)
+    pool.append_blocks(0, K.repeat(40, 1, 1, 1).contiguous(), V.repeat(40, 1, 1, 1).contiguous())
+    q, _ = queries(spec)
+    got = _run_step(pool, spec.with_(n_blocks=40), q.cuda(), _params(budget_blocks=7), 7)
+    assert got["sel"][0, :7].tolist() == list(range(7))
+    assert np.all(got["scores"][0, :40] == got["scores"][0, 0])
+
+
+# ------------------------------------------------------------------ several sessions, permuted pages
+
+def test_multi_session_ragged_lengths_and_permuted_pages():
+    spec = CONFIGS["batch8"].with_(name="batch3", n_sessions=3, n_blocks=150, n_planted=5, budget_blocks=20)
+    lens = [150, 97, 130]
+    pool = fill_pool(spec, lens)
+    osess = fill_oracle(spec, lens)
+    q, qb = queries(spec)
+    got = _run_step(pool, spec, q.cuda(), _params(budget_blocks=spec.budget_blocks), spec.budget_blocks)
+    for s in range(3):
+        ref = _oracle_step(spec, osess[s], qb, s, spec.budget_blocks)
+        sel_gpu, _ = _compare_step(spec, got, s, ref)
+        same = _oracle_step(spec, osess[s], qb, s, spec.budget_blocks, sel_override=sel_gpu)
+        _compare_view_and_attention(spec, got, s, same)
+
+
+def test_gather_in_isolation_with_oracle_ids():
+    spec = SMALL
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    ids = np.array([0, 3, 4, 77, 128, 199], np.int32)
+    dev = torch.device("cuda", 0)
+    sel = torch.from_numpy(ids).to(dev).view(1, -1).contiguous()
+    n_sel = torch.tensor([len(ids)], dtype=torch.int32, device=dev)
+    view = pool.new_view(1, 8 * spec.block_tokens)
+    view.k.fill_(7.0)
+    pool.materialize(sel, n_sel, view)
+    assert pool.device_status() == 0
+    vK, vV = orc.gather(osess.repo, osess.table, ids, 8 * spec.block_tokens)
+    T = len(ids) * spec.block_tokens
+    assert np.array_equal(bits(view.k[0])[:, :, :T], vK[:, :, :T]) and np.array_equal(bits(view.v[0])[:, :, :T], vV[:, :, :T])
+    assert torch.all(view.k[0][:, :, T:] == 7.0)                 # tokens past the view are untouched
+
+
+def test_out_of_range_ids_are_flagged_not_dereferenced():
+    from paper_2609_04852_b200.kvmem import E_DEVICE_RANGE
+    spec = SMALL
+    pool = fill_pool(spec)
+    dev = torch.device("cuda", 0)
+    sel = torch.tensor([[1, 5000, 7]], dtype=torch.int32, device=dev)
+    n_sel = torch.tensor([3], dtype=torch.int32, device=dev)
+    view = pool.new_view(1, 4 * spec.block_tokens)
+    pool.materialize(sel, n_sel, view)
+    assert pool.device_status() == E_DEVICE_RANGE
+    assert pool.device_status() == 0                              # reading clears the word
+
+
+# ------------------------------------------------------------------ host-side errors leave the pool unchanged
+
+def test_argument_and_capacity_errors():
+    from paper_2609_04852_b200 import KvmemError, Pool
+    from paper_2609_04852_b200.kvmem import E_CAPACITY, E_INVALID, E_STATE, E_UNSUPPORTED
+    spec = SMALL.with_(n_blocks=8)
+    dev = torch.device("cuda", 0)
+    pool = Pool(1, 32, 8, 128, 64, 1, 8, 8, 0)
+    from kvmem_workloads import kv_blocks
+    K, V = kv_blocks(spec, 0, 0, 4, dev)
+    pool.append_blocks(0, K, V, [0, 1, 2, 3])
+    with pytest.raises(KvmemError) as e:
+        pool.append_blocks(0, K, V, [3, 4, 5, 6])                 # page 3 is taken
+    assert e.value.status == E_STATE and pool.session_blocks(0) == 4
+    with pytest.raises(KvmemError) as e:
+        pool.append_blocks(0, K[:100], V[:100])                   # partial block
+    assert e.value.status == E_INVALID
+    pool.append_blocks(0, K, V)
+    with pytest.raises(KvmemError) as e:
+        pool.append_blocks(0, K, V)                               # session and pool are full
+    assert e.value.status == E_CAPACITY and pool.session_blocks(0) == 8
+    q, _ = queries(spec)
+    sel = torch.zeros(1, 2, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    with pytest.raises(KvmemError) as e:
+        pool.select(q.cuda(), _params(budget_blocks=4), sel, n_sel)   # sel_stride 2 < k = 4
+    assert e.value.status == E_CAPACITY
+    with pytest.raises(KvmemError) as e:
+        Pool(1, 32, 5, 128, 64, 1, 8, 8, 0)                       # 32 % 5 != 0
+    assert e.value.status == E_INVALID
+    q17 = torch.zeros(1, 5, 1, 32, 128, dtype=torch.bfloat16, device=dev)
+    view = pool.new_view(1, 8 * 64)
+    out, lse = pool.new_outputs(1, 5)
+    with pytest.raises(KvmemError) as e:
+        pool.view_attend(q17, view, n_sel, out, lse)              # 5 tokens x 4 heads per KV head > 16 rows
+    assert e.value.status == E_UNSUPPORTED
+    pool.session_reset(0)
+    assert pool.session_blocks(0) == 0
+    pool.append_blocks(0, K, V)
+    assert pool.session_blocks(0) == 4 and pool.device_status() == 0
