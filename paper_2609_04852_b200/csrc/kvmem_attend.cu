@@ -265,31 +265,29 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     }
 }
 
-// Merge the splits of one (session, layer, KV head) in split order; write O and LSE.
+// Merge the splits of one query row of one (session, layer, KV head) in split order; write O and LSE.
 __global__ void __launch_bounds__(128)
 attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, float* __restrict__ out,
-                    float* __restrict__ lse, int M, int L, int H, int G, int r, int rows, int n_splits) {
-    const int z = blockIdx.x, LG = L * G;
+                    float* __restrict__ lse, int M, int L, int H, int G, int r, int n_splits) {
+    const int row = blockIdx.x, z = blockIdx.y, LG = L * G;
     const int s = z / LG, lg = z % LG, l = lg / G, g = lg % G;
     const int col = threadIdx.x;
-    for (int row = 0; row < rows; ++row) {
-        float mx = -INFINITY;
-        for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, part_ml[((size_t)z * n_splits + sp) * kRowsPad + row].x);
-        float acc = 0.0f, lsum = 0.0f;
-        for (int sp = 0; sp < n_splits; ++sp) {
-            const size_t pi = ((size_t)z * n_splits + sp) * kRowsPad + row;
-            const float2 ml = part_ml[pi];
-            if (ml.x > -INFINITY) {
-                const float f = exp2f(ml.x - mx);
-                acc += f * part_o[pi * kD + col];
-                lsum += f * ml.y;
-            }
-        }
-        const int m = row / r, hr = row % r;
-        const size_t orow = (((size_t)s * M + m) * L + l) * H + (size_t)g * r + hr;
-        out[orow * kD + col] = lsum > 0.0f ? acc / lsum : 0.0f;
-        if (col == 0) lse[orow] = lsum > 0.0f ? (mx + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
+    const size_t p0 = (size_t)z * n_splits * kRowsPad + row;          // split sp lives at p0 + sp * kRowsPad
+    float mx = -INFINITY;
+    for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, part_ml[p0 + (size_t)sp * kRowsPad].x);
+    float acc = 0.0f, lsum = 0.0f;
+#pragma unroll 4
+    for (int sp = 0; sp < n_splits; ++sp) {
+        const size_t pi = p0 + (size_t)sp * kRowsPad;
+        const float2 ml = part_ml[pi];
+        const float f = ml.x > -INFINITY ? exp2f(ml.x - mx) : 0.0f;
+        acc += f * part_o[pi * kD + col];
+        lsum += f * ml.y;
     }
+    const int m = row / r, hr = row % r;
+    const size_t orow = (((size_t)s * M + m) * L + l) * H + (size_t)g * r + hr;
+    out[orow * kD + col] = lsum > 0.0f ? acc / lsum : 0.0f;
+    if (col == 0) lse[orow] = lsum > 0.0f ? (mx + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
 }
 
 static PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
@@ -348,7 +346,8 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     attend_split_kernel<<<grid, kAttThreads, kAttSmem, st>>>(map_k, map_v, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    attend_merge_kernel<<<heads, kD, 0, st>>>(a.part_o, a.part_ml, out, lse, M, g.L, g.H, g.G, g.r, a.rows, a.n_splits);
+    attend_merge_kernel<<<dim3((unsigned)a.rows, (unsigned)heads), kD, 0, st>>>(a.part_o, a.part_ml, out, lse, M, g.L, g.H, g.G,
+                                                                            g.r, a.n_splits);
     return cudaGetLastError();
 }
 

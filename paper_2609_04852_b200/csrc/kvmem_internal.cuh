@@ -75,7 +75,7 @@ cudaError_t launch_append(const kvmem_pool& p, int session, int b_first, int n_b
 
 struct ScoreWorkspace {
     float* logits;     // [ns][L][G][rows_pad][nb_pad]
-    float2* partials;  // [ns][L][G][rows_pad][n_chunks]
+    float2* partials;  // [ns][L][G][rows_pad][n_parts]: per-CTA (max, sum-exp) of each row
     float* scores;     // [ns][max_bps]  (used when the caller passes no score buffer)
     size_t logits_bytes, partials_bytes, scores_bytes, total;
     int rows, rows_pad, nb_pad, n_chunks;

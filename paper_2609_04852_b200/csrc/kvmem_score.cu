@@ -1,24 +1,30 @@
 // Query-conditioned block scoring for decode-sized queries (Eq. "kvmem-block-score", Sec. 4.3):
 //   R_b = sum_m (1/(L*H)) sum_{l,h} softmax_{b'}( q[l][m][h] . kbar[l][b'][g(h)] / sqrt(d) )_b
 //
-// The index is streamed once.  A CTA owns 128 consecutive blocks of one (session, layer, KV
-// head); a half-warp owns one Mean-K vector (16 lanes x one 128-bit load = 256 B), so a warp reads
-// 512 contiguous bytes per step.  The M*r query rows that share this KV head sit in registers as
+// The index is streamed once.  About one persistent CTA per SM owns a contiguous range of
+// 128-block tiles of one (session, layer, KV head); tiles (32 KiB, contiguous in the index) arrive
+// through a ring of shared-memory stages filled by 1-D TMA bulk copies (mbarrier completion, bounded
+// waits).  A half-warp owns one Mean-K vector (16 lanes x one 128-bit shared-memory load = 256 B).  The M*r query rows that share this KV head sit in registers as
 // fp32; every lane forms its 8-dimension partial dot product for all rows, and a transposing
 // butterfly (15 shuffles for 16 rows) leaves lane i of the half-warp with the finished logit of
 // row i.  Logits (already multiplied by log2(e)/sqrt(d)) are staged in shared memory, written out
-// coalesced, and each CTA records per-row (max, sum-exp) of its tile: the cross-tile softmax
+// coalesced, and each CTA carries per-row (max, sum-exp) across its tiles: the cross-tile softmax
 // statistics that Sec. 5.2 describes for tiled scoring.  A second small kernel merges the tile
 // statistics per row and reduces rows in a fixed order, so results are run-to-run identical.
 #include <math.h>
 
+#include <algorithm>
+
 #include "kvmem_internal.cuh"
+#include "kvmem_ptx.cuh"
 
 namespace kvmem {
 
 constexpr int kChunk = 128;       // blocks per CTA tile
 constexpr int kScoreThreads = 256;
 constexpr int kMaxDecodeTokens = 16;
+constexpr int kScoreStages = 4;   // 32 KiB index tiles in flight per CTA
+constexpr int kMaxScoreParts = 64;
 
 ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, char* base) {
     ScoreWorkspace w{};
@@ -30,7 +36,7 @@ ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions
     const size_t lg = (size_t)c.n_layers * c.n_kv_heads;
     const int rows_store = n_q_tokens <= kMaxDecodeTokens ? w.rows_pad : 16;
     w.logits_bytes = align_up((size_t)n_sessions * lg * rows_store * w.nb_pad * sizeof(float), 256);
-    w.partials_bytes = align_up((size_t)n_sessions * lg * rows_store * w.n_chunks * sizeof(float2), 256);
+    w.partials_bytes = align_up((size_t)n_sessions * lg * rows_store * kMaxScoreParts * sizeof(float2), 256);
     w.scores_bytes = align_up((size_t)n_sessions * c.max_blocks_per_session * sizeof(float), 256);
     w.total = w.logits_bytes + w.partials_bytes + w.scores_bytes;
     if (base) {
@@ -82,25 +88,46 @@ __global__ void __launch_bounds__(kScoreThreads, 1)
 score_logits_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ index,
                     const int32_t* __restrict__ nblocks_dev, int session_first, int M, int L, int H, int G,
                     int max_bps, size_t index_elems_per_session, float* __restrict__ logits,
-                    float2* __restrict__ partials, int rows, int rows_pad, int nb_pad, int n_chunks,
-                    float scale_log2e) {
+                    float2* __restrict__ partials, int rows, int rows_pad, int nb_pad, int n_parts,
+                    float scale_log2e, int32_t* __restrict__ status) {
     constexpr int SH = (RP == 16) ? 0 : (RP == 8) ? 1 : 2;   // lanes per finished row = 1 << SH
+    constexpr int RPW = (RP + 7) / 8;                        // rows whose statistics one warp carries
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ uint64_t full_bar[kScoreStages];
     __shared__ float slog[RP][kChunk + 4];
+    uint4* stage_mem = reinterpret_cast<uint4*>(smem_raw);   // [kScoreStages][kChunk][16] x 16 B
 
-    const int s = blockIdx.z, lg = blockIdx.y, chunk = blockIdx.x;
+    const int s = blockIdx.z, lg = blockIdx.y, part = blockIdx.x;
     const int l = lg / G, g = lg % G, r = H / G;
     const int NB = nblocks_dev[session_first + s];
-    const int b0 = chunk * kChunk;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int hl = lane & 15, hw = tid >> 4;               // lane in half-warp, half-warp in CTA (0..15)
     const size_t slab = ((size_t)s * L * G + lg) * rows_pad;  // first row of this (s, l, g)
-
     const __nv_bfloat16* idx_lg =
         index + (size_t)(session_first + s) * index_elems_per_session + (size_t)lg * max_bps * 128;
 
-    for (int pass = 0; pass * RP < rows_pad; ++pass) {
+    // this CTA's contiguous range of 128-block chunks
+    const int n_chunks = (NB + kChunk - 1) / kChunk;
+    const int c_begin = (int)((long long)n_chunks * part / n_parts), c_end = (int)((long long)n_chunks * (part + 1) / n_parts);
+    const int n_mine = c_end - c_begin;
+
+    if (tid == 0) {
+        for (int i = 0; i < kScoreStages; ++i) ptx::mbar_init(&full_bar[i], 1);
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+
+    int issued = 0, waited = 0;                            // running counts over all passes (barrier phases)
+    auto issue = [&](int chunk) {                          // thread 0 only
+        const int st = issued % kScoreStages;
+        const int b0 = chunk * kChunk;
+        const uint32_t bytes = (uint32_t)min(kChunk, NB - b0) * 256u;
+        ptx::mbar_expect_tx(&full_bar[st], bytes);
+        ptx::bulk_g2s(stage_mem + (size_t)st * kChunk * 16, idx_lg + (size_t)b0 * 128, bytes, &full_bar[st]);
+    };
+
+    for (int pass = 0; pass * RP < rows; ++pass) {
         const int row0 = pass * RP;
-        if (row0 >= rows && pass > 0) break;
         // query rows of this pass, dims [8*hl, 8*hl + 8), as fp32 registers
         float qr[RP][8];
 #pragma unroll
@@ -116,14 +143,31 @@ score_logits_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 for (int c = 0; c < 8; ++c) qr[j][c] = 0.0f;
             }
         }
-        if (b0 < NB) {
+        float run_m[RPW], run_l[RPW];
+#pragma unroll
+        for (int i = 0; i < RPW; ++i) { run_m[i] = -INFINITY; run_l[i] = 0.0f; }
+
+        if (tid == 0) {
+            for (int i = 0; i < min(kScoreStages - 1, n_mine); ++i) { issue(c_begin + i); ++issued; }
+        }
+        for (int i = 0; i < n_mine; ++i) {
+            const int chunk = c_begin + i, b0 = chunk * kChunk;
+            const int st = waited % kScoreStages;
+            const bool ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((waited / kScoreStages) & 1));
+            ++waited;
+            if (__syncthreads_or(!ok)) {                  // CTA-uniform: somebody gave up
+                if (tid == 0) atomicExch(status, (int)KVMEM_E_TIMEOUT);
+                return;
+            }
+            // stage (i - 1) was released by the barrier above: refill it
+            if (tid == 0 && i + kScoreStages - 1 < n_mine) { issue(chunk + kScoreStages - 1); ++issued; }
+            const uint4* tile = stage_mem + (size_t)st * kChunk * 16;
 #pragma unroll 2
             for (int it = 0; it < kChunk / 16; ++it) {
                 const int col = it * 16 + hw;
-                const int blk = b0 + col;
-                const bool valid = blk < NB;
+                const bool valid = b0 + col < NB;
                 uint4 u = make_uint4(0, 0, 0, 0);
-                if (valid) u = __ldg(reinterpret_cast<const uint4*>(idx_lg + (size_t)blk * 128 + hl * 8));
+                if (valid) u = tile[col * 16 + hl];
                 float kf[8];
                 unpack8(u, kf);
                 float acc[RP];
@@ -137,54 +181,59 @@ score_logits_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 halfwarp_transpose_reduce<RP>(acc, hl);
                 if ((hl & ((1 << SH) - 1)) == 0) slog[hl >> SH][col] = valid ? acc[0] * scale_log2e : -INFINITY;
             }
+            __syncthreads();
+            // per-row statistics of this tile (folded into the running pair) and coalesced logit store
+#pragma unroll
+            for (int jj = 0; jj < RPW; ++jj) {
+                const int j = warp + 8 * jj;
+                if (j < RP) {
+                    float mx = -INFINITY, v[kChunk / 32];
+#pragma unroll
+                    for (int t = 0; t < kChunk / 32; ++t) {
+                        v[t] = slog[j][lane + 32 * t];
+                        mx = fmaxf(mx, v[t]);
+                    }
+#pragma unroll
+                    for (int o = 16; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                    const float mn = fmaxf(run_m[jj], mx);      // finite: a chunk holds at least one block
+                    float sum = 0.0f;
+#pragma unroll
+                    for (int t = 0; t < kChunk / 32; ++t) sum += exp2f(v[t] - mn);
+#pragma unroll
+                    for (int o = 16; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+                    run_l[jj] = run_l[jj] * exp2f(run_m[jj] - mn) + sum;
+                    run_m[jj] = mn;
+                    float* dst = logits + (slab + row0 + j) * (size_t)nb_pad + b0;
+#pragma unroll
+                    for (int t = 0; t < kChunk / 32; ++t) dst[lane + 32 * t] = v[t];
+                }
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        // per-row statistics of this tile and coalesced logit store
-        for (int j = warp; j < RP; j += kScoreThreads / 32) {
-            const int row = row0 + j;
-            float mx = -INFINITY, v[kChunk / 32];
 #pragma unroll
-            for (int i = 0; i < kChunk / 32; ++i) {
-                v[i] = (b0 < NB) ? slog[j][lane + 32 * i] : -INFINITY;
-                mx = fmaxf(mx, v[i]);
-            }
-#pragma unroll
-            for (int o = 16; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            float sum = 0.0f;
-            if (mx > -INFINITY) {
-#pragma unroll
-                for (int i = 0; i < kChunk / 32; ++i) sum += exp2f(v[i] - mx);
-            }
-#pragma unroll
-            for (int o = 16; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (row < rows_pad) {
-                if (lane == 0) partials[(slab + row) * n_chunks + chunk] = make_float2(mx, sum);
-                float* dst = logits + (slab + row) * (size_t)nb_pad + b0;
-#pragma unroll
-                for (int i = 0; i < kChunk / 32; ++i) dst[lane + 32 * i] = v[i];
-            }
+        for (int jj = 0; jj < RPW; ++jj) {
+            const int j = warp + 8 * jj;
+            if (j < RP && lane == 0) partials[(slab + row0 + j) * n_parts + part] = make_float2(run_m[jj], run_l[jj]);
         }
-        __syncthreads();
     }
 }
 
-// Merge the tile statistics of every row, then R_b = (1/(L*H)) sum_rows exp2(logit - max_row) / Z_row.
+// Merge the per-CTA statistics of every row, then R_b = (1/(L*H)) sum_rows exp2(logit - max_row) / Z_row.
 __global__ void __launch_bounds__(256)
 score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__ partials,
                     const int32_t* __restrict__ nblocks_dev, int session_first, int LG, int rows, int rows_pad,
-                    int nb_pad, int n_chunks, float inv_LH, float* __restrict__ scores, int scores_stride) {
+                    int nb_pad, int n_parts, float inv_LH, float* __restrict__ scores, int scores_stride) {
     extern __shared__ float2 rowstat[];   // [LG * rows] : (max, 1/Z)
     const int s = blockIdx.y;
     const int NB = nblocks_dev[session_first + s];
     if ((int)(blockIdx.x * blockDim.x) >= NB) return;
-    const int live_chunks = min(n_chunks, (NB + kChunk - 1) / kChunk);
     for (int i = threadIdx.x; i < LG * rows; i += blockDim.x) {
         const int lg = i / rows, j = i % rows;
-        const float2* p = partials + (((size_t)s * LG + lg) * rows_pad + j) * n_chunks;
+        const float2* p = partials + (((size_t)s * LG + lg) * rows_pad + j) * n_parts;
         float mx = -INFINITY;
-        for (int c = 0; c < live_chunks; ++c) mx = fmaxf(mx, p[c].x);
+        for (int c = 0; c < n_parts; ++c) mx = fmaxf(mx, p[c].x);
         float z = 0.0f;
-        for (int c = 0; c < live_chunks; ++c) {
+        for (int c = 0; c < n_parts; ++c) {
             const float2 t = p[c];
             if (t.x > -INFINITY) z += t.y * exp2f(t.x - mx);
         }
@@ -197,6 +246,7 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
     for (int lg = 0; lg < LG; ++lg) {
         const float* base = logits + (((size_t)s * LG + lg) * rows_pad) * (size_t)nb_pad + b;
         float part = 0.0f;
+#pragma unroll 8
         for (int j = 0; j < rows; ++j) {
             const float2 st = rowstat[lg * rows + j];
             part += exp2f(base[(size_t)j * nb_pad] - st.x) * st.y;
@@ -214,30 +264,40 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     int max_nb = 0;
     for (int s = session_first; s < session_first + n_sessions; ++s) max_nb = std::max(max_nb, p.sess_blocks[s]);
     if (max_nb == 0) return cudaSuccess;
-    const int chunks = (max_nb + kChunk - 1) / kChunk;
-    dim3 grid((unsigned)chunks, (unsigned)(g.L * g.G), (unsigned)n_sessions);
-#define KVMEM_SCORE_ARGS                                                                                           \
-    q, p.index, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, p.lay.index_elems_per_session, ws.logits, \
-        ws.partials, ws.rows, ws.rows_pad, ws.nb_pad, ws.n_chunks, scale_log2e
-    if (ws.rows <= 4)
-        score_logits_kernel<4><<<grid, kScoreThreads, 0, st>>>(KVMEM_SCORE_ARGS);
-    else if (ws.rows <= 8)
-        score_logits_kernel<8><<<grid, kScoreThreads, 0, st>>>(KVMEM_SCORE_ARGS);
-    else
-        score_logits_kernel<16><<<grid, kScoreThreads, 0, st>>>(KVMEM_SCORE_ARGS);
-#undef KVMEM_SCORE_ARGS
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
     const int LG = g.L * g.G;
-    const size_t smem = (size_t)LG * ws.rows * sizeof(float2);
-    if (smem > 48 * 1024) {
-        e = cudaFuncSetAttribute(score_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const int chunks = (max_nb + kChunk - 1) / kChunk;
+    // persistent CTAs: about one per SM, each streaming a contiguous range of chunks of one (session, l, g)
+    const int n_parts = std::max(1, std::min({chunks, kMaxScoreParts, p.sm_count / std::max(1, LG * n_sessions)}));
+    const size_t smem = (size_t)kScoreStages * kChunk * 256;
+    dim3 grid((unsigned)n_parts, (unsigned)LG, (unsigned)n_sessions);
+    cudaError_t e;
+#define KVMEM_SCORE_LAUNCH(RP)                                                                                         \
+    do {                                                                                                               \
+        static bool attr_done = false;                                                                                 \
+        if (!attr_done) {                                                                                              \
+            e = cudaFuncSetAttribute(score_logits_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+            if (e != cudaSuccess) return e;                                                                            \
+            attr_done = true;                                                                                          \
+        }                                                                                                              \
+        score_logits_kernel<RP><<<grid, kScoreThreads, smem, st>>>(                                                    \
+            q, p.index, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, p.lay.index_elems_per_session,      \
+            ws.logits, ws.partials, ws.rows, ws.rows_pad, ws.nb_pad, n_parts, scale_log2e, p.status_dev);              \
+    } while (0)
+    if (ws.rows <= 4) KVMEM_SCORE_LAUNCH(4);
+    else if (ws.rows <= 8) KVMEM_SCORE_LAUNCH(8);
+    else KVMEM_SCORE_LAUNCH(16);
+#undef KVMEM_SCORE_LAUNCH
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t fsmem = (size_t)LG * ws.rows * sizeof(float2);
+    if (fsmem > 48 * 1024) {
+        e = cudaFuncSetAttribute(score_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsmem);
         if (e != cudaSuccess) return e;
     }
     dim3 fgrid((unsigned)((max_nb + 255) / 256), (unsigned)n_sessions);
-    score_finish_kernel<<<fgrid, 256, smem, st>>>(ws.logits, ws.partials, p.nblocks_dev, session_first, LG, ws.rows,
-                                                  ws.rows_pad, ws.nb_pad, ws.n_chunks, 1.0f / (float)(g.L * g.H),
-                                                  scores, scores_stride);
+    score_finish_kernel<<<fgrid, 256, fsmem, st>>>(ws.logits, ws.partials, p.nblocks_dev, session_first, LG, ws.rows,
+                                                   ws.rows_pad, ws.nb_pad, n_parts, 1.0f / (float)(g.L * g.H),
+                                                   scores, scores_stride);
     return cudaGetLastError();
 }
 

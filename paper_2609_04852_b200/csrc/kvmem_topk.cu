@@ -12,31 +12,37 @@
 namespace kvmem {
 
 constexpr int kTopkThreads = 1024;
+constexpr int kItems = 16;                                  // consecutive block ids per thread and tile
+constexpr int kTopkTile = kTopkThreads * kItems;            // 16,384 ids per sweep
 
 struct TopkShared {
     unsigned int hist[256];
-    unsigned int warp_a[32], warp_b[32];
-    unsigned int prefix, remaining, carry_eq, carry_sel;
+    unsigned int warp_tot[32];
+    unsigned int prefix, remaining;
 };
 
-// exclusive scan of two flags across the CTA; returns (rank_a, rank_b) and adds the totals to the carries
-__device__ __forceinline__ void block_scan2(bool fa, bool fb, TopkShared& sh, unsigned& ra, unsigned& rb,
-                                            unsigned& tot_a, unsigned& tot_b) {
+// exclusive prefix of `val` over the CTA (thread order) and the CTA total; two barriers
+__device__ __forceinline__ unsigned block_exclusive_scan(unsigned val, TopkShared& sh, unsigned& total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const unsigned ba = __ballot_sync(0xffffffffu, fa), bb = __ballot_sync(0xffffffffu, fb);
-    const unsigned lt = (1u << lane) - 1u;
-    if (lane == 0) { sh.warp_a[warp] = __popc(ba); sh.warp_b[warp] = __popc(bb); }
-    __syncthreads();
-    unsigned oa = 0, ob = 0, ta = 0, tb = 0;
-    for (int w = 0; w < kTopkThreads / 32; ++w) {
-        const unsigned ca = sh.warp_a[w], cb = sh.warp_b[w];
-        if (w < warp) { oa += ca; ob += cb; }
-        ta += ca; tb += cb;
+    unsigned inc = val;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
     }
-    ra = oa + __popc(ba & lt);
-    rb = ob + __popc(bb & lt);
-    tot_a = ta; tot_b = tb;
+    if (lane == 31) sh.warp_tot[warp] = inc;
     __syncthreads();
+    const unsigned wt = sh.warp_tot[lane];                  // kTopkThreads / 32 == 32 warps
+    unsigned winc = wt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += t;
+    }
+    const unsigned warp_off = __shfl_sync(0xffffffffu, winc - wt, warp);
+    total = __shfl_sync(0xffffffffu, winc, 31);
+    __syncthreads();
+    return warp_off + inc - val;
 }
 
 __global__ void __launch_bounds__(kTopkThreads)
@@ -44,7 +50,7 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
             int session_first, int B, kvmem_select_params_t prm, int32_t* __restrict__ sel_ids, int sel_stride,
             int32_t* __restrict__ n_sel, int32_t* __restrict__ status) {
     __shared__ TopkShared sh;
-    const int s = blockIdx.x, tid = threadIdx.x;
+    const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     const int NB = nblocks_dev[session_first + s];
     const unsigned int* bits = reinterpret_cast<const unsigned int*>(scores + (size_t)s * scores_stride);
     int32_t* out = sel_ids + (size_t)s * sel_stride;
@@ -82,9 +88,19 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
             __syncthreads();
             const unsigned int prefix = sh.prefix;
             const unsigned int mask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
-            for (int b = n_sink + tid; b < recent_lo; b += kTopkThreads) {
-                const unsigned int v = bits[b];
-                if ((v & mask) == prefix) atomicAdd(&sh.hist[(v >> shift) & 255u], 1u);
+            for (int base = 0; base < NB; base += kTopkTile) {
+                const int b0 = base + tid * kItems;
+#pragma unroll 4
+                for (int i = 0; i < kItems; ++i) {
+                    const int b = b0 + i;
+                    unsigned int v = 0;
+                    bool live = b >= n_sink && b < recent_lo;
+                    if (live) { v = bits[b]; live = (v & mask) == prefix; }
+                    // one shared-memory atomic per distinct digit in the warp
+                    const unsigned int digit = live ? ((v >> shift) & 255u) : 256u;
+                    const unsigned int peers = __match_any_sync(0xffffffffu, digit);
+                    if (live && lane == __ffs(peers) - 1) atomicAdd(&sh.hist[digit], (unsigned)__popc(peers));
+                }
             }
             __syncthreads();
             if (tid == 0) {
@@ -103,34 +119,38 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
         T = sh.prefix;
         need_eq = sh.remaining;
     }
-    if (tid == 0) { sh.carry_eq = 0u; sh.carry_sel = 0u; }
-    __syncthreads();
 
-    for (int base = 0; base < NB; base += kTopkThreads) {
-        const int b = base + tid;
-        bool reserved = false, eq = false, gt = false;
-        if (b < NB) {
-            reserved = (b < n_sink) || (b >= recent_lo);
-            if (!reserved && kc > 0) {
-                const unsigned int v = bits[b];
-                gt = v > T;
-                eq = v == T;
+    // ascending sweep: each thread owns kItems consecutive ids, so thread order is id order
+    unsigned carry_eq = 0, carry_sel = 0;
+    for (int base = 0; base < NB; base += kTopkTile) {
+        const int b0 = base + tid * kItems;
+        unsigned flags_res = 0, flags_gt = 0, flags_eq = 0;
+#pragma unroll
+        for (int i = 0; i < kItems; ++i) {
+            const int b = b0 + i;
+            if (b < NB) {
+                if (b < n_sink || b >= recent_lo) flags_res |= 1u << i;
+                else if (kc > 0) {
+                    const unsigned int v = bits[b];
+                    if (v > T) flags_gt |= 1u << i;
+                    else if (v == T) flags_eq |= 1u << i;
+                }
             }
         }
-        const unsigned carry_eq = sh.carry_eq, carry_sel = sh.carry_sel;
-        unsigned r_eq, r_dummy, t_eq, t_dummy;
-        block_scan2(eq, false, sh, r_eq, r_dummy, t_eq, t_dummy);
-        const bool take = reserved || gt || (eq && (carry_eq + r_eq) < need_eq);
-        unsigned r_sel, t_sel;
-        block_scan2(take, false, sh, r_sel, r_dummy, t_sel, t_dummy);
-        if (take) {
-            const unsigned pos = carry_sel + r_sel;
-            if (pos < (unsigned)sel_stride) out[pos] = b;
-        }
-        if (tid == 0) { sh.carry_eq = carry_eq + t_eq; sh.carry_sel = carry_sel + t_sel; }
-        __syncthreads();
+        unsigned tot_eq, tot_sel;
+        unsigned eq_rank = carry_eq + block_exclusive_scan(__popc(flags_eq), sh, tot_eq);
+        unsigned take = flags_res | flags_gt;
+#pragma unroll
+        for (int i = 0; i < kItems; ++i)
+            if (flags_eq & (1u << i)) { if (eq_rank < need_eq) take |= 1u << i; ++eq_rank; }
+        unsigned pos = carry_sel + block_exclusive_scan(__popc(take), sh, tot_sel);
+#pragma unroll
+        for (int i = 0; i < kItems; ++i)
+            if (take & (1u << i)) { if (pos < (unsigned)sel_stride) out[pos] = b0 + i; ++pos; }
+        carry_eq += tot_eq;
+        carry_sel += tot_sel;
     }
-    if (tid == 0) n_sel[s] = (int32_t)min(sh.carry_sel, (unsigned)sel_stride);
+    if (tid == 0) n_sel[s] = (int32_t)min(carry_sel, (unsigned)sel_stride);
 }
 
 cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, const float* scores,

@@ -29,14 +29,14 @@ class OracleSession:
 
 
 def fill_oracle(spec: WorkloadSpec, n_blocks: Optional[List[int]] = None, gen_device="cpu") -> List[OracleSession]:
-    """Oracle-side repositories (one per session, each with the whole page pool's id space)."""
+    """Oracle-side state: one repository of physical pages shared by the sessions, one index each."""
     tables = page_table(spec).numpy()
-    n_pages = spec.n_sessions * spec.n_blocks
+    lens = [spec.n_blocks if n_blocks is None else n_blocks[s] for s in range(spec.n_sessions)]
+    n_pages = max(int(tables[s, :lens[s]].max(initial=0)) + 1 for s in range(spec.n_sessions))
+    repo = orc.Repository.empty(n_pages, spec.block_tokens, spec.n_layers, spec.n_kv_heads, spec.head_dim)
     out = []
     for s in range(spec.n_sessions):
-        nb = spec.n_blocks if n_blocks is None else n_blocks[s]
-        repo = orc.Repository.empty(n_pages if spec.permute_pages else max(int(tables[s, :nb].max()) + 1, 1),
-                                    spec.block_tokens, spec.n_layers, spec.n_kv_heads, spec.head_dim)
+        nb = lens[s]
         idx = np.zeros((spec.n_layers, spec.n_kv_heads, max(nb, 1), spec.head_dim), np.uint16)
         step = 512
         for b0 in range(0, nb, step):

@@ -1,0 +1,86 @@
+"""Parity at the full benchmark sizes (128K, 1M, 8 x 256K), in the launch configuration the
+benchmark times.  The oracle gets the same bytes: the generator is bit-identical on CPU and GPU
+(checked below), so the history is generated on the device and copied to the host for the oracle.
+"""
+import numpy as np
+import pytest
+import torch
+
+from kvmem_harness import ATTN_ATOL, bits, check_scores, check_selection, fill_oracle, fill_pool, queries
+from kvmem_workloads import CONFIGS, kv_blocks, planted_blocks, select_params
+from oracle import kvmem_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+
+def test_generator_is_bit_identical_on_cpu_and_gpu():
+    spec = CONFIGS["128k"]
+    Kc, Vc = kv_blocks(spec, 0, 100, 108, "cpu")
+    Kg, Vg = kv_blocks(spec, 0, 100, 108, torch.device("cuda", 0))
+    assert torch.equal(Kc, Kg.cpu()) and torch.equal(Vc, Vg.cpu())
+    spec = CONFIGS["1m"]
+    ids = planted_blocks(spec, 0)[0][:2].tolist()
+    for b in ids:
+        Kc, _ = kv_blocks(spec, 0, b, b + 1, "cpu")
+        Kg, _ = kv_blocks(spec, 0, b, b + 1, torch.device("cuda", 0))
+        assert torch.equal(Kc, Kg.cpu())
+
+
+def _full_step(spec, qsets=(0,), gap_forced_budget=None):
+    from paper_2609_04852_b200 import SelectParams, budget_blocks
+    dev = torch.device("cuda", 0)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec, gen_device=dev)
+    prm_d = select_params(spec)
+    if gap_forced_budget is not None:
+        prm_d["budget_blocks"] = gap_forced_budget
+    prm = SelectParams(**prm_d)
+    ns, B, M = spec.n_sessions, spec.block_tokens, spec.n_q_tokens
+    k = budget_blocks(prm, B, spec.n_blocks)
+    sel = torch.zeros(ns, k, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(ns, dtype=torch.int32, device=dev)
+    scores = torch.zeros(ns, spec.n_blocks, dtype=torch.float32, device=dev)
+    view = pool.new_view(ns, k * B)
+    out, lse = pool.new_outputs(ns, M)
+    for s in range(ns):
+        assert np.array_equal(bits(pool.index(s)), osess[s].idx), "Mean-K index differs"
+    modes = []
+    for qset in qsets:
+        q, qb = queries(spec, qset)
+        qd = q.to(dev)
+        pool.select(qd, prm, sel, n_sel, scores)
+        pool.materialize(sel, n_sel, view)
+        pool.view_attend(qd, view, n_sel, out, lse)
+        torch.cuda.synchronize()
+        assert pool.device_status() == 0
+        sel_h, n_h, sc_h = sel.cpu().numpy(), n_sel.cpu().numpy(), scores.cpu().numpy()
+        out_h, lse_h = out.cpu().numpy(), lse.cpu().numpy()
+        for s in range(ns):
+            R, _ = orc.block_scores(qb[s], osess[s].idx, spec.n_blocks)
+            ref_sel = orc.select(R, B, prm_d["budget_blocks"], prm_d["max_view_tokens"])
+            check_scores(sc_h[s], R, M)
+            sel_gpu = sel_h[s, : n_h[s]]
+            assert n_h[s] == k == len(ref_sel) and k * B <= spec.max_view_tokens
+            modes.append(check_selection(sel_gpu, R, ref_sel))
+            vK, vV = orc.gather(osess[s].repo, osess[s].table, np.ascontiguousarray(sel_gpu), k * B)
+            assert np.array_equal(bits(view.k[s]), vK) and np.array_equal(bits(view.v[s]), vV), "gathered view differs"
+            ref_out, ref_lse = orc.attend(qb[s], vK, vV, k * B)
+            err_o, err_l = np.abs(out_h[s] - ref_out).max(), np.abs(lse_h[s] - ref_lse).max()
+            assert err_o <= ATTN_ATOL and err_l <= ATTN_ATOL, f"attention error {err_o:.2e}, lse {err_l:.2e}"
+            assert err_o <= 5e-2 * np.abs(ref_out).max(), "attention error is large relative to the output scale"
+    return modes
+
+
+def test_config_128k_full():
+    spec = CONFIGS["128k"]
+    _full_step(spec, qsets=(0, 1))
+    modes = _full_step(spec, gap_forced_budget=spec.n_planted)       # k = planted count: the boundary gap is wide
+    assert modes == ["exact"]
+
+
+def test_config_1m_full():
+    _full_step(CONFIGS["1m"])
+
+
+def test_config_batch8_full():
+    _full_step(CONFIGS["batch8"])
