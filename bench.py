@@ -130,6 +130,7 @@ def fill_pool(spec, device, seed_shift=0):
 def run_native(args):
     import torch.distributed as dist
     from paper_2609_04852_b200 import SelectParams
+    from paper_2609_04852_b200.sharding import max_over_ranks, whole_job_rate
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -243,10 +244,7 @@ def run_native(args):
     else:
         clock_note = "sampled during the timed region"
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(times[0]), float(times[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], device=device)     # slowest rank decides
 
     if rank == 0:
         clocks = sampler.stop()
@@ -259,7 +257,7 @@ def run_native(args):
         step_gbs = world * K * ns * ab["total"] / (total_ms * 1e-3) / 1e9 / world      # per GPU
         rows = ns * M * spec.n_layers * spec.n_q_heads
         line = {
-            "metric": METRIC, "value": world * K / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "metric": METRIC, "value": whole_job_rate(K, world, total_ms), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded; shapes of the paper's agent workspaces)",
             "config": {"workload": f"{spec.name}: {ns} session(s) x {spec.n_blocks} blocks of {B} tokens "
@@ -269,7 +267,7 @@ def run_native(args):
                        "l2": "flushed between steps (256 MiB write)" if flush is not None else
                              "no flush: every step streams far more than the 126 MB L2",
                        "parallelism": f"{world} independent session replica(s), one per GPU"},
-            "e2e": {"value": world * Ke / (e2e_ms * 1e-3), "unit": UNIT, "steps": Ke,
+            "e2e": {"value": whole_job_rate(Ke, world, e2e_ms), "unit": UNIT, "steps": Ke,
                     "h2d_bytes_per_step": rows * spec.head_dim * 2,
                     "d2h_bytes_per_step": rows * spec.head_dim * 4 + rows * 4,
                     "api": "kvmem_recall_step_host (pinned host query in, host O and LSE out, synchronous)"},

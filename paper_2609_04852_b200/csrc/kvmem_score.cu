@@ -219,14 +219,18 @@ score_logits_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 }
 
 // Merge the per-CTA statistics of every row, then R_b = (1/(L*H)) sum_rows exp2(logit - max_row) / Z_row.
+// A CTA owns 32 consecutive blocks; thread (lgs, bl) sums the rows of heads lgs, lgs + 8, ... for block
+// bl (16 independent coalesced loads in flight), and the 8 partial sums are added in a fixed order.
+constexpr int kFinishBlocks = 32;
 __global__ void __launch_bounds__(256)
 score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__ partials,
                     const int32_t* __restrict__ nblocks_dev, int session_first, int LG, int rows, int rows_pad,
                     int nb_pad, int n_parts, float inv_LH, float* __restrict__ scores, int scores_stride) {
     extern __shared__ float2 rowstat[];   // [LG * rows] : (max, 1/Z)
+    __shared__ float red[8][kFinishBlocks];
     const int s = blockIdx.y;
     const int NB = nblocks_dev[session_first + s];
-    if ((int)(blockIdx.x * blockDim.x) >= NB) return;
+    if ((int)(blockIdx.x * kFinishBlocks) >= NB) return;
     for (int i = threadIdx.x; i < LG * rows; i += blockDim.x) {
         const int lg = i / rows, j = i % rows;
         const float2* p = partials + (((size_t)s * LG + lg) * rows_pad + j) * n_parts;
@@ -240,20 +244,29 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
         rowstat[i] = make_float2(mx, 1.0f / z);
     }
     __syncthreads();
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= NB) return;
-    float total = 0.0f;
-    for (int lg = 0; lg < LG; ++lg) {
-        const float* base = logits + (((size_t)s * LG + lg) * rows_pad) * (size_t)nb_pad + b;
-        float part = 0.0f;
-#pragma unroll 8
-        for (int j = 0; j < rows; ++j) {
-            const float2 st = rowstat[lg * rows + j];
-            part += exp2f(base[(size_t)j * nb_pad] - st.x) * st.y;
+    const int bl = threadIdx.x & (kFinishBlocks - 1), lgs = threadIdx.x / kFinishBlocks;
+    const int b = blockIdx.x * kFinishBlocks + bl;
+    float part = 0.0f;
+    if (b < NB) {
+        for (int lg = lgs; lg < LG; lg += 8) {
+            const float* base = logits + (((size_t)s * LG + lg) * rows_pad) * (size_t)nb_pad + b;
+            float sub = 0.0f;
+#pragma unroll 16
+            for (int j = 0; j < rows; ++j) {
+                const float2 st = rowstat[lg * rows + j];
+                sub += exp2f(base[(size_t)j * nb_pad] - st.x) * st.y;
+            }
+            part += sub;
         }
-        total += part;
     }
-    scores[(size_t)s * scores_stride + b] = total * inv_LH;
+    red[lgs][bl] = part;
+    __syncthreads();
+    if (lgs == 0 && b < NB) {
+        float total = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) total += red[i][bl];
+        scores[(size_t)s * scores_stride + b] = total * inv_LH;
+    }
 }
 
 cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q,
@@ -294,7 +307,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
         e = cudaFuncSetAttribute(score_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsmem);
         if (e != cudaSuccess) return e;
     }
-    dim3 fgrid((unsigned)((max_nb + 255) / 256), (unsigned)n_sessions);
+    dim3 fgrid((unsigned)((max_nb + kFinishBlocks - 1) / kFinishBlocks), (unsigned)n_sessions);
     score_finish_kernel<<<fgrid, 256, fsmem, st>>>(ws.logits, ws.partials, p.nblocks_dev, session_first, LG, ws.rows,
                                                    ws.rows_pad, ws.nb_pad, n_parts, 1.0f / (float)(g.L * g.H),
                                                    scores, scores_stride);

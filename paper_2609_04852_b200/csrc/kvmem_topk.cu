@@ -103,16 +103,34 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
                 }
             }
             __syncthreads();
-            if (tid == 0) {
-                unsigned int rem = sh.remaining;
-                int bin = 255;
-                for (; bin > 0; --bin) {
-                    const unsigned int c = sh.hist[bin];
-                    if (c >= rem) break;
-                    rem -= c;
+            if (tid < 32) {
+                // warp 0 walks the 256 bins from the top: lane i owns bins [255 - 8i - 7, 255 - 8i]
+                const unsigned int rem = sh.remaining;
+                unsigned int c[8], mine = 0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { c[j] = sh.hist[255 - 8 * lane - j]; mine += c[j]; }
+                unsigned int inc = mine;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned int t = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc += t;
                 }
-                sh.prefix = prefix | ((unsigned)bin << shift);
-                sh.remaining = rem;                        // how many of value-prefix "bin" are still needed
+                const unsigned int before = inc - mine;            // candidates in bins above this lane's
+                const bool here = before < rem && rem <= inc;      // the k-th largest falls into my bins
+                // (if the counts were inconsistent nobody would claim it; the last lane then takes bin 0)
+                const unsigned int claim = __ballot_sync(0xffffffffu, here);
+                if (here || (claim == 0u && lane == 31)) {
+                    unsigned int left = rem - before;
+                    int bin = 255 - 8 * lane;
+#pragma unroll
+                    for (int j = 0; j < 7; ++j) {
+                        if (c[j] >= left) break;
+                        left -= c[j];
+                        --bin;
+                    }
+                    sh.prefix = prefix | ((unsigned)bin << shift);
+                    sh.remaining = left;                           // how many of this digit are still needed
+                }
             }
             __syncthreads();
         }
