@@ -165,6 +165,26 @@ int kvmem_view_attend(kvmem_pool_t* pool, int32_t n_sessions, const void* q /*DE
                       const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
                       void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
+/* kvmem_view_attend for callers that cannot allocate device memory.  (The paper has no counterpart.)
+ * Who needs it: a serving process that gave all of HBM to its KV pool at start-up and runs with
+ * its allocator frozen, a plug-in that only ever sees the buffers of one request, or a latency path
+ * where a device-synchronising cudaMalloc is not acceptable.  Same arguments, definitions and
+ * results as kvmem_view_attend, except that the split-K workspace is a fixed array inside the
+ * library (about 4 MiB, held on every GPU that loads the library until the process exits).
+ *   - Limit: n_sessions * n_layers * n_kv_heads <= 8 per call; more returns KVMEM_E_CAPACITY with
+ *     a message, and nothing is enqueued.
+ *   - The call allocates nothing: no cudaMalloc, cudaFree or allocating library routine.
+ *   - The first call on a device looks up the array's device address (the pool's device must be
+ *     the current device); make that first call before starting any stream capture.
+ *   - All calls in the process share the array and it keeps the previous call's contents.  Nothing
+ *     in it needs clearing (every slot that is read is overwritten first), but two calls whose
+ *     kernels overlap on the GPU (different streams, or different pools on one device) race on it:
+ *     keep them on one stream or order them with events. */
+int kvmem_view_attend_static(kvmem_pool_t* pool, int32_t n_sessions, const void* q /*DEVICE*/, int32_t n_q_tokens,
+                             const void* view_k /*DEVICE*/, const void* view_v /*DEVICE*/, int32_t view_cap_tokens,
+                             const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
+                             void* stream);
+
 /* The whole recall step for callers whose query and results live in HOST memory: copies q to the
  * device, runs kvmem_select, kvmem_materialize and kvmem_view_attend, copies out and lse back and
  * waits for the stream (synchronous).  Same definitions and limits as the three calls above.
