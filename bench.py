@@ -47,6 +47,20 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "source": "fallback"}
 
 
+def measured_tensor_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"tflops": float(p["bf16_tflops"]), "source": "measured"}
+    return {"tflops": 1590.0, "source": "fallback"}
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one gather launch, from the ncu capture summarised in
+# profiles/dram_traffic_1m.md (1M workload)
+GATHER_TRAFFIC = {"1m": 2099369984}
+
+
 def algorithmic_bytes(spec, k):
     """Bytes the method must move per step (per session): index read + view read/write + view read."""
     view = 2 * k * spec.block_tokens * spec.n_layers * spec.n_kv_heads * spec.head_dim * 2       # K and V, bf16
@@ -143,8 +157,10 @@ def run_native(args):
         dist.init_process_group("nccl", device_id=device)
 
     base = CONFIGS[args.workload]
-    if not base.attend:
-        raise SystemExit(f"workload {base.name} has no attend stage; the benchmark times the whole step")
+    if args.blocks:      # a shrunken history of the same recipe: the small case for ncu captures
+        f = args.blocks / base.n_blocks
+        base = base.with_(name=f"{base.name}@{args.blocks}", n_blocks=args.blocks,
+                          n_planted=max(1, int(base.n_planted * f)), budget_blocks=max(1, int(base.budget_blocks * f)))
     pool, spec = fill_pool(base, device, seed_shift=1000 * rank)     # one independent replica per rank
     ns, M, B = spec.n_sessions, spec.n_q_tokens, spec.block_tokens
     prm = SelectParams(**select_params(spec))
@@ -224,8 +240,17 @@ def run_native(args):
     barrier()
     ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ee0.record(stream)
+    q_stage = torch.empty_like(q_dev[0])
+    sel_pin = torch.empty(sel.shape, dtype=torch.int32).pin_memory()
     for i in range(Ke):
-        pool.recall_step_host(q_pin[i % len(q_pin)], prm, sel, n_sel, view, out_pin, lse_pin)
+        if spec.attend:
+            pool.recall_step_host(q_pin[i % len(q_pin)], prm, sel, n_sel, view, out_pin, lse_pin)
+        else:       # chunked scoring has no attend stage: host query in, selected ids out
+            q_stage.copy_(q_pin[i % len(q_pin)], non_blocking=True)
+            pool.select(q_stage, prm, sel, n_sel)
+            pool.materialize(sel, n_sel, view)
+            sel_pin.copy_(sel, non_blocking=True)
+            torch.cuda.synchronize(device)
     ee1.record(stream)
     barrier()
     e2e_ms = ee0.elapsed_time(ee1)
@@ -277,13 +302,27 @@ def run_native(args):
                          "achieved": gather_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gather_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "algorithmic_bytes_per_launch": ns * ab["gather"], "avg_launch_ms": gather_s * 1e3,
-                         "traffic": None},
+                         "traffic": GATHER_TRAFFIC.get(base.name)},
             "step_hbm": {"algorithmic_bytes_per_step": ns * ab["total"], "achieved_gbs": step_gbs,
                          "frac_of_peak": step_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "nominal_peak_gbs": 8000.0},
             "stages_ms": {"select": med(sel_ms), "materialize": med(gat_ms), "attend": med(att_ms),
                           "step_median": med(step_ms), "step_min": min(step_ms)},
         }
+        if not spec.attend:
+            # the chunked configuration is bounded by the tensor pipe: two passes of the 2*M*H*NB*d contraction
+            flop_alg = 2.0 * ns * M * spec.n_layers * spec.n_q_heads * spec.n_blocks * spec.head_dim
+            sel_s = (sum(sel_ms) / K) * 1e-3
+            tpeak = measured_tensor_peak()
+            line["e2e"]["h2d_bytes_per_step"] = rows * spec.head_dim * 2
+            line["e2e"]["d2h_bytes_per_step"] = ns * k * 4
+            line["e2e"]["api"] = "pinned host query in, selected ids out, around kvmem_select + kvmem_materialize"
+            line["gpu_launches"] = K * 5
+            line["roofline"] = {"bound": "tensor", "kernel": "score_chunk_kernel<1> + <2> (inside kvmem_select; time includes the finish and top-k kernels)",
+                                "achieved": 2 * flop_alg / sel_s / 1e12, "peak": tpeak["tflops"], "unit": "TFLOP/s",
+                                "frac": 2 * flop_alg / sel_s / 1e12 / tpeak["tflops"], "peak_source": f"of {tpeak['source']} (burst)",
+                                "executed_flop_per_launch_pair": 2 * flop_alg, "algorithmic_flop": flop_alg,
+                                "algorithmic_tflops": flop_alg / sel_s / 1e12, "avg_select_ms": sel_s * 1e3, "traffic": None}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(base, args.cpu_sample_blocks)
         print(json.dumps(line), flush=True)
@@ -393,6 +432,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["native", "reference"], default="native")
     ap.add_argument("--workload", choices=sorted(CONFIGS), default="1m")
+    ap.add_argument("--blocks", type=int, default=0, help="shrink the history to this many blocks (profiling)")
     ap.add_argument("--flush-l2", action="store_true", help="write 256 MiB between steps (for workloads near L2 size)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)

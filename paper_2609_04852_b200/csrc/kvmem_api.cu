@@ -111,6 +111,7 @@ size_t kvmem_select_workspace_bytes(const kvmem_pool_config_t* cfg, int32_t n_se
         set_error("invalid arguments to kvmem_select_workspace_bytes");
         return 0;
     }
+    if (n_q_tokens > kMaxDecodeTokens) return plan_chunk_workspace(*cfg, n_sessions, n_q_tokens, nullptr).total;
     return plan_score_workspace(*cfg, n_sessions, n_q_tokens, nullptr).total;
 }
 
@@ -257,12 +258,28 @@ int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, con
     for (int s = session_first; s < session_first + n_sessions; ++s)
         max_k = std::max(max_k, kvmem_budget_blocks(prm, p->cfg.block_tokens, p->sess_blocks[s]));
     if (sel_stride < max_k) { set_error("sel_stride %d is below the clamped budget %d", sel_stride, max_k); return KVMEM_E_CAPACITY; }
-    ScoreWorkspace ws = plan_score_workspace(p->cfg, n_sessions, n_q_tokens, (char*)workspace);
-    if (workspace_bytes < ws.total) { set_error("select workspace holds %zu bytes, %zu needed", workspace_bytes, ws.total); return KVMEM_E_CAPACITY; }
     cudaStream_t st = (cudaStream_t)stream;
-    float* sc = scores ? scores : ws.scores;
-    cudaError_t e = launch_score_decode(*p, session_first, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, ws, sc,
-                                        p->cfg.max_blocks_per_session, st);
+    float* sc = nullptr;
+    cudaError_t e;
+    if (n_q_tokens > kMaxDecodeTokens) {
+        // a multi-token chunk makes scoring a dense contraction: tensor-core path
+        if (!chunked_scoring_supported(p->cfg, n_q_tokens)) {
+            set_error("chunked scoring needs head_dim 128, H/G dividing 128 and n_q_tokens * H/G <= 4096 "
+                      "(scores are additive over query tokens: split a longer chunk and add)");
+            return KVMEM_E_UNSUPPORTED;
+        }
+        ChunkWorkspace cw = plan_chunk_workspace(p->cfg, n_sessions, n_q_tokens, (char*)workspace);
+        if (workspace_bytes < cw.total) { set_error("select workspace holds %zu bytes, %zu needed", workspace_bytes, cw.total); return KVMEM_E_CAPACITY; }
+        sc = scores ? scores : cw.scores;
+        e = launch_score_chunked(*p, session_first, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, cw, sc,
+                                 p->cfg.max_blocks_per_session, st);
+    } else {
+        ScoreWorkspace ws = plan_score_workspace(p->cfg, n_sessions, n_q_tokens, (char*)workspace);
+        if (workspace_bytes < ws.total) { set_error("select workspace holds %zu bytes, %zu needed", workspace_bytes, ws.total); return KVMEM_E_CAPACITY; }
+        sc = scores ? scores : ws.scores;
+        e = launch_score_decode(*p, session_first, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, ws, sc,
+                                p->cfg.max_blocks_per_session, st);
+    }
     if (e != cudaSuccess) return cuda_fail("score kernel launch", e);
     e = launch_topk(*p, session_first, n_sessions, sc, p->cfg.max_blocks_per_session, *prm, sel_ids, sel_stride, n_sel, st);
     if (e != cudaSuccess) return cuda_fail("top-k kernel launch", e);

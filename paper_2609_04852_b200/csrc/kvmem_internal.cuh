@@ -85,6 +85,20 @@ ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions
 cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q,
                                 int M, const ScoreWorkspace& ws, float* scores, int scores_stride, cudaStream_t st);
 
+// multi-token query chunks: tcgen05 two-pass contraction
+struct ChunkWorkspace {
+    float2* rowstat;   // [ns][L][G][rows_pad] (max, log2 Z)
+    float* colsum;     // [ns][L][G][nb_pad]: per-head sums of the softmax weights over the head's query rows
+    float* scores;     // [ns][max_bps]
+    size_t rowstat_bytes, colsum_bytes, scores_bytes, total;
+    int rows, rows_pad, n_panels, nb_pad;
+};
+ChunkWorkspace plan_chunk_workspace(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, char* base);
+bool chunked_scoring_supported(const kvmem_pool_config_t& c, int n_q_tokens);
+constexpr int kMaxDecodeTokens = 16;   // more query tokens than this take the tensor-core path
+cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q, int M,
+                                 const ChunkWorkspace& ws, float* scores, int scores_stride, cudaStream_t st);
+
 cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, const float* scores,
                         int scores_stride, const kvmem_select_params_t& prm, int32_t* sel_ids, int sel_stride,
                         int32_t* n_sel, cudaStream_t st);

@@ -22,7 +22,6 @@ namespace kvmem {
 
 constexpr int kChunk = 128;       // blocks per CTA tile
 constexpr int kScoreThreads = 256;
-constexpr int kMaxDecodeTokens = 16;
 constexpr int kScoreStages = 4;   // 32 KiB index tiles in flight per CTA
 constexpr int kMaxScoreParts = 64;
 
@@ -34,7 +33,7 @@ ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions
     w.nb_pad = (c.max_blocks_per_session + kChunk - 1) / kChunk * kChunk;
     w.n_chunks = w.nb_pad / kChunk;
     const size_t lg = (size_t)c.n_layers * c.n_kv_heads;
-    const int rows_store = n_q_tokens <= kMaxDecodeTokens ? w.rows_pad : 16;
+    const int rows_store = w.rows_pad;
     w.logits_bytes = align_up((size_t)n_sessions * lg * rows_store * w.nb_pad * sizeof(float), 256);
     w.partials_bytes = align_up((size_t)n_sessions * lg * rows_store * kMaxScoreParts * sizeof(float2), 256);
     w.scores_bytes = align_up((size_t)n_sessions * c.max_blocks_per_session * sizeof(float), 256);

@@ -1,0 +1,581 @@
+// Block scoring for a multi-token query chunk (Eq. "kvmem-block-score", Sec. 4.3) as a dense
+// contraction on the 5th-generation tensor cores.
+//
+// Per (session, layer, KV head): logits S = Q_g K̄_g^T with Q_g the M*(H/G) query rows of the head
+// group (2,048 x 128 for a 512-token chunk) and K̄_g the head's Mean-K index (NB x 128).  The
+// 2,048 x 16,384 logit matrix (1 GiB in fp32 over 8 heads) is never stored; the exact softmax needs
+// row statistics before column sums, so the contraction runs twice:
+//   pass 1 (S   = Q K̄^T): per query row, running max and sum-exp over all blocks -> rowstat (max, log2 Z)
+//   pass 2 (S^T = K̄ Q^T): p = exp2(s - max - log2 Z) summed over all query rows    -> headsum[l][g][b]
+// and a small kernel adds the heads in a fixed order: R_b = (1/(L*H)) sum_{l,g} headsum.
+// tcgen05.ld hands each epilogue thread one accumulator row (one TMEM lane).  Pass 1 puts query rows
+// on the lanes, so the row statistics are thread-local; pass 2 swaps the operands and puts blocks on
+// the lanes, so the sum over query rows is thread-local too: no shuffles, no atomics, and the
+// per-row shifts -(max + log2 Z) are broadcast reads from shared memory.
+//
+// Both passes: UMMA M = 128, N = 256, K = 128 (8 instructions of K = 16), bf16 in, fp32 accumulate.
+// Warp 0 is the TMA producer (stationary operand once per work item, streamed operand through a
+// shared-memory ring, 128-byte swizzle), one thread of warp 1 issues tcgen05.mma into two 256-column
+// TMEM accumulators, warps 2-5 are the epilogue.  The epilogue of tile t overlaps the MMAs of tile
+// t + 1.  Pass 1: one CTA per 128-row query panel, sweeping all blocks.  Pass 2: persistent CTAs, one
+// work item = 128 blocks of one head, sweeping that head's query rows.  All mbarrier waits are bounded.
+#include <cudaTypedefs.h>
+#include <math.h>
+
+#include <algorithm>
+
+#include "kvmem_internal.cuh"
+#include "kvmem_ptx.cuh"
+
+namespace kvmem {
+
+constexpr int kCkBM = 128;                    // rows per panel
+constexpr int kCkBN = 256;                    // blocks per tile
+constexpr int kCkStages = 2;                  // index tiles in flight
+constexpr int kCkThreads = 192;               // TMA warp, MMA warp, 4 epilogue warps
+constexpr int kCkAHalf = kCkBM * 128;         // bytes of one 64-dim half of the Q panel  (16 KiB)
+constexpr int kCkBHalf = kCkBN * 128;         // bytes of one 64-dim half of an index tile (32 KiB)
+constexpr int kCkTmemCols = 512;              // two fp32 accumulators of 256 columns
+constexpr size_t kCkSmem = 2 * kCkAHalf + (size_t)kCkStages * 2 * kCkBHalf + 1024;
+
+namespace t5 {   // tcgen05 wrappers
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(dst_smem)), "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, one CTA
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// mbarrier arrives once all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(ptx::smem_u32(bar)) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// issue the load of 32 columns without waiting for it
+__device__ __forceinline__ void ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1,024 bytes apart.  `addr` may point 32*k bytes into the swizzle span (K advance).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)0 << 16;                            // leading byte offset: unused for swizzled K-major
+    d |= (uint64_t)(1024u >> 4) << 32;                 // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                            // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                            // layout type: 128-byte swizzle
+    return d;
+}
+
+}  // namespace t5
+
+__device__ __forceinline__ void tma_load_4d(void* dst_smem, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::
+            "r"(ptx::smem_u32(dst_smem)),
+        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(ptx::smem_u32(bar))
+        : "memory");
+}
+
+struct ChunkArgs {
+    const int32_t* nblocks_dev;
+    float2* rowstat;      // [ns][LG][rows_pad]   (max, log2 Z) of every query row, log2 domain
+    float* headsum;       // [ns][LG][nb_pad]     sum over the head's query rows of the softmax weights
+    int32_t* status;
+    int session_first, n_sessions, M, L, G, r, rows, rows_pad, nb_pad, n_bpanels;
+    float scale_log2e;
+};
+
+// fp32 accumulate, bf16 x bf16, both operands K-major, N = 256, M = 128
+__device__ __forceinline__ uint32_t chunk_idesc() {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kCkBN >> 3) << 17) | ((uint32_t)(kCkBM >> 4) << 24);
+}
+
+// one 128 x 256 x 128 tile: 8 MMAs of K = 16 (32 bytes inside the 128-byte swizzle span)
+__device__ __forceinline__ void issue_tile_mma(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
+    const uint32_t idesc = chunk_idesc();
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const uint32_t koff = (uint32_t)(k & 3) * 32u;
+        const uint64_t da = t5::smem_desc_sw128(a_addr + (uint32_t)(k >> 2) * kCkAHalf + koff);
+        const uint64_t db = t5::smem_desc_sw128(b_addr + (uint32_t)(k >> 2) * kCkBHalf + koff);
+        t5::mma_bf16(d_tmem, da, db, idesc, k > 0 ? 1u : 0u);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Pass 1.  Grid (query panel, layer x KV head, session).  TMEM lane = query row.
+__global__ void __launch_bounds__(kCkThreads, 1)
+score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_idx,
+                           ChunkArgs a) {
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ uint64_t a_full, b_full[kCkStages], b_empty[kCkStages], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+
+    unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    unsigned char* smem_a = base;                              // Q panel: 2 halves x 16 KiB
+    unsigned char* smem_b = base + 2 * kCkAHalf;               // index tiles: stages x 2 halves x 32 KiB
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int panel = blockIdx.x, lg = blockIdx.y, s = blockIdx.z;
+    const int l = lg / a.G, g = lg % a.G;
+    const int LG = a.L * a.G;
+    const int NB = a.nblocks_dev[a.session_first + s];
+    const int n_tiles = (NB + kCkBN - 1) / kCkBN;
+
+    if (tid == 0) {
+        ptx::mbar_init(&a_full, 1);
+        for (int i = 0; i < kCkStages; ++i) { ptx::mbar_init(&b_full[i], 1); ptx::mbar_init(&b_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 4); }
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {                     // one warp allocates the tensor memory for the whole CTA
+        t5::tmem_alloc(&tmem_base_slot, kCkTmemCols);
+        t5::tmem_relinquish();
+    }
+    t5::fence_before();
+    __syncthreads();
+    t5::fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0 && n_tiles > 0) {
+            ptx::prefetch_tensormap(&map_q);
+            ptx::prefetch_tensormap(&map_idx);
+            // Q panel: rows j = m * r + hr of this KV head; 128 rows = 128 / r tokens x r heads
+            const int m0 = s * a.M + panel * (kCkBM / a.r);
+            ptx::mbar_expect_tx(&a_full, 2 * kCkAHalf);
+            tma_load_4d(smem_a, &map_q, 0, g * a.r, l, m0, &a_full);
+            tma_load_4d(smem_a + kCkAHalf, &map_q, 64, g * a.r, l, m0, &a_full);
+            const int z = ((a.session_first + s) * a.L + l) * a.G + g;
+            for (int t = 0; t < n_tiles; ++t) {
+                const int st = t % kCkStages;
+                if (t >= kCkStages && !ptx::mbar_wait(&b_empty[st], (uint32_t)(((t / kCkStages) & 1) ^ 1))) {
+                    atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+                    break;
+                }
+                unsigned char* dst = smem_b + (size_t)st * 2 * kCkBHalf;
+                ptx::mbar_expect_tx(&b_full[st], 2 * kCkBHalf);
+                ptx::tma_load_3d(dst, &map_idx, 0, t * kCkBN, z, &b_full[st]);
+                ptx::tma_load_3d(dst + kCkBHalf, &map_idx, 64, t * kCkBN, z, &b_full[st]);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0 && n_tiles > 0) {
+            bool ok = ptx::mbar_wait(&a_full, 0);
+            const uint32_t a_addr = ptx::smem_u32(smem_a);
+            for (int t = 0; ok && t < n_tiles; ++t) {
+                const int st = t % kCkStages, acc = t & 1;
+                ok = ptx::mbar_wait(&b_full[st], (uint32_t)((t / kCkStages) & 1));
+                if (ok && t >= 2) ok = ptx::mbar_wait(&acc_empty[acc], (uint32_t)(((t >> 1) & 1) ^ 1));
+                if (!ok) break;
+                t5::fence_after();
+                issue_tile_mma(tmem_base + (uint32_t)acc * kCkBN, a_addr, ptx::smem_u32(smem_b + (size_t)st * 2 * kCkBHalf));
+                t5::commit(&b_empty[st]);                  // the index tile may be overwritten
+                t5::commit(&acc_full[acc]);                // the accumulator may be read
+            }
+            if (!ok) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+        }
+    } else {
+        // ------------------------------------------------ epilogue (4 warps, one TMEM lane quarter each)
+        const int quarter = warp & 3;                      // warps 2,3,4,5 -> quarters 2,3,0,1
+        const int row = panel * kCkBM + quarter * 32 + lane;   // row of this (session, l, g): m * r + hr
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        float run_m = -INFINITY, run_z = 0.0f;
+        for (int t = 0; t < n_tiles; ++t) {
+            const int acc = t & 1;
+            const bool arrived = ptx::mbar_wait(&acc_full[acc], (uint32_t)((t >> 1) & 1));
+            if (!__all_sync(0xffffffffu, arrived)) {
+                if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+                break;
+            }
+            t5::fence_after();
+            const int col0 = t * kCkBN;
+            const bool ragged = col0 + kCkBN > NB;
+            uint32_t buf[2][32];
+            t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN), buf[0]);
+#pragma unroll 2
+            for (int c = 0; c < kCkBN / 32; ++c) {
+                t5::ld_wait();
+                if (c + 1 < kCkBN / 32) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + (c + 1) * 32), buf[(c + 1) & 1]);
+                float v[32];
+                float mx = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float x = __uint_as_float(buf[c & 1][i]) * a.scale_log2e;
+                    v[i] = (ragged && col0 + c * 32 + i >= NB) ? -INFINITY : x;
+                    mx = fmaxf(mx, v[i]);
+                }
+                const float mn = fmaxf(run_m, mx);
+                if (mn > -INFINITY) {
+                    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        s0 += t5::ex2(v[i] - mn); s1 += t5::ex2(v[i + 1] - mn);
+                        s2 += t5::ex2(v[i + 2] - mn); s3 += t5::ex2(v[i + 3] - mn);
+                    }
+                    run_z = run_z * t5::ex2(run_m - mn) + ((s0 + s1) + (s2 + s3));
+                    run_m = mn;
+                }
+            }
+            t5::fence_before();                            // the accumulator has been drained into registers
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
+        }
+        if (row < a.rows) a.rowstat[((size_t)s * LG + lg) * a.rows_pad + row] = make_float2(run_m, log2f(run_z));
+    }
+
+    t5::fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        t5::fence_after();
+        t5::tmem_dealloc(tmem_base, kCkTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Pass 2.  Persistent CTAs; work item = (session, layer x KV head, 128-block panel).  TMEM lane = block.
+// Stationary operand: the panel's Mean-K vectors; streamed operand: the head's query rows, 256 at a time.
+constexpr int kCkShiftMax = 4096;                // query rows per (session, l, g) the shift vector can hold
+constexpr size_t kCkSmem2 = 2 * 2 * kCkAHalf + (size_t)kCkStages * 2 * kCkBHalf + kCkShiftMax * sizeof(float) + 1024;
+
+__global__ void __launch_bounds__(kCkThreads, 1)
+score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_idx,
+                          ChunkArgs a) {
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ uint64_t a_full[2], a_empty[2], b_full[kCkStages], b_empty[kCkStages], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+
+    unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    unsigned char* smem_a = base;                                  // index panels: 2 stages x 2 halves x 16 KiB
+    unsigned char* smem_b = base + 2 * 2 * kCkAHalf;               // query tiles:  stages x 2 halves x 32 KiB
+    float* shift = reinterpret_cast<float*>(smem_b + (size_t)kCkStages * 2 * kCkBHalf);   // [n_qtiles * 256]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int LG = a.L * a.G;
+    const int n_items = a.n_sessions * LG * a.n_bpanels;           // panel index fastest: neighbours share a head's Q
+    const int n_qtiles = (a.rows + kCkBN - 1) / kCkBN;
+    const int tokens_per_qtile = kCkBN / a.r;
+
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(&a_full[i], 1); ptx::mbar_init(&a_empty[i], 1);
+            ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 4);
+        }
+        for (int i = 0; i < kCkStages; ++i) { ptx::mbar_init(&b_full[i], 1); ptx::mbar_init(&b_empty[i], 1); }
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {
+        t5::tmem_alloc(&tmem_base_slot, kCkTmemCols);
+        t5::tmem_relinquish();
+    }
+    t5::fence_before();
+    __syncthreads();
+    t5::fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    // every role walks the same item sequence and skips the same (empty) items
+    auto item_live = [&](int item, int& s, int& lg, int& bp) {
+        bp = item % a.n_bpanels;
+        lg = (item / a.n_bpanels) % LG;
+        s = item / (a.n_bpanels * LG);
+        return bp * kCkBM < a.nblocks_dev[a.session_first + s];
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            ptx::prefetch_tensormap(&map_q);
+            ptx::prefetch_tensormap(&map_idx);
+            int li = 0, tt = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+                int s, lg, bp;
+                if (!item_live(item, s, lg, bp)) continue;
+                const int l = lg / a.G, g = lg % a.G;
+                const int as = li & 1;
+                if (li >= 2) ok = ptx::mbar_wait(&a_empty[as], (uint32_t)(((li >> 1) & 1) ^ 1));
+                if (!ok) break;
+                unsigned char* adst = smem_a + (size_t)as * 2 * kCkAHalf;
+                const int z = ((a.session_first + s) * a.L + l) * a.G + g;
+                ptx::mbar_expect_tx(&a_full[as], 2 * kCkAHalf);
+                ptx::tma_load_3d(adst, &map_idx, 0, bp * kCkBM, z, &a_full[as]);
+                ptx::tma_load_3d(adst + kCkAHalf, &map_idx, 64, bp * kCkBM, z, &a_full[as]);
+                for (int qt = 0; qt < n_qtiles; ++qt, ++tt) {
+                    const int st = tt % kCkStages;
+                    if (tt >= kCkStages) ok = ptx::mbar_wait(&b_empty[st], (uint32_t)(((tt / kCkStages) & 1) ^ 1));
+                    if (!ok) break;
+                    unsigned char* dst = smem_b + (size_t)st * 2 * kCkBHalf;
+                    const int m0 = s * a.M + qt * tokens_per_qtile;
+                    ptx::mbar_expect_tx(&b_full[st], 2 * kCkBHalf);
+                    tma_load_4d(dst, &map_q, 0, g * a.r, l, m0, &b_full[st]);
+                    tma_load_4d(dst + kCkBHalf, &map_q, 64, g * a.r, l, m0, &b_full[st]);
+                }
+                ++li;
+            }
+            if (!ok) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int li = 0, tt = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+                int s, lg, bp;
+                if (!item_live(item, s, lg, bp)) continue;
+                const int as = li & 1;
+                ok = ptx::mbar_wait(&a_full[as], (uint32_t)((li >> 1) & 1));
+                const uint32_t a_addr = ptx::smem_u32(smem_a + (size_t)as * 2 * kCkAHalf);
+                for (int qt = 0; ok && qt < n_qtiles; ++qt, ++tt) {
+                    const int st = tt % kCkStages, acc = tt & 1;
+                    ok = ptx::mbar_wait(&b_full[st], (uint32_t)((tt / kCkStages) & 1));
+                    if (ok && tt >= 2) ok = ptx::mbar_wait(&acc_empty[acc], (uint32_t)(((tt >> 1) & 1) ^ 1));
+                    if (!ok) break;
+                    t5::fence_after();
+                    issue_tile_mma(tmem_base + (uint32_t)acc * kCkBN, a_addr, ptx::smem_u32(smem_b + (size_t)st * 2 * kCkBHalf));
+                    t5::commit(&b_empty[st]);
+                    t5::commit(&acc_full[acc]);
+                }
+                if (ok) t5::commit(&a_empty[as]);          // the index panel may be overwritten
+                ++li;
+            }
+            if (!ok) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+        }
+    } else {
+        // ------------------------------------------------ epilogue
+        const int quarter = warp & 3;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const int et = tid - 64;                           // 0..127 among the epilogue threads
+        int tt = 0, cur_head = -1;
+        bool failed = false;                               // a warp that gave up still meets every named barrier
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            int s, lg, bp;
+            if (!item_live(item, s, lg, bp)) continue;
+            if (s * LG + lg != cur_head) {
+                // shifts -(max + log2 Z) of this head's query rows; -inf switches a padding row off
+                cur_head = s * LG + lg;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const float2* rs = a.rowstat + (size_t)cur_head * a.rows_pad;
+                for (int j = et; j < n_qtiles * kCkBN; j += 128) {
+                    float sh = -INFINITY;
+                    if (j < a.rows) { const float2 st = rs[j]; sh = -(st.x + st.y); }
+                    shift[j] = sh;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+            float total = 0.0f;
+            for (int qt = 0; qt < n_qtiles; ++qt, ++tt) {
+                if (failed) continue;
+                const int acc = tt & 1;
+                const bool arrived = ptx::mbar_wait(&acc_full[acc], (uint32_t)((tt >> 1) & 1));
+                if (!__all_sync(0xffffffffu, arrived)) {
+                    if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+                    failed = true;
+                    continue;
+                }
+                t5::fence_after();
+                const float4* sh4 = reinterpret_cast<const float4*>(shift + qt * kCkBN);
+                uint32_t buf[2][32];
+                t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN), buf[0]);
+                float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+#pragma unroll 2
+                for (int c = 0; c < kCkBN / 32; ++c) {
+                    t5::ld_wait();
+                    if (c + 1 < kCkBN / 32) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + (c + 1) * 32), buf[(c + 1) & 1]);
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        const float4 sh = sh4[c * 8 + (i >> 2)];            // same address in every lane: broadcast
+                        s0 += t5::ex2(fmaf(__uint_as_float(buf[c & 1][i]), a.scale_log2e, sh.x));
+                        s1 += t5::ex2(fmaf(__uint_as_float(buf[c & 1][i + 1]), a.scale_log2e, sh.y));
+                        s2 += t5::ex2(fmaf(__uint_as_float(buf[c & 1][i + 2]), a.scale_log2e, sh.z));
+                        s3 += t5::ex2(fmaf(__uint_as_float(buf[c & 1][i + 3]), a.scale_log2e, sh.w));
+                    }
+                }
+                total += (s0 + s1) + (s2 + s3);
+                t5::fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
+            }
+            const int b = bp * kCkBM + quarter * 32 + lane;
+            if (!failed && b < a.nblocks_dev[a.session_first + s])
+                a.headsum[((size_t)s * LG + lg) * a.nb_pad + b] = total;
+        }
+    }
+
+    t5::fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        t5::fence_after();
+        t5::tmem_dealloc(tmem_base, kCkTmemCols);
+    }
+}
+
+// R_b = (1/(L*H)) * sum over (layer, KV head) of the head sums, in a fixed order.
+__global__ void __launch_bounds__(256)
+score_chunk_finish_kernel(const float* __restrict__ headsum, const int32_t* __restrict__ nblocks_dev, int session_first,
+                          int LG, int nb_pad, float inv_LH, float* __restrict__ scores, int scores_stride) {
+    const int s = blockIdx.y;
+    const int NB = nblocks_dev[session_first + s];
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= NB) return;
+    const float* p = headsum + (size_t)s * LG * nb_pad + b;
+    float total = 0.0f;
+    for (int i = 0; i < LG; ++i) total += p[(size_t)i * nb_pad];
+    scores[(size_t)s * scores_stride + b] = total * inv_LH;
+}
+
+static PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+    }
+    return fn;
+}
+
+ChunkWorkspace plan_chunk_workspace(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, char* base) {
+    ChunkWorkspace w{};
+    const int r = c.n_q_heads / c.n_kv_heads;
+    w.rows = n_q_tokens * r;
+    w.n_panels = (w.rows + kCkBM - 1) / kCkBM;
+    w.rows_pad = w.n_panels * kCkBM;
+    w.nb_pad = (c.max_blocks_per_session + kCkBN - 1) / kCkBN * kCkBN;
+    const size_t lg = (size_t)c.n_layers * c.n_kv_heads;
+    w.rowstat_bytes = align_up((size_t)n_sessions * lg * w.rows_pad * sizeof(float2), 256);
+    w.colsum_bytes = align_up((size_t)n_sessions * lg * w.nb_pad * sizeof(float), 256);
+    w.scores_bytes = align_up((size_t)n_sessions * c.max_blocks_per_session * sizeof(float), 256);
+    w.total = w.rowstat_bytes + w.colsum_bytes + w.scores_bytes;
+    if (base) {
+        w.rowstat = reinterpret_cast<float2*>(base);
+        w.colsum = reinterpret_cast<float*>(base + w.rowstat_bytes);
+        w.scores = reinterpret_cast<float*>(base + w.rowstat_bytes + w.colsum_bytes);
+    }
+    return w;
+}
+
+bool chunked_scoring_supported(const kvmem_pool_config_t& c, int n_q_tokens) {
+    const int r = c.n_q_heads / c.n_kv_heads;
+    return c.head_dim == 128 && r >= 1 && kCkBM % r == 0 && (long long)n_q_tokens * r <= kCkShiftMax;
+}
+
+// q [ns*M][L][H][128] as a 4-D tensor; box = 64 dims x r heads x 1 layer x (rows / r) tokens = `rows` rows of 128 B
+static bool make_q_map(PFN_cuTensorMapEncodeTiled_v12000 enc, CUtensorMap* map, const __nv_bfloat16* q, const Geometry& g,
+                       int n_tokens_total, int rows) {
+    cuuint64_t dims[4] = {128, (cuuint64_t)g.H, (cuuint64_t)g.L, (cuuint64_t)n_tokens_total};
+    cuuint64_t strides[3] = {256, (cuuint64_t)g.H * 256, (cuuint64_t)g.L * g.H * 256};
+    cuuint32_t box[4] = {64, (cuuint32_t)g.r, 1, (cuuint32_t)(rows / g.r)};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(q), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// index [max_sessions * L * G][max_bps][128]; box = 64 dims x `rows` blocks x 1
+static bool make_index_map(PFN_cuTensorMapEncodeTiled_v12000 enc, CUtensorMap* map, const kvmem_pool& p, int rows) {
+    const Geometry& g = p.geo;
+    cuuint64_t dims[3] = {128, (cuuint64_t)g.max_bps, (cuuint64_t)g.max_sessions * g.L * g.G};
+    cuuint64_t strides[2] = {256, (cuuint64_t)g.max_bps * 256};
+    cuuint32_t box[3] = {64, (cuuint32_t)rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, p.index, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q, int M,
+                                 const ChunkWorkspace& ws, float* scores, int scores_stride, cudaStream_t st) {
+    const Geometry& g = p.geo;
+    PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode_fn();
+    if (!enc) return cudaErrorNotSupported;
+    int max_nb = 0;
+    for (int s = session_first; s < session_first + n_sessions; ++s) max_nb = std::max(max_nb, p.sess_blocks[s]);
+    if (max_nb == 0) return cudaSuccess;
+
+    CUtensorMap q_panel, q_tile, idx_tile, idx_panel;      // 128- and 256-row boxes of each operand
+    if (!make_q_map(enc, &q_panel, q, g, n_sessions * M, kCkBM) || !make_q_map(enc, &q_tile, q, g, n_sessions * M, kCkBN) ||
+        !make_index_map(enc, &idx_tile, p, kCkBN) || !make_index_map(enc, &idx_panel, p, kCkBM))
+        return cudaErrorInvalidValue;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(score_chunk_rowstat_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCkSmem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(score_chunk_colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCkSmem2);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    ChunkArgs a{};
+    a.nblocks_dev = p.nblocks_dev; a.rowstat = ws.rowstat; a.headsum = ws.colsum; a.status = p.status_dev;
+    a.session_first = session_first; a.n_sessions = n_sessions; a.M = M; a.L = g.L; a.G = g.G; a.r = g.r;
+    a.rows = ws.rows; a.rows_pad = ws.rows_pad; a.nb_pad = ws.nb_pad;
+    a.n_bpanels = (max_nb + kCkBM - 1) / kCkBM;
+    a.scale_log2e = 1.4426950408889634f / sqrtf((float)g.d);
+    const int LG = g.L * g.G;
+    dim3 grid1((unsigned)ws.n_panels, (unsigned)LG, (unsigned)n_sessions);
+    score_chunk_rowstat_kernel<<<grid1, kCkThreads, kCkSmem, st>>>(q_panel, idx_tile, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int n_items = n_sessions * LG * a.n_bpanels;
+    score_chunk_colsum_kernel<<<std::min(n_items, p.sm_count), kCkThreads, kCkSmem2, st>>>(q_tile, idx_panel, a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    dim3 fgrid((unsigned)((max_nb + 255) / 256), (unsigned)n_sessions);
+    score_chunk_finish_kernel<<<fgrid, 256, 0, st>>>(ws.colsum, p.nblocks_dev, session_first, LG, ws.nb_pad,
+                                                     1.0f / (float)(g.L * g.H), scores, scores_stride);
+    return cudaGetLastError();
+}
+
+}  // namespace kvmem

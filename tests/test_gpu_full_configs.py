@@ -84,3 +84,34 @@ def test_config_1m_full():
 
 def test_config_batch8_full():
     _full_step(CONFIGS["batch8"])
+
+
+def test_config_chunk512_full():
+    """512-token chunk against the 1M index: score (tensor cores) -> select -> materialize."""
+    from paper_2609_04852_b200 import SelectParams, budget_blocks
+    spec = CONFIGS["chunk512"]
+    dev = torch.device("cuda", 0)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec, gen_device=dev)[0]
+    prm_d = select_params(spec)
+    prm = SelectParams(**prm_d)
+    B = spec.block_tokens
+    k = budget_blocks(prm, B, spec.n_blocks)
+    sel = torch.zeros(1, k, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    scores = torch.zeros(1, spec.n_blocks, dtype=torch.float32, device=dev)
+    view = pool.new_view(1, k * B)
+    q, qb = queries(spec, 0)
+    pool.select(q.to(dev), prm, sel, n_sel, scores)
+    pool.materialize(sel, n_sel, view)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    R, _ = orc.block_scores(qb[0], osess.idx, spec.n_blocks)
+    check_scores(scores.cpu().numpy()[0], R, spec.n_q_tokens)
+    ref_sel = orc.select(R, B, prm_d["budget_blocks"], prm_d["max_view_tokens"])
+    sel_gpu = sel.cpu().numpy()[0, : int(n_sel.item())]
+    assert len(sel_gpu) == k
+    check_selection(sel_gpu, R, ref_sel)
+    assert set(planted_blocks(spec, 0)[0].tolist()) <= set(sel_gpu.tolist())
+    vK, vV = orc.gather(osess.repo, osess.table, np.ascontiguousarray(sel_gpu), k * B)
+    assert np.array_equal(bits(view.k[0]), vK) and np.array_equal(bits(view.v[0]), vV)

@@ -181,6 +181,31 @@ def test_duplicate_blocks_tie_break_by_lower_id():
     assert np.all(got["scores"][0, :40] == got["scores"][0, 0])
 
 
+# ------------------------------------------------------------------ multi-token chunks (tensor-core scoring)
+
+@pytest.mark.parametrize("M,n_blocks,n_sessions", [(32, 200, 1), (40, 300, 1), (17, 517, 2), (64, 256, 1)])
+def test_chunked_scoring_matches_oracle(M, n_blocks, n_sessions):
+    # M * 4 rows per KV head: one full 128-row panel, ragged panels (160, 68 rows), ragged 256-block tiles
+    spec = CONFIGS["batch8"].with_(name="chunk", n_sessions=n_sessions, n_blocks=n_blocks, n_planted=6,
+                                   budget_blocks=24, n_q_tokens=M, permute_pages=False)
+    lens = [n_blocks - 37 * s for s in range(n_sessions)]
+    pool = fill_pool(spec, lens)
+    osess = fill_oracle(spec, lens)
+    q, qb = queries(spec)
+    got = _run_step(pool, spec, q.cuda(), _params(budget_blocks=spec.budget_blocks), spec.budget_blocks, attend=False)
+    for s in range(n_sessions):
+        R, _ = orc.block_scores(qb[s], osess[s].idx, osess[s].n_blocks)
+        assert abs(got["scores"][s, :lens[s]].sum() - M) < 1e-3 * M
+        check_scores(got["scores"][s, :lens[s]], R, M)
+        ref_sel = orc.select(R, spec.block_tokens, spec.budget_blocks, 1 << 30)
+        sel_gpu = got["sel"][s, : int(got["n_sel"][s])]
+        check_selection(sel_gpu, R, ref_sel)
+        vK, vV = orc.gather(osess[s].repo, osess[s].table, np.ascontiguousarray(sel_gpu), spec.budget_blocks * spec.block_tokens)
+        T = len(sel_gpu) * spec.block_tokens
+        assert np.array_equal(bits(got["view"].k[s])[:, :, :T], vK[:, :, :T])
+        assert np.array_equal(bits(got["view"].v[s])[:, :, :T], vV[:, :, :T])
+
+
 # ------------------------------------------------------------------ several sessions, permuted pages
 
 def test_multi_session_ragged_lengths_and_permuted_pages():
