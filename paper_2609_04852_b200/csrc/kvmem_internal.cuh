@@ -87,8 +87,8 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
 
 // multi-token query chunks: tcgen05 two-pass contraction
 struct ChunkWorkspace {
-    float2* rowstat;   // [ns][L][G][rows_pad] (max, log2 Z)
-    float* colsum;     // [ns][L][G][nb_pad]: per-head sums of the softmax weights over the head's query rows
+    float2* rowstat;   // [ns][L][G][4][rows_pad] (max, sum-exp) per slice of the tile columns
+    float* colsum;     // [ns][L][G][4][nb_pad]: per-head, per-column-slice sums of the softmax weights over the head's query rows
     float* scores;     // [ns][max_bps]
     size_t rowstat_bytes, colsum_bytes, scores_bytes, total;
     int rows, rows_pad, n_panels, nb_pad;

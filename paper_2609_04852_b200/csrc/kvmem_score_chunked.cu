@@ -16,7 +16,7 @@
 // Both passes: UMMA M = 128, N = 256, K = 128 (8 instructions of K = 16), bf16 in, fp32 accumulate.
 // Warp 0 is the TMA producer (stationary operand once per work item, streamed operand through a
 // shared-memory ring, 128-byte swizzle), one thread of warp 1 issues tcgen05.mma into two 256-column
-// TMEM accumulators, warps 2-5 are the epilogue.  The epilogue of tile t overlaps the MMAs of tile
+// TMEM accumulators, warps 2-17 are the epilogue (four per TMEM lane quarter, a quarter of a tile's columns each).  The epilogue of tile t overlaps the MMAs of tile
 // t + 1.  Pass 1: one CTA per 128-row query panel, sweeping all blocks.  Pass 2: persistent CTAs, one
 // work item = 128 blocks of one head, sweeping that head's query rows.  All mbarrier waits are bounded.
 #include <cudaTypedefs.h>
@@ -29,14 +29,20 @@
 
 namespace kvmem {
 
-constexpr int kCkBM = 128;                    // rows per panel
-constexpr int kCkBN = 256;                    // blocks per tile
-constexpr int kCkStages = 2;                  // index tiles in flight
-constexpr int kCkThreads = 192;               // TMA warp, MMA warp, 4 epilogue warps
-constexpr int kCkAHalf = kCkBM * 128;         // bytes of one 64-dim half of the Q panel  (16 KiB)
-constexpr int kCkBHalf = kCkBN * 128;         // bytes of one 64-dim half of an index tile (32 KiB)
-constexpr int kCkTmemCols = 512;              // two fp32 accumulators of 256 columns
-constexpr size_t kCkSmem = 2 * kCkAHalf + (size_t)kCkStages * 2 * kCkBHalf + 1024;
+constexpr int kCkBM = 128;                    // accumulator rows (UMMA M): one TMEM lane each
+constexpr int kCkBN = 256;                    // accumulator columns per tile (UMMA N): the largest N halves the
+                                              // MMA instructions per flop, which one issuing thread must sustain
+constexpr int kCkAccs = 2;                    // TMEM accumulators of 256 columns in flight
+constexpr int kCkStages1 = 3;                 // streamed tiles in flight, pass 1
+constexpr int kCkStages2 = 2;                 // streamed tiles in flight, pass 2 (two stationary panels + shifts also live in smem)
+constexpr int kCkEpiWarps = 16;               // four per TMEM lane quarter, each takes a quarter of a tile's columns
+constexpr int kCkSplit = kCkEpiWarps / 4;     // column slices per tile
+constexpr int kCkThreads = 64 + 32 * kCkEpiWarps;   // TMA warp, MMA warp, epilogue warps
+constexpr int kCkHalfCols = kCkBN / kCkSplit; // columns per epilogue warp and tile
+constexpr int kCkAHalf = kCkBM * 128;         // bytes of one 64-dim half of the 128-row operand tile (16 KiB)
+constexpr int kCkBHalf = kCkBN * 128;         // bytes of one 64-dim half of the 256-row operand tile (32 KiB)
+constexpr int kCkTmemCols = kCkAccs * kCkBN;  // 512: all of tensor memory
+constexpr size_t kCkSmem = 2 * kCkAHalf + (size_t)kCkStages1 * 2 * kCkBHalf + 1024;
 
 namespace t5 {   // tcgen05 wrappers
 
@@ -105,17 +111,12 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
-// 8-row groups 1,024 bytes apart.  `addr` may point 32*k bytes into the swizzle span (K advance).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3ffffu) >> 4);          // start address, 16-byte units
-    d |= (uint64_t)0 << 16;                            // leading byte offset: unused for swizzled K-major
-    d |= (uint64_t)(1024u >> 4) << 32;                 // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                            // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                            // layout type: 128-byte swizzle
-    return d;
-}
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, 8-row groups
+// 1,024 bytes apart.  Only the low word depends on the address; advancing K by 16 elements (32 bytes,
+// inside the swizzle span) adds 2 to it, and the second 64-dim half adds half_bytes / 16.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // SBO, descriptor version 1, SWIZZLE_128B
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr) { return (addr & 0x3ffffu) >> 4; }
+__device__ __forceinline__ uint64_t make_desc(uint32_t lo) { return ((uint64_t)kDescHi << 32) | (uint64_t)lo; }
 
 }  // namespace t5
 
@@ -129,8 +130,8 @@ __device__ __forceinline__ void tma_load_4d(void* dst_smem, const CUtensorMap* m
 
 struct ChunkArgs {
     const int32_t* nblocks_dev;
-    float2* rowstat;      // [ns][LG][rows_pad]   (max, log2 Z) of every query row, log2 domain
-    float* headsum;       // [ns][LG][nb_pad]     sum over the head's query rows of the softmax weights
+    float2* rowstat;      // [ns][LG][kCkSplit][rows_pad]  (max, sum-exp) of every query row over one slice of the tile columns, log2 domain
+    float* headsum;       // [ns][LG][kCkSplit][nb_pad]    per column slice: sum over the head's query rows of the softmax weights
     int32_t* status;
     int session_first, n_sessions, M, L, G, r, rows, rows_pad, nb_pad, n_bpanels;
     float scale_log2e;
@@ -141,16 +142,39 @@ __device__ __forceinline__ uint32_t chunk_idesc() {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kCkBN >> 3) << 17) | ((uint32_t)(kCkBM >> 4) << 24);
 }
 
-// one 128 x 256 x 128 tile: 8 MMAs of K = 16 (32 bytes inside the 128-byte swizzle span)
-__device__ __forceinline__ void issue_tile_mma(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
+// one 128 x 256 x 128 tile: 8 MMAs of K = 16
+__device__ __forceinline__ void issue_tile_mma(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo) {
     const uint32_t idesc = chunk_idesc();
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        const uint32_t koff = (uint32_t)(k & 3) * 32u;
-        const uint64_t da = t5::smem_desc_sw128(a_addr + (uint32_t)(k >> 2) * kCkAHalf + koff);
-        const uint64_t db = t5::smem_desc_sw128(b_addr + (uint32_t)(k >> 2) * kCkBHalf + koff);
-        t5::mma_bf16(d_tmem, da, db, idesc, k > 0 ? 1u : 0u);
+        const uint32_t ka = (uint32_t)(k >> 2) * (kCkAHalf >> 4) + (uint32_t)(k & 3) * 2u;
+        const uint32_t kb = (uint32_t)(k >> 2) * (kCkBHalf >> 4) + (uint32_t)(k & 3) * 2u;
+        t5::mma_bf16(d_tmem, t5::make_desc(a_lo + ka), t5::make_desc(b_lo + kb), idesc, k > 0 ? 1u : 0u);
     }
+}
+
+// Fold 32 raw logits of one query row into its running (max, sum-exp), exp2 domain.  `live` (ragged
+// tiles only) is how many of the 32 columns are real blocks.
+template <bool RAGGED>
+__device__ __forceinline__ void rowstat_chunk(const uint32_t (&raw)[32], int live, float scale_log2e, float& run_m, float& run_z) {
+    float v[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = (RAGGED && i >= live) ? -INFINITY : __uint_as_float(raw[i]);
+    // maximum of the raw logits by a tree (the scale is positive, so it commutes with max)
+    float m8[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m8[i] = fmaxf(fmaxf(v[i], v[i + 8]), fmaxf(v[i + 16], v[i + 24]));
+    const float mx = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
+    const float mn = fmaxf(run_m, mx * scale_log2e);
+    if (RAGGED && !(mn > -INFINITY)) return;
+    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        s0 += t5::ex2(fmaf(v[i], scale_log2e, -mn)); s1 += t5::ex2(fmaf(v[i + 1], scale_log2e, -mn));
+        s2 += t5::ex2(fmaf(v[i + 2], scale_log2e, -mn)); s3 += t5::ex2(fmaf(v[i + 3], scale_log2e, -mn));
+    }
+    run_z = run_z * t5::ex2(run_m - mn) + ((s0 + s1) + (s2 + s3));
+    run_m = mn;
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -159,7 +183,7 @@ __global__ void __launch_bounds__(kCkThreads, 1)
 score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_idx,
                            ChunkArgs a) {
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ uint64_t a_full, b_full[kCkStages], b_empty[kCkStages], acc_full[2], acc_empty[2];
+    __shared__ uint64_t a_full, b_full[kCkStages1], b_empty[kCkStages1], acc_full[kCkAccs], acc_empty[kCkAccs];
     __shared__ uint32_t tmem_base_slot;
 
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -175,8 +199,8 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 
     if (tid == 0) {
         ptx::mbar_init(&a_full, 1);
-        for (int i = 0; i < kCkStages; ++i) { ptx::mbar_init(&b_full[i], 1); ptx::mbar_init(&b_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 4); }
+        for (int i = 0; i < kCkStages1; ++i) { ptx::mbar_init(&b_full[i], 1); ptx::mbar_init(&b_empty[i], 1); }
+        for (int i = 0; i < kCkAccs; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], kCkEpiWarps); }
         ptx::fence_mbar_init();
     }
     if (warp == 1) {                     // one warp allocates the tensor memory for the whole CTA
@@ -200,8 +224,8 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             tma_load_4d(smem_a + kCkAHalf, &map_q, 64, g * a.r, l, m0, &a_full);
             const int z = ((a.session_first + s) * a.L + l) * a.G + g;
             for (int t = 0; t < n_tiles; ++t) {
-                const int st = t % kCkStages;
-                if (t >= kCkStages && !ptx::mbar_wait(&b_empty[st], (uint32_t)(((t / kCkStages) & 1) ^ 1))) {
+                const int st = t % kCkStages1;
+                if (t >= kCkStages1 && !ptx::mbar_wait(&b_empty[st], (uint32_t)(((t / kCkStages1) & 1) ^ 1))) {
                     atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                     break;
                 }
@@ -215,66 +239,53 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         // ------------------------------------------------ MMA issuer
         if (lane == 0 && n_tiles > 0) {
             bool ok = ptx::mbar_wait(&a_full, 0);
-            const uint32_t a_addr = ptx::smem_u32(smem_a);
+            const uint32_t a_lo = t5::desc_lo(ptx::smem_u32(smem_a)), b_lo0 = t5::desc_lo(ptx::smem_u32(smem_b));
             for (int t = 0; ok && t < n_tiles; ++t) {
-                const int st = t % kCkStages, acc = t & 1;
-                ok = ptx::mbar_wait(&b_full[st], (uint32_t)((t / kCkStages) & 1));
-                if (ok && t >= 2) ok = ptx::mbar_wait(&acc_empty[acc], (uint32_t)(((t >> 1) & 1) ^ 1));
+                const int st = t % kCkStages1, acc = t % kCkAccs;
+                ok = ptx::mbar_wait(&b_full[st], (uint32_t)((t / kCkStages1) & 1));
+                if (ok && t >= kCkAccs) ok = ptx::mbar_wait(&acc_empty[acc], (uint32_t)(((t / kCkAccs) & 1) ^ 1));
                 if (!ok) break;
                 t5::fence_after();
-                issue_tile_mma(tmem_base + (uint32_t)acc * kCkBN, a_addr, ptx::smem_u32(smem_b + (size_t)st * 2 * kCkBHalf));
+                issue_tile_mma(tmem_base + (uint32_t)acc * kCkBN, a_lo, b_lo0 + (uint32_t)st * (2 * kCkBHalf >> 4));
                 t5::commit(&b_empty[st]);                  // the index tile may be overwritten
                 t5::commit(&acc_full[acc]);                // the accumulator may be read
             }
             if (!ok) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
         }
     } else {
-        // ------------------------------------------------ epilogue (4 warps, one TMEM lane quarter each)
-        const int quarter = warp & 3;                      // warps 2,3,4,5 -> quarters 2,3,0,1
+        // ------------------------------------------------ epilogue: warp -> (TMEM lane quarter, column half)
+        const int quarter = warp & 3;                      // warps 2..17 -> quarters 2,3,0,1,...
+        const int half = (warp - 2) >> 2;
         const int row = panel * kCkBM + quarter * 32 + lane;   // row of this (session, l, g): m * r + hr
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * kCkHalfCols);
         float run_m = -INFINITY, run_z = 0.0f;
         for (int t = 0; t < n_tiles; ++t) {
-            const int acc = t & 1;
-            const bool arrived = ptx::mbar_wait(&acc_full[acc], (uint32_t)((t >> 1) & 1));
+            const int acc = t % kCkAccs;
+            const bool arrived = ptx::mbar_wait(&acc_full[acc], (uint32_t)((t / kCkAccs) & 1));
             if (!__all_sync(0xffffffffu, arrived)) {
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
             }
             t5::fence_after();
-            const int col0 = t * kCkBN;
-            const bool ragged = col0 + kCkBN > NB;
-            uint32_t buf[2][32];
-            t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN), buf[0]);
-#pragma unroll 2
-            for (int c = 0; c < kCkBN / 32; ++c) {
-                t5::ld_wait();
-                if (c + 1 < kCkBN / 32) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + (c + 1) * 32), buf[(c + 1) & 1]);
-                float v[32];
-                float mx = -INFINITY;
+            const int col0 = t * kCkBN + half * kCkHalfCols;
+            const bool ragged = col0 + kCkHalfCols > NB;
+            uint32_t buf[kCkHalfCols / 32][32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float x = __uint_as_float(buf[c & 1][i]) * a.scale_log2e;
-                    v[i] = (ragged && col0 + c * 32 + i >= NB) ? -INFINITY : x;
-                    mx = fmaxf(mx, v[i]);
-                }
-                const float mn = fmaxf(run_m, mx);
-                if (mn > -INFINITY) {
-                    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        s0 += t5::ex2(v[i] - mn); s1 += t5::ex2(v[i + 1] - mn);
-                        s2 += t5::ex2(v[i + 2] - mn); s3 += t5::ex2(v[i + 3] - mn);
-                    }
-                    run_z = run_z * t5::ex2(run_m - mn) + ((s0 + s1) + (s2 + s3));
-                    run_m = mn;
-                }
-            }
-            t5::fence_before();                            // the accumulator has been drained into registers
+            for (int c = 0; c < kCkHalfCols / 32; ++c) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf[c]);
+            t5::ld_wait();
+            // the accumulator now lives in registers: hand it back before doing the arithmetic
+            t5::fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
+            if (!ragged) {
+#pragma unroll
+                for (int c = 0; c < kCkHalfCols / 32; ++c) rowstat_chunk<false>(buf[c], 0, a.scale_log2e, run_m, run_z);
+            } else {
+#pragma unroll
+                for (int c = 0; c < kCkHalfCols / 32; ++c) rowstat_chunk<true>(buf[c], NB - (col0 + c * 32), a.scale_log2e, run_m, run_z);
+            }
         }
-        if (row < a.rows) a.rowstat[((size_t)s * LG + lg) * a.rows_pad + row] = make_float2(run_m, log2f(run_z));
+        if (row < a.rows) a.rowstat[(((size_t)s * LG + lg) * kCkSplit + half) * a.rows_pad + row] = make_float2(run_m, run_z);
     }
 
     t5::fence_before();
@@ -289,32 +300,33 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 // Pass 2.  Persistent CTAs; work item = (session, layer x KV head, 128-block panel).  TMEM lane = block.
 // Stationary operand: the panel's Mean-K vectors; streamed operand: the head's query rows, 256 at a time.
 constexpr int kCkShiftMax = 4096;                // query rows per (session, l, g) the shift vector can hold
-constexpr size_t kCkSmem2 = 2 * 2 * kCkAHalf + (size_t)kCkStages * 2 * kCkBHalf + kCkShiftMax * sizeof(float) + 1024;
+constexpr size_t kCkSmem2 = 2 * 2 * kCkAHalf + (size_t)kCkStages2 * 2 * kCkBHalf + kCkShiftMax * sizeof(float) + 1024;
 
 __global__ void __launch_bounds__(kCkThreads, 1)
 score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_idx,
                           ChunkArgs a) {
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ uint64_t a_full[2], a_empty[2], b_full[kCkStages], b_empty[kCkStages], acc_full[2], acc_empty[2];
+    __shared__ uint64_t a_full[2], a_empty[2], b_full[kCkStages2], b_empty[kCkStages2], acc_full[kCkAccs], acc_empty[kCkAccs];
     __shared__ uint32_t tmem_base_slot;
 
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     unsigned char* smem_a = base;                                  // index panels: 2 stages x 2 halves x 16 KiB
     unsigned char* smem_b = base + 2 * 2 * kCkAHalf;               // query tiles:  stages x 2 halves x 32 KiB
-    float* shift = reinterpret_cast<float*>(smem_b + (size_t)kCkStages * 2 * kCkBHalf);   // [n_qtiles * 256]
+    float* shift = reinterpret_cast<float*>(smem_b + (size_t)kCkStages2 * 2 * kCkBHalf);  // [n_qtiles * 256]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int LG = a.L * a.G;
     const int n_items = a.n_sessions * LG * a.n_bpanels;           // panel index fastest: neighbours share a head's Q
+    // a contiguous range of items per CTA: the head (and with it the shift vector) changes at most a few times
+    const int item_begin = (int)((long long)n_items * blockIdx.x / gridDim.x);
+    const int item_end = (int)((long long)n_items * (blockIdx.x + 1) / gridDim.x);
     const int n_qtiles = (a.rows + kCkBN - 1) / kCkBN;
     const int tokens_per_qtile = kCkBN / a.r;
 
     if (tid == 0) {
-        for (int i = 0; i < 2; ++i) {
-            ptx::mbar_init(&a_full[i], 1); ptx::mbar_init(&a_empty[i], 1);
-            ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 4);
-        }
-        for (int i = 0; i < kCkStages; ++i) { ptx::mbar_init(&b_full[i], 1); ptx::mbar_init(&b_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&a_full[i], 1); ptx::mbar_init(&a_empty[i], 1); }
+        for (int i = 0; i < kCkAccs; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], kCkEpiWarps); }
+        for (int i = 0; i < kCkStages2; ++i) { ptx::mbar_init(&b_full[i], 1); ptx::mbar_init(&b_empty[i], 1); }
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
@@ -341,7 +353,7 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
             ptx::prefetch_tensormap(&map_idx);
             int li = 0, tt = 0;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+            for (int item = item_begin; ok && item < item_end; ++item) {
                 int s, lg, bp;
                 if (!item_live(item, s, lg, bp)) continue;
                 const int l = lg / a.G, g = lg % a.G;
@@ -354,8 +366,8 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 ptx::tma_load_3d(adst, &map_idx, 0, bp * kCkBM, z, &a_full[as]);
                 ptx::tma_load_3d(adst + kCkAHalf, &map_idx, 64, bp * kCkBM, z, &a_full[as]);
                 for (int qt = 0; qt < n_qtiles; ++qt, ++tt) {
-                    const int st = tt % kCkStages;
-                    if (tt >= kCkStages) ok = ptx::mbar_wait(&b_empty[st], (uint32_t)(((tt / kCkStages) & 1) ^ 1));
+                    const int st = tt % kCkStages2;
+                    if (tt >= kCkStages2) ok = ptx::mbar_wait(&b_empty[st], (uint32_t)(((tt / kCkStages2) & 1) ^ 1));
                     if (!ok) break;
                     unsigned char* dst = smem_b + (size_t)st * 2 * kCkBHalf;
                     const int m0 = s * a.M + qt * tokens_per_qtile;
@@ -372,19 +384,20 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         if (lane == 0) {
             int li = 0, tt = 0;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+            for (int item = item_begin; ok && item < item_end; ++item) {
                 int s, lg, bp;
                 if (!item_live(item, s, lg, bp)) continue;
                 const int as = li & 1;
                 ok = ptx::mbar_wait(&a_full[as], (uint32_t)((li >> 1) & 1));
-                const uint32_t a_addr = ptx::smem_u32(smem_a + (size_t)as * 2 * kCkAHalf);
+                const uint32_t a_lo = t5::desc_lo(ptx::smem_u32(smem_a + (size_t)as * 2 * kCkAHalf));
+                const uint32_t b_lo0 = t5::desc_lo(ptx::smem_u32(smem_b));
                 for (int qt = 0; ok && qt < n_qtiles; ++qt, ++tt) {
-                    const int st = tt % kCkStages, acc = tt & 1;
-                    ok = ptx::mbar_wait(&b_full[st], (uint32_t)((tt / kCkStages) & 1));
-                    if (ok && tt >= 2) ok = ptx::mbar_wait(&acc_empty[acc], (uint32_t)(((tt >> 1) & 1) ^ 1));
+                    const int st = tt % kCkStages2, acc = tt % kCkAccs;
+                    ok = ptx::mbar_wait(&b_full[st], (uint32_t)((tt / kCkStages2) & 1));
+                    if (ok && tt >= kCkAccs) ok = ptx::mbar_wait(&acc_empty[acc], (uint32_t)(((tt / kCkAccs) & 1) ^ 1));
                     if (!ok) break;
                     t5::fence_after();
-                    issue_tile_mma(tmem_base + (uint32_t)acc * kCkBN, a_addr, ptx::smem_u32(smem_b + (size_t)st * 2 * kCkBHalf));
+                    issue_tile_mma(tmem_base + (uint32_t)acc * kCkBN, a_lo, b_lo0 + (uint32_t)st * (2 * kCkBHalf >> 4));
                     t5::commit(&b_empty[st]);
                     t5::commit(&acc_full[acc]);
                 }
@@ -394,63 +407,75 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
             if (!ok) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
         }
     } else {
-        // ------------------------------------------------ epilogue
+        // ------------------------------------------------ epilogue: warp -> (TMEM lane quarter, column half)
         const int quarter = warp & 3;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        const int et = tid - 64;                           // 0..127 among the epilogue threads
+        const int half = (warp - 2) >> 2;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * kCkHalfCols);
+        const int et = tid - 64;                           // index among the epilogue threads
         int tt = 0, cur_head = -1;
         bool failed = false;                               // a warp that gave up still meets every named barrier
-        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        for (int item = item_begin; item < item_end; ++item) {
             int s, lg, bp;
             if (!item_live(item, s, lg, bp)) continue;
             if (s * LG + lg != cur_head) {
-                // shifts -(max + log2 Z) of this head's query rows; -inf switches a padding row off
+                // shifts -(max + log2 Z) of this head's query rows, merging the column slices of
+                // pass 1; -inf switches a padding row off
                 cur_head = s * LG + lg;
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                const float2* rs = a.rowstat + (size_t)cur_head * a.rows_pad;
-                for (int j = et; j < n_qtiles * kCkBN; j += 128) {
+                asm volatile("bar.sync 1, %0;" ::"n"(32 * kCkEpiWarps) : "memory");
+                const float2* rs = a.rowstat + ((size_t)cur_head * kCkSplit) * a.rows_pad;
+                for (int j = et; j < n_qtiles * kCkBN; j += 32 * kCkEpiWarps) {
                     float sh = -INFINITY;
-                    if (j < a.rows) { const float2 st = rs[j]; sh = -(st.x + st.y); }
+                    if (j < a.rows) {
+                        float2 pp[kCkSplit];
+                        float mx = -INFINITY;
+#pragma unroll
+                        for (int h = 0; h < kCkSplit; ++h) { pp[h] = rs[(size_t)h * a.rows_pad + j]; mx = fmaxf(mx, pp[h].x); }
+                        float z = 0.0f;
+#pragma unroll
+                        for (int h = 0; h < kCkSplit; ++h) z += pp[h].x > -INFINITY ? pp[h].y * exp2f(pp[h].x - mx) : 0.0f;
+                        sh = -(mx + log2f(z));
+                    }
                     shift[j] = sh;
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, %0;" ::"n"(32 * kCkEpiWarps) : "memory");
             }
             float total = 0.0f;
             for (int qt = 0; qt < n_qtiles; ++qt, ++tt) {
                 if (failed) continue;
-                const int acc = tt & 1;
-                const bool arrived = ptx::mbar_wait(&acc_full[acc], (uint32_t)((tt >> 1) & 1));
+                const int acc = tt % kCkAccs;
+                const bool arrived = ptx::mbar_wait(&acc_full[acc], (uint32_t)((tt / kCkAccs) & 1));
                 if (!__all_sync(0xffffffffu, arrived)) {
                     if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                     failed = true;
                     continue;
                 }
                 t5::fence_after();
-                const float4* sh4 = reinterpret_cast<const float4*>(shift + qt * kCkBN);
-                uint32_t buf[2][32];
-                t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN), buf[0]);
-                float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
-#pragma unroll 2
-                for (int c = 0; c < kCkBN / 32; ++c) {
-                    t5::ld_wait();
-                    if (c + 1 < kCkBN / 32) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + (c + 1) * 32), buf[(c + 1) & 1]);
+                const float4* sh4 = reinterpret_cast<const float4*>(shift + qt * kCkBN + half * kCkHalfCols);
+                uint32_t buf[kCkHalfCols / 32][32];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        const float4 sh = sh4[c * 8 + (i >> 2)];            // same address in every lane: broadcast
-                        s0 += t5::ex2(fmaf(__uint_as_float(buf[c & 1][i]), a.scale_log2e, sh.x));
-                        s1 += t5::ex2(fmaf(__uint_as_float(buf[c & 1][i + 1]), a.scale_log2e, sh.y));
-                        s2 += t5::ex2(fmaf(__uint_as_float(buf[c & 1][i + 2]), a.scale_log2e, sh.z));
-                        s3 += t5::ex2(fmaf(__uint_as_float(buf[c & 1][i + 3]), a.scale_log2e, sh.w));
-                    }
-                }
-                total += (s0 + s1) + (s2 + s3);
+                for (int c = 0; c < kCkHalfCols / 32; ++c) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf[c]);
+                t5::ld_wait();
+                // the accumulator now lives in registers: hand it back before doing the arithmetic
                 t5::fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
+                float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+#pragma unroll
+                for (int c = 0; c < kCkHalfCols / 32; ++c) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        const float4 sh = sh4[c * 8 + (i >> 2)];            // same address in every lane: broadcast
+                        s0 += t5::ex2(fmaf(__uint_as_float(buf[c][i]), a.scale_log2e, sh.x));
+                        s1 += t5::ex2(fmaf(__uint_as_float(buf[c][i + 1]), a.scale_log2e, sh.y));
+                        s2 += t5::ex2(fmaf(__uint_as_float(buf[c][i + 2]), a.scale_log2e, sh.z));
+                        s3 += t5::ex2(fmaf(__uint_as_float(buf[c][i + 3]), a.scale_log2e, sh.w));
+                    }
+                }
+                total += (s0 + s1) + (s2 + s3);
             }
             const int b = bp * kCkBM + quarter * 32 + lane;
             if (!failed && b < a.nblocks_dev[a.session_first + s])
-                a.headsum[((size_t)s * LG + lg) * a.nb_pad + b] = total;
+                a.headsum[(((size_t)s * LG + lg) * kCkSplit + half) * a.nb_pad + b] = total;
         }
     }
 
@@ -462,7 +487,7 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     }
 }
 
-// R_b = (1/(L*H)) * sum over (layer, KV head) of the head sums, in a fixed order.
+// R_b = (1/(L*H)) * sum over (layer, KV head, column half) of the head sums, in a fixed order.
 __global__ void __launch_bounds__(256)
 score_chunk_finish_kernel(const float* __restrict__ headsum, const int32_t* __restrict__ nblocks_dev, int session_first,
                           int LG, int nb_pad, float inv_LH, float* __restrict__ scores, int scores_stride) {
@@ -494,10 +519,10 @@ ChunkWorkspace plan_chunk_workspace(const kvmem_pool_config_t& c, int n_sessions
     w.rows = n_q_tokens * r;
     w.n_panels = (w.rows + kCkBM - 1) / kCkBM;
     w.rows_pad = w.n_panels * kCkBM;
-    w.nb_pad = (c.max_blocks_per_session + kCkBN - 1) / kCkBN * kCkBN;
+    w.nb_pad = (c.max_blocks_per_session + 255) / 256 * 256;
     const size_t lg = (size_t)c.n_layers * c.n_kv_heads;
-    w.rowstat_bytes = align_up((size_t)n_sessions * lg * w.rows_pad * sizeof(float2), 256);
-    w.colsum_bytes = align_up((size_t)n_sessions * lg * w.nb_pad * sizeof(float), 256);
+    w.rowstat_bytes = align_up((size_t)n_sessions * lg * kCkSplit * w.rows_pad * sizeof(float2), 256);
+    w.colsum_bytes = align_up((size_t)n_sessions * lg * kCkSplit * w.nb_pad * sizeof(float), 256);
     w.scores_bytes = align_up((size_t)n_sessions * c.max_blocks_per_session * sizeof(float), 256);
     w.total = w.rowstat_bytes + w.colsum_bytes + w.scores_bytes;
     if (base) {
@@ -573,7 +598,7 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     dim3 fgrid((unsigned)((max_nb + 255) / 256), (unsigned)n_sessions);
-    score_chunk_finish_kernel<<<fgrid, 256, 0, st>>>(ws.colsum, p.nblocks_dev, session_first, LG, ws.nb_pad,
+    score_chunk_finish_kernel<<<fgrid, 256, 0, st>>>(ws.colsum, p.nblocks_dev, session_first, kCkSplit * LG, ws.nb_pad,
                                                      1.0f / (float)(g.L * g.H), scores, scores_stride);
     return cudaGetLastError();
 }
