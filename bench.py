@@ -35,7 +35,7 @@ from kvmem_workloads import CONFIGS, kv_blocks, make_queries, page_table, select
 
 METRIC = "select+materialize+attend steps/s"
 UNIT = "steps/s"
-KERNELS_PER_STEP = 6      # score_logits, score_finish, topk, gather, attend_split, attend_merge
+KERNELS_PER_STEP = 6      # score_logits, score_finish, topk, gather, attend_split, attend_merge (5 when fused)
 
 
 def measured_peaks():
@@ -178,17 +178,23 @@ def run_native(args):
     lse_pin = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device) if args.flush_l2 else None
     stream = torch.cuda.current_stream(device)
+    fused = spec.attend and not args.unfused
 
     def step(i, ev=None):
         q = q_dev[i % len(q_dev)]
         pool.select(q, prm, sel, n_sel)
         if ev is not None:
             ev[0].record(stream)
-        pool.materialize(sel, n_sel, view)
-        if ev is not None:
-            ev[1].record(stream)
-        if spec.attend:
-            pool.view_attend(q, view, n_sel, out, lse)
+        if fused:
+            pool.materialize_attend(q, sel, n_sel, view, out, lse)      # one pass: view written while attended
+            if ev is not None:
+                ev[1].record(stream)
+        else:
+            pool.materialize(sel, n_sel, view)
+            if ev is not None:
+                ev[1].record(stream)
+            if spec.attend:
+                pool.view_attend(q, view, n_sel, out, lse)
         if ev is not None:
             ev[2].record(stream)
 
@@ -279,7 +285,9 @@ def run_native(args):
         med = statistics.median
         gather_s = (sum(gat_ms) / K) * 1e-3
         gather_gbs = ns * ab["gather"] / gather_s / 1e9
-        step_gbs = world * K * ns * ab["total"] / (total_ms * 1e-3) / 1e9 / world      # per GPU
+        # fused: every view byte is read once (from the pages) and written once; separate calls read it a second time
+        step_bytes = ns * (ab["total"] - (ab["attend"] if fused else 0))
+        step_gbs = world * K * step_bytes / (total_ms * 1e-3) / 1e9 / world      # per GPU
         rows = ns * M * spec.n_layers * spec.n_q_heads
         line = {
             "metric": METRIC, "value": whole_job_rate(K, world, total_ms), "unit": UNIT, "n_gpus": world, "steps": K,
@@ -291,19 +299,25 @@ def run_native(args):
                        "history_tokens": spec.tokens, "view_tokens": cap, "query_sets": len(qsets),
                        "l2": "flushed between steps (256 MiB write)" if flush is not None else
                              "no flush: every step streams far more than the 126 MB L2",
-                       "parallelism": f"{world} independent session replica(s), one per GPU"},
+                       "parallelism": f"{world} independent session replica(s), one per GPU",
+                       "calls": "kvmem_select + kvmem_materialize_attend" if fused else
+                                "kvmem_select + kvmem_materialize" + (" + kvmem_view_attend" if spec.attend else "")},
             "e2e": {"value": whole_job_rate(Ke, world, e2e_ms), "unit": UNIT, "steps": Ke,
                     "h2d_bytes_per_step": rows * spec.head_dim * 2,
                     "d2h_bytes_per_step": rows * spec.head_dim * 4 + rows * 4,
                     "api": "kvmem_recall_step_host (pinned host query in, host O and LSE out, synchronous)"},
-            "gpu_launches": K * KERNELS_PER_STEP,
+            "gpu_launches": K * (KERNELS_PER_STEP - (1 if fused else 0)),
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "gather_bulk_kernel (kvmem_materialize)",
+            "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<true> + merge (kvmem_materialize_attend: view written while attended)"
+                                                   if fused else "gather_bulk_kernel (kvmem_materialize)",
                          "achieved": gather_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gather_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "algorithmic_bytes_per_launch": ns * ab["gather"], "avg_launch_ms": gather_s * 1e3,
-                         "traffic": GATHER_TRAFFIC.get(base.name)},
-            "step_hbm": {"algorithmic_bytes_per_step": ns * ab["total"], "achieved_gbs": step_gbs,
+                         "traffic": None if fused else GATHER_TRAFFIC.get(base.name)},
+            "step_hbm": {"algorithmic_bytes_per_step": step_bytes,
+                         "accounting": "index + view read + view write (fused pass)" if fused else
+                                       "index + gather read/write + attend read (separate calls)",
+                         "bytes_if_separate_calls": ns * ab["total"], "achieved_gbs": step_gbs,
                          "frac_of_peak": step_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "nominal_peak_gbs": 8000.0},
             "stages_ms": {"select": med(sel_ms), "materialize": med(gat_ms), "attend": med(att_ms),
@@ -434,6 +448,7 @@ def main():
     ap.add_argument("--workload", choices=sorted(CONFIGS), default="1m")
     ap.add_argument("--blocks", type=int, default=0, help="shrink the history to this many blocks (profiling)")
     ap.add_argument("--flush-l2", action="store_true", help="write 256 MiB between steps (for workloads near L2 size)")
+    ap.add_argument("--unfused", action="store_true", help="separate kvmem_materialize and kvmem_view_attend calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)
     args = ap.parse_args()

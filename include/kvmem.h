@@ -165,6 +165,18 @@ int kvmem_view_attend(kvmem_pool_t* pool, int32_t n_sessions, const void* q /*DE
                       const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
                       void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
+/* kvmem_materialize followed by kvmem_view_attend as ONE pass over the selected blocks (Sec. 4.4 execution
+ * view + Sec. 5.2 decode over it): each selected K/V tile is read once from the page pool through the
+ * block table, written to its place in the view, and attended over while it sits in shared memory.
+ * Same arguments, results, limits and error behaviour as the two separate calls; the view it leaves
+ * behind is bit-identical to kvmem_materialize's, and out/lse are those of kvmem_view_attend on it.
+ * HBM traffic per view byte drops from 2 reads + 1 write to 1 read + 1 write. */
+int kvmem_materialize_attend(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
+                             int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
+                             const int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/, void* view_v /*DEVICE*/,
+                             int32_t view_cap_tokens, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
+                             void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
 /* kvmem_view_attend for callers that cannot allocate device memory.  (The paper has no counterpart.)
  * Who needs it: a serving process that gave all of HBM to its KV pool at start-up and runs with
  * its allocator frozen, a plug-in that only ever sees the buffers of one request, or a latency path
@@ -186,8 +198,8 @@ int kvmem_view_attend_static(kvmem_pool_t* pool, int32_t n_sessions, const void*
                              void* stream);
 
 /* The whole recall step for callers whose query and results live in HOST memory: copies q to the
- * device, runs kvmem_select, kvmem_materialize and kvmem_view_attend, copies out and lse back and
- * waits for the stream (synchronous).  Same definitions and limits as the three calls above.
+ * device, runs kvmem_select and kvmem_materialize_attend, copies out and lse back and waits for the
+ * stream (synchronous).  Same definitions and limits as the individual calls.
  *   q_host     HOST bf16 [n_sessions][n_q_tokens][L][H][d]   (pinned memory makes the copies asynchronous)
  *   out_host   HOST fp32 [n_sessions][n_q_tokens][L][H][d];  lse_host HOST fp32 [n_sessions][n_q_tokens][L][H]
  *   staging    DEVICE, kvmem_step_staging_bytes(), 256-byte aligned: device copies of q, out, lse

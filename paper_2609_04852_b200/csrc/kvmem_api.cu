@@ -378,10 +378,8 @@ int kvmem_recall_step_host(kvmem_pool_t* p, int32_t session_first, int32_t n_ses
     int rc = kvmem_select(p, session_first, n_sessions, q_dev, n_q_tokens, prm, sel_ids, sel_stride, n_sel, nullptr,
                           select_ws, select_ws_bytes, stream);
     if (rc != KVMEM_OK) return rc;
-    rc = kvmem_materialize(p, session_first, n_sessions, sel_ids, sel_stride, n_sel, view_k, view_v, view_cap_tokens, stream);
-    if (rc != KVMEM_OK) return rc;
-    rc = kvmem_view_attend(p, n_sessions, q_dev, n_q_tokens, view_k, view_v, view_cap_tokens, n_sel, scale, out_dev,
-                           lse_dev, attend_ws, attend_ws_bytes, stream);
+    rc = kvmem_materialize_attend(p, session_first, n_sessions, q_dev, n_q_tokens, sel_ids, sel_stride, n_sel, view_k, view_v,
+                                  view_cap_tokens, scale, out_dev, lse_dev, attend_ws, attend_ws_bytes, stream);
     if (rc != KVMEM_OK) return rc;
     e = cudaMemcpyAsync(out_host, out_dev, rows * p->cfg.head_dim * 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(lse_host, lse_dev, rows * 4, cudaMemcpyDeviceToHost, st);
@@ -395,6 +393,41 @@ int kvmem_set_option(const char* name, int32_t value) {
     if (strcmp(name, "gather_mode") == 0 && (value == 0 || value == 1)) { g_gather_mode = value; return KVMEM_OK; }
     set_error("unknown option or value: %s = %d", name, value);
     return KVMEM_E_INVALID;
+}
+
+int kvmem_materialize_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                             const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v,
+                             int32_t view_cap_tokens, float scale, float* out, float* lse, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!q || !sel_ids || !n_sel || !view_k || !view_v || !out || !lse || !workspace || !aligned(q, 16) ||
+        !aligned(view_k, 128) || !aligned(view_v, 128) || !aligned(workspace, 256) || !aligned(out, 16)) {
+        set_error("kvmem_materialize_attend: null or misaligned pointer (views need 128-byte alignment)");
+        return KVMEM_E_INVALID;
+    }
+    if (n_q_tokens < 1 || sel_stride < 1) { set_error("n_q_tokens and sel_stride must be positive"); return KVMEM_E_INVALID; }
+    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
+        set_error("attention kernel is built for head_dim 128 and 64-token blocks");
+        return KVMEM_E_UNSUPPORTED;
+    }
+    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (view_cap_tokens < p->cfg.block_tokens || view_cap_tokens % p->cfg.block_tokens != 0) {
+        set_error("view_cap_tokens must be a positive multiple of block_tokens");
+        return KVMEM_E_INVALID;
+    }
+    if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
+    if ((int64_t)p->cfg.max_blocks * 2 * p->cfg.n_layers * p->cfg.n_kv_heads * p->cfg.block_tokens > 0x7fffffffll) {
+        set_error("page pool too large for 32-bit TMA row coordinates");
+        return KVMEM_E_UNSUPPORTED;
+    }
+    AttendPlan plan = plan_attend(p->cfg, n_sessions, n_q_tokens, p->sm_count);
+    if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
+    cudaError_t e = launch_attend(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, (const __nv_bfloat16*)view_k,
+                                  (const __nv_bfloat16*)view_v, view_cap_tokens, n_sel, scale, out, lse, workspace,
+                                  (cudaStream_t)stream, sel_ids, sel_stride, session_first);
+    if (e != cudaSuccess) return cuda_fail("fused materialize+attend kernel launch", e);
+    return KVMEM_OK;
 }
 
 int kvmem_get_index(kvmem_pool_t* p, int32_t session, const void** index, int32_t* n_blocks) {

@@ -41,6 +41,11 @@ struct AttendArgs {
     int32_t* status;
     int M, L, H, G, r, rows, n_splits, cap_tokens;
     float scale_log2e;
+    // fused view assembly (attend_split_kernel<true>): tiles come from the page pool through the block table
+    const int32_t* sel_ids;      // [n_sessions][sel_stride]
+    const int32_t* tables;       // [max_sessions][max_bps]
+    const int32_t* nblocks_dev;  // [max_sessions]
+    int session_first, sel_stride, max_bps, max_blocks;
 };
 
 AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, int sm_count) {
@@ -68,8 +73,15 @@ static int choose_splits(int heads, int max_tiles, int sms) {
     return best;
 }
 
-__global__ void __launch_bounds__(kAttThreads, 1)
-attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, AttendArgs a) {
+// FUSED = false: tiles are read from the materialised view.
+// FUSED = true : tiles are read from the page pool through the block table (what the gather reads), one
+//                extra warp stores every tile into the view with TMA while the consumers attend over it,
+//                so the view is assembled and attended in one pass: 1 read + 1 write per view byte
+//                instead of 2 reads + 1 write.
+template <bool FUSED>
+__global__ void __launch_bounds__(kAttThreads + (FUSED ? 32 : 0), 1)
+attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                    const __grid_constant__ CUtensorMap map_pages, AttendArgs a) {
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages];
     __shared__ float merge_m[kAttConsumers][kRowsPad], merge_l[kAttConsumers][kRowsPad];
@@ -88,7 +100,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     const int n_tiles = t1 - t0;
 
     if (tid == 0) {
-        for (int i = 0; i < kAttStages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kAttConsumers / kAttGroups); }
+        for (int i = 0; i < kAttStages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kAttConsumers / kAttGroups + (FUSED ? 1 : 0)); }
         ptx::fence_mbar_init();
     }
     __syncthreads();
@@ -100,23 +112,87 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 
     if (warp == kAttConsumers) {
         // ---------------- producer ----------------
+        if (!FUSED) {
+            if (lane == 0 && n_tiles > 0) {
+                ptx::prefetch_tensormap(&map_k);
+                ptx::prefetch_tensormap(&map_v);
+                for (int it = 0; it < n_tiles; ++it) {
+                    const int st = it % kAttStages;
+                    if (it >= kAttStages && !ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kAttStages) & 1) ^ 1))) {
+                        atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+                        break;
+                    }
+                    unsigned char* dst = stages + (size_t)st * kStageBytes;
+                    const int y = (t0 + it) * kTile;
+                    ptx::mbar_expect_tx(&full_bar[st], kStageBytes);
+                    ptx::tma_load_3d(dst, &map_k, 0, y, z, &full_bar[st]);
+                    ptx::tma_load_3d(dst + kHalfBytes, &map_k, 64, y, z, &full_bar[st]);
+                    ptx::tma_load_3d(dst + 2 * kHalfBytes, &map_v, 0, y, z, &full_bar[st]);
+                    ptx::tma_load_3d(dst + 3 * kHalfBytes, &map_v, 64, y, z, &full_bar[st]);
+                }
+            }
+        } else if (n_tiles > 0) {
+            // the whole warp looks up pages, 32 tiles at a time; lane 0 issues the loads
+            if (lane == 0) ptx::prefetch_tensormap(&map_pages);
+            const int NB = a.nblocks_dev[a.session_first + s];
+            int base_it = 0, my_page = 0;
+            auto lookup = [&](int it) -> int {
+                if (it >= n_tiles) return 0;
+                const int id = a.sel_ids[(size_t)s * a.sel_stride + t0 + it];
+                int pg = -1;
+                if (id >= 0 && id < NB) pg = a.tables[(size_t)(a.session_first + s) * a.max_bps + id];
+                if (pg < 0 || pg >= a.max_blocks) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); pg = 0; }
+                return pg;           // a flagged id reads page 0 instead of faulting; the status word reports it
+            };
+            my_page = lookup(lane);
+            bool ok = true;
+            for (int it = 0; it < n_tiles; ++it) {
+                if (it >= base_it + 32) { base_it = it; my_page = lookup(base_it + lane); }
+                const int page = __shfl_sync(0xffffffffu, my_page, it - base_it);
+                if (lane == 0) {
+                    const int st = it % kAttStages;
+                    if (it >= kAttStages) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kAttStages) & 1) ^ 1));
+                    if (ok) {
+                        unsigned char* dst = stages + (size_t)st * kStageBytes;
+                        // page layout [K|V][L*G][64 tokens][128]: rows of 256 B
+                        const int yk = ((page * 2 + 0) * LG + lg) * kTile, yv = ((page * 2 + 1) * LG + lg) * kTile;
+                        ptx::mbar_expect_tx(&full_bar[st], kStageBytes);
+                        ptx::tma_load_2d(dst, &map_pages, 0, yk, &full_bar[st]);
+                        ptx::tma_load_2d(dst + kHalfBytes, &map_pages, 64, yk, &full_bar[st]);
+                        ptx::tma_load_2d(dst + 2 * kHalfBytes, &map_pages, 0, yv, &full_bar[st]);
+                        ptx::tma_load_2d(dst + 3 * kHalfBytes, &map_pages, 64, yv, &full_bar[st]);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
+            }
+        }
+    } else if (FUSED && warp == kAttConsumers + 1) {
+        // ---------------- view writer: every tile that lands in shared memory is stored to the view ----------------
         if (lane == 0 && n_tiles > 0) {
             ptx::prefetch_tensormap(&map_k);
             ptx::prefetch_tensormap(&map_v);
+            bool ok = true;
             for (int it = 0; it < n_tiles; ++it) {
                 const int st = it % kAttStages;
-                if (it >= kAttStages && !ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kAttStages) & 1) ^ 1))) {
-                    atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
-                    break;
-                }
-                unsigned char* dst = stages + (size_t)st * kStageBytes;
+                ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kAttStages) & 1));
+                if (!ok) break;
+                unsigned char* src = stages + (size_t)st * kStageBytes;
                 const int y = (t0 + it) * kTile;
-                ptx::mbar_expect_tx(&full_bar[st], kStageBytes);
-                ptx::tma_load_3d(dst, &map_k, 0, y, z, &full_bar[st]);
-                ptx::tma_load_3d(dst + kHalfBytes, &map_k, 64, y, z, &full_bar[st]);
-                ptx::tma_load_3d(dst + 2 * kHalfBytes, &map_v, 0, y, z, &full_bar[st]);
-                ptx::tma_load_3d(dst + 3 * kHalfBytes, &map_v, 64, y, z, &full_bar[st]);
+                ptx::tma_store_3d(&map_k, src, 0, y, z);
+                ptx::tma_store_3d(&map_k, src + kHalfBytes, 64, y, z);
+                ptx::tma_store_3d(&map_v, src + 2 * kHalfBytes, 0, y, z);
+                ptx::tma_store_3d(&map_v, src + 3 * kHalfBytes, 64, y, z);
+                ptx::bulk_commit();
+                if (it > 0) {                              // all but the newest store have left shared memory
+                    ptx::bulk_wait_read<1>();
+                    ptx::mbar_arrive(&empty_bar[(it - 1) % kAttStages]);
+                }
             }
+            ptx::bulk_wait_read<0>();
+            if (ok) ptx::mbar_arrive(&empty_bar[(n_tiles - 1) % kAttStages]);
+            else atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+            ptx::bulk_wait<0>();                           // the view is complete before the kernel ends
         }
     } else {
         // ---------------- consumers ----------------
@@ -316,18 +392,41 @@ static bool make_view_map(CUtensorMap* map, const __nv_bfloat16* view, int heads
     return r == CUDA_SUCCESS;
 }
 
+// page pool [max_blocks * 2 * L*G * 64 rows][128] bf16 as a 2-D tensor; box = 64 dims x 64 tokens, 128-byte swizzle
+static bool make_pages_map(CUtensorMap* map, const kvmem_pool& p) {
+    PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
+    if (!enc) return false;
+    const Geometry& g = p.geo;
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)g.max_blocks * 2 * g.L * g.G * kTile};
+    cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.pages, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// sel_ids == nullptr: attend over an already materialised view.  Otherwise: assemble the view from the
+// pages of sessions [session_first, session_first + n_sessions) and attend over it in the same kernel.
 cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M,
                           const __nv_bfloat16* view_k, const __nv_bfloat16* view_v, int view_cap_tokens,
                           const int32_t* n_sel, float scale, float* out, float* lse, void* workspace,
-                          cudaStream_t st) {
+                          cudaStream_t st, const int32_t* sel_ids, int sel_stride, int session_first) {
     const Geometry& g = p.geo;
     const int LG = g.L * g.G, heads = n_sessions * LG;
-    CUtensorMap map_k, map_v;
+    const bool fused = sel_ids != nullptr;
+    CUtensorMap map_k, map_v, map_pages;
     if (!make_view_map(&map_k, view_k, heads, view_cap_tokens) || !make_view_map(&map_v, view_v, heads, view_cap_tokens))
         return cudaErrorInvalidValue;
+    if (fused) {
+        if (!make_pages_map(&map_pages, p)) return cudaErrorInvalidValue;
+    } else {
+        map_pages = map_k;
+    }
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attend_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        cudaError_t e = cudaFuncSetAttribute(attend_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attend_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -342,8 +441,13 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     a.cap_tokens = view_cap_tokens;
     const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
     a.scale_log2e = sc * 1.4426950408889634f;
+    a.sel_ids = sel_ids; a.tables = p.tables; a.nblocks_dev = p.nblocks_dev;
+    a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
-    attend_split_kernel<<<grid, kAttThreads, kAttSmem, st>>>(map_k, map_v, a);
+    if (fused)
+        attend_split_kernel<true><<<grid, kAttThreads + 32, kAttSmem, st>>>(map_k, map_v, map_pages, a);
+    else
+        attend_split_kernel<false><<<grid, kAttThreads, kAttSmem, st>>>(map_k, map_v, map_pages, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     attend_merge_kernel<<<dim3((unsigned)a.rows, (unsigned)heads), kD, 0, st>>>(a.part_o, a.part_ml, out, lse, M, g.L, g.H, g.G,

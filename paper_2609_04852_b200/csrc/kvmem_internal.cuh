@@ -117,6 +117,6 @@ AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tok
 cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M,
                           const __nv_bfloat16* view_k, const __nv_bfloat16* view_v, int view_cap_tokens,
                           const int32_t* n_sel, float scale, float* out, float* lse, void* workspace,
-                          cudaStream_t st);
+                          cudaStream_t st, const int32_t* sel_ids = nullptr, int sel_stride = 0, int session_first = 0);
 
 }  // namespace kvmem

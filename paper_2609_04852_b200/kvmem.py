@@ -71,6 +71,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_get_block_table": (C.c_int, [vp, i32, C.POINTER(vp), C.POINTER(i32)]),
         "kvmem_device_status": (C.c_int, [vp, C.POINTER(i32), vp]),
         "kvmem_set_option": (C.c_int, [C.c_char_p, i32]),
+        "kvmem_materialize_attend": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
         "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
         "kvmem_recall_step_host": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, i32, f32, vp, vp,
@@ -89,7 +90,7 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_session_reset", "kvmem_session_blocks", "kvmem_append_blocks", "kvmem_select",
             "kvmem_materialize", "kvmem_view_attend", "kvmem_get_index", "kvmem_get_block_table",
             "kvmem_device_status", "kvmem_set_option", "kvmem_step_staging_bytes", "kvmem_recall_step_host",
-            "kvmem_view_attend_static")
+            "kvmem_view_attend_static", "kvmem_materialize_attend")
 
 
 def _check(status: int) -> None:
@@ -222,6 +223,17 @@ class Pool:
                                           _dev(view.v, torch.bfloat16), view.cap_tokens, _dev(n_sel, torch.int32),
                                           scale, _dev(out, torch.float32), _dev(lse, torch.float32),
                                           ws.data_ptr(), ws.numel(), _stream()))
+
+    def materialize_attend(self, q: torch.Tensor, sel_ids: torch.Tensor, n_sel: torch.Tensor, view: View,
+                           out: torch.Tensor, lse: torch.Tensor, scale: float = 0.0, session_first: int = 0) -> None:
+        """materialize + view_attend in one pass over the selected blocks (same results, a third less HBM traffic)."""
+        ns, M = q.shape[0], q.shape[1]
+        ws = self.attend_workspace(ns, M)
+        _check(self.lib.kvmem_materialize_attend(self.handle, session_first, ns, _dev(q, torch.bfloat16), M,
+                                                 _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
+                                                 _dev(view.k, torch.bfloat16), _dev(view.v, torch.bfloat16),
+                                                 view.cap_tokens, scale, _dev(out, torch.float32),
+                                                 _dev(lse, torch.float32), ws.data_ptr(), ws.numel(), _stream()))
 
     def view_attend_static(self, q: torch.Tensor, view: View, n_sel: torch.Tensor, out: torch.Tensor,
                            lse: torch.Tensor, scale: float = 0.0) -> None:

@@ -51,8 +51,15 @@ def _full_step(spec, qsets=(0,), gap_forced_budget=None):
         pool.select(qd, prm, sel, n_sel, scores)
         pool.materialize(sel, n_sel, view)
         pool.view_attend(qd, view, n_sel, out, lse)
+        # the fused call (what the benchmark times) must leave the same view and the same results
+        view2 = pool.new_view(ns, k * B)
+        out2, lse2 = pool.new_outputs(ns, M)
+        pool.materialize_attend(qd, sel, n_sel, view2, out2, lse2)
         torch.cuda.synchronize()
         assert pool.device_status() == 0
+        assert torch.equal(view.k, view2.k) and torch.equal(view.v, view2.v)
+        assert torch.equal(out, out2) and torch.equal(lse, lse2)
+        del view2
         sel_h, n_h, sc_h = sel.cpu().numpy(), n_sel.cpu().numpy(), scores.cpu().numpy()
         out_h, lse_h = out.cpu().numpy(), lse.cpu().numpy()
         for s in range(ns):

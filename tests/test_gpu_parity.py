@@ -181,6 +181,54 @@ def test_duplicate_blocks_tie_break_by_lower_id():
     assert np.all(got["scores"][0, :40] == got["scores"][0, 0])
 
 
+# ------------------------------------------------------------------ fused view assembly + attention
+
+@pytest.mark.parametrize("n_sessions,M,budget", [(1, 4, 150), (3, 1, 20), (1, 2, 1)])
+def test_fused_materialize_attend_equals_separate_calls_and_oracle(n_sessions, M, budget):
+    spec = CONFIGS["batch8"].with_(name="fused", n_sessions=n_sessions, n_blocks=300, n_planted=6, budget_blocks=budget,
+                                   n_q_tokens=M)
+    lens = [300 - 41 * s for s in range(n_sessions)]
+    pool = fill_pool(spec, lens)
+    osess = fill_oracle(spec, lens)
+    dev = torch.device("cuda", 0)
+    q, qb = queries(spec)
+    qd = q.to(dev)
+    sel = torch.full((n_sessions, budget), -1, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(n_sessions, dtype=torch.int32, device=dev)
+    pool.select(qd, _params(budget_blocks=budget), sel, n_sel)
+    view_a, view_b = pool.new_view(n_sessions, budget * 64), pool.new_view(n_sessions, budget * 64)
+    out_a, lse_a = pool.new_outputs(n_sessions, M)
+    out_b, lse_b = pool.new_outputs(n_sessions, M)
+    pool.materialize(sel, n_sel, view_a)
+    pool.view_attend(qd, view_a, n_sel, out_a, lse_a)
+    pool.materialize_attend(qd, sel, n_sel, view_b, out_b, lse_b)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    assert torch.equal(view_a.k, view_b.k) and torch.equal(view_a.v, view_b.v), "fused view differs from the gathered view"
+    assert torch.equal(out_a, out_b) and torch.equal(lse_a, lse_b), "same tiles, same order: results must be identical"
+    for s in range(n_sessions):
+        ids = sel[s, : int(n_sel[s])].cpu().numpy()
+        vK, vV = orc.gather(osess[s].repo, osess[s].table, np.ascontiguousarray(ids), budget * 64)
+        assert np.array_equal(bits(view_b.k[s]), vK) and np.array_equal(bits(view_b.v[s]), vV)
+        ref_out, ref_lse = orc.attend(qb[s], vK, vV, len(ids) * 64)
+        assert np.abs(out_b[s].cpu().numpy() - ref_out).max() <= ATTN_ATOL
+        assert np.abs(lse_b[s].cpu().numpy() - ref_lse).max() <= ATTN_ATOL
+
+
+def test_fused_path_flags_out_of_range_ids():
+    from paper_2609_04852_b200.kvmem import E_DEVICE_RANGE
+    spec = SMALL
+    pool = fill_pool(spec)
+    dev = torch.device("cuda", 0)
+    q, _ = queries(spec)
+    sel = torch.tensor([[1, 5000, 7]], dtype=torch.int32, device=dev)
+    n_sel = torch.tensor([3], dtype=torch.int32, device=dev)
+    view = pool.new_view(1, 4 * spec.block_tokens)
+    out, lse = pool.new_outputs(1, spec.n_q_tokens)
+    pool.materialize_attend(q.to(dev), sel, n_sel, view, out, lse)
+    assert pool.device_status() == E_DEVICE_RANGE
+
+
 # ------------------------------------------------------------------ multi-token chunks (tensor-core scoring)
 
 @pytest.mark.parametrize("M,n_blocks,n_sessions", [(32, 200, 1), (40, 300, 1), (17, 517, 2), (64, 256, 1)])
