@@ -231,7 +231,8 @@ int kvmem_device_status(kvmem_pool_t* pool, int32_t* status /*HOST*/, void* stre
 
 /* Process-wide implementation switches used to compare kernel variants; they never change results.
  * (No counterpart in the paper.)  "gather_mode": 1 = bulk asynchronous copies through shared memory
- * (default), 0 = 128-bit load/store copy. */
+ * (default), 0 = 128-bit load/store copy.  "score_mode" (decode-sized queries): 1 = dot products on the
+ * tensor cores (default), 0 = fp32 ALU kernel that reduces the query rows with warp shuffles. */
 int kvmem_set_option(const char* name /*HOST*/, int32_t value);
 
 #ifdef __cplusplus

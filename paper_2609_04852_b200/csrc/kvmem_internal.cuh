@@ -65,6 +65,7 @@ constexpr uint64_t kMagic = 0x4b564d454d423230ull;  // "KVMEMB20"
 void set_error(const char* fmt, ...);
 
 // tuning switches (kvmem_set_option)
+extern int g_score_mode;    // 1: tensor-core decode scoring (default), 0: fp32 ALU + warp-shuffle kernel
 extern int g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
 
 // ---- kernel launchers (each defined next to its kernel) ----------------------------------------

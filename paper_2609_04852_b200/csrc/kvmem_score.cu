@@ -11,6 +11,7 @@
 // coalesced, and each CTA carries per-row (max, sum-exp) across its tiles: the cross-tile softmax
 // statistics that Sec. 5.2 describes for tiled scoring.  A second small kernel merges the tile
 // statistics per row and reduces rows in a fixed order, so results are run-to-run identical.
+#include <cudaTypedefs.h>
 #include <math.h>
 
 #include <algorithm>
@@ -217,22 +218,186 @@ score_logits_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     }
 }
 
+// Same contract as score_logits_kernel, with the dot products on the tensor cores: the M*r <= 16 query
+// rows of a pass form one m16 MMA tile (bf16 mma.sync, fp32 accumulate), each warp takes 16 of the
+// tile's 128 Mean-K vectors.  Index tiles arrive by tiled TMA with the 128-byte swizzle, so the
+// ldmatrix reads are conflict-free.  This removes the fp32-ALU bound of the shuffle kernel (16 rows
+// x 128 dims = 2,048 FMAs per 256-byte vector) and leaves the kernel bound by the index stream.
+__global__ void __launch_bounds__(kScoreThreads, 1)
+score_logits_mma_kernel(const __grid_constant__ CUtensorMap map_idx, const __nv_bfloat16* __restrict__ q,
+                        const int32_t* __restrict__ nblocks_dev, int session_first, int M, int L, int H, int G,
+                        int max_bps, float* __restrict__ logits, float2* __restrict__ partials, int rows, int rows_pad,
+                        int nb_pad, int n_parts, float scale_log2e, int32_t* __restrict__ status) {
+    constexpr int RP = 16;
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ uint64_t full_bar[kScoreStages];
+    __shared__ float slog[RP][kChunk + 4];
+    unsigned char* stage_mem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    constexpr uint32_t kHalf = kChunk * 128;                 // one 64-dim half of a tile: 128 rows x 128 B
+    constexpr uint32_t kStage = 2 * kHalf;
+
+    const int s = blockIdx.z, lg = blockIdx.y, part = blockIdx.x;
+    const int l = lg / G, g = lg % G, r = H / G;
+    const int NB = nblocks_dev[session_first + s];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const size_t slab = ((size_t)s * L * G + lg) * rows_pad;
+    const int row_base = ((session_first + s) * L * G + lg) * max_bps;     // first index row of this (session, l, g)
+
+    const int n_chunks = (NB + kChunk - 1) / kChunk;
+    const int c_begin = (int)((long long)n_chunks * part / n_parts), c_end = (int)((long long)n_chunks * (part + 1) / n_parts);
+    const int n_mine = c_end - c_begin;
+
+    if (tid == 0) {
+        for (int i = 0; i < kScoreStages; ++i) ptx::mbar_init(&full_bar[i], 1);
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&map_idx);
+    }
+    __syncthreads();
+
+    int issued = 0, waited = 0;
+    auto issue = [&](int chunk) {                          // thread 0 only
+        const int st = issued % kScoreStages;
+        unsigned char* dst = stage_mem + (size_t)st * kStage;
+        ptx::mbar_expect_tx(&full_bar[st], kStage);
+        ptx::tma_load_2d(dst, &map_idx, 0, row_base + chunk * kChunk, &full_bar[st]);
+        ptx::tma_load_2d(dst + kHalf, &map_idx, 64, row_base + chunk * kChunk, &full_bar[st]);
+    };
+    const uint32_t stage0 = ptx::smem_u32(stage_mem);
+    const int mj = lane >> 3, mr = lane & 7;               // ldmatrix: matrix index and row within it
+
+    for (int pass = 0; pass * RP < rows; ++pass) {
+        const int row0 = pass * RP;
+        // Q fragments (A operand, m16k16 x 8 k-steps): row j = m * r + hr -> q[s][m][l][g*r + hr]
+        uint32_t qf[8][4];
+        {
+            const int ra = row0 + (lane >> 2), rb = ra + 8;
+            const __nv_bfloat16* qa = nullptr;
+            const __nv_bfloat16* qb = nullptr;
+            if (ra < rows) qa = q + ((((size_t)s * M + ra / r) * L + l) * H + (size_t)g * r + ra % r) * 128;
+            if (rb < rows) qb = q + ((((size_t)s * M + rb / r) * L + l) * H + (size_t)g * r + rb % r) * 128;
+            const int kq = 2 * (lane & 3);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                qf[ks][0] = qa ? *reinterpret_cast<const uint32_t*>(qa + ks * 16 + kq) : 0u;
+                qf[ks][1] = qb ? *reinterpret_cast<const uint32_t*>(qb + ks * 16 + kq) : 0u;
+                qf[ks][2] = qa ? *reinterpret_cast<const uint32_t*>(qa + ks * 16 + kq + 8) : 0u;
+                qf[ks][3] = qb ? *reinterpret_cast<const uint32_t*>(qb + ks * 16 + kq + 8) : 0u;
+            }
+        }
+        float run_m[2] = {-INFINITY, -INFINITY}, run_l[2] = {0.0f, 0.0f};
+
+        if (tid == 0) {
+            for (int i = 0; i < min(kScoreStages - 1, n_mine); ++i) { issue(c_begin + i); ++issued; }
+        }
+        for (int i = 0; i < n_mine; ++i) {
+            const int chunk = c_begin + i, b0 = chunk * kChunk;
+            const int st = waited % kScoreStages;
+            const bool ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((waited / kScoreStages) & 1));
+            ++waited;
+            if (__syncthreads_or(!ok)) {                  // CTA-uniform: somebody gave up
+                if (tid == 0) atomicExch(status, (int)KVMEM_E_TIMEOUT);
+                return;
+            }
+            if (tid == 0 && i + kScoreStages - 1 < n_mine) { issue(chunk + kScoreStages - 1); ++issued; }
+            const uint32_t tile = stage0 + (uint32_t)st * kStage;
+            // S = Q Kbar^T for this warp's 16 vectors: 2 n-tiles x 8 k-steps
+            float sc[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) { sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.0f; }
+#pragma unroll
+            for (int kp = 0; kp < 4; ++kp) {
+                const int cg = kp * 4 + mj;
+                const uint32_t half_off = (uint32_t)(cg >> 3) * kHalf;
+                const int c = cg & 7;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    const int rowi = warp * 16 + nt * 8 + mr;
+                    const uint32_t addr = tile + half_off + (uint32_t)rowi * 128u + (uint32_t)((c ^ (rowi & 7)) << 4);
+                    uint32_t b0r, b1r, b2r, b3r;
+                    ptx::ldmatrix_x4(addr, b0r, b1r, b2r, b3r);
+                    ptx::mma_bf16_16816(sc[nt], qf[2 * kp], b0r, b1r);
+                    ptx::mma_bf16_16816(sc[nt], qf[2 * kp + 1], b2r, b3r);
+                }
+            }
+            {
+                const int ra = lane >> 2, rb = ra + 8;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    const int col = warp * 16 + nt * 8 + 2 * (lane & 3);
+                    const bool v0 = b0 + col < NB, v1 = b0 + col + 1 < NB;
+                    slog[ra][col] = v0 ? sc[nt][0] * scale_log2e : -INFINITY;
+                    slog[ra][col + 1] = v1 ? sc[nt][1] * scale_log2e : -INFINITY;
+                    slog[rb][col] = v0 ? sc[nt][2] * scale_log2e : -INFINITY;
+                    slog[rb][col + 1] = v1 ? sc[nt][3] * scale_log2e : -INFINITY;
+                }
+            }
+            __syncthreads();
+            // per-row statistics of this tile (folded into the running pair) and coalesced logit store
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = warp + 8 * jj;
+                float mx = -INFINITY, v[kChunk / 32];
+#pragma unroll
+                for (int t = 0; t < kChunk / 32; ++t) {
+                    v[t] = slog[j][lane + 32 * t];
+                    mx = fmaxf(mx, v[t]);
+                }
+#pragma unroll
+                for (int o = 16; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                const float mn = fmaxf(run_m[jj], mx);      // finite: a chunk holds at least one block
+                float sum = 0.0f;
+#pragma unroll
+                for (int t = 0; t < kChunk / 32; ++t) sum += exp2f(v[t] - mn);
+#pragma unroll
+                for (int o = 16; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+                run_l[jj] = run_l[jj] * exp2f(run_m[jj] - mn) + sum;
+                run_m[jj] = mn;
+                float* dst = logits + (slab + row0 + j) * (size_t)nb_pad + b0;
+#pragma unroll
+                for (int t = 0; t < kChunk / 32; ++t) dst[lane + 32 * t] = v[t];
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+            const int j = warp + 8 * jj;
+            if (lane == 0) partials[(slab + row0 + j) * n_parts + part] = make_float2(run_m[jj], run_l[jj]);
+        }
+    }
+}
+
 // Merge the per-CTA statistics of every row, then R_b = (1/(L*H)) sum_rows exp2(logit - max_row) / Z_row.
-// A CTA owns 32 consecutive blocks; thread (lgs, bl) sums the rows of heads lgs, lgs + 8, ... for block
-// bl (16 independent coalesced loads in flight), and the 8 partial sums are added in a fixed order.
-constexpr int kFinishBlocks = 32;
+// A CTA owns 128 consecutive blocks.  The per-CTA (max, sum-exp) pairs are first staged in shared
+// memory with independent coalesced loads and merged there, one thread per row.  Then thread
+// (lgs, bl) sums the rows of heads lgs, lgs + 8, ... for blocks bl, bl + 32, bl + 64, bl + 96
+// (independent coalesced loads), and the 8 partial sums are added in a fixed order.
+constexpr int kFinishBlocks = 128;
 __global__ void __launch_bounds__(256)
 score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__ partials,
                     const int32_t* __restrict__ nblocks_dev, int session_first, int LG, int rows, int rows_pad,
-                    int nb_pad, int n_parts, float inv_LH, float* __restrict__ scores, int scores_stride) {
-    extern __shared__ float2 rowstat[];   // [LG * rows] : (max, 1/Z)
+                    int nb_pad, int n_parts, float inv_LH, float* __restrict__ scores, int scores_stride, int stage_parts) {
+    extern __shared__ float2 fin_smem[];  // rowstat [LG * rows] : (max, 1/Z); then staged partials [LG * rows][n_parts]
+    float2* rowstat = fin_smem;
+    float2* staged = fin_smem + LG * rows;
     __shared__ float red[8][kFinishBlocks];
     const int s = blockIdx.y;
     const int NB = nblocks_dev[session_first + s];
     if ((int)(blockIdx.x * kFinishBlocks) >= NB) return;
-    for (int i = threadIdx.x; i < LG * rows; i += blockDim.x) {
+    const int n_rows = LG * rows;
+    if (stage_parts) {
+        // warp w copies rows w, w + 8, ...; lane c copies pair c: independent loads, several rows in flight
+        const int wid = threadIdx.x >> 5, ln = threadIdx.x & 31;
+#pragma unroll 8
+        for (int row = wid; row < n_rows; row += 8) {
+            const int lg = row / rows, j = row % rows;
+            const float2* src = partials + (((size_t)s * LG + lg) * rows_pad + j) * n_parts;
+            for (int c = ln; c < n_parts; c += 32) staged[row * n_parts + c] = src[c];
+        }
+        __syncthreads();
+    }
+    for (int i = threadIdx.x; i < n_rows; i += blockDim.x) {
         const int lg = i / rows, j = i % rows;
-        const float2* p = partials + (((size_t)s * LG + lg) * rows_pad + j) * n_parts;
+        const float2* p = stage_parts ? staged + (size_t)i * n_parts : partials + (((size_t)s * LG + lg) * rows_pad + j) * n_parts;
         float mx = -INFINITY;
         for (int c = 0; c < n_parts; ++c) mx = fmaxf(mx, p[c].x);
         float z = 0.0f;
@@ -243,29 +408,57 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
         rowstat[i] = make_float2(mx, 1.0f / z);
     }
     __syncthreads();
-    const int bl = threadIdx.x & (kFinishBlocks - 1), lgs = threadIdx.x / kFinishBlocks;
-    const int b = blockIdx.x * kFinishBlocks + bl;
-    float part = 0.0f;
-    if (b < NB) {
-        for (int lg = lgs; lg < LG; lg += 8) {
-            const float* base = logits + (((size_t)s * LG + lg) * rows_pad) * (size_t)nb_pad + b;
-            float sub = 0.0f;
-#pragma unroll 16
-            for (int j = 0; j < rows; ++j) {
-                const float2 st = rowstat[lg * rows + j];
-                sub += exp2f(base[(size_t)j * nb_pad] - st.x) * st.y;
-            }
-            part += sub;
+    const int bl = threadIdx.x & 31, lgs = threadIdx.x >> 5;
+    const int b0 = blockIdx.x * kFinishBlocks + bl;
+    float part[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    for (int lg = lgs; lg < LG; lg += 8) {
+        const float* base = logits + (((size_t)s * LG + lg) * rows_pad) * (size_t)nb_pad + b0;
+        float sub[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 8
+        for (int j = 0; j < rows; ++j) {
+            const float2 st = rowstat[lg * rows + j];
+            const float* rp = base + (size_t)j * nb_pad;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (b0 + 32 * u < NB) sub[u] += exp2f(rp[32 * u] - st.x) * st.y;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) part[u] += sub[u];
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) red[lgs][bl + 32 * u] = part[u];
+    __syncthreads();
+    if (threadIdx.x < kFinishBlocks) {
+        const int b = blockIdx.x * kFinishBlocks + threadIdx.x;
+        if (b < NB) {
+            float total = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) total += red[i][threadIdx.x];
+            scores[(size_t)s * scores_stride + b] = total * inv_LH;
         }
     }
-    red[lgs][bl] = part;
-    __syncthreads();
-    if (lgs == 0 && b < NB) {
-        float total = 0.0f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) total += red[i][bl];
-        scores[(size_t)s * scores_stride + b] = total * inv_LH;
+}
+
+int g_score_mode = 1;   // 1: tensor-core dot products (default), 0: fp32 ALU + warp-shuffle kernel
+
+// index [max_sessions * L * G * max_bps rows][128] bf16 as a 2-D tensor; box = 64 dims x 128 rows, 128-byte swizzle
+static bool make_score_index_map(CUtensorMap* map, const kvmem_pool& p) {
+    static PFN_cuTensorMapEncodeTiled_v12000 enc = nullptr;
+    if (!enc) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return false;
+        enc = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
     }
+    const Geometry& g = p.geo;
+    cuuint64_t dims[2] = {128, (cuuint64_t)g.max_sessions * g.L * g.G * g.max_bps};
+    cuuint64_t strides[1] = {256};
+    cuuint32_t box[2] = {64, (cuuint32_t)kChunk};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.index, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q,
@@ -283,6 +476,20 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     const size_t smem = (size_t)kScoreStages * kChunk * 256;
     dim3 grid((unsigned)n_parts, (unsigned)LG, (unsigned)n_sessions);
     cudaError_t e;
+    const long long index_rows = (long long)g.max_sessions * g.L * g.G * g.max_bps;
+    if (g_score_mode == 1 && index_rows <= 0x7fffffffll) {     // TMA row coordinates are 32-bit
+        CUtensorMap map_idx;
+        if (!make_score_index_map(&map_idx, p)) return cudaErrorInvalidValue;
+        static bool attr_done = false;
+        if (!attr_done) {
+            e = cudaFuncSetAttribute(score_logits_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem + 1024));
+            if (e != cudaSuccess) return e;
+            attr_done = true;
+        }
+        score_logits_mma_kernel<<<grid, kScoreThreads, smem + 1024, st>>>(
+            map_idx, q, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, ws.logits, ws.partials, ws.rows,
+            ws.rows_pad, ws.nb_pad, n_parts, scale_log2e, p.status_dev);
+    } else {
 #define KVMEM_SCORE_LAUNCH(RP)                                                                                         \
     do {                                                                                                               \
         static bool attr_done = false;                                                                                 \
@@ -295,13 +502,17 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
             q, p.index, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, p.lay.index_elems_per_session,      \
             ws.logits, ws.partials, ws.rows, ws.rows_pad, ws.nb_pad, n_parts, scale_log2e, p.status_dev);              \
     } while (0)
-    if (ws.rows <= 4) KVMEM_SCORE_LAUNCH(4);
-    else if (ws.rows <= 8) KVMEM_SCORE_LAUNCH(8);
-    else KVMEM_SCORE_LAUNCH(16);
+        if (ws.rows <= 4) KVMEM_SCORE_LAUNCH(4);
+        else if (ws.rows <= 8) KVMEM_SCORE_LAUNCH(8);
+        else KVMEM_SCORE_LAUNCH(16);
 #undef KVMEM_SCORE_LAUNCH
+    }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const size_t fsmem = (size_t)LG * ws.rows * sizeof(float2);
+    size_t fsmem = (size_t)LG * ws.rows * sizeof(float2);
+    const size_t stage_bytes = fsmem * n_parts;
+    const int stage_parts = fsmem + stage_bytes <= 96 * 1024 ? 1 : 0;       // stage the pairs when they fit
+    if (stage_parts) fsmem += stage_bytes;
     if (fsmem > 48 * 1024) {
         e = cudaFuncSetAttribute(score_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsmem);
         if (e != cudaSuccess) return e;
@@ -309,7 +520,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     dim3 fgrid((unsigned)((max_nb + kFinishBlocks - 1) / kFinishBlocks), (unsigned)n_sessions);
     score_finish_kernel<<<fgrid, 256, fsmem, st>>>(ws.logits, ws.partials, p.nblocks_dev, session_first, LG, ws.rows,
                                                    ws.rows_pad, ws.nb_pad, n_parts, 1.0f / (float)(g.L * g.H),
-                                                   scores, scores_stride);
+                                                   scores, scores_stride, stage_parts);
     return cudaGetLastError();
 }
 

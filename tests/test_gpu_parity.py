@@ -92,11 +92,12 @@ def test_index_and_block_table_bit_exact(spec):
 # ------------------------------------------------------------------ whole step on small workspaces
 
 @pytest.mark.parametrize("M", [1, 2, 4])
-@pytest.mark.parametrize("gather_mode", [1, 0])
-def test_step_matches_oracle_small(M, gather_mode):
+@pytest.mark.parametrize("gather_mode,score_mode", [(1, 1), (0, 0)])
+def test_step_matches_oracle_small(M, gather_mode, score_mode):
     from paper_2609_04852_b200 import set_option
     spec = SMALL.with_(n_q_tokens=M)
     set_option("gather_mode", gather_mode)
+    set_option("score_mode", score_mode)
     try:
         pool = fill_pool(spec)
         osess = fill_oracle(spec)[0]
@@ -109,6 +110,25 @@ def test_step_matches_oracle_small(M, gather_mode):
             _compare_view_and_attention(spec, got, 0, same)
     finally:
         set_option("gather_mode", 1)
+        set_option("score_mode", 1)
+
+
+@pytest.mark.parametrize("M,score_mode", [(8, 1), (8, 0), (16, 1), (5, 0)])
+def test_scoring_with_more_than_sixteen_rows_per_kv_head(M, score_mode):
+    # M * 4 rows per KV head > 16: the decode scorer walks the rows in passes of 16
+    from paper_2609_04852_b200 import set_option
+    spec = SMALL.with_(n_q_tokens=M, n_blocks=333)
+    set_option("score_mode", score_mode)
+    try:
+        pool = fill_pool(spec)
+        osess = fill_oracle(spec)[0]
+        q, qb = queries(spec)
+        got = _run_step(pool, spec, q.cuda(), _params(budget_blocks=spec.budget_blocks), spec.budget_blocks, attend=False)
+        R, _ = orc.block_scores(qb[0], osess.idx, spec.n_blocks)
+        check_scores(got["scores"][0], R, M)
+        check_selection(got["sel"][0, : int(got["n_sel"][0])], R, orc.select(R, 64, spec.budget_blocks, 1 << 30))
+    finally:
+        set_option("score_mode", 1)
 
 
 def test_gap_forced_selection_is_identical_and_recovers_planted_blocks():
@@ -179,6 +199,23 @@ def test_duplicate_blocks_tie_break_by_lower_id():
     got = _run_step(pool, spec.with_(n_blocks=40), q.cuda(), _params(budget_blocks=7), 7)
     assert got["sel"][0, :7].tolist() == list(range(7))
     assert np.all(got["scores"][0, :40] == got["scores"][0, 0])
+
+
+def test_long_session_takes_the_general_top_k_path():
+    # more than 16,384 blocks: the selector re-reads the scores from global memory in every pass
+    spec = CONFIGS["tiny"].with_(name="long", n_blocks=16384 + 517, block_tokens=16, n_planted=40, budget_blocks=300)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    q, qb = queries(spec)
+    for budget in (300, 40):
+        got = _run_step(pool, spec, q.cuda(), _params(budget_blocks=budget), budget, attend=False)
+        R, _ = orc.block_scores(qb[0], osess.idx, spec.n_blocks)
+        check_scores(got["scores"][0], R, spec.n_q_tokens)
+        sel_gpu = got["sel"][0, : int(got["n_sel"][0])]
+        check_selection(sel_gpu, R, orc.select(R, spec.block_tokens, budget, 1 << 30))
+        vK, vV = orc.gather(osess.repo, osess.table, np.ascontiguousarray(sel_gpu), budget * spec.block_tokens)
+        T = len(sel_gpu) * spec.block_tokens
+        assert np.array_equal(bits(got["view"].k[0])[:, :, :T], vK[:, :, :T])
 
 
 # ------------------------------------------------------------------ fused view assembly + attention
