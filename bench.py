@@ -185,7 +185,11 @@ def run_native(args):
         pool.select(q, prm, sel, n_sel)
         if ev is not None:
             ev[0].record(stream)
-        if fused:
+        if args.paged:
+            pool.paged_attend(q, sel, n_sel, out, lse)                  # copy-free view: no materialisation at all
+            if ev is not None:
+                ev[1].record(stream)
+        elif fused:
             pool.materialize_attend(q, sel, n_sel, view, out, lse)      # one pass: view written while attended
             if ev is not None:
                 ev[1].record(stream)
@@ -287,6 +291,8 @@ def run_native(args):
         gather_gbs = ns * ab["gather"] / gather_s / 1e9
         # fused: every view byte is read once (from the pages) and written once; separate calls read it a second time
         step_bytes = ns * (ab["total"] - (ab["attend"] if fused else 0))
+        if args.paged:
+            step_bytes = ns * (ab["index"] + ab["attend"])
         step_gbs = world * K * step_bytes / (total_ms * 1e-3) / 1e9 / world      # per GPU
         rows = ns * M * spec.n_layers * spec.n_q_heads
         line = {
@@ -300,7 +306,8 @@ def run_native(args):
                        "l2": "flushed between steps (256 MiB write)" if flush is not None else
                              "no flush: every step streams far more than the 126 MB L2",
                        "parallelism": f"{world} independent session replica(s), one per GPU",
-                       "calls": "kvmem_select + kvmem_materialize_attend" if fused else
+                       "calls": "kvmem_select + kvmem_paged_attend (NO materialize: copy-free view variant)" if args.paged else
+                                "kvmem_select + kvmem_materialize_attend" if fused else
                                 "kvmem_select + kvmem_materialize" + (" + kvmem_view_attend" if spec.attend else "")},
             "e2e": {"value": whole_job_rate(Ke, world, e2e_ms), "unit": UNIT, "steps": Ke,
                     "h2d_bytes_per_step": rows * spec.head_dim * 2,
@@ -315,7 +322,8 @@ def run_native(args):
                          "algorithmic_bytes_per_launch": ns * ab["gather"], "avg_launch_ms": gather_s * 1e3,
                          "traffic": None if fused else GATHER_TRAFFIC.get(base.name)},
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes,
-                         "accounting": "index + view read + view write (fused pass)" if fused else
+                         "accounting": "index + one read of the selected pages (copy-free view, nothing materialised)" if args.paged else
+                                       "index + view read + view write (fused pass)" if fused else
                                        "index + gather read/write + attend read (separate calls)",
                          "bytes_if_separate_calls": ns * ab["total"], "achieved_gbs": step_gbs,
                          "frac_of_peak": step_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
@@ -448,6 +456,8 @@ def main():
     ap.add_argument("--workload", choices=sorted(CONFIGS), default="1m")
     ap.add_argument("--blocks", type=int, default=0, help="shrink the history to this many blocks (profiling)")
     ap.add_argument("--flush-l2", action="store_true", help="write 256 MiB between steps (for workloads near L2 size)")
+    ap.add_argument("--paged", action="store_true",
+                    help="copy-free execution view: kvmem_select + kvmem_paged_attend (no view is materialised; not the headline step)")
     ap.add_argument("--unfused", action="store_true", help="separate kvmem_materialize and kvmem_view_attend calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)

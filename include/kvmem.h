@@ -177,6 +177,17 @@ int kvmem_materialize_attend(kvmem_pool_t* pool, int32_t session_first, int32_t 
                              int32_t view_cap_tokens, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
                              void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
+/* Copy-free execution view (Sec. 4.4: the view as a page table over non-contiguous physical pages;
+ * Sec. 5.3 "Copy-free execution-view assembly"): GQA decode attention straight over the selected
+ * blocks' pages, in the order of sel_ids, through the block table.  No contiguous view is written.
+ * out and lse equal kvmem_view_attend's on the view kvmem_materialize would build from the same ids
+ * (same tiles, same order, same arithmetic).  HBM traffic: one read per view byte.
+ * Arguments as in kvmem_materialize_attend, without the view buffers. */
+int kvmem_paged_attend(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
+                       int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
+                       const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
+                       void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
 /* kvmem_view_attend for callers that cannot allocate device memory.  (The paper has no counterpart.)
  * Who needs it: a serving process that gave all of HBM to its KV pool at start-up and runs with
  * its allocator frozen, a plug-in that only ever sees the buffers of one request, or a latency path

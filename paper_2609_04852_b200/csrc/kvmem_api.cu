@@ -431,6 +431,37 @@ int kvmem_materialize_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_s
     return KVMEM_OK;
 }
 
+int kvmem_paged_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                       const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, float scale, float* out, float* lse,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!q || !sel_ids || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(workspace, 256) || !aligned(out, 16)) {
+        set_error("kvmem_paged_attend: null or misaligned pointer");
+        return KVMEM_E_INVALID;
+    }
+    if (n_q_tokens < 1 || sel_stride < 1) { set_error("n_q_tokens and sel_stride must be positive"); return KVMEM_E_INVALID; }
+    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
+        set_error("attention kernel is built for head_dim 128 and 64-token blocks");
+        return KVMEM_E_UNSUPPORTED;
+    }
+    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
+    if ((int64_t)p->cfg.max_blocks * 2 * p->cfg.n_layers * p->cfg.n_kv_heads * p->cfg.block_tokens > 0x7fffffffll) {
+        set_error("page pool too large for 32-bit TMA row coordinates");
+        return KVMEM_E_UNSUPPORTED;
+    }
+    AttendPlan plan = plan_attend(p->cfg, n_sessions, n_q_tokens, p->sm_count);
+    if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
+    // the "view" is only virtual here: its length bound is sel_stride blocks
+    const int64_t cap_tokens = (int64_t)sel_stride * p->cfg.block_tokens;
+    if (cap_tokens > 0x7fffffffll) { set_error("sel_stride too large"); return KVMEM_E_INVALID; }
+    cudaError_t e = launch_attend(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, nullptr, nullptr, (int)cap_tokens, n_sel,
+                                  scale, out, lse, workspace, (cudaStream_t)stream, sel_ids, sel_stride, session_first);
+    if (e != cudaSuccess) return cuda_fail("paged attention kernel launch", e);
+    return KVMEM_OK;
+}
+
 int kvmem_get_index(kvmem_pool_t* p, int32_t session, const void** index, int32_t* n_blocks) {
     if (!pool_ok(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;

@@ -73,15 +73,19 @@ static int choose_splits(int heads, int max_tiles, int sms) {
     return best;
 }
 
-// FUSED = false: tiles are read from the materialised view.
-// FUSED = true : tiles are read from the page pool through the block table (what the gather reads), one
-//                extra warp stores every tile into the view with TMA while the consumers attend over it,
-//                so the view is assembled and attended in one pass: 1 read + 1 write per view byte
-//                instead of 2 reads + 1 write.
-template <bool FUSED>
-__global__ void __launch_bounds__(kAttThreads + (FUSED ? 32 : 0), 1)
+// MODE 0: tiles are read from the materialised view.
+// MODE 1: tiles are read from the page pool through the block table (what the gather reads), one
+//         extra warp stores every tile into the view with TMA while the consumers attend over it,
+//         so the view is assembled and attended in one pass: 1 read + 1 write per view byte
+//         instead of 2 reads + 1 write.
+// MODE 2: copy-free execution view (Sec. 5.3 "Copy-free execution-view assembly"): tiles are read from
+//         the pages through the block table and attended over; no contiguous view is written.
+template <int MODE>
+__global__ void __launch_bounds__(kAttThreads + (MODE == 1 ? 32 : 0), 1)
 attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_pages, AttendArgs a) {
+    constexpr bool FUSED = MODE == 1;      // a view-writer warp shares every stage with the consumers
+    constexpr bool PAGED = MODE != 0;      // the producer reads pages through the block table
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages];
     __shared__ float merge_m[kAttConsumers][kRowsPad], merge_l[kAttConsumers][kRowsPad];
@@ -112,7 +116,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 
     if (warp == kAttConsumers) {
         // ---------------- producer ----------------
-        if (!FUSED) {
+        if (!PAGED) {
             if (lane == 0 && n_tiles > 0) {
                 ptx::prefetch_tensormap(&map_k);
                 ptx::prefetch_tensormap(&map_v);
@@ -414,19 +418,22 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     const Geometry& g = p.geo;
     const int LG = g.L * g.G, heads = n_sessions * LG;
     const bool fused = sel_ids != nullptr;
+    const bool paged_only = fused && view_k == nullptr;     // copy-free: attend straight over the pages
     CUtensorMap map_k, map_v, map_pages;
-    if (!make_view_map(&map_k, view_k, heads, view_cap_tokens) || !make_view_map(&map_v, view_v, heads, view_cap_tokens))
+    if (fused && !make_pages_map(&map_pages, p)) return cudaErrorInvalidValue;
+    if (paged_only) {
+        map_k = map_pages; map_v = map_pages;               // unused by this mode
+    } else if (!make_view_map(&map_k, view_k, heads, view_cap_tokens) || !make_view_map(&map_v, view_v, heads, view_cap_tokens)) {
         return cudaErrorInvalidValue;
-    if (fused) {
-        if (!make_pages_map(&map_pages, p)) return cudaErrorInvalidValue;
-    } else {
-        map_pages = map_k;
     }
+    if (!fused) map_pages = map_k;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attend_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        cudaError_t e = cudaFuncSetAttribute(attend_split_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attend_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+            e = cudaFuncSetAttribute(attend_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attend_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -444,10 +451,12 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     a.sel_ids = sel_ids; a.tables = p.tables; a.nblocks_dev = p.nblocks_dev;
     a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
-    if (fused)
-        attend_split_kernel<true><<<grid, kAttThreads + 32, kAttSmem, st>>>(map_k, map_v, map_pages, a);
+    if (paged_only)
+        attend_split_kernel<2><<<grid, kAttThreads, kAttSmem, st>>>(map_k, map_v, map_pages, a);
+    else if (fused)
+        attend_split_kernel<1><<<grid, kAttThreads + 32, kAttSmem, st>>>(map_k, map_v, map_pages, a);
     else
-        attend_split_kernel<false><<<grid, kAttThreads, kAttSmem, st>>>(map_k, map_v, map_pages, a);
+        attend_split_kernel<0><<<grid, kAttThreads, kAttSmem, st>>>(map_k, map_v, map_pages, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     attend_merge_kernel<<<dim3((unsigned)a.rows, (unsigned)heads), kD, 0, st>>>(a.part_o, a.part_ml, out, lse, M, g.L, g.H, g.G,

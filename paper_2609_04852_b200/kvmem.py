@@ -72,6 +72,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_device_status": (C.c_int, [vp, C.POINTER(i32), vp]),
         "kvmem_set_option": (C.c_int, [C.c_char_p, i32]),
         "kvmem_materialize_attend": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp]),
+        "kvmem_paged_attend": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
         "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
         "kvmem_recall_step_host": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, i32, f32, vp, vp,
@@ -90,7 +91,8 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_session_reset", "kvmem_session_blocks", "kvmem_append_blocks", "kvmem_select",
             "kvmem_materialize", "kvmem_view_attend", "kvmem_get_index", "kvmem_get_block_table",
             "kvmem_device_status", "kvmem_set_option", "kvmem_step_staging_bytes", "kvmem_recall_step_host",
-            "kvmem_view_attend_static", "kvmem_materialize_attend")
+            "kvmem_view_attend_static", "kvmem_materialize_attend",
+            "kvmem_paged_attend")
 
 
 def _check(status: int) -> None:
@@ -234,6 +236,16 @@ class Pool:
                                                  _dev(view.k, torch.bfloat16), _dev(view.v, torch.bfloat16),
                                                  view.cap_tokens, scale, _dev(out, torch.float32),
                                                  _dev(lse, torch.float32), ws.data_ptr(), ws.numel(), _stream()))
+
+    def paged_attend(self, q: torch.Tensor, sel_ids: torch.Tensor, n_sel: torch.Tensor, out: torch.Tensor,
+                     lse: torch.Tensor, scale: float = 0.0, session_first: int = 0) -> None:
+        """Copy-free execution view: attention straight over the selected blocks' pages (no view written)."""
+        ns, M = q.shape[0], q.shape[1]
+        ws = self.attend_workspace(ns, M)
+        _check(self.lib.kvmem_paged_attend(self.handle, session_first, ns, _dev(q, torch.bfloat16), M,
+                                           _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
+                                           scale, _dev(out, torch.float32), _dev(lse, torch.float32),
+                                           ws.data_ptr(), ws.numel(), _stream()))
 
     def view_attend_static(self, q: torch.Tensor, view: View, n_sel: torch.Tensor, out: torch.Tensor,
                            lse: torch.Tensor, scale: float = 0.0) -> None:

@@ -243,6 +243,11 @@ def test_fused_materialize_attend_equals_separate_calls_and_oracle(n_sessions, M
     assert pool.device_status() == 0
     assert torch.equal(view_a.k, view_b.k) and torch.equal(view_a.v, view_b.v), "fused view differs from the gathered view"
     assert torch.equal(out_a, out_b) and torch.equal(lse_a, lse_b), "same tiles, same order: results must be identical"
+    out_c, lse_c = pool.new_outputs(n_sessions, M)            # copy-free view: attention straight over the pages
+    pool.paged_attend(qd, sel, n_sel, out_c, lse_c)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    assert torch.equal(out_a, out_c) and torch.equal(lse_a, lse_c), "paged attention differs from attention over the view"
     for s in range(n_sessions):
         ids = sel[s, : int(n_sel[s])].cpu().numpy()
         vK, vV = orc.gather(osess[s].repo, osess[s].table, np.ascontiguousarray(ids), budget * 64)
