@@ -288,7 +288,8 @@ def run_native(args):
         ab = algorithmic_bytes(spec, k)
         med = statistics.median
         gather_s = (sum(gat_ms) / K) * 1e-3
-        gather_gbs = ns * ab["gather"] / gather_s / 1e9
+        dom_bytes = ns * (ab["attend"] if args.paged else ab["gather"])    # paged: one read of the selected pages
+        gather_gbs = dom_bytes / gather_s / 1e9
         # fused: every view byte is read once (from the pages) and written once; separate calls read it a second time
         step_bytes = ns * (ab["total"] - (ab["attend"] if fused else 0))
         if args.paged:
@@ -315,11 +316,12 @@ def run_native(args):
                     "api": "kvmem_recall_step_host (pinned host query in, host O and LSE out, synchronous)"},
             "gpu_launches": K * (KERNELS_PER_STEP - (1 if fused else 0)),
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<true> + merge (kvmem_materialize_attend: view written while attended)"
+            "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<2> + merge (kvmem_paged_attend)" if args.paged else
+                                                   "attend_split_kernel<1> + merge (kvmem_materialize_attend: view written while attended)"
                                                    if fused else "gather_bulk_kernel (kvmem_materialize)",
                          "achieved": gather_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gather_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
-                         "algorithmic_bytes_per_launch": ns * ab["gather"], "avg_launch_ms": gather_s * 1e3,
+                         "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": gather_s * 1e3,
                          "traffic": None if fused else GATHER_TRAFFIC.get(base.name)},
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes,
                          "accounting": "index + one read of the selected pages (copy-free view, nothing materialised)" if args.paged else
