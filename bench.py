@@ -59,6 +59,8 @@ def measured_tensor_peak():
 # dram__bytes_read.sum + dram__bytes_write.sum of one gather launch, from the ncu capture summarised in
 # profiles/dram_traffic_1m.md (1M workload)
 GATHER_TRAFFIC = {"1m": 2099369984}
+# the same for one launch of the fused pass (attend_split_kernel<1>)
+FUSED_TRAFFIC = {"1m": 2101969664}
 
 
 def algorithmic_bytes(spec, k):
@@ -322,7 +324,7 @@ def run_native(args):
                          "achieved": gather_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gather_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": gather_s * 1e3,
-                         "traffic": None if fused else GATHER_TRAFFIC.get(base.name)},
+                         "traffic": None if args.paged else FUSED_TRAFFIC.get(base.name) if fused else GATHER_TRAFFIC.get(base.name)},
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes,
                          "accounting": "index + one read of the selected pages (copy-free view, nothing materialised)" if args.paged else
                                        "index + view read + view write (fused pass)" if fused else
