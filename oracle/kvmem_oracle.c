@@ -276,3 +276,77 @@ int kvo_threads(void) {
 #endif
     return n;
 }
+
+/* =======================================================================================
+ * Position-consistent materialisation (Sec. 4.3 "Mean-K Retrieval-Index Construction":
+ * positional encoding is removed before indexing and from the query; Sec. 4.4: RoPE is
+ * applied to raw K at the block's assigned compact position, V is copied unchanged, with
+ * precomputed sine/cosine tables).
+ *
+ * Readings (the paper names RoPE but prints no formula): rotate-half pairing (i, i + d/2),
+ * frequency of pair i = theta^(-2i/d), angle = position * frequency.  The table holds
+ * cos and sin of the fp64 angle rounded once to fp32.  A rotated bf16 element is a
+ * quantised code, so its arithmetic is fixed: four fp32 products and two fp32 sums (no fused
+ * multiply-add), one round-to-nearest-even to bf16; the CUDA kernels do the same.
+ */
+
+/* tab[p][i] = (cos, sin) of p * theta^(-2i/d) as fp32 pairs; tab is [n_pos][d/2][2] */
+void kvo_rope_table(int64_t n_pos, int d, double theta, float* tab) {
+    const int half = d / 2;
+#pragma omp parallel for schedule(static)
+    for (int64_t p = 0; p < n_pos; ++p)
+        for (int i = 0; i < half; ++i) {
+            const double freq = pow(theta, -2.0 * (double)i / (double)d);
+            const double ang = (double)p * freq;
+            tab[(p * half + i) * 2 + 0] = (float)cos(ang);
+            tab[(p * half + i) * 2 + 1] = (float)sin(ang);
+        }
+}
+
+/* one vector of d elements at position p; inverse != 0 rotates by -p (removes the encoding) */
+static void kvo_rotate_vec(const bf16_t* x, bf16_t* y, int d, const float* tab_row, int inverse) {
+    const int half = d / 2;
+    for (int i = 0; i < half; ++i) {
+        const float a = bf16_to_f32(x[i]), b = bf16_to_f32(x[i + half]);
+        const float c = tab_row[2 * i], s = inverse ? -tab_row[2 * i + 1] : tab_row[2 * i + 1];
+        const float ac = a * c, bs = b * s, bc = b * c, as = a * s;
+        const float lo = ac - bs, hi = bc + as;
+        y[i] = f32_to_bf16_rne(lo);
+        y[i + half] = f32_to_bf16_rne(hi);
+    }
+}
+
+/* x, y: [n_rows][n_vec][d] bf16; every vector of row r is rotated by pos[r] (or by -pos[r]).
+ * Returns -1 if a position is outside the table. */
+int kvo_rope_rotate(const bf16_t* x, bf16_t* y, int64_t n_rows, int n_vec, int d, const int32_t* pos,
+                    const float* tab, int64_t n_pos, int inverse) {
+    for (int64_t r = 0; r < n_rows; ++r)
+        if (pos[r] < 0 || pos[r] >= n_pos) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < n_rows; ++r)
+        for (int v = 0; v < n_vec; ++v)
+            kvo_rotate_vec(x + (r * n_vec + v) * d, y + (r * n_vec + v) * d, d, tab + (size_t)pos[r] * (d / 2) * 2, inverse);
+    return 0;
+}
+
+/* Execution view with position-consistent keys: as kvo_gather, but the raw key of view token
+ * j*B + t is rotated to compact position first_pos + j*B + t; values are copied unchanged. */
+int kvo_gather_rope(const bf16_t* pagesK, const bf16_t* pagesV, const int32_t* table, const int32_t* sel,
+                    int64_t n_sel, int B, int L, int G, int d, bf16_t* viewK, bf16_t* viewV, int64_t cap_tokens,
+                    int64_t first_pos, const float* tab, int64_t n_pos) {
+    if (first_pos < 0 || first_pos + n_sel * B > n_pos) return -1;
+    const size_t page = (size_t)B * L * G * d;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n_sel; ++j) {
+        const size_t src = (size_t)table[sel[j]] * page;
+        for (int t = 0; t < B; ++t)
+            for (int l = 0; l < L; ++l)
+                for (int g = 0; g < G; ++g) {
+                    const size_t s = src + (((size_t)t * L + l) * G + g) * d;
+                    const size_t o = (((size_t)l * G + g) * cap_tokens + (size_t)j * B + t) * d;
+                    kvo_rotate_vec(pagesK + s, viewK + o, d, tab + (size_t)(first_pos + j * B + t) * (d / 2) * 2, 0);
+                    memcpy(viewV + o, pagesV + s, (size_t)d * sizeof(bf16_t));
+                }
+    }
+    return 0;
+}

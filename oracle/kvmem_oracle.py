@@ -4,12 +4,13 @@ Only ``tests/``, the smoke check and the benchmark's CPU-baseline leg may import
 It imports nothing from the CUDA package.  Arrays are NumPy; bf16 tensors travel as
 ``uint16`` bit patterns (``torch_tensor.view(torch.int16).numpy().view(np.uint16)``).
 
-Parity pins: every function here is pinned by ``tests/test_oracle_pins.py`` against closed
+Parity pins: every function here is pinned by ``tests/test_oracle_pins.py`` (and the RoPE
+functions by ``tests/test_oracle_rope_pins.py``) against closed
 forms, invariants of the equations, special cases that reduce to textbook softmax
 attention, and brute force on tiny inputs.  What stays *parity unpinned* is only what the
 paper never prints: the authors' sink/recent sizes, whether their candidate set excludes
-reserved blocks, their index element type, their query-head to KV-head mapping and their
-tie-break.  The readings taken are stated in ``kvmem_oracle.c``.
+reserved blocks, their index element type, their query-head to KV-head mapping, their
+tie-break, and their RoPE variant (pairing and base).  The readings taken are stated in ``kvmem_oracle.c``.
 """
 from __future__ import annotations
 
@@ -55,6 +56,12 @@ def lib():
         L.kvo_gather.restype = None
         L.kvo_attend.argtypes = [p, p, p, i64, i64, i32, i32, i32, i32, i32, dbl, p, p]
         L.kvo_attend.restype = None
+        L.kvo_rope_table.argtypes = [i64, i32, dbl, p]
+        L.kvo_rope_table.restype = None
+        L.kvo_rope_rotate.argtypes = [p, p, i64, i32, i32, p, p, i64, i32]
+        L.kvo_rope_rotate.restype = i32
+        L.kvo_gather_rope.argtypes = [p, p, p, p, i64, i32, i32, i32, i32, p, p, i64, i64, p, i64]
+        L.kvo_gather_rope.restype = i32
         L.kvo_threads.argtypes = []
         L.kvo_threads.restype = i32
         _lib = L
@@ -170,3 +177,40 @@ def attend(q: np.ndarray, viewK: np.ndarray, viewV: np.ndarray, T: int, scale: O
     lse = np.zeros((M, L, H), np.float32)
     lib().kvo_attend(_ptr(q), _ptr(viewK), _ptr(viewV), T, cap, M, L, H, G, d, float(scale), _ptr(out), _ptr(lse))
     return out, lse
+
+
+# ---- position-consistent materialisation (RoPE) ------------------------------------------------
+
+def rope_table(n_pos: int, d: int, theta: float) -> np.ndarray:
+    """fp32 [n_pos][d/2][2] = (cos, sin) of position * theta^(-2i/d)."""
+    tab = np.zeros((n_pos, d // 2, 2), np.float32)
+    lib().kvo_rope_table(n_pos, d, float(theta), _ptr(tab))
+    return tab
+
+
+def rope_rotate(x: np.ndarray, pos: np.ndarray, tab: np.ndarray, inverse: bool = False) -> np.ndarray:
+    """x uint16 [n_rows][n_vec][d]; every vector of row r rotated by pos[r] (inverse: by -pos[r])."""
+    _u16(x)
+    n_rows, n_vec, d = x.shape
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    assert pos.shape == (n_rows,) and tab.dtype == np.float32 and tab.shape[1] == d // 2
+    y = np.zeros_like(x)
+    rc = lib().kvo_rope_rotate(_ptr(x), _ptr(y), n_rows, n_vec, d, _ptr(pos), _ptr(tab), tab.shape[0], int(inverse))
+    if rc != 0:
+        raise ValueError("position outside the RoPE table")
+    return y
+
+
+def gather_rope(repo: Repository, table: np.ndarray, sel: np.ndarray, cap_tokens: int, first_pos: int,
+                tab: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Execution view whose keys carry RoPE at their compact positions first_pos + j*B + t."""
+    _, B, L, G, d = repo.pagesK.shape
+    assert table.dtype == np.int32 and sel.dtype == np.int32 and len(sel) * B <= cap_tokens
+    viewK = np.zeros((L, G, cap_tokens, d), np.uint16)
+    viewV = np.zeros((L, G, cap_tokens, d), np.uint16)
+    rc = lib().kvo_gather_rope(_ptr(repo.pagesK), _ptr(repo.pagesV), _ptr(np.ascontiguousarray(table)),
+                               _ptr(np.ascontiguousarray(sel)), len(sel), B, L, G, d, _ptr(viewK), _ptr(viewV),
+                               cap_tokens, first_pos, _ptr(tab), tab.shape[0])
+    if rc != 0:
+        raise ValueError("compact positions outside the RoPE table")
+    return viewK, viewV
