@@ -59,6 +59,11 @@ typedef struct {
     int32_t max_blocks;             /* physical pages in the pool                                      */
     int32_t max_blocks_per_session; /* rows of one session's block table and index                     */
     int32_t device;                 /* CUDA device ordinal                                             */
+    int32_t rope_max_positions;     /* 0: no rotary support.  Else the pool holds a cos/sin table for
+                                       positions [0, rope_max_positions): the native window, since every
+                                       token is encoded and re-encoded inside an execution view (8 bytes x
+                                       head_dim / 2 per position)                                      */
+    float rope_theta;               /* rotary base (e.g. 1e6); used when rope_max_positions > 0        */
 } kvmem_pool_config_t;
 
 /* Selection budget (Eq. "active_budget", Eq. "active_capacity" in Sec. 3.1; selector in
@@ -78,7 +83,7 @@ typedef struct {
 /* ---- pure host helpers (no CUDA call) -------------------------------------------------- */
 
 /* Bytes of DEVICE storage kvmem_pool_create needs for this geometry (0 if cfg is invalid).
- * Holds the K/V pages, the Mean-K index, the block tables and a status word. */
+ * Holds the K/V pages, the Mean-K index, the block tables, a status word and, if enabled, the rotary table. */
 size_t kvmem_pool_bytes(const kvmem_pool_config_t* cfg /*HOST*/);
 
 /* The budget clamp above for a session of n_blocks blocks; never negative. */
@@ -121,6 +126,34 @@ int32_t kvmem_session_blocks(const kvmem_pool_t* pool, int32_t session);
  * Errors: KVMEM_E_CAPACITY (session or pool full), KVMEM_E_STATE (page in use), KVMEM_E_INVALID. */
 int kvmem_append_blocks(kvmem_pool_t* pool, int32_t session, const void* k /*DEVICE*/, const void* v /*DEVICE*/,
                         int32_t n_blocks, const int32_t* phys_ids /*HOST*/, void* stream);
+
+/* ---- position-consistent keys (Sec. 4.3: positional encoding removed before indexing and from the
+ * query; Sec. 4.4: RoPE applied to raw K at the assigned compact position, V copied unchanged, with
+ * precomputed sine/cosine tables).  Needs rope_max_positions > 0.  Rotary variant: pairs (i, i + d/2),
+ * frequency theta^(-2i/d), table = fp32 cos/sin of the fp64 angle; a rotated element is four fp32
+ * products and two fp32 sums (no fused multiply-add), rounded once to bf16. ------------------------ */
+
+/* kvmem_append_blocks for keys that still carry RoPE: token t of new block i was encoded at position
+ * block_pos0[i] + t (its position in the execution window it was computed in).  The encoding is removed,
+ * the raw keys are stored in the pages and indexed; block_pos0 is kept in the block record.
+ *   block_pos0  HOST int32 [n_blocks]; every position must lie in [0, rope_max_positions) */
+int kvmem_append_blocks_rope(kvmem_pool_t* pool, int32_t session, const void* k_roped /*DEVICE*/, const void* v /*DEVICE*/,
+                             int32_t n_blocks, const int32_t* phys_ids /*HOST*/, const int32_t* block_pos0 /*HOST*/,
+                             void* stream);
+
+/* Rotate n_rows x n_vec vectors of head_dim elements: y[r][v] = RoPE(x[r][v], positions[r]), or the
+ * inverse rotation (inverse != 0), e.g. to bring the current query into the position-independent space
+ * the index lives in.  x, y DEVICE bf16 [n_rows][n_vec][head_dim] (may alias); positions DEVICE int32
+ * [n_rows].  Rows with a position outside the table are left unwritten and flagged in the status word. */
+int kvmem_rope_rotate(kvmem_pool_t* pool, const void* x /*DEVICE*/, void* y /*DEVICE*/, int64_t n_rows, int32_t n_vec,
+                      const int32_t* positions /*DEVICE*/, int32_t inverse, void* stream);
+
+/* kvmem_materialize with position-consistent keys: the key of view token j*B + t is the raw key rotated
+ * to compact position first_position + j*B + t; values are copied unchanged.
+ * first_position + budget * B must not exceed rope_max_positions (KVMEM_E_INVALID otherwise). */
+int kvmem_materialize_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids /*DEVICE*/,
+                           int32_t sel_stride, const int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/,
+                           void* view_v /*DEVICE*/, int32_t view_cap_tokens, int32_t first_position, void* stream);
 
 /* ---- the recall step ----------------------------------------------------------------------- */
 

@@ -1,5 +1,6 @@
 // C ABI of libkvmem_b200: argument checking, pool and session bookkeeping, launch sequencing.
 // Every step of the recall path runs in the kernels of the sibling files; nothing here computes.
+#include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
 #include <string.h>
@@ -33,6 +34,9 @@ bool config_valid(const kvmem_pool_config_t& c, const char** why) {
     if (c.max_blocks_per_session < 1 || c.max_blocks_per_session > c.max_blocks)
         return bad("max_blocks_per_session must be in [1, max_blocks]");
     if (c.device < 0) return bad("device must be a CUDA ordinal");
+    if (c.rope_max_positions < 0) return bad("rope_max_positions must be non-negative");
+    if (c.rope_max_positions > 0 && !(c.rope_theta > 1.0f)) return bad("rope_theta must exceed 1 when rotary support is on");
+    if (c.rope_max_positions > 0 && c.head_dim % 16 != 0) return bad("rotary support needs head_dim to be a multiple of 16");
     return true;
 }
 
@@ -52,6 +56,10 @@ Layout make_layout(const kvmem_pool_config_t& c) {
     off = align_up(off + (size_t)c.max_sessions * 4, 256);
     l.status_off = off;
     off = align_up(off + 256, 256);
+    l.pos0_off = off;
+    if (c.rope_max_positions > 0) off = align_up(off + (size_t)c.max_sessions * c.max_blocks_per_session * 4, 256);
+    l.rope_off = off;
+    if (c.rope_max_positions > 0) off = align_up(off + (size_t)c.rope_max_positions * (c.head_dim / 2) * sizeof(float2), 256);
     l.total = off;
     return l;
 }
@@ -166,7 +174,26 @@ int kvmem_pool_create(const kvmem_pool_config_t* cfg, void* storage, size_t byte
     p->page_used.assign(cfg->max_blocks, 0);
     p->free_hint = 0;
     p->sm_count = prop.multiProcessorCount;
-    e = cudaMemset(p->base + lay.tables_off, 0, lay.total - lay.tables_off);
+    p->pos0_dev = cfg->rope_max_positions > 0 ? (int32_t*)(p->base + lay.pos0_off) : nullptr;
+    p->rope_dev = cfg->rope_max_positions > 0 ? (float2*)(p->base + lay.rope_off) : nullptr;
+    e = cudaMemset(p->base + lay.tables_off, 0, lay.rope_off - lay.tables_off);
+    if (e == cudaSuccess && cfg->rope_max_positions > 0) {
+        // cos/sin of position * theta^(-2i/d): angle in fp64, one rounding to fp32 (built here, on the host)
+        const int half = cfg->head_dim / 2;
+        std::vector<double> freq(half);
+        for (int i = 0; i < half; ++i) freq[i] = pow((double)cfg->rope_theta, -2.0 * (double)i / (double)cfg->head_dim);
+        const int chunk = 4096;
+        std::vector<float2> rows((size_t)chunk * half);
+        for (int p0 = 0; e == cudaSuccess && p0 < cfg->rope_max_positions; p0 += chunk) {
+            const int n = std::min(chunk, cfg->rope_max_positions - p0);
+            for (int r = 0; r < n; ++r)
+                for (int i = 0; i < half; ++i) {
+                    const double ang = (double)(p0 + r) * freq[i];
+                    rows[(size_t)r * half + i] = make_float2((float)cos(ang), (float)sin(ang));
+                }
+            e = cudaMemcpy(p->rope_dev + (size_t)p0 * half, rows.data(), (size_t)n * half * sizeof(float2), cudaMemcpyHostToDevice);
+        }
+    }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete p; return cuda_fail("clearing pool metadata", e); }
     *out = p;
@@ -196,8 +223,8 @@ int32_t kvmem_session_blocks(const kvmem_pool_t* p, int32_t session) {
     return p->sess_blocks[session];
 }
 
-int kvmem_append_blocks(kvmem_pool_t* p, int32_t session, const void* k, const void* v, int32_t n_blocks,
-                        const int32_t* phys_ids, void* stream) {
+static int append_impl(kvmem_pool_t* p, int32_t session, const void* k, const void* v, int32_t n_blocks,
+                       const int32_t* phys_ids, const int32_t* block_pos0, void* stream) {
     if (!pool_ok(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;
     if (n_blocks < 0) { set_error("n_blocks is negative"); return KVMEM_E_INVALID; }
@@ -227,6 +254,15 @@ int kvmem_append_blocks(kvmem_pool_t* p, int32_t session, const void* k, const v
             if (!p->page_used[pg]) ids[got++] = pg;
         if (got < n_blocks) { set_error("pool has %d free pages, %d needed", got, n_blocks); return KVMEM_E_CAPACITY; }
     }
+    if (block_pos0) {
+        if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
+        for (int i = 0; i < n_blocks; ++i)
+            if (block_pos0[i] < 0 || (int64_t)block_pos0[i] + p->cfg.block_tokens > p->cfg.rope_max_positions) {
+                set_error("block %d: positions [%d, %d) outside the rotary table [0, %d)", i, block_pos0[i],
+                          block_pos0[i] + p->cfg.block_tokens, p->cfg.rope_max_positions);
+                return KVMEM_E_INVALID;
+            }
+    }
     cudaStream_t st = (cudaStream_t)stream;
     int32_t* table = p->tables + (size_t)session * p->cfg.max_blocks_per_session;
     cudaError_t e = cudaMemcpyAsync(table + have, ids.data(), (size_t)n_blocks * 4, cudaMemcpyHostToDevice, st);
@@ -234,11 +270,68 @@ int kvmem_append_blocks(kvmem_pool_t* p, int32_t session, const void* k, const v
     const int32_t total = have + n_blocks;
     e = cudaMemcpyAsync(p->nblocks_dev + session, &total, 4, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail("block count upload", e);
-    e = launch_append(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st);
+    if (block_pos0) {
+        e = cudaMemcpyAsync(p->pos0_dev + (size_t)session * p->cfg.max_blocks_per_session + have, block_pos0,
+                            (size_t)n_blocks * 4, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return cuda_fail("block position upload", e);
+    }
+    e = launch_append(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st, block_pos0 != nullptr);
     if (e != cudaSuccess) return cuda_fail("append kernel launch", e);
     for (int32_t pg : ids) { p->page_used[pg] = 1; p->sess_pages[session].push_back(pg); }
     if (!phys_ids) p->free_hint = ids.back() + 1;
     p->sess_blocks[session] = total;
+    return KVMEM_OK;
+}
+
+int kvmem_append_blocks(kvmem_pool_t* p, int32_t session, const void* k, const void* v, int32_t n_blocks,
+                        const int32_t* phys_ids, void* stream) {
+    return append_impl(p, session, k, v, n_blocks, phys_ids, nullptr, stream);
+}
+
+int kvmem_append_blocks_rope(kvmem_pool_t* p, int32_t session, const void* k_roped, const void* v, int32_t n_blocks,
+                             const int32_t* phys_ids, const int32_t* block_pos0, void* stream) {
+    if (!block_pos0) { set_error("block_pos0 is null"); return KVMEM_E_INVALID; }
+    return append_impl(p, session, k_roped, v, n_blocks, phys_ids, block_pos0, stream);
+}
+
+int kvmem_rope_rotate(kvmem_pool_t* p, const void* x, void* y, int64_t n_rows, int32_t n_vec, const int32_t* positions,
+                      int32_t inverse, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
+    if (!x || !y || !positions || !aligned(x, 16) || !aligned(y, 16) || n_rows < 0 || n_vec < 1) {
+        set_error("kvmem_rope_rotate: null or misaligned pointer, or bad sizes");
+        return KVMEM_E_INVALID;
+    }
+    if (n_rows == 0) return KVMEM_OK;
+    cudaError_t e = launch_rope_rotate(*p, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, n_rows, n_vec, positions, inverse,
+                                       (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("rotary kernel launch", e);
+    return KVMEM_OK;
+}
+
+int kvmem_materialize_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids,
+                           int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v, int32_t view_cap_tokens,
+                           int32_t first_position, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
+    if (!sel_ids || !n_sel || !view_k || !view_v || !aligned(view_k, 16) || !aligned(view_v, 16)) {
+        set_error("kvmem_materialize_rope: null or misaligned pointer");
+        return KVMEM_E_INVALID;
+    }
+    if (sel_stride < 1 || view_cap_tokens < p->cfg.block_tokens || view_cap_tokens % p->cfg.block_tokens != 0) {
+        set_error("view_cap_tokens must be a positive multiple of block_tokens and sel_stride positive");
+        return KVMEM_E_INVALID;
+    }
+    const int64_t last = (int64_t)first_position + std::min<int64_t>((int64_t)sel_stride * p->cfg.block_tokens, view_cap_tokens);
+    if (first_position < 0 || last > p->cfg.rope_max_positions) {
+        set_error("compact positions [%d, %lld) outside the rotary table [0, %d)", first_position, (long long)last,
+                  p->cfg.rope_max_positions);
+        return KVMEM_E_INVALID;
+    }
+    cudaError_t e = launch_gather_rope(*p, session_first, n_sessions, sel_ids, sel_stride, n_sel, (__nv_bfloat16*)view_k,
+                                       (__nv_bfloat16*)view_v, view_cap_tokens, first_position, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("rotary gather kernel launch", e);
     return KVMEM_OK;
 }
 

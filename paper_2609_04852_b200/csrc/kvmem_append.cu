@@ -14,7 +14,8 @@ __global__ void __launch_bounds__(256)
 append_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* __restrict__ v_in,
               __nv_bfloat16* __restrict__ pages, __nv_bfloat16* __restrict__ index_sess,
               const int32_t* __restrict__ table_sess, int32_t* __restrict__ status,
-              int b_first, int L, int G, int B, int d, int max_blocks, int max_bps, size_t page_elems) {
+              int b_first, int L, int G, int B, int d, int max_blocks, int max_bps, size_t page_elems,
+              const int32_t* __restrict__ pos0_sess, const float2* __restrict__ rope, int rope_positions) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __nv_bfloat16* tile = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [B][d]
 
@@ -39,10 +40,32 @@ append_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* __res
         const uint4 kk = *reinterpret_cast<const uint4*>(ksrc + (size_t)t * row_stride + j * 8);
         const uint4 vv = *reinterpret_cast<const uint4*>(vsrc + (size_t)t * row_stride + j * 8);
         *reinterpret_cast<uint4*>(tile + (size_t)t * d + j * 8) = kk;
-        *reinterpret_cast<uint4*>(kdst + (size_t)t * d + j * 8) = kk;
         *reinterpret_cast<uint4*>(vdst + (size_t)t * d + j * 8) = vv;
     }
     __syncthreads();
+    if (rope) {
+        // the keys still carry RoPE of positions pos0 + t: rotate back by the same angles (Sec. 4.3), so
+        // that the pages hold raw keys and the index is position-independent.  fp32 products and sums
+        // without fused multiply-add, one rounding to bf16: the defined arithmetic of a rotated element.
+        const int pos0 = pos0_sess[b_first + i];
+        const int half = d / 2;
+        for (int e = threadIdx.x; e < B * half; e += blockDim.x) {
+            const int t = e / half, x = e % half;
+            const int pos = pos0 + t;
+            if (pos < 0 || pos >= rope_positions) { atomicExch(status, (int)KVMEM_E_DEVICE_RANGE); continue; }
+            const float2 cs = rope[(size_t)pos * half + x];
+            const float a = __bfloat162float(tile[(size_t)t * d + x]), b = __bfloat162float(tile[(size_t)t * d + x + half]);
+            const float lo = __fadd_rn(__fmul_rn(a, cs.x), __fmul_rn(b, cs.y));     // inverse rotation: sin -> -sin
+            const float hi = __fsub_rn(__fmul_rn(b, cs.x), __fmul_rn(a, cs.y));
+            tile[(size_t)t * d + x] = __float2bfloat16_rn(lo);
+            tile[(size_t)t * d + x + half] = __float2bfloat16_rn(hi);
+        }
+        __syncthreads();
+    }
+    for (int c = threadIdx.x; c < n_chunks; c += blockDim.x) {
+        const int t = c / chunks_per_row, j = c % chunks_per_row;
+        *reinterpret_cast<uint4*>(kdst + (size_t)t * d + j * 8) = *reinterpret_cast<const uint4*>(tile + (size_t)t * d + j * 8);
+    }
 
     const float inv = 1.0f / (float)B;
     __nv_bfloat16* idx_row = index_sess + ((size_t)lg * max_bps + (size_t)(b_first + i)) * d;
@@ -54,7 +77,7 @@ append_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* __res
 }
 
 cudaError_t launch_append(const kvmem_pool& p, int session, int b_first, int n_blocks, const __nv_bfloat16* k,
-                          const __nv_bfloat16* v, cudaStream_t st) {
+                          const __nv_bfloat16* v, cudaStream_t st, bool derope) {
     const Geometry& g = p.geo;
     const size_t smem = (size_t)g.B * g.d * sizeof(__nv_bfloat16);
     if (smem > 48 * 1024) {
@@ -66,7 +89,9 @@ cudaError_t launch_append(const kvmem_pool& p, int session, int b_first, int n_b
     // gridDim.x is limited to 2^31-1 blocks and gridDim.y to 65535: L*G stays far below that
     dim3 grid((unsigned)n_blocks, (unsigned)(g.L * g.G));
     append_kernel<<<grid, 256, smem, st>>>(k, v, p.pages, index, table, p.status_dev, b_first, g.L, g.G, g.B, g.d,
-                                           g.max_blocks, g.max_bps, p.lay.page_elems);
+                                           g.max_blocks, g.max_bps, p.lay.page_elems,
+                                           derope ? p.pos0_dev + (size_t)session * g.max_bps : nullptr,
+                                           derope ? p.rope_dev : nullptr, p.cfg.rope_max_positions);
     return cudaGetLastError();
 }
 

@@ -21,8 +21,10 @@ constexpr uint64_t kWaitLimitNs = 1000ull * 1000 * 1000;  // ... or about one se
 //   tables  [max_sessions][max_blocks_per_session] int32 (logical -> physical page)
 //   nblocks [max_sessions] int32
 //   status  int32 (sticky device status word)
+//   pos0    [max_sessions][max_blocks_per_session] int32: original position of each block's first token (rotary pools)
+//   rope    [rope_max_positions][d/2] float2 (cos, sin)                                         (rotary pools)
 struct Layout {
-    size_t pages_off, index_off, tables_off, nblocks_off, status_off, total;
+    size_t pages_off, index_off, tables_off, nblocks_off, status_off, pos0_off, rope_off, total;
     size_t page_elems;  // bf16 elements per page
     size_t tile_elems;  // B * d
     size_t index_elems_per_session;
@@ -51,6 +53,8 @@ struct kvmem_pool {
     int32_t* tables;
     int32_t* nblocks_dev;
     int32_t* status_dev;
+    int32_t* pos0_dev;                  // null unless rope_max_positions > 0
+    float2* rope_dev;
     std::vector<int32_t> sess_blocks;               // host mirror of nblocks
     std::vector<std::vector<int32_t>> sess_pages;   // host mirror of tables
     std::vector<uint8_t> page_used;
@@ -72,7 +76,7 @@ extern int g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
 // All return cudaGetLastError() after the launch.
 
 cudaError_t launch_append(const kvmem_pool& p, int session, int b_first, int n_blocks, const __nv_bfloat16* k,
-                          const __nv_bfloat16* v, cudaStream_t st);
+                          const __nv_bfloat16* v, cudaStream_t st, bool derope = false);
 
 struct ScoreWorkspace {
     float* logits;     // [ns][L][G][rows_pad][nb_pad]
@@ -85,6 +89,13 @@ ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions
 
 cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q,
                                 int M, const ScoreWorkspace& ws, float* scores, int scores_stride, cudaStream_t st);
+
+// rotary position embedding (kvmem_rope.cu)
+cudaError_t launch_rope_rotate(const kvmem_pool& p, const __nv_bfloat16* x, __nv_bfloat16* y, long long n_rows, int n_vec,
+                               const int32_t* positions, int inverse, cudaStream_t st);
+cudaError_t launch_gather_rope(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids,
+                               int sel_stride, const int32_t* n_sel, __nv_bfloat16* view_k, __nv_bfloat16* view_v,
+                               int view_cap_tokens, int first_position, cudaStream_t st);
 
 // multi-token query chunks: tcgen05 two-pass contraction
 struct ChunkWorkspace {

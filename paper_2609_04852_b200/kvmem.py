@@ -28,7 +28,8 @@ class KvmemError(RuntimeError):
 
 class PoolConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "block_tokens",
-                                          "max_sessions", "max_blocks", "max_blocks_per_session", "device")]
+                                          "max_sessions", "max_blocks", "max_blocks_per_session", "device",
+                                          "rope_max_positions")] + [("rope_theta", C.c_float)]
 
 
 class SelectParams(C.Structure):
@@ -72,6 +73,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_device_status": (C.c_int, [vp, C.POINTER(i32), vp]),
         "kvmem_set_option": (C.c_int, [C.c_char_p, i32]),
         "kvmem_materialize_attend": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp]),
+        "kvmem_append_blocks_rope": (C.c_int, [vp, i32, vp, vp, i32, C.POINTER(i32), C.POINTER(i32), vp]),
+        "kvmem_rope_rotate": (C.c_int, [vp, vp, vp, C.c_int64, i32, vp, i32, vp]),
+        "kvmem_materialize_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, i32, vp]),
         "kvmem_paged_attend": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
         "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
@@ -92,7 +96,7 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_materialize", "kvmem_view_attend", "kvmem_get_index", "kvmem_get_block_table",
             "kvmem_device_status", "kvmem_set_option", "kvmem_step_staging_bytes", "kvmem_recall_step_host",
             "kvmem_view_attend_static", "kvmem_materialize_attend",
-            "kvmem_paged_attend")
+            "kvmem_paged_attend", "kvmem_append_blocks_rope", "kvmem_rope_rotate", "kvmem_materialize_rope")
 
 
 def _check(status: int) -> None:
@@ -132,10 +136,11 @@ class Pool:
     """A paged KV repository with its Mean-K index, living in one torch uint8 tensor."""
 
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, block_tokens: int,
-                 max_sessions: int, max_blocks: int, max_blocks_per_session: int, device: int = 0):
+                 max_sessions: int, max_blocks: int, max_blocks_per_session: int, device: int = 0,
+                 rope_max_positions: int = 0, rope_theta: float = 0.0):
         self.lib = load_library()
         self.cfg = PoolConfig(n_layers, n_q_heads, n_kv_heads, head_dim, block_tokens, max_sessions, max_blocks,
-                              max_blocks_per_session, device)
+                              max_blocks_per_session, device, rope_max_positions, rope_theta)
         nbytes = self.lib.kvmem_pool_bytes(C.byref(self.cfg))
         if nbytes == 0:
             raise KvmemError(E_INVALID, self.lib.kvmem_last_error().decode())
@@ -183,6 +188,40 @@ class Pool:
             ids = (C.c_int32 * n)(*[int(x) for x in phys_ids])
         _check(self.lib.kvmem_append_blocks(self.handle, session, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16),
                                             n, ids, _stream()))
+
+    # ---- position-consistent keys
+    def append_blocks_rope(self, session: int, k_roped: torch.Tensor, v: torch.Tensor, block_pos0: Sequence[int],
+                           phys_ids: Optional[Sequence[int]] = None) -> None:
+        """append_blocks for keys that carry RoPE: token t of block i was encoded at block_pos0[i] + t."""
+        c = self.cfg
+        per_block = c.block_tokens * c.n_layers * c.n_kv_heads * c.head_dim
+        if k_roped.numel() % per_block or k_roped.shape != v.shape:
+            raise KvmemError(E_INVALID, "k and v must hold whole blocks of identical shape")
+        n = k_roped.numel() // per_block
+        if len(block_pos0) != n or (phys_ids is not None and len(phys_ids) != n):
+            raise KvmemError(E_INVALID, "one position (and page id) per block")
+        ids = None if phys_ids is None else (C.c_int32 * n)(*[int(x) for x in phys_ids])
+        pos = (C.c_int32 * n)(*[int(x) for x in block_pos0])
+        _check(self.lib.kvmem_append_blocks_rope(self.handle, session, _dev(k_roped, torch.bfloat16),
+                                                 _dev(v, torch.bfloat16), n, ids, pos, _stream()))
+
+    def rope_rotate(self, x: torch.Tensor, positions: torch.Tensor, out: Optional[torch.Tensor] = None,
+                    inverse: bool = False) -> torch.Tensor:
+        """x bf16 [n_rows][n_vec][head_dim], positions int32 [n_rows] -> rotated copy (inverse: encoding removed)."""
+        if out is None:
+            out = torch.empty_like(x)
+        n_rows, n_vec = x.shape[0], x.numel() // (x.shape[0] * self.cfg.head_dim)
+        _check(self.lib.kvmem_rope_rotate(self.handle, _dev(x, torch.bfloat16), _dev(out, torch.bfloat16), n_rows, n_vec,
+                                          _dev(positions, torch.int32), int(inverse), _stream()))
+        return out
+
+    def materialize_rope(self, sel_ids: torch.Tensor, n_sel: torch.Tensor, view: View, first_position: int = 0,
+                         session_first: int = 0) -> None:
+        """materialize with keys rotated to their compact positions first_position + j*B + t; values copied."""
+        ns = n_sel.shape[0]
+        _check(self.lib.kvmem_materialize_rope(self.handle, session_first, ns, _dev(sel_ids, torch.int32),
+                                               sel_ids.shape[-1], _dev(n_sel, torch.int32), _dev(view.k, torch.bfloat16),
+                                               _dev(view.v, torch.bfloat16), view.cap_tokens, first_position, _stream()))
 
     # ---- the recall step
     def select_workspace(self, n_sessions: int, n_q_tokens: int) -> torch.Tensor:
