@@ -61,6 +61,8 @@ def measured_tensor_peak():
 GATHER_TRAFFIC = {"1m": 2099369984}
 # the same for one launch of the fused pass (attend_split_kernel<1>)
 FUSED_TRAFFIC = {"1m": 2101969664}
+# and of the rotating gather (gather_rope_kernel), profiles/dram_traffic_1m_rope_step.md
+ROPE_GATHER_TRAFFIC = {"1m": 2298386176}
 
 
 def algorithmic_bytes(spec, k):
@@ -128,16 +130,30 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- native arm
 
-def fill_pool(spec, device, seed_shift=0):
+ROPE_THETA = 1.0e6
+
+
+def rope_window(spec):
+    """Positions the rotary table must cover: the native window plus the step's query tokens."""
+    return spec.max_view_tokens + 64
+
+
+def fill_pool(spec, device, seed_shift=0, rope=False):
     from paper_2609_04852_b200 import Pool
     spec = spec.with_(seed=spec.seed + seed_shift)
     pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.block_tokens,
-                spec.n_sessions, spec.n_sessions * spec.n_blocks, spec.n_blocks, device.index)
+                spec.n_sessions, spec.n_sessions * spec.n_blocks, spec.n_blocks, device.index,
+                rope_window(spec) if rope else 0, ROPE_THETA if rope else 0.0)
     tables = page_table(spec)
+    B = spec.block_tokens
     for s in range(spec.n_sessions):
         for b0 in range(0, spec.n_blocks, 1024):
             b1 = min(spec.n_blocks, b0 + 1024)
             K, V = kv_blocks(spec, s, b0, b1, device)
+            if rope:    # the keys are taken as encoded at the positions they had inside their execution window
+                pos0 = [(b * B) % (spec.max_view_tokens - B) for b in range(b0, b1)]
+                pool.append_blocks_rope(s, K, V, pos0, tables[s, b0:b1].tolist())
+                continue
             pool.append_blocks(s, K, V, tables[s, b0:b1].tolist())
         torch.cuda.synchronize(device)
     return pool, spec
@@ -163,7 +179,7 @@ def run_native(args):
         f = args.blocks / base.n_blocks
         base = base.with_(name=f"{base.name}@{args.blocks}", n_blocks=args.blocks,
                           n_planted=max(1, int(base.n_planted * f)), budget_blocks=max(1, int(base.budget_blocks * f)))
-    pool, spec = fill_pool(base, device, seed_shift=1000 * rank)     # one independent replica per rank
+    pool, spec = fill_pool(base, device, seed_shift=1000 * rank, rope=args.rope)     # one independent replica per rank
     ns, M, B = spec.n_sessions, spec.n_q_tokens, spec.block_tokens
     prm = SelectParams(**select_params(spec))
     from paper_2609_04852_b200 import budget_blocks
@@ -180,10 +196,30 @@ def run_native(args):
     lse_pin = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device) if args.flush_l2 else None
     stream = torch.cuda.current_stream(device)
-    fused = spec.attend and not args.unfused
+    fused = spec.attend and not args.unfused and not args.rope
+
+    if args.rope:
+        if not spec.attend or spec.n_sessions != 1:
+            raise SystemExit("--rope is measured on the single-session attend workloads")
+        H, d = spec.n_q_heads, spec.head_dim
+        q_pos = torch.arange(k * B, k * B + M, dtype=torch.int32, device=device)     # the query sits right after the view
+        q_raw = torch.empty_like(q_dev[0])
 
     def step(i, ev=None):
         q = q_dev[i % len(q_dev)]
+        if args.rope:
+            # the model's query carries RoPE: remove it for retrieval (Sec. 4.3), keep it for attention
+            pool.rope_rotate(q.view(M, H, d), q_pos, out=q_raw.view(M, H, d), inverse=True)
+            pool.select(q_raw, prm, sel, n_sel)
+            if ev is not None:
+                ev[0].record(stream)
+            pool.materialize_rope(sel, n_sel, view, 0)
+            if ev is not None:
+                ev[1].record(stream)
+            pool.view_attend(q, view, n_sel, out, lse)
+            if ev is not None:
+                ev[2].record(stream)
+            return
         pool.select(q, prm, sel, n_sel)
         if ev is not None:
             ev[0].record(stream)
@@ -255,7 +291,16 @@ def run_native(args):
     q_stage = torch.empty_like(q_dev[0])
     sel_pin = torch.empty(sel.shape, dtype=torch.int32).pin_memory()
     for i in range(Ke):
-        if spec.attend:
+        if args.rope:   # same position-consistent step, query from pinned host memory, results back to the host
+            q_stage.copy_(q_pin[i % len(q_pin)], non_blocking=True)
+            pool.rope_rotate(q_stage.view(M, H, d), q_pos, out=q_raw.view(M, H, d), inverse=True)
+            pool.select(q_raw, prm, sel, n_sel)
+            pool.materialize_rope(sel, n_sel, view, 0)
+            pool.view_attend(q_stage, view, n_sel, out, lse)
+            out_pin.copy_(out, non_blocking=True)
+            lse_pin.copy_(lse, non_blocking=True)
+            torch.cuda.synchronize(device)
+        elif spec.attend:
             pool.recall_step_host(q_pin[i % len(q_pin)], prm, sel, n_sel, view, out_pin, lse_pin)
         else:       # chunked scoring has no attend stage: host query in, selected ids out
             q_stage.copy_(q_pin[i % len(q_pin)], non_blocking=True)
@@ -309,22 +354,25 @@ def run_native(args):
                        "l2": "flushed between steps (256 MiB write)" if flush is not None else
                              "no flush: every step streams far more than the 126 MB L2",
                        "parallelism": f"{world} independent session replica(s), one per GPU",
-                       "calls": "kvmem_select + kvmem_paged_attend (NO materialize: copy-free view variant)" if args.paged else
+                       "calls": "kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_rope + kvmem_view_attend" if args.rope else
+                                "kvmem_select + kvmem_paged_attend (NO materialize: copy-free view variant)" if args.paged else
                                 "kvmem_select + kvmem_materialize_attend" if fused else
                                 "kvmem_select + kvmem_materialize" + (" + kvmem_view_attend" if spec.attend else "")},
             "e2e": {"value": whole_job_rate(Ke, world, e2e_ms), "unit": UNIT, "steps": Ke,
                     "h2d_bytes_per_step": rows * spec.head_dim * 2,
                     "d2h_bytes_per_step": rows * spec.head_dim * 4 + rows * 4,
                     "api": "kvmem_recall_step_host (pinned host query in, host O and LSE out, synchronous)"},
-            "gpu_launches": K * (KERNELS_PER_STEP - (1 if fused else 0)),
+            "gpu_launches": K * (KERNELS_PER_STEP - (1 if fused else 0) + (1 if args.rope else 0)),
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<2> + merge (kvmem_paged_attend)" if args.paged else
+            "roofline": {"bound": "hbm", "kernel": "gather_rope_kernel (kvmem_materialize_rope)" if args.rope else
+                                                   "attend_split_kernel<2> + merge (kvmem_paged_attend)" if args.paged else
                                                    "attend_split_kernel<1> + merge (kvmem_materialize_attend: view written while attended)"
                                                    if fused else "gather_bulk_kernel (kvmem_materialize)",
                          "achieved": gather_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gather_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": gather_s * 1e3,
-                         "traffic": None if args.paged else FUSED_TRAFFIC.get(base.name) if fused else GATHER_TRAFFIC.get(base.name)},
+                         "traffic": None if args.paged else ROPE_GATHER_TRAFFIC.get(base.name) if args.rope else
+                                    FUSED_TRAFFIC.get(base.name) if fused else GATHER_TRAFFIC.get(base.name)},
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes,
                          "accounting": "index + one read of the selected pages (copy-free view, nothing materialised)" if args.paged else
                                        "index + view read + view write (fused pass)" if fused else
@@ -349,6 +397,8 @@ def run_native(args):
                                 "frac": 2 * flop_alg / sel_s / 1e12 / tpeak["tflops"], "peak_source": f"of {tpeak['source']} (burst)",
                                 "executed_flop_per_launch_pair": 2 * flop_alg, "algorithmic_flop": flop_alg,
                                 "algorithmic_tflops": flop_alg / sel_s / 1e12, "avg_select_ms": sel_s * 1e3, "traffic": None}
+        if args.rope:
+            line["e2e"]["api"] = "pinned host query in, host O and LSE out, around the four calls of the position-consistent step"
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(base, args.cpu_sample_blocks)
         print(json.dumps(line), flush=True)
@@ -460,6 +510,9 @@ def main():
     ap.add_argument("--workload", choices=sorted(CONFIGS), default="1m")
     ap.add_argument("--blocks", type=int, default=0, help="shrink the history to this many blocks (profiling)")
     ap.add_argument("--flush-l2", action="store_true", help="write 256 MiB between steps (for workloads near L2 size)")
+    ap.add_argument("--rope", action="store_true",
+                    help="position-consistent view: keys de-rotated at append, query de-rotated for retrieval, RoPE at the "
+                         "compact position fused into the gather (kvmem_materialize_rope), then kvmem_view_attend")
     ap.add_argument("--paged", action="store_true",
                     help="copy-free execution view: kvmem_select + kvmem_paged_attend (no view is materialised; not the headline step)")
     ap.add_argument("--unfused", action="store_true", help="separate kvmem_materialize and kvmem_view_attend calls")
