@@ -221,6 +221,22 @@ int kvmem_paged_attend(kvmem_pool_t* pool, int32_t session_first, int32_t n_sess
                        const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
                        void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
+/* Working-set delta between two consecutive steps (Eq. "kvmem-working-set-delta", Sec. 4.4):
+ *     retained R = W_next n W_prev,   incoming L = W_next \ W_prev,   outgoing E = W_prev \ W_next.
+ * prev_ids / next_ids are the ascending id lists kvmem_select wrote at the two steps, a block's slot is
+ * its index in its list (compact position / block_tokens).  All DEVICE int32:
+ *   prev_ids, next_ids [n_sessions][stride];  n_prev, n_next [n_sessions]
+ *   retained [n_sessions][stride][3] = (id, slot in prev, slot in next)   ascending ids
+ *   incoming [n_sessions][stride][2] = (id, slot in next);  outgoing [n_sessions][stride] = id
+ *   counts   [n_sessions][3] = (|R|, |L|, |E|)
+ * A retained block whose slot moved needs its resident keys re-rotated by (new - old) * block_tokens
+ * positions (kvmem_rope_rotate); only incoming blocks have to be fetched. */
+int kvmem_working_set_delta(kvmem_pool_t* pool, int32_t n_sessions, const int32_t* prev_ids /*DEVICE*/,
+                            const int32_t* n_prev /*DEVICE*/, const int32_t* next_ids /*DEVICE*/,
+                            const int32_t* n_next /*DEVICE*/, int32_t stride, int32_t* retained /*DEVICE*/,
+                            int32_t* incoming /*DEVICE*/, int32_t* outgoing /*DEVICE*/, int32_t* counts /*DEVICE*/,
+                            void* stream);
+
 /* kvmem_view_attend for callers that cannot allocate device memory.  (The paper has no counterpart.)
  * Who needs it: a serving process that gave all of HBM to its KV pool at start-up and runs with
  * its allocator frozen, a plug-in that only ever sees the buffers of one request, or a latency path

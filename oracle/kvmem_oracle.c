@@ -350,3 +350,34 @@ int kvo_gather_rope(const bf16_t* pagesK, const bf16_t* pagesV, const int32_t* t
     }
     return 0;
 }
+
+/* =======================================================================================
+ * Working-set delta (Eq. "kvmem-working-set-delta", Sec. 4.4): with W_prev and W_next the block
+ * sets of two consecutive steps,
+ *     R = W_next n W_prev (retained),  L = W_next \ W_prev (incoming),  E = W_prev \ W_next (outgoing).
+ * Inputs are the chronological (ascending) id lists; a block's slot is its index in its list, i.e. its
+ * compact position divided by B.  Outputs, all in ascending id order:
+ *   retained [nR][3] = (id, slot in prev, slot in next); incoming [nL][2] = (id, slot in next);
+ *   outgoing [nE] = id.  counts = (nR, nL, nE).
+ */
+void kvo_working_set_delta(const int32_t* prev, int64_t n_prev, const int32_t* next, int64_t n_next,
+                           int32_t* retained, int32_t* incoming, int32_t* outgoing, int32_t* counts) {
+    int64_t nR = 0, nL = 0, nE = 0;
+    for (int64_t j = 0; j < n_next; ++j) {
+        int64_t found = -1;
+        for (int64_t i = 0; i < n_prev; ++i)
+            if (prev[i] == next[j]) { found = i; break; }
+        if (found >= 0) {
+            retained[3 * nR] = next[j]; retained[3 * nR + 1] = (int32_t)found; retained[3 * nR + 2] = (int32_t)j; ++nR;
+        } else {
+            incoming[2 * nL] = next[j]; incoming[2 * nL + 1] = (int32_t)j; ++nL;
+        }
+    }
+    for (int64_t i = 0; i < n_prev; ++i) {
+        int found = 0;
+        for (int64_t j = 0; j < n_next; ++j)
+            if (next[j] == prev[i]) { found = 1; break; }
+        if (!found) outgoing[nE++] = prev[i];
+    }
+    counts[0] = (int32_t)nR; counts[1] = (int32_t)nL; counts[2] = (int32_t)nE;
+}

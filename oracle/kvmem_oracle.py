@@ -62,6 +62,8 @@ def lib():
         L.kvo_rope_rotate.restype = i32
         L.kvo_gather_rope.argtypes = [p, p, p, p, i64, i32, i32, i32, i32, p, p, i64, i64, p, i64]
         L.kvo_gather_rope.restype = i32
+        L.kvo_working_set_delta.argtypes = [p, i64, p, i64, p, p, p, p]
+        L.kvo_working_set_delta.restype = None
         L.kvo_threads.argtypes = []
         L.kvo_threads.restype = i32
         _lib = L
@@ -214,3 +216,17 @@ def gather_rope(repo: Repository, table: np.ndarray, sel: np.ndarray, cap_tokens
     if rc != 0:
         raise ValueError("compact positions outside the RoPE table")
     return viewK, viewV
+
+
+# ---- working-set delta ---------------------------------------------------------------------------
+
+def working_set_delta(prev: np.ndarray, nxt: np.ndarray):
+    """Ascending int32 id lists -> (retained [nR][3] = id, old slot, new slot; incoming [nL][2] = id, new slot;
+    outgoing [nE])."""
+    prev, nxt = np.ascontiguousarray(prev, np.int32), np.ascontiguousarray(nxt, np.int32)
+    ret = np.zeros((max(len(nxt), 1), 3), np.int32)
+    inc = np.zeros((max(len(nxt), 1), 2), np.int32)
+    out = np.zeros(max(len(prev), 1), np.int32)
+    cnt = np.zeros(3, np.int32)
+    lib().kvo_working_set_delta(_ptr(prev), len(prev), _ptr(nxt), len(nxt), _ptr(ret), _ptr(inc), _ptr(out), _ptr(cnt))
+    return ret[: cnt[0]].copy(), inc[: cnt[1]].copy(), out[: cnt[2]].copy()

@@ -555,6 +555,21 @@ int kvmem_paged_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_session
     return KVMEM_OK;
 }
 
+int kvmem_working_set_delta(kvmem_pool_t* p, int32_t n_sessions, const int32_t* prev_ids, const int32_t* n_prev,
+                            const int32_t* next_ids, const int32_t* n_next, int32_t stride, int32_t* retained,
+                            int32_t* incoming, int32_t* outgoing, int32_t* counts, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (n_sessions < 1 || stride < 1 || !prev_ids || !n_prev || !next_ids || !n_next || !retained || !incoming || !outgoing ||
+        !counts) {
+        set_error("kvmem_working_set_delta: null pointer or non-positive size");
+        return KVMEM_E_INVALID;
+    }
+    cudaError_t e = launch_working_set_delta(*p, n_sessions, prev_ids, n_prev, next_ids, n_next, stride, retained, incoming,
+                                             outgoing, counts, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("working-set delta kernel launch", e);
+    return KVMEM_OK;
+}
+
 int kvmem_get_index(kvmem_pool_t* p, int32_t session, const void** index, int32_t* n_blocks) {
     if (!pool_ok(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;

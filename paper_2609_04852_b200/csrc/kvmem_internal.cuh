@@ -90,6 +90,11 @@ ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions
 cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q,
                                 int M, const ScoreWorkspace& ws, float* scores, int scores_stride, cudaStream_t st);
 
+// working-set delta (kvmem_delta.cu)
+cudaError_t launch_working_set_delta(const kvmem_pool& p, int n_sessions, const int32_t* prev_ids, const int32_t* n_prev,
+                                     const int32_t* next_ids, const int32_t* n_next, int stride, int32_t* retained,
+                                     int32_t* incoming, int32_t* outgoing, int32_t* counts, cudaStream_t st);
+
 // rotary position embedding (kvmem_rope.cu)
 cudaError_t launch_rope_rotate(const kvmem_pool& p, const __nv_bfloat16* x, __nv_bfloat16* y, long long n_rows, int n_vec,
                                const int32_t* positions, int inverse, cudaStream_t st);

@@ -76,6 +76,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_append_blocks_rope": (C.c_int, [vp, i32, vp, vp, i32, C.POINTER(i32), C.POINTER(i32), vp]),
         "kvmem_rope_rotate": (C.c_int, [vp, vp, vp, C.c_int64, i32, vp, i32, vp]),
         "kvmem_materialize_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, i32, vp]),
+        "kvmem_working_set_delta": (C.c_int, [vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]),
         "kvmem_paged_attend": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
         "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
@@ -96,7 +97,8 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_materialize", "kvmem_view_attend", "kvmem_get_index", "kvmem_get_block_table",
             "kvmem_device_status", "kvmem_set_option", "kvmem_step_staging_bytes", "kvmem_recall_step_host",
             "kvmem_view_attend_static", "kvmem_materialize_attend",
-            "kvmem_paged_attend", "kvmem_append_blocks_rope", "kvmem_rope_rotate", "kvmem_materialize_rope")
+            "kvmem_paged_attend", "kvmem_append_blocks_rope", "kvmem_rope_rotate", "kvmem_materialize_rope",
+            "kvmem_working_set_delta")
 
 
 def _check(status: int) -> None:
@@ -188,6 +190,24 @@ class Pool:
             ids = (C.c_int32 * n)(*[int(x) for x in phys_ids])
         _check(self.lib.kvmem_append_blocks(self.handle, session, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16),
                                             n, ids, _stream()))
+
+    # ---- working-set delta
+    def working_set_delta(self, prev_ids: torch.Tensor, n_prev: torch.Tensor, next_ids: torch.Tensor,
+                          n_next: torch.Tensor):
+        """Retained / incoming / outgoing blocks between two selections (ascending int32 id lists of equal stride).
+        Returns (retained [ns][stride][3], incoming [ns][stride][2], outgoing [ns][stride], counts [ns][3])."""
+        ns, stride = prev_ids.shape
+        if next_ids.shape != prev_ids.shape:
+            raise ValueError("both id lists must have the same [n_sessions][stride] shape")
+        dev = prev_ids.device
+        ret = torch.zeros(ns, stride, 3, dtype=torch.int32, device=dev)
+        inc = torch.zeros(ns, stride, 2, dtype=torch.int32, device=dev)
+        out = torch.zeros(ns, stride, dtype=torch.int32, device=dev)
+        cnt = torch.zeros(ns, 3, dtype=torch.int32, device=dev)
+        _check(self.lib.kvmem_working_set_delta(self.handle, ns, _dev(prev_ids, torch.int32), _dev(n_prev, torch.int32),
+                                                _dev(next_ids, torch.int32), _dev(n_next, torch.int32), stride,
+                                                ret.data_ptr(), inc.data_ptr(), out.data_ptr(), cnt.data_ptr(), _stream()))
+        return ret, inc, out, cnt
 
     # ---- position-consistent keys
     def append_blocks_rope(self, session: int, k_roped: torch.Tensor, v: torch.Tensor, block_pos0: Sequence[int],

@@ -218,6 +218,35 @@ def test_long_session_takes_the_general_top_k_path():
         assert np.array_equal(bits(got["view"].k[0])[:, :, :T], vK[:, :, :T])
 
 
+# ------------------------------------------------------------------ working-set delta
+
+def test_working_set_delta_between_two_steps():
+    spec = CONFIGS["batch8"].with_(name="delta", n_sessions=2, n_blocks=3000, n_planted=40, budget_blocks=1500,
+                                   block_tokens=16, n_q_tokens=1, permute_pages=False)
+    pool = fill_pool(spec)
+    dev = torch.device("cuda", 0)
+    k = spec.budget_blocks
+    sels, counts = [], []
+    for qset, budget in ((0, 1500), (5, 1100)):                 # two consecutive steps with different queries and budgets
+        q = queries(spec, qset)[0].to(dev)
+        sel = torch.full((2, k), -1, dtype=torch.int32, device=dev)
+        n_sel = torch.zeros(2, dtype=torch.int32, device=dev)
+        pool.select(q, _params(budget_blocks=budget), sel, n_sel)
+        sels.append(sel); counts.append(n_sel)
+    ret, inc, out, cnt = pool.working_set_delta(sels[0], counts[0], sels[1], counts[1])
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    for s in range(2):
+        prev = sels[0][s, : int(counts[0][s])].cpu().numpy()
+        nxt = sels[1][s, : int(counts[1][s])].cpu().numpy()
+        r_ref, i_ref, o_ref = orc.working_set_delta(prev, nxt)
+        nR, nL, nE = (int(x) for x in cnt[s].cpu())
+        assert (nR, nL, nE) == (len(r_ref), len(i_ref), len(o_ref)) and nR > 0 and nL > 0 and nE > 0
+        assert np.array_equal(ret[s, :nR].cpu().numpy(), r_ref)
+        assert np.array_equal(inc[s, :nL].cpu().numpy(), i_ref)
+        assert np.array_equal(out[s, :nE].cpu().numpy(), o_ref)
+
+
 # ------------------------------------------------------------------ fused view assembly + attention
 
 @pytest.mark.parametrize("n_sessions,M,budget", [(1, 4, 150), (3, 1, 20), (1, 2, 1)])

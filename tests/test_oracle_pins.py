@@ -424,3 +424,21 @@ def test_tiny_config_planted_recovery():
     planted = set(planted_blocks(spec, 0)[0].tolist())
     assert planted <= set(res["sel"].tolist()) and len(res["sel"]) == 32
     assert abs(res["R"].sum() - spec.n_q_tokens) < 1e-5
+
+
+# ------------------------------------------------------------------ working-set delta (Eq. kvmem-working-set-delta)
+
+def test_working_set_delta_matches_set_algebra():
+    for n_prev, n_next, universe in [(0, 5, 20), (7, 0, 20), (12, 12, 15), (40, 33, 60), (9, 9, 9)]:
+        prev = np.sort(rng.choice(universe, n_prev, replace=False)).astype(np.int32)
+        nxt = np.sort(rng.choice(universe, n_next, replace=False)).astype(np.int32)
+        ret, inc, out = orc.working_set_delta(prev, nxt)
+        P, N = set(prev.tolist()), set(nxt.tolist())
+        assert ret[:, 0].tolist() == sorted(P & N) and inc[:, 0].tolist() == sorted(N - P) and out.tolist() == sorted(P - N)
+        assert len(ret) + len(inc) == n_next and len(ret) + len(out) == n_prev
+        for bid, old, new in ret.tolist():
+            assert prev[old] == bid and nxt[new] == bid           # slots index the chronological lists
+        for bid, new in inc.tolist():
+            assert nxt[new] == bid
+    ret, inc, out = orc.working_set_delta(np.array([1, 4, 6], np.int32), np.array([2, 4, 6, 9], np.int32))
+    assert ret.tolist() == [[4, 1, 1], [6, 2, 2]] and inc.tolist() == [[2, 0], [9, 3]] and out.tolist() == [1]
