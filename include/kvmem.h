@@ -157,6 +157,11 @@ int kvmem_materialize_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_
 
 /* ---- the recall step ----------------------------------------------------------------------- */
 
+/* Scores only (Eq. "kvmem-block-score", Sec. 4.3): the first half of kvmem_select, same arguments and
+ * definitions; scores (required) receives R for every session. */
+int kvmem_score(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/, int32_t n_q_tokens,
+                float* scores /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
 /* Score and select (Sec. 4.3, Eq. "kvmem-block-score"; selector; Sec. 5.2 tiled scoring with the
  * softmax kept global across tiles).  For each session s in [session_first, session_first + n_sessions):
  *     R_b = sum_m (1/(L*H)) sum_{l,h} softmax_{b' in all blocks of s}( q[m][l][h] . kbar[l][b'][g(h)] / sqrt(d) )_b

@@ -335,23 +335,15 @@ int kvmem_materialize_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_ses
     return KVMEM_OK;
 }
 
-int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
-                 const kvmem_select_params_t* prm, int32_t* sel_ids, int32_t sel_stride, int32_t* n_sel, float* scores,
-                 void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
-    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
-    if (!q || !aligned(q, 16) || !prm || !sel_ids || !n_sel || !workspace || !aligned(workspace, 256)) {
-        set_error("kvmem_select: null or misaligned pointer");
+// scoring stage shared by kvmem_score and kvmem_select; *sc_out receives where the scores were written
+static int score_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                      float* scores, void* workspace, size_t workspace_bytes, cudaStream_t st, float** sc_out) {
+    if (!q || !aligned(q, 16) || !workspace || !aligned(workspace, 256)) {
+        set_error("scoring: null or misaligned pointer");
         return KVMEM_E_INVALID;
     }
     if (n_q_tokens < 1) { set_error("n_q_tokens must be positive"); return KVMEM_E_INVALID; }
-    if (prm->n_sink_blocks < 0 || prm->n_recent_blocks < 0) { set_error("sink/recent counts must be non-negative"); return KVMEM_E_INVALID; }
     if (p->cfg.head_dim != 128) { set_error("scoring kernels are built for head_dim 128"); return KVMEM_E_UNSUPPORTED; }
-    int max_k = 0;
-    for (int s = session_first; s < session_first + n_sessions; ++s)
-        max_k = std::max(max_k, kvmem_budget_blocks(prm, p->cfg.block_tokens, p->sess_blocks[s]));
-    if (sel_stride < max_k) { set_error("sel_stride %d is below the clamped budget %d", sel_stride, max_k); return KVMEM_E_CAPACITY; }
-    cudaStream_t st = (cudaStream_t)stream;
     float* sc = nullptr;
     cudaError_t e;
     if (n_q_tokens > kMaxDecodeTokens) {
@@ -374,7 +366,35 @@ int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, con
                                 p->cfg.max_blocks_per_session, st);
     }
     if (e != cudaSuccess) return cuda_fail("score kernel launch", e);
-    e = launch_topk(*p, session_first, n_sessions, sc, p->cfg.max_blocks_per_session, *prm, sel_ids, sel_stride, n_sel, st);
+    *sc_out = sc;
+    return KVMEM_OK;
+}
+
+int kvmem_score(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens, float* scores,
+                void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!scores) { set_error("scores is null"); return KVMEM_E_INVALID; }
+    float* sc = nullptr;
+    return score_impl(p, session_first, n_sessions, q, n_q_tokens, scores, workspace, workspace_bytes, (cudaStream_t)stream, &sc);
+}
+
+int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                 const kvmem_select_params_t* prm, int32_t* sel_ids, int32_t sel_stride, int32_t* n_sel, float* scores,
+                 void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!prm || !sel_ids || !n_sel) { set_error("kvmem_select: null pointer"); return KVMEM_E_INVALID; }
+    if (prm->n_sink_blocks < 0 || prm->n_recent_blocks < 0) { set_error("sink/recent counts must be non-negative"); return KVMEM_E_INVALID; }
+    int max_k = 0;
+    for (int s = session_first; s < session_first + n_sessions; ++s)
+        max_k = std::max(max_k, kvmem_budget_blocks(prm, p->cfg.block_tokens, p->sess_blocks[s]));
+    if (sel_stride < max_k) { set_error("sel_stride %d is below the clamped budget %d", sel_stride, max_k); return KVMEM_E_CAPACITY; }
+    cudaStream_t st = (cudaStream_t)stream;
+    float* sc = nullptr;
+    int rc = score_impl(p, session_first, n_sessions, q, n_q_tokens, scores, workspace, workspace_bytes, st, &sc);
+    if (rc != KVMEM_OK) return rc;
+    cudaError_t e = launch_topk(*p, session_first, n_sessions, sc, p->cfg.max_blocks_per_session, *prm, sel_ids, sel_stride, n_sel, st);
     if (e != cudaSuccess) return cuda_fail("top-k kernel launch", e);
     return KVMEM_OK;
 }

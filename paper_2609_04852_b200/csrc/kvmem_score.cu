@@ -367,11 +367,12 @@ score_logits_mma_kernel(const __grid_constant__ CUtensorMap map_idx, const __nv_
 }
 
 // Merge the per-CTA statistics of every row, then R_b = (1/(L*H)) sum_rows exp2(logit - max_row) / Z_row.
-// A CTA owns 128 consecutive blocks.  The per-CTA (max, sum-exp) pairs are first staged in shared
+// A CTA owns 32 * kFinishU consecutive blocks.  The per-CTA (max, sum-exp) pairs are first staged in shared
 // memory with independent coalesced loads and merged there, one thread per row.  Then thread
-// (lgs, bl) sums the rows of heads lgs, lgs + 8, ... for blocks bl, bl + 32, bl + 64, bl + 96
+// (lgs, bl) sums the rows of heads lgs, lgs + 8, ... for blocks bl, bl + 32, ...
 // (independent coalesced loads), and the 8 partial sums are added in a fixed order.
-constexpr int kFinishBlocks = 128;
+constexpr int kFinishU = 1;                      // blocks per thread
+constexpr int kFinishBlocks = 32 * kFinishU;
 __global__ void __launch_bounds__(256)
 score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__ partials,
                     const int32_t* __restrict__ nblocks_dev, int session_first, int LG, int rows, int rows_pad,
@@ -410,23 +411,27 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
     __syncthreads();
     const int bl = threadIdx.x & 31, lgs = threadIdx.x >> 5;
     const int b0 = blockIdx.x * kFinishBlocks + bl;
-    float part[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    float part[kFinishU];
+#pragma unroll
+    for (int u = 0; u < kFinishU; ++u) part[u] = 0.0f;
     for (int lg = lgs; lg < LG; lg += 8) {
         const float* base = logits + (((size_t)s * LG + lg) * rows_pad) * (size_t)nb_pad + b0;
-        float sub[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        float sub[kFinishU];
+#pragma unroll
+        for (int u = 0; u < kFinishU; ++u) sub[u] = 0.0f;
 #pragma unroll 8
         for (int j = 0; j < rows; ++j) {
             const float2 st = rowstat[lg * rows + j];
             const float* rp = base + (size_t)j * nb_pad;
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < kFinishU; ++u)
                 if (b0 + 32 * u < NB) sub[u] += exp2f(rp[32 * u] - st.x) * st.y;
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) part[u] += sub[u];
+        for (int u = 0; u < kFinishU; ++u) part[u] += sub[u];
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) red[lgs][bl + 32 * u] = part[u];
+    for (int u = 0; u < kFinishU; ++u) red[lgs][bl + 32 * u] = part[u];
     __syncthreads();
     if (threadIdx.x < kFinishBlocks) {
         const int b = blockIdx.x * kFinishBlocks + threadIdx.x;

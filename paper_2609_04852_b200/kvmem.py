@@ -65,6 +65,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_session_reset": (C.c_int, [vp, i32]),
         "kvmem_session_blocks": (i32, [vp, i32]),
         "kvmem_append_blocks": (C.c_int, [vp, i32, vp, vp, i32, C.POINTER(i32), vp]),
+        "kvmem_score": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, sz, vp]),
         "kvmem_select": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, sz, vp]),
         "kvmem_materialize": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, vp]),
         "kvmem_view_attend": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
@@ -98,7 +99,7 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_device_status", "kvmem_set_option", "kvmem_step_staging_bytes", "kvmem_recall_step_host",
             "kvmem_view_attend_static", "kvmem_materialize_attend",
             "kvmem_paged_attend", "kvmem_append_blocks_rope", "kvmem_rope_rotate", "kvmem_materialize_rope",
-            "kvmem_working_set_delta")
+            "kvmem_working_set_delta", "kvmem_score")
 
 
 def _check(status: int) -> None:
@@ -259,6 +260,13 @@ class Pool:
         if self._attend_ws is None or self._attend_ws.numel() < need:
             self._attend_ws = torch.empty(need, dtype=torch.uint8, device=self.device)
         return self._attend_ws
+
+    def score(self, q: torch.Tensor, scores: torch.Tensor, session_first: int = 0) -> None:
+        """Block relevance only: q bf16 [n_sessions][M][L][H][d] -> scores fp32 [n_sessions][max_blocks_per_session]."""
+        ns, M = q.shape[0], q.shape[1]
+        ws = self.select_workspace(ns, M)
+        _check(self.lib.kvmem_score(self.handle, session_first, ns, _dev(q, torch.bfloat16), M,
+                                    _dev(scores, torch.float32), ws.data_ptr(), ws.numel(), _stream()))
 
     def select(self, q: torch.Tensor, params: SelectParams, sel_ids: torch.Tensor, n_sel: torch.Tensor,
                scores: Optional[torch.Tensor] = None, session_first: int = 0) -> None:

@@ -325,6 +325,26 @@ def test_chunked_scoring_matches_oracle(M, n_blocks, n_sessions):
         assert np.array_equal(bits(got["view"].v[s])[:, :, :T], vV[:, :, :T])
 
 
+@pytest.mark.parametrize("M,n_blocks,n_sessions", [(1, 333, 2), (4, 200, 1), (40, 300, 2)])
+def test_score_alone_equals_the_scores_select_reports_and_the_oracle(M, n_blocks, n_sessions):
+    spec = CONFIGS["batch8"].with_(name="score", n_sessions=n_sessions, n_blocks=n_blocks, n_planted=6,
+                                   budget_blocks=24, n_q_tokens=M, permute_pages=False)
+    lens = [n_blocks - 41 * s for s in range(n_sessions)]
+    pool = fill_pool(spec, lens)
+    osess = fill_oracle(spec, lens)
+    q, qb = queries(spec)
+    got = _run_step(pool, spec, q.cuda(), _params(budget_blocks=spec.budget_blocks), spec.budget_blocks, attend=False)
+    sc = torch.full((n_sessions, spec.n_blocks), -1.0, dtype=torch.float32, device="cuda")
+    pool.score(q.cuda(), sc)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    sc = sc.cpu().numpy()
+    for s in range(n_sessions):
+        R, _ = orc.block_scores(qb[s], osess[s].idx, osess[s].n_blocks)
+        check_scores(sc[s, :lens[s]], R, M)
+        assert np.array_equal(sc[s, :lens[s]], got["scores"][s, :lens[s]])     # same kernels, fixed merge order
+
+
 # ------------------------------------------------------------------ several sessions, permuted pages
 
 def test_multi_session_ragged_lengths_and_permuted_pages():
