@@ -171,6 +171,10 @@ def run_native(args):
         raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
+    for opt in args.option:
+        from paper_2609_04852_b200 import set_option
+        name, _, value = opt.partition("=")
+        set_option(name, int(value))
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
 
@@ -527,6 +531,8 @@ def main():
     ap.add_argument("--paged", action="store_true",
                     help="copy-free execution view: kvmem_select + kvmem_paged_attend (no view is materialised; not the headline step)")
     ap.add_argument("--unfused", action="store_true", help="separate kvmem_materialize and kvmem_view_attend calls")
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
+                    help="kernel-variant switch passed to kvmem_set_option (e.g. chunk_poly=0)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)
     args = ap.parse_args()

@@ -294,10 +294,12 @@ int kvmem_get_block_table(kvmem_pool_t* pool, int32_t session, const int32_t** t
  * KVMEM_E_TIMEOUT or KVMEM_E_DEVICE_RANGE.  Returns KVMEM_OK if the read itself worked. */
 int kvmem_device_status(kvmem_pool_t* pool, int32_t* status /*HOST*/, void* stream);
 
-/* Process-wide implementation switches used to compare kernel variants; they never change results.
- * (No counterpart in the paper.)  "gather_mode": 1 = bulk asynchronous copies through shared memory
+/* Process-wide implementation switches used to compare kernel variants; "gather_mode" and "score_mode"
+ * never change results, "chunk_poly" moves scores by a few 1e-6 relative.  (No counterpart in the paper.)  "gather_mode": 1 = bulk asynchronous copies through shared memory
  * (default), 0 = 128-bit load/store copy.  "score_mode" (decode-sized queries): 1 = dot products on the
- * tensor cores (default), 0 = fp32 ALU kernel that reduces the query rows with warp shuffles. */
+ * tensor cores (default), 0 = fp32 ALU kernel that reduces the query rows with warp shuffles.
+ * "chunk_poly" (multi-token chunks): n in 2..5 = every n-th exponential of the two softmax passes is a
+ * degree-4 polynomial on the FMA pipe instead of a special-function-unit instruction (default 5), 0 = none. */
 int kvmem_set_option(const char* name /*HOST*/, int32_t value);
 
 #ifdef __cplusplus

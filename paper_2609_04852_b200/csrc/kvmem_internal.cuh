@@ -70,6 +70,7 @@ void set_error(const char* fmt, ...);
 
 // tuning switches (kvmem_set_option)
 extern int g_score_mode;    // 1: tensor-core decode scoring (default), 0: fp32 ALU + warp-shuffle kernel
+extern int g_chunk_poly;    // chunked scoring: every n-th exponential on the FMA pipe (0: all on the special-function unit)
 extern int g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
 
 // ---- kernel launchers (each defined next to its kernel) ----------------------------------------
@@ -104,11 +105,12 @@ cudaError_t launch_gather_rope(const kvmem_pool& p, int session_first, int n_ses
 
 // multi-token query chunks: tcgen05 two-pass contraction
 struct ChunkWorkspace {
-    float2* rowstat;   // [ns][L][G][4][rows_pad] (max, sum-exp) per slice of the tile columns
+    float2* rowstat;   // [ns][L][G][n_chunks][4][rows_pad] (max, sum-exp) per run of block tiles and slice of the tile columns
+    float* shift;      // [ns][L][G][shift_stride]: -(max + log2 Z) of every query row, -inf on padding rows
     float* colsum;     // [ns][L][G][4][nb_pad]: per-head, per-column-slice sums of the softmax weights over the head's query rows
     float* scores;     // [ns][max_bps]
-    size_t rowstat_bytes, colsum_bytes, scores_bytes, total;
-    int rows, rows_pad, n_panels, nb_pad;
+    size_t rowstat_bytes, shift_bytes, colsum_bytes, scores_bytes, total;
+    int rows, rows_pad, n_panels, nb_pad, n_chunks, shift_stride;
 };
 ChunkWorkspace plan_chunk_workspace(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, char* base);
 bool chunked_scoring_supported(const kvmem_pool_config_t& c, int n_q_tokens);

@@ -59,6 +59,29 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     return false;
 }
 
+// Same bound, for waits that are expected to be long (a control warp waiting for the warps that do the
+// arithmetic): every attempt may stay suspended in hardware for up to kSuspendNs, so the waiting warp
+// issues almost no instructions and leaves the issue slots and the shared-memory pipe to the others.
+constexpr uint32_t kSuspendNs = 20000u;
+__device__ __forceinline__ bool mbar_wait_suspended(uint64_t* bar, uint32_t parity) {
+    uint64_t t0 = 0;
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs)
+            : "memory");
+        if (ok) return true;
+        const uint64_t now = globaltimer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > kWaitLimitNs) return false;
+    }
+    return false;
+}
+
 // 1-D bulk copy global -> shared, completion on an mbarrier (bytes % 16 == 0, both 16-byte aligned)
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(

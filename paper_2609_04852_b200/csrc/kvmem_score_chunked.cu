@@ -39,6 +39,7 @@ constexpr int kCkEpiWarps = 16;               // four per TMEM lane quarter, eac
 constexpr int kCkSplit = kCkEpiWarps / 4;     // column slices per tile
 constexpr int kCkThreads = 64 + 32 * kCkEpiWarps;   // TMA warp, MMA warp, epilogue warps
 constexpr int kCkHalfCols = kCkBN / kCkSplit; // columns per epilogue warp and tile
+constexpr int kCkChunks = kCkHalfCols / 32;   // 32-column register chunks per epilogue warp and tile
 constexpr int kCkAHalf = kCkBM * 128;         // bytes of one 64-dim half of the 128-row operand tile (16 KiB)
 constexpr int kCkBHalf = kCkBN * 128;         // bytes of one 64-dim half of the 256-row operand tile (32 KiB)
 constexpr int kCkTmemCols = kCkAccs * kCkBN;  // 512: all of tensor memory
@@ -72,24 +73,6 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint6
 __device__ __forceinline__ void commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(ptx::smem_u32(bar)) : "memory");
 }
-// 32 consecutive fp32 columns of this thread's TMEM lane
-__device__ __forceinline__ void ld32(uint32_t taddr, float (&v)[32]) {
-    uint32_t r[32];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
 // issue the load of 32 columns without waiting for it
 __device__ __forceinline__ void ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -130,10 +113,11 @@ __device__ __forceinline__ void tma_load_4d(void* dst_smem, const CUtensorMap* m
 
 struct ChunkArgs {
     const int32_t* nblocks_dev;
-    float2* rowstat;      // [ns][LG][kCkSplit][rows_pad]  (max, sum-exp) of every query row over one slice of the tile columns, log2 domain
-    float* headsum;       // [ns][LG][kCkSplit][nb_pad]    per column slice: sum over the head's query rows of the softmax weights
+    float2* rowstat;      // [ns][LG][n_chunks][kCkSplit][rows_pad]  (max, sum-exp) of every query row over one run of block tiles and one slice of the tile columns, log2 domain
+    float* shift;         // [ns][LG][shift_stride]                  -(max + log2 Z) per query row
+    float* headsum;       // [ns][LG][kCkSplit][nb_pad]              per column slice: sum over the head's query rows of the softmax weights
     int32_t* status;
-    int session_first, n_sessions, M, L, G, r, rows, rows_pad, nb_pad, n_bpanels;
+    int session_first, n_sessions, M, L, G, r, rows, rows_pad, nb_pad, n_bpanels, n_panels, n_chunks, shift_stride;
     float scale_log2e;
 };
 
@@ -153,9 +137,33 @@ __device__ __forceinline__ void issue_tile_mma(uint32_t d_tmem, uint32_t a_lo, u
     }
 }
 
+// 2^x on the FMA and integer pipes, for the share of the exponentials that the special-function unit
+// (16 results per clock and SM, the limiter of both passes) is spared.  x = n + f with n the nearest
+// integer and |f| <= 1/2; 2^f by a degree-4 polynomial (relative error below 3e-6), 2^n by adding n to
+// the exponent field.  Arguments below -125 (including -inf) return about 2^-125 instead of 0, which
+// is immaterial next to weights that sum to one per query row.
+__device__ __forceinline__ float ex2_poly(float x) {
+    x = fmaxf(x, -125.0f);
+    const float t = x + 12582912.0f;                 // 1.5 * 2^23: n sits in the low mantissa bits
+    const float f = x - (t - 12582912.0f);
+    float p = fmaf(0.009570100344717503f, f, 0.05591785907745361f);
+    p = fmaf(p, f, 0.240247443318367f);
+    p = fmaf(p, f, 0.6931217908859253f);
+    p = fmaf(p, f, 0.9999992847442627f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
+// element `idx` of a tile slice takes the polynomial when every POLY-th exponential is moved off the
+// special-function unit (POLY = 0: none)
+template <int POLY>
+__device__ __forceinline__ float ex2_mix(float x, int idx) {
+    if (POLY > 0 && idx % POLY == POLY - 1) return ex2_poly(x);
+    return t5::ex2(x);
+}
+
 // Fold 32 raw logits of one query row into its running (max, sum-exp), exp2 domain.  `live` (ragged
 // tiles only) is how many of the 32 columns are real blocks.
-template <bool RAGGED>
+template <bool RAGGED, int POLY>
 __device__ __forceinline__ void rowstat_chunk(const uint32_t (&raw)[32], int live, float scale_log2e, float& run_m, float& run_z) {
     float v[32];
 #pragma unroll
@@ -170,20 +178,29 @@ __device__ __forceinline__ void rowstat_chunk(const uint32_t (&raw)[32], int liv
     float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
-        s0 += t5::ex2(fmaf(v[i], scale_log2e, -mn)); s1 += t5::ex2(fmaf(v[i + 1], scale_log2e, -mn));
-        s2 += t5::ex2(fmaf(v[i + 2], scale_log2e, -mn)); s3 += t5::ex2(fmaf(v[i + 3], scale_log2e, -mn));
+        // a ragged slice keeps every exponential on the special-function unit: exp2(-inf) must be 0 there
+        s0 += ex2_mix<RAGGED ? 0 : POLY>(fmaf(v[i], scale_log2e, -mn), i);
+        s1 += ex2_mix<RAGGED ? 0 : POLY>(fmaf(v[i + 1], scale_log2e, -mn), i + 1);
+        s2 += ex2_mix<RAGGED ? 0 : POLY>(fmaf(v[i + 2], scale_log2e, -mn), i + 2);
+        s3 += ex2_mix<RAGGED ? 0 : POLY>(fmaf(v[i + 3], scale_log2e, -mn), i + 3);
     }
     run_z = run_z * t5::ex2(run_m - mn) + ((s0 + s1) + (s2 + s3));
     run_m = mn;
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Pass 1.  Grid (query panel, layer x KV head, session).  TMEM lane = query row.
+// Pass 1.  Persistent CTAs; work item = (session, layer x KV head, 128-row query panel, run of
+// kCkChunkTiles block tiles), run index fastest, a contiguous range of items per CTA: the panel in
+// shared memory changes at most a few times per CTA and all SMs carry the same number of tiles to
+// within one item.  TMEM lane = query row.
+constexpr int kCkChunkTiles = 8;
+
+template <int POLY>
 __global__ void __launch_bounds__(kCkThreads, 1)
 score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_idx,
                            ChunkArgs a) {
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ uint64_t a_full, b_full[kCkStages1], b_empty[kCkStages1], acc_full[kCkAccs], acc_empty[kCkAccs];
+    __shared__ uint64_t a_full, a_empty, b_full[kCkStages1], b_empty[kCkStages1], acc_full[kCkAccs], acc_empty[kCkAccs];
     __shared__ uint32_t tmem_base_slot;
 
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -191,14 +208,14 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     unsigned char* smem_b = base + 2 * kCkAHalf;               // index tiles: stages x 2 halves x 32 KiB
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int panel = blockIdx.x, lg = blockIdx.y, s = blockIdx.z;
-    const int l = lg / a.G, g = lg % a.G;
     const int LG = a.L * a.G;
-    const int NB = a.nblocks_dev[a.session_first + s];
-    const int n_tiles = (NB + kCkBN - 1) / kCkBN;
+    const int n_items = a.n_sessions * LG * a.n_panels * a.n_chunks;
+    const int item_begin = (int)((long long)n_items * blockIdx.x / gridDim.x);
+    const int item_end = (int)((long long)n_items * (blockIdx.x + 1) / gridDim.x);
 
     if (tid == 0) {
         ptx::mbar_init(&a_full, 1);
+        ptx::mbar_init(&a_empty, 1);
         for (int i = 0; i < kCkStages1; ++i) { ptx::mbar_init(&b_full[i], 1); ptx::mbar_init(&b_empty[i], 1); }
         for (int i = 0; i < kCkAccs; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], kCkEpiWarps); }
         ptx::fence_mbar_init();
@@ -212,80 +229,126 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     t5::fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
+    // every role walks the same item sequence and skips the same (empty) items; t0..t1 are the item's tiles
+    auto item_live = [&](int item, int& s, int& lg, int& panel, int& chunk, int& t0, int& t1, int& NB) {
+        chunk = item % a.n_chunks;
+        panel = (item / a.n_chunks) % a.n_panels;
+        lg = (item / (a.n_chunks * a.n_panels)) % LG;
+        s = item / (a.n_chunks * a.n_panels * LG);
+        NB = a.nblocks_dev[a.session_first + s];
+        const int n_tiles = (NB + kCkBN - 1) / kCkBN;
+        t0 = chunk * kCkChunkTiles;
+        t1 = min(t0 + kCkChunkTiles, n_tiles);
+        return t0 < t1;
+    };
+
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
-        if (lane == 0 && n_tiles > 0) {
+        if (lane == 0) {
             ptx::prefetch_tensormap(&map_q);
             ptx::prefetch_tensormap(&map_idx);
-            // Q panel: rows j = m * r + hr of this KV head; 128 rows = 128 / r tokens x r heads
-            const int m0 = s * a.M + panel * (kCkBM / a.r);
-            ptx::mbar_expect_tx(&a_full, 2 * kCkAHalf);
-            tma_load_4d(smem_a, &map_q, 0, g * a.r, l, m0, &a_full);
-            tma_load_4d(smem_a + kCkAHalf, &map_q, 64, g * a.r, l, m0, &a_full);
-            const int z = ((a.session_first + s) * a.L + l) * a.G + g;
-            for (int t = 0; t < n_tiles; ++t) {
-                const int st = t % kCkStages1;
-                if (t >= kCkStages1 && !ptx::mbar_wait(&b_empty[st], (uint32_t)(((t / kCkStages1) & 1) ^ 1))) {
-                    atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
-                    break;
+            int la = 0, tt = 0, cur_panel = -1;
+            bool ok = true;
+            for (int item = item_begin; ok && item < item_end; ++item) {
+                int s, lg, panel, chunk, t0, t1, NB;
+                if (!item_live(item, s, lg, panel, chunk, t0, t1, NB)) continue;
+                const int l = lg / a.G, g = lg % a.G;
+                if (item / a.n_chunks != cur_panel) {
+                    // Q panel: rows j = m * r + hr of this KV head; 128 rows = 128 / r tokens x r heads.
+                    // The previous panel must have been consumed by every MMA that reads it.
+                    cur_panel = item / a.n_chunks;
+                    if (la >= 1) ok = ptx::mbar_wait_suspended(&a_empty, (uint32_t)((la - 1) & 1));
+                    if (!ok) break;
+                    const int m0 = s * a.M + panel * (kCkBM / a.r);
+                    ptx::mbar_expect_tx(&a_full, 2 * kCkAHalf);
+                    tma_load_4d(smem_a, &map_q, 0, g * a.r, l, m0, &a_full);
+                    tma_load_4d(smem_a + kCkAHalf, &map_q, 64, g * a.r, l, m0, &a_full);
+                    ++la;
                 }
-                unsigned char* dst = smem_b + (size_t)st * 2 * kCkBHalf;
-                ptx::mbar_expect_tx(&b_full[st], 2 * kCkBHalf);
-                ptx::tma_load_3d(dst, &map_idx, 0, t * kCkBN, z, &b_full[st]);
-                ptx::tma_load_3d(dst + kCkBHalf, &map_idx, 64, t * kCkBN, z, &b_full[st]);
+                const int z = ((a.session_first + s) * a.L + l) * a.G + g;
+                for (int t = t0; t < t1; ++t, ++tt) {
+                    const int st = tt % kCkStages1;
+                    if (tt >= kCkStages1) ok = ptx::mbar_wait_suspended(&b_empty[st], (uint32_t)(((tt / kCkStages1) & 1) ^ 1));
+                    if (!ok) break;
+                    unsigned char* dst = smem_b + (size_t)st * 2 * kCkBHalf;
+                    ptx::mbar_expect_tx(&b_full[st], 2 * kCkBHalf);
+                    ptx::tma_load_3d(dst, &map_idx, 0, t * kCkBN, z, &b_full[st]);
+                    ptx::tma_load_3d(dst + kCkBHalf, &map_idx, 64, t * kCkBN, z, &b_full[st]);
+                }
             }
+            if (!ok) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
-        if (lane == 0 && n_tiles > 0) {
-            bool ok = ptx::mbar_wait(&a_full, 0);
+        if (lane == 0) {
             const uint32_t a_lo = t5::desc_lo(ptx::smem_u32(smem_a)), b_lo0 = t5::desc_lo(ptx::smem_u32(smem_b));
-            for (int t = 0; ok && t < n_tiles; ++t) {
-                const int st = t % kCkStages1, acc = t % kCkAccs;
-                ok = ptx::mbar_wait(&b_full[st], (uint32_t)((t / kCkStages1) & 1));
-                if (ok && t >= kCkAccs) ok = ptx::mbar_wait(&acc_empty[acc], (uint32_t)(((t / kCkAccs) & 1) ^ 1));
-                if (!ok) break;
-                t5::fence_after();
-                issue_tile_mma(tmem_base + (uint32_t)acc * kCkBN, a_lo, b_lo0 + (uint32_t)st * (2 * kCkBHalf >> 4));
-                t5::commit(&b_empty[st]);                  // the index tile may be overwritten
-                t5::commit(&acc_full[acc]);                // the accumulator may be read
+            int la = 0, tt = 0, cur_panel = -1;
+            bool ok = true;
+            for (int item = item_begin; ok && item < item_end; ++item) {
+                int s, lg, panel, chunk, t0, t1, NB;
+                if (!item_live(item, s, lg, panel, chunk, t0, t1, NB)) continue;
+                if (item / a.n_chunks != cur_panel) {
+                    cur_panel = item / a.n_chunks;
+                    if (la >= 1) t5::commit(&a_empty);     // arrives once every MMA on the old panel is done
+                    ok = ptx::mbar_wait_suspended(&a_full, (uint32_t)(la & 1));
+                    ++la;
+                }
+                for (int t = t0; ok && t < t1; ++t, ++tt) {
+                    const int st = tt % kCkStages1, acc = tt % kCkAccs;
+                    ok = ptx::mbar_wait_suspended(&b_full[st], (uint32_t)((tt / kCkStages1) & 1));
+                    if (ok && tt >= kCkAccs) ok = ptx::mbar_wait_suspended(&acc_empty[acc], (uint32_t)(((tt / kCkAccs) & 1) ^ 1));
+                    if (!ok) break;
+                    t5::fence_after();
+                    issue_tile_mma(tmem_base + (uint32_t)acc * kCkBN, a_lo, b_lo0 + (uint32_t)st * (2 * kCkBHalf >> 4));
+                    t5::commit(&b_empty[st]);                  // the index tile may be overwritten
+                    t5::commit(&acc_full[acc]);                // the accumulator may be read
+                }
             }
             if (!ok) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
         }
     } else {
-        // ------------------------------------------------ epilogue: warp -> (TMEM lane quarter, column half)
+        // ------------------------------------------------ epilogue: warp -> (TMEM lane quarter, column slice)
         const int quarter = warp & 3;                      // warps 2..17 -> quarters 2,3,0,1,...
         const int half = (warp - 2) >> 2;
-        const int row = panel * kCkBM + quarter * 32 + lane;   // row of this (session, l, g): m * r + hr
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * kCkHalfCols);
-        float run_m = -INFINITY, run_z = 0.0f;
-        for (int t = 0; t < n_tiles; ++t) {
-            const int acc = t % kCkAccs;
-            const bool arrived = ptx::mbar_wait(&acc_full[acc], (uint32_t)((t / kCkAccs) & 1));
-            if (!__all_sync(0xffffffffu, arrived)) {
-                if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
-                break;
+        int tt = 0;
+        bool failed = false;
+        for (int item = item_begin; !failed && item < item_end; ++item) {
+            int s, lg, panel, chunk, t0, t1, NB;
+            if (!item_live(item, s, lg, panel, chunk, t0, t1, NB)) continue;
+            const int row = panel * kCkBM + quarter * 32 + lane;   // row of this (session, l, g): m * r + hr
+            float run_m = -INFINITY, run_z = 0.0f;
+            for (int t = t0; t < t1; ++t, ++tt) {
+                const int acc = tt % kCkAccs;
+                const bool arrived = ptx::mbar_wait_suspended(&acc_full[acc], (uint32_t)((tt / kCkAccs) & 1));
+                if (!__all_sync(0xffffffffu, arrived)) {
+                    if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+                    failed = true;
+                    break;
+                }
+                t5::fence_after();
+                const int col0 = t * kCkBN + half * kCkHalfCols;
+                const bool ragged = col0 + kCkHalfCols > NB;
+                uint32_t buf[kCkChunks][32];
+#pragma unroll
+                for (int c = 0; c < kCkChunks; ++c) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf[c]);
+                t5::ld_wait();
+                // the accumulator now lives in registers: hand it back before doing the arithmetic
+                t5::fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
+                if (!ragged) {
+#pragma unroll
+                    for (int c = 0; c < kCkChunks; ++c) rowstat_chunk<false, POLY>(buf[c], 0, a.scale_log2e, run_m, run_z);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < kCkChunks; ++c)
+                        rowstat_chunk<true, POLY>(buf[c], NB - (col0 + c * 32), a.scale_log2e, run_m, run_z);
+                }
             }
-            t5::fence_after();
-            const int col0 = t * kCkBN + half * kCkHalfCols;
-            const bool ragged = col0 + kCkHalfCols > NB;
-            uint32_t buf[kCkHalfCols / 32][32];
-#pragma unroll
-            for (int c = 0; c < kCkHalfCols / 32; ++c) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf[c]);
-            t5::ld_wait();
-            // the accumulator now lives in registers: hand it back before doing the arithmetic
-            t5::fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
-            if (!ragged) {
-#pragma unroll
-                for (int c = 0; c < kCkHalfCols / 32; ++c) rowstat_chunk<false>(buf[c], 0, a.scale_log2e, run_m, run_z);
-            } else {
-#pragma unroll
-                for (int c = 0; c < kCkHalfCols / 32; ++c) rowstat_chunk<true>(buf[c], NB - (col0 + c * 32), a.scale_log2e, run_m, run_z);
-            }
+            if (!failed && row < a.rows)
+                a.rowstat[((((size_t)s * LG + lg) * a.n_chunks + chunk) * kCkSplit + half) * a.rows_pad + row] = make_float2(run_m, run_z);
         }
-        if (row < a.rows) a.rowstat[(((size_t)s * LG + lg) * kCkSplit + half) * a.rows_pad + row] = make_float2(run_m, run_z);
     }
 
     t5::fence_before();
@@ -296,12 +359,42 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     }
 }
 
+// Between the passes: shift = -(max + log2 Z) of every query row, merging the row statistics of all
+// tile runs and column slices in a fixed order; -inf switches a padding row off in pass 2.
+__global__ void __launch_bounds__(256)
+score_chunk_shift_kernel(ChunkArgs a) {
+    const int LG = a.L * a.G;
+    const long long total = (long long)a.n_sessions * LG * a.shift_stride;
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const int j = (int)(e % a.shift_stride);
+    const int head = (int)(e / a.shift_stride);
+    const int NB = a.nblocks_dev[a.session_first + head / LG];
+    const int n_tiles = (NB + kCkBN - 1) / kCkBN;
+    const int live_chunks = (n_tiles + kCkChunkTiles - 1) / kCkChunkTiles;
+    float sh = -INFINITY;
+    if (j < a.rows && live_chunks > 0) {
+        const float2* rs = a.rowstat + ((size_t)head * a.n_chunks * kCkSplit) * a.rows_pad + j;
+        const int n_part = live_chunks * kCkSplit;
+        float mx = -INFINITY;
+        for (int h = 0; h < n_part; ++h) mx = fmaxf(mx, rs[(size_t)h * a.rows_pad].x);
+        float z = 0.0f;
+        for (int h = 0; h < n_part; ++h) {
+            const float2 pp = rs[(size_t)h * a.rows_pad];
+            z += pp.x > -INFINITY ? pp.y * exp2f(pp.x - mx) : 0.0f;
+        }
+        sh = -(mx + log2f(z));
+    }
+    a.shift[e] = sh;
+}
+
 // ---------------------------------------------------------------------------------------------------
 // Pass 2.  Persistent CTAs; work item = (session, layer x KV head, 128-block panel).  TMEM lane = block.
 // Stationary operand: the panel's Mean-K vectors; streamed operand: the head's query rows, 256 at a time.
 constexpr int kCkShiftMax = 4096;                // query rows per (session, l, g) the shift vector can hold
 constexpr size_t kCkSmem2 = 2 * 2 * kCkAHalf + (size_t)kCkStages2 * 2 * kCkBHalf + kCkShiftMax * sizeof(float) + 1024;
 
+template <int POLY>
 __global__ void __launch_bounds__(kCkThreads, 1)
 score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_idx,
                           ChunkArgs a) {
@@ -358,7 +451,7 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 if (!item_live(item, s, lg, bp)) continue;
                 const int l = lg / a.G, g = lg % a.G;
                 const int as = li & 1;
-                if (li >= 2) ok = ptx::mbar_wait(&a_empty[as], (uint32_t)(((li >> 1) & 1) ^ 1));
+                if (li >= 2) ok = ptx::mbar_wait_suspended(&a_empty[as], (uint32_t)(((li >> 1) & 1) ^ 1));
                 if (!ok) break;
                 unsigned char* adst = smem_a + (size_t)as * 2 * kCkAHalf;
                 const int z = ((a.session_first + s) * a.L + l) * a.G + g;
@@ -367,7 +460,7 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 ptx::tma_load_3d(adst + kCkAHalf, &map_idx, 64, bp * kCkBM, z, &a_full[as]);
                 for (int qt = 0; qt < n_qtiles; ++qt, ++tt) {
                     const int st = tt % kCkStages2;
-                    if (tt >= kCkStages2) ok = ptx::mbar_wait(&b_empty[st], (uint32_t)(((tt / kCkStages2) & 1) ^ 1));
+                    if (tt >= kCkStages2) ok = ptx::mbar_wait_suspended(&b_empty[st], (uint32_t)(((tt / kCkStages2) & 1) ^ 1));
                     if (!ok) break;
                     unsigned char* dst = smem_b + (size_t)st * 2 * kCkBHalf;
                     const int m0 = s * a.M + qt * tokens_per_qtile;
@@ -388,13 +481,13 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 int s, lg, bp;
                 if (!item_live(item, s, lg, bp)) continue;
                 const int as = li & 1;
-                ok = ptx::mbar_wait(&a_full[as], (uint32_t)((li >> 1) & 1));
+                ok = ptx::mbar_wait_suspended(&a_full[as], (uint32_t)((li >> 1) & 1));
                 const uint32_t a_lo = t5::desc_lo(ptx::smem_u32(smem_a + (size_t)as * 2 * kCkAHalf));
                 const uint32_t b_lo0 = t5::desc_lo(ptx::smem_u32(smem_b));
                 for (int qt = 0; ok && qt < n_qtiles; ++qt, ++tt) {
                     const int st = tt % kCkStages2, acc = tt % kCkAccs;
-                    ok = ptx::mbar_wait(&b_full[st], (uint32_t)((tt / kCkStages2) & 1));
-                    if (ok && tt >= kCkAccs) ok = ptx::mbar_wait(&acc_empty[acc], (uint32_t)(((tt / kCkAccs) & 1) ^ 1));
+                    ok = ptx::mbar_wait_suspended(&b_full[st], (uint32_t)((tt / kCkStages2) & 1));
+                    if (ok && tt >= kCkAccs) ok = ptx::mbar_wait_suspended(&acc_empty[acc], (uint32_t)(((tt / kCkAccs) & 1) ^ 1));
                     if (!ok) break;
                     t5::fence_after();
                     issue_tile_mma(tmem_base + (uint32_t)acc * kCkBN, a_lo, b_lo0 + (uint32_t)st * (2 * kCkBHalf >> 4));
@@ -418,32 +511,18 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
             int s, lg, bp;
             if (!item_live(item, s, lg, bp)) continue;
             if (s * LG + lg != cur_head) {
-                // shifts -(max + log2 Z) of this head's query rows, merging the column slices of
-                // pass 1; -inf switches a padding row off
+                // shifts -(max + log2 Z) of this head's query rows (-inf on padding rows)
                 cur_head = s * LG + lg;
                 asm volatile("bar.sync 1, %0;" ::"n"(32 * kCkEpiWarps) : "memory");
-                const float2* rs = a.rowstat + ((size_t)cur_head * kCkSplit) * a.rows_pad;
-                for (int j = et; j < n_qtiles * kCkBN; j += 32 * kCkEpiWarps) {
-                    float sh = -INFINITY;
-                    if (j < a.rows) {
-                        float2 pp[kCkSplit];
-                        float mx = -INFINITY;
-#pragma unroll
-                        for (int h = 0; h < kCkSplit; ++h) { pp[h] = rs[(size_t)h * a.rows_pad + j]; mx = fmaxf(mx, pp[h].x); }
-                        float z = 0.0f;
-#pragma unroll
-                        for (int h = 0; h < kCkSplit; ++h) z += pp[h].x > -INFINITY ? pp[h].y * exp2f(pp[h].x - mx) : 0.0f;
-                        sh = -(mx + log2f(z));
-                    }
-                    shift[j] = sh;
-                }
+                const float* gs = a.shift + (size_t)cur_head * a.shift_stride;
+                for (int j = et; j < n_qtiles * kCkBN; j += 32 * kCkEpiWarps) shift[j] = gs[j];
                 asm volatile("bar.sync 1, %0;" ::"n"(32 * kCkEpiWarps) : "memory");
             }
             float total = 0.0f;
             for (int qt = 0; qt < n_qtiles; ++qt, ++tt) {
                 if (failed) continue;
                 const int acc = tt % kCkAccs;
-                const bool arrived = ptx::mbar_wait(&acc_full[acc], (uint32_t)((tt / kCkAccs) & 1));
+                const bool arrived = ptx::mbar_wait_suspended(&acc_full[acc], (uint32_t)((tt / kCkAccs) & 1));
                 if (!__all_sync(0xffffffffu, arrived)) {
                     if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                     failed = true;
@@ -451,9 +530,9 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 }
                 t5::fence_after();
                 const float4* sh4 = reinterpret_cast<const float4*>(shift + qt * kCkBN + half * kCkHalfCols);
-                uint32_t buf[kCkHalfCols / 32][32];
+                uint32_t buf[kCkChunks][32];
 #pragma unroll
-                for (int c = 0; c < kCkHalfCols / 32; ++c) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf[c]);
+                for (int c = 0; c < kCkChunks; ++c) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf[c]);
                 t5::ld_wait();
                 // the accumulator now lives in registers: hand it back before doing the arithmetic
                 t5::fence_before();
@@ -461,14 +540,14 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
                 float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
 #pragma unroll
-                for (int c = 0; c < kCkHalfCols / 32; ++c) {
+                for (int c = 0; c < kCkChunks; ++c) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 4) {
                         const float4 sh = sh4[c * 8 + (i >> 2)];            // same address in every lane: broadcast
-                        s0 += t5::ex2(fmaf(__uint_as_float(buf[c][i]), a.scale_log2e, sh.x));
-                        s1 += t5::ex2(fmaf(__uint_as_float(buf[c][i + 1]), a.scale_log2e, sh.y));
-                        s2 += t5::ex2(fmaf(__uint_as_float(buf[c][i + 2]), a.scale_log2e, sh.z));
-                        s3 += t5::ex2(fmaf(__uint_as_float(buf[c][i + 3]), a.scale_log2e, sh.w));
+                        s0 += ex2_mix<POLY>(fmaf(__uint_as_float(buf[c][i]), a.scale_log2e, sh.x), i);
+                        s1 += ex2_mix<POLY>(fmaf(__uint_as_float(buf[c][i + 1]), a.scale_log2e, sh.y), i + 1);
+                        s2 += ex2_mix<POLY>(fmaf(__uint_as_float(buf[c][i + 2]), a.scale_log2e, sh.z), i + 2);
+                        s3 += ex2_mix<POLY>(fmaf(__uint_as_float(buf[c][i + 3]), a.scale_log2e, sh.w), i + 3);
                     }
                 }
                 total += (s0 + s1) + (s2 + s3);
@@ -520,15 +599,19 @@ ChunkWorkspace plan_chunk_workspace(const kvmem_pool_config_t& c, int n_sessions
     w.n_panels = (w.rows + kCkBM - 1) / kCkBM;
     w.rows_pad = w.n_panels * kCkBM;
     w.nb_pad = (c.max_blocks_per_session + 255) / 256 * 256;
+    w.n_chunks = std::max(1, (w.nb_pad / kCkBN + kCkChunkTiles - 1) / kCkChunkTiles);
+    w.shift_stride = (w.rows + kCkBN - 1) / kCkBN * kCkBN;
     const size_t lg = (size_t)c.n_layers * c.n_kv_heads;
-    w.rowstat_bytes = align_up((size_t)n_sessions * lg * kCkSplit * w.rows_pad * sizeof(float2), 256);
+    w.rowstat_bytes = align_up((size_t)n_sessions * lg * w.n_chunks * kCkSplit * w.rows_pad * sizeof(float2), 256);
+    w.shift_bytes = align_up((size_t)n_sessions * lg * w.shift_stride * sizeof(float), 256);
     w.colsum_bytes = align_up((size_t)n_sessions * lg * kCkSplit * w.nb_pad * sizeof(float), 256);
     w.scores_bytes = align_up((size_t)n_sessions * c.max_blocks_per_session * sizeof(float), 256);
-    w.total = w.rowstat_bytes + w.colsum_bytes + w.scores_bytes;
+    w.total = w.rowstat_bytes + w.shift_bytes + w.colsum_bytes + w.scores_bytes;
     if (base) {
         w.rowstat = reinterpret_cast<float2*>(base);
-        w.colsum = reinterpret_cast<float*>(base + w.rowstat_bytes);
-        w.scores = reinterpret_cast<float*>(base + w.rowstat_bytes + w.colsum_bytes);
+        w.shift = reinterpret_cast<float*>(base + w.rowstat_bytes);
+        w.colsum = reinterpret_cast<float*>(base + w.rowstat_bytes + w.shift_bytes);
+        w.scores = reinterpret_cast<float*>(base + w.rowstat_bytes + w.shift_bytes + w.colsum_bytes);
     }
     return w;
 }
@@ -561,6 +644,8 @@ static bool make_index_map(PFN_cuTensorMapEncodeTiled_v12000 enc, CUtensorMap* m
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int g_chunk_poly = 5;   // every n-th exponential of the chunked passes on the FMA pipe; 0: none
+
 cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q, int M,
                                  const ChunkWorkspace& ws, float* scores, int scores_stride, cudaStream_t st) {
     const Geometry& g = p.geo;
@@ -574,29 +659,49 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
     if (!make_q_map(enc, &q_panel, q, g, n_sessions * M, kCkBM) || !make_q_map(enc, &q_tile, q, g, n_sessions * M, kCkBN) ||
         !make_index_map(enc, &idx_tile, p, kCkBN) || !make_index_map(enc, &idx_panel, p, kCkBM))
         return cudaErrorInvalidValue;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(score_chunk_rowstat_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCkSmem);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(score_chunk_colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCkSmem2);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
     ChunkArgs a{};
-    a.nblocks_dev = p.nblocks_dev; a.rowstat = ws.rowstat; a.headsum = ws.colsum; a.status = p.status_dev;
+    a.nblocks_dev = p.nblocks_dev; a.rowstat = ws.rowstat; a.shift = ws.shift; a.headsum = ws.colsum; a.status = p.status_dev;
     a.session_first = session_first; a.n_sessions = n_sessions; a.M = M; a.L = g.L; a.G = g.G; a.r = g.r;
-    a.rows = ws.rows; a.rows_pad = ws.rows_pad; a.nb_pad = ws.nb_pad;
+    a.rows = ws.rows; a.rows_pad = ws.rows_pad; a.nb_pad = ws.nb_pad; a.n_panels = ws.n_panels;
     a.n_bpanels = (max_nb + kCkBM - 1) / kCkBM;
+    a.n_chunks = ((max_nb + kCkBN - 1) / kCkBN + kCkChunkTiles - 1) / kCkChunkTiles;
+    a.shift_stride = ws.shift_stride;
     a.scale_log2e = 1.4426950408889634f / sqrtf((float)g.d);
     const int LG = g.L * g.G;
-    dim3 grid1((unsigned)ws.n_panels, (unsigned)LG, (unsigned)n_sessions);
-    score_chunk_rowstat_kernel<<<grid1, kCkThreads, kCkSmem, st>>>(q_panel, idx_tile, a);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    const int n_items = n_sessions * LG * a.n_bpanels;
-    score_chunk_colsum_kernel<<<std::min(n_items, p.sm_count), kCkThreads, kCkSmem2, st>>>(q_tile, idx_panel, a);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    const int n_items1 = n_sessions * LG * a.n_panels * a.n_chunks;
+    const int n_items2 = n_sessions * LG * a.n_bpanels;
+    const int grid1 = std::min(n_items1, p.sm_count), grid2 = std::min(n_items2, p.sm_count);
+    const long long n_shift = (long long)n_sessions * LG * a.shift_stride;
+    const int sgrid = (int)((n_shift + 255) / 256);
+    cudaError_t e = cudaSuccess;
+#define KVMEM_CHUNK_PASSES(POLY)                                                                                              \
+    do {                                                                                                                      \
+        static bool attr_done = false;                                                                                        \
+        if (!attr_done) {                                                                                                     \
+            e = cudaFuncSetAttribute(score_chunk_rowstat_kernel<POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCkSmem); \
+            if (e == cudaSuccess)                                                                                             \
+                e = cudaFuncSetAttribute(score_chunk_colsum_kernel<POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCkSmem2); \
+            if (e != cudaSuccess) return e;                                                                                   \
+            attr_done = true;                                                                                                 \
+        }                                                                                                                     \
+        score_chunk_rowstat_kernel<POLY><<<grid1, kCkThreads, kCkSmem, st>>>(q_panel, idx_tile, a);                           \
+        e = cudaGetLastError();                                                                                               \
+        if (e != cudaSuccess) return e;                                                                                       \
+        score_chunk_shift_kernel<<<sgrid, 256, 0, st>>>(a);                                                                   \
+        e = cudaGetLastError();                                                                                               \
+        if (e != cudaSuccess) return e;                                                                                       \
+        score_chunk_colsum_kernel<POLY><<<grid2, kCkThreads, kCkSmem2, st>>>(q_tile, idx_panel, a);                           \
+        e = cudaGetLastError();                                                                                               \
+        if (e != cudaSuccess) return e;                                                                                       \
+    } while (0)
+    switch (g_chunk_poly) {
+        case 2: KVMEM_CHUNK_PASSES(2); break;
+        case 3: KVMEM_CHUNK_PASSES(3); break;
+        case 4: KVMEM_CHUNK_PASSES(4); break;
+        case 5: KVMEM_CHUNK_PASSES(5); break;
+        default: KVMEM_CHUNK_PASSES(0); break;
+    }
+#undef KVMEM_CHUNK_PASSES
     dim3 fgrid((unsigned)((max_nb + 255) / 256), (unsigned)n_sessions);
     score_chunk_finish_kernel<<<fgrid, 256, 0, st>>>(ws.colsum, p.nblocks_dev, session_first, kCkSplit * LG, ws.nb_pad,
                                                      1.0f / (float)(g.L * g.H), scores, scores_stride);
