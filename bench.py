@@ -407,7 +407,7 @@ def run_native(args):
             line["e2e"]["d2h_bytes_per_step"] = ns * k * 4
             line["e2e"]["api"] = "pinned host query in, selected ids out, around kvmem_select + kvmem_materialize"
             line["gpu_launches"] = K * 5
-            line["roofline"] = {"bound": "tensor", "kernel": "score_chunk_rowstat_kernel + score_chunk_colsum_kernel + finish (kvmem_score, timed alone over 50 calls)",
+            line["roofline"] = {"bound": "tensor", "kernel": "score_chunk_rowstat_kernel + shift + score_chunk_colsum_kernel + finish (kvmem_score, timed alone over 50 calls)",
                                 "achieved": 2 * flop_alg / sel_s / 1e12, "peak": tpeak["tflops"], "unit": "TFLOP/s",
                                 "frac": 2 * flop_alg / sel_s / 1e12 / tpeak["tflops"], "peak_source": f"of {tpeak['source']} (burst)",
                                 "executed_flop_per_launch_pair": 2 * flop_alg, "algorithmic_flop": flop_alg,

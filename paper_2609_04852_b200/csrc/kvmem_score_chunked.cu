@@ -137,53 +137,111 @@ __device__ __forceinline__ void issue_tile_mma(uint32_t d_tmem, uint32_t a_lo, u
     }
 }
 
-// 2^x on the FMA and integer pipes, for the share of the exponentials that the special-function unit
-// (16 results per clock and SM, the limiter of both passes) is spared.  x = n + f with n the nearest
+// Packed fp32 arithmetic (two lanes per instruction, operands in 64-bit register pairs): the scale-and-
+// shift, the accumulation and the polynomial below cost half the issue slots of their scalar forms, which
+// matters because the epilogue is bounded by the special-function unit first and by issue slots second.
+namespace f2 {
+__device__ __forceinline__ uint64_t pk(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t pk(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpk(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ void unpk(uint64_t v, uint32_t& lo, uint32_t& hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+}  // namespace f2
+
+// 2^x for a pair, on the FMA and integer pipes: the share of the exponentials that the special-function
+// unit (16 results per clock and SM, the limiter of both passes) is spared.  x = n + f with n the nearest
 // integer and |f| <= 1/2; 2^f by a degree-4 polynomial (relative error below 3e-6), 2^n by adding n to
 // the exponent field.  Arguments below -125 (including -inf) return about 2^-125 instead of 0, which
 // is immaterial next to weights that sum to one per query row.
-__device__ __forceinline__ float ex2_poly(float x) {
-    x = fmaxf(x, -125.0f);
-    const float t = x + 12582912.0f;                 // 1.5 * 2^23: n sits in the low mantissa bits
-    const float f = x - (t - 12582912.0f);
-    float p = fmaf(0.009570100344717503f, f, 0.05591785907745361f);
-    p = fmaf(p, f, 0.240247443318367f);
-    p = fmaf(p, f, 0.6931217908859253f);
-    p = fmaf(p, f, 0.9999992847442627f);
-    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+__device__ __forceinline__ uint64_t ex2_poly2(uint64_t x2) {
+    float x0, x1;
+    f2::unpk(x2, x0, x1);
+    const uint64_t x = f2::pk(fmaxf(x0, -125.0f), fmaxf(x1, -125.0f));
+    const uint64_t t = f2::add(x, f2::pk(12582912.0f, 12582912.0f));         // 1.5 * 2^23: n sits in the low mantissa bits
+    const uint64_t n = f2::add(t, f2::pk(-12582912.0f, -12582912.0f));
+    const uint64_t f = f2::fma(n, f2::pk(-1.0f, -1.0f), x);                   // exact
+    uint64_t p = f2::fma(f2::pk(0.009570100344717503f, 0.009570100344717503f), f, f2::pk(0.05591785907745361f, 0.05591785907745361f));
+    p = f2::fma(p, f, f2::pk(0.240247443318367f, 0.240247443318367f));
+    p = f2::fma(p, f, f2::pk(0.6931217908859253f, 0.6931217908859253f));
+    p = f2::fma(p, f, f2::pk(0.9999992847442627f, 0.9999992847442627f));
+    uint32_t p0, p1, t0, t1;
+    f2::unpk(p, p0, p1);
+    f2::unpk(t, t0, t1);
+    return f2::pk(p0 + (t0 << 23), p1 + (t1 << 23));
 }
 
-// element `idx` of a tile slice takes the polynomial when every POLY-th exponential is moved off the
-// special-function unit (POLY = 0: none)
+// pair number `pidx` of a 32-column chunk takes the polynomial when every POLY-th pair of exponentials
+// is moved off the special-function unit (POLY = 0: none)
 template <int POLY>
-__device__ __forceinline__ float ex2_mix(float x, int idx) {
-    if (POLY > 0 && idx % POLY == POLY - 1) return ex2_poly(x);
-    return t5::ex2(x);
+__device__ __forceinline__ uint64_t ex2_pair(uint64_t x2, int pidx) {
+    if (POLY > 0 && pidx % POLY == POLY - 1) return ex2_poly2(x2);
+    float x0, x1;
+    f2::unpk(x2, x0, x1);
+    return f2::pk(t5::ex2(x0), t5::ex2(x1));
 }
 
 // Fold 32 raw logits of one query row into its running (max, sum-exp), exp2 domain.  `live` (ragged
 // tiles only) is how many of the 32 columns are real blocks.
 template <bool RAGGED, int POLY>
 __device__ __forceinline__ void rowstat_chunk(const uint32_t (&raw)[32], int live, float scale_log2e, float& run_m, float& run_z) {
-    float v[32];
+    if (RAGGED) {
+        // rare (the last tile of a session): scalar, every exponential on the special-function unit so
+        // that a switched-off column contributes exactly 0
+        float v[32];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = (RAGGED && i >= live) ? -INFINITY : __uint_as_float(raw[i]);
-    // maximum of the raw logits by a tree (the scale is positive, so it commutes with max)
-    float m8[8];
+        for (int i = 0; i < 32; ++i) v[i] = i >= live ? -INFINITY : __uint_as_float(raw[i]);
+        float mx = v[0];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) m8[i] = fmaxf(fmaxf(v[i], v[i + 8]), fmaxf(v[i + 16], v[i + 24]));
-    const float mx = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
+        for (int i = 1; i < 32; ++i) mx = fmaxf(mx, v[i]);
+        const float mn = fmaxf(run_m, mx * scale_log2e);
+        if (!(mn > -INFINITY)) return;
+        float sum = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) sum += t5::ex2(fmaf(v[i], scale_log2e, -mn));
+        run_z = run_z * t5::ex2(run_m - mn) + sum;
+        run_m = mn;
+        return;
+    }
+    // maximum of the raw logits by a tree of three-input maxima (the scale is positive, so it commutes with max)
+    float m[11];
+#pragma unroll
+    for (int i = 0; i < 10; ++i)
+        m[i] = f2::max3(__uint_as_float(raw[3 * i]), __uint_as_float(raw[3 * i + 1]), __uint_as_float(raw[3 * i + 2]));
+    m[10] = fmaxf(__uint_as_float(raw[30]), __uint_as_float(raw[31]));
+    const float mx = f2::max3(f2::max3(f2::max3(m[0], m[1], m[2]), f2::max3(m[3], m[4], m[5]), f2::max3(m[6], m[7], m[8])), m[9], m[10]);
     const float mn = fmaxf(run_m, mx * scale_log2e);
-    if (RAGGED && !(mn > -INFINITY)) return;
-    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+    const uint64_t sc2 = f2::pk(scale_log2e, scale_log2e), nm2 = f2::pk(-mn, -mn);
+    uint64_t acc0 = f2::pk(0.0f, 0.0f), acc1 = acc0;
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
-        // a ragged slice keeps every exponential on the special-function unit: exp2(-inf) must be 0 there
-        s0 += ex2_mix<RAGGED ? 0 : POLY>(fmaf(v[i], scale_log2e, -mn), i);
-        s1 += ex2_mix<RAGGED ? 0 : POLY>(fmaf(v[i + 1], scale_log2e, -mn), i + 1);
-        s2 += ex2_mix<RAGGED ? 0 : POLY>(fmaf(v[i + 2], scale_log2e, -mn), i + 2);
-        s3 += ex2_mix<RAGGED ? 0 : POLY>(fmaf(v[i + 3], scale_log2e, -mn), i + 3);
+        acc0 = f2::add(acc0, ex2_pair<POLY>(f2::fma(f2::pk(raw[i], raw[i + 1]), sc2, nm2), i >> 1));
+        acc1 = f2::add(acc1, ex2_pair<POLY>(f2::fma(f2::pk(raw[i + 2], raw[i + 3]), sc2, nm2), (i >> 1) + 1));
     }
+    float s0, s1, s2, s3;
+    f2::unpk(acc0, s0, s1);
+    f2::unpk(acc1, s2, s3);
     run_z = run_z * t5::ex2(run_m - mn) + ((s0 + s1) + (s2 + s3));
     run_m = mn;
 }
@@ -538,18 +596,20 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 t5::fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
-                float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+                const uint64_t sc2 = f2::pk(a.scale_log2e, a.scale_log2e);
+                uint64_t acc0 = f2::pk(0.0f, 0.0f), acc1 = acc0;
 #pragma unroll
                 for (int c = 0; c < kCkChunks; ++c) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 4) {
                         const float4 sh = sh4[c * 8 + (i >> 2)];            // same address in every lane: broadcast
-                        s0 += ex2_mix<POLY>(fmaf(__uint_as_float(buf[c][i]), a.scale_log2e, sh.x), i);
-                        s1 += ex2_mix<POLY>(fmaf(__uint_as_float(buf[c][i + 1]), a.scale_log2e, sh.y), i + 1);
-                        s2 += ex2_mix<POLY>(fmaf(__uint_as_float(buf[c][i + 2]), a.scale_log2e, sh.z), i + 2);
-                        s3 += ex2_mix<POLY>(fmaf(__uint_as_float(buf[c][i + 3]), a.scale_log2e, sh.w), i + 3);
+                        acc0 = f2::add(acc0, ex2_pair<POLY>(f2::fma(f2::pk(buf[c][i], buf[c][i + 1]), sc2, f2::pk(sh.x, sh.y)), i >> 1));
+                        acc1 = f2::add(acc1, ex2_pair<POLY>(f2::fma(f2::pk(buf[c][i + 2], buf[c][i + 3]), sc2, f2::pk(sh.z, sh.w)), (i >> 1) + 1));
                     }
                 }
+                float s0, s1, s2, s3;
+                f2::unpk(acc0, s0, s1);
+                f2::unpk(acc1, s2, s3);
                 total += (s0 + s1) + (s2 + s3);
             }
             const int b = bp * kCkBM + quarter * 32 + lane;
@@ -644,7 +704,7 @@ static bool make_index_map(PFN_cuTensorMapEncodeTiled_v12000 enc, CUtensorMap* m
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int g_chunk_poly = 5;   // every n-th exponential of the chunked passes on the FMA pipe; 0: none
+int g_chunk_poly = 4;   // every n-th exponential of the chunked passes on the FMA pipe; 0: none
 
 cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q, int M,
                                  const ChunkWorkspace& ws, float* scores, int scores_stride, cudaStream_t st) {
