@@ -3,11 +3,13 @@
 //
 // One CTA per session.  Scores are non-negative fp32, so their bit patterns order like unsigned
 // integers.  MSB-first 8-bit radix passes over the non-reserved candidates, starting at the highest
-// bit in which two candidates differ, find the value T of the k'-th largest score and how many
-// candidates are strictly larger (histograms in shared memory, 8 copies to spread the atomics).  A final ascending sweep
-// over block ids flags reserved blocks, every candidate above T, and the first (k' - above) ones
-// equal to T, i.e. equal scores go to the lower id, and compacts the flagged ids with a block-wide
-// prefix sum: the output is chronological without a sort, and identical from run to run.
+// bit in which two candidates differ, narrow down the value T of the k'-th largest score and how many
+// candidates are strictly larger (histograms in shared memory, 8 copies to spread the atomics).  The
+// passes stop as soon as the bin that holds the k'-th largest is needed whole, or holds at most 32
+// candidates, which one warp then ranks directly.  A final ascending sweep over block ids flags reserved
+// blocks, every candidate above T, and the first (k' - above) ones equal to T, i.e. equal scores go to
+// the lower id, compacts the flagged ids with a block-wide prefix sum into shared memory and writes
+// them out coalesced: the output is chronological without a sort, and identical from run to run.
 #include <algorithm>
 
 #include "kvmem_internal.cuh"
@@ -24,7 +26,9 @@ struct TopkShared {
     unsigned int hist[kHistCopies][256];
     unsigned int warp_tot[32];
     unsigned int warp_min[32], warp_max[32];
-    unsigned int prefix, remaining;
+    unsigned int bin_tot[256];
+    unsigned int small[32];                     // the candidates of the boundary bin, once there are at most 32
+    unsigned int prefix, remaining, bin_count, n_small;
 };
 
 // exclusive prefix of `val` over the CTA (thread order) and the CTA total; two barriers
@@ -62,15 +66,37 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
             int session_first, int B, kvmem_select_params_t prm, int32_t* __restrict__ sel_ids, int sel_stride,
             int32_t* __restrict__ n_sel, int32_t* __restrict__ status) {
     __shared__ TopkShared sh;
-    extern __shared__ __align__(16) unsigned int stage[];   // REG only: [kTopkThreads][kStagePitch]
+    extern __shared__ __align__(16) unsigned int stage[];   // [kTopkThreads][kStagePitch] score staging (REG), then kTopkTile output ids
     const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     const int NB = nblocks_dev[session_first + s];
     const unsigned int* bits = reinterpret_cast<const unsigned int*>(scores + (size_t)s * scores_stride);
     int32_t* out = sel_ids + (size_t)s * sel_stride;
     unsigned int vreg[kItems];
     if (REG) {
-        for (int idx = tid; idx < kTopkTile; idx += kTopkThreads)          // coalesced global reads
-            stage[(idx / kItems) * kStagePitch + (idx % kItems)] = idx < NB ? bits[idx] : 0u;
+        if ((reinterpret_cast<uintptr_t>(bits) & 15u) == 0) {
+            // coalesced 128-bit global reads, all of a thread's loads in flight before the first use
+            uint4 u[kItems / 4];
+#pragma unroll
+            for (int j = 0; j < kItems / 4; ++j) {
+                const int g4 = j * kTopkThreads + tid;                     // group of ids 4*g4 .. 4*g4 + 3
+                u[j] = make_uint4(0u, 0u, 0u, 0u);
+                if (4 * g4 + 3 < NB) {
+                    u[j] = *reinterpret_cast<const uint4*>(bits + 4 * g4);
+                } else if (4 * g4 < NB) {
+                    u[j].x = bits[4 * g4];
+                    if (4 * g4 + 1 < NB) u[j].y = bits[4 * g4 + 1];
+                    if (4 * g4 + 2 < NB) u[j].z = bits[4 * g4 + 2];
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < kItems / 4; ++j) {
+                const int g4 = j * kTopkThreads + tid;
+                *reinterpret_cast<uint4*>(&stage[(g4 / (kItems / 4)) * kStagePitch + (g4 % (kItems / 4)) * 4]) = u[j];
+            }
+        } else {
+            for (int idx = tid; idx < kTopkTile; idx += kTopkThreads)      // coalesced 32-bit reads
+                stage[(idx / kItems) * kStagePitch + (idx % kItems)] = idx < NB ? bits[idx] : 0u;
+        }
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < kItems; i += 4) {
@@ -83,7 +109,7 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
 
     // budget clamp
     long long room = (long long)prm.max_view_tokens - (long long)prm.mandatory_tokens;
-    long long kk = room > 0 ? room / B : 0;
+    long long kk = room <= 0 ? 0 : room <= 0x7fffffffll ? (long long)((int)room / B) : room / B;   // 32-bit division on the usual path
     if (prm.budget_blocks < kk) kk = prm.budget_blocks;
     if (NB < kk) kk = NB;
     if (kk < 0) kk = 0;
@@ -129,11 +155,11 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
         } else {
             const int hb = 31 - __clz(lo ^ hi);            // highest bit in which two candidates differ
             unsigned int known = hb >= 31 ? 0u : ~((2u << hb) - 1u);
-            if (tid == 0) { sh.prefix = hi & known; sh.remaining = (unsigned)kc; }
+            if (tid == 0) { sh.prefix = hi & known; sh.remaining = (unsigned)kc; sh.n_small = 0u; }
+            for (int i = tid; i < kHistCopies * 256; i += kTopkThreads) (&sh.hist[0][0])[i] = 0u;
+            __syncthreads();
             int shift = max(hb - 7, 0);
             while (true) {
-                for (int i = tid; i < kHistCopies * 256; i += kTopkThreads) (&sh.hist[0][0])[i] = 0u;
-                __syncthreads();
                 const unsigned int prefix = sh.prefix;
                 unsigned int* my_hist = sh.hist[(tid >> 5) % kHistCopies];
                 for (int base = 0; base < NB; base += kTopkTile) {
@@ -148,17 +174,20 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
                     }
                 }
                 __syncthreads();
+                if (tid < 256) {
+                    // thread t adds the copies of bin t (conflict-free) and leaves them zeroed for the next pass
+                    unsigned int t = 0;
+#pragma unroll
+                    for (int k2 = 0; k2 < kHistCopies; ++k2) { t += sh.hist[k2][tid]; sh.hist[k2][tid] = 0u; }
+                    sh.bin_tot[tid] = t;
+                }
+                __syncthreads();
                 if (tid < 32) {
                     // warp 0 walks the 256 bins from the top: lane i owns bins [255 - 8i - 7, 255 - 8i]
                     const unsigned int rem = sh.remaining;
                     unsigned int c[8], mine = 0;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        unsigned int t = 0;
-#pragma unroll
-                        for (int k2 = 0; k2 < kHistCopies; ++k2) t += sh.hist[k2][255 - 8 * lane - j];
-                        c[j] = t; mine += t;
-                    }
+                    for (int j = 0; j < 8; ++j) { c[j] = sh.bin_tot[255 - 8 * lane - j]; mine += c[j]; }
                     unsigned int inc = mine;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
@@ -171,24 +200,61 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
                     const unsigned int claim = __ballot_sync(0xffffffffu, here);
                     if (here || (claim == 0u && lane == 31)) {
                         unsigned int left = rem - before;
-                        int bin = 255 - 8 * lane;
-#pragma unroll
-                        for (int j = 0; j < 7; ++j) {
+                        int bin = 255 - 8 * lane, j = 0;
+                        for (; j < 7; ++j) {
                             if (c[j] >= left) break;
                             left -= c[j];
                             --bin;
                         }
                         sh.prefix = (prefix & ~(255u << shift)) | ((unsigned)bin << shift);
                         sh.remaining = left;                           // how many of this digit are still needed
+                        sh.bin_count = c[j];                           // how many candidates carry this digit
                     }
                 }
                 __syncthreads();
                 known |= 255u << shift;
-                if (shift == 0) break;
+                const unsigned int left = sh.remaining, in_bin = sh.bin_count;
+                if (shift == 0) { T = sh.prefix; need_eq = left; break; }
+                if (in_bin <= left) {
+                    // the whole bin is needed: everything at or above its lowest possible value is kept
+                    T = sh.prefix; need_eq = 0xffffffffu;
+                    break;
+                }
+                if (in_bin <= 32u) {
+                    // few candidates left: collect them (order does not matter) and let one warp rank them
+                    const unsigned int pfx = sh.prefix;
+                    for (int base = 0; base < NB; base += kTopkTile) {
+                        const int b0 = base + tid * kItems;
+#pragma unroll
+                        for (int i = 0; i < kItems; ++i) {
+                            const int b = b0 + i;
+                            if (b >= n_sink && b < recent_lo) {
+                                const unsigned int v = KVMEM_TOPK_VAL(base, i);
+                                if ((v & known) == pfx) {
+                                    const unsigned int slot = atomicAdd(&sh.n_small, 1u);
+                                    if (slot < 32u) sh.small[slot] = v;
+                                }
+                            }
+                        }
+                    }
+                    __syncthreads();
+                    if (tid < 32) {
+                        const unsigned int n = min(sh.n_small, 32u);
+                        const unsigned int mine = lane < n ? sh.small[lane] : 0u;
+                        unsigned int gt = 0, eq = 0;
+                        for (unsigned int j = 0; j < n; ++j) {
+                            const unsigned int o = __shfl_sync(0xffffffffu, mine, (int)j);
+                            gt += o > mine;
+                            eq += o == mine;
+                        }
+                        if (lane < n && gt < left && left <= gt + eq) { sh.prefix = mine; sh.remaining = left - gt; }
+                    }
+                    __syncthreads();
+                    T = sh.prefix; need_eq = sh.remaining;
+                    break;
+                }
                 shift = max(shift - 8, 0);
             }
-            T = sh.prefix;
-            need_eq = sh.remaining;
         }
     }
 
@@ -209,16 +275,29 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
                 }
             }
         }
-        unsigned tot_eq, tot_sel;
-        unsigned eq_rank = carry_eq + block_exclusive_scan(__popc(flags_eq), sh, tot_eq);
-        unsigned take = flags_res | flags_gt;
+        // one scan of (kept for sure | equal to T) counts, 16 bits each (a sweep covers 16,384 ids); the
+        // equal ones are kept in id order until need_eq of them are in
+        const unsigned sure = flags_res | flags_gt;
+        unsigned tot_packed;
+        const unsigned ex = block_exclusive_scan((unsigned)__popc(sure) | ((unsigned)__popc(flags_eq) << 16), sh, tot_packed);
+        unsigned eq_rank = carry_eq + (ex >> 16);
+        const unsigned tot_eq = tot_packed >> 16;
+        const unsigned eq_left_before = need_eq > carry_eq ? need_eq - carry_eq : 0u;     // equal ones this sweep may still take
+        const unsigned tot_sel = (tot_packed & 0xffffu) + min(tot_eq, eq_left_before);
+        unsigned rel = (ex & 0xffffu) + min(ex >> 16, eq_left_before);
+        unsigned take = sure;
 #pragma unroll
         for (int i = 0; i < kItems; ++i)
             if (flags_eq & (1u << i)) { if (eq_rank < need_eq) take |= 1u << i; ++eq_rank; }
-        unsigned pos = carry_sel + block_exclusive_scan(__popc(take), sh, tot_sel);
+        // compact into shared memory (scattered 4-byte writes are cheap there), then write out coalesced
+        int* outbuf = reinterpret_cast<int*>(stage);                   // at most kTopkTile ids per sweep
 #pragma unroll
         for (int i = 0; i < kItems; ++i)
-            if (take & (1u << i)) { if (pos < (unsigned)sel_stride) out[pos] = b0 + i; ++pos; }
+            if (take & (1u << i)) outbuf[rel++] = b0 + i;
+        __syncthreads();
+        for (unsigned i = tid; i < tot_sel; i += kTopkThreads)
+            if (carry_sel + i < (unsigned)sel_stride) out[carry_sel + i] = outbuf[i];
+        __syncthreads();
         carry_eq += tot_eq;
         carry_sel += tot_sel;
     }
@@ -231,20 +310,21 @@ cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, 
                         int32_t* n_sel, cudaStream_t st) {
     int max_nb = 0;
     for (int s = session_first; s < session_first + n_sessions; ++s) max_nb = std::max(max_nb, p.sess_blocks[s]);
-    if (max_nb <= kTopkTile) {
-        const size_t smem = (size_t)kTopkThreads * kStagePitch * sizeof(unsigned int);
-        static bool attr_done = false;
-        if (!attr_done) {
-            cudaError_t e = cudaFuncSetAttribute(topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return e;
-            attr_done = true;
-        }
+    const size_t smem = (size_t)kTopkThreads * kStagePitch * sizeof(unsigned int);
+    static_assert(kTopkThreads * kStagePitch >= kTopkTile, "the staging buffer doubles as the output buffer of one sweep");
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    if (max_nb <= kTopkTile)
         topk_kernel<true><<<n_sessions, kTopkThreads, smem, st>>>(scores, scores_stride, p.nblocks_dev, session_first,
                                                                   p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev);
-    } else {
-        topk_kernel<false><<<n_sessions, kTopkThreads, 0, st>>>(scores, scores_stride, p.nblocks_dev, session_first,
-                                                                p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev);
-    }
+    else
+        topk_kernel<false><<<n_sessions, kTopkThreads, smem, st>>>(scores, scores_stride, p.nblocks_dev, session_first,
+                                                                   p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev);
     return cudaGetLastError();
 }
 
