@@ -367,71 +367,74 @@ score_logits_mma_kernel(const __grid_constant__ CUtensorMap map_idx, const __nv_
 }
 
 // Merge the per-CTA statistics of every row, then R_b = (1/(L*H)) sum_rows exp2(logit - max_row) / Z_row.
-// A CTA owns 32 * kFinishU consecutive blocks.  The per-CTA (max, sum-exp) pairs are first staged in shared
-// memory with independent coalesced loads and merged there, one thread per row.  Then thread
-// (lgs, bl) sums the rows of heads lgs, lgs + 8, ... for blocks bl, bl + 32, ...
-// (independent coalesced loads), and the 8 partial sums are added in a fixed order.
-constexpr int kFinishU = 1;                      // blocks per thread
-constexpr int kFinishBlocks = 32 * kFinishU;
+// A CTA owns 32 consecutive blocks.  The session's (max, sum-exp) pairs are contiguous: they are staged
+// in shared memory by one flat 128-bit copy (all loads independent) and merged there by a group of
+// threads per row (fixed tree order).  Then thread (lgs, bl) sums the rows of heads lgs, lgs + 8, ...
+// for block bl (independent coalesced loads), and the 8 partial sums are added in a fixed order.
+constexpr int kFinishBlocks = 32;
 __global__ void __launch_bounds__(256)
 score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__ partials,
                     const int32_t* __restrict__ nblocks_dev, int session_first, int LG, int rows, int rows_pad,
                     int nb_pad, int n_parts, float inv_LH, float* __restrict__ scores, int scores_stride, int stage_parts) {
-    extern __shared__ float2 fin_smem[];  // rowstat [LG * rows] : (max, 1/Z); then staged partials [LG * rows][n_parts]
+    extern __shared__ float2 fin_smem[];  // rowstat [LG * rows_pad] : (max, 1/Z); then staged partials [LG * rows_pad][n_parts]
     float2* rowstat = fin_smem;
-    float2* staged = fin_smem + LG * rows;
+    float2* staged = fin_smem + LG * rows_pad;
     __shared__ float red[8][kFinishBlocks];
     const int s = blockIdx.y;
     const int NB = nblocks_dev[session_first + s];
     if ((int)(blockIdx.x * kFinishBlocks) >= NB) return;
-    const int n_rows = LG * rows;
+    const int n_slots = LG * rows_pad;                        // rows incl. padding: slot = lg * rows_pad + j
+    const float2* sess_parts = partials + (size_t)s * n_slots * n_parts;
     if (stage_parts) {
-        // warp w copies rows w, w + 8, ...; lane c copies pair c: independent loads, several rows in flight
-        const int wid = threadIdx.x >> 5, ln = threadIdx.x & 31;
-#pragma unroll 8
-        for (int row = wid; row < n_rows; row += 8) {
-            const int lg = row / rows, j = row % rows;
-            const float2* src = partials + (((size_t)s * LG + lg) * rows_pad + j) * n_parts;
-            for (int c = ln; c < n_parts; c += 32) staged[row * n_parts + c] = src[c];
-        }
+        const int n16 = n_slots * n_parts / 2;                // rows_pad is a multiple of 16: an even number of pairs
+        const uint4* src = reinterpret_cast<const uint4*>(sess_parts);
+        uint4* dst = reinterpret_cast<uint4*>(staged);
+#pragma unroll 4
+        for (int i = threadIdx.x; i < n16; i += 256) dst[i] = src[i];
         __syncthreads();
     }
-    for (int i = threadIdx.x; i < n_rows; i += blockDim.x) {
-        const int lg = i / rows, j = i % rows;
-        const float2* p = stage_parts ? staged + (size_t)i * n_parts : partials + (((size_t)s * LG + lg) * rows_pad + j) * n_parts;
-        float mx = -INFINITY;
-        for (int c = 0; c < n_parts; ++c) mx = fmaxf(mx, p[c].x);
-        float z = 0.0f;
-        for (int c = 0; c < n_parts; ++c) {
-            const float2 t = p[c];
-            if (t.x > -INFINITY) z += t.y * exp2f(t.x - mx);
+    // tpr threads per row (a power of two, at most 32): each merges a strided share of the parts, then a butterfly
+    int tpr = 1;
+    while (tpr < 32 && tpr * 2 * n_slots <= 256 && tpr * 2 <= n_parts) tpr *= 2;
+    for (int base = 0; base < n_slots; base += 256 / tpr) {
+        const int slot = base + (int)threadIdx.x / tpr, sub = (int)threadIdx.x % tpr;
+        const bool live = slot < n_slots && (slot % rows_pad) < rows;
+        float mx = -INFINITY, z = 0.0f;
+        if (live) {
+            const float2* pr = stage_parts ? staged + (size_t)slot * n_parts : sess_parts + (size_t)slot * n_parts;
+            for (int c = sub; c < n_parts; c += tpr) mx = fmaxf(mx, pr[c].x);
+            for (int c = sub; c < n_parts; c += tpr) {
+                const float2 t = pr[c];
+                if (t.x > -INFINITY) z += t.y * exp2f(t.x - mx);
+            }
         }
-        rowstat[i] = make_float2(mx, 1.0f / z);
+        for (int o = 1; o < tpr; o <<= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, mx, o), oz = __shfl_xor_sync(0xffffffffu, z, o);
+            const float nm = fmaxf(mx, om);
+            const float za = mx > -INFINITY ? z * exp2f(mx - nm) : 0.0f, zb = om > -INFINITY ? oz * exp2f(om - nm) : 0.0f;
+            // the same operand order on both partners, so every thread of the group ends with identical bits
+            z = (sub & o) ? zb + za : za + zb;
+            mx = nm;
+        }
+        if (live && sub == 0) rowstat[slot] = make_float2(mx, 1.0f / z);
     }
     __syncthreads();
     const int bl = threadIdx.x & 31, lgs = threadIdx.x >> 5;
     const int b0 = blockIdx.x * kFinishBlocks + bl;
-    float part[kFinishU];
-#pragma unroll
-    for (int u = 0; u < kFinishU; ++u) part[u] = 0.0f;
-    for (int lg = lgs; lg < LG; lg += 8) {
-        const float* base = logits + (((size_t)s * LG + lg) * rows_pad) * (size_t)nb_pad + b0;
-        float sub[kFinishU];
-#pragma unroll
-        for (int u = 0; u < kFinishU; ++u) sub[u] = 0.0f;
-#pragma unroll 8
-        for (int j = 0; j < rows; ++j) {
-            const float2 st = rowstat[lg * rows + j];
-            const float* rp = base + (size_t)j * nb_pad;
-#pragma unroll
-            for (int u = 0; u < kFinishU; ++u)
-                if (b0 + 32 * u < NB) sub[u] += exp2f(rp[32 * u] - st.x) * st.y;
+    float part = 0.0f;
+    if (b0 < NB) {
+        for (int lg = lgs; lg < LG; lg += 8) {
+            const float* base = logits + (((size_t)s * LG + lg) * rows_pad) * (size_t)nb_pad + b0;
+            float sub = 0.0f;
+#pragma unroll 16
+            for (int j = 0; j < rows; ++j) {
+                const float2 st = rowstat[lg * rows_pad + j];
+                sub += exp2f(base[(size_t)j * nb_pad] - st.x) * st.y;
+            }
+            part += sub;
         }
-#pragma unroll
-        for (int u = 0; u < kFinishU; ++u) part[u] += sub[u];
     }
-#pragma unroll
-    for (int u = 0; u < kFinishU; ++u) red[lgs][bl + 32 * u] = part[u];
+    red[lgs][bl] = part;
     __syncthreads();
     if (threadIdx.x < kFinishBlocks) {
         const int b = blockIdx.x * kFinishBlocks + threadIdx.x;
@@ -514,7 +517,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    size_t fsmem = (size_t)LG * ws.rows * sizeof(float2);
+    size_t fsmem = (size_t)LG * ws.rows_pad * sizeof(float2);
     const size_t stage_bytes = fsmem * n_parts;
     const int stage_parts = fsmem + stage_bytes <= 96 * 1024 ? 1 : 0;       // stage the pairs when they fit
     if (stage_parts) fsmem += stage_bytes;
