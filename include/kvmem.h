@@ -299,7 +299,9 @@ int kvmem_device_status(kvmem_pool_t* pool, int32_t* status /*HOST*/, void* stre
  * (default), 0 = 128-bit load/store copy.  "score_mode" (decode-sized queries): 1 = dot products on the
  * tensor cores (default), 0 = fp32 ALU kernel that reduces the query rows with warp shuffles.
  * "chunk_poly" (multi-token chunks): n in 2..5 = every n-th exponential of the two softmax passes is a
- * degree-4 polynomial on the FMA pipe instead of a special-function-unit instruction (default 4), 0 = none. */
+ * degree-4 polynomial on the FMA pipe instead of a special-function-unit instruction (default 4), 0 = none.
+ * "pdl": 1 = the kernels of a step are launched with programmatic stream serialization, so that the
+ * launch latency of each overlaps the tail of the one before (default), 0 = plain launches. */
 int kvmem_set_option(const char* name /*HOST*/, int32_t value);
 
 #ifdef __cplusplus

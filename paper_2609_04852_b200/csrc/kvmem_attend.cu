@@ -84,6 +84,7 @@ template <int MODE>
 __global__ void __launch_bounds__(kAttThreads + (MODE == 1 ? 32 : 0), 1)
 attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_pages, AttendArgs a) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
     constexpr bool FUSED = MODE == 1;      // a view-writer warp shares every stage with the consumers
     constexpr bool PAGED = MODE != 0;      // the producer reads pages through the block table
     extern __shared__ unsigned char smem_dyn[];
@@ -349,6 +350,8 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 __global__ void __launch_bounds__(128)
 attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, float* __restrict__ out,
                     float* __restrict__ lse, int M, int L, int H, int G, int r, int n_splits) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     const int row = blockIdx.x, z = blockIdx.y, LG = L * G;
     const int s = z / LG, lg = z % LG, l = lg / G, g = lg % G;
     const int col = threadIdx.x;
@@ -452,14 +455,14 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
     if (paged_only)
-        attend_split_kernel<2><<<grid, kAttThreads, kAttSmem, st>>>(map_k, map_v, map_pages, a);
+        launch_pdl(attend_split_kernel<2>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);
     else if (fused)
-        attend_split_kernel<1><<<grid, kAttThreads + 32, kAttSmem, st>>>(map_k, map_v, map_pages, a);
+        launch_pdl(attend_split_kernel<1>, dim3(grid), dim3(kAttThreads + 32), kAttSmem, st, map_k, map_v, map_pages, a);
     else
-        attend_split_kernel<0><<<grid, kAttThreads, kAttSmem, st>>>(map_k, map_v, map_pages, a);
+        launch_pdl(attend_split_kernel<0>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    attend_merge_kernel<<<dim3((unsigned)a.rows, (unsigned)heads), kD, 0, st>>>(a.part_o, a.part_ml, out, lse, M, g.L, g.H, g.G,
+    launch_pdl(attend_merge_kernel, dim3(dim3((unsigned)a.rows, (unsigned)heads)), dim3(kD), 0, st, a.part_o, a.part_ml, out, lse, M, g.L, g.H, g.G,
                                                                             g.r, a.n_splits);
     return cudaGetLastError();
 }

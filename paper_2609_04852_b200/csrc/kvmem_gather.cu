@@ -70,6 +70,7 @@ __device__ __forceinline__ void tile_addresses(const GatherArgs& a, int s, long 
 template <int STAGES>
 __global__ void __launch_bounds__(32)
 gather_bulk_kernel(GatherArgs a) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ uint64_t full[STAGES];
     const int s = blockIdx.y, lane = threadIdx.x;
@@ -149,6 +150,7 @@ gather_bulk_kernel(GatherArgs a) {
 
 __global__ void __launch_bounds__(256)
 gather_ldst_kernel(GatherArgs a) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
     const int s = blockIdx.y;
     const int NB = a.nblocks_dev[a.session_first + s];
     const int n_blk = usable_blocks(a, s);
@@ -178,6 +180,7 @@ gather_ldst_kernel(GatherArgs a) {
     }
 }
 
+int g_pdl = 1;           // programmatic dependent launch of the step's kernels
 int g_gather_mode = 1;   // 1: TMA bulk ring, 0: ld/st
 
 cudaError_t launch_gather(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids,
@@ -205,11 +208,11 @@ cudaError_t launch_gather(const kvmem_pool& p, int session_first, int n_sessions
         const int per_sm = std::max(1, (int)((220 * 1024) / (smem + 1024)));
         const int ctas = std::max(1, p.sm_count * per_sm / n_sessions);
         dim3 grid((unsigned)ctas, (unsigned)n_sessions);
-        gather_bulk_kernel<STAGES><<<grid, 32, smem, st>>>(a);
+        launch_pdl(gather_bulk_kernel<STAGES>, dim3(grid), dim3(32), smem, st, a);
     } else {
         const int ctas = std::max(1, p.sm_count * 8 / n_sessions);
         dim3 grid((unsigned)ctas, (unsigned)n_sessions);
-        gather_ldst_kernel<<<grid, 256, 0, st>>>(a);
+        launch_pdl(gather_ldst_kernel, dim3(grid), dim3(256), 0, st, a);
     }
     return cudaGetLastError();
 }

@@ -72,6 +72,30 @@ void set_error(const char* fmt, ...);
 extern int g_score_mode;    // 1: tensor-core decode scoring (default), 0: fp32 ALU + warp-shuffle kernel
 extern int g_chunk_poly;    // chunked scoring: every n-th exponential on the FMA pipe (0: all on the special-function unit)
 extern int g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
+extern int g_pdl;           // 1: the kernels of a step are launched with programmatic stream serialization (default), 0: plain launches
+
+// Programmatic dependent launch.  A kernel launched through launch_pdl may be scheduled while the previous
+// kernel of the stream is still running; its first statement is pdl_wait(), which returns once that
+// kernel (and, because every such kernel waits first, everything before it) has completed and its
+// writes are visible.  pdl_trigger() lets the next kernel's CTAs take their places early.  What is
+// hidden is the launch latency between the short dependent kernels of a step.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // ---- kernel launchers (each defined next to its kernel) ----------------------------------------
 // All return cudaGetLastError() after the launch.

@@ -79,6 +79,7 @@ struct GatherRopeArgs {
 
 __global__ void __launch_bounds__(256)
 gather_rope_kernel(GatherRopeArgs a) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
     const int s = blockIdx.y;
     const int NB = a.nblocks_dev[a.session_first + s];
     int n_blk = a.n_sel[s];
@@ -148,7 +149,7 @@ cudaError_t launch_gather_rope(const kvmem_pool& p, int session_first, int n_ses
     a.LG = g.L * g.G; a.B = g.B; a.d = g.d; a.cap_tokens = view_cap_tokens; a.first_position = first_position;
     a.rope_positions = p.cfg.rope_max_positions; a.page_elems = p.lay.page_elems;
     const int ctas = std::max(1, p.sm_count * 8 / n_sessions);
-    gather_rope_kernel<<<dim3((unsigned)ctas, (unsigned)n_sessions), 256, 0, st>>>(a);
+    launch_pdl(gather_rope_kernel, dim3(dim3((unsigned)ctas, (unsigned)n_sessions)), dim3(256), 0, st, a);
     return cudaGetLastError();
 }
 

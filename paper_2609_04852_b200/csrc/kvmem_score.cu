@@ -90,6 +90,8 @@ score_logits_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                     int max_bps, size_t index_elems_per_session, float* __restrict__ logits,
                     float2* __restrict__ partials, int rows, int rows_pad, int nb_pad, int n_parts,
                     float scale_log2e, int32_t* __restrict__ status) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     constexpr int SH = (RP == 16) ? 0 : (RP == 8) ? 1 : 2;   // lanes per finished row = 1 << SH
     constexpr int RPW = (RP + 7) / 8;                        // rows whose statistics one warp carries
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -228,6 +230,8 @@ score_logits_mma_kernel(const __grid_constant__ CUtensorMap map_idx, const __nv_
                         const int32_t* __restrict__ nblocks_dev, int session_first, int M, int L, int H, int G,
                         int max_bps, float* __restrict__ logits, float2* __restrict__ partials, int rows, int rows_pad,
                         int nb_pad, int n_parts, float scale_log2e, int32_t* __restrict__ status) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     constexpr int RP = 16;
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint64_t full_bar[kScoreStages];
@@ -376,6 +380,8 @@ __global__ void __launch_bounds__(256)
 score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__ partials,
                     const int32_t* __restrict__ nblocks_dev, int session_first, int LG, int rows, int rows_pad,
                     int nb_pad, int n_parts, float inv_LH, float* __restrict__ scores, int scores_stride, int stage_parts) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     extern __shared__ float2 fin_smem[];  // rowstat [LG * rows_pad] : (max, 1/Z); then staged partials [LG * rows_pad][n_parts]
     float2* rowstat = fin_smem;
     float2* staged = fin_smem + LG * rows_pad;
@@ -494,7 +500,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
             if (e != cudaSuccess) return e;
             attr_done = true;
         }
-        score_logits_mma_kernel<<<grid, kScoreThreads, smem + 1024, st>>>(
+        launch_pdl(score_logits_mma_kernel, dim3(grid), dim3(kScoreThreads), smem + 1024, st, 
             map_idx, q, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, ws.logits, ws.partials, ws.rows,
             ws.rows_pad, ws.nb_pad, n_parts, scale_log2e, p.status_dev);
     } else {
@@ -506,7 +512,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
             if (e != cudaSuccess) return e;                                                                            \
             attr_done = true;                                                                                          \
         }                                                                                                              \
-        score_logits_kernel<RP><<<grid, kScoreThreads, smem, st>>>(                                                    \
+        launch_pdl(score_logits_kernel<RP>, dim3(grid), dim3(kScoreThreads), smem, st,                                                     \
             q, p.index, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, p.lay.index_elems_per_session,      \
             ws.logits, ws.partials, ws.rows, ws.rows_pad, ws.nb_pad, n_parts, scale_log2e, p.status_dev);              \
     } while (0)
@@ -526,7 +532,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
         if (e != cudaSuccess) return e;
     }
     dim3 fgrid((unsigned)((max_nb + kFinishBlocks - 1) / kFinishBlocks), (unsigned)n_sessions);
-    score_finish_kernel<<<fgrid, 256, fsmem, st>>>(ws.logits, ws.partials, p.nblocks_dev, session_first, LG, ws.rows,
+    launch_pdl(score_finish_kernel, dim3(fgrid), dim3(256), fsmem, st, ws.logits, ws.partials, p.nblocks_dev, session_first, LG, ws.rows,
                                                    ws.rows_pad, ws.nb_pad, n_parts, 1.0f / (float)(g.L * g.H),
                                                    scores, scores_stride, stage_parts);
     return cudaGetLastError();

@@ -257,6 +257,8 @@ template <int POLY>
 __global__ void __launch_bounds__(kCkThreads, 1)
 score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_idx,
                            ChunkArgs a) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint64_t a_full, a_empty, b_full[kCkStages1], b_empty[kCkStages1], acc_full[kCkAccs], acc_empty[kCkAccs];
     __shared__ uint32_t tmem_base_slot;
@@ -421,6 +423,8 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 // tile runs and column slices in a fixed order; -inf switches a padding row off in pass 2.
 __global__ void __launch_bounds__(256)
 score_chunk_shift_kernel(ChunkArgs a) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     const int LG = a.L * a.G;
     const long long total = (long long)a.n_sessions * LG * a.shift_stride;
     const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;
@@ -456,6 +460,8 @@ template <int POLY>
 __global__ void __launch_bounds__(kCkThreads, 1)
 score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_idx,
                           ChunkArgs a) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint64_t a_full[2], a_empty[2], b_full[kCkStages2], b_empty[kCkStages2], acc_full[kCkAccs], acc_empty[kCkAccs];
     __shared__ uint32_t tmem_base_slot;
@@ -630,6 +636,8 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
 __global__ void __launch_bounds__(256)
 score_chunk_finish_kernel(const float* __restrict__ headsum, const int32_t* __restrict__ nblocks_dev, int session_first,
                           int LG, int nb_pad, float inv_LH, float* __restrict__ scores, int scores_stride) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     const int s = blockIdx.y;
     const int NB = nblocks_dev[session_first + s];
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
@@ -744,13 +752,13 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
             if (e != cudaSuccess) return e;                                                                                   \
             attr_done = true;                                                                                                 \
         }                                                                                                                     \
-        score_chunk_rowstat_kernel<POLY><<<grid1, kCkThreads, kCkSmem, st>>>(q_panel, idx_tile, a);                           \
+        launch_pdl(score_chunk_rowstat_kernel<POLY>, dim3(grid1), dim3(kCkThreads), kCkSmem, st, q_panel, idx_tile, a);                           \
         e = cudaGetLastError();                                                                                               \
         if (e != cudaSuccess) return e;                                                                                       \
-        score_chunk_shift_kernel<<<sgrid, 256, 0, st>>>(a);                                                                   \
+        launch_pdl(score_chunk_shift_kernel, dim3(sgrid), dim3(256), 0, st, a);                                                                   \
         e = cudaGetLastError();                                                                                               \
         if (e != cudaSuccess) return e;                                                                                       \
-        score_chunk_colsum_kernel<POLY><<<grid2, kCkThreads, kCkSmem2, st>>>(q_tile, idx_panel, a);                           \
+        launch_pdl(score_chunk_colsum_kernel<POLY>, dim3(grid2), dim3(kCkThreads), kCkSmem2, st, q_tile, idx_panel, a);                           \
         e = cudaGetLastError();                                                                                               \
         if (e != cudaSuccess) return e;                                                                                       \
     } while (0)
@@ -763,7 +771,7 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
     }
 #undef KVMEM_CHUNK_PASSES
     dim3 fgrid((unsigned)((max_nb + 255) / 256), (unsigned)n_sessions);
-    score_chunk_finish_kernel<<<fgrid, 256, 0, st>>>(ws.colsum, p.nblocks_dev, session_first, kCkSplit * LG, ws.nb_pad,
+    launch_pdl(score_chunk_finish_kernel, dim3(fgrid), dim3(256), 0, st, ws.colsum, p.nblocks_dev, session_first, kCkSplit * LG, ws.nb_pad,
                                                      1.0f / (float)(g.L * g.H), scores, scores_stride);
     return cudaGetLastError();
 }

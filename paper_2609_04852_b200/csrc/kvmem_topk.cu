@@ -65,6 +65,8 @@ __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* __restrict__ nblocks_dev,
             int session_first, int B, kvmem_select_params_t prm, int32_t* __restrict__ sel_ids, int sel_stride,
             int32_t* __restrict__ n_sel, int32_t* __restrict__ status) {
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     __shared__ TopkShared sh;
     extern __shared__ __align__(16) unsigned int stage[];   // [kTopkThreads][kStagePitch] score staging (REG), then kTopkTile output ids
     const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
@@ -320,10 +322,10 @@ cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, 
         attr_done = true;
     }
     if (max_nb <= kTopkTile)
-        topk_kernel<true><<<n_sessions, kTopkThreads, smem, st>>>(scores, scores_stride, p.nblocks_dev, session_first,
+        launch_pdl(topk_kernel<true>, dim3(n_sessions), dim3(kTopkThreads), smem, st, scores, scores_stride, p.nblocks_dev, session_first,
                                                                   p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev);
     else
-        topk_kernel<false><<<n_sessions, kTopkThreads, smem, st>>>(scores, scores_stride, p.nblocks_dev, session_first,
+        launch_pdl(topk_kernel<false>, dim3(n_sessions), dim3(kTopkThreads), smem, st, scores, scores_stride, p.nblocks_dev, session_first,
                                                                    p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev);
     return cudaGetLastError();
 }
