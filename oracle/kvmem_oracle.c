@@ -381,3 +381,112 @@ void kvo_working_set_delta(const int32_t* prev, int64_t n_prev, const int32_t* n
     }
     counts[0] = (int32_t)nR; counts[1] = (int32_t)nL; counts[2] = (int32_t)nE;
 }
+
+/* =======================================================================================
+ * Execution cache with working-set reuse and bounded delta re-RoPE (Sec. 4.4, "Retrieval-Aware
+ * Hierarchical Reuse" and the paragraph on the two views).
+ *
+ * The cache is `cap` slots (the paper's active GPU pages); a slot holds one block: K encoded for the
+ * block's current compact position and an unchanged copy of V.  State per slot: slot_block (block id,
+ * -1 = empty), slot_pos (compact block index the keys are encoded for), slot_cnt (delta re-RoPE
+ * operations since the keys were last built from raw K).  One update takes the cache from the
+ * previous working set to `sel` (ascending ids, n_sel <= cap), in the paper's order:
+ *   1. delta (Eq. "kvmem-working-set-delta"): a resident block that is selected again is retained
+ *      and keeps its slot; every other slot is reclaimed;
+ *   2. incoming blocks, in ascending id order, take the free slots in ascending slot order; their
+ *      keys are built from raw K with RoPE at the new compact position, their values are copied;
+ *   3. a retained block whose compact position changed is re-encoded: by a delta rotation of its
+ *      current keys by (new - old) positions while slot_cnt < max_delta (slot_cnt += 1), otherwise
+ *      rebuilt from raw K at the new position (slot_cnt = 0).  A retained block that did not move is
+ *      left alone.
+ * view_slots[j] = slot of the j-th selected block (the execution view's page table).
+ * stats = (retained and unmoved, delta re-RoPEd, rebuilt, incoming).
+ * Readings: the slot policy (lowest free slot, ascending ids) and the counter semantics (a limit on
+ * operations between reconstructions, reset by a reconstruction) are ours; the paper fixes neither.
+ * cacheK / cacheV: [cap][B][L][G][d] (token-major, like the repository pages of this file).
+ * d <= 1024.  Returns -1 if n_sel > cap or the compact positions leave the table.
+ */
+int kvo_view_cache_update(const bf16_t* pagesK, const bf16_t* pagesV, const int32_t* table, const int32_t* sel,
+                          int64_t n_sel, int B, int L, int G, int d, int64_t cap, int64_t max_delta,
+                          int64_t first_pos, const float* tab, int64_t n_pos, bf16_t* cacheK, bf16_t* cacheV,
+                          int32_t* slot_block, int32_t* slot_pos, int32_t* slot_cnt, int32_t* view_slots,
+                          int32_t* stats) {
+    if (n_sel > cap || first_pos < 0 || first_pos + n_sel * B > n_pos) return -1;
+    const size_t page = (size_t)B * L * G * d;
+    const int n_vec = L * G;
+    stats[0] = stats[1] = stats[2] = stats[3] = 0;
+    for (int64_t j = 0; j < n_sel; ++j) view_slots[j] = -1;
+    /* 1. retained blocks keep their slot, all other slots are reclaimed */
+    for (int64_t s = 0; s < cap; ++s) {
+        int64_t found = -1;
+        if (slot_block[s] >= 0)
+            for (int64_t j = 0; j < n_sel; ++j)
+                if (sel[j] == slot_block[s]) { found = j; break; }
+        if (found >= 0) view_slots[found] = (int32_t)s;
+        else slot_block[s] = -1;
+    }
+    /* 2. incoming blocks take the lowest free slots */
+    int64_t next_free = 0;
+    for (int64_t j = 0; j < n_sel; ++j) {
+        if (view_slots[j] >= 0) continue;
+        while (slot_block[next_free] >= 0) ++next_free;
+        const int64_t s = next_free;
+        const size_t src = (size_t)table[sel[j]] * page, dst = (size_t)s * page;
+        for (int t = 0; t < B; ++t)
+            for (int v = 0; v < n_vec; ++v) {
+                const size_t o = ((size_t)t * n_vec + v) * d;
+                kvo_rotate_vec(pagesK + src + o, cacheK + dst + o, d, tab + (size_t)(first_pos + j * B + t) * (d / 2) * 2, 0);
+            }
+        memcpy(cacheV + dst, pagesV + src, page * sizeof(bf16_t));
+        slot_block[s] = sel[j]; slot_pos[s] = (int32_t)j; slot_cnt[s] = 0;
+        view_slots[j] = (int32_t)s;
+        stats[3] += 1;
+    }
+    /* 3. retained blocks that moved */
+    for (int64_t j = 0; j < n_sel; ++j) {
+        const int64_t s = view_slots[j];
+        if (slot_pos[s] == j) continue;                            /* unmoved, or loaded in step 2 */
+        const size_t dst = (size_t)s * page;
+        if (slot_cnt[s] < max_delta) {
+            const int64_t delta = (j - slot_pos[s]) * B;           /* positions; the same for every token of the block */
+            const int64_t mag = delta < 0 ? -delta : delta;
+            for (int t = 0; t < B; ++t)
+                for (int v = 0; v < n_vec; ++v) {
+                    const size_t o = ((size_t)t * n_vec + v) * d;
+                    bf16_t tmp[1024];
+                    memcpy(tmp, cacheK + dst + o, (size_t)d * sizeof(bf16_t));
+                    kvo_rotate_vec(tmp, cacheK + dst + o, d, tab + (size_t)mag * (d / 2) * 2, delta < 0);
+                }
+            slot_cnt[s] += 1;
+            stats[1] += 1;
+        } else {
+            const size_t src = (size_t)table[sel[j]] * page;
+            for (int t = 0; t < B; ++t)
+                for (int v = 0; v < n_vec; ++v) {
+                    const size_t o = ((size_t)t * n_vec + v) * d;
+                    kvo_rotate_vec(pagesK + src + o, cacheK + dst + o, d, tab + (size_t)(first_pos + j * B + t) * (d / 2) * 2, 0);
+                }
+            slot_cnt[s] = 0;
+            stats[2] += 1;
+        }
+        slot_pos[s] = (int32_t)j;
+    }
+    stats[0] = (int32_t)n_sel - stats[1] - stats[2] - stats[3];
+    return 0;
+}
+
+/* The execution view as attention sees it: slot view_slots[j] supplies view tokens [j*B, (j+1)*B).
+ * viewK / viewV: [L][G][cap_tokens][d]. */
+void kvo_view_cache_view(const bf16_t* cacheK, const bf16_t* cacheV, const int32_t* view_slots, int64_t n_sel,
+                         int B, int L, int G, int d, bf16_t* viewK, bf16_t* viewV, int64_t cap_tokens) {
+    const size_t page = (size_t)B * L * G * d;
+    for (int64_t j = 0; j < n_sel; ++j)
+        for (int t = 0; t < B; ++t)
+            for (int l = 0; l < L; ++l)
+                for (int g = 0; g < G; ++g) {
+                    const size_t s = (size_t)view_slots[j] * page + (((size_t)t * L + l) * G + g) * d;
+                    const size_t o = (((size_t)l * G + g) * cap_tokens + (size_t)j * B + t) * d;
+                    memcpy(viewK + o, cacheK + s, (size_t)d * sizeof(bf16_t));
+                    memcpy(viewV + o, cacheV + s, (size_t)d * sizeof(bf16_t));
+                }
+}

@@ -64,6 +64,10 @@ def lib():
         L.kvo_gather_rope.restype = i32
         L.kvo_working_set_delta.argtypes = [p, i64, p, i64, p, p, p, p]
         L.kvo_working_set_delta.restype = None
+        L.kvo_view_cache_update.argtypes = [p, p, p, p, i64, i32, i32, i32, i32, i64, i64, i64, p, i64, p, p, p, p, p, p, p]
+        L.kvo_view_cache_update.restype = i32
+        L.kvo_view_cache_view.argtypes = [p, p, p, i64, i32, i32, i32, i32, p, p, i64]
+        L.kvo_view_cache_view.restype = None
         L.kvo_threads.argtypes = []
         L.kvo_threads.restype = i32
         _lib = L
@@ -230,3 +234,45 @@ def working_set_delta(prev: np.ndarray, nxt: np.ndarray):
     cnt = np.zeros(3, np.int32)
     lib().kvo_working_set_delta(_ptr(prev), len(prev), _ptr(nxt), len(nxt), _ptr(ret), _ptr(inc), _ptr(out), _ptr(cnt))
     return ret[: cnt[0]].copy(), inc[: cnt[1]].copy(), out[: cnt[2]].copy()
+
+
+# ---- execution cache: working-set reuse with bounded delta re-RoPE -----------------------------------
+
+class ViewCache:
+    """Oracle state of the execution cache (Sec. 4.4): `cap` slots of one block each, token-major
+    [cap][B][L][G][d] keys (encoded for their compact position) and values, plus the slot records."""
+
+    def __init__(self, repo: Repository, cap: int):
+        _, B, L, G, d = repo.pagesK.shape
+        self.cap, self.dims = cap, (B, L, G, d)
+        self.K = np.zeros((cap, B, L, G, d), np.uint16)
+        self.V = np.zeros((cap, B, L, G, d), np.uint16)
+        self.slot_block = np.full(cap, -1, np.int32)
+        self.slot_pos = np.zeros(cap, np.int32)
+        self.slot_cnt = np.zeros(cap, np.int32)
+        self.view_slots = np.full(cap, -1, np.int32)
+        self.n_view = 0
+
+    def update(self, repo: Repository, table: np.ndarray, sel: np.ndarray, max_delta: int, first_pos: int,
+               tab: np.ndarray) -> np.ndarray:
+        """Move the cache to the working set `sel`; returns stats (unmoved, delta re-RoPEd, rebuilt, incoming)."""
+        B, L, G, d = self.dims
+        sel = np.ascontiguousarray(sel, np.int32)
+        stats = np.zeros(4, np.int32)
+        rc = lib().kvo_view_cache_update(_ptr(repo.pagesK), _ptr(repo.pagesV), _ptr(np.ascontiguousarray(table)), _ptr(sel),
+                                         len(sel), B, L, G, d, self.cap, max_delta, first_pos, _ptr(tab), tab.shape[0],
+                                         _ptr(self.K), _ptr(self.V), _ptr(self.slot_block), _ptr(self.slot_pos),
+                                         _ptr(self.slot_cnt), _ptr(self.view_slots), _ptr(stats))
+        if rc != 0:
+            raise ValueError("selection larger than the cache, or compact positions outside the RoPE table")
+        self.n_view = len(sel)
+        return stats
+
+    def view(self, cap_tokens: int) -> Tuple[np.ndarray, np.ndarray]:
+        """The execution view in attention order: [L][G][cap_tokens][d] keys and values."""
+        B, L, G, d = self.dims
+        viewK = np.zeros((L, G, cap_tokens, d), np.uint16)
+        viewV = np.zeros((L, G, cap_tokens, d), np.uint16)
+        lib().kvo_view_cache_view(_ptr(self.K), _ptr(self.V), _ptr(self.view_slots), self.n_view, B, L, G, d,
+                                  _ptr(viewK), _ptr(viewV), cap_tokens)
+        return viewK, viewV
