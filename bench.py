@@ -406,7 +406,7 @@ def run_native(args):
             line["e2e"]["h2d_bytes_per_step"] = rows * spec.head_dim * 2
             line["e2e"]["d2h_bytes_per_step"] = ns * k * 4
             line["e2e"]["api"] = "pinned host query in, selected ids out, around kvmem_select + kvmem_materialize"
-            line["gpu_launches"] = K * 5
+            line["gpu_launches"] = K * 6
             line["roofline"] = {"bound": "tensor", "kernel": "score_chunk_rowstat_kernel + shift + score_chunk_colsum_kernel + finish (kvmem_score, timed alone over 50 calls)",
                                 "achieved": 2 * flop_alg / sel_s / 1e12, "peak": tpeak["tflops"], "unit": "TFLOP/s",
                                 "frac": 2 * flop_alg / sel_s / 1e12 / tpeak["tflops"], "peak_source": f"of {tpeak['source']} (burst)",
@@ -419,6 +419,146 @@ def run_native(args):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- execution cache (working-set reuse)
+
+def run_cache(args):
+    """Position-consistent step with the execution view kept across steps (Sec. 4.4): de-RoPE the query, select,
+    update the cache as a working-set delta (bounded delta re-RoPE), attend over the cache through its page table."""
+    from paper_2609_04852_b200 import SelectParams, budget_blocks, set_option
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1:
+        raise SystemExit("--cache is a single-GPU measurement")
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    for opt in args.option:
+        name, _, value = opt.partition("=")
+        set_option(name, int(value))
+    base = CONFIGS[args.workload]
+    if not base.attend or base.n_sessions != 1:
+        raise SystemExit("--cache is measured on the single-session attend workloads")
+    pool, spec = fill_pool(base, device, rope=True)
+    M, B, H, d = spec.n_q_tokens, spec.block_tokens, spec.n_q_heads, spec.head_dim
+    prm = SelectParams(**select_params(spec))
+    k = budget_blocks(prm, B, spec.n_blocks)
+    q_dev = [make_queries(spec, i, drift=args.drift).to(device) for i in range(spec.n_query_sets)]
+    sel = torch.zeros(1, k, dtype=torch.int32, device=device)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=device)
+    cache = pool.new_view_cache(k, args.max_delta, 0)
+    out, lse = pool.new_outputs(1, M)
+    q_pos = torch.arange(k * B, k * B + M, dtype=torch.int32, device=device)
+    q_raw = torch.empty_like(q_dev[0])
+    stream = torch.cuda.current_stream(device)
+
+    def step(i, ev=None):
+        q = q_dev[i % len(q_dev)]
+        pool.rope_rotate(q.view(M, H, d), q_pos, out=q_raw.view(M, H, d), inverse=True)
+        pool.select(q_raw, prm, sel, n_sel)
+        if ev is not None:
+            ev[0].record(stream)
+        cache.update(0, sel[0], n_sel)
+        if ev is not None:
+            ev[1].record(stream)
+        cache.attend(q[0], out[0], lse[0])
+        if ev is not None:
+            ev[2].record(stream)
+
+    # steady-state statistics of the working-set delta (untimed pass over two rounds of the query sets)
+    acc = torch.zeros(4, dtype=torch.int64, device=device)
+    n_stat = 2 * len(q_dev)
+    for i in range(n_stat):
+        step(i)
+        if i >= len(q_dev):
+            acc += cache.stats
+    torch.cuda.synchronize(device)
+    stats = (acc.cpu().double() / (n_stat - len(q_dev))).tolist()
+    for i in range(max(args.warmup, 3)):
+        step(n_stat + i)
+    torch.cuda.synchronize(device)
+    assert pool.device_status() == 0
+    sampler = ClockSampler(device.index)
+    sampler.start()
+    time.sleep(0.25)
+    K = args.steps
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    begins = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(device)
+    t0 = time.time()
+    e0.record(stream)
+    for i in range(K):
+        begins[i].record(stream)
+        step(n_stat + 3 + i, marks[i])
+    e1.record(stream)
+    torch.cuda.synchronize(device)
+    t1 = time.time()
+    if t1 - t0 < 0.5:       # keep the load up long enough for the clock sampler
+        t0 = time.time()
+        i = 0
+        while time.time() < t0 + 0.6:
+            step(i); i += 1
+            if i % 50 == 0:
+                torch.cuda.synchronize(device)
+        torch.cuda.synchronize(device)
+        t1 = time.time()
+    sampler.window(t0, t1)
+    clocks = sampler.stop()
+    assert pool.device_status() == 0
+    total_ms = e0.elapsed_time(e1)
+    med = statistics.median
+    sel_ms = med([begins[i].elapsed_time(marks[i][0]) for i in range(K)])
+    upd_ms = med([marks[i][0].elapsed_time(marks[i][1]) for i in range(K)])
+    att_ms = med([marks[i][1].elapsed_time(marks[i][2]) for i in range(K)])
+    # end to end: query from pinned host memory, O and LSE back to the host, every step
+    q_pin = [make_queries(spec, i, drift=args.drift).pin_memory() for i in range(spec.n_query_sets)]
+    out_pin, lse_pin = torch.empty(out.shape).pin_memory(), torch.empty(lse.shape).pin_memory()
+    q_stage = torch.empty_like(q_dev[0])
+    Ke = min(K, 200)
+    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ee0.record(stream)
+    for i in range(Ke):
+        q_stage.copy_(q_pin[i % len(q_pin)], non_blocking=True)
+        pool.rope_rotate(q_stage.view(M, H, d), q_pos, out=q_raw.view(M, H, d), inverse=True)
+        pool.select(q_raw, prm, sel, n_sel)
+        cache.update(0, sel[0], n_sel)
+        cache.attend(q_stage[0], out[0], lse[0])
+        out_pin.copy_(out, non_blocking=True)
+        lse_pin.copy_(lse, non_blocking=True)
+        torch.cuda.synchronize(device)
+    ee1.record(stream)
+    torch.cuda.synchronize(device)
+    peaks = measured_peaks()
+    page_bytes = 2 * spec.n_layers * spec.n_kv_heads * B * d * 2
+    # bytes the update has to move: an incoming block is read and written (K and V), a re-encoded one K only
+    upd_bytes = stats[3] * 2 * page_bytes + (stats[1] + stats[2]) * page_bytes
+    att_bytes = k * page_bytes
+    rows = M * spec.n_layers * H
+    line = {
+        "metric": METRIC, "value": K / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic (seeded; shapes of the paper's agent workspaces)",
+        "config": {"workload": f"{spec.name}: 1 session x {spec.n_blocks} blocks of {B} tokens, {M} query token(s), budget {k} blocks, "
+                               f"execution cache of {k} slots, query drift {args.drift}, at most {args.max_delta} delta re-RoPE "
+                               "operations between reconstructions",
+                   "history_tokens": spec.tokens, "view_tokens": k * B, "query_sets": len(q_dev),
+                   "l2": "no flush: every step streams far more than the 126 MB L2",
+                   "parallelism": "1 session on 1 GPU",
+                   "calls": "kvmem_rope_rotate(q) + kvmem_select + kvmem_view_cache_update + kvmem_view_cache_attend"},
+        "e2e": {"value": Ke / (ee0.elapsed_time(ee1) * 1e-3), "unit": UNIT, "steps": Ke,
+                "h2d_bytes_per_step": rows * d * 2, "d2h_bytes_per_step": rows * d * 4 + rows * 4,
+                "api": "pinned host query in, host O and LSE out, around the four calls"},
+        "gpu_launches": K * 8, "clocks": clocks,
+        "cache": {"avg_blocks_per_step": {"unmoved": stats[0], "delta_roped": stats[1], "rebuilt": stats[2], "incoming": stats[3]},
+                  "update_bytes_per_step": upd_bytes, "view_bytes": att_bytes},
+        "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<2> + merge over the cache slots (kvmem_view_cache_attend)",
+                     "achieved": att_bytes / (att_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": att_bytes / (att_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+                     "algorithmic_bytes_per_launch": att_bytes, "avg_launch_ms": att_ms, "traffic": None},
+        "update_roofline": {"kernel": "view_cache_plan_kernel + view_cache_apply_kernel", "achieved_gbs": upd_bytes / (upd_ms * 1e-3) / 1e9,
+                            "frac": upd_bytes / (upd_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "avg_ms": upd_ms},
+        "stages_ms": {"select": sel_ms, "cache_update": upd_ms, "attend": att_ms},
+    }
+    print(json.dumps(line), flush=True)
 
 
 # ----------------------------------------------------------------------------- oracle arm / CPU baseline
@@ -533,6 +673,10 @@ def main():
     ap.add_argument("--unfused", action="store_true", help="separate kvmem_materialize and kvmem_view_attend calls")
     ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
                     help="kernel-variant switch passed to kvmem_set_option (e.g. chunk_poly=0)")
+    ap.add_argument("--cache", action="store_true", help="position-consistent step over an execution cache kept across "
+                    "steps (working-set reuse, bounded delta re-RoPE); not the headline step")
+    ap.add_argument("--drift", type=float, default=1.0, help="--cache: how far consecutive queries move (1 = independent)")
+    ap.add_argument("--max-delta", type=int, default=4, help="--cache: delta re-RoPE operations between reconstructions")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)
     args = ap.parse_args()
@@ -541,7 +685,10 @@ def main():
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the native arm")
-        run_native(args)
+        if args.cache:
+            run_cache(args)
+        else:
+            run_native(args)
 
 
 if __name__ == "__main__":

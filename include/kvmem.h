@@ -242,6 +242,47 @@ int kvmem_working_set_delta(kvmem_pool_t* pool, int32_t n_sessions, const int32_
                             int32_t* incoming /*DEVICE*/, int32_t* outgoing /*DEVICE*/, int32_t* counts /*DEVICE*/,
                             void* stream);
 
+/* Execution cache: the execution view kept across steps, with working-set reuse and bounded delta
+ * re-RoPE (Sec. 4.4: the two views; "Retrieval-Aware Hierarchical Reuse"; Eq. "kvmem-working-set-delta").
+ *
+ * The cache is cap_blocks slots ("active GPU pages") in caller-owned DEVICE memory of
+ * kvmem_view_cache_bytes() bytes, 256-byte aligned, for ONE session.  A slot holds one block in the
+ * pool's page format ([K|V][L][G][block_tokens][d] bf16): K encoded for the block's current compact
+ * position, V unchanged.  The pool's pages must hold raw (position-independent) keys and the pool must
+ * have a rotary table.  kvmem_view_cache_update moves the cache from the previous working set to
+ * sel_ids (ascending, as kvmem_select writes them; *n_sel <= cap_blocks):
+ *   - a block that is resident and selected again keeps its slot (no data moves); every other slot is
+ *     reclaimed; incoming blocks, in ascending id order, take the free slots in ascending slot order,
+ *     their K built from raw K with RoPE at compact position first_position + j*block_tokens + t (j =
+ *     index in sel_ids), their V copied;
+ *   - a retained block whose index j changed has its keys re-encoded: rotated in place by
+ *     (j_new - j_old) * block_tokens positions while fewer than max_delta_ropes such rotations have been
+ *     applied since its keys were last built from raw K, otherwise rebuilt from raw K (counter reset).
+ *     max_delta_ropes = 0 rebuilds every moved block, i.e. the cache always equals
+ *     kvmem_materialize_rope's view.
+ * Rotation arithmetic as in kvmem_rope_rotate (fp32 products and sums, no fused multiply-add, one
+ * rounding to bf16), so cache contents are reproducible bit for bit.
+ * stats (DEVICE int32[4], may be NULL) = (retained and unmoved, delta re-RoPEd, rebuilt, incoming).
+ * Records inside the cache, at the byte offsets kvmem_view_cache_layout writes to offsets[6] (HOST):
+ *   [0] pages  [1] slot_block int32[cap] (-1 = empty)  [2] slot_pos int32[cap]  [3] slot_cnt int32[cap]
+ *   [4] view_slots int32[cap]: slot of the j-th selected block (the view's page table)  [5] n_view int32.
+ * kvmem_view_cache_attend: GQA decode attention over the cached view through view_slots (no compaction);
+ * q [M][L][H][d] bf16, out/lse/workspace/scale as in kvmem_view_attend with n_sessions = 1.
+ * Errors: KVMEM_E_STATE without a rotary table; KVMEM_E_INVALID for bad pointers, cap_blocks outside
+ * [1, 32768] or positions outside the table; KVMEM_E_CAPACITY if cache_bytes is too small.  A selection
+ * longer than cap_blocks or an id outside the session is clamped / skipped on the device and reported as
+ * KVMEM_E_DEVICE_RANGE by kvmem_device_status.  Calls on one cache must be ordered (same stream). */
+size_t kvmem_view_cache_bytes(const kvmem_pool_t* pool, int32_t cap_blocks);
+int kvmem_view_cache_layout(const kvmem_pool_t* pool, int32_t cap_blocks, size_t* offsets /*HOST [6]*/);
+int kvmem_view_cache_reset(kvmem_pool_t* pool, void* cache /*DEVICE*/, size_t cache_bytes, int32_t cap_blocks, void* stream);
+int kvmem_view_cache_update(kvmem_pool_t* pool, int32_t session, const int32_t* sel_ids /*DEVICE*/,
+                            const int32_t* n_sel /*DEVICE*/, void* cache /*DEVICE*/, size_t cache_bytes,
+                            int32_t cap_blocks, int32_t max_delta_ropes, int32_t first_position,
+                            int32_t* stats /*DEVICE, may be NULL*/, void* stream);
+int kvmem_view_cache_attend(kvmem_pool_t* pool, const void* q /*DEVICE*/, int32_t n_q_tokens, void* cache /*DEVICE*/,
+                            size_t cache_bytes, int32_t cap_blocks, float scale, float* out /*DEVICE*/,
+                            float* lse /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
 /* kvmem_view_attend for callers that cannot allocate device memory.  (The paper has no counterpart.)
  * Who needs it: a serving process that gave all of HBM to its KV pool at start-up and runs with
  * its allocator frozen, a plug-in that only ever sees the buffers of one request, or a latency path

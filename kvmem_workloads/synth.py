@@ -189,12 +189,19 @@ def kv_blocks(spec: WorkloadSpec, session: int, b0: int, b1: int, device="cpu"
     return k.to(torch.bfloat16), v.to(torch.bfloat16)
 
 
-def make_queries(spec: WorkloadSpec, qset: int = 0) -> torch.Tensor:
-    """Query set ``qset``: bf16 ``[n_sessions][M][L][H][d]`` on the CPU."""
+def make_queries(spec: WorkloadSpec, qset: int = 0, drift: float = 1.0) -> torch.Tensor:
+    """Query set ``qset``: bf16 ``[n_sessions][M][L][H][d]`` on the CPU.
+
+    ``drift`` < 1 models consecutive agent steps whose queries stay close: the free part of query set
+    ``qset`` is sqrt(1 - drift^2) * (that of set 0) + drift * (its own), so consecutive selections overlap
+    more the smaller ``drift`` is; 1.0 (default) gives independent query sets."""
     M, L, H, d, r = spec.n_q_tokens, spec.n_layers, spec.n_q_heads, spec.head_dim, spec.group
     out = torch.empty(spec.n_sessions, M, L, H, d, dtype=torch.float32)
     for s in range(spec.n_sessions):
         z = _normal(0, M * L * H * d, _key(spec.seed, _S_Q, s, qset), "cpu").view(M, L, H, d)
+        if drift < 1.0 and qset != 0:
+            z0 = _normal(0, M * L * H * d, _key(spec.seed, _S_Q, s, 0), "cpu").view(M, L, H, d)
+            z = math.sqrt(1.0 - drift * drift) * z0 + drift * z
         u = planted_directions(spec, s)                       # [L][G][d]
         u_h = u.repeat_interleave(r, dim=1)                   # query head h looks at KV head h // r
         out[s] = z + math.sqrt(d) * u_h.view(1, L, H, d)

@@ -592,6 +592,87 @@ int kvmem_working_set_delta(kvmem_pool_t* p, int32_t n_sessions, const int32_t* 
     return KVMEM_OK;
 }
 
+// ---- execution cache: working-set reuse with bounded delta re-RoPE ----
+
+static int cache_ok(kvmem_pool_t* p, const void* cache, size_t cache_bytes, int32_t cap_blocks, const char* who) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (p->cfg.rope_max_positions <= 0) { set_error("%s: the pool was created without rotary support", who); return KVMEM_E_STATE; }
+    if (cap_blocks < 1 || cap_blocks > 32768) { set_error("%s: cap_blocks must be in [1, 32768]", who); return KVMEM_E_INVALID; }
+    if (!cache || !aligned(cache, 256)) { set_error("%s: cache is null or not 256-byte aligned", who); return KVMEM_E_INVALID; }
+    const size_t need = cache_layout(p->lay.page_elems, cap_blocks).total;
+    if (cache_bytes < need) { set_error("%s: cache holds %zu bytes, %zu needed", who, cache_bytes, need); return KVMEM_E_CAPACITY; }
+    return KVMEM_OK;
+}
+
+size_t kvmem_view_cache_bytes(const kvmem_pool_t* p, int32_t cap_blocks) {
+    if (!p || cap_blocks < 1 || cap_blocks > 32768) return 0;
+    return cache_layout(p->lay.page_elems, cap_blocks).total;
+}
+
+int kvmem_view_cache_layout(const kvmem_pool_t* p, int32_t cap_blocks, size_t* offsets) {
+    if (!p || !offsets || cap_blocks < 1 || cap_blocks > 32768) { set_error("kvmem_view_cache_layout: bad argument"); return KVMEM_E_INVALID; }
+    const CacheLayout c = cache_layout(p->lay.page_elems, cap_blocks);
+    offsets[0] = c.pages; offsets[1] = c.slot_block; offsets[2] = c.slot_pos; offsets[3] = c.slot_cnt;
+    offsets[4] = c.view_slots; offsets[5] = c.n_view;
+    return KVMEM_OK;
+}
+
+int kvmem_view_cache_reset(kvmem_pool_t* p, void* cache, size_t cache_bytes, int32_t cap_blocks, void* stream) {
+    const int rc = cache_ok(p, cache, cache_bytes, cap_blocks, "kvmem_view_cache_reset");
+    if (rc != KVMEM_OK) return rc;
+    cudaError_t e = launch_view_cache_reset(*p, cache, cap_blocks, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("execution-cache reset kernel launch", e);
+    return KVMEM_OK;
+}
+
+int kvmem_view_cache_update(kvmem_pool_t* p, int32_t session, const int32_t* sel_ids, const int32_t* n_sel, void* cache,
+                            size_t cache_bytes, int32_t cap_blocks, int32_t max_delta_ropes, int32_t first_position,
+                            int32_t* stats, void* stream) {
+    const int rc = cache_ok(p, cache, cache_bytes, cap_blocks, "kvmem_view_cache_update");
+    if (rc != KVMEM_OK) return rc;
+    if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;
+    if (!sel_ids || !n_sel) { set_error("kvmem_view_cache_update: null pointer"); return KVMEM_E_INVALID; }
+    if (max_delta_ropes < 0) { set_error("max_delta_ropes must be non-negative"); return KVMEM_E_INVALID; }
+    const int64_t last = (int64_t)first_position + (int64_t)cap_blocks * p->cfg.block_tokens;
+    if (first_position < 0 || last > p->cfg.rope_max_positions) {
+        set_error("compact positions [%d, %lld) outside the rotary table [0, %d)", first_position, (long long)last,
+                  p->cfg.rope_max_positions);
+        return KVMEM_E_INVALID;
+    }
+    if (p->cfg.head_dim % 16 != 0) { set_error("rotary kernels need head_dim to be a multiple of 16"); return KVMEM_E_UNSUPPORTED; }
+    cudaError_t e = launch_view_cache_update(*p, session, sel_ids, n_sel, cache, cap_blocks, max_delta_ropes, first_position,
+                                             stats, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("execution-cache update kernel launch", e);
+    return KVMEM_OK;
+}
+
+int kvmem_view_cache_attend(kvmem_pool_t* p, const void* q, int32_t n_q_tokens, void* cache, size_t cache_bytes,
+                            int32_t cap_blocks, float scale, float* out, float* lse, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+    const int rc = cache_ok(p, cache, cache_bytes, cap_blocks, "kvmem_view_cache_attend");
+    if (rc != KVMEM_OK) return rc;
+    if (!q || !out || !lse || !workspace || !aligned(q, 16) || !aligned(workspace, 256) || !aligned(out, 16)) {
+        set_error("kvmem_view_cache_attend: null or misaligned pointer");
+        return KVMEM_E_INVALID;
+    }
+    if (n_q_tokens < 1) { set_error("n_q_tokens must be positive"); return KVMEM_E_INVALID; }
+    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
+        set_error("attention kernel is built for head_dim 128 and 64-token blocks");
+        return KVMEM_E_UNSUPPORTED;
+    }
+    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
+    AttendPlan plan = plan_attend(p->cfg, 1, n_q_tokens, p->sm_count);
+    if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
+    PagedSource src{};
+    view_cache_paged_source(*p, cache, cap_blocks, &src);
+    const int64_t cap_tokens = (int64_t)cap_blocks * p->cfg.block_tokens;
+    cudaError_t e = launch_attend(*p, 1, (const __nv_bfloat16*)q, n_q_tokens, nullptr, nullptr, (int)cap_tokens, src.n_sel, scale,
+                                  out, lse, workspace, (cudaStream_t)stream, src.sel_ids, cap_blocks, 0, &src);
+    if (e != cudaSuccess) return cuda_fail("execution-cache attention kernel launch", e);
+    return KVMEM_OK;
+}
+
 int kvmem_get_index(kvmem_pool_t* p, int32_t session, const void** index, int32_t* n_blocks) {
     if (!pool_ok(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;

@@ -400,15 +400,15 @@ static bool make_view_map(CUtensorMap* map, const __nv_bfloat16* view, int heads
 }
 
 // page pool [max_blocks * 2 * L*G * 64 rows][128] bf16 as a 2-D tensor; box = 64 dims x 64 tokens, 128-byte swizzle
-static bool make_pages_map(CUtensorMap* map, const kvmem_pool& p) {
+static bool make_pages_map(CUtensorMap* map, const kvmem_pool& p, const __nv_bfloat16* pages, int n_pages) {
     PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
     if (!enc) return false;
     const Geometry& g = p.geo;
-    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)g.max_blocks * 2 * g.L * g.G * kTile};
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)n_pages * 2 * g.L * g.G * kTile};
     cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
     cuuint32_t box[2] = {64, (cuuint32_t)kTile};
     cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.pages, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(pages), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -417,13 +417,14 @@ static bool make_pages_map(CUtensorMap* map, const kvmem_pool& p) {
 cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M,
                           const __nv_bfloat16* view_k, const __nv_bfloat16* view_v, int view_cap_tokens,
                           const int32_t* n_sel, float scale, float* out, float* lse, void* workspace,
-                          cudaStream_t st, const int32_t* sel_ids, int sel_stride, int session_first) {
+                          cudaStream_t st, const int32_t* sel_ids, int sel_stride, int session_first, const PagedSource* alt) {
     const Geometry& g = p.geo;
     const int LG = g.L * g.G, heads = n_sessions * LG;
     const bool fused = sel_ids != nullptr;
     const bool paged_only = fused && view_k == nullptr;     // copy-free: attend straight over the pages
     CUtensorMap map_k, map_v, map_pages;
-    if (fused && !make_pages_map(&map_pages, p)) return cudaErrorInvalidValue;
+    // alt: the pages and tables are not the pool's own (attention over an execution cache)
+    if (fused && !make_pages_map(&map_pages, p, alt ? alt->pages : p.pages, alt ? alt->n_pages : g.max_blocks)) return cudaErrorInvalidValue;
     if (paged_only) {
         map_k = map_pages; map_v = map_pages;               // unused by this mode
     } else if (!make_view_map(&map_k, view_k, heads, view_cap_tokens) || !make_view_map(&map_v, view_v, heads, view_cap_tokens)) {
@@ -453,6 +454,9 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     a.scale_log2e = sc * 1.4426950408889634f;
     a.sel_ids = sel_ids; a.tables = p.tables; a.nblocks_dev = p.nblocks_dev;
     a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
+    if (alt) {
+        a.tables = alt->tables; a.nblocks_dev = alt->nblocks_dev; a.max_bps = alt->table_stride; a.max_blocks = alt->n_pages;
+    }
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
     if (paged_only)
         launch_pdl(attend_split_kernel<2>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);

@@ -142,6 +142,27 @@ constexpr int kMaxDecodeTokens = 16;   // more query tokens than this take the t
 cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q, int M,
                                  const ChunkWorkspace& ws, float* scores, int scores_stride, cudaStream_t st);
 
+// Execution cache (working-set reuse with bounded delta re-RoPE): offsets inside the caller's buffer
+struct CacheLayout {
+    size_t pages, slot_block, slot_pos, slot_cnt, view_slots, n_view, iota, action, old_pos, free_list, total;
+};
+CacheLayout cache_layout(size_t page_elems, int cap);
+// where paged attention finds its pages and tables when they are not the pool's own
+struct PagedSource {
+    const __nv_bfloat16* pages;
+    int n_pages;
+    const int32_t* tables;
+    int table_stride;
+    const int32_t* nblocks_dev;
+    const int32_t* sel_ids;
+    const int32_t* n_sel;
+};
+cudaError_t launch_view_cache_reset(const kvmem_pool& p, void* cache, int cap, cudaStream_t st);
+cudaError_t launch_view_cache_update(const kvmem_pool& p, int session, const int32_t* sel_ids, const int32_t* n_sel,
+                                     void* cache, int cap, int max_delta, int first_position, int32_t* stats,
+                                     cudaStream_t st);
+void view_cache_paged_source(const kvmem_pool& p, void* cache, int cap, PagedSource* src);
+
 cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, const float* scores,
                         int scores_stride, const kvmem_select_params_t& prm, int32_t* sel_ids, int sel_stride,
                         int32_t* n_sel, cudaStream_t st);
@@ -160,6 +181,7 @@ AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tok
 cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M,
                           const __nv_bfloat16* view_k, const __nv_bfloat16* view_v, int view_cap_tokens,
                           const int32_t* n_sel, float scale, float* out, float* lse, void* workspace,
-                          cudaStream_t st, const int32_t* sel_ids = nullptr, int sel_stride = 0, int session_first = 0);
+                          cudaStream_t st, const int32_t* sel_ids = nullptr, int sel_stride = 0, int session_first = 0,
+                          const PagedSource* alt = nullptr);
 
 }  // namespace kvmem

@@ -78,6 +78,11 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_rope_rotate": (C.c_int, [vp, vp, vp, C.c_int64, i32, vp, i32, vp]),
         "kvmem_materialize_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, i32, vp]),
         "kvmem_working_set_delta": (C.c_int, [vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]),
+        "kvmem_view_cache_bytes": (sz, [vp, i32]),
+        "kvmem_view_cache_layout": (C.c_int, [vp, i32, C.POINTER(sz)]),
+        "kvmem_view_cache_reset": (C.c_int, [vp, vp, sz, i32, vp]),
+        "kvmem_view_cache_update": (C.c_int, [vp, i32, vp, vp, vp, sz, i32, i32, i32, vp, vp]),
+        "kvmem_view_cache_attend": (C.c_int, [vp, vp, i32, vp, sz, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_paged_attend": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
         "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
@@ -99,7 +104,8 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_device_status", "kvmem_set_option", "kvmem_step_staging_bytes", "kvmem_recall_step_host",
             "kvmem_view_attend_static", "kvmem_materialize_attend",
             "kvmem_paged_attend", "kvmem_append_blocks_rope", "kvmem_rope_rotate", "kvmem_materialize_rope",
-            "kvmem_working_set_delta", "kvmem_score")
+            "kvmem_working_set_delta", "kvmem_score", "kvmem_view_cache_bytes", "kvmem_view_cache_layout",
+            "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend")
 
 
 def _check(status: int) -> None:
@@ -209,6 +215,10 @@ class Pool:
                                                 _dev(next_ids, torch.int32), _dev(n_next, torch.int32), stride,
                                                 ret.data_ptr(), inc.data_ptr(), out.data_ptr(), cnt.data_ptr(), _stream()))
         return ret, inc, out, cnt
+
+    # ---- execution cache: working-set reuse with bounded delta re-RoPE
+    def new_view_cache(self, cap_blocks: int, max_delta_ropes: int, first_position: int = 0) -> "ViewCache":
+        return ViewCache(self, cap_blocks, max_delta_ropes, first_position)
 
     # ---- position-consistent keys
     def append_blocks_rope(self, session: int, k_roped: torch.Tensor, v: torch.Tensor, block_pos0: Sequence[int],
@@ -379,3 +389,54 @@ class Pool:
         st = C.c_int32()
         _check(self.lib.kvmem_device_status(self.handle, C.byref(st), _stream()))
         return st.value
+
+
+class ViewCache:
+    """The execution view kept across steps for one session: `cap_blocks` slots of one block each (keys
+    encoded for their compact position, values unchanged), updated as a working-set delta."""
+
+    def __init__(self, pool: Pool, cap_blocks: int, max_delta_ropes: int, first_position: int = 0):
+        self.pool, self.cap, self.max_delta, self.first_position = pool, cap_blocks, max_delta_ropes, first_position
+        need = pool.lib.kvmem_view_cache_bytes(pool.handle, cap_blocks)
+        if need == 0:
+            raise KvmemError(E_INVALID, "cap_blocks must be in [1, 32768]")
+        self.buf = torch.empty(need, dtype=torch.uint8, device=pool.device)
+        offs = (C.c_size_t * 6)()
+        _check(pool.lib.kvmem_view_cache_layout(pool.handle, cap_blocks, offs))
+        self.offsets = list(offs)
+        self.stats = torch.zeros(4, dtype=torch.int32, device=pool.device)
+        _check(pool.lib.kvmem_view_cache_reset(pool.handle, self.buf.data_ptr(), self.buf.numel(), cap_blocks, _stream()))
+
+    def update(self, session: int, sel_ids: torch.Tensor, n_sel: torch.Tensor) -> None:
+        """sel_ids int32 [>= n] ascending (one session's row), n_sel int32 [1]; stats land in self.stats."""
+        p = self.pool
+        _check(p.lib.kvmem_view_cache_update(p.handle, session, _dev(sel_ids, torch.int32), _dev(n_sel, torch.int32),
+                                             self.buf.data_ptr(), self.buf.numel(), self.cap, self.max_delta,
+                                             self.first_position, self.stats.data_ptr(), _stream()))
+
+    def attend(self, q: torch.Tensor, out: torch.Tensor, lse: torch.Tensor, scale: float = 0.0) -> None:
+        """q bf16 [M][L][H][d] (one session) -> out fp32 [M][L][H][d], lse fp32 [M][L][H]."""
+        p = self.pool
+        M = q.shape[0]
+        ws = p.attend_workspace(1, M)
+        _check(p.lib.kvmem_view_cache_attend(p.handle, _dev(q, torch.bfloat16), M, self.buf.data_ptr(), self.buf.numel(),
+                                             self.cap, scale, _dev(out, torch.float32), _dev(lse, torch.float32),
+                                             ws.data_ptr(), ws.numel(), _stream()))
+
+    # ---- inspection (copies)
+    def _ints(self, which: int, n: int) -> torch.Tensor:
+        o = self.offsets[which]
+        return self.buf[o:o + 4 * n].view(torch.int32).clone()
+
+    def records(self):
+        """(slot_block, slot_pos, slot_cnt, view_slots, n_view) as CPU tensors / int."""
+        torch.cuda.synchronize(self.pool.device)
+        return (self._ints(1, self.cap).cpu(), self._ints(2, self.cap).cpu(), self._ints(3, self.cap).cpu(),
+                self._ints(4, self.cap).cpu(), int(self._ints(5, 1).cpu()[0]))
+
+    def pages(self) -> torch.Tensor:
+        """bf16 [cap][2][L][G][B][d]: the slots in the pool's page format (a view of the cache buffer)."""
+        c = self.pool.cfg
+        n = self.cap * 2 * c.n_layers * c.n_kv_heads * c.block_tokens * c.head_dim
+        o = self.offsets[0]
+        return self.buf[o:o + 2 * n].view(torch.bfloat16).view(self.cap, 2, c.n_layers, c.n_kv_heads, c.block_tokens, c.head_dim)
