@@ -217,6 +217,12 @@ def run_native(args):
             pool.select(q_raw, prm, sel, n_sel)
             if ev is not None:
                 ev[0].record(stream)
+            if args.paged:      # copy-free: raw key tiles are RoPE'd in shared memory on their way to the tensor cores
+                pool.paged_attend_rope(q, sel, n_sel, out, lse, 0)
+                if ev is not None:
+                    ev[1].record(stream)
+                    ev[2].record(stream)
+                return
             pool.materialize_rope(sel, n_sel, view, 0)
             if ev is not None:
                 ev[1].record(stream)
@@ -299,8 +305,11 @@ def run_native(args):
             q_stage.copy_(q_pin[i % len(q_pin)], non_blocking=True)
             pool.rope_rotate(q_stage.view(M, H, d), q_pos, out=q_raw.view(M, H, d), inverse=True)
             pool.select(q_raw, prm, sel, n_sel)
-            pool.materialize_rope(sel, n_sel, view, 0)
-            pool.view_attend(q_stage, view, n_sel, out, lse)
+            if args.paged:
+                pool.paged_attend_rope(q_stage, sel, n_sel, out, lse, 0)
+            else:
+                pool.materialize_rope(sel, n_sel, view, 0)
+                pool.view_attend(q_stage, view, n_sel, out, lse)
             out_pin.copy_(out, non_blocking=True)
             lse_pin.copy_(lse, non_blocking=True)
             torch.cuda.synchronize(device)
@@ -358,7 +367,9 @@ def run_native(args):
                        "l2": "flushed between steps (256 MiB write)" if flush is not None else
                              "no flush: every step streams far more than the 126 MB L2",
                        "parallelism": f"{world} independent session replica(s), one per GPU",
-                       "calls": "kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_rope + kvmem_view_attend" if args.rope else
+                       "calls": "kvmem_rope_rotate(q) + kvmem_select + kvmem_paged_attend_rope (copy-free, keys RoPE'd in shared memory)"
+                                if args.rope and args.paged else
+                                "kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_rope + kvmem_view_attend" if args.rope else
                                 "kvmem_select + kvmem_paged_attend (NO materialize: copy-free view variant)" if args.paged else
                                 "kvmem_select + kvmem_materialize_attend" if fused else
                                 "kvmem_select + kvmem_materialize" + (" + kvmem_view_attend" if spec.attend else "")},
@@ -366,9 +377,10 @@ def run_native(args):
                     "h2d_bytes_per_step": rows * spec.head_dim * 2,
                     "d2h_bytes_per_step": rows * spec.head_dim * 4 + rows * 4,
                     "api": "kvmem_recall_step_host (pinned host query in, host O and LSE out, synchronous)"},
-            "gpu_launches": K * (KERNELS_PER_STEP - (1 if fused else 0) + (1 if args.rope else 0)),
+            "gpu_launches": K * (KERNELS_PER_STEP - (1 if fused or args.paged else 0) + (1 if args.rope else 0)),
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "gather_rope_kernel (kvmem_materialize_rope)" if args.rope else
+            "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<3> + merge (kvmem_paged_attend_rope)" if args.rope and args.paged else
+                                                   "gather_rope_kernel (kvmem_materialize_rope)" if args.rope else
                                                    "attend_split_kernel<2> + merge (kvmem_paged_attend)" if args.paged else
                                                    "attend_split_kernel<1> + merge (kvmem_materialize_attend: view written while attended)"
                                                    if fused else "gather_bulk_kernel (kvmem_materialize)",

@@ -226,6 +226,21 @@ int kvmem_paged_attend(kvmem_pool_t* pool, int32_t session_first, int32_t n_sess
                        const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
                        void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
+/* Copy-free execution view with position-consistent keys (Sec. 4.4: the view is a page table over the
+ * physical pages, and RoPE is applied to raw K at the block's assigned compact position): as
+ * kvmem_paged_attend, but every key tile is rotated in shared memory, between its arrival from the
+ * pages and its use, to compact position first_position + j*block_tokens + t (j = index in sel_ids),
+ * with the arithmetic of kvmem_rope_rotate.  out and lse equal kvmem_view_attend's on the view
+ * kvmem_materialize_rope would build from the same ids; nothing is written besides out and lse.  The
+ * pool's pages must hold raw keys and q must carry RoPE at its own position.  HBM traffic: one read per
+ * view byte plus the rotary table rows of the view's positions.
+ * Extra errors: KVMEM_E_STATE without a rotary table; KVMEM_E_INVALID if
+ * [first_position, first_position + sel_stride*block_tokens) leaves the table. */
+int kvmem_paged_attend_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
+                            int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
+                            const int32_t* n_sel /*DEVICE*/, int32_t first_position, float scale, float* out /*DEVICE*/,
+                            float* lse /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
 /* Working-set delta between two consecutive steps (Eq. "kvmem-working-set-delta", Sec. 4.4):
  *     retained R = W_next n W_prev,   incoming L = W_next \ W_prev,   outgoing E = W_prev \ W_next.
  * prev_ids / next_ids are the ascending id lists kvmem_select wrote at the two steps, a block's slot is

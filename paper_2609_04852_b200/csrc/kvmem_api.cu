@@ -546,9 +546,9 @@ int kvmem_materialize_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_s
     return KVMEM_OK;
 }
 
-int kvmem_paged_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
-                       const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, float scale, float* out, float* lse,
-                       void* workspace, size_t workspace_bytes, void* stream) {
+static int paged_attend_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                             const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, int32_t rope_first_position,
+                             float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
     if (!pool_ok(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q || !sel_ids || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(workspace, 256) || !aligned(out, 16)) {
@@ -572,9 +572,32 @@ int kvmem_paged_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_session
     const int64_t cap_tokens = (int64_t)sel_stride * p->cfg.block_tokens;
     if (cap_tokens > 0x7fffffffll) { set_error("sel_stride too large"); return KVMEM_E_INVALID; }
     cudaError_t e = launch_attend(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, nullptr, nullptr, (int)cap_tokens, n_sel,
-                                  scale, out, lse, workspace, (cudaStream_t)stream, sel_ids, sel_stride, session_first);
+                                  scale, out, lse, workspace, (cudaStream_t)stream, sel_ids, sel_stride, session_first, nullptr,
+                                  rope_first_position);
     if (e != cudaSuccess) return cuda_fail("paged attention kernel launch", e);
     return KVMEM_OK;
+}
+
+int kvmem_paged_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                       const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, float scale, float* out, float* lse,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    return paged_attend_impl(p, session_first, n_sessions, q, n_q_tokens, sel_ids, sel_stride, n_sel, -1, scale, out, lse,
+                             workspace, workspace_bytes, stream);
+}
+
+int kvmem_paged_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                            const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, int32_t first_position,
+                            float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
+    const int64_t last = (int64_t)first_position + (int64_t)sel_stride * p->cfg.block_tokens;
+    if (first_position < 0 || sel_stride < 1 || last > p->cfg.rope_max_positions) {
+        set_error("compact positions [%d, %lld) outside the rotary table [0, %d)", first_position, (long long)last,
+                  p->cfg.rope_max_positions);
+        return KVMEM_E_INVALID;
+    }
+    return paged_attend_impl(p, session_first, n_sessions, q, n_q_tokens, sel_ids, sel_stride, n_sel, first_position, scale, out,
+                             lse, workspace, workspace_bytes, stream);
 }
 
 int kvmem_working_set_delta(kvmem_pool_t* p, int32_t n_sessions, const int32_t* prev_ids, const int32_t* n_prev,

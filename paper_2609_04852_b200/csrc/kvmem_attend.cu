@@ -16,6 +16,7 @@
 
 #include "kvmem_internal.cuh"
 #include "kvmem_ptx.cuh"
+#include "kvmem_rope.cuh"
 
 namespace kvmem {
 
@@ -24,8 +25,12 @@ constexpr int kAttConsumers = 8;
 constexpr int kAttGroups = 2;                   // consumer groups; kAttStages % kAttGroups == 0
 static_assert(kAttStages % kAttGroups == 0, "each group must own whole stages");
 constexpr int kAttThreads = (kAttConsumers + 1) * 32;
+constexpr int kAttRopeStages = 4;               // data stages in that mode: two stages' room holds the rotary rows of two tiles
 constexpr int kTile = 64;                       // tokens per tile == block_tokens
 constexpr int kD = 128;
+constexpr int kTabBytes = kTile * (kD / 2) * 8; // (cos, sin) fp32 of 64 pairs for 64 positions: 32 KiB
+static_assert(kAttRopeStages % kAttGroups == 0 && kAttRopeStages * 4 * kTile * 128 + 2 * kTabBytes <= kAttStages * 4 * kTile * 128,
+              "the rotary mode's data stages and table ring must fit the ring of the other modes");
 constexpr int kHalfBytes = kTile * 128;         // one 64-dim half of a tile: 64 rows x 128 B
 constexpr int kStageBytes = 4 * kHalfBytes;     // K lo, K hi, V lo, V hi
 constexpr int kMaxSplits = 64;
@@ -46,6 +51,9 @@ struct AttendArgs {
     const int32_t* tables;       // [max_sessions][max_bps]
     const int32_t* nblocks_dev;  // [max_sessions]
     int session_first, sel_stride, max_bps, max_blocks;
+    // position-consistent copy-free view (attend_split_kernel<3>): raw keys are rotated in shared memory
+    const float2* rope;          // [rope_positions][64] (cos, sin)
+    int first_position;          // compact position of view token 0
 };
 
 AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, int sm_count) {
@@ -78,6 +86,11 @@ static int choose_splits(int heads, int max_tiles, int sms) {
 //         extra warp stores every tile into the view with TMA while the consumers attend over it,
 //         so the view is assembled and attended in one pass: 1 read + 1 write per view byte
 //         instead of 2 reads + 1 write.
+// MODE 3: MODE 2 with position-consistent keys (Sec. 4.4: RoPE is applied to raw K at the block's compact
+//         position): the rotary rows of a tile's 64 positions ride along in a small ring of their own,
+//         and each consumer warp rotates its key fragments in registers between ldmatrix and the MMAs, with
+//         the arithmetic of kvmem_rope_rotate (fp32 products and sums, no fused multiply-add, one rounding
+//         to bf16).  The result equals attention over kvmem_materialize_rope's view and no byte is written.
 // MODE 2: copy-free execution view (Sec. 5.3 "Copy-free execution-view assembly"): tiles are read from
 //         the pages through the block table and attended over; no contiguous view is written.
 template <int MODE>
@@ -87,8 +100,10 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     pdl_wait();        // everything earlier in the stream is complete and visible from here on
     constexpr bool FUSED = MODE == 1;      // a view-writer warp shares every stage with the consumers
     constexpr bool PAGED = MODE != 0;      // the producer reads pages through the block table
+    constexpr bool ROPE = MODE == 3;       // the consumers re-encode their key fragments in registers before the MMAs
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages];
+    constexpr int STAGES = ROPE ? kAttRopeStages : kAttStages;   // the rotary mode gives two stages' room to the table ring
+    __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages], tab_full[kAttGroups], tab_empty[kAttGroups];
     __shared__ float merge_m[kAttConsumers][kRowsPad], merge_l[kAttConsumers][kRowsPad];
 
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -105,7 +120,11 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     const int n_tiles = t1 - t0;
 
     if (tid == 0) {
-        for (int i = 0; i < kAttStages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kAttConsumers / kAttGroups + (FUSED ? 1 : 0)); }
+        for (int i = 0; i < STAGES; ++i) {
+            ptx::mbar_init(&full_bar[i], 1);
+            ptx::mbar_init(&empty_bar[i], kAttConsumers / kAttGroups + (FUSED ? 1 : 0));
+        }
+        for (int i = 0; i < kAttGroups; ++i) { ptx::mbar_init(&tab_full[i], 1); ptx::mbar_init(&tab_empty[i], kAttConsumers / kAttGroups); }
         ptx::fence_mbar_init();
     }
     __syncthreads();
@@ -122,8 +141,8 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 ptx::prefetch_tensormap(&map_k);
                 ptx::prefetch_tensormap(&map_v);
                 for (int it = 0; it < n_tiles; ++it) {
-                    const int st = it % kAttStages;
-                    if (it >= kAttStages && !ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kAttStages) & 1) ^ 1))) {
+                    const int st = it % STAGES;
+                    if (it >= STAGES && !ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1))) {
                         atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                         break;
                     }
@@ -155,8 +174,18 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (it >= base_it + 32) { base_it = it; my_page = lookup(base_it + lane); }
                 const int page = __shfl_sync(0xffffffffu, my_page, it - base_it);
                 if (lane == 0) {
-                    const int st = it % kAttStages;
-                    if (it >= kAttStages) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kAttStages) & 1) ^ 1));
+                    const int st = it % STAGES;
+                    if (it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
+                    if (ROPE && ok) {
+                        // the (cos, sin) rows of the tile's 64 compact positions are contiguous: one 32 KiB bulk copy
+                        const int tb = it % kAttGroups;              // group tb consumes tile it: one table buffer per group
+                        if (it >= kAttGroups) ok = ptx::mbar_wait(&tab_empty[tb], (uint32_t)(((it / kAttGroups) & 1) ^ 1));
+                        if (ok) {
+                            const float2* rows = a.rope + (size_t)(a.first_position + (t0 + it) * kTile) * (kD / 2);
+                            ptx::mbar_expect_tx(&tab_full[tb], kTabBytes);
+                            ptx::bulk_g2s(stages + (size_t)STAGES * kStageBytes + (size_t)tb * kTabBytes, rows, kTabBytes, &tab_full[tb]);
+                        }
+                    }
                     if (ok) {
                         unsigned char* dst = stages + (size_t)st * kStageBytes;
                         // page layout [K|V][L*G][64 tokens][128]: rows of 256 B
@@ -179,8 +208,8 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             ptx::prefetch_tensormap(&map_v);
             bool ok = true;
             for (int it = 0; it < n_tiles; ++it) {
-                const int st = it % kAttStages;
-                ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kAttStages) & 1));
+                const int st = it % STAGES;
+                ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / STAGES) & 1));
                 if (!ok) break;
                 unsigned char* src = stages + (size_t)st * kStageBytes;
                 const int y = (t0 + it) * kTile;
@@ -191,11 +220,11 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 ptx::bulk_commit();
                 if (it > 0) {                              // all but the newest store have left shared memory
                     ptx::bulk_wait_read<1>();
-                    ptx::mbar_arrive(&empty_bar[(it - 1) % kAttStages]);
+                    ptx::mbar_arrive(&empty_bar[(it - 1) % STAGES]);
                 }
             }
             ptx::bulk_wait_read<0>();
-            if (ok) ptx::mbar_arrive(&empty_bar[(n_tiles - 1) % kAttStages]);
+            if (ok) ptx::mbar_arrive(&empty_bar[(n_tiles - 1) % STAGES]);
             else atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
             ptx::bulk_wait<0>();                           // the view is complete before the kernel ends
         }
@@ -226,8 +255,9 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         const int grp = warp >> 2, wq = warp & 3;
 
         for (int it = grp; it < n_tiles; it += kAttGroups) {
-            const int st = it % kAttStages;
-            const bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kAttStages) & 1));
+            const int st = it % STAGES;
+            bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / STAGES) & 1));
+            if (ROPE) arrived = arrived && ptx::mbar_wait(&tab_full[grp], (uint32_t)((it / kAttGroups) & 1));
             if (!__all_sync(0xffffffffu, arrived)) {          // warp-uniform decision
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
@@ -239,19 +269,61 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             float sc[2][4];
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) { sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.0f; }
+            if (!ROPE) {
 #pragma unroll
-            for (int kp = 0; kp < 4; ++kp) {            // 32 dims = 4 chunks of 16 B = 2 k-steps
-                const int cg = kp * 4 + mj;             // 16-byte chunk along d (0..15)
-                const uint32_t half_off = (uint32_t)(cg >> 3) * kHalfBytes;
-                const int c = cg & 7;
+                for (int kp = 0; kp < 4; ++kp) {            // 32 dims = 4 chunks of 16 B = 2 k-steps
+                    const int cg = kp * 4 + mj;             // 16-byte chunk along d (0..15)
+                    const uint32_t half_off = (uint32_t)(cg >> 3) * kHalfBytes;
+                    const int c = cg & 7;
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) {
+                        const int tok = wq * 16 + nt * 8 + mr;
+                        const uint32_t addr = kbase + half_off + (uint32_t)tok * 128u + (uint32_t)((c ^ (tok & 7)) << 4);
+                        uint32_t b0, b1, b2, b3;
+                        ptx::ldmatrix_x4(addr, b0, b1, b2, b3);
+                        ptx::mma_bf16_16816(sc[nt], qf[2 * kp], b0, b1);
+                        ptx::mma_bf16_16816(sc[nt], qf[2 * kp + 1], b2, b3);
+                    }
+                }
+            } else {
+                // Dimension i pairs with i + 64: the fragment of chunk cg (low half) and the one of chunk cg + 8
+                // (high half) sit in the same lane, so a lane rotates what it holds: registers lo[j], hi[j] carry
+                // dims 8 (4 kp + j) + 2 (lane & 3) + {0, 1} (+ 64) of token wq*16 + nt*8 + lane/4.
+                const unsigned char* tab = stages + (size_t)STAGES * kStageBytes + (size_t)grp * kTabBytes;   // [64 positions][64 pairs] (cos, sin)
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt) {
                     const int tok = wq * 16 + nt * 8 + mr;
-                    const uint32_t addr = kbase + half_off + (uint32_t)tok * 128u + (uint32_t)((c ^ (tok & 7)) << 4);
-                    uint32_t b0, b1, b2, b3;
-                    ptx::ldmatrix_x4(addr, b0, b1, b2, b3);
-                    ptx::mma_bf16_16816(sc[nt], qf[2 * kp], b0, b1);
-                    ptx::mma_bf16_16816(sc[nt], qf[2 * kp + 1], b2, b3);
+                    const int rtok = wq * 16 + nt * 8 + (lane >> 2);              // the token whose elements this lane holds
+                    uint32_t lo[2][4], hi[2][4];
+#pragma unroll
+                    for (int kp = 0; kp < 2; ++kp) {
+                        const int c = kp * 4 + mj;
+                        const uint32_t addr = kbase + (uint32_t)tok * 128u + (uint32_t)((c ^ (tok & 7)) << 4);
+                        ptx::ldmatrix_x4(addr, lo[kp][0], lo[kp][1], lo[kp][2], lo[kp][3]);
+                        ptx::ldmatrix_x4(addr + kHalfBytes, hi[kp][0], hi[kp][1], hi[kp][2], hi[kp][3]);
+                        const float4* row = reinterpret_cast<const float4*>(tab + (size_t)rtok * (kD * 4)) + (kp * 16 + (lane & 3));
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float4 t = row[j * 4];                          // pairs 8 (4 kp + j) + 2 (lane & 3) + {0, 1}
+                            const float a0 = __uint_as_float(lo[kp][j] << 16), a1 = __uint_as_float(lo[kp][j] & 0xffff0000u);
+                            const float b0 = __uint_as_float(hi[kp][j] << 16), b1 = __uint_as_float(hi[kp][j] & 0xffff0000u);
+                            const float l0 = __fsub_rn(__fmul_rn(a0, t.x), __fmul_rn(b0, t.y)), h0 = __fadd_rn(__fmul_rn(b0, t.x), __fmul_rn(a0, t.y));
+                            const float l1 = __fsub_rn(__fmul_rn(a1, t.z), __fmul_rn(b1, t.w)), h1 = __fadd_rn(__fmul_rn(b1, t.z), __fmul_rn(a1, t.w));
+                            lo[kp][j] = ptx::pack_bf16x2(l0, l1);
+                            hi[kp][j] = ptx::pack_bf16x2(h0, h1);
+                        }
+                    }
+                    // the k-steps in the order of the other modes, so that the logits are the same bits
+#pragma unroll
+                    for (int kp = 0; kp < 2; ++kp) {
+                        ptx::mma_bf16_16816(sc[nt], qf[2 * kp], lo[kp][0], lo[kp][1]);
+                        ptx::mma_bf16_16816(sc[nt], qf[2 * kp + 1], lo[kp][2], lo[kp][3]);
+                    }
+#pragma unroll
+                    for (int kp = 0; kp < 2; ++kp) {
+                        ptx::mma_bf16_16816(sc[nt], qf[2 * kp + 4], hi[kp][0], hi[kp][1]);
+                        ptx::mma_bf16_16816(sc[nt], qf[2 * kp + 5], hi[kp][2], hi[kp][3]);
+                    }
                 }
             }
             // online softmax (exp2 domain); this thread holds rows lane/4 (c0,c1) and lane/4 + 8 (c2,c3)
@@ -299,7 +371,10 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 }
             }
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&empty_bar[st]);
+            if (lane == 0) {
+                ptx::mbar_arrive(&empty_bar[st]);
+                if (ROPE) ptx::mbar_arrive(&tab_empty[grp]);
+            }
         }
         // row sums live spread over the 4 lanes of a quad
         l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1); l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
@@ -417,7 +492,8 @@ static bool make_pages_map(CUtensorMap* map, const kvmem_pool& p, const __nv_bfl
 cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M,
                           const __nv_bfloat16* view_k, const __nv_bfloat16* view_v, int view_cap_tokens,
                           const int32_t* n_sel, float scale, float* out, float* lse, void* workspace,
-                          cudaStream_t st, const int32_t* sel_ids, int sel_stride, int session_first, const PagedSource* alt) {
+                          cudaStream_t st, const int32_t* sel_ids, int sel_stride, int session_first, const PagedSource* alt,
+                          int rope_first_position) {
     const Geometry& g = p.geo;
     const int LG = g.L * g.G, heads = n_sessions * LG;
     const bool fused = sel_ids != nullptr;
@@ -438,6 +514,8 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
             e = cudaFuncSetAttribute(attend_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attend_split_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -457,8 +535,11 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     if (alt) {
         a.tables = alt->tables; a.nblocks_dev = alt->nblocks_dev; a.max_bps = alt->table_stride; a.max_blocks = alt->n_pages;
     }
+    a.rope = p.rope_dev; a.first_position = rope_first_position;
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
-    if (paged_only)
+    if (paged_only && rope_first_position >= 0)
+        launch_pdl(attend_split_kernel<3>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);
+    else if (paged_only)
         launch_pdl(attend_split_kernel<2>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);
     else if (fused)
         launch_pdl(attend_split_kernel<1>, dim3(grid), dim3(kAttThreads + 32), kAttSmem, st, map_k, map_v, map_pages, a);

@@ -182,6 +182,6 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
                           const __nv_bfloat16* view_k, const __nv_bfloat16* view_v, int view_cap_tokens,
                           const int32_t* n_sel, float scale, float* out, float* lse, void* workspace,
                           cudaStream_t st, const int32_t* sel_ids = nullptr, int sel_stride = 0, int session_first = 0,
-                          const PagedSource* alt = nullptr);
+                          const PagedSource* alt = nullptr, int rope_first_position = -1);
 
 }  // namespace kvmem

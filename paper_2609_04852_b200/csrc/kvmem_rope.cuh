@@ -6,15 +6,14 @@
 
 namespace kvmem {
 
-// 8 (lo, hi) pairs -> rotated pairs.  sgn = +1 forward, -1 inverse.
-__device__ __forceinline__ void rotate8(const uint4& lo_in, const uint4& hi_in, const float2* __restrict__ cs, float sgn,
-                                        uint4& lo_out, uint4& hi_out) {
+// 8 (lo, hi) pairs -> rotated pairs; t[w] = (cos, sin, cos, sin) of pairs 2w and 2w + 1.  sgn = +1 forward, -1 inverse.
+__device__ __forceinline__ void rotate8_cs(const uint4& lo_in, const uint4& hi_in, const float4 (&t4)[4], float sgn,
+                                           uint4& lo_out, uint4& hi_out) {
     const uint32_t li[4] = {lo_in.x, lo_in.y, lo_in.z, lo_in.w}, hi[4] = {hi_in.x, hi_in.y, hi_in.z, hi_in.w};
     uint32_t lo_o[4], hi_o[4];
-    const float4* cs4 = reinterpret_cast<const float4*>(cs);      // (cos0, sin0, cos1, sin1)
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
-        const float4 t = __ldg(cs4 + w);
+        const float4 t = t4[w];
         const float a0 = __uint_as_float(li[w] << 16), a1 = __uint_as_float(li[w] & 0xffff0000u);
         const float b0 = __uint_as_float(hi[w] << 16), b1 = __uint_as_float(hi[w] & 0xffff0000u);
         const float s0 = sgn * t.y, s1 = sgn * t.w;
@@ -26,6 +25,16 @@ __device__ __forceinline__ void rotate8(const uint4& lo_in, const uint4& hi_in, 
     }
     lo_out = make_uint4(lo_o[0], lo_o[1], lo_o[2], lo_o[3]);
     hi_out = make_uint4(hi_o[0], hi_o[1], hi_o[2], hi_o[3]);
+}
+
+// the same with the table row in global memory: cs points at the (cos, sin) of the first of the 8 pairs
+__device__ __forceinline__ void rotate8(const uint4& lo_in, const uint4& hi_in, const float2* __restrict__ cs, float sgn,
+                                        uint4& lo_out, uint4& hi_out) {
+    const float4* cs4 = reinterpret_cast<const float4*>(cs);
+    float4 t4[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) t4[w] = __ldg(cs4 + w);
+    rotate8_cs(lo_in, hi_in, t4, sgn, lo_out, hi_out);
 }
 
 }  // namespace kvmem

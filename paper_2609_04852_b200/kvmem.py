@@ -84,6 +84,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_view_cache_update": (C.c_int, [vp, i32, vp, vp, vp, sz, i32, i32, i32, vp, vp]),
         "kvmem_view_cache_attend": (C.c_int, [vp, vp, i32, vp, sz, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_paged_attend": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
+        "kvmem_paged_attend_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
         "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
         "kvmem_recall_step_host": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, i32, f32, vp, vp,
@@ -105,7 +106,7 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_view_attend_static", "kvmem_materialize_attend",
             "kvmem_paged_attend", "kvmem_append_blocks_rope", "kvmem_rope_rotate", "kvmem_materialize_rope",
             "kvmem_working_set_delta", "kvmem_score", "kvmem_view_cache_bytes", "kvmem_view_cache_layout",
-            "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend")
+            "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend", "kvmem_paged_attend_rope")
 
 
 def _check(status: int) -> None:
@@ -323,6 +324,17 @@ class Pool:
                                            _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
                                            scale, _dev(out, torch.float32), _dev(lse, torch.float32),
                                            ws.data_ptr(), ws.numel(), _stream()))
+
+    def paged_attend_rope(self, q: torch.Tensor, sel_ids: torch.Tensor, n_sel: torch.Tensor, out: torch.Tensor,
+                          lse: torch.Tensor, first_position: int = 0, scale: float = 0.0, session_first: int = 0) -> None:
+        """Copy-free view with position-consistent keys: raw key tiles are RoPE'd in shared memory on their way
+        to the tensor cores (same results as materialize_rope + view_attend, no view written)."""
+        ns, M = q.shape[0], q.shape[1]
+        ws = self.attend_workspace(ns, M)
+        _check(self.lib.kvmem_paged_attend_rope(self.handle, session_first, ns, _dev(q, torch.bfloat16), M,
+                                                _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
+                                                first_position, scale, _dev(out, torch.float32), _dev(lse, torch.float32),
+                                                ws.data_ptr(), ws.numel(), _stream()))
 
     def view_attend_static(self, q: torch.Tensor, view: View, n_sel: torch.Tensor, out: torch.Tensor,
                            lse: torch.Tensor, scale: float = 0.0) -> None:

@@ -106,6 +106,35 @@ def test_step_with_position_consistent_view(first_position):
     assert np.array_equal(bits(view.k[0]), vK), "rotated keys differ from the defined code"
     ref_out, ref_lse = orc.attend(qb[0], vK, vV, k * B)
     assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+    # the copy-free variant rotates the same raw tiles in shared memory: same keys bit for bit, same tile order
+    out2, lse2 = pool.new_outputs(1, M)
+    pool.paged_attend_rope(qd, sel, n_sel, out2, lse2, first_position)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    assert np.abs(out2.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse2.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+    assert torch.equal(out2, out) and torch.equal(lse2, lse)
+
+
+@pytest.mark.parametrize("n_blocks,budget,M", [(700, 60, 4), (90, 1, 1), (64, 64, 2)])
+def test_position_consistent_paged_attention_over_long_and_short_views(n_blocks, budget, M):
+    # several tiles per split and a ragged split range; a single tile; every block selected
+    spec = SPEC.with_(n_blocks=n_blocks, budget_blocks=budget, n_q_tokens=M)
+    dev = torch.device("cuda", 0)
+    pool, repo, idx, tab, table = _fill_both(spec)
+    B = spec.block_tokens
+    rng = np.random.default_rng(n_blocks)
+    ids = np.sort(rng.choice(n_blocks, size=budget, replace=False)).astype(np.int32)
+    first = 17 if (17 + budget * B) <= WINDOW else 0
+    q, qb = queries(spec)
+    sel = torch.from_numpy(ids).view(1, -1).to(dev)
+    n_sel = torch.tensor([budget], dtype=torch.int32, device=dev)
+    out, lse = pool.new_outputs(1, M)
+    pool.paged_attend_rope(q.to(dev), sel, n_sel, out, lse, first)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    vK, vV = orc.gather_rope(repo, table, ids, budget * B, first, tab)
+    ref_out, ref_lse = orc.attend(qb[0], vK, vV, budget * B)
+    assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
 
 
 def test_rotary_errors():
@@ -129,4 +158,12 @@ def test_rotary_errors():
     with pytest.raises(KvmemError) as e:
         pool.materialize_rope(sel, n_sel, view, WINDOW - 64)         # compact positions would leave the table
     assert e.value.status == E_INVALID
+    out, lse = pool.new_outputs(1, 1)
+    q = torch.zeros(1, 1, 1, spec.n_q_heads, spec.head_dim, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(KvmemError) as e:
+        pool.paged_attend_rope(q, sel, n_sel, out, lse, WINDOW - 64)
+    assert e.value.status == E_INVALID
+    with pytest.raises(KvmemError) as e:
+        plain.paged_attend_rope(q, sel, n_sel, out, lse, 0)
+    assert e.value.status == E_STATE
     assert pool.device_status() == 0
