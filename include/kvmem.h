@@ -197,7 +197,10 @@ int kvmem_materialize(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessi
  *   lse      DEVICE fp32 [n_sessions][n_q_tokens][n_layers][n_q_heads]
  *   scale    0 selects 1/sqrt(head_dim)
  *   workspace DEVICE, kvmem_attend_workspace_bytes(), 256-byte aligned
- * T = 0 gives out = 0 and lse = -inf.  n_q_tokens * (H/G) <= 16 per call. */
+ * T = 0 gives out = 0 and lse = -inf.  n_q_tokens * (H/G) <= 16 per call.  Any block size the pool accepts
+ * (the view is walked in 64-token tiles; a shorter last tile is masked); head_dim 128.  The calls that read
+ * pages through the block table (kvmem_materialize_attend, kvmem_paged_attend*, kvmem_view_cache_attend) are
+ * built for 64-token blocks and return KVMEM_E_UNSUPPORTED otherwise. */
 int kvmem_view_attend(kvmem_pool_t* pool, int32_t n_sessions, const void* q /*DEVICE*/, int32_t n_q_tokens,
                       const void* view_k /*DEVICE*/, const void* view_v /*DEVICE*/, int32_t view_cap_tokens,
                       const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,

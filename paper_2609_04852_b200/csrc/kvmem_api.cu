@@ -429,8 +429,8 @@ int kvmem_view_attend(kvmem_pool_t* p, int32_t n_sessions, const void* q, int32_
         return KVMEM_E_INVALID;
     }
     if (n_q_tokens < 1) { set_error("n_q_tokens must be positive"); return KVMEM_E_INVALID; }
-    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
-        set_error("attention kernel is built for head_dim 128 and 64-token blocks");
+    if (p->cfg.head_dim != 128) {       // any block size the pool accepts (a multiple of 16): the view is walked in 64-token tiles
+        set_error("attention kernel is built for head_dim 128");
         return KVMEM_E_UNSUPPORTED;
     }
     if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }

@@ -52,6 +52,7 @@ struct AttendArgs {
     const int32_t* nblocks_dev;  // [max_sessions]
     int session_first, sel_stride, max_bps, max_blocks;
     // position-consistent copy-free view (attend_split_kernel<3>): raw keys are rotated in shared memory
+    int block_tokens;            // tokens per selected block (view length = n_sel * block_tokens); 64 in the paged modes
     const float2* rope;          // [rope_positions][64] (cos, sin)
     int first_position;          // compact position of view token 0
 };
@@ -113,8 +114,12 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     const int z = s * LG + lg;
     const int l = lg / a.G, g = lg % a.G;
 
-    int n_blk = a.n_sel[s];
-    n_blk = max(0, min(n_blk, a.cap_tokens / kTile));
+    // view length in tokens; the kernel works in 64-token tiles, whatever the block size of the view (a multiple of
+    // 16, so each consumer warp's 16 tokens are all inside or all outside the view)
+    const int btok = PAGED ? kTile : a.block_tokens;
+    const long long n_tok_ll = min((long long)max(a.n_sel[s], 0) * btok, (long long)a.cap_tokens);
+    const int n_tok = (int)n_tok_ll;
+    const int n_blk = (n_tok + kTile - 1) / kTile;
     const int t0 = (int)((long long)n_blk * split / a.n_splits);
     const int t1 = (int)((long long)n_blk * (split + 1) / a.n_splits);
     const int n_tiles = t1 - t0;
@@ -261,6 +266,11 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             if (!__all_sync(0xffffffffu, arrived)) {          // warp-uniform decision
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
+            }
+            if (!PAGED && (t0 + it) * kTile + wq * 16 >= n_tok) {      // this warp's 16 tokens lie beyond a ragged view end
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&empty_bar[st]);
+                continue;
             }
             const uint32_t kbase = stage0 + (uint32_t)st * kStageBytes;
             const uint32_t vbase = kbase + 2 * kHalfBytes;
@@ -535,7 +545,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     if (alt) {
         a.tables = alt->tables; a.nblocks_dev = alt->nblocks_dev; a.max_bps = alt->table_stride; a.max_blocks = alt->n_pages;
     }
-    a.rope = p.rope_dev; a.first_position = rope_first_position;
+    a.rope = p.rope_dev; a.first_position = rope_first_position; a.block_tokens = g.B;
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
     if (paged_only && rope_first_position >= 0)
         launch_pdl(attend_split_kernel<3>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);

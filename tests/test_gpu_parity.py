@@ -113,6 +113,22 @@ def test_step_matches_oracle_small(M, gather_mode, score_mode):
         set_option("score_mode", 1)
 
 
+@pytest.mark.parametrize("block_tokens,budget", [(32, 21), (32, 24), (16, 37), (128, 5)])
+def test_step_with_other_block_sizes(block_tokens, budget):
+    # the paper's default block is 32 tokens; the view is walked in 64-token tiles, so an odd number of 32-token
+    # blocks (or any count of 16-token blocks not divisible by 4) ends in a partly filled tile
+    spec = SMALL.with_(block_tokens=block_tokens, budget_blocks=budget, n_q_tokens=2)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    q, qb = queries(spec)
+    got = _run_step(pool, spec, q.cuda(), _params(budget_blocks=budget), budget)
+    ref = _oracle_step(spec, osess, qb, 0, budget)
+    sel_gpu, _ = _compare_step(spec, got, 0, ref)
+    assert len(sel_gpu) == budget
+    same = _oracle_step(spec, osess, qb, 0, budget, sel_override=sel_gpu)
+    _compare_view_and_attention(spec, got, 0, same)
+
+
 @pytest.mark.parametrize("M,score_mode", [(8, 1), (8, 0), (16, 1), (5, 0)])
 def test_scoring_with_more_than_sixteen_rows_per_kv_head(M, score_mode):
     # M * 4 rows per KV head > 16: the decode scorer walks the rows in passes of 16
