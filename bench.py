@@ -181,8 +181,11 @@ def run_native(args):
     base = CONFIGS[args.workload]
     if args.blocks:      # a shrunken history of the same recipe: the small case for ncu captures
         f = args.blocks / base.n_blocks
-        base = base.with_(name=f"{base.name}@{args.blocks}", n_blocks=args.blocks,
-                          n_planted=max(1, int(base.n_planted * f)), budget_blocks=max(1, int(base.budget_blocks * f)))
+        if base.name == "table4":     # the workspace sweep keeps the 64K view and grows only the history
+            base = base.with_(name=f"{base.name}@{args.blocks}", n_blocks=args.blocks)
+        else:
+            base = base.with_(name=f"{base.name}@{args.blocks}", n_blocks=args.blocks,
+                              n_planted=max(1, int(base.n_planted * f)), budget_blocks=max(1, int(base.budget_blocks * f)))
     pool, spec = fill_pool(base, device, seed_shift=1000 * rank, rope=args.rope)     # one independent replica per rank
     ns, M, B = spec.n_sessions, spec.n_q_tokens, spec.block_tokens
     prm = SelectParams(**select_params(spec))

@@ -86,6 +86,11 @@ CONFIGS: Dict[str, WorkloadSpec] = {
     # 512-token chunk against the 1M index: score + select + materialize only
     "chunk512": _spec("chunk512", 1, 16384, 512, 1024, 3.0, 0.0, 4096, seed=4, attend=False),
 }
+# The paper's workspace-scaling experiment (its table of retrieval latency against workspace size): 32-token
+# blocks, a 128-token query, a 64K-token execution view; the history is swept from 256K to 10M tokens
+# (8,192 to 312,500 blocks) by the benchmark.  Base size 1M tokens.  Score + select + materialize only.
+CONFIGS["table4"] = replace(_spec("table4", 1, 32768, 128, 256, 3.0, 0.0, 2048, seed=5, attend=False),
+                            block_tokens=32, n_query_sets=4)
 
 
 # ----------------------------------------------------------------------------- hashing

@@ -122,3 +122,37 @@ def test_config_chunk512_full():
     assert set(planted_blocks(spec, 0)[0].tolist()) <= set(sel_gpu.tolist())
     vK, vV = orc.gather(osess.repo, osess.table, np.ascontiguousarray(sel_gpu), k * B)
     assert np.array_equal(bits(view.k[0]), vK) and np.array_equal(bits(view.v[0]), vV)
+
+
+def test_workspace_scaling_recipe_at_reduced_size():
+    """The workspace-scaling recipe (32-token blocks, 128-token query, 64K view) with a 20K-block history: the
+    general top-k path (more than 16,384 blocks) fed by tensor-core scoring, then the gather of 32-token blocks."""
+    from paper_2609_04852_b200 import SelectParams, budget_blocks
+    spec = CONFIGS["table4"].with_(name="table4-small", n_blocks=20000, n_planted=64, budget_blocks=300)
+    dev = torch.device("cuda", 0)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec, gen_device=dev)[0]
+    prm_d = select_params(spec)
+    prm = SelectParams(**prm_d)
+    B = spec.block_tokens
+    k = budget_blocks(prm, B, spec.n_blocks)
+    assert B == 32 and k == 300
+    sel = torch.zeros(1, k, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    scores = torch.zeros(1, spec.n_blocks, dtype=torch.float32, device=dev)
+    view = pool.new_view(1, k * B)
+    q, qb = queries(spec, 0)
+    pool.select(q.to(dev), prm, sel, n_sel, scores)
+    pool.materialize(sel, n_sel, view)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    assert np.array_equal(bits(pool.index(0)), osess.idx)
+    R, _ = orc.block_scores(qb[0], osess.idx, spec.n_blocks)
+    check_scores(scores.cpu().numpy()[0], R, spec.n_q_tokens)
+    ref_sel = orc.select(R, B, prm_d["budget_blocks"], prm_d["max_view_tokens"])
+    sel_gpu = sel.cpu().numpy()[0, : int(n_sel.item())]
+    assert len(sel_gpu) == k
+    check_selection(sel_gpu, R, ref_sel)
+    assert set(planted_blocks(spec, 0)[0].tolist()) <= set(sel_gpu.tolist())
+    vK, vV = orc.gather(osess.repo, osess.table, np.ascontiguousarray(sel_gpu), k * B)
+    assert np.array_equal(bits(view.k[0]), vK) and np.array_equal(bits(view.v[0]), vV)
