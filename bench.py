@@ -427,6 +427,25 @@ def run_native(args):
                                 "frac": 2 * flop_alg / sel_s / 1e12 / tpeak["tflops"], "peak_source": f"of {tpeak['source']} (burst)",
                                 "executed_flop_per_launch_pair": 2 * flop_alg, "algorithmic_flop": flop_alg,
                                 "algorithmic_tflops": flop_alg / sel_s / 1e12, "avg_score_ms": sel_s * 1e3, "traffic": None}
+        if args.host_index and spec.attend and ns == 1:
+            # the memory-bounded variant: the index stays in pinned host memory and is streamed over PCIe in tiles
+            idx_host = pool.index(0).cpu().contiguous().pin_memory()
+            sc_buf = torch.zeros(spec.n_blocks, dtype=torch.float32, device=device)
+            hres = {}
+            for tile in (2048, 4096, 8192):
+                for i in range(3):
+                    pool.score_host_index(idx_host, spec.n_blocks, q_dev[i % len(q_dev)][0], sc_buf, tile)
+                h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize(device)
+                h0.record(stream)
+                for i in range(20):
+                    pool.score_host_index(idx_host, spec.n_blocks, q_dev[i % len(q_dev)][0], sc_buf, tile)
+                h1.record(stream)
+                torch.cuda.synchronize(device)
+                ms = h0.elapsed_time(h1) / 20
+                hres[str(tile)] = {"ms": ms, "h2d_gbs": idx_host.numel() * 2 / (ms * 1e-3) / 1e9}
+            line["host_index_scoring"] = {"api": "kvmem_score_host_index", "index_bytes": idx_host.numel() * 2,
+                                          "by_tile_blocks": hres}
         if args.rope:
             line["e2e"]["api"] = "pinned host query in, host O and LSE out, around the four calls of the position-consistent step"
         if world == 1 and not args.no_cpu_baseline:
@@ -692,6 +711,7 @@ def main():
                     "steps (working-set reuse, bounded delta re-RoPE); not the headline step")
     ap.add_argument("--drift", type=float, default=1.0, help="--cache: how far consecutive queries move (1 = independent)")
     ap.add_argument("--max-delta", type=int, default=4, help="--cache: delta re-RoPE operations between reconstructions")
+    ap.add_argument("--host-index", action="store_true", help="also time scoring against the index kept in pinned host memory")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)
     args = ap.parse_args()

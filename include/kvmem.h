@@ -162,6 +162,36 @@ int kvmem_materialize_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_
 int kvmem_score(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/, int32_t n_q_tokens,
                 float* scores /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
+/* Selection alone (Sec. 4.3: reserve sink and recent blocks, fill the budget with the largest R_b, ties to the
+ * lower id, chronological output): the second half of kvmem_select, for scores the caller already has (for
+ * example from kvmem_score_host_index).  scores DEVICE fp32 [n_sessions][scores_stride], non-negative; the
+ * session lengths are the pool's.  sel_ids, sel_stride, n_sel and errors as in kvmem_select. */
+int kvmem_topk(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const float* scores /*DEVICE*/,
+               int32_t scores_stride, const kvmem_select_params_t* params /*HOST*/, int32_t* sel_ids /*DEVICE*/,
+               int32_t sel_stride, int32_t* n_sel /*DEVICE*/, void* stream);
+
+/* Block relevance against an index that lives in HOST memory (Sec. 5.2: the index is streamed to the GPU in
+ * tiles and softmax statistics are carried across tiles; Sec. 5.3 "Incremental Indexing" keeps the index small
+ * enough for that).  R is the same quantity kvmem_score computes (Eq. "kvmem-block-score"), for one session.
+ *   index_host  HOST bf16 [n_layers][n_kv_heads][index_stride_blocks][head_dim], 16-byte aligned; page-locked
+ *               memory makes the copies asynchronous and fast, pageable memory works but serialises
+ *   n_blocks    blocks to score (<= index_stride_blocks)
+ *   q           DEVICE bf16 [n_q_tokens][n_layers][n_q_heads][head_dim], 1..16 query tokens
+ *   tile_blocks blocks per head and tile, a multiple of 128
+ *   scores      DEVICE fp32 [n_blocks]
+ *   staging     DEVICE, kvmem_score_host_staging_bytes(): two tiles, 256-byte aligned
+ *   workspace   DEVICE, kvmem_score_host_workspace_bytes(): fp32 logits of all blocks and the per-tile statistics
+ * Tile i + 1 is copied (on a stream the pool owns) while tile i is scored on `stream`; the two are ordered by
+ * events only.  When the call returns, work is queued on both streams; `stream` alone has to be waited for.
+ * index_host must stay valid until then.  Calls on one pool must not overlap.  Errors: KVMEM_E_INVALID,
+ * KVMEM_E_CAPACITY, KVMEM_E_CUDA as elsewhere. */
+size_t kvmem_score_host_workspace_bytes(const kvmem_pool_t* pool, int32_t n_blocks, int32_t n_q_tokens, int32_t tile_blocks);
+size_t kvmem_score_host_staging_bytes(const kvmem_pool_t* pool, int32_t tile_blocks);
+int kvmem_score_host_index(kvmem_pool_t* pool, const void* index_host /*HOST*/, int32_t n_blocks, int32_t index_stride_blocks,
+                           const void* q /*DEVICE*/, int32_t n_q_tokens, int32_t tile_blocks, float* scores /*DEVICE*/,
+                           void* staging /*DEVICE*/, size_t staging_bytes, void* workspace /*DEVICE*/,
+                           size_t workspace_bytes, void* stream);
+
 /* Score and select (Sec. 4.3, Eq. "kvmem-block-score"; selector; Sec. 5.2 tiled scoring with the
  * softmax kept global across tiles).  For each session s in [session_first, session_first + n_sessions):
  *     R_b = sum_m (1/(L*H)) sum_{l,h} softmax_{b' in all blocks of s}( q[m][l][h] . kbar[l][b'][g(h)] / sqrt(d) )_b

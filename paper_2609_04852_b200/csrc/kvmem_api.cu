@@ -203,6 +203,15 @@ int kvmem_pool_create(const kvmem_pool_config_t* cfg, void* storage, size_t byte
 int kvmem_pool_destroy(kvmem_pool_t* pool) {
     if (!pool_ok(pool)) return KVMEM_E_STATE;
     pool->magic = 0;
+    if (pool->copy_stream) {            // the copy stream of host-resident index scoring: drain it, then let it go
+        cudaStreamSynchronize(pool->copy_stream);
+        for (int i = 0; i < 2; ++i) {
+            if (pool->ev_ready[i]) cudaEventDestroy(pool->ev_ready[i]);
+            if (pool->ev_free[i]) cudaEventDestroy(pool->ev_free[i]);
+        }
+        if (pool->ev_start) cudaEventDestroy(pool->ev_start);
+        cudaStreamDestroy(pool->copy_stream);
+    }
     delete pool;
     return KVMEM_OK;
 }
@@ -377,6 +386,69 @@ int kvmem_score(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, cons
     if (!scores) { set_error("scores is null"); return KVMEM_E_INVALID; }
     float* sc = nullptr;
     return score_impl(p, session_first, n_sessions, q, n_q_tokens, scores, workspace, workspace_bytes, (cudaStream_t)stream, &sc);
+}
+
+// ---- index in host memory, streamed in tiles
+
+static bool host_score_args_ok(const kvmem_pool_t* p, int32_t n_blocks, int32_t n_q_tokens, int32_t tile_blocks) {
+    if (n_blocks < 1 || n_q_tokens < 1 || n_q_tokens > kMaxDecodeTokens) {
+        set_error("host-index scoring takes 1..%d query tokens and at least one block", kMaxDecodeTokens);
+        return false;
+    }
+    if (tile_blocks < 128 || tile_blocks % 128 != 0) { set_error("tile_blocks must be a positive multiple of 128"); return false; }
+    if (p->cfg.head_dim != 128) { set_error("scoring kernels are built for head_dim 128"); return false; }
+    if ((int64_t)p->cfg.n_layers * p->cfg.n_kv_heads * tile_blocks > 0x7fffffffll) { set_error("tile too large"); return false; }
+    return true;
+}
+
+size_t kvmem_score_host_workspace_bytes(const kvmem_pool_t* p, int32_t n_blocks, int32_t n_q_tokens, int32_t tile_blocks) {
+    if (!p || !host_score_args_ok(p, n_blocks, n_q_tokens, tile_blocks)) return 0;
+    return plan_host_score(p->cfg, n_blocks, n_q_tokens, tile_blocks, p->sm_count, nullptr).total;
+}
+
+size_t kvmem_score_host_staging_bytes(const kvmem_pool_t* p, int32_t tile_blocks) {
+    if (!p || !host_score_args_ok(p, 1, 1, tile_blocks)) return 0;
+    return plan_host_score(p->cfg, 1, 1, tile_blocks, p->sm_count, nullptr).staging_bytes;
+}
+
+int kvmem_score_host_index(kvmem_pool_t* p, const void* index_host, int32_t n_blocks, int32_t index_stride_blocks, const void* q,
+                           int32_t n_q_tokens, int32_t tile_blocks, float* scores, void* staging, size_t staging_bytes,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!host_score_args_ok(p, n_blocks, n_q_tokens, tile_blocks)) return KVMEM_E_INVALID;
+    if (!index_host || !q || !scores || !staging || !workspace || !aligned(index_host, 16) || !aligned(q, 16) ||
+        !aligned(staging, 256) || !aligned(workspace, 256)) {
+        set_error("kvmem_score_host_index: null or misaligned pointer");
+        return KVMEM_E_INVALID;
+    }
+    if (index_stride_blocks < n_blocks) { set_error("index_stride_blocks is below n_blocks"); return KVMEM_E_INVALID; }
+    HostScorePlan plan = plan_host_score(p->cfg, n_blocks, n_q_tokens, tile_blocks, p->sm_count, (char*)workspace);
+    if (workspace_bytes < plan.total) { set_error("workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
+    if (staging_bytes < plan.staging_bytes) { set_error("staging holds %zu bytes, %zu needed", staging_bytes, plan.staging_bytes); return KVMEM_E_CAPACITY; }
+    cudaError_t e = launch_score_host_index(*p, (const __nv_bfloat16*)index_host, n_blocks, index_stride_blocks,
+                                            (const __nv_bfloat16*)q, n_q_tokens, tile_blocks, staging, plan, scores,
+                                            (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("host-index scoring", e);
+    return KVMEM_OK;
+}
+
+int kvmem_topk(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const float* scores, int32_t scores_stride,
+               const kvmem_select_params_t* prm, int32_t* sel_ids, int32_t sel_stride, int32_t* n_sel, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!scores || !prm || !sel_ids || !n_sel) { set_error("kvmem_topk: null pointer"); return KVMEM_E_INVALID; }
+    if (prm->n_sink_blocks < 0 || prm->n_recent_blocks < 0) { set_error("sink/recent counts must be non-negative"); return KVMEM_E_INVALID; }
+    int max_k = 0, max_nb = 0;
+    for (int s = session_first; s < session_first + n_sessions; ++s) {
+        max_k = std::max(max_k, kvmem_budget_blocks(prm, p->cfg.block_tokens, p->sess_blocks[s]));
+        max_nb = std::max(max_nb, p->sess_blocks[s]);
+    }
+    if (sel_stride < max_k) { set_error("sel_stride %d is below the clamped budget %d", sel_stride, max_k); return KVMEM_E_CAPACITY; }
+    if (scores_stride < max_nb) { set_error("scores_stride %d is below the session length %d", scores_stride, max_nb); return KVMEM_E_INVALID; }
+    cudaError_t e = launch_topk(*p, session_first, n_sessions, scores, scores_stride, *prm, sel_ids, sel_stride, n_sel,
+                                (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("top-k kernel launch", e);
+    return KVMEM_OK;
 }
 
 int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,

@@ -60,6 +60,9 @@ struct kvmem_pool {
     std::vector<uint8_t> page_used;
     int32_t free_hint;
     int sm_count;
+    // host-resident index scoring: a copy stream and its events, created on first use
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_ready[2] = {nullptr, nullptr}, ev_free[2] = {nullptr, nullptr}, ev_start = nullptr;
 };
 
 namespace kvmem {
@@ -115,6 +118,18 @@ ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions
 cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q,
                                 int M, const ScoreWorkspace& ws, float* scores, int scores_stride, cudaStream_t st);
 
+// scoring against a host-resident index, streamed in tiles (kvmem_score.cu)
+struct HostScorePlan {
+    float* logits;      // [L][G][rows_pad][nb_pad]
+    float2* partials;   // [L][G][rows_pad][part_stride]: (max, sum-exp) per row, tile and CTA
+    float2* merged;     // [L][G][rows_pad]
+    size_t logits_bytes, partials_bytes, merged_bytes, total, staging_bytes;
+    int rows, rows_pad, nb_pad, n_tiles, parts_per_tile, part_stride;
+};
+HostScorePlan plan_host_score(const kvmem_pool_config_t& c, int n_blocks, int n_q_tokens, int tile_blocks, int sm_count, char* base);
+cudaError_t launch_score_host_index(kvmem_pool& p, const __nv_bfloat16* index_host, int n_blocks, int stride_blocks,
+                                    const __nv_bfloat16* q, int M, int tile_blocks, void* staging, const HostScorePlan& ws,
+                                    float* scores, cudaStream_t st);
 // working-set delta (kvmem_delta.cu)
 cudaError_t launch_working_set_delta(const kvmem_pool& p, int n_sessions, const int32_t* prev_ids, const int32_t* n_prev,
                                      const int32_t* next_ids, const int32_t* n_next, int stride, int32_t* retained,

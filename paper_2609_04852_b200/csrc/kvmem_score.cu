@@ -229,7 +229,10 @@ __global__ void __launch_bounds__(kScoreThreads, 1)
 score_logits_mma_kernel(const __grid_constant__ CUtensorMap map_idx, const __nv_bfloat16* __restrict__ q,
                         const int32_t* __restrict__ nblocks_dev, int session_first, int M, int L, int H, int G,
                         int max_bps, float* __restrict__ logits, float2* __restrict__ partials, int rows, int rows_pad,
-                        int nb_pad, int n_parts, float scale_log2e, int32_t* __restrict__ status) {
+                        int nb_pad, int n_parts, float scale_log2e, int32_t* __restrict__ status,
+                        int nb_override, int col_off, int part_stride, int part_off) {
+    // nb_override >= 0: the tensor map covers one staged tile of a host-resident index (nb_override blocks per head,
+    // max_bps rows apart); its logits go to columns col_off.. and its statistics to slots part_off.. of part_stride
     pdl_wait();        // everything earlier in the stream is complete and visible from here on
     pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     constexpr int RP = 16;
@@ -242,7 +245,7 @@ score_logits_mma_kernel(const __grid_constant__ CUtensorMap map_idx, const __nv_
 
     const int s = blockIdx.z, lg = blockIdx.y, part = blockIdx.x;
     const int l = lg / G, g = lg % G, r = H / G;
-    const int NB = nblocks_dev[session_first + s];
+    const int NB = nb_override >= 0 ? nb_override : nblocks_dev[session_first + s];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const size_t slab = ((size_t)s * L * G + lg) * rows_pad;
     const int row_base = ((session_first + s) * L * G + lg) * max_bps;     // first index row of this (session, l, g)
@@ -356,7 +359,7 @@ score_logits_mma_kernel(const __grid_constant__ CUtensorMap map_idx, const __nv_
                 for (int o = 16; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
                 run_l[jj] = run_l[jj] * exp2f(run_m[jj] - mn) + sum;
                 run_m[jj] = mn;
-                float* dst = logits + (slab + row0 + j) * (size_t)nb_pad + b0;
+                float* dst = logits + (slab + row0 + j) * (size_t)nb_pad + col_off + b0;
 #pragma unroll
                 for (int t = 0; t < kChunk / 32; ++t) dst[lane + 32 * t] = v[t];
             }
@@ -365,7 +368,7 @@ score_logits_mma_kernel(const __grid_constant__ CUtensorMap map_idx, const __nv_
 #pragma unroll
         for (int jj = 0; jj < 2; ++jj) {
             const int j = warp + 8 * jj;
-            if (lane == 0) partials[(slab + row0 + j) * n_parts + part] = make_float2(run_m[jj], run_l[jj]);
+            if (lane == 0) partials[(slab + row0 + j) * part_stride + part_off + part] = make_float2(run_m[jj], run_l[jj]);
         }
     }
 }
@@ -379,7 +382,8 @@ constexpr int kFinishBlocks = 32;
 __global__ void __launch_bounds__(256)
 score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__ partials,
                     const int32_t* __restrict__ nblocks_dev, int session_first, int LG, int rows, int rows_pad,
-                    int nb_pad, int n_parts, float inv_LH, float* __restrict__ scores, int scores_stride, int stage_parts) {
+                    int nb_pad, int n_parts, float inv_LH, float* __restrict__ scores, int scores_stride, int stage_parts,
+                    int nb_override) {
     pdl_wait();        // everything earlier in the stream is complete and visible from here on
     pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     extern __shared__ float2 fin_smem[];  // rowstat [LG * rows_pad] : (max, 1/Z); then staged partials [LG * rows_pad][n_parts]
@@ -387,7 +391,7 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
     float2* staged = fin_smem + LG * rows_pad;
     __shared__ float red[8][kFinishBlocks];
     const int s = blockIdx.y;
-    const int NB = nblocks_dev[session_first + s];
+    const int NB = nb_override >= 0 ? nb_override : nblocks_dev[session_first + s];
     if ((int)(blockIdx.x * kFinishBlocks) >= NB) return;
     const int n_slots = LG * rows_pad;                        // rows incl. padding: slot = lg * rows_pad + j
     const float2* sess_parts = partials + (size_t)s * n_slots * n_parts;
@@ -456,7 +460,7 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
 int g_score_mode = 1;   // 1: tensor-core dot products (default), 0: fp32 ALU + warp-shuffle kernel
 
 // index [max_sessions * L * G * max_bps rows][128] bf16 as a 2-D tensor; box = 64 dims x 128 rows, 128-byte swizzle
-static bool make_score_index_map(CUtensorMap* map, const kvmem_pool& p) {
+static bool make_score_index_map(CUtensorMap* map, const __nv_bfloat16* index, long long index_rows) {
     static PFN_cuTensorMapEncodeTiled_v12000 enc = nullptr;
     if (!enc) {
         void* ptr = nullptr;
@@ -466,12 +470,11 @@ static bool make_score_index_map(CUtensorMap* map, const kvmem_pool& p) {
             return false;
         enc = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
     }
-    const Geometry& g = p.geo;
-    cuuint64_t dims[2] = {128, (cuuint64_t)g.max_sessions * g.L * g.G * g.max_bps};
+    cuuint64_t dims[2] = {128, (cuuint64_t)index_rows};
     cuuint64_t strides[1] = {256};
     cuuint32_t box[2] = {64, (cuuint32_t)kChunk};
     cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.index, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(index), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -493,7 +496,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     const long long index_rows = (long long)g.max_sessions * g.L * g.G * g.max_bps;
     if (g_score_mode == 1 && index_rows <= 0x7fffffffll) {     // TMA row coordinates are 32-bit
         CUtensorMap map_idx;
-        if (!make_score_index_map(&map_idx, p)) return cudaErrorInvalidValue;
+        if (!make_score_index_map(&map_idx, p.index, index_rows)) return cudaErrorInvalidValue;
         static bool attr_done = false;
         if (!attr_done) {
             e = cudaFuncSetAttribute(score_logits_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem + 1024));
@@ -502,7 +505,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
         }
         launch_pdl(score_logits_mma_kernel, dim3(grid), dim3(kScoreThreads), smem + 1024, st, 
             map_idx, q, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, ws.logits, ws.partials, ws.rows,
-            ws.rows_pad, ws.nb_pad, n_parts, scale_log2e, p.status_dev);
+            ws.rows_pad, ws.nb_pad, n_parts, scale_log2e, p.status_dev, -1, 0, n_parts, 0);
     } else {
 #define KVMEM_SCORE_LAUNCH(RP)                                                                                         \
     do {                                                                                                               \
@@ -534,7 +537,116 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     dim3 fgrid((unsigned)((max_nb + kFinishBlocks - 1) / kFinishBlocks), (unsigned)n_sessions);
     launch_pdl(score_finish_kernel, dim3(fgrid), dim3(256), fsmem, st, ws.logits, ws.partials, p.nblocks_dev, session_first, LG, ws.rows,
                                                    ws.rows_pad, ws.nb_pad, n_parts, 1.0f / (float)(g.L * g.H),
-                                                   scores, scores_stride, stage_parts);
+                                                   scores, scores_stride, stage_parts, -1);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Scoring against an index that lives in HOST memory (Sec. 5.2: the index is streamed to the GPU in
+// tiles and the softmax statistics are carried across tiles).  Tiles of tile_blocks blocks per (layer,
+// KV head) are copied into one of two device staging buffers on the pool's copy stream while the
+// previous tile is scored on the caller's stream (events in both directions, no device-wide
+// synchronisation).  Every tile adds its per-row (max, sum-exp) pairs to the partials array; the logits
+// of all blocks stay on the device (fp32, [rows][NB]); after the last tile the pairs are merged per row
+// in a fixed order and the finish kernel normalises, exactly as for an index in device memory.
+
+// (max, sum-exp) pairs of one row -> one pair, in slot order
+__global__ void __launch_bounds__(128)
+score_merge_partials_kernel(const float2* __restrict__ partials, float2* __restrict__ merged, int n_rows, int n_parts) {
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= n_rows) return;
+    const float2* p = partials + (size_t)row * n_parts;
+    float mx = -INFINITY;
+    for (int c = 0; c < n_parts; ++c) mx = fmaxf(mx, p[c].x);
+    float z = 0.0f;
+    for (int c = 0; c < n_parts; ++c) {
+        const float2 t = p[c];
+        if (t.x > -INFINITY) z += t.y * exp2f(t.x - mx);
+    }
+    merged[row] = make_float2(mx, z);
+}
+
+HostScorePlan plan_host_score(const kvmem_pool_config_t& c, int n_blocks, int n_q_tokens, int tile_blocks, int sm_count, char* base) {
+    HostScorePlan w{};
+    const int r = c.n_q_heads / c.n_kv_heads, LG = c.n_layers * c.n_kv_heads;
+    w.rows = n_q_tokens * r;
+    w.rows_pad = (w.rows + 15) / 16 * 16;
+    w.nb_pad = (n_blocks + kChunk - 1) / kChunk * kChunk;
+    w.n_tiles = (n_blocks + tile_blocks - 1) / tile_blocks;
+    w.parts_per_tile = std::max(1, std::min({tile_blocks / kChunk, kMaxScoreParts, sm_count / std::max(1, LG)}));
+    w.part_stride = w.n_tiles * w.parts_per_tile;
+    w.logits_bytes = align_up((size_t)LG * w.rows_pad * w.nb_pad * sizeof(float), 256);
+    w.partials_bytes = align_up((size_t)LG * w.rows_pad * w.part_stride * sizeof(float2), 256);
+    w.merged_bytes = align_up((size_t)LG * w.rows_pad * sizeof(float2), 256);
+    w.total = w.logits_bytes + w.partials_bytes + w.merged_bytes;
+    w.staging_bytes = 2 * align_up((size_t)LG * tile_blocks * 256, 256);
+    if (base) {
+        w.logits = reinterpret_cast<float*>(base);
+        w.partials = reinterpret_cast<float2*>(base + w.logits_bytes);
+        w.merged = reinterpret_cast<float2*>(base + w.logits_bytes + w.partials_bytes);
+    }
+    return w;
+}
+
+cudaError_t launch_score_host_index(kvmem_pool& p, const __nv_bfloat16* index_host, int n_blocks, int stride_blocks,
+                                    const __nv_bfloat16* q, int M, int tile_blocks, void* staging, const HostScorePlan& ws,
+                                    float* scores, cudaStream_t st) {
+    const Geometry& g = p.geo;
+    const int LG = g.L * g.G;
+    cudaError_t e;
+    if (!p.copy_stream) {                                  // created on first use, destroyed with the pool
+        e = cudaStreamCreateWithFlags(&p.copy_stream, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return e;
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            e = cudaEventCreateWithFlags(&p.ev_ready[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p.ev_free[i], cudaEventDisableTiming);
+        }
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p.ev_start, cudaEventDisableTiming);
+        if (e != cudaSuccess) return e;
+    }
+    static bool attr_done = false;
+    const size_t smem = (size_t)kScoreStages * kChunk * 256 + 1024;
+    if (!attr_done) {
+        e = cudaFuncSetAttribute(score_logits_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    const size_t buf_bytes = align_up((size_t)LG * tile_blocks * 256, 256);
+    const float scale_log2e = 1.4426950408889634f / sqrtf((float)g.d);
+    // whatever the caller's stream did with the staging buffers before (an earlier call) is finished first
+    if ((e = cudaEventRecord(p.ev_start, st)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(p.copy_stream, p.ev_start, 0)) != cudaSuccess) return e;
+    for (int i = 0; i < ws.n_tiles; ++i) {
+        const int b0 = i * tile_blocks, nb = std::min(tile_blocks, n_blocks - b0), buf = i & 1;
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(staging) + (size_t)buf * buf_bytes);
+        if (i >= 2 && (e = cudaStreamWaitEvent(p.copy_stream, p.ev_free[buf], 0)) != cudaSuccess) return e;
+        // one strided copy: nb * 256 bytes of each of the L*G heads
+        e = cudaMemcpy2DAsync(dst, (size_t)tile_blocks * 256, index_host + (size_t)b0 * g.d, (size_t)stride_blocks * 256,
+                              (size_t)nb * 256, (size_t)LG, cudaMemcpyHostToDevice, p.copy_stream);
+        if (e != cudaSuccess) return e;
+        if ((e = cudaEventRecord(p.ev_ready[buf], p.copy_stream)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(st, p.ev_ready[buf], 0)) != cudaSuccess) return e;
+        CUtensorMap map_idx;
+        if (!make_score_index_map(&map_idx, dst, (long long)LG * tile_blocks)) return cudaErrorInvalidValue;
+        dim3 grid((unsigned)ws.parts_per_tile, (unsigned)LG, 1);
+        score_logits_mma_kernel<<<grid, kScoreThreads, smem, st>>>(map_idx, q, p.nblocks_dev, 0, M, g.L, g.H, g.G, tile_blocks,
+                                                                  ws.logits, ws.partials, ws.rows, ws.rows_pad, ws.nb_pad,
+                                                                  ws.parts_per_tile, scale_log2e, p.status_dev, nb, b0,
+                                                                  ws.part_stride, i * ws.parts_per_tile);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if ((e = cudaEventRecord(p.ev_free[buf], st)) != cudaSuccess) return e;
+    }
+    const int n_rows = LG * ws.rows_pad;
+    score_merge_partials_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(ws.partials, ws.merged, n_rows, ws.part_stride);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const size_t fsmem = 2 * (size_t)LG * ws.rows_pad * sizeof(float2);
+    if (fsmem > 48 * 1024) {
+        e = cudaFuncSetAttribute(score_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsmem);
+        if (e != cudaSuccess) return e;
+    }
+    dim3 fgrid((unsigned)((n_blocks + kFinishBlocks - 1) / kFinishBlocks), 1);
+    score_finish_kernel<<<fgrid, 256, fsmem, st>>>(ws.logits, ws.merged, nullptr, 0, LG, ws.rows, ws.rows_pad, ws.nb_pad, 1,
+                                                   1.0f / (float)(g.L * g.H), scores, n_blocks, 1, n_blocks);
     return cudaGetLastError();
 }
 

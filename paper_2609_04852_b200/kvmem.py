@@ -66,6 +66,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_session_blocks": (i32, [vp, i32]),
         "kvmem_append_blocks": (C.c_int, [vp, i32, vp, vp, i32, C.POINTER(i32), vp]),
         "kvmem_score": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, sz, vp]),
+        "kvmem_topk": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp]),
+        "kvmem_score_host_workspace_bytes": (sz, [vp, i32, i32, i32]),
+        "kvmem_score_host_staging_bytes": (sz, [vp, i32]),
+        "kvmem_score_host_index": (C.c_int, [vp, vp, i32, i32, vp, i32, i32, vp, vp, sz, vp, sz, vp]),
         "kvmem_select": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, sz, vp]),
         "kvmem_materialize": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, vp]),
         "kvmem_view_attend": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
@@ -106,7 +110,8 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_view_attend_static", "kvmem_materialize_attend",
             "kvmem_paged_attend", "kvmem_append_blocks_rope", "kvmem_rope_rotate", "kvmem_materialize_rope",
             "kvmem_working_set_delta", "kvmem_score", "kvmem_view_cache_bytes", "kvmem_view_cache_layout",
-            "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend", "kvmem_paged_attend_rope")
+            "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend", "kvmem_paged_attend_rope", "kvmem_topk", "kvmem_score_host_workspace_bytes",
+            "kvmem_score_host_staging_bytes", "kvmem_score_host_index")
 
 
 def _check(status: int) -> None:
@@ -160,6 +165,8 @@ class Pool:
         _check(self.lib.kvmem_pool_create(C.byref(self.cfg), self.storage.data_ptr(), nbytes, C.byref(self.handle)))
         self._select_ws: Optional[torch.Tensor] = None
         self._attend_ws: Optional[torch.Tensor] = None
+        self._host_ws: Optional[torch.Tensor] = None
+        self._host_staging: Optional[torch.Tensor] = None
         self._staging: Optional[torch.Tensor] = None
 
     # ---- lifetime
@@ -278,6 +285,34 @@ class Pool:
         ws = self.select_workspace(ns, M)
         _check(self.lib.kvmem_score(self.handle, session_first, ns, _dev(q, torch.bfloat16), M,
                                     _dev(scores, torch.float32), ws.data_ptr(), ws.numel(), _stream()))
+
+    def topk(self, scores: torch.Tensor, params: SelectParams, sel_ids: torch.Tensor, n_sel: torch.Tensor,
+             session_first: int = 0) -> None:
+        """Selection from scores the caller already has: scores fp32 [n_sessions][stride] on the device."""
+        ns = scores.shape[0]
+        _check(self.lib.kvmem_topk(self.handle, session_first, ns, _dev(scores, torch.float32), scores.shape[1],
+                                   C.byref(params), _dev(sel_ids, torch.int32), sel_ids.shape[-1],
+                                   _dev(n_sel, torch.int32), _stream()))
+
+    def score_host_index(self, index_host: torch.Tensor, n_blocks: int, q: torch.Tensor, scores: torch.Tensor,
+                         tile_blocks: int = 4096) -> None:
+        """Block relevance against an index in HOST memory (bf16 [L][G][stride][d], ideally pinned), streamed to the
+        GPU in tiles of tile_blocks blocks; q bf16 [M][L][H][d] and scores fp32 [n_blocks] on the device."""
+        if index_host.is_cuda or index_host.dtype != torch.bfloat16 or not index_host.is_contiguous():
+            raise ValueError("index_host must be a contiguous CPU bf16 tensor")
+        M = q.shape[0]
+        need_ws = self.lib.kvmem_score_host_workspace_bytes(self.handle, n_blocks, M, tile_blocks)
+        need_st = self.lib.kvmem_score_host_staging_bytes(self.handle, tile_blocks)
+        if need_ws == 0 or need_st == 0:
+            raise KvmemError(E_INVALID, self.lib.kvmem_last_error().decode())
+        if self._host_ws is None or self._host_ws.numel() < need_ws:
+            self._host_ws = torch.empty(need_ws, dtype=torch.uint8, device=self.device)
+        if self._host_staging is None or self._host_staging.numel() < need_st:
+            self._host_staging = torch.empty(need_st, dtype=torch.uint8, device=self.device)
+        _check(self.lib.kvmem_score_host_index(self.handle, index_host.data_ptr(), n_blocks, index_host.shape[2],
+                                               _dev(q, torch.bfloat16), M, tile_blocks, _dev(scores, torch.float32),
+                                               self._host_staging.data_ptr(), self._host_staging.numel(),
+                                               self._host_ws.data_ptr(), self._host_ws.numel(), _stream()))
 
     def select(self, q: torch.Tensor, params: SelectParams, sel_ids: torch.Tensor, n_sel: torch.Tensor,
                scores: Optional[torch.Tensor] = None, session_first: int = 0) -> None:

@@ -361,6 +361,60 @@ def test_score_alone_equals_the_scores_select_reports_and_the_oracle(M, n_blocks
         assert np.array_equal(sc[s, :lens[s]], got["scores"][s, :lens[s]])     # same kernels, fixed merge order
 
 
+# ------------------------------------------------------------------ index in host memory, streamed in tiles
+
+@pytest.mark.parametrize("n_blocks,tile_blocks,M,pinned", [(1000, 256, 4, True), (333, 128, 1, True), (700, 1024, 2, False),
+                                                          (2100, 128, 3, True)])
+def test_scoring_from_a_host_resident_index_in_tiles(n_blocks, tile_blocks, M, pinned):
+    # several tiles with a ragged last one, one tile larger than the index, many tiles (statistics carried across 17)
+    from paper_2609_04852_b200 import SelectParams
+    spec = SMALL.with_(n_blocks=n_blocks, n_q_tokens=M, budget_blocks=40)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    q, qb = queries(spec)
+    dev = torch.device("cuda", 0)
+    idx_host = pool.index(0).cpu().contiguous()                 # [L][G][n_blocks][d]: the index, now in host memory
+    assert np.array_equal(bits(idx_host), osess.idx[:, :, :n_blocks])
+    if pinned:
+        idx_host = idx_host.pin_memory()
+    R, _ = orc.block_scores(qb[0], osess.idx, n_blocks)
+    scores = torch.full((1, n_blocks), -1.0, dtype=torch.float32, device=dev)
+    for _ in range(2):                                          # the second call reuses the staging buffers
+        pool.score_host_index(idx_host, n_blocks, q[0].to(dev), scores[0], tile_blocks)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    got = scores.cpu().numpy()[0]
+    assert abs(got.sum() - M) < 1e-3 * M
+    check_scores(got, R, M)
+    # selection from these scores, on the device
+    sel = torch.zeros(1, 40, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    pool.topk(scores, _params(budget_blocks=40, n_sink_blocks=1, n_recent_blocks=2), sel, n_sel)
+    torch.cuda.synchronize()
+    ref_sel = orc.select(R, spec.block_tokens, 40, 1 << 30, 0, 1, 2)
+    check_selection(sel.cpu().numpy()[0, : int(n_sel[0])], R, ref_sel, 1, 2)
+    # and the same scores as the index in device memory gives, to rounding
+    dev_scores = torch.zeros(1, n_blocks, dtype=torch.float32, device=dev)
+    pool.score(q.to(dev), dev_scores)
+    assert np.allclose(dev_scores.cpu().numpy()[0], got, rtol=1e-4, atol=1e-9)
+
+
+def test_host_index_argument_errors():
+    from paper_2609_04852_b200 import KvmemError
+    spec = SMALL.with_(n_blocks=300)
+    pool = fill_pool(spec)
+    dev = torch.device("cuda", 0)
+    idx_host = pool.index(0).cpu().contiguous()
+    q, _ = queries(spec)
+    scores = torch.zeros(300, dtype=torch.float32, device=dev)
+    with pytest.raises(KvmemError):
+        pool.score_host_index(idx_host, 300, q[0].to(dev), scores, 100)          # tile not a multiple of 128
+    with pytest.raises(KvmemError):
+        pool.score_host_index(idx_host, 400, q[0].to(dev), scores, 128)          # more blocks than the index holds
+    with pytest.raises(ValueError):
+        pool.score_host_index(idx_host.to(dev), 300, q[0].to(dev), scores, 128)  # not a host tensor
+
+
 # ------------------------------------------------------------------ several sessions, permuted pages
 
 def test_multi_session_ragged_lengths_and_permuted_pages():
