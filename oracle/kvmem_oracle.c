@@ -490,3 +490,112 @@ void kvo_view_cache_view(const bf16_t* cacheK, const bf16_t* cacheV, const int32
                     memcpy(viewV + o, cacheV + s, (size_t)d * sizeof(bf16_t));
                 }
 }
+
+/* =======================================================================================
+ * FP8 execution view (the paper's evaluation keeps the KV cache in FP8, Sec. 6.1).
+ *
+ * Format: E4M3 in its finite-only form (1 sign, 4 exponent, 3 mantissa bits, bias 7, no
+ * infinities, largest finite value 448, codes 0x7f / 0xff are NaN).  A stored element is the
+ * code of x * inv_scale (one fp32 product), rounded to nearest with ties to the even code and
+ * saturated to +-448: a quantised code, so both implementations take that decision on the same
+ * fp32 value.  Readings: one static scale per tensor (keys, values), given by the caller, as FP8
+ * KV caches are commonly run; the paper states no scaling rule.
+ * View layout: keys [L][G][cap_tokens][d] bytes; values transposed inside every 64-token tile,
+ * [L][G][cap_tokens/64][d][64] bytes (so that both operands of the attention contractions are read
+ * along their contraction index).
+ */
+static float e4m3_to_f32(uint8_t c) {
+    const int e = (c >> 3) & 15, m = c & 7;
+    float v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexpf((float)m, -9);                       /* subnormal: m * 2^-9 */
+    else v = ldexpf(1.0f + (float)m / 8.0f, e - 7);
+    return (c & 0x80) ? -v : v;
+}
+
+static uint8_t f32_to_e4m3(float x) {
+    const uint8_t sign = signbit(x) ? 0x80 : 0x00;
+    const float a = fabsf(x);
+    if (isnan(x)) return 0x7f;
+    if (a >= 448.0f) return sign | 0x7e;                        /* saturate */
+    /* nearest of the 127 non-negative finite values; on a tie the even code */
+    int lo = 0, hi = 0x7e;                                      /* value(lo) <= a <= value(hi) */
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) / 2;
+        if (e4m3_to_f32((uint8_t)mid) <= a) lo = mid; else hi = mid;
+    }
+    const float vl = e4m3_to_f32((uint8_t)lo), vh = e4m3_to_f32((uint8_t)hi);
+    const double dl = (double)a - (double)vl, dh = (double)vh - (double)a;
+    int code;
+    if (dl < dh) code = lo;
+    else if (dh < dl) code = hi;
+    else code = (lo & 1) ? hi : lo;
+    return sign | (uint8_t)code;
+}
+
+void kvo_quantize_e4m3(const bf16_t* x, uint8_t* y, int64_t n, float inv_scale) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) y[i] = f32_to_e4m3(bf16_to_f32(x[i]) * inv_scale);
+}
+
+void kvo_dequantize_e4m3(const uint8_t* y, float* x, int64_t n, float scale) {
+    for (int64_t i = 0; i < n; ++i) x[i] = e4m3_to_f32(y[i]) * scale;
+}
+
+/* as kvo_gather, quantising on the way; cap_tokens is a multiple of 64 */
+void kvo_gather_fp8(const bf16_t* pagesK, const bf16_t* pagesV, const int32_t* table, const int32_t* sel,
+                    int64_t n_sel, int B, int L, int G, int d, float k_inv_scale, float v_inv_scale,
+                    uint8_t* viewK8, uint8_t* viewV8T, int64_t cap_tokens) {
+    const size_t page = (size_t)B * L * G * d;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n_sel; ++j) {
+        const size_t src = (size_t)table[sel[j]] * page;
+        for (int t = 0; t < B; ++t) {
+            const int64_t tok = j * B + t, tile = tok / 64, tt = tok % 64;
+            for (int l = 0; l < L; ++l)
+                for (int g = 0; g < G; ++g) {
+                    const size_t s = src + (((size_t)t * L + l) * G + g) * d;
+                    const size_t head = (size_t)l * G + g;
+                    for (int c = 0; c < d; ++c) {
+                        viewK8[(head * cap_tokens + (size_t)tok) * d + c] = f32_to_e4m3(bf16_to_f32(pagesK[s + c]) * k_inv_scale);
+                        viewV8T[((head * (size_t)(cap_tokens / 64) + (size_t)tile) * d + c) * 64 + (size_t)tt] =
+                            f32_to_e4m3(bf16_to_f32(pagesV[s + c]) * v_inv_scale);
+                    }
+                }
+        }
+    }
+}
+
+/* kvo_attend over an FP8 view: keys are code * k_scale, values code * v_scale */
+void kvo_attend_fp8(const bf16_t* q, const uint8_t* viewK8, const uint8_t* viewV8T, int64_t T, int64_t cap_tokens,
+                    int M, int L, int H, int G, int d, double scale, double k_scale, double v_scale, float* out, float* lse) {
+    const int r = H / G;
+    const int64_t rows = (int64_t)M * L * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t row = 0; row < rows; ++row) {
+        const int h = (int)(row % H);
+        const int l = (int)((row / H) % L);
+        const size_t head = (size_t)l * G + (size_t)(h / r);
+        const bf16_t* qv = q + row * d;
+        double* s = (double*)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1));
+        double* o = (double*)calloc((size_t)d, sizeof(double));
+        double best = -INFINITY;
+        for (int64_t t = 0; t < T; ++t) {
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c)
+                acc += (double)bf16_to_f32(qv[c]) * ((double)e4m3_to_f32(viewK8[(head * cap_tokens + (size_t)t) * d + c]) * k_scale);
+            s[t] = acc * scale;
+            if (s[t] > best) best = s[t];
+        }
+        double sum = 0.0;
+        for (int64_t t = 0; t < T; ++t) sum += exp(s[t] - best);
+        for (int64_t t = 0; t < T; ++t) {
+            const double p = exp(s[t] - best) / sum;
+            const size_t vbase = (head * (size_t)(cap_tokens / 64) + (size_t)(t / 64)) * d;
+            for (int c = 0; c < d; ++c) o[c] += p * ((double)e4m3_to_f32(viewV8T[(vbase + c) * 64 + (size_t)(t % 64)]) * v_scale);
+        }
+        for (int c = 0; c < d; ++c) out[row * d + c] = (float)o[c];
+        lse[row] = T > 0 ? (float)(best + log(sum)) : -INFINITY;
+        free(s); free(o);
+    }
+}

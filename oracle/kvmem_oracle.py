@@ -68,6 +68,15 @@ def lib():
         L.kvo_view_cache_update.restype = i32
         L.kvo_view_cache_view.argtypes = [p, p, p, i64, i32, i32, i32, i32, p, p, i64]
         L.kvo_view_cache_view.restype = None
+        f32 = C.c_float
+        L.kvo_quantize_e4m3.argtypes = [p, p, i64, f32]
+        L.kvo_quantize_e4m3.restype = None
+        L.kvo_dequantize_e4m3.argtypes = [p, p, i64, f32]
+        L.kvo_dequantize_e4m3.restype = None
+        L.kvo_gather_fp8.argtypes = [p, p, p, p, i64, i32, i32, i32, i32, f32, f32, p, p, i64]
+        L.kvo_gather_fp8.restype = None
+        L.kvo_attend_fp8.argtypes = [p, p, p, i64, i64, i32, i32, i32, i32, i32, dbl, dbl, dbl, p, p]
+        L.kvo_attend_fp8.restype = None
         L.kvo_threads.argtypes = []
         L.kvo_threads.restype = i32
         _lib = L
@@ -276,3 +285,49 @@ class ViewCache:
         lib().kvo_view_cache_view(_ptr(self.K), _ptr(self.V), _ptr(self.view_slots), self.n_view, B, L, G, d,
                                   _ptr(viewK), _ptr(viewV), cap_tokens)
         return viewK, viewV
+
+
+# ---- FP8 (E4M3) execution view ------------------------------------------------------------------------
+
+def quantize_e4m3(x: np.ndarray, inv_scale: float = 1.0) -> np.ndarray:
+    """bf16 bit patterns (uint16) -> E4M3 codes (uint8) of x * inv_scale, round to nearest even, saturating at 448."""
+    x = np.ascontiguousarray(_u16(x))
+    y = np.zeros(x.shape, np.uint8)
+    lib().kvo_quantize_e4m3(_ptr(x), _ptr(y), x.size, float(inv_scale))
+    return y
+
+
+def dequantize_e4m3(y: np.ndarray, scale: float = 1.0) -> np.ndarray:
+    y = np.ascontiguousarray(y, np.uint8)
+    x = np.zeros(y.shape, np.float32)
+    lib().kvo_dequantize_e4m3(_ptr(y), _ptr(x), y.size, float(scale))
+    return x
+
+
+def gather_fp8(repo: Repository, table: np.ndarray, sel: np.ndarray, cap_tokens: int, k_inv_scale: float = 1.0,
+               v_inv_scale: float = 1.0) -> Tuple[np.ndarray, np.ndarray]:
+    """FP8 execution view: keys uint8 [L][G][cap][d]; values uint8 [L][G][cap/64][d][64] (transposed per 64-token tile)."""
+    _, B, L, G, d = repo.pagesK.shape
+    assert cap_tokens % 64 == 0 and len(sel) * B <= cap_tokens and table.dtype == np.int32 and sel.dtype == np.int32
+    vK = np.zeros((L, G, cap_tokens, d), np.uint8)
+    vV = np.zeros((L, G, cap_tokens // 64, d, 64), np.uint8)
+    lib().kvo_gather_fp8(_ptr(repo.pagesK), _ptr(repo.pagesV), _ptr(np.ascontiguousarray(table)),
+                         _ptr(np.ascontiguousarray(sel)), len(sel), B, L, G, d, float(k_inv_scale), float(v_inv_scale),
+                         _ptr(vK), _ptr(vV), cap_tokens)
+    return vK, vV
+
+
+def attend_fp8(q: np.ndarray, viewK8: np.ndarray, viewV8T: np.ndarray, T: int, k_scale: float = 1.0, v_scale: float = 1.0,
+               scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """q uint16 [M][L][H][d] over an FP8 view -> (O fp32 [M][L][H][d], LSE fp32 [M][L][H])."""
+    _u16(q)
+    M, L, H, d = q.shape
+    G, cap = viewK8.shape[1], viewK8.shape[2]
+    assert viewK8.dtype == np.uint8 and viewV8T.dtype == np.uint8 and viewV8T.shape == (L, G, cap // 64, d, 64) and T <= cap
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    out = np.zeros((M, L, H, d), np.float32)
+    lse = np.zeros((M, L, H), np.float32)
+    lib().kvo_attend_fp8(_ptr(q), _ptr(viewK8), _ptr(viewV8T), T, cap, M, L, H, G, d, float(scale), float(k_scale),
+                         float(v_scale), _ptr(out), _ptr(lse))
+    return out, lse
