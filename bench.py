@@ -203,7 +203,11 @@ def run_native(args):
     lse_pin = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device) if args.flush_l2 else None
     stream = torch.cuda.current_stream(device)
-    fused = spec.attend and not args.unfused and not args.rope
+    fused = spec.attend and not args.unfused and not args.rope and not args.fp8
+    if args.fp8:
+        if not spec.attend:
+            raise SystemExit("--fp8 is measured on the attend workloads")
+        k8, v8t = pool.new_view_fp8(ns, cap)
 
     if args.rope:
         if not spec.attend or spec.n_sessions != 1:
@@ -236,6 +240,14 @@ def run_native(args):
         pool.select(q, prm, sel, n_sel)
         if ev is not None:
             ev[0].record(stream)
+        if args.fp8:           # FP8 (E4M3) view: quantise while gathering, attend over half the bytes
+            pool.materialize_fp8(sel, n_sel, k8, v8t)
+            if ev is not None:
+                ev[1].record(stream)
+            pool.view_attend_fp8(q, k8, v8t, n_sel, out, lse)
+            if ev is not None:
+                ev[2].record(stream)
+            return
         if args.paged:
             pool.paged_attend(q, sel, n_sel, out, lse)                  # copy-free view: no materialisation at all
             if ev is not None:
@@ -313,6 +325,14 @@ def run_native(args):
             else:
                 pool.materialize_rope(sel, n_sel, view, 0)
                 pool.view_attend(q_stage, view, n_sel, out, lse)
+            out_pin.copy_(out, non_blocking=True)
+            lse_pin.copy_(lse, non_blocking=True)
+            torch.cuda.synchronize(device)
+        elif args.fp8:
+            q_stage.copy_(q_pin[i % len(q_pin)], non_blocking=True)
+            pool.select(q_stage, prm, sel, n_sel)
+            pool.materialize_fp8(sel, n_sel, k8, v8t)
+            pool.view_attend_fp8(q_stage, k8, v8t, n_sel, out, lse)
             out_pin.copy_(out, non_blocking=True)
             lse_pin.copy_(lse, non_blocking=True)
             torch.cuda.synchronize(device)
@@ -446,6 +466,26 @@ def run_native(args):
                 hres[str(tile)] = {"ms": ms, "h2d_gbs": idx_host.numel() * 2 / (ms * 1e-3) / 1e9}
             line["host_index_scoring"] = {"api": "kvmem_score_host_index", "index_bytes": idx_host.numel() * 2,
                                           "by_tile_blocks": hres}
+        if args.fp8:
+            # FP8 view: the gather reads the bf16 pages (2 B per element) and writes 1 B; attention reads 1 B
+            g_bytes = ns * ab["gather"] * 3 // 4
+            a_bytes = ns * ab["attend"] // 2
+            g_s, a_s = med(gat_ms) * 1e-3, med(att_ms) * 1e-3
+            line["config"]["calls"] = "kvmem_select + kvmem_materialize_fp8 + kvmem_view_attend_fp8 (E4M3 view, static scales 1.0)"
+            line["dtype"] = "bf16 pages and query, E4M3 view, f16 tensor-core products, fp32 accumulation"
+            line["roofline"] = {"bound": "hbm", "kernel": "gather_fp8_kernel (kvmem_materialize_fp8)", "achieved": g_bytes / g_s / 1e9,
+                                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": g_bytes / g_s / 1e9 / peaks["hbm_gbs"],
+                                "peak_source": f"of {peaks['source']}", "algorithmic_bytes_per_launch": g_bytes,
+                                "avg_launch_ms": g_s * 1e3, "traffic": None}
+            line["attend_roofline"] = {"kernel": "attend_fp8_split_kernel + merge (kvmem_view_attend_fp8)", "achieved_gbs": a_bytes / a_s / 1e9,
+                                       "frac": a_bytes / a_s / 1e9 / peaks["hbm_gbs"], "algorithmic_bytes_per_launch": a_bytes,
+                                       "avg_ms": a_s * 1e3}
+            fp8_step = ns * ab["index"] + g_bytes + a_bytes
+            line["step_hbm"] = {"algorithmic_bytes_per_step": fp8_step, "accounting": "index + bf16 page read + FP8 view write + FP8 view read",
+                                "achieved_gbs": K * fp8_step / (total_ms * 1e-3) / 1e9,
+                                "frac_of_peak": K * fp8_step / (total_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                "peak_source": f"of {peaks['source']}", "nominal_peak_gbs": 8000.0}
+            line["e2e"]["api"] = "pinned host query in, host O and LSE out, around the three calls of the FP8-view step"
         if args.rope:
             line["e2e"]["api"] = "pinned host query in, host O and LSE out, around the four calls of the position-consistent step"
         if world == 1 and not args.no_cpu_baseline:
@@ -711,6 +751,7 @@ def main():
                     "steps (working-set reuse, bounded delta re-RoPE); not the headline step")
     ap.add_argument("--drift", type=float, default=1.0, help="--cache: how far consecutive queries move (1 = independent)")
     ap.add_argument("--max-delta", type=int, default=4, help="--cache: delta re-RoPE operations between reconstructions")
+    ap.add_argument("--fp8", action="store_true", help="FP8 (E4M3) execution view: materialize_fp8 + view_attend_fp8 (not the headline step)")
     ap.add_argument("--host-index", action="store_true", help="also time scoring against the index kept in pinned host memory")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)

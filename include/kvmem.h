@@ -290,6 +290,30 @@ int kvmem_working_set_delta(kvmem_pool_t* pool, int32_t n_sessions, const int32_
                             int32_t* incoming /*DEVICE*/, int32_t* outgoing /*DEVICE*/, int32_t* counts /*DEVICE*/,
                             void* stream);
 
+/* FP8 execution view (the paper's evaluation keeps the KV cache in FP8, Sec. 6.1): kvmem_materialize and
+ * kvmem_view_attend for a view that stores one byte per element.
+ * Element = E4M3 code (1 sign, 4 exponent, 3 mantissa bits, bias 7, no infinities, largest value 448) of
+ * x * (1 / scale): one fp32 product, round to nearest with ties to even, saturated to +-448; one static scale
+ * per tensor (k_scale for keys, v_scale for values), > 0.  (The paper states no scaling rule; static
+ * per-tensor scales are how FP8 KV caches are commonly run.)
+ *   view_k8   DEVICE uint8 [n_sessions][n_layers][n_kv_heads][view_cap_tokens][head_dim]
+ *   view_v8t  DEVICE uint8 [n_sessions][n_layers][n_kv_heads][view_cap_tokens / 64][head_dim][64]: values are
+ *             transposed inside every 64-token tile, so that attention reads both operands along the index it
+ *             contracts over
+ *   both 128-byte aligned; view_cap_tokens a multiple of 64; other arguments as in kvmem_materialize /
+ *   kvmem_view_attend.  Built for head_dim 128 and 64-token blocks (KVMEM_E_UNSUPPORTED otherwise).
+ * kvmem_materialize_fp8 reads the bf16 pages through the block table and writes the codes (2 bytes read + 1
+ * byte written per element).  kvmem_view_attend_fp8 computes out = softmax(q . (k8 * k_scale)^T * scale)
+ * (v8 * v_scale) and lse over the first n_sel[s] * 64 view tokens: half the bytes of the bf16 view; the codes
+ * are widened to f16 (exactly) in registers and contracted on the tensor cores with fp32 accumulation. */
+int kvmem_materialize_fp8(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids /*DEVICE*/,
+                          int32_t sel_stride, const int32_t* n_sel /*DEVICE*/, void* view_k8 /*DEVICE*/,
+                          void* view_v8t /*DEVICE*/, int32_t view_cap_tokens, float k_scale, float v_scale, void* stream);
+int kvmem_view_attend_fp8(kvmem_pool_t* pool, int32_t n_sessions, const void* q /*DEVICE*/, int32_t n_q_tokens,
+                          const void* view_k8 /*DEVICE*/, const void* view_v8t /*DEVICE*/, int32_t view_cap_tokens,
+                          const int32_t* n_sel /*DEVICE*/, float scale, float k_scale, float v_scale, float* out /*DEVICE*/,
+                          float* lse /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
 /* Execution cache: the execution view kept across steps, with working-set reuse and bounded delta
  * re-RoPE (Sec. 4.4: the two views; "Retrieval-Aware Hierarchical Reuse"; Eq. "kvmem-working-set-delta").
  *

@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <cmath>
 #include <new>
 
 #include "kvmem_internal.cuh"
@@ -684,6 +685,64 @@ int kvmem_working_set_delta(kvmem_pool_t* p, int32_t n_sessions, const int32_t* 
     cudaError_t e = launch_working_set_delta(*p, n_sessions, prev_ids, n_prev, next_ids, n_next, stride, retained, incoming,
                                              outgoing, counts, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail("working-set delta kernel launch", e);
+    return KVMEM_OK;
+}
+
+// ---- FP8 execution view ----
+
+static int fp8_common_ok(kvmem_pool_t* p, int32_t view_cap_tokens, float k_scale, float v_scale, const char* who) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
+        set_error("%s: the FP8 view kernels are built for head_dim 128 and 64-token blocks", who);
+        return KVMEM_E_UNSUPPORTED;
+    }
+    if (view_cap_tokens < 64 || view_cap_tokens % 64 != 0) { set_error("%s: view_cap_tokens must be a positive multiple of 64", who); return KVMEM_E_INVALID; }
+    if (!(k_scale > 0.0f) || !(v_scale > 0.0f) || !std::isfinite(k_scale) || !std::isfinite(v_scale)) {
+        set_error("%s: scales must be positive and finite", who);
+        return KVMEM_E_INVALID;
+    }
+    return KVMEM_OK;
+}
+
+int kvmem_materialize_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids, int32_t sel_stride,
+                          const int32_t* n_sel, void* view_k8, void* view_v8t, int32_t view_cap_tokens, float k_scale,
+                          float v_scale, void* stream) {
+    const int rc = fp8_common_ok(p, view_cap_tokens, k_scale, v_scale, "kvmem_materialize_fp8");
+    if (rc != KVMEM_OK) return rc;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!sel_ids || !n_sel || !view_k8 || !view_v8t || !aligned(view_k8, 128) || !aligned(view_v8t, 128) || sel_stride < 1) {
+        set_error("kvmem_materialize_fp8: null or misaligned pointer (views need 128-byte alignment), or sel_stride < 1");
+        return KVMEM_E_INVALID;
+    }
+    cudaError_t e = launch_gather_fp8(*p, session_first, n_sessions, sel_ids, sel_stride, n_sel, (uint8_t*)view_k8,
+                                      (uint8_t*)view_v8t, view_cap_tokens, k_scale, v_scale, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("FP8 gather kernel launch", e);
+    return KVMEM_OK;
+}
+
+int kvmem_view_attend_fp8(kvmem_pool_t* p, int32_t n_sessions, const void* q, int32_t n_q_tokens, const void* view_k8,
+                          const void* view_v8t, int32_t view_cap_tokens, const int32_t* n_sel, float scale, float k_scale,
+                          float v_scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = fp8_common_ok(p, view_cap_tokens, k_scale, v_scale, "kvmem_view_attend_fp8");
+    if (rc != KVMEM_OK) return rc;
+    if (n_sessions < 1 || n_q_tokens < 1) { set_error("n_sessions and n_q_tokens must be positive"); return KVMEM_E_INVALID; }
+    if (!q || !view_k8 || !view_v8t || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(view_k8, 128) ||
+        !aligned(view_v8t, 128) || !aligned(workspace, 256) || !aligned(out, 16)) {
+        set_error("kvmem_view_attend_fp8: null or misaligned pointer (views need 128-byte alignment)");
+        return KVMEM_E_INVALID;
+    }
+    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
+    if ((int64_t)n_sessions * p->cfg.n_layers * p->cfg.n_kv_heads * view_cap_tokens > 0x7fffffffll) {
+        set_error("view too large for 32-bit TMA row coordinates");
+        return KVMEM_E_UNSUPPORTED;
+    }
+    AttendPlan plan = plan_attend(p->cfg, n_sessions, n_q_tokens, p->sm_count);
+    if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
+    cudaError_t e = launch_attend_fp8(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, (const uint8_t*)view_k8,
+                                      (const uint8_t*)view_v8t, view_cap_tokens, n_sel, scale, k_scale, v_scale, out, lse,
+                                      workspace, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("FP8 attention kernel launch", e);
     return KVMEM_OK;
 }
 

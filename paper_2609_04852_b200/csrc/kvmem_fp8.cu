@@ -1,0 +1,443 @@
+// FP8 (E4M3) execution view (the paper's evaluation keeps the KV cache in FP8, Sec. 6.1): assembly of
+// the view with quantisation on the way, and split-K decode attention over it.
+//
+// A stored element is the E4M3 code of x * inv_scale (one fp32 product, round to nearest even,
+// saturating at +-448), one static scale per tensor.  Layout: keys [heads][cap_tokens][128] bytes; values
+// transposed inside every 64-token tile, [heads][cap_tokens / 64][128][64] bytes, so that both
+// operands of the two attention contractions are read along their contraction index with plain
+// ldmatrix loads: a 32-bit ldmatrix register then holds four consecutive elements of the contraction
+// index, which two cvt instructions turn into the two f16x2 registers of an m16n8k16 B fragment.  The
+// k-slots of the MMA are a permutation of the contraction index that the A fragments (the query for
+// Q K^T, the probabilities for P V) follow, so no data is shuffled.
+#include <cuda_fp8.h>
+#include <cudaTypedefs.h>
+#include <math.h>
+
+#include <algorithm>
+
+#include "kvmem_internal.cuh"
+#include "kvmem_ptx.cuh"
+
+namespace kvmem {
+
+constexpr int kF8Tile = 64;                      // tokens per tile == block_tokens on this path
+constexpr int kF8D = 128;
+
+__device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d, float inv) {
+    const __nv_fp8x2_storage_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(a, inv), __fmul_rn(b, inv)), __NV_SATFINITE, __NV_E4M3);
+    const __nv_fp8x2_storage_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(c, inv), __fmul_rn(d, inv)), __NV_SATFINITE, __NV_E4M3);
+    return (uint32_t)lo | ((uint32_t)hi << 16);
+}
+
+// 8 bf16 (one 128-bit load) -> 8 E4M3 bytes
+__device__ __forceinline__ uint2 quant8(const uint4& v, float inv) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+    return make_uint2(quant4(f[0], f[1], f[2], f[3], inv), quant4(f[4], f[5], f[6], f[7], inv));
+}
+
+struct GatherF8Args {
+    const __nv_bfloat16* pages;
+    const int32_t* tables;
+    const int32_t* nblocks_dev;
+    const int32_t* sel_ids;
+    const int32_t* n_sel;
+    uint8_t* view_k;
+    uint8_t* view_v;
+    int32_t* status;
+    int session_first, sel_stride, max_bps, max_blocks, LG, cap_tokens;
+    float k_inv_scale, v_inv_scale;
+    size_t page_elems;
+};
+
+// One CTA pass = one (selected block, layer x KV head): the K tile is quantised straight through, the V
+// tile goes through shared memory to come out transposed.  HBM: 2 bytes read + 1 byte written per element.
+constexpr int kF8Pitch = kF8D + 4;               // bytes per token row of the staging buffer (33 words: conflict-free columns)
+__global__ void __launch_bounds__(256)
+gather_fp8_kernel(GatherF8Args a) {
+    pdl_wait();
+    __shared__ __align__(16) uint8_t sv[kF8Tile * kF8Pitch];
+    const int s = blockIdx.y;
+    const int NB = a.nblocks_dev[a.session_first + s];
+    int n_blk = a.n_sel[s];
+    const int cap_blocks = a.cap_tokens / kF8Tile;
+    if (n_blk > a.sel_stride || n_blk > cap_blocks) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE);
+        n_blk = min(min(n_blk, a.sel_stride), cap_blocks);
+    }
+    n_blk = max(n_blk, 0);
+    const long long n_items = (long long)n_blk * a.LG;
+    const int tile_elems = kF8Tile * kF8D;
+    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int j = (int)(item / a.LG), lg = (int)(item % a.LG);
+        const int id = a.sel_ids[(size_t)s * a.sel_stride + j];
+        int page = -1;
+        if (id >= 0 && id < NB) page = a.tables[(size_t)(a.session_first + s) * a.max_bps + id];
+        if (page < 0 || page >= a.max_blocks) { if (threadIdx.x == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); continue; }
+        const __nv_bfloat16* ksrc = a.pages + (size_t)page * a.page_elems + (size_t)lg * tile_elems;
+        const __nv_bfloat16* vsrc = ksrc + (size_t)a.LG * tile_elems;
+        const size_t head = (size_t)s * a.LG + lg;
+        uint8_t* kdst = a.view_k + (head * a.cap_tokens + (size_t)j * kF8Tile) * kF8D;
+        uint8_t* vdst = a.view_v + (head * cap_blocks + (size_t)j) * (size_t)tile_elems;
+        // 1,024 groups of 8 elements per tile: 4 per thread
+        uint4 kv[4], vv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int e = threadIdx.x + 256 * i;
+            kv[i] = __ldg(reinterpret_cast<const uint4*>(ksrc) + e);
+            vv[i] = __ldg(reinterpret_cast<const uint4*>(vsrc) + e);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int e = threadIdx.x + 256 * i;                  // token e / 16, dims 8 * (e % 16) ..
+            *reinterpret_cast<uint2*>(kdst + (size_t)e * 8) = quant8(kv[i], a.k_inv_scale);
+            const uint2 q = quant8(vv[i], a.v_inv_scale);
+            uint32_t* row = reinterpret_cast<uint32_t*>(sv + (e >> 4) * kF8Pitch + (e & 15) * 8);
+            row[0] = q.x; row[1] = q.y;
+        }
+        __syncthreads();
+        // transposed store: 512 pieces of 16 tokens of one dimension, 2 per thread
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int pce = threadIdx.x + 256 * i;
+            const int dim = pce >> 2, tg = pce & 3;
+            uint32_t w[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                uint32_t x = 0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) x |= (uint32_t)sv[(tg * 16 + k * 4 + b) * kF8Pitch + dim] << (8 * b);
+                w[k] = x;
+            }
+            *reinterpret_cast<uint4*>(vdst + (size_t)dim * kF8Tile + tg * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Split-K decode attention over the FP8 view.  Same structure as the bf16 kernel (producer warp with
+// TMA, two groups of four consumer warps, one partial per split, merge kernel), with 16 KiB stages
+// (an 8 KiB K tile and an 8 KiB transposed V tile) and f16 tensor-core MMAs on converted fragments.
+constexpr int kF8Stages = 8;
+constexpr int kF8Consumers = 8;
+constexpr int kF8Groups = 2;
+static_assert(kF8Stages % kF8Groups == 0, "each group must own whole stages");
+constexpr int kF8Threads = (kF8Consumers + 1) * 32;
+constexpr int kF8TileBytes = kF8Tile * kF8D;     // 8 KiB: 64 rows of 128 bytes, for K (row = token) and V^T (row = two dims)
+constexpr int kF8StageBytes = 2 * kF8TileBytes;
+constexpr int kF8RowsPad = 16;
+constexpr int kF8MergeStride = 136;
+constexpr size_t kF8Smem = (size_t)kF8Stages * kF8StageBytes + 1024;
+static_assert((size_t)kF8Consumers * kF8RowsPad * kF8MergeStride * sizeof(float) <= (size_t)kF8Stages * kF8StageBytes,
+              "the ring is reused for the merge of the consumer warps");
+
+struct AttendF8Args {
+    const __nv_bfloat16* q;
+    const int32_t* n_sel;
+    float* part_o;      // [ns*LG][n_splits][16][128]
+    float2* part_ml;    // [ns*LG][n_splits][16]
+    int32_t* status;
+    int M, L, H, G, r, rows, n_splits, cap_tokens;
+    float scale_log2e;  // softmax scale * k_scale * log2(e)
+    float v_scale;
+};
+
+__global__ void __launch_bounds__(kF8Threads, 1)
+attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, AttendF8Args a) {
+    pdl_wait();
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ uint64_t full_bar[kF8Stages], empty_bar[kF8Stages];
+    __shared__ float merge_m[kF8Consumers][kF8RowsPad], merge_l[kF8Consumers][kF8RowsPad];
+
+    unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int split = blockIdx.x, lg = blockIdx.y, s = blockIdx.z;
+    const int LG = a.L * a.G;
+    const int z = s * LG + lg;
+    const int l = lg / a.G, g = lg % a.G;
+
+    const int n_blk = max(0, min(a.n_sel[s], a.cap_tokens / kF8Tile));
+    const int t0 = (int)((long long)n_blk * split / a.n_splits);
+    const int t1 = (int)((long long)n_blk * (split + 1) / a.n_splits);
+    const int n_tiles = t1 - t0;
+    const int cap_tiles = a.cap_tokens / kF8Tile;
+
+    if (tid == 0) {
+        for (int i = 0; i < kF8Stages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kF8Consumers / kF8Groups); }
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+
+    float o[16][4];           // O accumulators: 16 n-tiles of 8 dims
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f; }
+
+    if (warp == kF8Consumers) {
+        // ---------------- producer ----------------
+        if (lane == 0 && n_tiles > 0) {
+            ptx::prefetch_tensormap(&map_k);
+            ptx::prefetch_tensormap(&map_v);
+            for (int it = 0; it < n_tiles; ++it) {
+                const int st = it % kF8Stages;
+                if (it >= kF8Stages && !ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kF8Stages) & 1) ^ 1))) {
+                    atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+                    break;
+                }
+                unsigned char* dst = stages + (size_t)st * kF8StageBytes;
+                ptx::mbar_expect_tx(&full_bar[st], kF8StageBytes);
+                ptx::tma_load_2d(dst, &map_k, 0, (z * cap_tiles + t0 + it) * kF8Tile, &full_bar[st]);                 // 64 tokens x 128 B
+                ptx::tma_load_2d(dst + kF8TileBytes, &map_v, 0, (z * cap_tiles + t0 + it) * kF8Tile, &full_bar[st]);  // 64 dim pairs x 128 B
+            }
+        }
+    } else {
+        // ---------------- consumers ----------------
+        // Q fragments in f16.  k-slot permutation inside a k16 step: slots {2c, 2c+1} of lane quad position c hold
+        // dims 16 ks + 4c + {0, 1}, slots {2c+8, 2c+9} hold dims 16 ks + 4c + {2, 3}: what one ldmatrix register of
+        // FP8 keys (four consecutive dims of a token) converts to.
+        uint32_t qf[8][4];
+        {
+            const int row_a = lane >> 2, row_b = row_a + 8;
+            const __nv_bfloat16* qa = nullptr;
+            const __nv_bfloat16* qb = nullptr;
+            if (row_a < a.rows) qa = a.q + ((((size_t)s * a.M + row_a / a.r) * a.L + l) * a.H + (size_t)g * a.r + row_a % a.r) * kF8D;
+            if (row_b < a.rows) qb = a.q + ((((size_t)s * a.M + row_b / a.r) * a.L + l) * a.H + (size_t)g * a.r + row_b % a.r) * kF8D;
+            const int kq = 4 * (lane & 3);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                float fa[4] = {0.f, 0.f, 0.f, 0.f}, fb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (qa) fa[i] = __bfloat162float(qa[ks * 16 + kq + i]);
+                    if (qb) fb[i] = __bfloat162float(qb[ks * 16 + kq + i]);
+                }
+                qf[ks][0] = ptx::pack_f16x2(fa[0], fa[1]);
+                qf[ks][1] = ptx::pack_f16x2(fb[0], fb[1]);
+                qf[ks][2] = ptx::pack_f16x2(fa[2], fa[3]);
+                qf[ks][3] = ptx::pack_f16x2(fb[2], fb[3]);
+            }
+        }
+        const uint32_t stage0 = ptx::smem_u32(stages);
+        const int mj = lane >> 3, mr = lane & 7;        // ldmatrix: matrix index and row within it
+        const int grp = warp >> 2, wq = warp & 3;       // group grp takes tiles grp, grp + 2, ...; warp wq tokens [16 wq, 16 wq + 16)
+
+        for (int it = grp; it < n_tiles; it += kF8Groups) {
+            const int st = it % kF8Stages;
+            const bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kF8Stages) & 1));
+            if (!__all_sync(0xffffffffu, arrived)) {
+                if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+                break;
+            }
+            const uint32_t kbase = stage0 + (uint32_t)st * kF8StageBytes;
+            const uint32_t vbase = kbase + kF8TileBytes;
+
+            // S = Q K^T for this warp's 16 tokens.  Column n of n-tile nt is token 4 (n / 2) + 2 nt + (n % 2) of the 16,
+            // so that a lane ends up with the probabilities of four consecutive tokens: the same four an ldmatrix register
+            // of transposed FP8 values carries.
+            float sc[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) { sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.0f; }
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                const int tok = wq * 16 + 4 * (mr >> 1) + 2 * nt + (mr & 1);
+#pragma unroll
+                for (int kh = 0; kh < 2; ++kh) {            // 64 dims = 4 chunks of 16 B = 4 k-steps
+                    const int c = kh * 4 + mj;
+                    const uint32_t addr = kbase + (uint32_t)tok * 128u + (uint32_t)((c ^ (tok & 7)) << 4);
+                    uint32_t kr[4];
+                    ptx::ldmatrix_x4(addr, kr[0], kr[1], kr[2], kr[3]);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint32_t b0, b1;
+                        ptx::e4m3x4_to_f16x2x2(kr[j], b0, b1);
+                        ptx::mma_f16_16816(sc[nt], qf[kh * 4 + j], b0, b1);
+                    }
+                }
+            }
+            // online softmax (exp2 domain); this thread holds rows lane/4 (c0,c1) and lane/4 + 8 (c2,c3)
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                sc[nt][0] *= a.scale_log2e; sc[nt][1] *= a.scale_log2e; sc[nt][2] *= a.scale_log2e; sc[nt][3] *= a.scale_log2e;
+                mx0 = fmaxf(mx0, fmaxf(sc[nt][0], sc[nt][1]));
+                mx1 = fmaxf(mx1, fmaxf(sc[nt][2], sc[nt][3]));
+            }
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+            const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+            const bool grew = (mn0 != m_run[0]) || (mn1 != m_run[1]);
+            if (__any_sync(0xffffffffu, grew)) {
+                const float corr0 = exp2f(m_run[0] - mn0), corr1 = exp2f(m_run[1] - mn1);
+                l_run[0] *= corr0; l_run[1] *= corr1;
+#pragma unroll
+                for (int nd = 0; nd < 16; ++nd) { o[nd][0] *= corr0; o[nd][1] *= corr0; o[nd][2] *= corr1; o[nd][3] *= corr1; }
+                m_run[0] = mn0; m_run[1] = mn1;
+            }
+            uint32_t pa[4];
+            {
+                const float p00 = exp2f(sc[0][0] - mn0), p01 = exp2f(sc[0][1] - mn0);
+                const float p02 = exp2f(sc[0][2] - mn1), p03 = exp2f(sc[0][3] - mn1);
+                const float p10 = exp2f(sc[1][0] - mn0), p11 = exp2f(sc[1][1] - mn0);
+                const float p12 = exp2f(sc[1][2] - mn1), p13 = exp2f(sc[1][3] - mn1);
+                l_run[0] += (p00 + p01) + (p10 + p11);
+                l_run[1] += (p02 + p03) + (p12 + p13);
+                pa[0] = ptx::pack_f16x2(p00, p01); pa[1] = ptx::pack_f16x2(p02, p03);
+                pa[2] = ptx::pack_f16x2(p10, p11); pa[3] = ptx::pack_f16x2(p12, p13);
+            }
+            // O += P V: the transposed V tile has row = dim / 2; the 16 bytes of chunk (dim & 1) * 4 + wq are this warp's
+            // 16 tokens of that dim, and a lane's register holds tokens 4 (lane & 3) .. + 3 of dim 8 nd + lane / 4
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                const int dim = (np * 4 + mj) * 8 + mr;
+                const int vr = dim >> 1, c = (dim & 1) * 4 + wq;
+                const uint32_t addr = vbase + (uint32_t)vr * 128u + (uint32_t)((c ^ (vr & 7)) << 4);
+                uint32_t vreg[4];
+                ptx::ldmatrix_x4(addr, vreg[0], vreg[1], vreg[2], vreg[3]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t b0, b1;
+                    ptx::e4m3x4_to_f16x2x2(vreg[j], b0, b1);
+                    ptx::mma_f16_16816(o[np * 4 + j], pa, b0, b1);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&empty_bar[st]);
+        }
+        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1); l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
+        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1); l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
+    }
+
+    __syncthreads();
+    float* merge_o = reinterpret_cast<float*>(stages);          // [consumer][16][kF8MergeStride]
+    if (warp < kF8Consumers) {
+        const int row_a = lane >> 2, row_b = row_a + 8, col = 2 * (lane & 3);
+        float* base = merge_o + (size_t)warp * kF8RowsPad * kF8MergeStride;
+#pragma unroll
+        for (int nd = 0; nd < 16; ++nd) {
+            *reinterpret_cast<float2*>(base + row_a * kF8MergeStride + nd * 8 + col) = make_float2(o[nd][0], o[nd][1]);
+            *reinterpret_cast<float2*>(base + row_b * kF8MergeStride + nd * 8 + col) = make_float2(o[nd][2], o[nd][3]);
+        }
+        if ((lane & 3) == 0) {
+            merge_m[warp][row_a] = m_run[0]; merge_l[warp][row_a] = l_run[0];
+            merge_m[warp][row_b] = m_run[1]; merge_l[warp][row_b] = l_run[1];
+        }
+    }
+    __syncthreads();
+    if (tid < 256) {
+        const int col = tid & 127, r0 = (tid >> 7) * 8;
+        const size_t pbase = ((size_t)z * a.n_splits + split) * kF8RowsPad;
+        for (int row = r0; row < r0 + 8; ++row) {
+            float mx = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kF8Consumers; ++w) mx = fmaxf(mx, merge_m[w][row]);
+            float acc = 0.0f, lsum = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kF8Consumers; ++w) {
+                const float mw = merge_m[w][row];
+                if (mw > -INFINITY) {
+                    const float f = exp2f(mw - mx);
+                    acc += f * merge_o[((size_t)w * kF8RowsPad + row) * kF8MergeStride + col];
+                    lsum += f * merge_l[w][row];
+                }
+            }
+            a.part_o[(pbase + row) * kF8D + col] = acc * a.v_scale;
+            if (col == 0) a.part_ml[pbase + row] = make_float2(mx, lsum);
+        }
+    }
+}
+
+// defined with the bf16 kernel: merges the splits of a head in split order
+__global__ void attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, float* __restrict__ out,
+                                    float* __restrict__ lse, int M, int L, int H, int G, int r, int n_splits);
+
+static PFN_cuTensorMapEncodeTiled_v12000 f8_encode() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+    }
+    return fn;
+}
+
+// [rows][128] bytes; box = 128 bytes x 64 rows, 128-byte swizzle
+static bool make_f8_map(CUtensorMap* map, const uint8_t* base, long long rows) {
+    PFN_cuTensorMapEncodeTiled_v12000 enc = f8_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {128, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {128};
+    cuuint32_t box[2] = {128, (cuuint32_t)kF8Tile};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t launch_gather_fp8(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids, int sel_stride,
+                              const int32_t* n_sel, uint8_t* view_k, uint8_t* view_v, int view_cap_tokens, float k_scale,
+                              float v_scale, cudaStream_t st) {
+    const Geometry& g = p.geo;
+    GatherF8Args a{};
+    a.pages = p.pages; a.tables = p.tables; a.nblocks_dev = p.nblocks_dev; a.sel_ids = sel_ids; a.n_sel = n_sel;
+    a.view_k = view_k; a.view_v = view_v; a.status = p.status_dev;
+    a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
+    a.LG = g.L * g.G; a.cap_tokens = view_cap_tokens; a.k_inv_scale = 1.0f / k_scale; a.v_inv_scale = 1.0f / v_scale;
+    a.page_elems = p.lay.page_elems;
+    const int ctas = std::max(1, p.sm_count * 8 / n_sessions);
+    launch_pdl(gather_fp8_kernel, dim3((unsigned)ctas, (unsigned)n_sessions), dim3(256), 0, st, a);
+    return cudaGetLastError();
+}
+
+static int f8_choose_splits(int heads, int max_tiles, int sms) {
+    const int overhead = 6;
+    long long best_cost = -1;
+    int best = 1;
+    for (int s = 1; s <= 64 && s <= std::max(1, max_tiles); ++s) {
+        const long long waves = ((long long)heads * s + sms - 1) / sms;
+        const long long cost = waves * ((max_tiles + s - 1) / s + overhead);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    }
+    return best;
+}
+
+cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M, const uint8_t* view_k,
+                              const uint8_t* view_v, int view_cap_tokens, const int32_t* n_sel, float scale, float k_scale,
+                              float v_scale, float* out, float* lse, void* workspace, cudaStream_t st) {
+    const Geometry& g = p.geo;
+    const int LG = g.L * g.G, heads = n_sessions * LG;
+    CUtensorMap map_k, map_v;
+    if (!make_f8_map(&map_k, view_k, (long long)heads * view_cap_tokens) || !make_f8_map(&map_v, view_v, (long long)heads * view_cap_tokens))
+        return cudaErrorInvalidValue;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(attend_fp8_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    AttendPlan plan = plan_attend(p.cfg, n_sessions, M, p.sm_count);
+    AttendF8Args a{};
+    a.q = q; a.n_sel = n_sel;
+    a.part_o = reinterpret_cast<float*>(workspace);
+    a.part_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(workspace) + plan.part_o_bytes);
+    a.status = p.status_dev;
+    a.M = M; a.L = g.L; a.H = g.H; a.G = g.G; a.r = g.r; a.rows = M * g.r;
+    a.n_splits = f8_choose_splits(heads, view_cap_tokens / kF8Tile, p.sm_count);
+    a.cap_tokens = view_cap_tokens;
+    const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
+    a.scale_log2e = sc * k_scale * 1.4426950408889634f;
+    a.v_scale = v_scale;
+    dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
+    launch_pdl(attend_fp8_split_kernel, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    launch_pdl(attend_merge_kernel, dim3((unsigned)a.rows, (unsigned)heads), dim3(kF8D), 0, st, a.part_o, a.part_ml, out, lse, M, g.L,
+               g.H, g.G, g.r, a.n_splits);
+    return cudaGetLastError();
+}
+
+}  // namespace kvmem

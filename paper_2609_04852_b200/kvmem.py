@@ -89,6 +89,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_view_cache_attend": (C.c_int, [vp, vp, i32, vp, sz, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_paged_attend": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
         "kvmem_paged_attend_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, i32, f32, vp, vp, vp, sz, vp]),
+        "kvmem_materialize_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, f32, f32, vp]),
+        "kvmem_view_attend_fp8": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, f32, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
         "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
         "kvmem_recall_step_host": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, i32, f32, vp, vp,
@@ -111,7 +113,7 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_paged_attend", "kvmem_append_blocks_rope", "kvmem_rope_rotate", "kvmem_materialize_rope",
             "kvmem_working_set_delta", "kvmem_score", "kvmem_view_cache_bytes", "kvmem_view_cache_layout",
             "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend", "kvmem_paged_attend_rope", "kvmem_topk", "kvmem_score_host_workspace_bytes",
-            "kvmem_score_host_staging_bytes", "kvmem_score_host_index")
+            "kvmem_score_host_staging_bytes", "kvmem_score_host_index", "kvmem_materialize_fp8", "kvmem_view_attend_fp8")
 
 
 def _check(status: int) -> None:
@@ -370,6 +372,31 @@ class Pool:
                                                 _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
                                                 first_position, scale, _dev(out, torch.float32), _dev(lse, torch.float32),
                                                 ws.data_ptr(), ws.numel(), _stream()))
+
+    # ---- FP8 (E4M3) execution view
+    def new_view_fp8(self, n_sessions: int, cap_tokens: int) -> Tuple[torch.Tensor, torch.Tensor]:
+        """(keys uint8 [ns][L][G][cap][d], values uint8 [ns][L][G][cap/64][d][64]) for materialize_fp8."""
+        c = self.cfg
+        k8 = torch.zeros(n_sessions, c.n_layers, c.n_kv_heads, cap_tokens, c.head_dim, dtype=torch.uint8, device=self.device)
+        v8t = torch.zeros(n_sessions, c.n_layers, c.n_kv_heads, cap_tokens // 64, c.head_dim, 64, dtype=torch.uint8,
+                          device=self.device)
+        return k8, v8t
+
+    def materialize_fp8(self, sel_ids: torch.Tensor, n_sel: torch.Tensor, k8: torch.Tensor, v8t: torch.Tensor,
+                        k_scale: float = 1.0, v_scale: float = 1.0, session_first: int = 0) -> None:
+        ns = sel_ids.shape[0]
+        _check(self.lib.kvmem_materialize_fp8(self.handle, session_first, ns, _dev(sel_ids, torch.int32), sel_ids.shape[-1],
+                                              _dev(n_sel, torch.int32), _dev(k8, torch.uint8), _dev(v8t, torch.uint8),
+                                              k8.shape[3], k_scale, v_scale, _stream()))
+
+    def view_attend_fp8(self, q: torch.Tensor, k8: torch.Tensor, v8t: torch.Tensor, n_sel: torch.Tensor, out: torch.Tensor,
+                        lse: torch.Tensor, k_scale: float = 1.0, v_scale: float = 1.0, scale: float = 0.0) -> None:
+        ns, M = q.shape[0], q.shape[1]
+        ws = self.attend_workspace(ns, M)
+        _check(self.lib.kvmem_view_attend_fp8(self.handle, ns, _dev(q, torch.bfloat16), M, _dev(k8, torch.uint8),
+                                              _dev(v8t, torch.uint8), k8.shape[3], _dev(n_sel, torch.int32), scale, k_scale,
+                                              v_scale, _dev(out, torch.float32), _dev(lse, torch.float32), ws.data_ptr(),
+                                              ws.numel(), _stream()))
 
     def view_attend_static(self, q: torch.Tensor, view: View, n_sel: torch.Tensor, out: torch.Tensor,
                            lse: torch.Tensor, scale: float = 0.0) -> None:

@@ -17,7 +17,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def _declared_functions():
     text = open(os.path.join(ROOT, "include", "kvmem.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(kvmem_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(kvmem_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_builds_loads_and_exports_every_declared_symbol():
