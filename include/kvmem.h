@@ -413,6 +413,8 @@ int kvmem_device_status(kvmem_pool_t* pool, int32_t* status /*HOST*/, void* stre
  * tensor cores (default), 0 = fp32 ALU kernel that reduces the query rows with warp shuffles.
  * "chunk_poly" (multi-token chunks): n in 2..5 = every n-th exponential of the two softmax passes is a
  * degree-4 polynomial on the FMA pipe instead of a special-function-unit instruction (default 4), 0 = none.
+ * "topk_cluster" (sessions above 16,384 blocks): 1 = selection by a thread-block cluster of 8 CTAs that merge
+ * their histograms through distributed shared memory (default), 0 = by one CTA that re-reads the scores per pass.
  * "pdl": 1 = the kernels of a step are launched with programmatic stream serialization, so that the
  * launch latency of each overlaps the tail of the one before (default), 0 = plain launches. */
 int kvmem_set_option(const char* name /*HOST*/, int32_t value);

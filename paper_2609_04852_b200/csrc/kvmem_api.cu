@@ -578,6 +578,7 @@ int kvmem_set_option(const char* name, int32_t value) {
     if (!name) { set_error("option name is null"); return KVMEM_E_INVALID; }
     if (strcmp(name, "gather_mode") == 0 && (value == 0 || value == 1)) { g_gather_mode = value; return KVMEM_OK; }
     if (strcmp(name, "chunk_poly") == 0 && (value == 0 || (value >= 2 && value <= 5))) { g_chunk_poly = value; return KVMEM_OK; }
+    if (strcmp(name, "topk_cluster") == 0 && (value == 0 || value == 1)) { g_topk_cluster = value; return KVMEM_OK; }
     if (strcmp(name, "pdl") == 0 && (value == 0 || value == 1)) { g_pdl = value; return KVMEM_OK; }
     if (strcmp(name, "score_mode") == 0 && (value == 0 || value == 1)) { g_score_mode = value; return KVMEM_OK; }
     set_error("unknown option or value: %s = %d", name, value);

@@ -12,6 +12,8 @@
 // them out coalesced: the output is chronological without a sort, and identical from run to run.
 #include <algorithm>
 
+#include <cooperative_groups.h>
+
 #include "kvmem_internal.cuh"
 
 namespace kvmem {
@@ -307,6 +309,325 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
 #undef KVMEM_TOPK_VAL
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Sessions of more than 16,384 blocks: the same selection by a thread-block cluster.  Tile t (16,384
+// consecutive ids) belongs to CTA t mod 8 of the cluster.  Every radix pass builds its histogram per CTA,
+// the eight histograms are added through distributed shared memory, and every CTA takes the same
+// decision from the same totals; the final sweep ranks the tiles through per-tile counts published the
+// same way.  All cluster-wide steps are hardware cluster barriers (no spinning), and every CTA meets
+// the same barriers because every branch between them depends on cluster-wide values only.
+constexpr int kTopkCluster = 8;
+constexpr int kTopkMaxOwnTiles = 64;             // tiles per CTA: 8 * 64 * 16,384 blocks per session at most
+
+struct TopkClusterShared {
+    unsigned int hist[kHistCopies][256];
+    unsigned int bin_tot[256];                   // this CTA's bin totals of the current pass (read by the others)
+    unsigned int all_tot[256];                   // the cluster's totals
+    unsigned int warp_tot[32];
+    unsigned int warp_min[32], warp_max[32];
+    unsigned int cta_min, cta_max;               // (read by the others)
+    unsigned int small[32], n_small;             // this CTA's candidates of a small boundary bin (read by the others)
+    unsigned int tile_counts[kTopkMaxOwnTiles];  // per own tile: kept for sure | equal to T << 16 (read by the others)
+    unsigned int prefix, remaining, bin_count;
+    unsigned int carry_sel, carry_eq;
+};
+
+__device__ __forceinline__ unsigned cluster_block_scan(unsigned val, unsigned int* warp_tot, unsigned& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned inc = val;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    const unsigned wt = warp_tot[lane];
+    unsigned winc = wt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += t;
+    }
+    const unsigned warp_off = __shfl_sync(0xffffffffu, winc - wt, warp);
+    total = __shfl_sync(0xffffffffu, winc, 31);
+    __syncthreads();
+    return warp_off + inc - val;
+}
+
+__global__ void __launch_bounds__(kTopkThreads)
+topk_cluster_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* __restrict__ nblocks_dev,
+                    int session_first, int B, kvmem_select_params_t prm, int32_t* __restrict__ sel_ids, int sel_stride,
+                    int32_t* __restrict__ n_sel, int32_t* __restrict__ status) {
+    pdl_wait();
+    pdl_trigger();
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    __shared__ TopkClusterShared sh;
+    extern __shared__ __align__(16) unsigned int stage[];   // [kTopkThreads][kStagePitch] scores of a tile, then its output ids
+    const int rank = (int)cluster.block_rank();
+    const int s = blockIdx.x / kTopkCluster, tid = threadIdx.x, lane = tid & 31;
+    const int NB = nblocks_dev[session_first + s];
+    const unsigned int* bits = reinterpret_cast<const unsigned int*>(scores + (size_t)s * scores_stride);
+    int32_t* out = sel_ids + (size_t)s * sel_stride;
+    const int n_tiles = (NB + kTopkTile - 1) / kTopkTile;
+    auto remote = [&](int r) { return cluster.map_shared_rank(&sh, r); };
+
+    long long room = (long long)prm.max_view_tokens - (long long)prm.mandatory_tokens;
+    long long kk = room <= 0 ? 0 : room <= 0x7fffffffll ? (long long)((int)room / B) : room / B;
+    if (prm.budget_blocks < kk) kk = prm.budget_blocks;
+    if (NB < kk) kk = NB;
+    if (kk < 0) kk = 0;
+    if (kk > sel_stride) {
+        if (tid == 0 && rank == 0) atomicExch(status, (int)KVMEM_E_DEVICE_RANGE);
+        kk = sel_stride;
+    }
+    const int k = (int)kk;
+    if (k == 0) {                                // cluster-uniform: nobody waits for anybody
+        if (tid == 0 && rank == 0) n_sel[s] = 0;
+        return;
+    }
+    const int n_sink = min(prm.n_sink_blocks, k);
+    int recent_lo = max(NB - prm.n_recent_blocks, n_sink);
+    recent_lo = max(recent_lo, NB - (k - n_sink));
+    recent_lo = min(max(recent_lo, 0), NB);
+    const int n_cand = recent_lo - n_sink;
+    const int kc = k - n_sink - (NB - recent_lo);
+    unsigned int T = 0xffffffffu, need_eq = 0;
+    if (tid == 0) sh.n_small = 0u;
+
+    if (kc > 0 && kc >= n_cand) {
+        T = 0u; need_eq = 0xffffffffu;
+    } else if (kc > 0) {
+        unsigned int lo = 0xffffffffu, hi = 0u;
+        // order does not matter in the counting passes: consecutive lanes read consecutive ids
+        for (int t = rank; t < n_tiles; t += kTopkCluster) {
+#pragma unroll
+            for (int i = 0; i < kItems; ++i) {
+                const int b = t * kTopkTile + i * kTopkThreads + tid;
+                if (b >= n_sink && b < recent_lo) { const unsigned int v = bits[b]; lo = min(lo, v); hi = max(hi, v); }
+            }
+        }
+        lo = __reduce_min_sync(0xffffffffu, lo);
+        hi = __reduce_max_sync(0xffffffffu, hi);
+        if (lane == 0) { sh.warp_min[tid >> 5] = lo; sh.warp_max[tid >> 5] = hi; }
+        __syncthreads();
+        if (tid < 32) {
+            lo = __reduce_min_sync(0xffffffffu, sh.warp_min[lane]);
+            hi = __reduce_max_sync(0xffffffffu, sh.warp_max[lane]);
+            if (lane == 0) { sh.cta_min = lo; sh.cta_max = hi; }
+        }
+        cluster.sync();
+        lo = 0xffffffffu; hi = 0u;
+        for (int r = 0; r < kTopkCluster; ++r) { lo = min(lo, remote(r)->cta_min); hi = max(hi, remote(r)->cta_max); }
+        if (lo == hi) {
+            T = lo; need_eq = (unsigned)kc;
+        } else {
+            const int hb = 31 - __clz(lo ^ hi);
+            unsigned int known = hb >= 31 ? 0u : ~((2u << hb) - 1u);
+            unsigned int prefix = hi & known, remaining = (unsigned)kc;      // identical in every thread of the cluster
+            for (int i = tid; i < kHistCopies * 256; i += kTopkThreads) (&sh.hist[0][0])[i] = 0u;
+            __syncthreads();
+            int shift = max(hb - 7, 0);
+            while (true) {
+                unsigned int* my_hist = sh.hist[(tid >> 5) % kHistCopies];
+                for (int t = rank; t < n_tiles; t += kTopkCluster) {
+#pragma unroll
+                    for (int i = 0; i < kItems; ++i) {
+                        const int b = t * kTopkTile + i * kTopkThreads + tid;
+                        if (b >= n_sink && b < recent_lo) {
+                            const unsigned int v = bits[b];
+                            if ((v & known) == prefix) atomicAdd(&my_hist[(v >> shift) & 255u], 1u);
+                        }
+                    }
+                }
+                __syncthreads();
+                if (tid < 256) {
+                    unsigned int t = 0;
+#pragma unroll
+                    for (int k2 = 0; k2 < kHistCopies; ++k2) { t += sh.hist[k2][tid]; sh.hist[k2][tid] = 0u; }
+                    sh.bin_tot[tid] = t;
+                }
+                cluster.sync();                              // every CTA's bin totals are in place
+                if (tid < 256) {
+                    unsigned int t = 0;
+                    for (int r = 0; r < kTopkCluster; ++r) t += remote(r)->bin_tot[tid];
+                    sh.all_tot[tid] = t;
+                }
+                __syncthreads();
+                if (tid < 32) {
+                    unsigned int c[8], mine = 0;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { c[j] = sh.all_tot[255 - 8 * lane - j]; mine += c[j]; }
+                    unsigned int inc = mine;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const unsigned int t = __shfl_up_sync(0xffffffffu, inc, o);
+                        if (lane >= o) inc += t;
+                    }
+                    const unsigned int before = inc - mine;
+                    const bool here = before < remaining && remaining <= inc;
+                    const unsigned int claim = __ballot_sync(0xffffffffu, here);
+                    if (here || (claim == 0u && lane == 31)) {
+                        unsigned int left = remaining - before;
+                        int bin = 255 - 8 * lane, j = 0;
+                        for (; j < 7; ++j) {
+                            if (c[j] >= left) break;
+                            left -= c[j];
+                            --bin;
+                        }
+                        sh.prefix = (prefix & ~(255u << shift)) | ((unsigned)bin << shift);
+                        sh.remaining = left;
+                        sh.bin_count = c[j];
+                    }
+                }
+                __syncthreads();
+                cluster.sync();                              // everybody has read everybody's totals: they may be rewritten
+                known |= 255u << shift;
+                prefix = sh.prefix; remaining = sh.remaining;
+                const unsigned int in_bin = sh.bin_count;
+                if (shift == 0) { T = prefix; need_eq = remaining; break; }
+                if (in_bin <= remaining) { T = prefix; need_eq = 0xffffffffu; break; }
+                if (in_bin <= 32u) {
+                    for (int t = rank; t < n_tiles; t += kTopkCluster) {
+#pragma unroll
+                        for (int i = 0; i < kItems; ++i) {
+                            const int b = t * kTopkTile + i * kTopkThreads + tid;
+                            if (b >= n_sink && b < recent_lo) {
+                                const unsigned int v = bits[b];
+                                if ((v & known) == prefix) {
+                                    const unsigned int slot = atomicAdd(&sh.n_small, 1u);
+                                    if (slot < 32u) sh.small[slot] = v;
+                                }
+                            }
+                        }
+                    }
+                    cluster.sync();                          // every CTA's short list is complete
+                    if (tid < 32) {
+                        // lane i takes the i-th candidate of the cluster (ranks in order, then slots in order)
+                        unsigned int mine = 0, n = 0;
+                        for (int r = 0; r < kTopkCluster; ++r) {
+                            const unsigned int nr = min(remote(r)->n_small, 32u);
+                            if ((unsigned)lane >= n && (unsigned)lane < n + nr) mine = remote(r)->small[lane - n];
+                            n += nr;
+                        }
+                        n = min(n, 32u);
+                        unsigned int gt = 0, eq = 0;
+                        for (unsigned int j = 0; j < n; ++j) {
+                            const unsigned int o = __shfl_sync(0xffffffffu, mine, (int)j);
+                            gt += o > mine;
+                            eq += o == mine;
+                        }
+                        if ((unsigned)lane < n && gt < remaining && remaining <= gt + eq) { sh.prefix = mine; sh.remaining = remaining - gt; }
+                    }
+                    __syncthreads();
+                    T = sh.prefix; need_eq = sh.remaining;
+                    break;
+                }
+                shift = max(shift - 8, 0);
+            }
+        }
+    }
+
+    // per-tile counts of what is kept for sure and of what equals T, published to the cluster
+    int n_own = 0;
+    for (int t = rank; t < n_tiles; t += kTopkCluster, ++n_own) {
+        unsigned cnt = 0;
+#pragma unroll
+        for (int i = 0; i < kItems; ++i) {
+            const int b = t * kTopkTile + i * kTopkThreads + tid;
+            if (b < NB) {
+                if (b < n_sink || b >= recent_lo) cnt += 1u;
+                else if (kc > 0) {
+                    const unsigned int v = bits[b];
+                    if (v > T) cnt += 1u;
+                    else if (v == T) cnt += 1u << 16;
+                }
+            }
+        }
+        unsigned total;
+        cluster_block_scan(cnt, sh.warp_tot, total);
+        if (tid == 0 && n_own < kTopkMaxOwnTiles) sh.tile_counts[n_own] = total;
+    }
+    cluster.sync();
+    // the ascending sweep over this CTA's tiles
+    for (int t = rank; t < n_tiles; t += kTopkCluster) {
+        if (tid == 0) {
+            // what the tiles before t keep (sequential: an equal score is kept only while need_eq lasts)
+            unsigned cs = 0, ce = 0;
+            for (int u = 0; u < t; ++u) {
+                const unsigned pc = remote(u % kTopkCluster)->tile_counts[u / kTopkCluster];
+                const unsigned eqs = pc >> 16, left = need_eq > ce ? need_eq - ce : 0u;
+                cs += (pc & 0xffffu) + min(eqs, left);
+                ce += eqs;
+            }
+            sh.carry_sel = cs; sh.carry_eq = ce;
+        }
+        __syncthreads();
+        const unsigned carry_sel = sh.carry_sel, carry_eq = sh.carry_eq;
+        const int b0 = t * kTopkTile + tid * kItems;
+        // the sweep needs id order inside a thread: coalesced loads into shared memory, then 16 consecutive ids each
+        unsigned int vreg[kItems];
+        for (int idx = tid; idx < kTopkTile; idx += kTopkThreads) {
+            const int b = t * kTopkTile + idx;
+            stage[(idx / kItems) * kStagePitch + (idx % kItems)] = b < NB ? bits[b] : 0u;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kItems; i += 4) {
+            const uint4 u = *reinterpret_cast<const uint4*>(&stage[tid * kStagePitch + i]);
+            vreg[i] = u.x; vreg[i + 1] = u.y; vreg[i + 2] = u.z; vreg[i + 3] = u.w;
+        }
+        __syncthreads();                                    // the buffer becomes the output buffer below
+        unsigned flags_res = 0, flags_gt = 0, flags_eq = 0;
+#pragma unroll
+        for (int i = 0; i < kItems; ++i) {
+            const int b = b0 + i;
+            if (b < NB) {
+                if (b < n_sink || b >= recent_lo) flags_res |= 1u << i;
+                else if (kc > 0) {
+                    const unsigned int v = vreg[i];
+                    if (v > T) flags_gt |= 1u << i;
+                    else if (v == T) flags_eq |= 1u << i;
+                }
+            }
+        }
+        const unsigned sure = flags_res | flags_gt;
+        unsigned tot_packed;
+        const unsigned ex = cluster_block_scan((unsigned)__popc(sure) | ((unsigned)__popc(flags_eq) << 16), sh.warp_tot, tot_packed);
+        unsigned eq_rank = carry_eq + (ex >> 16);
+        const unsigned tot_eq = tot_packed >> 16;
+        const unsigned eq_left_before = need_eq > carry_eq ? need_eq - carry_eq : 0u;
+        const unsigned tot_sel = (tot_packed & 0xffffu) + min(tot_eq, eq_left_before);
+        unsigned rel = (ex & 0xffffu) + min(ex >> 16, eq_left_before);
+        unsigned take = sure;
+#pragma unroll
+        for (int i = 0; i < kItems; ++i)
+            if (flags_eq & (1u << i)) { if (eq_rank < need_eq) take |= 1u << i; ++eq_rank; }
+        int* outbuf = reinterpret_cast<int*>(stage);
+#pragma unroll
+        for (int i = 0; i < kItems; ++i)
+            if (take & (1u << i)) outbuf[rel++] = b0 + i;
+        __syncthreads();
+        for (unsigned i = tid; i < tot_sel; i += kTopkThreads)
+            if (carry_sel + i < (unsigned)sel_stride) out[carry_sel + i] = outbuf[i];
+        __syncthreads();
+    }
+    if (tid == 0 && rank == 0) {
+        unsigned cs = 0, ce = 0;
+        for (int u = 0; u < n_tiles; ++u) {
+            const unsigned pc = remote(u % kTopkCluster)->tile_counts[u / kTopkCluster];
+            const unsigned eqs = pc >> 16, left = need_eq > ce ? need_eq - ce : 0u;
+            cs += (pc & 0xffffu) + min(eqs, left);
+            ce += eqs;
+        }
+        n_sel[s] = (int32_t)min(cs, (unsigned)sel_stride);
+    }
+    cluster.sync();                                          // nobody leaves while its shared memory may still be read
+}
+
+int g_topk_cluster = 1;   // sessions above 16,384 blocks: 1 = cluster of 8 CTAs, 0 = one CTA re-reading the scores
+
 cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, const float* scores,
                         int scores_stride, const kvmem_select_params_t& prm, int32_t* sel_ids, int sel_stride,
                         int32_t* n_sel, cudaStream_t st) {
@@ -320,6 +641,30 @@ cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, 
         if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_done = true;
+    }
+    const int max_tiles = (max_nb + kTopkTile - 1) / kTopkTile;
+    if (max_nb > kTopkTile && g_topk_cluster && max_tiles <= kTopkCluster * kTopkMaxOwnTiles) {
+        // long sessions: one cluster of 8 CTAs per session
+        static bool cattr_done = false;
+        if (!cattr_done) {
+            cudaError_t e = cudaFuncSetAttribute(topk_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            cattr_done = true;
+        }
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)(kTopkCluster * n_sessions));
+        cfg.blockDim = dim3(kTopkThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kTopkCluster;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, topk_cluster_kernel, scores, scores_stride, (const int32_t*)p.nblocks_dev, session_first,
+                                  p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev);
     }
     if (max_nb <= kTopkTile)
         launch_pdl(topk_kernel<true>, dim3(n_sessions), dim3(kTopkThreads), smem, st, scores, scores_stride, p.nblocks_dev, session_first,

@@ -234,6 +234,41 @@ def test_long_session_takes_the_general_top_k_path():
         assert np.array_equal(bits(got["view"].k[0])[:, :, :T], vK[:, :, :T])
 
 
+@pytest.mark.parametrize("n_scores,budget,sink,recent,kind", [
+    (16385, 300, 0, 0, "normal"), (50000, 4096, 3, 5, "normal"), (140000, 2048, 0, 0, "normal"),   # 2, 4 and 9 tiles
+    (40000, 1000, 2, 2, "ties"), (33000, 500, 0, 0, "constant"), (20000, 19990, 4, 4, "normal"), (70000, 70000, 0, 0, "normal")])
+def test_selection_from_given_scores_in_long_sessions(n_scores, budget, sink, recent, kind):
+    """kvmem_topk on sessions above 16,384 blocks: the cluster kernel and the single-CTA kernel against the oracle's
+    selector, bit for bit (scores are given, so there is nothing to tolerate), with heavy ties and reservations."""
+    from paper_2609_04852_b200 import Pool, set_option
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(n_scores)
+    if kind == "normal":
+        R = rng.random(n_scores).astype(np.float32) ** 8                    # skewed, like softmax mass
+    elif kind == "ties":
+        R = rng.integers(0, 6, n_scores).astype(np.float32) / 8.0           # six distinct values: thousands of ties
+    else:
+        R = np.full(n_scores, 0.25, np.float32)
+    # a pool that only carries the session length (tiny head geometry, no data needed for selection)
+    pool = Pool(1, 1, 1, 128, 16, 1, n_scores, n_scores, 0)
+    K = torch.zeros(n_scores * 16, 1, 1, 128, dtype=torch.bfloat16, device=dev)
+    pool.append_blocks(0, K, K)
+    scores = torch.from_numpy(R).view(1, -1).to(dev)
+    ref = orc.select(R, 16, budget, 1 << 30, 0, sink, recent)
+    for mode in (1, 0):
+        set_option("topk_cluster", mode)
+        try:
+            sel = torch.full((1, budget), -1, dtype=torch.int32, device=dev)
+            n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+            pool.topk(scores, _params(budget_blocks=budget, n_sink_blocks=sink, n_recent_blocks=recent), sel, n_sel)
+            torch.cuda.synchronize()
+            assert pool.device_status() == 0
+            got = sel.cpu().numpy()[0, : int(n_sel[0])]
+            assert np.array_equal(got, ref), f"mode {mode}: {len(got)} ids, oracle {len(ref)}"
+        finally:
+            set_option("topk_cluster", 1)
+
+
 # ------------------------------------------------------------------ working-set delta
 
 def test_working_set_delta_between_two_steps():
