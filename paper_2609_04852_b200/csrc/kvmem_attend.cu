@@ -14,6 +14,8 @@
 #include <cudaTypedefs.h>
 #include <math.h>
 
+#include <algorithm>
+
 #include "kvmem_internal.cuh"
 #include "kvmem_ptx.cuh"
 #include "kvmem_rope.cuh"
@@ -52,6 +54,7 @@ struct AttendArgs {
     const int32_t* nblocks_dev;  // [max_sessions]
     int session_first, sel_stride, max_bps, max_blocks;
     // position-consistent copy-free view (attend_split_kernel<3>): raw keys are rotated in shared memory
+    int lookahead;               // tiles the producer may run ahead of the consumers (0: as many as there are stages)
     int block_tokens;            // tokens per selected block (view length = n_sel * block_tokens); 64 in the paged modes
     const float2* rope;          // [rope_positions][64] (cos, sin)
     int first_position;          // compact position of view token 0
@@ -68,6 +71,9 @@ AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tok
     p.total = p.part_o_bytes + p.part_ml_bytes;
     return p;
 }
+
+int g_attend_lookahead = 0;   // 0: chosen in launch_attend; > 0: forced number of tiles in flight per CTA
+int g_attend_splits = 0;   // 0: chosen by the cost model below; > 0: forced (kernel-variant switch)
 
 // splits per head: fewest waves of CTAs over the SMs, counting a fixed per-CTA cost in tiles
 static int choose_splits(int heads, int max_tiles, int sms) {
@@ -123,6 +129,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     const int t0 = (int)((long long)n_blk * split / a.n_splits);
     const int t1 = (int)((long long)n_blk * (split + 1) / a.n_splits);
     const int n_tiles = t1 - t0;
+    const int ahead = a.lookahead > 0 ? min(a.lookahead, STAGES) : STAGES;
 
     if (tid == 0) {
         for (int i = 0; i < STAGES; ++i) {
@@ -147,7 +154,13 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 ptx::prefetch_tensormap(&map_v);
                 for (int it = 0; it < n_tiles; ++it) {
                     const int st = it % STAGES;
-                    if (it >= STAGES && !ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1))) {
+                    bool ok = true;
+                    if (ahead < STAGES && it >= ahead) {          // at most `ahead` tiles in flight (see the paged producer)
+                        const int jt = it - ahead;
+                        ok = ptx::mbar_wait(&empty_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1));
+                    }
+                    if (ok && it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
+                    if (!ok) {
                         atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                         break;
                     }
@@ -180,7 +193,13 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 const int page = __shfl_sync(0xffffffffu, my_page, it - base_it);
                 if (lane == 0) {
                     const int st = it % STAGES;
-                    if (it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
+                    // at most `ahead` tiles in flight: tile it - ahead has left its stage (the same phase is waited for
+                    // again, and found complete, when that stage is refilled)
+                    if (ok && ahead < STAGES && it >= ahead) {
+                        const int jt = it - ahead;
+                        ok = ptx::mbar_wait(&empty_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1));
+                    }
+                    if (ok && it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
                     if (ROPE && ok) {
                         // the (cos, sin) rows of the tile's 64 compact positions are contiguous: one 32 KiB bulk copy
                         const int tb = it % kAttGroups;              // group tb consumes tile it: one table buffer per group
@@ -536,7 +555,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     a.part_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(workspace) + plan.part_o_bytes);
     a.status = p.status_dev;
     a.M = M; a.L = g.L; a.H = g.H; a.G = g.G; a.r = g.r; a.rows = M * g.r;
-    a.n_splits = choose_splits(heads, view_cap_tokens / kTile, p.sm_count);
+    a.n_splits = g_attend_splits > 0 ? std::min(g_attend_splits, kMaxSplits) : choose_splits(heads, view_cap_tokens / kTile, p.sm_count);
     a.cap_tokens = view_cap_tokens;
     const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
     a.scale_log2e = sc * 1.4426950408889634f;
@@ -546,6 +565,19 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         a.tables = alt->tables; a.nblocks_dev = alt->nblocks_dev; a.max_bps = alt->table_stride; a.max_blocks = alt->n_pages;
     }
     a.rope = p.rope_dev; a.first_position = rope_first_position; a.block_tokens = g.B;
+    // How far the producers run ahead.  Measured on this part: a long single-wave stream is fastest with about 14 MiB
+    // in flight over all SMs when the kernel also writes the view (read/write turn-arounds in HBM grow with the number
+    // of outstanding requests) and about 19 MiB when it only reads; more stages in flight than that cost 5-7 %.
+    // Short streams and multi-wave grids keep every stage in flight.
+    a.lookahead = g_attend_lookahead;
+    if (a.lookahead == 0) {
+        const long long ctas = (long long)a.n_splits * heads;
+        const int tiles_per_cta = (view_cap_tokens / kTile + a.n_splits - 1) / a.n_splits;
+        if (ctas <= p.sm_count && tiles_per_cta >= 64) {
+            const double target = (fused && !paged_only ? 14.0 : 19.0) * 1024.0 * 1024.0;
+            a.lookahead = std::max(2, std::min(kAttStages, (int)(target / ((double)ctas * kStageBytes) + 0.5)));
+        }
+    }
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
     if (paged_only && rope_first_position >= 0)
         launch_pdl(attend_split_kernel<3>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);

@@ -76,6 +76,9 @@ extern int g_score_mode;    // 1: tensor-core decode scoring (default), 0: fp32 
 extern int g_chunk_poly;    // chunked scoring: every n-th exponential on the FMA pipe (0: all on the special-function unit)
 extern int g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
 extern int g_topk_cluster;  // 1: sessions above 16,384 blocks are selected by a cluster of 8 CTAs (default), 0: by one CTA
+extern int g_gather_ctas;
+extern int g_attend_lookahead;
+extern int g_attend_splits; // 0: split count from the cost model (default); > 0: forced
 extern int g_pdl;           // 1: the kernels of a step are launched with programmatic stream serialization (default), 0: plain launches
 
 // Programmatic dependent launch.  A kernel launched through launch_pdl may be scheduled while the previous
