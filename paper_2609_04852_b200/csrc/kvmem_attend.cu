@@ -27,12 +27,15 @@ constexpr int kAttConsumers = 8;
 constexpr int kAttGroups = 2;                   // consumer groups; kAttStages % kAttGroups == 0
 static_assert(kAttStages % kAttGroups == 0, "each group must own whole stages");
 constexpr int kAttThreads = (kAttConsumers + 1) * 32;
-constexpr int kAttRopeStages = 4;               // data stages in that mode: two stages' room holds the rotary rows of two tiles
+constexpr int kAttRopeStages = 4;               // the position-consistent paged mode: data stages,
+constexpr int kAttRopeGroups = 2;               // consumer groups (one table buffer of rotary rows each)
+constexpr int kAttRopeConsumers = 8;            // and consumer warps (12 warps in 3 groups spill at the 128-register cap: 345 us against 257)
 constexpr int kTile = 64;                       // tokens per tile == block_tokens
 constexpr int kD = 128;
 constexpr int kTabBytes = kTile * (kD / 2) * 8; // (cos, sin) fp32 of 64 pairs for 64 positions: 32 KiB
-static_assert(kAttRopeStages % kAttGroups == 0 && kAttRopeStages * 4 * kTile * 128 + 2 * kTabBytes <= kAttStages * 4 * kTile * 128,
-              "the rotary mode's data stages and table ring must fit the ring of the other modes");
+static_assert(kAttRopeStages % kAttRopeGroups == 0 && kAttRopeConsumers % kAttRopeGroups == 0 &&
+                  kAttRopeStages * 4 * kTile * 128 + kAttRopeGroups * kTabBytes <= kAttStages * 4 * kTile * 128,
+              "the rotary mode's data stages and table buffers must fit the ring of the other modes");
 constexpr int kHalfBytes = kTile * 128;         // one 64-dim half of a tile: 64 rows x 128 B
 constexpr int kStageBytes = 4 * kHalfBytes;     // K lo, K hi, V lo, V hi
 constexpr int kMaxSplits = 64;
@@ -101,7 +104,7 @@ static int choose_splits(int heads, int max_tiles, int sms) {
 // MODE 2: copy-free execution view (Sec. 5.3 "Copy-free execution-view assembly"): tiles are read from
 //         the pages through the block table and attended over; no contiguous view is written.
 template <int MODE>
-__global__ void __launch_bounds__(kAttThreads + (MODE == 1 ? 32 : 0), 1)
+__global__ void __launch_bounds__(MODE == 3 ? (kAttRopeConsumers + 1) * 32 : kAttThreads + (MODE == 1 ? 32 : 0), 1)
 attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_pages, AttendArgs a) {
     pdl_wait();        // everything earlier in the stream is complete and visible from here on
@@ -109,9 +112,12 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     constexpr bool PAGED = MODE != 0;      // the producer reads pages through the block table
     constexpr bool ROPE = MODE == 3;       // the consumers re-encode their key fragments in registers before the MMAs
     extern __shared__ unsigned char smem_dyn[];
-    constexpr int STAGES = ROPE ? kAttRopeStages : kAttStages;   // the rotary mode gives two stages' room to the table ring
-    __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages], tab_full[kAttGroups], tab_empty[kAttGroups];
-    __shared__ float merge_m[kAttConsumers][kRowsPad], merge_l[kAttConsumers][kRowsPad];
+    // the rotary mode gives the room of two data stages to one buffer of rotary rows per consumer group
+    constexpr int STAGES = ROPE ? kAttRopeStages : kAttStages;
+    constexpr int CONSUMERS = ROPE ? kAttRopeConsumers : kAttConsumers;
+    constexpr int GROUPS = ROPE ? kAttRopeGroups : kAttGroups;
+    __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages], tab_full[kAttRopeGroups], tab_empty[kAttRopeGroups];
+    __shared__ float merge_m[kAttRopeConsumers][kRowsPad], merge_l[kAttRopeConsumers][kRowsPad];
 
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -134,9 +140,9 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     if (tid == 0) {
         for (int i = 0; i < STAGES; ++i) {
             ptx::mbar_init(&full_bar[i], 1);
-            ptx::mbar_init(&empty_bar[i], kAttConsumers / kAttGroups + (FUSED ? 1 : 0));
+            ptx::mbar_init(&empty_bar[i], CONSUMERS / GROUPS + (FUSED ? 1 : 0));
         }
-        for (int i = 0; i < kAttGroups; ++i) { ptx::mbar_init(&tab_full[i], 1); ptx::mbar_init(&tab_empty[i], kAttConsumers / kAttGroups); }
+        for (int i = 0; i < GROUPS; ++i) { ptx::mbar_init(&tab_full[i], 1); ptx::mbar_init(&tab_empty[i], CONSUMERS / GROUPS); }
         ptx::fence_mbar_init();
     }
     __syncthreads();
@@ -146,7 +152,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #pragma unroll
     for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f; }
 
-    if (warp == kAttConsumers) {
+    if (warp == CONSUMERS) {
         // ---------------- producer ----------------
         if (!PAGED) {
             if (lane == 0 && n_tiles > 0) {
@@ -202,8 +208,8 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     if (ok && it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
                     if (ROPE && ok) {
                         // the (cos, sin) rows of the tile's 64 compact positions are contiguous: one 32 KiB bulk copy
-                        const int tb = it % kAttGroups;              // group tb consumes tile it: one table buffer per group
-                        if (it >= kAttGroups) ok = ptx::mbar_wait(&tab_empty[tb], (uint32_t)(((it / kAttGroups) & 1) ^ 1));
+                        const int tb = it % GROUPS;              // group tb consumes tile it: one table buffer per group
+                        if (it >= GROUPS) ok = ptx::mbar_wait(&tab_empty[tb], (uint32_t)(((it / GROUPS) & 1) ^ 1));
                         if (ok) {
                             const float2* rows = a.rope + (size_t)(a.first_position + (t0 + it) * kTile) * (kD / 2);
                             ptx::mbar_expect_tx(&tab_full[tb], kTabBytes);
@@ -225,7 +231,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (!ok) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
             }
         }
-    } else if (FUSED && warp == kAttConsumers + 1) {
+    } else if (FUSED && warp == CONSUMERS + 1) {
         // ---------------- view writer: every tile that lands in shared memory is stored to the view ----------------
         if (lane == 0 && n_tiles > 0) {
             ptx::prefetch_tensormap(&map_k);
@@ -278,10 +284,10 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         // parity wait requires.  Inside a tile, warp wq owns tokens [16 wq, 16 wq + 16).
         const int grp = warp >> 2, wq = warp & 3;
 
-        for (int it = grp; it < n_tiles; it += kAttGroups) {
+        for (int it = grp; it < n_tiles; it += GROUPS) {
             const int st = it % STAGES;
             bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / STAGES) & 1));
-            if (ROPE) arrived = arrived && ptx::mbar_wait(&tab_full[grp], (uint32_t)((it / kAttGroups) & 1));
+            if (ROPE) arrived = arrived && ptx::mbar_wait(&tab_full[grp], (uint32_t)((it / GROUPS) & 1));
             if (!__all_sync(0xffffffffu, arrived)) {          // warp-uniform decision
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
@@ -413,7 +419,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     // every issued tile has been consumed (or a wait gave up): the ring can be reused for the merge
     __syncthreads();
     float* merge_o = reinterpret_cast<float*>(stages);          // [consumer][16][kMergeStride]
-    if (warp < kAttConsumers) {
+    if (warp < CONSUMERS) {
         const int row_a = lane >> 2, row_b = row_a + 8, col = 2 * (lane & 3);
         float* base = merge_o + (size_t)warp * kRowsPad * kMergeStride;
 #pragma unroll
@@ -433,10 +439,10 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         for (int row = r0; row < r0 + 8; ++row) {
             float mx = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < kAttConsumers; ++w) mx = fmaxf(mx, merge_m[w][row]);
+            for (int w = 0; w < CONSUMERS; ++w) mx = fmaxf(mx, merge_m[w][row]);
             float acc = 0.0f, lsum = 0.0f;
 #pragma unroll
-            for (int w = 0; w < kAttConsumers; ++w) {
+            for (int w = 0; w < CONSUMERS; ++w) {
                 const float mw = merge_m[w][row];
                 if (mw > -INFINITY) {
                     const float f = exp2f(mw - mx);
@@ -580,7 +586,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     }
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
     if (paged_only && rope_first_position >= 0)
-        launch_pdl(attend_split_kernel<3>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);
+        launch_pdl(attend_split_kernel<3>, dim3(grid), dim3((kAttRopeConsumers + 1) * 32), kAttSmem, st, map_k, map_v, map_pages, a);
     else if (paged_only)
         launch_pdl(attend_split_kernel<2>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);
     else if (fused)
