@@ -396,6 +396,48 @@ def test_score_alone_equals_the_scores_select_reports_and_the_oracle(M, n_blocks
         assert np.array_equal(sc[s, :lens[s]], got["scores"][s, :lens[s]])     # same kernels, fixed merge order
 
 
+# ------------------------------------------------------------------ kernel-variant switches
+
+@pytest.mark.parametrize("name,value,bit_exact", [("pdl", 0, True), ("attend_lookahead", 2, True), ("gather_ctas", 148, True),
+                                                  ("attend_splits", 5, False), ("attend_splits", 37, False)])
+def test_kernel_variant_switches_do_not_change_results(name, value, bit_exact):
+    # scheduling knobs (launch attributes, tiles in flight, CTA counts) leave every byte alone; a different split count
+    # changes only the order of the split-K merge
+    from paper_2609_04852_b200 import set_option
+    spec = SMALL.with_(n_blocks=700, budget_blocks=333, n_q_tokens=4)
+    pool = fill_pool(spec)
+    q, _ = queries(spec)
+    dev = torch.device("cuda", 0)
+
+    def run():
+        sel = torch.zeros(1, 333, dtype=torch.int32, device=dev)
+        n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+        pool.select(q.to(dev), _params(budget_blocks=333), sel, n_sel)
+        view, view2 = pool.new_view(1, 333 * 64), pool.new_view(1, 333 * 64)
+        out, lse = pool.new_outputs(1, 4)
+        out2, lse2 = pool.new_outputs(1, 4)
+        out3, lse3 = pool.new_outputs(1, 4)
+        pool.materialize(sel, n_sel, view)
+        pool.view_attend(q.to(dev), view, n_sel, out, lse)
+        pool.materialize_attend(q.to(dev), sel, n_sel, view2, out2, lse2)
+        pool.paged_attend(q.to(dev), sel, n_sel, out3, lse3)
+        torch.cuda.synchronize()
+        assert pool.device_status() == 0
+        return sel, view.k, view.v, view2.k, view2.v, out, lse, out2, lse2, out3, lse3
+
+    base = run()
+    set_option(name, value)
+    try:
+        got = run()
+    finally:
+        set_option(name, 1 if name == "pdl" else 0)
+    for i, (a, b) in enumerate(zip(base, got)):
+        if bit_exact or i < 5:
+            assert torch.equal(a, b), (name, i)
+        else:
+            assert (a - b).abs().max().item() <= ATTN_ATOL, (name, i)
+
+
 # ------------------------------------------------------------------ index in host memory, streamed in tiles
 
 @pytest.mark.parametrize("n_blocks,tile_blocks,M,pinned", [(1000, 256, 4, True), (333, 128, 1, True), (700, 1024, 2, False),
