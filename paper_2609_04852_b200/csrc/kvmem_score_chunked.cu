@@ -420,14 +420,17 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 }
 
 // Between the passes: shift = -(max + log2 Z) of every query row, merging the row statistics of all
-// tile runs and column slices in a fixed order; -inf switches a padding row off in pass 2.
+// tile runs and column slices; -inf switches a padding row off in pass 2.  One warp per row (a long
+// history has hundreds of partials per row): every lane folds a strided share, then a butterfly whose
+// operand order is fixed, so the result is the same bits in every lane and from run to run.
 __global__ void __launch_bounds__(256)
 score_chunk_shift_kernel(ChunkArgs a) {
-    pdl_wait();        // everything earlier in the stream is complete and visible from here on
-    pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
+    pdl_wait();
+    pdl_trigger();
     const int LG = a.L * a.G;
     const long long total = (long long)a.n_sessions * LG * a.shift_stride;
-    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    const long long e = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;      // one warp per row
+    const int lane = threadIdx.x & 31;
     if (e >= total) return;
     const int j = (int)(e % a.shift_stride);
     const int head = (int)(e / a.shift_stride);
@@ -438,16 +441,26 @@ score_chunk_shift_kernel(ChunkArgs a) {
     if (j < a.rows && live_chunks > 0) {
         const float2* rs = a.rowstat + ((size_t)head * a.n_chunks * kCkSplit) * a.rows_pad + j;
         const int n_part = live_chunks * kCkSplit;
-        float mx = -INFINITY;
-        for (int h = 0; h < n_part; ++h) mx = fmaxf(mx, rs[(size_t)h * a.rows_pad].x);
-        float z = 0.0f;
-        for (int h = 0; h < n_part; ++h) {
+        float mx = -INFINITY, z = 0.0f;
+        for (int h = lane; h < n_part; h += 32) {
             const float2 pp = rs[(size_t)h * a.rows_pad];
-            z += pp.x > -INFINITY ? pp.y * exp2f(pp.x - mx) : 0.0f;
+            if (pp.x > -INFINITY) {
+                const float nm = fmaxf(mx, pp.x);
+                z = z * exp2f(mx - nm) + pp.y * exp2f(pp.x - nm);
+                mx = nm;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, mx, o), oz = __shfl_xor_sync(0xffffffffu, z, o);
+            const float nm = fmaxf(mx, om);
+            const float za = mx > -INFINITY ? z * exp2f(mx - nm) : 0.0f, zb = om > -INFINITY ? oz * exp2f(om - nm) : 0.0f;
+            z = (lane & o) ? zb + za : za + zb;         // same operand order on both partners: identical bits in every lane
+            mx = nm;
         }
         sh = -(mx + log2f(z));
     }
-    a.shift[e] = sh;
+    if (lane == 0) a.shift[e] = sh;
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -740,7 +753,7 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
     const int n_items2 = n_sessions * LG * a.n_bpanels;
     const int grid1 = std::min(n_items1, p.sm_count), grid2 = std::min(n_items2, p.sm_count);
     const long long n_shift = (long long)n_sessions * LG * a.shift_stride;
-    const int sgrid = (int)((n_shift + 255) / 256);
+    const int sgrid = (int)((n_shift * 32 + 255) / 256);             // one warp per row
     cudaError_t e = cudaSuccess;
 #define KVMEM_CHUNK_PASSES(POLY)                                                                                              \
     do {                                                                                                                      \
