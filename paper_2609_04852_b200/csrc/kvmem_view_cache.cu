@@ -70,7 +70,7 @@ view_cache_reset_kernel(CachePtrs c, int cap) {
 constexpr int kPlanThreads = 1024;
 
 // position of `id` in the ascending list ids[0..n), or -1
-__device__ __forceinline__ int find_sorted(const int32_t* __restrict__ ids, int n, int id) {
+__device__ __forceinline__ int find_sorted(const int32_t* ids, int n, int id) {
     int lo = 0, hi = n;
     while (lo < hi) {
         const int mid = (lo + hi) >> 1;
@@ -87,6 +87,7 @@ view_cache_plan_kernel(CachePtrs c, int cap, const int32_t* __restrict__ sel_ids
     pdl_trigger();
     __shared__ unsigned int warp_tot[32];
     __shared__ int sh_stats[4];
+    extern __shared__ int32_t sel_sm[];             // the selection, for the binary searches: [cap]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int n = *n_sel;
     if (n < 0 || n > cap) {
@@ -95,12 +96,12 @@ view_cache_plan_kernel(CachePtrs c, int cap, const int32_t* __restrict__ sel_ids
     }
     const int NB = nblocks_dev[session];
     if (tid < 4) sh_stats[tid] = 0;
-    for (int j = tid; j < cap; j += kPlanThreads) c.view_slots[j] = -1;
+    for (int j = tid; j < cap; j += kPlanThreads) { c.view_slots[j] = -1; sel_sm[j] = j < n ? sel_ids[j] : 0x7fffffff; }
     __syncthreads();
     // 1. retained blocks keep their slot; every other slot is reclaimed
     for (int s = tid; s < cap; s += kPlanThreads) {
         const int b = c.slot_block[s];
-        const int j = b >= 0 ? find_sorted(sel_ids, n, b) : -1;
+        const int j = b >= 0 ? find_sorted(sel_sm, n, b) : -1;
         if (j >= 0) c.view_slots[j] = s;
         else c.slot_block[s] = -1;
     }
@@ -138,7 +139,7 @@ view_cache_plan_kernel(CachePtrs c, int cap, const int32_t* __restrict__ sel_ids
     int st[4] = {0, 0, 0, 0};
     for (int j = r0; j < r1; ++j) {
         if (j >= n) break;
-        const int id = sel_ids[j];
+        const int id = sel_sm[j];
         if (id < 0 || id >= NB) atomicExch(status, (int)KVMEM_E_DEVICE_RANGE);
         int slot = c.view_slots[j], act, old = j;
         if (slot < 0) {
@@ -253,7 +254,12 @@ cudaError_t launch_view_cache_update(const kvmem_pool& p, int session, const int
     const Geometry& g = p.geo;
     const CacheLayout lay = cache_layout(p.lay.page_elems, cap);
     const CachePtrs c = cache_ptrs(cache, lay);
-    launch_pdl(view_cache_plan_kernel, dim3(1), dim3(kPlanThreads), 0, st, c, cap, sel_ids, n_sel, p.nblocks_dev, session,
+    const size_t plan_smem = (size_t)cap * sizeof(int32_t);
+    if (plan_smem > 48 * 1024) {
+        cudaError_t ea = cudaFuncSetAttribute(view_cache_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_smem);
+        if (ea != cudaSuccess) return ea;
+    }
+    launch_pdl(view_cache_plan_kernel, dim3(1), dim3(kPlanThreads), plan_smem, st, c, cap, sel_ids, n_sel, p.nblocks_dev, session,
                max_delta, stats, p.status_dev);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
