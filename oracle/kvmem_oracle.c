@@ -330,10 +330,14 @@ int kvo_rope_rotate(const bf16_t* x, bf16_t* y, int64_t n_rows, int n_vec, int d
 }
 
 /* Execution view with position-consistent keys: as kvo_gather, but the raw key of view token
- * j*B + t is rotated to compact position first_pos + j*B + t; values are copied unchanged. */
+ * j*B + t is rotated to compact position first_pos + j*B + t; values are copied unchanged.
+ * in_block != 0: the pages hold keys that already carry the rotation of their offset t inside
+ * their block (a position-independent encoding too: t never changes); the view key is then the
+ * stored key rotated by the block's compact position first_pos + j*B alone, which is the same
+ * rotation R(first_pos + j*B + t) of the raw key up to the rounding of the stored key. */
 int kvo_gather_rope(const bf16_t* pagesK, const bf16_t* pagesV, const int32_t* table, const int32_t* sel,
                     int64_t n_sel, int B, int L, int G, int d, bf16_t* viewK, bf16_t* viewV, int64_t cap_tokens,
-                    int64_t first_pos, const float* tab, int64_t n_pos) {
+                    int64_t first_pos, const float* tab, int64_t n_pos, int in_block) {
     if (first_pos < 0 || first_pos + n_sel * B > n_pos) return -1;
     const size_t page = (size_t)B * L * G * d;
 #pragma omp parallel for schedule(static)
@@ -344,7 +348,7 @@ int kvo_gather_rope(const bf16_t* pagesK, const bf16_t* pagesV, const int32_t* t
                 for (int g = 0; g < G; ++g) {
                     const size_t s = src + (((size_t)t * L + l) * G + g) * d;
                     const size_t o = (((size_t)l * G + g) * cap_tokens + (size_t)j * B + t) * d;
-                    kvo_rotate_vec(pagesK + s, viewK + o, d, tab + (size_t)(first_pos + j * B + t) * (d / 2) * 2, 0);
+                    kvo_rotate_vec(pagesK + s, viewK + o, d, tab + (size_t)(first_pos + j * B + (in_block ? 0 : t)) * (d / 2) * 2, 0);
                     memcpy(viewV + o, pagesV + s, (size_t)d * sizeof(bf16_t));
                 }
     }
@@ -404,13 +408,14 @@ void kvo_working_set_delta(const int32_t* prev, int64_t n_prev, const int32_t* n
  * Readings: the slot policy (lowest free slot, ascending ids) and the counter semantics (a limit on
  * operations between reconstructions, reset by a reconstruction) are ours; the paper fixes neither.
  * cacheK / cacheV: [cap][B][L][G][d] (token-major, like the repository pages of this file).
- * d <= 1024.  Returns -1 if n_sel > cap or the compact positions leave the table.
+ * in_block: as in kvo_gather_rope (keys stored with the rotation of their in-block offset; loads and rebuilds
+ * rotate by the block's position alone).  d <= 1024.  Returns -1 if n_sel > cap or positions leave the table.
  */
 int kvo_view_cache_update(const bf16_t* pagesK, const bf16_t* pagesV, const int32_t* table, const int32_t* sel,
                           int64_t n_sel, int B, int L, int G, int d, int64_t cap, int64_t max_delta,
                           int64_t first_pos, const float* tab, int64_t n_pos, bf16_t* cacheK, bf16_t* cacheV,
                           int32_t* slot_block, int32_t* slot_pos, int32_t* slot_cnt, int32_t* view_slots,
-                          int32_t* stats) {
+                          int32_t* stats, int in_block) {
     if (n_sel > cap || first_pos < 0 || first_pos + n_sel * B > n_pos) return -1;
     const size_t page = (size_t)B * L * G * d;
     const int n_vec = L * G;
@@ -435,7 +440,7 @@ int kvo_view_cache_update(const bf16_t* pagesK, const bf16_t* pagesV, const int3
         for (int t = 0; t < B; ++t)
             for (int v = 0; v < n_vec; ++v) {
                 const size_t o = ((size_t)t * n_vec + v) * d;
-                kvo_rotate_vec(pagesK + src + o, cacheK + dst + o, d, tab + (size_t)(first_pos + j * B + t) * (d / 2) * 2, 0);
+                kvo_rotate_vec(pagesK + src + o, cacheK + dst + o, d, tab + (size_t)(first_pos + j * B + (in_block ? 0 : t)) * (d / 2) * 2, 0);
             }
         memcpy(cacheV + dst, pagesV + src, page * sizeof(bf16_t));
         slot_block[s] = sel[j]; slot_pos[s] = (int32_t)j; slot_cnt[s] = 0;
@@ -464,7 +469,7 @@ int kvo_view_cache_update(const bf16_t* pagesK, const bf16_t* pagesV, const int3
             for (int t = 0; t < B; ++t)
                 for (int v = 0; v < n_vec; ++v) {
                     const size_t o = ((size_t)t * n_vec + v) * d;
-                    kvo_rotate_vec(pagesK + src + o, cacheK + dst + o, d, tab + (size_t)(first_pos + j * B + t) * (d / 2) * 2, 0);
+                    kvo_rotate_vec(pagesK + src + o, cacheK + dst + o, d, tab + (size_t)(first_pos + j * B + (in_block ? 0 : t)) * (d / 2) * 2, 0);
                 }
             slot_cnt[s] = 0;
             stats[2] += 1;
@@ -593,6 +598,51 @@ void kvo_attend_fp8(const bf16_t* q, const uint8_t* viewK8, const uint8_t* viewV
             const double p = exp(s[t] - best) / sum;
             const size_t vbase = (head * (size_t)(cap_tokens / 64) + (size_t)(t / 64)) * d;
             for (int c = 0; c < d; ++c) o[c] += p * ((double)e4m3_to_f32(viewV8T[(vbase + c) * 64 + (size_t)(t % 64)]) * v_scale);
+        }
+        for (int c = 0; c < d; ++c) out[row * d + c] = (float)o[c];
+        lse[row] = T > 0 ? (float)(best + log(sum)) : -INFINITY;
+        free(s); free(o);
+    }
+}
+
+/* =======================================================================================
+ * Attention with position-consistent keys when the pages hold in-block-rotated keys k' = R(t) k
+ * (kvo_gather_rope with in_block): the logit q . R(p0 + t) k equals (R(-p0) q) . k', so the
+ * query is rotated back by the compact position p0 = first_pos + tile*B of each tile of B tokens
+ * instead of the keys forward.  The rotated query is a bf16 vector (the arithmetic of
+ * kvo_rope_rotate, inverse), which is what the tensor cores are fed; everything after it is
+ * kvo_attend.  viewK: plain gather (kvo_gather) of the stored keys k'.  B = tokens per tile.
+ */
+void kvo_attend_qrot(const bf16_t* q, const bf16_t* viewK, const bf16_t* viewV, int64_t T, int64_t cap_tokens,
+                     int M, int L, int H, int G, int d, int B, int64_t first_pos, const float* tab, double scale,
+                     float* out, float* lse) {
+    const int r = H / G;
+    const int64_t rows = (int64_t)M * L * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t row = 0; row < rows; ++row) {
+        const int h = (int)(row % H);
+        const int l = (int)((row / H) % L);
+        const int g = h / r;
+        const bf16_t* qv = q + row * d;
+        const bf16_t* Kg = viewK + ((size_t)l * G + g) * (size_t)cap_tokens * d;
+        const bf16_t* Vg = viewV + ((size_t)l * G + g) * (size_t)cap_tokens * d;
+        double* s = (double*)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1));
+        double* o = (double*)calloc((size_t)d, sizeof(double));
+        bf16_t qr[1024];
+        double best = -INFINITY;
+        for (int64_t t = 0; t < T; ++t) {
+            if (t % B == 0) kvo_rotate_vec(qv, qr, d, tab + (size_t)(first_pos + t) * (d / 2) * 2, 1);
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c)
+                acc += (double)bf16_to_f32(qr[c]) * (double)bf16_to_f32(Kg[(size_t)t * d + c]);
+            s[t] = acc * scale;
+            if (s[t] > best) best = s[t];
+        }
+        double sum = 0.0;
+        for (int64_t t = 0; t < T; ++t) sum += exp(s[t] - best);
+        for (int64_t t = 0; t < T; ++t) {
+            const double p = exp(s[t] - best) / sum;
+            for (int c = 0; c < d; ++c) o[c] += p * (double)bf16_to_f32(Vg[(size_t)t * d + c]);
         }
         for (int c = 0; c < d; ++c) out[row * d + c] = (float)o[c];
         lse[row] = T > 0 ? (float)(best + log(sum)) : -INFINITY;

@@ -60,11 +60,13 @@ def lib():
         L.kvo_rope_table.restype = None
         L.kvo_rope_rotate.argtypes = [p, p, i64, i32, i32, p, p, i64, i32]
         L.kvo_rope_rotate.restype = i32
-        L.kvo_gather_rope.argtypes = [p, p, p, p, i64, i32, i32, i32, i32, p, p, i64, i64, p, i64]
+        L.kvo_gather_rope.argtypes = [p, p, p, p, i64, i32, i32, i32, i32, p, p, i64, i64, p, i64, i32]
         L.kvo_gather_rope.restype = i32
         L.kvo_working_set_delta.argtypes = [p, i64, p, i64, p, p, p, p]
         L.kvo_working_set_delta.restype = None
-        L.kvo_view_cache_update.argtypes = [p, p, p, p, i64, i32, i32, i32, i32, i64, i64, i64, p, i64, p, p, p, p, p, p, p]
+        L.kvo_view_cache_update.argtypes = [p, p, p, p, i64, i32, i32, i32, i32, i64, i64, i64, p, i64, p, p, p, p, p, p, p, i32]
+        L.kvo_attend_qrot.argtypes = [p, p, p, i64, i64, i32, i32, i32, i32, i32, i32, i64, p, dbl, p, p]
+        L.kvo_attend_qrot.restype = None
         L.kvo_view_cache_update.restype = i32
         L.kvo_view_cache_view.argtypes = [p, p, p, i64, i32, i32, i32, i32, p, p, i64]
         L.kvo_view_cache_view.restype = None
@@ -217,18 +219,35 @@ def rope_rotate(x: np.ndarray, pos: np.ndarray, tab: np.ndarray, inverse: bool =
 
 
 def gather_rope(repo: Repository, table: np.ndarray, sel: np.ndarray, cap_tokens: int, first_pos: int,
-                tab: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
-    """Execution view whose keys carry RoPE at their compact positions first_pos + j*B + t."""
+                tab: np.ndarray, in_block: bool = False) -> Tuple[np.ndarray, np.ndarray]:
+    """Execution view whose keys carry RoPE at their compact positions first_pos + j*B + t.  in_block: the pages
+    hold keys already rotated by their offset t inside the block; the view rotates them by first_pos + j*B."""
     _, B, L, G, d = repo.pagesK.shape
     assert table.dtype == np.int32 and sel.dtype == np.int32 and len(sel) * B <= cap_tokens
     viewK = np.zeros((L, G, cap_tokens, d), np.uint16)
     viewV = np.zeros((L, G, cap_tokens, d), np.uint16)
     rc = lib().kvo_gather_rope(_ptr(repo.pagesK), _ptr(repo.pagesV), _ptr(np.ascontiguousarray(table)),
                                _ptr(np.ascontiguousarray(sel)), len(sel), B, L, G, d, _ptr(viewK), _ptr(viewV),
-                               cap_tokens, first_pos, _ptr(tab), tab.shape[0])
+                               cap_tokens, first_pos, _ptr(tab), tab.shape[0], int(in_block))
     if rc != 0:
         raise ValueError("compact positions outside the RoPE table")
     return viewK, viewV
+
+
+def attend_qrot(q: np.ndarray, viewK: np.ndarray, viewV: np.ndarray, T: int, block_tokens: int, first_pos: int,
+                tab: np.ndarray, scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Attention over a plain gather of in-block-rotated keys, the query rotated back by each tile's position."""
+    _u16(q), _u16(viewK), _u16(viewV)
+    M, L, H, d = q.shape
+    G, cap = viewK.shape[1], viewK.shape[2]
+    assert first_pos + T <= tab.shape[0] and T <= cap
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    out = np.zeros((M, L, H, d), np.float32)
+    lse = np.zeros((M, L, H), np.float32)
+    lib().kvo_attend_qrot(_ptr(q), _ptr(viewK), _ptr(viewV), T, cap, M, L, H, G, d, block_tokens, first_pos, _ptr(tab),
+                          float(scale), _ptr(out), _ptr(lse))
+    return out, lse
 
 
 # ---- working-set delta ---------------------------------------------------------------------------
@@ -263,7 +282,7 @@ class ViewCache:
         self.n_view = 0
 
     def update(self, repo: Repository, table: np.ndarray, sel: np.ndarray, max_delta: int, first_pos: int,
-               tab: np.ndarray) -> np.ndarray:
+               tab: np.ndarray, in_block: bool = False) -> np.ndarray:
         """Move the cache to the working set `sel`; returns stats (unmoved, delta re-RoPEd, rebuilt, incoming)."""
         B, L, G, d = self.dims
         sel = np.ascontiguousarray(sel, np.int32)
@@ -271,7 +290,7 @@ class ViewCache:
         rc = lib().kvo_view_cache_update(_ptr(repo.pagesK), _ptr(repo.pagesV), _ptr(np.ascontiguousarray(table)), _ptr(sel),
                                          len(sel), B, L, G, d, self.cap, max_delta, first_pos, _ptr(tab), tab.shape[0],
                                          _ptr(self.K), _ptr(self.V), _ptr(self.slot_block), _ptr(self.slot_pos),
-                                         _ptr(self.slot_cnt), _ptr(self.view_slots), _ptr(stats))
+                                         _ptr(self.slot_cnt), _ptr(self.view_slots), _ptr(stats), int(in_block))
         if rc != 0:
             raise ValueError("selection larger than the cache, or compact positions outside the RoPE table")
         self.n_view = len(sel)

@@ -149,3 +149,17 @@ def test_selection_larger_than_the_cache_is_refused():
     except ValueError:
         return
     raise AssertionError("expected a refusal")
+
+
+def test_in_block_layout_loads_and_rebuilds_with_the_block_position_only():
+    rng, K, V, table, repo, tab, cache = _setup(cap=8, n_pos=512)
+    # store k' = R(t) k instead of the raw keys
+    t_in_block = (np.arange(NB * B) % B).astype(np.int32)
+    Kp = orc.rope_rotate(np.ascontiguousarray(K.reshape(NB * B, L * G, d)), t_in_block, tab).reshape(K.shape)
+    stored = orc.Repository.empty(NB, B, L, G, d)
+    stored.place(Kp, V, table)
+    for step, sel in enumerate([_ids(3, 6, 9, 12), _ids(6, 9, 12, 20), _ids(1, 6, 12, 20, 22)]):
+        cache.update(stored, table, sel, max_delta=0, first_pos=10, tab=tab, in_block=True)     # always rebuilt
+        vK, vV = cache.view(8 * B)
+        gK, gV = orc.gather_rope(stored, table, sel, 8 * B, 10, tab, in_block=True)
+        assert np.array_equal(vK, gK) and np.array_equal(vV, gV), step

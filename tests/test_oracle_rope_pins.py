@@ -116,3 +116,73 @@ def test_gather_rope_rotates_keys_to_compact_positions_and_copies_values():
     # with an all-zero position table offset (first_pos = 0, single block at j = 0, t = 0) the first token is unrotated
     vK0, _ = orc.gather_rope(repo, table, sel[:1], B, 0, tab)
     assert np.array_equal(vK0[:, :, 0, :], K[sel[0] * B])
+
+
+# ---- keys stored with the rotation of their offset inside the block ("in-block" layout) -------------------
+
+def _in_block_repo(B=8, L=1, G=2, d=32, NB=10, seed=21, n_pos=512):
+    r = np.random.default_rng(seed)
+    K = to_bits(r.standard_normal((NB * B, L, G, d)).astype(np.float32))
+    V = to_bits(r.standard_normal((NB * B, L, G, d)).astype(np.float32))
+    tab = orc.rope_table(n_pos, d, THETA)
+    t_in_block = (np.arange(NB * B) % B).astype(np.int32)
+    Kp = orc.rope_rotate(K.reshape(NB * B, L * G, d), t_in_block, tab).reshape(K.shape)      # k' = R(t) k
+    table = r.permutation(NB).astype(np.int32)
+    raw, stored = orc.Repository.empty(NB, B, L, G, d), orc.Repository.empty(NB, B, L, G, d)
+    raw.place(K, V, table)
+    stored.place(Kp, V, table)
+    return r, K, V, Kp, table, raw, stored, tab
+
+
+def test_in_block_view_rotates_stored_keys_by_the_block_position_only():
+    _, _, _, Kp, table, raw, stored, tab = _in_block_repo()
+    B, L, G, d = 8, 1, 2, 32
+    sel = np.array([1, 4, 7, 8], np.int32)
+    first = 19
+    vK, vV = orc.gather_rope(stored, table, sel, 5 * B, first, tab, in_block=True)
+    for j, b in enumerate(sel):
+        rows = np.ascontiguousarray(Kp[b * B:(b + 1) * B].reshape(B, L * G, d))
+        want = orc.rope_rotate(rows, np.full(B, first + j * B, np.int32), tab).reshape(B, L, G, d)   # one angle per block
+        assert np.array_equal(vK[:, :, j * B:(j + 1) * B].transpose(2, 0, 1, 3), want)
+    # the same keys, to two bf16 roundings, as rotating the raw keys to first + j*B + t (rotations add)
+    rK, rV = orc.gather_rope(raw, table, sel, 5 * B, first, tab)
+    assert np.array_equal(vV, rV)
+    assert np.abs(from_bits(vK) - from_bits(rK)).max() <= 2.0 ** -5
+
+
+def test_query_rotation_gives_the_logits_of_rotated_keys():
+    r, _, _, _, table, raw, stored, tab = _in_block_repo(seed=33)
+    B, L, G, d, H, M = 8, 1, 2, 32, 4, 2
+    sel = np.array([0, 2, 3, 6, 9], np.int32)
+    T, cap, first = len(sel) * B, 6 * B, 40
+    q = to_bits(r.standard_normal((M, L, H, d)).astype(np.float32))
+    sK, sV = orc.gather(stored, table, sel, cap)                         # the stored keys, not rotated further
+    O1, lse1 = orc.attend_qrot(q, sK, sV, T, B, first, tab)
+    # (R(-p0) q) . k' = q . R(p0) k': attention over the view that kvo_gather_rope builds from the same pages
+    vK, vV = orc.gather_rope(stored, table, sel, cap, first, tab, in_block=True)
+    O2, lse2 = orc.attend(q, vK, vV, T)
+    assert np.abs(O1 - O2).max() < 2e-2 and np.abs(lse1 - lse2).max() < 2e-2
+    # and over the view of raw keys rotated to their compact positions
+    rK, rV = orc.gather_rope(raw, table, sel, cap, first, tab)
+    O3, lse3 = orc.attend(q, rK, rV, T)
+    assert np.abs(O1 - O3).max() < 3e-2 and np.abs(lse1 - lse3).max() < 3e-2
+
+
+def test_query_rotation_at_position_zero_is_plain_attention_over_the_stored_keys():
+    r, _, _, _, table, _, stored, tab = _in_block_repo(seed=5)
+    B, d = 8, 32
+    q = to_bits(r.standard_normal((1, 1, 4, d)).astype(np.float32))
+    sel = np.array([3], np.int32)
+    sK, sV = orc.gather(stored, table, sel, B)
+    O1, lse1 = orc.attend_qrot(q, sK, sV, B, B, 0, tab)                   # one tile at position 0: R(0) = identity
+    O2, lse2 = orc.attend(q, sK, sV, B)
+    assert np.array_equal(O1, O2) and np.array_equal(lse1, lse2)
+    # the rotated query itself: each tile uses the bf16 query of kvo_rope_rotate(inverse) at its position
+    sel2 = np.array([3, 5], np.int32)
+    sK2, sV2 = orc.gather(stored, table, sel2, 2 * B)
+    q_rot = orc.rope_rotate(np.ascontiguousarray(q.reshape(1, 4, d)), np.array([B], np.int32), tab, inverse=True).reshape(q.shape)
+    # logits of the second tile alone, from LSEs: lse(both) = log(exp(lse(tile 0 with q)) + exp(lse(tile 1 with q_rot)))
+    _, l_both = orc.attend_qrot(q, sK2, sV2, 2 * B, B, 0, tab)
+    _, l0 = orc.attend(q, sK2[:, :, :B].copy(), sV2[:, :, :B].copy(), B)
+    _, l1 = orc.attend(q_rot, sK2[:, :, B:].copy(), sV2[:, :, B:].copy(), B)
+    assert np.allclose(l_both, np.logaddexp(l0, l1), atol=1e-5)
