@@ -138,12 +138,12 @@ def rope_window(spec):
     return spec.max_view_tokens + 64
 
 
-def fill_pool(spec, device, seed_shift=0, rope=False):
+def fill_pool(spec, device, seed_shift=0, rope=False, in_block=False):
     from paper_2609_04852_b200 import Pool
     spec = spec.with_(seed=spec.seed + seed_shift)
     pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.block_tokens,
                 spec.n_sessions, spec.n_sessions * spec.n_blocks, spec.n_blocks, device.index,
-                rope_window(spec) if rope else 0, ROPE_THETA if rope else 0.0)
+                rope_window(spec) if rope else 0, ROPE_THETA if rope else 0.0, rope_in_block_keys=in_block)
     tables = page_table(spec)
     B = spec.block_tokens
     for s in range(spec.n_sessions):
@@ -186,7 +186,7 @@ def run_native(args):
         else:
             base = base.with_(name=f"{base.name}@{args.blocks}", n_blocks=args.blocks,
                               n_planted=max(1, int(base.n_planted * f)), budget_blocks=max(1, int(base.budget_blocks * f)))
-    pool, spec = fill_pool(base, device, seed_shift=1000 * rank, rope=args.rope)     # one independent replica per rank
+    pool, spec = fill_pool(base, device, seed_shift=1000 * rank, rope=args.rope, in_block=args.in_block)     # one independent replica per rank
     ns, M, B = spec.n_sessions, spec.n_q_tokens, spec.block_tokens
     prm = SelectParams(**select_params(spec))
     from paper_2609_04852_b200 import budget_blocks
@@ -390,7 +390,9 @@ def run_native(args):
                        "l2": "flushed between steps (256 MiB write)" if flush is not None else
                              "no flush: every step streams far more than the 126 MB L2",
                        "parallelism": f"{world} independent session replica(s), one per GPU",
-                       "calls": "kvmem_rope_rotate(q) + kvmem_select + kvmem_paged_attend_rope (copy-free, keys RoPE'd in shared memory)"
+                       "calls": "kvmem_rope_rotate(q) + kvmem_select + kvmem_paged_attend_rope (copy-free, pages hold RoPE(k, in-block offset), "
+                                "the query rotated back once per block)" if args.rope and args.paged and args.in_block else
+                                "kvmem_rope_rotate(q) + kvmem_select + kvmem_paged_attend_rope (copy-free, keys RoPE'd in shared memory)"
                                 if args.rope and args.paged else
                                 "kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_rope + kvmem_view_attend" if args.rope else
                                 "kvmem_select + kvmem_paged_attend (NO materialize: copy-free view variant)" if args.paged else
@@ -402,7 +404,9 @@ def run_native(args):
                     "api": "kvmem_recall_step_host (pinned host query in, host O and LSE out, synchronous)"},
             "gpu_launches": K * (KERNELS_PER_STEP - (1 if fused or args.paged else 0) + (1 if args.rope else 0)),
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<3> + merge (kvmem_paged_attend_rope)" if args.rope and args.paged else
+            "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<4> + merge (kvmem_paged_attend_rope, in-block key layout)"
+                                                   if args.rope and args.paged and args.in_block else
+                                                   "attend_split_kernel<3> + merge (kvmem_paged_attend_rope)" if args.rope and args.paged else
                                                    "gather_rope_kernel (kvmem_materialize_rope)" if args.rope else
                                                    "attend_split_kernel<2> + merge (kvmem_paged_attend)" if args.paged else
                                                    "attend_split_kernel<1> + merge (kvmem_materialize_attend: view written while attended)"
@@ -511,7 +515,7 @@ def run_cache(args):
     base = CONFIGS[args.workload]
     if not base.attend or base.n_sessions != 1:
         raise SystemExit("--cache is measured on the single-session attend workloads")
-    pool, spec = fill_pool(base, device, rope=True)
+    pool, spec = fill_pool(base, device, rope=True, in_block=args.in_block)
     M, B, H, d = spec.n_q_tokens, spec.block_tokens, spec.n_q_heads, spec.head_dim
     prm = SelectParams(**select_params(spec))
     k = budget_blocks(prm, B, spec.n_blocks)
@@ -742,6 +746,9 @@ def main():
     ap.add_argument("--rope", action="store_true",
                     help="position-consistent view: keys de-rotated at append, query de-rotated for retrieval, RoPE at the "
                          "compact position fused into the gather (kvmem_materialize_rope), then kvmem_view_attend")
+    ap.add_argument("--in-block", action="store_true",
+                    help="with --rope: the pages hold RoPE(k, offset inside the block); the view rotates by the block's position "
+                         "alone and --paged rotates the query back once per block instead of every key")
     ap.add_argument("--paged", action="store_true",
                     help="copy-free execution view: kvmem_select + kvmem_paged_attend (no view is materialised; not the headline step)")
     ap.add_argument("--unfused", action="store_true", help="separate kvmem_materialize and kvmem_view_attend calls")
@@ -756,6 +763,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)
     args = ap.parse_args()
+    if args.in_block and not args.rope:
+        raise SystemExit("--in-block needs --rope")
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -64,6 +64,14 @@ typedef struct {
                                        token is encoded and re-encoded inside an execution view (8 bytes x
                                        head_dim / 2 per position)                                      */
     float rope_theta;               /* rotary base (e.g. 1e6); used when rope_max_positions > 0        */
+    int32_t rope_in_block_keys;     /* 0: the pages hold raw (position-free) keys.  1 (needs rotary support with
+                                       rope_max_positions >= block_tokens and 64-token blocks for the copy-free
+                                       attention): a page holds k' = RoPE(k, t), t the token's offset inside its
+                                       block, so that a block placed at compact position p0 needs the rotation
+                                       of p0 alone: the position-consistent view rotates by one angle set per
+                                       block, and the copy-free attention rotates the QUERY back by p0 once per
+                                       block instead of every key forward (q . R(p0 + t) k = (R(-p0) q) . R(t) k).
+                                       The Mean-K index is built from the raw keys either way              */
 } kvmem_pool_config_t;
 
 /* Selection budget (Eq. "active_budget", Eq. "active_capacity" in Sec. 3.1; selector in

@@ -38,6 +38,9 @@ bool config_valid(const kvmem_pool_config_t& c, const char** why) {
     if (c.rope_max_positions < 0) return bad("rope_max_positions must be non-negative");
     if (c.rope_max_positions > 0 && !(c.rope_theta > 1.0f)) return bad("rope_theta must exceed 1 when rotary support is on");
     if (c.rope_max_positions > 0 && c.head_dim % 16 != 0) return bad("rotary support needs head_dim to be a multiple of 16");
+    if (c.rope_in_block_keys != 0 && c.rope_in_block_keys != 1) return bad("rope_in_block_keys must be 0 or 1");
+    if (c.rope_in_block_keys && c.rope_max_positions < c.block_tokens)
+        return bad("rope_in_block_keys needs rotary support covering at least one block (rope_max_positions >= block_tokens)");
     return true;
 }
 

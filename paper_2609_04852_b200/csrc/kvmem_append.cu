@@ -15,7 +15,7 @@ append_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* __res
               __nv_bfloat16* __restrict__ pages, __nv_bfloat16* __restrict__ index_sess,
               const int32_t* __restrict__ table_sess, int32_t* __restrict__ status,
               int b_first, int L, int G, int B, int d, int max_blocks, int max_bps, size_t page_elems,
-              const int32_t* __restrict__ pos0_sess, const float2* __restrict__ rope, int rope_positions) {
+              const int32_t* __restrict__ pos0_sess, const float2* __restrict__ rope, int rope_positions, int in_block) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __nv_bfloat16* tile = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [B][d]
 
@@ -43,7 +43,7 @@ append_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* __res
         *reinterpret_cast<uint4*>(vdst + (size_t)t * d + j * 8) = vv;
     }
     __syncthreads();
-    if (rope) {
+    if (pos0_sess) {
         // the keys still carry RoPE of positions pos0 + t: rotate back by the same angles (Sec. 4.3), so
         // that the pages hold raw keys and the index is position-independent.  fp32 products and sums
         // without fused multiply-add, one rounding to bf16: the defined arithmetic of a rotated element.
@@ -62,17 +62,33 @@ append_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* __res
         }
         __syncthreads();
     }
-    for (int c = threadIdx.x; c < n_chunks; c += blockDim.x) {
-        const int t = c / chunks_per_row, j = c % chunks_per_row;
-        *reinterpret_cast<uint4*>(kdst + (size_t)t * d + j * 8) = *reinterpret_cast<const uint4*>(tile + (size_t)t * d + j * 8);
-    }
-
+    // the index entry comes from the raw keys (position-independent, Sec. 4.3), whatever the pages hold
     const float inv = 1.0f / (float)B;
     __nv_bfloat16* idx_row = index_sess + ((size_t)lg * max_bps + (size_t)(b_first + i)) * d;
     for (int c = threadIdx.x; c < d; c += blockDim.x) {
         float acc = 0.0f;
         for (int t = 0; t < B; ++t) acc = __fadd_rn(acc, __bfloat162float(tile[(size_t)t * d + c]));
         idx_row[c] = __float2bfloat16_rn(__fmul_rn(acc, inv));
+    }
+    if (in_block) {
+        // in-block layout: the page holds RoPE(k, t), t the offset inside the block, so that a later placement at
+        // compact position p0 is the rotation of p0 alone for the whole block.  Same defined arithmetic.
+        __syncthreads();
+        const int half = d / 2;
+        for (int e = threadIdx.x; e < B * half; e += blockDim.x) {
+            const int t = e / half, x = e % half;
+            const float2 cs = rope[(size_t)t * half + x];
+            const float a = __bfloat162float(tile[(size_t)t * d + x]), b = __bfloat162float(tile[(size_t)t * d + x + half]);
+            const float lo = __fsub_rn(__fmul_rn(a, cs.x), __fmul_rn(b, cs.y));
+            const float hi = __fadd_rn(__fmul_rn(b, cs.x), __fmul_rn(a, cs.y));
+            tile[(size_t)t * d + x] = __float2bfloat16_rn(lo);
+            tile[(size_t)t * d + x + half] = __float2bfloat16_rn(hi);
+        }
+        __syncthreads();
+    }
+    for (int c = threadIdx.x; c < n_chunks; c += blockDim.x) {
+        const int t = c / chunks_per_row, j = c % chunks_per_row;
+        *reinterpret_cast<uint4*>(kdst + (size_t)t * d + j * 8) = *reinterpret_cast<const uint4*>(tile + (size_t)t * d + j * 8);
     }
 }
 
@@ -91,7 +107,7 @@ cudaError_t launch_append(const kvmem_pool& p, int session, int b_first, int n_b
     append_kernel<<<grid, 256, smem, st>>>(k, v, p.pages, index, table, p.status_dev, b_first, g.L, g.G, g.B, g.d,
                                            g.max_blocks, g.max_bps, p.lay.page_elems,
                                            derope ? p.pos0_dev + (size_t)session * g.max_bps : nullptr,
-                                           derope ? p.rope_dev : nullptr, p.cfg.rope_max_positions);
+                                           p.rope_dev, p.cfg.rope_max_positions, p.cfg.rope_in_block_keys);
     return cudaGetLastError();
 }
 

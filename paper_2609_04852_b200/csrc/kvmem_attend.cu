@@ -42,6 +42,9 @@ constexpr int kMaxSplits = 64;
 constexpr int kRowsPad = 16;
 constexpr int kMergeStride = 136;               // floats per merged row in shared memory
 constexpr size_t kAttSmem = (size_t)kAttStages * kStageBytes + 1024;
+constexpr int kQrotBytes = kRowsPad * kD * 2;   // one rotated query tile: 16 rows x 256 B
+constexpr size_t kAttSmemQrot = kAttSmem + (size_t)kAttStages * kQrotBytes;
+constexpr int kQrotWarps = 2;                   // query-rotator warps; they take tiles alternately
 
 struct AttendArgs {
     const __nv_bfloat16* q;
@@ -61,6 +64,7 @@ struct AttendArgs {
     int block_tokens;            // tokens per selected block (view length = n_sel * block_tokens); 64 in the paged modes
     const float2* rope;          // [rope_positions][64] (cos, sin)
     int first_position;          // compact position of view token 0
+    int rope_positions;          // rows of the rotary table
 };
 
 AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, int sm_count) {
@@ -101,22 +105,28 @@ static int choose_splits(int heads, int max_tiles, int sms) {
 //         and each consumer warp rotates its key fragments in registers between ldmatrix and the MMAs, with
 //         the arithmetic of kvmem_rope_rotate (fp32 products and sums, no fused multiply-add, one rounding
 //         to bf16).  The result equals attention over kvmem_materialize_rope's view and no byte is written.
+// MODE 4: position-consistent keys over pages that hold k' = RoPE(k, t), t the offset inside the block: the logit
+//         q . R(p0 + t) k equals (R(-p0) q) . k', so two extra warps, taking tiles alternately, rotate the 16 query rows back by the tile's
+//         compact position p0 (one rotary row per tile instead of 64) into a small shared-memory ring, the
+//         consumers fetch their A fragments from it with ldmatrix, and the keys go to the MMAs as stored.
 // MODE 2: copy-free execution view (Sec. 5.3 "Copy-free execution-view assembly"): tiles are read from
 //         the pages through the block table and attended over; no contiguous view is written.
 template <int MODE>
-__global__ void __launch_bounds__(MODE == 3 ? (kAttRopeConsumers + 1) * 32 : kAttThreads + (MODE == 1 ? 32 : 0), 1)
+__global__ void __launch_bounds__(MODE == 3 ? (kAttRopeConsumers + 1) * 32 : kAttThreads + (MODE == 1 ? 32 : MODE == 4 ? 32 * kQrotWarps : 0), 1)
 attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_pages, AttendArgs a) {
     pdl_wait();        // everything earlier in the stream is complete and visible from here on
     constexpr bool FUSED = MODE == 1;      // a view-writer warp shares every stage with the consumers
     constexpr bool PAGED = MODE != 0;      // the producer reads pages through the block table
     constexpr bool ROPE = MODE == 3;       // the consumers re-encode their key fragments in registers before the MMAs
+    constexpr bool QROT = MODE == 4;       // a rotator warp re-encodes the query per tile instead
     extern __shared__ unsigned char smem_dyn[];
     // the rotary mode gives the room of two data stages to one buffer of rotary rows per consumer group
     constexpr int STAGES = ROPE ? kAttRopeStages : kAttStages;
     constexpr int CONSUMERS = ROPE ? kAttRopeConsumers : kAttConsumers;
     constexpr int GROUPS = ROPE ? kAttRopeGroups : kAttGroups;
     __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages], tab_full[kAttRopeGroups], tab_empty[kAttRopeGroups];
+    __shared__ uint64_t q_full[kAttStages];
     __shared__ float merge_m[kAttRopeConsumers][kRowsPad], merge_l[kAttRopeConsumers][kRowsPad];
 
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -143,6 +153,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             ptx::mbar_init(&empty_bar[i], CONSUMERS / GROUPS + (FUSED ? 1 : 0));
         }
         for (int i = 0; i < GROUPS; ++i) { ptx::mbar_init(&tab_full[i], 1); ptx::mbar_init(&tab_empty[i], CONSUMERS / GROUPS); }
+        for (int i = 0; i < kAttStages; ++i) ptx::mbar_init(&q_full[i], 1);
         ptx::fence_mbar_init();
     }
     __syncthreads();
@@ -258,11 +269,63 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             else atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
             ptx::bulk_wait<0>();                           // the view is complete before the kernel ends
         }
+    } else if (QROT && warp > CONSUMERS) {
+        // ---------------- query rotator: Q'(tile) = RoPE^-1(q, p0(tile)) for the 16 query rows ----------------
+        // Lane -> 16-byte chunk c = lane & 7 of the low half (dims 8c..8c+7, paired with 64+8c..) of rows
+        // (lane >> 3) + 4 i: the lane's 8 (cos, sin) pairs serve its four rows.  Q' is stored [16 rows][256 B] with
+        // the 16-byte chunk index XOR-ed with the row's low 3 bits, which keeps the consumers' ldmatrix conflict-free.
+        if (n_tiles > 0) {
+            const int c = lane & 7;
+            uint4 raw_lo[4], raw_hi[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = (lane >> 3) + 4 * i;
+                raw_lo[i] = raw_hi[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (row < a.rows) {
+                    const __nv_bfloat16* qr = a.q + ((((size_t)s * a.M + row / a.r) * a.L + l) * a.H + (size_t)g * a.r + row % a.r) * kD;
+                    raw_lo[i] = *reinterpret_cast<const uint4*>(qr + c * 8);
+                    raw_hi[i] = *reinterpret_cast<const uint4*>(qr + kD / 2 + c * 8);
+                }
+            }
+            unsigned char* qring = stages + (size_t)kAttStages * kStageBytes;
+            // the rotary row of a tile is fetched one of this warp's tiles ahead: an L2 round trip per tile would
+            // otherwise sit on the critical path of every tile
+            auto fetch_row = [&](int it, float4 (&t4)[4]) {
+                int p0 = a.first_position + (t0 + min(it, n_tiles - 1)) * kTile;
+                if (p0 < 0 || p0 >= a.rope_positions) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); p0 = 0; }
+                const float4* cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)p0 * (kD / 2) + c * 8);
+#pragma unroll
+                for (int w = 0; w < 4; ++w) t4[w] = __ldg(cs4 + w);
+            };
+            const int it_first = warp - CONSUMERS - 1;
+            float4 t4[4], t4_next[4];
+            fetch_row(it_first, t4_next);
+            for (int it = it_first; it < n_tiles; it += kQrotWarps) {
+                const int st = it % STAGES;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) t4[w] = t4_next[w];
+                fetch_row(it + kQrotWarps, t4_next);
+                bool ok = true;
+                if (it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
+                if (!__all_sync(0xffffffffu, ok)) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
+                unsigned char* qb = qring + (size_t)st * kQrotBytes;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = (lane >> 3) + 4 * i;
+                    uint4 lo_o, hi_o;
+                    rotate8_cs(raw_lo[i], raw_hi[i], t4, -1.0f, lo_o, hi_o);
+                    *reinterpret_cast<uint4*>(qb + row * 256 + ((c ^ (row & 7)) << 4)) = lo_o;
+                    *reinterpret_cast<uint4*>(qb + row * 256 + (((c + 8) ^ (row & 7)) << 4)) = hi_o;
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&q_full[st]);
+            }
+        }
     } else {
         // ---------------- consumers ----------------
         // Q fragments (A operand, m16k16 x 8 k-steps).  Row j = m * r + hr  ->  q[s][m][l][g*r + hr].
         uint32_t qf[8][4];
-        {
+        if (!QROT) {
             const int row_a = lane >> 2, row_b = row_a + 8;
             const __nv_bfloat16* qa = nullptr;
             const __nv_bfloat16* qb = nullptr;
@@ -288,6 +351,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             const int st = it % STAGES;
             bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / STAGES) & 1));
             if (ROPE) arrived = arrived && ptx::mbar_wait(&tab_full[grp], (uint32_t)((it / GROUPS) & 1));
+            if (QROT) arrived = arrived && ptx::mbar_wait(&q_full[st], (uint32_t)((it / STAGES) & 1));
             if (!__all_sync(0xffffffffu, arrived)) {          // warp-uniform decision
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
@@ -299,6 +363,9 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             }
             const uint32_t kbase = stage0 + (uint32_t)st * kStageBytes;
             const uint32_t vbase = kbase + 2 * kHalfBytes;
+            // QROT: this tile's rotated query; its A fragments are fetched two k-steps at a time, next to their use
+            const int qrow = mr + 8 * (mj & 1);
+            const uint32_t qaddr = stage0 + (uint32_t)kAttStages * kStageBytes + (uint32_t)st * kQrotBytes + (uint32_t)qrow * 256u;
 
             // S = Q K^T for this warp's 16 tokens: 2 n-tiles (8 tokens each) x 8 k-steps
             float sc[2][4];
@@ -310,6 +377,13 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     const int cg = kp * 4 + mj;             // 16-byte chunk along d (0..15)
                     const uint32_t half_off = (uint32_t)(cg >> 3) * kHalfBytes;
                     const int c = cg & 7;
+                    if (QROT) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int ks = 2 * kp + h;
+                            ptx::ldmatrix_x4(qaddr + (uint32_t)(((ks * 2 + (mj >> 1)) ^ (qrow & 7)) << 4), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+                        }
+                    }
 #pragma unroll
                     for (int nt = 0; nt < 2; ++nt) {
                         const int tok = wq * 16 + nt * 8 + mr;
@@ -551,6 +625,8 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
             e = cudaFuncSetAttribute(attend_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attend_split_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmemQrot);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -570,7 +646,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     if (alt) {
         a.tables = alt->tables; a.nblocks_dev = alt->nblocks_dev; a.max_bps = alt->table_stride; a.max_blocks = alt->n_pages;
     }
-    a.rope = p.rope_dev; a.first_position = rope_first_position; a.block_tokens = g.B;
+    a.rope = p.rope_dev; a.first_position = rope_first_position; a.block_tokens = g.B; a.rope_positions = p.cfg.rope_max_positions;
     // How far the producers run ahead.  Measured on this part: a long single-wave stream is fastest with about 14 MiB
     // in flight over all SMs when the kernel also writes the view (read/write turn-arounds in HBM grow with the number
     // of outstanding requests) and about 19 MiB when it only reads; more stages in flight than that cost 5-7 %.
@@ -585,7 +661,9 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         }
     }
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
-    if (paged_only && rope_first_position >= 0)
+    if (paged_only && rope_first_position >= 0 && p.cfg.rope_in_block_keys)
+        launch_pdl(attend_split_kernel<4>, dim3(grid), dim3(kAttThreads + 32 * kQrotWarps), kAttSmemQrot, st, map_k, map_v, map_pages, a);
+    else if (paged_only && rope_first_position >= 0)
         launch_pdl(attend_split_kernel<3>, dim3(grid), dim3((kAttRopeConsumers + 1) * 32), kAttSmem, st, map_k, map_v, map_pages, a);
     else if (paged_only)
         launch_pdl(attend_split_kernel<2>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);

@@ -52,7 +52,7 @@ struct GatherRopeArgs {
     __nv_bfloat16* view_v;
     const float2* rope;
     int32_t* status;
-    int session_first, sel_stride, max_bps, max_blocks, LG, B, d, cap_tokens, first_position, rope_positions;
+    int session_first, sel_stride, max_bps, max_blocks, LG, B, d, cap_tokens, first_position, rope_positions, in_block;
     size_t page_elems;
 };
 
@@ -93,7 +93,7 @@ gather_rope_kernel(GatherRopeArgs a) {
         } else {                                            // keys: rotate to the compact position
             for (int e = threadIdx.x; e < a.B * chunks; e += 256) {
                 const int t = e / chunks, c = e % chunks;
-                const int pos = a.first_position + j * a.B + t;
+                const int pos = a.first_position + j * a.B + (a.in_block ? 0 : t);      // in-block layout: t is already in the stored key
                 if (pos >= a.rope_positions) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); continue; }
                 const __nv_bfloat16* row = src + (size_t)t * a.d + c * 8;
                 const uint4 lo = __ldg(reinterpret_cast<const uint4*>(row)), hi = __ldg(reinterpret_cast<const uint4*>(row + half));
@@ -126,7 +126,7 @@ cudaError_t launch_gather_rope(const kvmem_pool& p, int session_first, int n_ses
     a.view_k = view_k; a.view_v = view_v; a.rope = p.rope_dev; a.status = p.status_dev;
     a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
     a.LG = g.L * g.G; a.B = g.B; a.d = g.d; a.cap_tokens = view_cap_tokens; a.first_position = first_position;
-    a.rope_positions = p.cfg.rope_max_positions; a.page_elems = p.lay.page_elems;
+    a.rope_positions = p.cfg.rope_max_positions; a.page_elems = p.lay.page_elems; a.in_block = p.cfg.rope_in_block_keys;
     const int ctas = std::max(1, p.sm_count * 8 / n_sessions);
     launch_pdl(gather_rope_kernel, dim3(dim3((unsigned)ctas, (unsigned)n_sessions)), dim3(256), 0, st, a);
     return cudaGetLastError();

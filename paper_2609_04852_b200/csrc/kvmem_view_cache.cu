@@ -177,7 +177,7 @@ struct CacheApplyArgs {
     const int32_t* sel_ids;
     const float2* rope;
     int32_t* status;
-    int cap, max_blocks, LG, B, d, first_position, rope_positions;
+    int cap, max_blocks, LG, B, d, first_position, rope_positions, in_block;
     size_t page_elems;
 };
 
@@ -225,10 +225,10 @@ view_cache_apply_kernel(CacheApplyArgs a) {
             const uint4* s4 = reinterpret_cast<const uint4*>(src);
             uint4* d4 = reinterpret_cast<uint4*>(dst);
             for (int v = threadIdx.x; v < tile_elems / 8; v += 256) d4[v] = __ldg(s4 + v);
-        } else {                                            // keys: raw K rotated to the compact position
+        } else {                                            // keys: stored K rotated to the compact position
             for (int e = threadIdx.x; e < a.B * chunks; e += 256) {
                 const int t = e / chunks, c = e % chunks;
-                const int pos = a.first_position + j * a.B + t;
+                const int pos = a.first_position + j * a.B + (a.in_block ? 0 : t);   // in-block layout: t is already in the stored key
                 if (pos >= a.rope_positions) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); continue; }
                 const __nv_bfloat16* row = src + (size_t)t * a.d + c * 8;
                 const uint4 lo = __ldg(reinterpret_cast<const uint4*>(row)), hi = __ldg(reinterpret_cast<const uint4*>(row + half));
@@ -266,7 +266,7 @@ cudaError_t launch_view_cache_update(const kvmem_pool& p, int session, const int
     CacheApplyArgs a{};
     a.c = c; a.pages = p.pages; a.table = p.tables + (size_t)session * g.max_bps; a.sel_ids = sel_ids; a.rope = p.rope_dev;
     a.status = p.status_dev; a.cap = cap; a.max_blocks = g.max_blocks; a.LG = g.L * g.G; a.B = g.B; a.d = g.d;
-    a.first_position = first_position; a.rope_positions = p.cfg.rope_max_positions; a.page_elems = p.lay.page_elems;
+    a.first_position = first_position; a.rope_positions = p.cfg.rope_max_positions; a.page_elems = p.lay.page_elems; a.in_block = p.cfg.rope_in_block_keys;
     launch_pdl(view_cache_apply_kernel, dim3(p.sm_count * 8), dim3(256), 0, st, a);
     return cudaGetLastError();
 }

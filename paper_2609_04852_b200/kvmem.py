@@ -29,7 +29,8 @@ class KvmemError(RuntimeError):
 class PoolConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "block_tokens",
                                           "max_sessions", "max_blocks", "max_blocks_per_session", "device",
-                                          "rope_max_positions")] + [("rope_theta", C.c_float)]
+                                          "rope_max_positions")] + [("rope_theta", C.c_float),
+                                                                   ("rope_in_block_keys", C.c_int32)]
 
 
 class SelectParams(C.Structure):
@@ -154,10 +155,10 @@ class Pool:
 
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, block_tokens: int,
                  max_sessions: int, max_blocks: int, max_blocks_per_session: int, device: int = 0,
-                 rope_max_positions: int = 0, rope_theta: float = 0.0):
+                 rope_max_positions: int = 0, rope_theta: float = 0.0, rope_in_block_keys: bool = False):
         self.lib = load_library()
         self.cfg = PoolConfig(n_layers, n_q_heads, n_kv_heads, head_dim, block_tokens, max_sessions, max_blocks,
-                              max_blocks_per_session, device, rope_max_positions, rope_theta)
+                              max_blocks_per_session, device, rope_max_positions, rope_theta, int(rope_in_block_keys))
         nbytes = self.lib.kvmem_pool_bytes(C.byref(self.cfg))
         if nbytes == 0:
             raise KvmemError(E_INVALID, self.lib.kvmem_last_error().decode())
