@@ -131,6 +131,8 @@ int32_t kvmem_session_blocks(const kvmem_pool_t* pool, int32_t session);
  *   k, v       DEVICE bf16 [n_blocks * block_tokens][n_layers][n_kv_heads][head_dim], 16-byte aligned;
  *              may be released once the stream has run the call
  *   phys_ids   HOST int32 [n_blocks] page ids to use, or NULL to take free pages in ascending order
+ * On a pool created with rope_in_block_keys, k holds raw keys, the index is built from them, and the
+ * page receives RoPE(k, t), t = the token's offset inside its block.
  * Errors: KVMEM_E_CAPACITY (session or pool full), KVMEM_E_STATE (page in use), KVMEM_E_INVALID. */
 int kvmem_append_blocks(kvmem_pool_t* pool, int32_t session, const void* k /*DEVICE*/, const void* v /*DEVICE*/,
                         int32_t n_blocks, const int32_t* phys_ids /*HOST*/, void* stream);
@@ -143,7 +145,8 @@ int kvmem_append_blocks(kvmem_pool_t* pool, int32_t session, const void* k /*DEV
 
 /* kvmem_append_blocks for keys that still carry RoPE: token t of new block i was encoded at position
  * block_pos0[i] + t (its position in the execution window it was computed in).  The encoding is removed,
- * the raw keys are stored in the pages and indexed; block_pos0 is kept in the block record.
+ * the raw keys are stored in the pages and indexed; block_pos0 is kept in the block record.  (With
+ * rope_in_block_keys the raw keys are indexed and the pages receive RoPE(raw, t), t the offset in the block.)
  *   block_pos0  HOST int32 [n_blocks]; every position must lie in [0, rope_max_positions) */
 int kvmem_append_blocks_rope(kvmem_pool_t* pool, int32_t session, const void* k_roped /*DEVICE*/, const void* v /*DEVICE*/,
                              int32_t n_blocks, const int32_t* phys_ids /*HOST*/, const int32_t* block_pos0 /*HOST*/,
@@ -157,7 +160,9 @@ int kvmem_rope_rotate(kvmem_pool_t* pool, const void* x /*DEVICE*/, void* y /*DE
                       const int32_t* positions /*DEVICE*/, int32_t inverse, void* stream);
 
 /* kvmem_materialize with position-consistent keys: the key of view token j*B + t is the raw key rotated
- * to compact position first_position + j*B + t; values are copied unchanged.
+ * to compact position first_position + j*B + t; values are copied unchanged.  With rope_in_block_keys the
+ * stored key already carries the rotation of t and is rotated by first_position + j*B: one set of angles per
+ * block (the result differs from the raw-key path by one extra bf16 rounding of the stored key).
  * first_position + budget * B must not exceed rope_max_positions (KVMEM_E_INVALID otherwise). */
 int kvmem_materialize_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids /*DEVICE*/,
                            int32_t sel_stride, const int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/,
@@ -275,6 +280,11 @@ int kvmem_paged_attend(kvmem_pool_t* pool, int32_t session_first, int32_t n_sess
  * kvmem_materialize_rope would build from the same ids; nothing is written besides out and lse.  The
  * pool's pages must hold raw keys and q must carry RoPE at its own position.  HBM traffic: one read per
  * view byte plus the rotary table rows of the view's positions.
+ * On a pool created with rope_in_block_keys (pages hold k' = RoPE(k, t)) no key is rotated: the logit
+ * q . R(p0 + t) k equals (R(-p0) q) . k', p0 = first_position + j*block_tokens, so the 16 query rows are rotated
+ * back by p0 once per block (arithmetic of kvmem_rope_rotate, inverse; the rotated query is a bf16 vector)
+ * and the stored keys feed the tensor cores as they are.  The result is the same mathematics as attention
+ * over kvmem_materialize_rope's view, one rounding of the query instead of one of each key apart.
  * Extra errors: KVMEM_E_STATE without a rotary table; KVMEM_E_INVALID if
  * [first_position, first_position + sel_stride*block_tokens) leaves the table. */
 int kvmem_paged_attend_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
