@@ -282,29 +282,45 @@ def run_native(args):
         sampler.start()
         time.sleep(0.25)
 
-    # ---- timed region: K steps, device-timed, inputs resident in HBM
+    # ---- timed region: K steps, device-timed, inputs resident in HBM.  No event is recorded between the calls of a
+    # step here: an event between two calls keeps the second kernel from launching programmatically behind the first
+    # (about 15 us per step at 1M).  The per-stage times come from a second pass of K steps below.
     K = args.steps
-    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    begins = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if flush is not None:
+        fb = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+        fe = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
     barrier()
     t_wall0 = time.time()
     e0.record(stream)
     for i in range(K):
         if flush is not None:
             flush.fill_(i & 255)
-        begins[i].record(stream)
-        step(i, marks[i])
+            fb[i].record(stream)
+        step(i)
+        if flush is not None:
+            fe[i].record(stream)
     e1.record(stream)
     barrier()
     t_wall1 = time.time()
     total_ms = e0.elapsed_time(e1)
+    if flush is not None:
+        total_ms = sum(fb[i].elapsed_time(fe[i]) for i in range(K))          # the flush writes are not part of a step
+    # ---- second pass of K steps with events after each call: stage times and the dominant kernel's launch duration
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    begins = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    barrier()
+    for i in range(K):
+        if flush is not None:
+            flush.fill_(i & 255)
+        begins[i].record(stream)
+        step(i, marks[i])
+    barrier()
+    t_wall1 = time.time()
     step_ms = [begins[i].elapsed_time(marks[i][2]) for i in range(K)]
     sel_ms = [begins[i].elapsed_time(marks[i][0]) for i in range(K)]
     gat_ms = [marks[i][0].elapsed_time(marks[i][1]) for i in range(K)]
     att_ms = [marks[i][1].elapsed_time(marks[i][2]) for i in range(K)]
-    if flush is not None:
-        total_ms = sum(step_ms)          # the flush writes are not part of a step
     sampler.window(t_wall0, t_wall1)
     assert pool.device_status() == 0, "device status word set during the timed region"
 
@@ -424,7 +440,9 @@ def run_native(args):
                          "frac_of_peak": step_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "nominal_peak_gbs": 8000.0},
             "stages_ms": {"select": med(sel_ms), "materialize": med(gat_ms), "attend": med(att_ms),
-                          "step_median": med(step_ms), "step_min": min(step_ms)},
+                          "step_median": med(step_ms), "step_min": min(step_ms),
+                          "note": "from a second pass of the same K steps with an event after each call; value and ms_per_step "
+                                  "come from the first pass, which records no event inside a step"},
         }
         if not spec.attend:
             # the chunked configuration is bounded by the tensor pipe: two passes of the 2*M*H*NB*d contraction.
@@ -639,6 +657,151 @@ def run_cache(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------- one session sharded by KV head
+
+def run_head_sharded(args):
+    """Strong scaling of ONE session over N GPUs: rank p holds the pages and index rows of KV heads
+    [p G/N, (p+1) G/N) and the query heads that map to them.  Step: score the own heads, all-reduce the NB fp32
+    block scores (NCCL; the only exchange), the same deterministic top-k on every rank, view assembly + attention
+    over the own heads.  At N = 1 it is the default step without the collective."""
+    import torch.distributed as dist
+    from paper_2609_04852_b200 import Pool, SelectParams, budget_blocks, set_option
+    from paper_2609_04852_b200.sharding import head_sharded_step, kv_heads_for_rank, max_over_ranks, query_heads_of
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world and world > 1:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    for opt in args.option:
+        name, _, value = opt.partition("=")
+        set_option(name, int(value))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    spec = CONFIGS[args.workload]
+    if not spec.attend or spec.n_sessions != 1:
+        raise SystemExit("--shard-heads is measured on the single-session attend workloads")
+    if args.blocks:
+        f = args.blocks / spec.n_blocks
+        spec = spec.with_(name=f"{spec.name}@{args.blocks}", n_blocks=args.blocks, n_planted=max(1, int(spec.n_planted * f)),
+                          budget_blocks=max(1, int(spec.budget_blocks * f)))
+    r = spec.n_q_heads // spec.n_kv_heads
+    g0, g1 = kv_heads_for_rank(spec.n_kv_heads, rank, world)
+    h0, h1 = query_heads_of((g0, g1), r)
+    G_loc, H_loc = g1 - g0, h1 - h0
+    M, B, d = spec.n_q_tokens, spec.block_tokens, spec.head_dim
+    pool = Pool(spec.n_layers, H_loc, G_loc, d, B, 1, spec.n_blocks, spec.n_blocks, device.index)
+    table = page_table(spec)[0]
+    for b0 in range(0, spec.n_blocks, 1024):          # every rank generates the same session and keeps its heads
+        b1 = min(spec.n_blocks, b0 + 1024)
+        K, V = kv_blocks(spec, 0, b0, b1, device)
+        pool.append_blocks(0, K[:, :, g0:g1].contiguous(), V[:, :, g0:g1].contiguous(), table[b0:b1].tolist())
+    torch.cuda.synchronize(device)
+    prm = SelectParams(**select_params(spec))
+    k = budget_blocks(prm, B, spec.n_blocks)
+    qsets = [make_queries(spec, i)[:, :, :, h0:h1].contiguous() for i in range(spec.n_query_sets)]
+    q_dev = [q.to(device) for q in qsets]
+    q_pin = [q.pin_memory() for q in qsets]
+    scores = torch.zeros(1, spec.n_blocks, dtype=torch.float32, device=device)
+    sel = torch.zeros(1, k, dtype=torch.int32, device=device)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=device)
+    view = pool.new_view(1, k * B)
+    out, lse = pool.new_outputs(1, M)
+    stream = torch.cuda.current_stream(device)
+
+    def step(i):
+        head_sharded_step(pool, q_dev[i % len(q_dev)], prm, scores, sel, n_sel, view, out, lse, world)
+
+    def barrier():
+        torch.cuda.synchronize(device)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    assert pool.device_status() == 0 and int(n_sel[0]) == k
+    if world > 1:       # every rank must hold the same selection: compare a checksum (bookkeeping, untimed)
+        chk = torch.stack([sel.sum(dtype=torch.int64), (sel.to(torch.int64) * torch.arange(1, k + 1, device=device)).sum()])
+        lo, hi = chk.clone(), chk.clone()
+        dist.all_reduce(lo, op=dist.ReduceOp.MIN)
+        dist.all_reduce(hi, op=dist.ReduceOp.MAX)
+        assert torch.equal(lo, hi), "ranks disagree on the selected ids"
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    K = args.steps
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.time()
+    e0.record(stream)
+    for i in range(K):
+        step(i)
+    e1.record(stream)
+    barrier()
+    t1 = time.time()
+    total_ms = e0.elapsed_time(e1)
+    # end to end: the own heads of the query from pinned host memory, the own heads of O and LSE back
+    out_pin, lse_pin = torch.empty(out.shape).pin_memory(), torch.empty(lse.shape).pin_memory()
+    q_stage = torch.empty_like(q_dev[0])
+    Ke = min(K, 200)
+    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ee0.record(stream)
+    for i in range(Ke):
+        q_stage.copy_(q_pin[i % len(q_pin)], non_blocking=True)
+        head_sharded_step(pool, q_stage, prm, scores, sel, n_sel, view, out, lse, world)
+        out_pin.copy_(out, non_blocking=True)
+        lse_pin.copy_(lse, non_blocking=True)
+        torch.cuda.synchronize(device)
+    ee1.record(stream)
+    barrier()
+    e2e_ms = ee0.elapsed_time(ee1)
+    if rank == 0 and t1 - t0 < 0.5:       # keep the load up long enough for the clock sampler (rank 0 alone: no collective)
+        t0 = time.time()
+        i = 0
+        while time.time() < t0 + 0.6:
+            pool.materialize_attend(q_dev[0], sel, n_sel, view, out, lse); i += 1
+            if i % 50 == 0:
+                torch.cuda.synchronize(device)
+        torch.cuda.synchronize(device)
+        t1 = time.time()
+    sampler.window(t0, t1)
+    assert pool.device_status() == 0
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], device=device)
+    if rank == 0:
+        clocks = sampler.stop()
+        peaks = measured_peaks()
+        rank_bytes = 2 * k * 2 * spec.n_layers * G_loc * B * d * 2 + spec.n_layers * G_loc * spec.n_blocks * d * 2
+        rows = M * spec.n_layers * H_loc
+        line = {
+            "metric": METRIC, "value": K / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded; shapes of the paper's agent workspaces)",
+            "config": {"workload": f"{spec.name}: 1 session x {spec.n_blocks} blocks of {B} tokens, {M} query token(s), "
+                                   f"{spec.n_q_heads}/{spec.n_kv_heads} heads, budget {k} blocks",
+                       "history_tokens": spec.tokens, "view_tokens": k * B, "query_sets": len(qsets),
+                       "l2": "no flush: every step streams far more than the 126 MB L2",
+                       "parallelism": f"one session sharded by KV head over {world} GPU(s): {G_loc} KV / {H_loc} query heads per rank, "
+                                      f"one all-reduce of {spec.n_blocks} fp32 block scores per step",
+                       "calls": "kvmem_score + all-reduce(R) + kvmem_topk + kvmem_materialize_attend"},
+            "e2e": {"value": Ke / (e2e_ms * 1e-3), "unit": UNIT, "steps": Ke, "h2d_bytes_per_step": rows * d * 2,
+                    "d2h_bytes_per_step": rows * d * 4 + rows * 4,
+                    "api": "pinned host query (own heads) in, host O and LSE (own heads) out, around the sharded step"},
+            "gpu_launches": K * 5, "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "whole step on one rank (index + view read + view write of its heads)",
+                         "achieved": rank_bytes / (total_ms / K * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": rank_bytes / (total_ms / K * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+                         "algorithmic_bytes_per_launch": rank_bytes, "avg_launch_ms": total_ms / K, "traffic": None},
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ----------------------------------------------------------------------------- oracle arm / CPU baseline
 
 def _bits(t):
@@ -751,6 +914,9 @@ def main():
                          "alone and --paged rotates the query back once per block instead of every key")
     ap.add_argument("--paged", action="store_true",
                     help="copy-free execution view: kvmem_select + kvmem_paged_attend (no view is materialised; not the headline step)")
+    ap.add_argument("--shard-heads", action="store_true",
+                    help="N GPUs share ONE session, each holding a slice of the KV heads; one all-reduce of the block scores "
+                         "per step (strong scaling; the default at N > 1 is one independent session replica per GPU)")
     ap.add_argument("--unfused", action="store_true", help="separate kvmem_materialize and kvmem_view_attend calls")
     ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
                     help="kernel-variant switch passed to kvmem_set_option (e.g. chunk_poly=0)")
@@ -772,6 +938,8 @@ def main():
             raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the native arm")
         if args.cache:
             run_cache(args)
+        elif args.shard_heads:
+            run_head_sharded(args)
         else:
             run_native(args)
 

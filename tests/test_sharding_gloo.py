@@ -70,3 +70,84 @@ def test_two_gloo_ranks_shard_sessions_and_take_the_max_time():
 
 def test_max_over_ranks_without_a_process_group_is_identity():
     assert max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
+
+
+# ---- sharding by KV head inside one session: one all-reduce of the block scores --------------------
+
+def test_head_partition_and_query_head_mapping():
+    from paper_2609_04852_b200.sharding import kv_heads_for_rank, query_heads_of
+    assert [kv_heads_for_rank(8, r, 4) for r in range(4)] == [(0, 2), (2, 4), (4, 6), (6, 8)]
+    assert query_heads_of((2, 4), 4) == (8, 16)
+    for bad in ((8, 3), (6, 4)):
+        try:
+            kv_heads_for_rank(bad[0], 0, bad[1])
+        except ValueError:
+            continue
+        raise AssertionError("uneven head split must be refused")
+
+
+def _head_worker(rank, world, port, ret):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        from kvmem_workloads import CONFIGS, kv_blocks, make_queries
+        from oracle import kvmem_oracle as orc
+        from paper_2609_04852_b200.sharding import combine_head_shard_scores, kv_heads_for_rank, query_heads_of
+        spec = CONFIGS["tiny"].with_(n_blocks=96, n_planted=6, budget_blocks=12, n_q_tokens=2)
+        r = spec.n_q_heads // spec.n_kv_heads
+        g0, g1 = kv_heads_for_rank(spec.n_kv_heads, rank, world)
+        h0, h1 = query_heads_of((g0, g1), r)
+        K, V = kv_blocks(spec, 0, 0, spec.n_blocks)
+        Kb = K.view(torch.int16).numpy().view(np.uint16)
+        Vb = V.view(torch.int16).numpy().view(np.uint16)
+        qb = make_queries(spec, 0)[0].contiguous().view(torch.int16).numpy().view(np.uint16)      # [M][L][H][d]
+        # this rank's shard: its KV heads of the keys, its query heads of the query
+        idx_local = orc.mean_k_index(np.ascontiguousarray(Kb[:, :, g0:g1]), spec.block_tokens)
+        q_local = np.ascontiguousarray(qb[:, :, h0:h1])
+        R_local, _ = orc.block_scores(q_local, idx_local, spec.n_blocks)
+        R = combine_head_shard_scores(torch.from_numpy(R_local.astype(np.float32)), world).numpy()
+        sel = orc.select(R, spec.block_tokens, spec.budget_blocks, spec.max_view_tokens)
+        # attention over the own heads only
+        table = np.arange(spec.n_blocks, dtype=np.int32)
+        repo = orc.Repository.empty(spec.n_blocks, spec.block_tokens, spec.n_layers, g1 - g0, spec.head_dim)
+        repo.place(np.ascontiguousarray(Kb[:, :, g0:g1]), np.ascontiguousarray(Vb[:, :, g0:g1]), table)
+        T = len(sel) * spec.block_tokens
+        vK, vV = orc.gather(repo, table, sel, T)
+        O_local, lse_local = orc.attend(q_local, vK, vV, T)
+        # the unsharded computation, for comparison (every rank can afford it at this size)
+        idx = orc.mean_k_index(Kb, spec.block_tokens)
+        R_full, _ = orc.block_scores(qb, idx, spec.n_blocks)
+        sel_full = orc.select(R_full, spec.block_tokens, spec.budget_blocks, spec.max_view_tokens)
+        full = orc.Repository.empty(spec.n_blocks, spec.block_tokens, spec.n_layers, spec.n_kv_heads, spec.head_dim)
+        full.place(Kb, Vb, table)
+        fK, fV = orc.gather(full, table, sel_full, T)
+        O_full, lse_full = orc.attend(qb, fK, fV, T)
+        gathered = [None] * world
+        dist.all_gather_object(gathered, (R.tobytes(), sel.tolist()))      # test bookkeeping only
+        ret[rank] = dict(
+            r_close=bool(np.allclose(R, R_full, rtol=1e-5, atol=1e-9)), sel_same=sel.tolist() == sel_full.tolist(),
+            out_same=bool(np.array_equal(O_local, O_full[:, :, h0:h1]) and np.array_equal(lse_local, lse_full[:, :, h0:h1])),
+            ranks_agree=all(g == gathered[0] for g in gathered), r_sum=float(R.sum()))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_kv_heads_with_one_all_reduce_of_the_scores():
+    world = 2
+    with mp.Manager() as mgr:
+        ret = mgr.dict()
+        mp.spawn(_head_worker, args=(world, _free_port(), ret), nprocs=world, join=True)
+        res = {k: dict(v) for k, v in ret.items()}
+    assert sorted(res) == [0, 1]
+    for r in res.values():
+        assert r["r_close"] and r["sel_same"] and r["out_same"] and r["ranks_agree"]
+        assert abs(r["r_sum"] - 2.0) < 1e-4                 # sum_b R_b = M query tokens
+
+
+def test_combining_scores_without_ranks_is_the_identity_and_an_injected_reduce_is_used():
+    from paper_2609_04852_b200.sharding import combine_head_shard_scores
+    x = torch.tensor([0.25, 0.75])
+    assert combine_head_shard_scores(x.clone(), 1).tolist() == [0.25, 0.75]
+    other = torch.tensor([0.5, 0.5])
+    y = combine_head_shard_scores(x.clone(), 2, all_reduce=lambda t: t.add_(other * 0.5))
+    assert y.tolist() == [0.375, 0.625]
