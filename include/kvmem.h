@@ -433,6 +433,8 @@ int kvmem_device_status(kvmem_pool_t* pool, int32_t* status /*HOST*/, void* stre
  * degree-4 polynomial on the FMA pipe instead of a special-function-unit instruction (default 4), 0 = none.
  * "topk_cluster" (sessions above 16,384 blocks): 1 = selection by a thread-block cluster of 8 CTAs that merge
  * their histograms through distributed shared memory (default), 0 = by one CTA that re-reads the scores per pass.
+ * "topk_items" (sessions of at most 16,384 blocks): 0 = the selection kernel holds the fewest scores per thread
+ * (1, 2, 4, 8 or 16) that cover the session (default), n = at least n; never changes a result.
  * "attend_splits" (0 = chosen by the library, else forced split-K count), "attend_lookahead" (0 = chosen by the
  * library, else tiles the attention producers may run ahead), "gather_ctas" (0 = chosen by the library, else the
  * number of copy CTAs): the knobs of the bytes-in-flight sweeps; only "attend_splits" can move a result, by the

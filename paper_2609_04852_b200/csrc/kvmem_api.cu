@@ -582,6 +582,10 @@ int kvmem_set_option(const char* name, int32_t value) {
     if (strcmp(name, "gather_mode") == 0 && (value == 0 || value == 1)) { g_gather_mode = value; return KVMEM_OK; }
     if (strcmp(name, "chunk_poly") == 0 && (value == 0 || (value >= 2 && value <= 5))) { g_chunk_poly = value; return KVMEM_OK; }
     if (strcmp(name, "topk_cluster") == 0 && (value == 0 || value == 1)) { g_topk_cluster = value; return KVMEM_OK; }
+    if (strcmp(name, "topk_items") == 0 && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) {
+        g_topk_items = value;
+        return KVMEM_OK;
+    }
     if (strcmp(name, "gather_ctas") == 0 && value >= 0) { g_gather_ctas = value; return KVMEM_OK; }
     if (strcmp(name, "attend_lookahead") == 0 && value >= 0 && value <= 8) { g_attend_lookahead = value; return KVMEM_OK; }
     if (strcmp(name, "attend_splits") == 0 && value >= 0 && value <= 64) { g_attend_splits = value; return KVMEM_OK; }

@@ -57,12 +57,15 @@ __device__ __forceinline__ unsigned block_exclusive_scan(unsigned val, TopkShare
     return warp_off + inc - val;
 }
 
-// REG = true (sessions of at most 16,384 blocks): the scores are staged once through shared memory with
-// coalesced loads and then live in registers, 16 consecutive ids per thread, for every later pass.
+// REG = true (sessions of at most 1,024 * ITEMS blocks): the scores are loaded once and then live in registers,
+// ITEMS consecutive ids per thread, for every later pass (ITEMS = 16: staged through shared memory so that the
+// global loads stay coalesced; fewer: each thread loads its own 4 to 32 contiguous bytes).  The kernel is bound by
+// instruction issue and barrier latency on its one SM, so a short session takes the instantiation with the
+// fewest items per thread that covers it.
 // REG = false: any length; every pass re-reads the scores from global memory.
 constexpr int kStagePitch = kItems + 4;                     // floats per thread in the staging buffer: conflict-free 128-bit reads
 
-template <bool REG>
+template <bool REG, int ITEMS>
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* __restrict__ nblocks_dev,
             int session_first, int B, kvmem_select_params_t prm, int32_t* __restrict__ sel_ids, int sel_stride,
@@ -75,8 +78,31 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
     const int NB = nblocks_dev[session_first + s];
     const unsigned int* bits = reinterpret_cast<const unsigned int*>(scores + (size_t)s * scores_stride);
     int32_t* out = sel_ids + (size_t)s * sel_stride;
+    constexpr int kItems = ITEMS, kTopkTile = kTopkThreads * ITEMS;      // shadow the file-scope values of the 16-item layout
     unsigned int vreg[kItems];
-    if (REG) {
+    if constexpr (REG && ITEMS < 16) {
+        if (ITEMS % 4 == 0 && (reinterpret_cast<uintptr_t>(bits) & 15u) == 0) {
+#pragma unroll
+            for (int j = 0; j < ITEMS / 4; ++j) {
+                const int g4 = tid * (ITEMS / 4) + j;                      // ids 4*g4 .. 4*g4 + 3
+                uint4 u = make_uint4(0u, 0u, 0u, 0u);
+                if (4 * g4 + 3 < NB) {
+                    u = *reinterpret_cast<const uint4*>(bits + 4 * g4);
+                } else if (4 * g4 < NB) {
+                    u.x = bits[4 * g4];
+                    if (4 * g4 + 1 < NB) u.y = bits[4 * g4 + 1];
+                    if (4 * g4 + 2 < NB) u.z = bits[4 * g4 + 2];
+                }
+                vreg[(4 * j) % ITEMS] = u.x; vreg[(4 * j + 1) % ITEMS] = u.y; vreg[(4 * j + 2) % ITEMS] = u.z; vreg[(4 * j + 3) % ITEMS] = u.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < ITEMS; ++i) {
+                const int idx = tid * ITEMS + i;
+                vreg[i] = idx < NB ? bits[idx] : 0u;
+            }
+        }
+    } else if constexpr (REG) {
         if ((reinterpret_cast<uintptr_t>(bits) & 15u) == 0) {
             // coalesced 128-bit global reads, all of a thread's loads in flight before the first use
             uint4 u[kItems / 4];
@@ -626,6 +652,7 @@ topk_cluster_kernel(const float* __restrict__ scores, int scores_stride, const i
     cluster.sync();                                          // nobody leaves while its shared memory may still be read
 }
 
+int g_topk_items = 0;     // 0: fewest items per thread that cover the session; 2..16: at least this many (kernel-variant switch)
 int g_topk_cluster = 1;   // sessions above 16,384 blocks: 1 = cluster of 8 CTAs, 0 = one CTA re-reading the scores
 
 cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, const float* scores,
@@ -637,8 +664,8 @@ cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, 
     static_assert(kTopkThreads * kStagePitch >= kTopkTile, "the staging buffer doubles as the output buffer of one sweep");
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(topk_kernel<true, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_kernel<false, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -666,12 +693,19 @@ cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, 
         return cudaLaunchKernelEx(&cfg, topk_cluster_kernel, scores, scores_stride, (const int32_t*)p.nblocks_dev, session_first,
                                   p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev);
     }
-    if (max_nb <= kTopkTile)
-        launch_pdl(topk_kernel<true>, dim3(n_sessions), dim3(kTopkThreads), smem, st, scores, scores_stride, p.nblocks_dev, session_first,
-                                                                  p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev);
-    else
-        launch_pdl(topk_kernel<false>, dim3(n_sessions), dim3(kTopkThreads), smem, st, scores, scores_stride, p.nblocks_dev, session_first,
-                                                                   p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev);
+#define KVMEM_TOPK_LAUNCH(REG, ITEMS, BYTES)                                                                            \
+    launch_pdl(topk_kernel<REG, ITEMS>, dim3(n_sessions), dim3(kTopkThreads), (size_t)(BYTES), st, scores, scores_stride, \
+               p.nblocks_dev, session_first, p.geo.B, prm, sel_ids, sel_stride, n_sel, p.status_dev)
+    // the shortest instantiation that holds the longest session in registers; its dynamic shared memory is the
+    // output buffer of one sweep (1,024 * ITEMS ids)
+    const int items = g_topk_items > 0 ? g_topk_items : 1;
+    if (max_nb <= kTopkThreads * 1 && items <= 1) KVMEM_TOPK_LAUNCH(true, 1, kTopkThreads * 1 * 4);
+    else if (max_nb <= kTopkThreads * 2 && items <= 2) KVMEM_TOPK_LAUNCH(true, 2, kTopkThreads * 2 * 4);
+    else if (max_nb <= kTopkThreads * 4 && items <= 4) KVMEM_TOPK_LAUNCH(true, 4, kTopkThreads * 4 * 4);
+    else if (max_nb <= kTopkThreads * 8 && items <= 8) KVMEM_TOPK_LAUNCH(true, 8, kTopkThreads * 8 * 4);
+    else if (max_nb <= kTopkTile) KVMEM_TOPK_LAUNCH(true, 16, smem);
+    else KVMEM_TOPK_LAUNCH(false, 16, smem);
+#undef KVMEM_TOPK_LAUNCH
     return cudaGetLastError();
 }
 

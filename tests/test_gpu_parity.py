@@ -269,6 +269,45 @@ def test_selection_from_given_scores_in_long_sessions(n_scores, budget, sink, re
             set_option("topk_cluster", 1)
 
 
+@pytest.mark.parametrize("n_scores,budget,sink,recent,kind", [
+    (1, 1, 0, 0, "normal"), (257, 32, 0, 0, "normal"), (1024, 100, 1, 2, "ties"), (1025, 1000, 0, 0, "normal"),
+    (2048, 512, 0, 0, "normal"), (2049, 7, 3, 0, "ties"), (4096, 4095, 0, 0, "normal"), (5000, 1234, 2, 9, "ties"),
+    (8192, 800, 0, 0, "constant"), (8193, 4096, 0, 0, "normal"), (16384, 4096, 0, 0, "normal"), (16384, 5000, 5, 5, "ties")])
+def test_selection_from_given_scores_in_short_sessions(n_scores, budget, sink, recent, kind):
+    """kvmem_topk up to 16,384 blocks: the register kernel's instantiations (1, 2, 4, 8 and 16 scores per thread;
+    the session picks the smallest that covers it, the switch forces larger ones) against the oracle's selector,
+    bit for bit, at the sizes where the instantiation changes."""
+    from paper_2609_04852_b200 import Pool, set_option
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(n_scores + budget)
+    if kind == "normal":
+        R = rng.random(n_scores).astype(np.float32) ** 8
+    elif kind == "ties":
+        R = rng.integers(0, 6, n_scores).astype(np.float32) / 8.0
+    else:
+        R = np.full(n_scores, 0.25, np.float32)
+    pool = Pool(1, 1, 1, 128, 16, 1, n_scores, n_scores, 0)
+    K = torch.zeros(n_scores * 16, 1, 1, 128, dtype=torch.bfloat16, device=dev)
+    pool.append_blocks(0, K, K)
+    ref = orc.select(R, 16, budget, 1 << 30, 0, sink, recent)
+    # an unaligned score pointer takes the scalar loads
+    for items, offset in ((0, 0), (16, 0), (4, 0), (0, 1), (8, 3)):
+        buf = torch.zeros(n_scores + 8, dtype=torch.float32, device=dev)
+        scores = buf[offset: offset + n_scores].view(1, -1)
+        scores.copy_(torch.from_numpy(R).view(1, -1))
+        set_option("topk_items", items)
+        try:
+            sel = torch.full((1, budget), -1, dtype=torch.int32, device=dev)
+            n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+            pool.topk(scores, _params(budget_blocks=budget, n_sink_blocks=sink, n_recent_blocks=recent), sel, n_sel)
+            torch.cuda.synchronize()
+            assert pool.device_status() == 0
+            got = sel.cpu().numpy()[0, : int(n_sel[0])]
+            assert np.array_equal(got, ref), f"items {items}, offset {offset}: {len(got)} ids, oracle {len(ref)}"
+        finally:
+            set_option("topk_items", 0)
+
+
 # ------------------------------------------------------------------ working-set delta
 
 def test_working_set_delta_between_two_steps():
@@ -399,7 +438,8 @@ def test_score_alone_equals_the_scores_select_reports_and_the_oracle(M, n_blocks
 # ------------------------------------------------------------------ kernel-variant switches
 
 @pytest.mark.parametrize("name,value,bit_exact", [("pdl", 0, True), ("attend_lookahead", 2, True), ("gather_ctas", 148, True),
-                                                  ("attend_splits", 5, False), ("attend_splits", 37, False)])
+                                                  ("attend_splits", 5, False), ("attend_splits", 37, False), ("topk_items", 16, True),
+                                                  ("topk_items", 2, True)])
 def test_kernel_variant_switches_do_not_change_results(name, value, bit_exact):
     # scheduling knobs (launch attributes, tiles in flight, CTA counts) leave every byte alone; a different split count
     # changes only the order of the split-K merge
