@@ -23,7 +23,7 @@ namespace kvmem {
 
 constexpr int kChunk = 128;       // blocks per CTA tile
 constexpr int kScoreThreads = 256;
-constexpr int kScoreStages = 4;   // 32 KiB index tiles in flight per CTA
+constexpr int kScoreStages = 3;   // 32 KiB index tiles in flight per CTA (two CTAs of the tensor-core kernel share an SM)
 constexpr int kMaxScoreParts = 64;
 
 ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, char* base) {
@@ -225,7 +225,7 @@ score_logits_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 // tile's 128 Mean-K vectors.  Index tiles arrive by tiled TMA with the 128-byte swizzle, so the
 // ldmatrix reads are conflict-free.  This removes the fp32-ALU bound of the shuffle kernel (16 rows
 // x 128 dims = 2,048 FMAs per 256-byte vector) and leaves the kernel bound by the index stream.
-__global__ void __launch_bounds__(kScoreThreads, 1)
+__global__ void __launch_bounds__(kScoreThreads, 2)
 score_logits_mma_kernel(const __grid_constant__ CUtensorMap map_idx, const __nv_bfloat16* __restrict__ q,
                         const int32_t* __restrict__ nblocks_dev, int session_first, int M, int L, int H, int G,
                         int max_bps, float* __restrict__ logits, float2* __restrict__ partials, int rows, int rows_pad,
@@ -489,7 +489,12 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     const int LG = g.L * g.G;
     const int chunks = (max_nb + kChunk - 1) / kChunk;
     // persistent CTAs: about one per SM, each streaming a contiguous range of chunks of one (session, l, g)
-    const int n_parts = std::max(1, std::min({chunks, kMaxScoreParts, p.sm_count / std::max(1, LG * n_sessions)}));
+    // Two CTAs of the tensor-core kernel fit on an SM.  The second one is used only while the row statistics stay
+    // short (many sessions or heads: at most 4 partials per row); a long single session is fastest with one CTA per
+    // SM and half as many partials to merge (measured at 1M: 18 parts 38.6 us, 36 parts 41.7 us for the select stage).
+    const int heads = std::max(1, LG * n_sessions);
+    const int fit1 = p.sm_count / heads, fit2 = g_score_mode == 1 ? 2 * p.sm_count / heads : fit1;
+    const int n_parts = std::max(1, std::min({chunks, kMaxScoreParts, fit2 <= 4 ? fit2 : fit1}));
     const size_t smem = (size_t)kScoreStages * kChunk * 256;
     dim3 grid((unsigned)n_parts, (unsigned)LG, (unsigned)n_sessions);
     cudaError_t e;
