@@ -417,7 +417,7 @@ def run_native(args):
             "e2e": {"value": whole_job_rate(Ke, world, e2e_ms), "unit": UNIT, "steps": Ke,
                     "h2d_bytes_per_step": rows * spec.head_dim * 2,
                     "d2h_bytes_per_step": rows * spec.head_dim * 4 + rows * 4,
-                    "api": "kvmem_recall_step_host (pinned host query in, host O and LSE out, synchronous)"},
+                    "api": "kvmem_recall_step_host (pinned host query copied in, O and LSE written into the pinned host buffers by the step's last kernel, synchronous)"},
             "gpu_launches": K * (KERNELS_PER_STEP - (1 if fused or args.paged else 0) + (1 if args.rope else 0)),
             "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<4> + merge (kvmem_paged_attend_rope, in-block key layout)"

@@ -398,6 +398,8 @@ int kvmem_view_attend_static(kvmem_pool_t* pool, int32_t n_sessions, const void*
  * stream (synchronous).  Same definitions and limits as the individual calls.
  *   q_host     HOST bf16 [n_sessions][n_q_tokens][L][H][d]   (pinned memory makes the copies asynchronous)
  *   out_host   HOST fp32 [n_sessions][n_q_tokens][L][H][d];  lse_host HOST fp32 [n_sessions][n_q_tokens][L][H]
+ *              (when both are pinned, device-mapped memory the last kernel of the step writes them directly
+ *              and no copy is issued; otherwise they are copied from the staging buffer)
  *   staging    DEVICE, kvmem_step_staging_bytes(), 256-byte aligned: device copies of q, out, lse
  * sel_ids, n_sel, views and workspaces are DEVICE buffers as in the individual calls and hold the
  * step's selection and view afterwards. */

@@ -542,6 +542,14 @@ size_t kvmem_step_staging_bytes(const kvmem_pool_config_t* cfg, int32_t n_sessio
     return a + b + c;
 }
 
+// the device-side address of a host buffer that the GPU can write directly (pinned and mapped), else null
+static float* mapped_host_pointer(float* host) {
+    cudaPointerAttributes at{};
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    if (at.type != cudaMemoryTypeHost || !at.devicePointer) return nullptr;
+    return static_cast<float*>(at.devicePointer);
+}
+
 int kvmem_recall_step_host(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q_host,
                            int32_t n_q_tokens, const kvmem_select_params_t* prm, int32_t* sel_ids, int32_t sel_stride,
                            int32_t* n_sel, void* view_k, void* view_v, int32_t view_cap_tokens, float scale,
@@ -567,11 +575,20 @@ int kvmem_recall_step_host(kvmem_pool_t* p, int32_t session_first, int32_t n_ses
     int rc = kvmem_select(p, session_first, n_sessions, q_dev, n_q_tokens, prm, sel_ids, sel_stride, n_sel, nullptr,
                           select_ws, select_ws_bytes, stream);
     if (rc != KVMEM_OK) return rc;
+    // Result buffers in pinned, device-mapped host memory are written by the merge kernel itself (the stores cross
+    // PCIe as they are issued and are complete when the stream is): two copy operations less on the critical path
+    // of a synchronous step.  Anything else (pageable memory) takes the staged copies.
+    float* out_map = mapped_host_pointer(out_host);
+    float* lse_map = mapped_host_pointer(lse_host);
+    const bool direct = out_map && lse_map && aligned(out_map, 16);
     rc = kvmem_materialize_attend(p, session_first, n_sessions, q_dev, n_q_tokens, sel_ids, sel_stride, n_sel, view_k, view_v,
-                                  view_cap_tokens, scale, out_dev, lse_dev, attend_ws, attend_ws_bytes, stream);
+                                  view_cap_tokens, scale, direct ? out_map : out_dev, direct ? lse_map : lse_dev, attend_ws,
+                                  attend_ws_bytes, stream);
     if (rc != KVMEM_OK) return rc;
-    e = cudaMemcpyAsync(out_host, out_dev, rows * p->cfg.head_dim * 4, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(lse_host, lse_dev, rows * 4, cudaMemcpyDeviceToHost, st);
+    if (!direct) {
+        e = cudaMemcpyAsync(out_host, out_dev, rows * p->cfg.head_dim * 4, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(lse_host, lse_dev, rows * 4, cudaMemcpyDeviceToHost, st);
+    }
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail("result download", e);
     return KVMEM_OK;

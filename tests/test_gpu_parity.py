@@ -619,3 +619,41 @@ def test_argument_and_capacity_errors():
     assert pool.session_blocks(0) == 0
     pool.append_blocks(0, K, V)
     assert pool.session_blocks(0) == 4 and pool.device_status() == 0
+
+
+# ------------------------------------------------------------------ the whole step with host buffers
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_recall_step_with_host_buffers_equals_the_device_calls(pinned):
+    """kvmem_recall_step_host: query from host memory, O and LSE into host memory.  Pinned result buffers are written by
+    the step's last kernel directly, pageable ones through the staging copies; both must give the bytes of
+    kvmem_select + kvmem_materialize_attend on device buffers, and match the oracle."""
+    spec = SMALL.with_(n_blocks=300, n_planted=12, budget_blocks=12, n_q_tokens=4)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    dev = torch.device("cuda", 0)
+    q, qb = queries(spec)
+    prm = _params(budget_blocks=12)
+    sel = torch.zeros(1, 12, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    view = pool.new_view(1, 12 * 64)
+    out, lse = pool.new_outputs(1, 4)
+    pool.select(q.to(dev), prm, sel, n_sel)
+    pool.materialize_attend(q.to(dev), sel, n_sel, view, out, lse)
+    torch.cuda.synchronize()
+    q_host = q.clone().pin_memory() if pinned else q.clone()
+    out_host = torch.full(out.shape, float("nan"), dtype=torch.float32)
+    lse_host = torch.full(lse.shape, float("nan"), dtype=torch.float32)
+    if pinned:
+        out_host, lse_host = out_host.pin_memory(), lse_host.pin_memory()
+    sel2 = torch.zeros_like(sel)
+    n_sel2 = torch.zeros_like(n_sel)
+    view2 = pool.new_view(1, 12 * 64)
+    for _ in range(2):                                          # the second call reuses the staging buffer
+        pool.recall_step_host(q_host, prm, sel2, n_sel2, view2, out_host, lse_host)      # synchronous
+    assert pool.device_status() == 0
+    assert torch.equal(sel2, sel) and torch.equal(view2.k, view.k) and torch.equal(view2.v, view.v)
+    assert torch.equal(out_host, out.cpu()) and torch.equal(lse_host, lse.cpu())
+    ref = _oracle_step(spec, osess, qb, 0, 12)
+    assert np.array_equal(sel2.cpu().numpy()[0], ref["sel"])     # budget = planted blocks: a resolvable gap
+    assert np.abs(out_host.numpy()[0] - ref["out"]).max() <= ATTN_ATOL and np.abs(lse_host.numpy()[0] - ref["lse"]).max() <= ATTN_ATOL
