@@ -230,6 +230,12 @@ def run_native(args):
                     ev[1].record(stream)
                     ev[2].record(stream)
                 return
+            if args.in_block:  # one pass: K tiles rotated by their block position in shared memory, stored and attended over
+                pool.materialize_attend_rope(q, sel, n_sel, view, out, lse, 0)
+                if ev is not None:
+                    ev[1].record(stream)
+                    ev[2].record(stream)
+                return
             pool.materialize_rope(sel, n_sel, view, 0)
             if ev is not None:
                 ev[1].record(stream)
@@ -339,8 +345,7 @@ def run_native(args):
             if args.paged:
                 pool.paged_attend_rope(q_stage, sel, n_sel, out, lse, 0)
             else:
-                pool.materialize_rope(sel, n_sel, view, 0)
-                pool.view_attend(q_stage, view, n_sel, out, lse)
+                pool.materialize_attend_rope(q_stage, sel, n_sel, view, out, lse, 0)
             out_pin.copy_(out, non_blocking=True)
             lse_pin.copy_(lse, non_blocking=True)
             torch.cuda.synchronize(device)
@@ -390,7 +395,8 @@ def run_native(args):
         dom_bytes = ns * (ab["attend"] if args.paged else ab["gather"])    # paged: one read of the selected pages
         gather_gbs = dom_bytes / gather_s / 1e9
         # fused: every view byte is read once (from the pages) and written once; separate calls read it a second time
-        step_bytes = ns * (ab["total"] - (ab["attend"] if fused else 0))
+        one_pass = fused or (args.rope and args.in_block and not args.paged)       # view written while attended
+        step_bytes = ns * (ab["total"] - (ab["attend"] if one_pass else 0))
         if args.paged:
             step_bytes = ns * (ab["index"] + ab["attend"])
         step_gbs = world * K * step_bytes / (total_ms * 1e-3) / 1e9 / world      # per GPU
@@ -410,6 +416,8 @@ def run_native(args):
                                 "the query rotated back once per block)" if args.rope and args.paged and args.in_block else
                                 "kvmem_rope_rotate(q) + kvmem_select + kvmem_paged_attend_rope (copy-free, keys RoPE'd in shared memory)"
                                 if args.rope and args.paged else
+                                "kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_attend_rope (one pass: K tiles rotated by their block "
+                                "position in shared memory, stored and attended over)" if args.rope and args.in_block else
                                 "kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_rope + kvmem_view_attend" if args.rope else
                                 "kvmem_select + kvmem_paged_attend (NO materialize: copy-free view variant)" if args.paged else
                                 "kvmem_select + kvmem_materialize_attend" if fused else
@@ -418,11 +426,13 @@ def run_native(args):
                     "h2d_bytes_per_step": rows * spec.head_dim * 2,
                     "d2h_bytes_per_step": rows * spec.head_dim * 4 + rows * 4,
                     "api": "kvmem_recall_step_host (pinned host query copied in, O and LSE written into the pinned host buffers by the step's last kernel, synchronous)"},
-            "gpu_launches": K * (KERNELS_PER_STEP - (1 if fused or args.paged else 0) + (1 if args.rope else 0)),
+            "gpu_launches": K * (KERNELS_PER_STEP - (1 if one_pass or args.paged else 0) + (1 if args.rope else 0)),
             "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "attend_split_kernel<4> + merge (kvmem_paged_attend_rope, in-block key layout)"
                                                    if args.rope and args.paged and args.in_block else
                                                    "attend_split_kernel<3> + merge (kvmem_paged_attend_rope)" if args.rope and args.paged else
+                                                   "attend_split_kernel<5> + merge (kvmem_materialize_attend_rope: K rotated in shared memory, "
+                                                   "view written while attended)" if args.rope and args.in_block else
                                                    "gather_rope_kernel (kvmem_materialize_rope)" if args.rope else
                                                    "attend_split_kernel<2> + merge (kvmem_paged_attend)" if args.paged else
                                                    "attend_split_kernel<1> + merge (kvmem_materialize_attend: view written while attended)"
@@ -434,7 +444,7 @@ def run_native(args):
                                     FUSED_TRAFFIC.get(base.name) if fused else GATHER_TRAFFIC.get(base.name)},
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes,
                          "accounting": "index + one read of the selected pages (copy-free view, nothing materialised)" if args.paged else
-                                       "index + view read + view write (fused pass)" if fused else
+                                       "index + view read + view write (fused pass)" if one_pass else
                                        "index + gather read/write + attend read (separate calls)",
                          "bytes_if_separate_calls": ns * ab["total"], "achieved_gbs": step_gbs,
                          "frac_of_peak": step_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",

@@ -292,6 +292,19 @@ int kvmem_paged_attend_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n
                             const int32_t* n_sel /*DEVICE*/, int32_t first_position, float scale, float* out /*DEVICE*/,
                             float* lse /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
+/* kvmem_materialize_rope followed by kvmem_view_attend in one call (Sec. 4.4: the execution view with keys
+ * encoded at their compact positions, then decode over it).  Same arguments as kvmem_materialize_attend plus
+ * first_position; the view left behind is kvmem_materialize_rope's, out/lse are kvmem_view_attend's on it with
+ * a q that carries RoPE at its own position.  On a pool with rope_in_block_keys this is ONE pass (each K tile is
+ * rotated by its block's compact position while it sits in shared memory, then stored and attended over: 1 read
+ * + 1 write per view byte); on a raw-key pool it runs the two kernels one after the other.
+ * Extra errors: KVMEM_E_STATE without a rotary table; KVMEM_E_INVALID if the compact positions leave it. */
+int kvmem_materialize_attend_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
+                                  int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
+                                  const int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/, void* view_v /*DEVICE*/,
+                                  int32_t view_cap_tokens, int32_t first_position, float scale, float* out /*DEVICE*/,
+                                  float* lse /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
 /* Working-set delta between two consecutive steps (Eq. "kvmem-working-set-delta", Sec. 4.4):
  *     retained R = W_next n W_prev,   incoming L = W_next \ W_prev,   outgoing E = W_prev \ W_next.
  * prev_ids / next_ids are the ascending id lists kvmem_select wrote at the two steps, a block's slot is
@@ -439,8 +452,9 @@ int kvmem_device_status(kvmem_pool_t* pool, int32_t* status /*HOST*/, void* stre
  * (1, 2, 4, 8 or 16) that cover the session (default), n = at least n; never changes a result.
  * "attend_splits" (0 = chosen by the library, else forced split-K count), "attend_lookahead" (0 = chosen by the
  * library, else tiles the attention producers may run ahead), "gather_ctas" (0 = chosen by the library, else the
- * number of copy CTAs): the knobs of the bytes-in-flight sweeps; only "attend_splits" can move a result, by the
- * rounding of a different split-K merge order.
+ * number of copy CTAs), "attend_landed" (-1 = chosen by the library, 1 / 0 = the lookahead counts tiles that have not
+ * landed in shared memory yet / that have not been consumed yet): the knobs of the bytes-in-flight sweeps; only
+ * "attend_splits" can move a result, by the rounding of a different split-K merge order.
  * "pdl": 1 = the kernels of a step are launched with programmatic stream serialization, so that the
  * launch latency of each overlaps the tail of the one before (default), 0 = plain launches. */
 int kvmem_set_option(const char* name /*HOST*/, int32_t value);

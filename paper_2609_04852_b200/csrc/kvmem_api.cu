@@ -605,6 +605,7 @@ int kvmem_set_option(const char* name, int32_t value) {
     }
     if (strcmp(name, "gather_ctas") == 0 && value >= 0) { g_gather_ctas = value; return KVMEM_OK; }
     if (strcmp(name, "attend_lookahead") == 0 && value >= 0 && value <= 8) { g_attend_lookahead = value; return KVMEM_OK; }
+    if (strcmp(name, "attend_landed") == 0 && (value >= -1 && value <= 1)) { g_attend_landed = value; return KVMEM_OK; }
     if (strcmp(name, "attend_splits") == 0 && value >= 0 && value <= 64) { g_attend_splits = value; return KVMEM_OK; }
     if (strcmp(name, "pdl") == 0 && (value == 0 || value == 1)) { g_pdl = value; return KVMEM_OK; }
     if (strcmp(name, "score_mode") == 0 && (value == 0 || value == 1)) { g_score_mode = value; return KVMEM_OK; }
@@ -612,10 +613,11 @@ int kvmem_set_option(const char* name, int32_t value) {
     return KVMEM_E_INVALID;
 }
 
-int kvmem_materialize_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
-                             const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v,
-                             int32_t view_cap_tokens, float scale, float* out, float* lse, void* workspace,
-                             size_t workspace_bytes, void* stream) {
+// rope_first_position < 0: plain views; otherwise the position-consistent fused pass (in-block key layout)
+static int materialize_attend_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                                   const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v,
+                                   int32_t view_cap_tokens, int32_t rope_first_position, float scale, float* out, float* lse,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
     if (!pool_ok(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q || !sel_ids || !n_sel || !view_k || !view_v || !out || !lse || !workspace || !aligned(q, 16) ||
@@ -642,9 +644,41 @@ int kvmem_materialize_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_s
     if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
     cudaError_t e = launch_attend(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, (const __nv_bfloat16*)view_k,
                                   (const __nv_bfloat16*)view_v, view_cap_tokens, n_sel, scale, out, lse, workspace,
-                                  (cudaStream_t)stream, sel_ids, sel_stride, session_first);
+                                  (cudaStream_t)stream, sel_ids, sel_stride, session_first, nullptr, rope_first_position);
     if (e != cudaSuccess) return cuda_fail("fused materialize+attend kernel launch", e);
     return KVMEM_OK;
+}
+
+int kvmem_materialize_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                             const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v,
+                             int32_t view_cap_tokens, float scale, float* out, float* lse, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    return materialize_attend_impl(p, session_first, n_sessions, q, n_q_tokens, sel_ids, sel_stride, n_sel, view_k, view_v,
+                                   view_cap_tokens, -1, scale, out, lse, workspace, workspace_bytes, stream);
+}
+
+int kvmem_materialize_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                                  const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v,
+                                  int32_t view_cap_tokens, int32_t first_position, float scale, float* out, float* lse,
+                                  void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
+    if (sel_stride < 1 || view_cap_tokens < 1) { set_error("sel_stride and view_cap_tokens must be positive"); return KVMEM_E_INVALID; }
+    const int64_t last = (int64_t)first_position + std::min<int64_t>((int64_t)sel_stride * p->cfg.block_tokens, view_cap_tokens);
+    if (first_position < 0 || last > p->cfg.rope_max_positions) {
+        set_error("compact positions [%d, %lld) outside the rotary table [0, %d)", first_position, (long long)last,
+                  p->cfg.rope_max_positions);
+        return KVMEM_E_INVALID;
+    }
+    if (p->cfg.rope_in_block_keys)      // one pass: every K tile is rotated by its block position on its way through shared memory
+        return materialize_attend_impl(p, session_first, n_sessions, q, n_q_tokens, sel_ids, sel_stride, n_sel, view_k, view_v,
+                                       view_cap_tokens, first_position, scale, out, lse, workspace, workspace_bytes, stream);
+    // raw keys need 64 sets of angles per tile: the rotating gather, then attention over the view
+    int rc = kvmem_materialize_rope(p, session_first, n_sessions, sel_ids, sel_stride, n_sel, view_k, view_v, view_cap_tokens,
+                                    first_position, stream);
+    if (rc != KVMEM_OK) return rc;
+    return kvmem_view_attend(p, n_sessions, q, n_q_tokens, view_k, view_v, view_cap_tokens, n_sel, scale, out, lse, workspace,
+                             workspace_bytes, stream);
 }
 
 static int paged_attend_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,

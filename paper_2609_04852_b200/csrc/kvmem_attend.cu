@@ -45,6 +45,7 @@ constexpr size_t kAttSmem = (size_t)kAttStages * kStageBytes + 1024;
 constexpr int kQrotBytes = kRowsPad * kD * 2;   // one rotated query tile: 16 rows x 256 B
 constexpr size_t kAttSmemQrot = kAttSmem + (size_t)kAttStages * kQrotBytes;
 constexpr int kQrotWarps = 2;                   // query-rotator warps; they take tiles alternately
+constexpr int kKrotWarps = 2;                   // key-tile rotator warps of the position-consistent fused pass; alternate tiles
 
 struct AttendArgs {
     const __nv_bfloat16* q;
@@ -61,6 +62,7 @@ struct AttendArgs {
     int session_first, sel_stride, max_bps, max_blocks;
     // position-consistent copy-free view (attend_split_kernel<3>): raw keys are rotated in shared memory
     int lookahead;               // tiles the producer may run ahead of the consumers (0: as many as there are stages)
+    int landed;                  // 1: the lookahead counts tiles that have not landed yet instead of tiles not yet consumed
     int block_tokens;            // tokens per selected block (view length = n_sel * block_tokens); 64 in the paged modes
     const float2* rope;          // [rope_positions][64] (cos, sin)
     int first_position;          // compact position of view token 0
@@ -79,6 +81,7 @@ AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tok
     return p;
 }
 
+int g_attend_landed = -1;     // -1: chosen in launch_attend; 0 / 1: the lookahead counts tiles not yet consumed / not yet landed
 int g_attend_lookahead = 0;   // 0: chosen in launch_attend; > 0: forced number of tiles in flight per CTA
 int g_attend_splits = 0;   // 0: chosen by the cost model below; > 0: forced (kernel-variant switch)
 
@@ -109,14 +112,20 @@ static int choose_splits(int heads, int max_tiles, int sms) {
 //         q . R(p0 + t) k equals (R(-p0) q) . k', so two extra warps, taking tiles alternately, rotate the 16 query rows back by the tile's
 //         compact position p0 (one rotary row per tile instead of 64) into a small shared-memory ring, the
 //         consumers fetch their A fragments from it with ldmatrix, and the keys go to the MMAs as stored.
+// MODE 5: MODE 1 for pages that hold k' = RoPE(k, t) (offset inside the block), leaving a position-consistent view: two
+//         extra warps, taking tiles alternately, rotate every K tile in place in shared memory by its compact
+//         position p0 (one set of angles per tile, arithmetic of kvmem_rope_rotate) as soon as it has landed; the
+//         consumers and the view writer wait for the rotated tile.  The view equals kvmem_materialize_rope's and
+//         out/lse equal kvmem_view_attend's on it, with 1 read + 1 write per view byte.
 // MODE 2: copy-free execution view (Sec. 5.3 "Copy-free execution-view assembly"): tiles are read from
 //         the pages through the block table and attended over; no contiguous view is written.
 template <int MODE>
-__global__ void __launch_bounds__(MODE == 3 ? (kAttRopeConsumers + 1) * 32 : kAttThreads + (MODE == 1 ? 32 : MODE == 4 ? 32 * kQrotWarps : 0), 1)
+__global__ void __launch_bounds__(MODE == 3 ? (kAttRopeConsumers + 1) * 32 : kAttThreads + (MODE == 1 ? 32 : MODE == 4 ? 32 * kQrotWarps : MODE == 5 ? 32 + 32 * kKrotWarps : 0), 1)
 attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_pages, AttendArgs a) {
     pdl_wait();        // everything earlier in the stream is complete and visible from here on
-    constexpr bool FUSED = MODE == 1;      // a view-writer warp shares every stage with the consumers
+    constexpr bool FUSED = MODE == 1 || MODE == 5;   // a view-writer warp shares every stage with the consumers
+    constexpr bool KROT = MODE == 5;       // rotator warps re-encode every K tile in place before anybody else reads it
     constexpr bool PAGED = MODE != 0;      // the producer reads pages through the block table
     constexpr bool ROPE = MODE == 3;       // the consumers re-encode their key fragments in registers before the MMAs
     constexpr bool QROT = MODE == 4;       // a rotator warp re-encodes the query per tile instead
@@ -126,7 +135,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     constexpr int CONSUMERS = ROPE ? kAttRopeConsumers : kAttConsumers;
     constexpr int GROUPS = ROPE ? kAttRopeGroups : kAttGroups;
     __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages], tab_full[kAttRopeGroups], tab_empty[kAttRopeGroups];
-    __shared__ uint64_t q_full[kAttStages];
+    __shared__ uint64_t q_full[kAttStages];     // MODE 4: rotated query of the stage's tile is in place; MODE 5: its K tile is rotated
     __shared__ float merge_m[kAttRopeConsumers][kRowsPad], merge_l[kAttRopeConsumers][kRowsPad];
 
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -174,7 +183,8 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     bool ok = true;
                     if (ahead < STAGES && it >= ahead) {          // at most `ahead` tiles in flight (see the paged producer)
                         const int jt = it - ahead;
-                        ok = ptx::mbar_wait(&empty_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1));
+                        ok = a.landed ? ptx::mbar_wait(&full_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1))
+                                      : ptx::mbar_wait(&empty_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1));
                     }
                     if (ok && it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
                     if (!ok) {
@@ -214,7 +224,10 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     // again, and found complete, when that stage is refilled)
                     if (ok && ahead < STAGES && it >= ahead) {
                         const int jt = it - ahead;
-                        ok = ptx::mbar_wait(&empty_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1));
+                        // KROT: a landed tile waits for its rotation in shared memory, which is no longer an HBM
+                        // request in flight; the limit applies to tiles that have not landed yet
+                        ok = (KROT || a.landed) ? ptx::mbar_wait(&full_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1))
+                                                : ptx::mbar_wait(&empty_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1));
                     }
                     if (ok && it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
                     if (ROPE && ok) {
@@ -251,6 +264,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             for (int it = 0; it < n_tiles; ++it) {
                 const int st = it % STAGES;
                 ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / STAGES) & 1));
+                if (KROT && ok) ok = ptx::mbar_wait(&q_full[st], (uint32_t)((it / STAGES) & 1));
                 if (!ok) break;
                 unsigned char* src = stages + (size_t)st * kStageBytes;
                 const int y = (t0 + it) * kTile;
@@ -268,6 +282,46 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             if (ok) ptx::mbar_arrive(&empty_bar[(n_tiles - 1) % STAGES]);
             else atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
             ptx::bulk_wait<0>();                           // the view is complete before the kernel ends
+        }
+    } else if (KROT && warp > CONSUMERS + 1) {
+        // ---------------- key rotators: K tile <- RoPE(K tile, p0(tile)), in place ----------------
+        // Lane -> 16-byte chunk c = lane & 7 of the low half (dims 8c..8c+7, paired with the same chunk of the high
+        // half) of tokens (lane >> 3) + 4 i: the lane's 8 (cos, sin) pairs serve its sixteen tokens.  A quarter-warp
+        // covers one 128-byte row of the swizzled tile: conflict-free 128-bit accesses.
+        if (n_tiles > 0) {
+            const int c = lane & 7;
+            auto fetch_row = [&](int it, float4 (&t4)[4]) {
+                int p0 = a.first_position + (t0 + min(it, n_tiles - 1)) * kTile;
+                if (p0 < 0 || p0 >= a.rope_positions) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); p0 = 0; }
+                const float4* cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)p0 * (kD / 2) + c * 8);
+#pragma unroll
+                for (int w = 0; w < 4; ++w) t4[w] = __ldg(cs4 + w);
+            };
+            const int it_first = warp - CONSUMERS - 2;
+            float4 t4[4], t4_next[4];
+            fetch_row(it_first, t4_next);
+            for (int it = it_first; it < n_tiles; it += kKrotWarps) {
+                const int st = it % STAGES;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) t4[w] = t4_next[w];
+                fetch_row(it + kKrotWarps, t4_next);
+                const bool ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / STAGES) & 1));
+                if (!__all_sync(0xffffffffu, ok)) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
+                unsigned char* klo = stages + (size_t)st * kStageBytes;
+#pragma unroll 4
+                for (int i = 0; i < kTile / 4; ++i) {
+                    const int tok = (lane >> 3) + 4 * i;
+                    unsigned char* plo = klo + tok * 128 + ((c ^ (tok & 7)) << 4);
+                    const uint4 lo = *reinterpret_cast<const uint4*>(plo), hi = *reinterpret_cast<const uint4*>(plo + kHalfBytes);
+                    uint4 lo_o, hi_o;
+                    rotate8_cs(lo, hi, t4, 1.0f, lo_o, hi_o);
+                    *reinterpret_cast<uint4*>(plo) = lo_o;
+                    *reinterpret_cast<uint4*>(plo + kHalfBytes) = hi_o;
+                }
+                ptx::fence_proxy_async_smem();      // the view writer's bulk stores read these bytes through the async proxy
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&q_full[st]);
+            }
         }
     } else if (QROT && warp > CONSUMERS) {
         // ---------------- query rotator: Q'(tile) = RoPE^-1(q, p0(tile)) for the 16 query rows ----------------
@@ -351,7 +405,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             const int st = it % STAGES;
             bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / STAGES) & 1));
             if (ROPE) arrived = arrived && ptx::mbar_wait(&tab_full[grp], (uint32_t)((it / GROUPS) & 1));
-            if (QROT) arrived = arrived && ptx::mbar_wait(&q_full[st], (uint32_t)((it / STAGES) & 1));
+            if (QROT || KROT) arrived = arrived && ptx::mbar_wait(&q_full[st], (uint32_t)((it / STAGES) & 1));
             if (!__all_sync(0xffffffffu, arrived)) {          // warp-uniform decision
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
@@ -627,6 +681,8 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
             e = cudaFuncSetAttribute(attend_split_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmemQrot);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attend_split_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -647,16 +703,20 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         a.tables = alt->tables; a.nblocks_dev = alt->nblocks_dev; a.max_bps = alt->table_stride; a.max_blocks = alt->n_pages;
     }
     a.rope = p.rope_dev; a.first_position = rope_first_position; a.block_tokens = g.B; a.rope_positions = p.cfg.rope_max_positions;
-    // How far the producers run ahead.  Measured on this part: a long single-wave stream is fastest with about 14 MiB
-    // in flight over all SMs when the kernel also writes the view (read/write turn-arounds in HBM grow with the number
-    // of outstanding requests) and about 19 MiB when it only reads; more stages in flight than that cost 5-7 %.
-    // Short streams and multi-wave grids keep every stage in flight.
+    // How far the producers run ahead.  Measured on this part: a long single-wave stream is fastest with a bounded number
+    // of bytes in flight over all SMs (more outstanding requests than the bandwidth-delay product only lengthen the queues
+    // in front of HBM and, where the kernel also writes, mix more reads and writes): about 19 MiB counted up to consumption
+    // when the kernel only reads, about 9.5 MiB counted up to arrival in shared memory when it also writes the view (a
+    // landed tile that waits for its consumers, its store or its rotation is no longer an HBM request: 338.8 us against
+    // 345.1 us with 14 MiB counted up to consumption).  Short streams and multi-wave grids keep every stage in flight.
     a.lookahead = g_attend_lookahead;
+    const bool writes_view = fused && !paged_only;
+    a.landed = g_attend_landed >= 0 ? g_attend_landed : (writes_view ? 1 : 0);
     if (a.lookahead == 0) {
         const long long ctas = (long long)a.n_splits * heads;
         const int tiles_per_cta = (view_cap_tokens / kTile + a.n_splits - 1) / a.n_splits;
         if (ctas <= p.sm_count && tiles_per_cta >= 64) {
-            const double target = (fused && !paged_only ? 14.0 : 19.0) * 1024.0 * 1024.0;
+            const double target = (writes_view ? (a.landed ? 9.5 : 14.0) : 19.0) * 1024.0 * 1024.0;
             a.lookahead = std::max(2, std::min(kAttStages, (int)(target / ((double)ctas * kStageBytes) + 0.5)));
         }
     }
@@ -667,6 +727,8 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         launch_pdl(attend_split_kernel<3>, dim3(grid), dim3((kAttRopeConsumers + 1) * 32), kAttSmem, st, map_k, map_v, map_pages, a);
     else if (paged_only)
         launch_pdl(attend_split_kernel<2>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);
+    else if (fused && rope_first_position >= 0)
+        launch_pdl(attend_split_kernel<5>, dim3(grid), dim3(kAttThreads + 32 + 32 * kKrotWarps), kAttSmem, st, map_k, map_v, map_pages, a);
     else if (fused)
         launch_pdl(attend_split_kernel<1>, dim3(grid), dim3(kAttThreads + 32), kAttSmem, st, map_k, map_v, map_pages, a);
     else

@@ -75,6 +75,7 @@ void set_error(const char* fmt, ...);
 extern int g_score_mode;    // 1: tensor-core decode scoring (default), 0: fp32 ALU + warp-shuffle kernel
 extern int g_chunk_poly;    // chunked scoring: every n-th exponential on the FMA pipe (0: all on the special-function unit)
 extern int g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
+extern int g_attend_landed;
 extern int g_topk_items;    // 0: the top-k kernel holds the fewest scores per thread that cover the session; 1..16: at least this many
 extern int g_topk_cluster;  // 1: sessions above 16,384 blocks are selected by a cluster of 8 CTAs (default), 0: by one CTA
 extern int g_gather_ctas;

@@ -439,7 +439,7 @@ def test_score_alone_equals_the_scores_select_reports_and_the_oracle(M, n_blocks
 
 @pytest.mark.parametrize("name,value,bit_exact", [("pdl", 0, True), ("attend_lookahead", 2, True), ("gather_ctas", 148, True),
                                                   ("attend_splits", 5, False), ("attend_splits", 37, False), ("topk_items", 16, True),
-                                                  ("topk_items", 2, True)])
+                                                  ("topk_items", 2, True), ("attend_landed", 0, True), ("attend_landed", 1, True)])
 def test_kernel_variant_switches_do_not_change_results(name, value, bit_exact):
     # scheduling knobs (launch attributes, tiles in flight, CTA counts) leave every byte alone; a different split count
     # changes only the order of the split-K merge
@@ -470,7 +470,7 @@ def test_kernel_variant_switches_do_not_change_results(name, value, bit_exact):
     try:
         got = run()
     finally:
-        set_option(name, 1 if name == "pdl" else 0)
+        set_option(name, 1 if name == "pdl" else -1 if name == "attend_landed" else 0)
     for i, (a, b) in enumerate(zip(base, got)):
         if bit_exact or i < 5:
             assert torch.equal(a, b), (name, i)

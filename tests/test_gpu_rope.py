@@ -106,6 +106,12 @@ def test_step_with_position_consistent_view(first_position):
     assert np.array_equal(bits(view.k[0]), vK), "rotated keys differ from the defined code"
     ref_out, ref_lse = orc.attend(qb[0], vK, vV, k * B)
     assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+    # one call for both steps (two kernels on a raw-key pool): the same bytes
+    view3 = pool.new_view(1, k * B)
+    out3, lse3 = pool.new_outputs(1, M)
+    pool.materialize_attend_rope(qd, sel, n_sel, view3, out3, lse3, first_position)
+    torch.cuda.synchronize()
+    assert torch.equal(view3.k, view.k) and torch.equal(view3.v, view.v) and torch.equal(out3, out) and torch.equal(lse3, lse)
     # the copy-free variant rotates the same raw tiles in shared memory: same keys bit for bit, same tile order
     out2, lse2 = pool.new_outputs(1, M)
     pool.paged_attend_rope(qd, sel, n_sel, out2, lse2, first_position)

@@ -107,6 +107,39 @@ def test_view_by_block_rotation_and_attention_with_the_query_rotated_back(n_bloc
     assert (out2 - out).abs().max().item() <= 3e-2 and (lse2 - lse).abs().max().item() <= 3e-2
 
 
+@pytest.mark.parametrize("n_blocks,budget,M,first", [(150, 20, 4, 517), (700, 60, 4, 17), (90, 1, 1, 0), (64, 64, 2, 0)])
+def test_fused_position_consistent_materialise_and_attend(n_blocks, budget, M, first):
+    # one pass: every K tile is rotated by its block position in shared memory, stored to the view and attended over
+    spec = SPEC.with_(n_blocks=n_blocks, budget_blocks=budget, n_q_tokens=M)
+    dev = torch.device("cuda", 0)
+    pool, repo, idx, tab, table = _fill_both(spec)
+    B = spec.block_tokens
+    ids = np.sort(np.random.default_rng(n_blocks + 1).choice(n_blocks, size=budget, replace=False)).astype(np.int32)
+    q, qb = queries(spec)
+    qd = q.to(dev)
+    sel = torch.from_numpy(ids).view(1, -1).to(dev)
+    n_sel = torch.tensor([budget], dtype=torch.int32, device=dev)
+    T = budget * B
+    view = pool.new_view(1, T)
+    out, lse = pool.new_outputs(1, M)
+    pool.materialize_attend_rope(qd, sel, n_sel, view, out, lse, first)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    vK, vV = orc.gather_rope(repo, table, ids, T, first, tab, in_block=True)
+    assert np.array_equal(bits(view.k[0]), vK), "fused pass: rotated keys differ from the defined code"
+    assert np.array_equal(bits(view.v[0]), vV)
+    ref_out, ref_lse = orc.attend(qb[0], vK, vV, T)
+    assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+    # the same bytes as the two separate calls
+    view2 = pool.new_view(1, T)
+    out2, lse2 = pool.new_outputs(1, M)
+    pool.materialize_rope(sel, n_sel, view2, first)
+    pool.view_attend(qd, view2, n_sel, out2, lse2)
+    torch.cuda.synchronize()
+    assert torch.equal(view2.k, view.k) and torch.equal(view2.v, view.v)
+    assert torch.equal(out2, out) and torch.equal(lse2, lse)
+
+
 def test_query_rotation_really_depends_on_the_compact_position():
     # the same selection at two different first positions must differ (a rotator that ignored p0 would pass the
     # tolerance test only by accident), and each must match its own oracle result
