@@ -60,7 +60,9 @@ def measured_tensor_peak():
 # profiles/dram_traffic_1m.md (1M workload)
 GATHER_TRAFFIC = {"1m": 2099369984}
 # the same for one launch of the fused pass (attend_split_kernel<1>)
-FUSED_TRAFFIC = {"1m": 2100752896}
+FUSED_TRAFFIC = {"1m": 2099557205}      # mean of six launches, profiles/launch_list_bench_1m.md
+# and of the position-consistent fused pass on the in-block key layout (attend_split_kernel<5>), profiles/bench_1m_position_consistent.md
+ROPE_FUSED_TRAFFIC = {"1m": 2098100000}
 # and of the rotating gather (gather_rope_kernel), profiles/dram_traffic_1m_rope_step.md
 ROPE_GATHER_TRAFFIC = {"1m": 2298386176}
 
@@ -440,7 +442,8 @@ def run_native(args):
                          "achieved": gather_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gather_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": gather_s * 1e3,
-                         "traffic": None if args.paged else ROPE_GATHER_TRAFFIC.get(base.name) if args.rope else
+                         "traffic": None if args.paged else ROPE_FUSED_TRAFFIC.get(base.name) if args.rope and args.in_block else
+                                    ROPE_GATHER_TRAFFIC.get(base.name) if args.rope else
                                     FUSED_TRAFFIC.get(base.name) if fused else GATHER_TRAFFIC.get(base.name)},
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes,
                          "accounting": "index + one read of the selected pages (copy-free view, nothing materialised)" if args.paged else
