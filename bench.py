@@ -140,12 +140,12 @@ def rope_window(spec):
     return spec.max_view_tokens + 64
 
 
-def fill_pool(spec, device, seed_shift=0, rope=False, in_block=False):
+def fill_pool(spec, device, seed_shift=0, rope=False, in_block=False, fp8_pages=False):
     from paper_2609_04852_b200 import Pool
     spec = spec.with_(seed=spec.seed + seed_shift)
     pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.block_tokens,
                 spec.n_sessions, spec.n_sessions * spec.n_blocks, spec.n_blocks, device.index,
-                rope_window(spec) if rope else 0, ROPE_THETA if rope else 0.0, rope_in_block_keys=in_block)
+                rope_window(spec) if rope else 0, ROPE_THETA if rope else 0.0, rope_in_block_keys=in_block, fp8_pages=fp8_pages)
     tables = page_table(spec)
     B = spec.block_tokens
     for s in range(spec.n_sessions):
@@ -188,7 +188,7 @@ def run_native(args):
         else:
             base = base.with_(name=f"{base.name}@{args.blocks}", n_blocks=args.blocks,
                               n_planted=max(1, int(base.n_planted * f)), budget_blocks=max(1, int(base.budget_blocks * f)))
-    pool, spec = fill_pool(base, device, seed_shift=1000 * rank, rope=args.rope, in_block=args.in_block)     # one independent replica per rank
+    pool, spec = fill_pool(base, device, seed_shift=1000 * rank, rope=args.rope, in_block=args.in_block, fp8_pages=args.fp8_pages)     # one independent replica per rank
     ns, M, B = spec.n_sessions, spec.n_q_tokens, spec.block_tokens
     prm = SelectParams(**select_params(spec))
     from paper_2609_04852_b200 import budget_blocks
@@ -248,7 +248,13 @@ def run_native(args):
         pool.select(q, prm, sel, n_sel)
         if ev is not None:
             ev[0].record(stream)
-        if args.fp8:           # FP8 (E4M3) view: quantise while gathering, attend over half the bytes
+        if args.fp8_pages and args.paged:       # FP8 repository, copy-free: attention straight over the 1-byte pages
+            pool.paged_attend_fp8(q, sel, n_sel, out, lse)
+            if ev is not None:
+                ev[1].record(stream)
+                ev[2].record(stream)
+            return
+        if args.fp8:           # FP8 (E4M3) view: quantise while gathering (or copy the tiles of an FP8 repository), attend over half the bytes
             pool.materialize_fp8(sel, n_sel, k8, v8t)
             if ev is not None:
                 ev[1].record(stream)
@@ -354,8 +360,11 @@ def run_native(args):
         elif args.fp8:
             q_stage.copy_(q_pin[i % len(q_pin)], non_blocking=True)
             pool.select(q_stage, prm, sel, n_sel)
-            pool.materialize_fp8(sel, n_sel, k8, v8t)
-            pool.view_attend_fp8(q_stage, k8, v8t, n_sel, out, lse)
+            if args.fp8_pages and args.paged:
+                pool.paged_attend_fp8(q_stage, sel, n_sel, out, lse)
+            else:
+                pool.materialize_fp8(sel, n_sel, k8, v8t)
+                pool.view_attend_fp8(q_stage, k8, v8t, n_sel, out, lse)
             out_pin.copy_(out, non_blocking=True)
             lse_pin.copy_(lse, non_blocking=True)
             torch.cuda.synchronize(device)
@@ -508,15 +517,27 @@ def run_native(args):
             g_s, a_s = med(gat_ms) * 1e-3, med(att_ms) * 1e-3
             line["config"]["calls"] = "kvmem_select + kvmem_materialize_fp8 + kvmem_view_attend_fp8 (E4M3 view, static scales 1.0)"
             line["dtype"] = "bf16 pages and query, E4M3 view, f16 tensor-core products, fp32 accumulation"
-            line["roofline"] = {"bound": "hbm", "kernel": "gather_fp8_kernel (kvmem_materialize_fp8)", "achieved": g_bytes / g_s / 1e9,
+            if args.fp8_pages:      # FP8 repository: the gather copies 1-byte tiles; --paged reads them in place
+                g_bytes = ns * ab["gather"] // 2
+                line["dtype"] = "E4M3 pages (quantised at append), bf16 query and index, f16 tensor-core products, fp32 accumulation"
+                line["config"]["calls"] = ("kvmem_select + kvmem_paged_attend_fp8 (copy-free view over an FP8 repository)" if args.paged else
+                                           "kvmem_select + kvmem_materialize_fp8 + kvmem_view_attend_fp8 over an FP8 repository")
+                if args.paged:
+                    g_bytes, a_bytes, a_s = a_bytes, 0, 1.0
+            line["roofline"] = {"bound": "hbm", "kernel": "attend_fp8_split_kernel<paged> + merge (kvmem_paged_attend_fp8)" if args.fp8_pages and args.paged else
+                                                           "gather_fp8_pages_kernel (kvmem_materialize_fp8)" if args.fp8_pages else
+                                                           "gather_fp8_kernel (kvmem_materialize_fp8)", "achieved": g_bytes / g_s / 1e9,
                                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": g_bytes / g_s / 1e9 / peaks["hbm_gbs"],
                                 "peak_source": f"of {peaks['source']}", "algorithmic_bytes_per_launch": g_bytes,
                                 "avg_launch_ms": g_s * 1e3, "traffic": None}
             line["attend_roofline"] = {"kernel": "attend_fp8_split_kernel + merge (kvmem_view_attend_fp8)", "achieved_gbs": a_bytes / a_s / 1e9,
                                        "frac": a_bytes / a_s / 1e9 / peaks["hbm_gbs"], "algorithmic_bytes_per_launch": a_bytes,
                                        "avg_ms": a_s * 1e3}
+            if args.fp8_pages and args.paged:
+                line.pop("attend_roofline")
             fp8_step = ns * ab["index"] + g_bytes + a_bytes
-            line["step_hbm"] = {"algorithmic_bytes_per_step": fp8_step, "accounting": "index + bf16 page read + FP8 view write + FP8 view read",
+            line["step_hbm"] = {"algorithmic_bytes_per_step": fp8_step, "accounting": "index + one read of the selected FP8 pages" if args.fp8_pages and args.paged else
+                                "index + FP8 page read + FP8 view write + FP8 view read" if args.fp8_pages else "index + bf16 page read + FP8 view write + FP8 view read",
                                 "achieved_gbs": K * fp8_step / (total_ms * 1e-3) / 1e9,
                                 "frac_of_peak": K * fp8_step / (total_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                 "peak_source": f"of {peaks['source']}", "nominal_peak_gbs": 8000.0}
@@ -937,11 +958,15 @@ def main():
                     "steps (working-set reuse, bounded delta re-RoPE); not the headline step")
     ap.add_argument("--drift", type=float, default=1.0, help="--cache: how far consecutive queries move (1 = independent)")
     ap.add_argument("--max-delta", type=int, default=4, help="--cache: delta re-RoPE operations between reconstructions")
+    ap.add_argument("--fp8-pages", action="store_true", help="FP8 repository: the pages hold E4M3 tiles quantised at append; with --paged "
+                    "the copy-free kvmem_paged_attend_fp8, else materialize_fp8 (a byte copy) + view_attend_fp8 (implies --fp8)")
     ap.add_argument("--fp8", action="store_true", help="FP8 (E4M3) execution view: materialize_fp8 + view_attend_fp8 (not the headline step)")
     ap.add_argument("--host-index", action="store_true", help="also time scoring against the index kept in pinned host memory")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)
     args = ap.parse_args()
+    if args.fp8_pages:
+        args.fp8 = True
     if args.in_block and not args.rope:
         raise SystemExit("--in-block needs --rope")
     if args.impl == "reference":

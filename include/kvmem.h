@@ -72,6 +72,16 @@ typedef struct {
                                        block, and the copy-free attention rotates the QUERY back by p0 once per
                                        block instead of every key forward (q . R(p0 + t) k = (R(-p0) q) . R(t) k).
                                        The Mean-K index is built from the raw keys either way              */
+    int32_t fp8_pages;              /* 0: pages hold bf16.  1 (head_dim 128, 64-token blocks, no rotary support): the
+                                       repository itself is FP8 (Sec. 6.1: the KV cache is kept in FP8): a page holds the
+                                       E4M3 codes of k / fp8_k_scale ([64 tokens][128] bytes per layer and KV head) and
+                                       of v / fp8_v_scale transposed ([128 dims][64 tokens] bytes), i.e. the tiles of the
+                                       FP8 execution view; half the memory and half the traffic of every pass over
+                                       pages.  kvmem_append_blocks still takes bf16 K and V and builds the bf16 Mean-K
+                                       index from them; kvmem_materialize_fp8 and kvmem_paged_attend_fp8 are the calls
+                                       that read such pages, the bf16 page readers return KVMEM_E_STATE            */
+    float fp8_k_scale;              /* static per-tensor scales of an FP8 repository (positive, finite)              */
+    float fp8_v_scale;
 } kvmem_pool_config_t;
 
 /* Selection budget (Eq. "active_budget", Eq. "active_capacity" in Sec. 3.1; selector in
@@ -344,6 +354,18 @@ int kvmem_view_attend_fp8(kvmem_pool_t* pool, int32_t n_sessions, const void* q 
                           const void* view_k8 /*DEVICE*/, const void* view_v8t /*DEVICE*/, int32_t view_cap_tokens,
                           const int32_t* n_sel /*DEVICE*/, float scale, float k_scale, float v_scale, float* out /*DEVICE*/,
                           float* lse /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
+/* On a pool created with fp8_pages: kvmem_materialize_fp8 copies the selected blocks' 8 KiB tiles as they are (1 byte
+ * read + 1 byte written per element; k_scale and v_scale must be the pool's, KVMEM_E_INVALID otherwise), and
+ * kvmem_paged_attend_fp8 is the copy-free execution view over such a repository (Sec. 5.3): attention straight
+ * over the selected pages through the block table, nothing written besides out and lse; results are those of
+ * kvmem_view_attend_fp8 on the view kvmem_materialize_fp8 would build, with the pool's scales (same tiles, same
+ * order, same arithmetic).  HBM traffic: one byte per element of the selected blocks.
+ * Arguments as kvmem_paged_attend.  KVMEM_E_STATE on a pool with bf16 pages. */
+int kvmem_paged_attend_fp8(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
+                           int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
+                           const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
+                           void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
 /* Execution cache: the execution view kept across steps, with working-set reuse and bounded delta
  * re-RoPE (Sec. 4.4: the two views; "Retrieval-Aware Hierarchical Reuse"; Eq. "kvmem-working-set-delta").

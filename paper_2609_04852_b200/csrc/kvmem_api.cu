@@ -41,6 +41,13 @@ bool config_valid(const kvmem_pool_config_t& c, const char** why) {
     if (c.rope_in_block_keys != 0 && c.rope_in_block_keys != 1) return bad("rope_in_block_keys must be 0 or 1");
     if (c.rope_in_block_keys && c.rope_max_positions < c.block_tokens)
         return bad("rope_in_block_keys needs rotary support covering at least one block (rope_max_positions >= block_tokens)");
+    if (c.fp8_pages != 0 && c.fp8_pages != 1) return bad("fp8_pages must be 0 or 1");
+    if (c.fp8_pages) {
+        if (c.head_dim != 128 || c.block_tokens != 64) return bad("an FP8 repository needs head_dim 128 and 64-token blocks");
+        if (c.rope_max_positions > 0) return bad("an FP8 repository cannot be combined with rotary support");
+        if (!(c.fp8_k_scale > 0.0f) || !(c.fp8_v_scale > 0.0f) || !std::isfinite(c.fp8_k_scale) || !std::isfinite(c.fp8_v_scale))
+            return bad("fp8_k_scale and fp8_v_scale must be positive and finite");
+    }
     return true;
 }
 
@@ -51,7 +58,7 @@ Layout make_layout(const kvmem_pool_config_t& c) {
     l.index_elems_per_session = (size_t)c.n_layers * c.n_kv_heads * c.max_blocks_per_session * c.head_dim;
     size_t off = 0;
     l.pages_off = off;
-    off = align_up(off + (size_t)c.max_blocks * l.page_elems * 2, 256);
+    off = align_up(off + (size_t)c.max_blocks * l.page_elems * (c.fp8_pages ? 1 : 2), 256);      // bf16 or E4M3 elements
     l.index_off = off;
     off = align_up(off + (size_t)c.max_sessions * l.index_elems_per_session * 2, 256);
     l.tables_off = off;
@@ -82,6 +89,13 @@ static bool sessions_ok(const kvmem_pool* p, int first, int n) {
         return false;
     }
     return true;
+}
+
+// the calls that read bf16 pages refuse an FP8 repository (and the other way round) instead of misreading it
+static bool pages_are(const kvmem_pool* p, bool fp8, const char* who) {
+    if ((p->cfg.fp8_pages != 0) == fp8) return true;
+    set_error("%s reads %s pages, the pool holds %s", who, fp8 ? "FP8" : "bf16", fp8 ? "bf16" : "FP8");
+    return false;
 }
 
 static int cuda_fail(const char* what, cudaError_t e) {
@@ -288,7 +302,8 @@ static int append_impl(kvmem_pool_t* p, int32_t session, const void* k, const vo
                             (size_t)n_blocks * 4, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) return cuda_fail("block position upload", e);
     }
-    e = launch_append(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st, block_pos0 != nullptr);
+    e = p->cfg.fp8_pages ? launch_append_fp8(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st)
+                         : launch_append(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st, block_pos0 != nullptr);
     if (e != cudaSuccess) return cuda_fail("append kernel launch", e);
     for (int32_t pg : ids) { p->page_used[pg] = 1; p->sess_pages[session].push_back(pg); }
     if (!phys_ids) p->free_hint = ids.back() + 1;
@@ -478,7 +493,7 @@ int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, con
 int kvmem_materialize(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids,
                       int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v, int32_t view_cap_tokens,
                       void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_ok(p) || !pages_are(p, false, "kvmem_materialize")) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!sel_ids || !n_sel || !view_k || !view_v || !aligned(view_k, 16) || !aligned(view_v, 16)) {
         set_error("kvmem_materialize: null or misaligned pointer");
@@ -618,7 +633,7 @@ static int materialize_attend_impl(kvmem_pool_t* p, int32_t session_first, int32
                                    const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v,
                                    int32_t view_cap_tokens, int32_t rope_first_position, float scale, float* out, float* lse,
                                    void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_ok(p) || !pages_are(p, false, "kvmem_materialize_attend")) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q || !sel_ids || !n_sel || !view_k || !view_v || !out || !lse || !workspace || !aligned(q, 16) ||
         !aligned(view_k, 128) || !aligned(view_v, 128) || !aligned(workspace, 256) || !aligned(out, 16)) {
@@ -684,7 +699,7 @@ int kvmem_materialize_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_
 static int paged_attend_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
                              const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, int32_t rope_first_position,
                              float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_ok(p) || !pages_are(p, false, "kvmem_paged_attend")) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q || !sel_ids || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(workspace, 256) || !aligned(out, 16)) {
         set_error("kvmem_paged_attend: null or misaligned pointer");
@@ -776,6 +791,11 @@ int kvmem_materialize_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_sess
         set_error("kvmem_materialize_fp8: null or misaligned pointer (views need 128-byte alignment), or sel_stride < 1");
         return KVMEM_E_INVALID;
     }
+    if (p->cfg.fp8_pages && (k_scale != p->cfg.fp8_k_scale || v_scale != p->cfg.fp8_v_scale)) {
+        set_error("kvmem_materialize_fp8: the pool's pages were quantised with scales %g / %g, not %g / %g", p->cfg.fp8_k_scale,
+                  p->cfg.fp8_v_scale, k_scale, v_scale);
+        return KVMEM_E_INVALID;
+    }
     cudaError_t e = launch_gather_fp8(*p, session_first, n_sessions, sel_ids, sel_stride, n_sel, (uint8_t*)view_k8,
                                       (uint8_t*)view_v8t, view_cap_tokens, k_scale, v_scale, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail("FP8 gather kernel launch", e);
@@ -805,6 +825,32 @@ int kvmem_view_attend_fp8(kvmem_pool_t* p, int32_t n_sessions, const void* q, in
                                       (const uint8_t*)view_v8t, view_cap_tokens, n_sel, scale, k_scale, v_scale, out, lse,
                                       workspace, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail("FP8 attention kernel launch", e);
+    return KVMEM_OK;
+}
+
+int kvmem_paged_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                           const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, float scale, float* out, float* lse,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p) || !pages_are(p, true, "kvmem_paged_attend_fp8")) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!q || !sel_ids || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(workspace, 256) || !aligned(out, 16)) {
+        set_error("kvmem_paged_attend_fp8: null or misaligned pointer");
+        return KVMEM_E_INVALID;
+    }
+    if (n_q_tokens < 1 || sel_stride < 1) { set_error("n_q_tokens and sel_stride must be positive"); return KVMEM_E_INVALID; }
+    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
+    if ((int64_t)p->cfg.max_blocks * 2 * p->cfg.n_layers * p->cfg.n_kv_heads * 64 > 0x7fffffffll) {
+        set_error("page pool too large for 32-bit TMA row coordinates");
+        return KVMEM_E_UNSUPPORTED;
+    }
+    if ((int64_t)sel_stride * 64 > 0x7fffffffll) { set_error("sel_stride too large"); return KVMEM_E_INVALID; }
+    AttendPlan plan = plan_attend(p->cfg, n_sessions, n_q_tokens, p->sm_count);
+    if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
+    cudaError_t e = launch_attend_fp8(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, nullptr, nullptr, sel_stride * 64, n_sel,
+                                      scale, p->cfg.fp8_k_scale, p->cfg.fp8_v_scale, out, lse, workspace, (cudaStream_t)stream,
+                                      sel_ids, sel_stride, session_first);
+    if (e != cudaSuccess) return cuda_fail("paged FP8 attention kernel launch", e);
     return KVMEM_OK;
 }
 

@@ -118,6 +118,113 @@ gather_fp8_kernel(GatherF8Args a) {
 }
 
 // ---------------------------------------------------------------------------------------------------
+// FP8 repository (pool created with fp8_pages): the pages hold the tiles of the FP8 view, so the append
+// quantises once (K straight, V transposed through shared memory, the same arithmetic as above), builds the
+// Mean-K entry from the bf16 keys it was given (Eq. "mean_k_index": fp32 sum in ascending token order, one
+// rounding to bf16), and every later pass moves one byte per element.
+__global__ void __launch_bounds__(256)
+append_fp8_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* __restrict__ v_in, uint8_t* __restrict__ pages8,
+                  __nv_bfloat16* __restrict__ index_sess, const int32_t* __restrict__ table_sess, int32_t* __restrict__ status,
+                  int b_first, int L, int G, int max_blocks, int max_bps, size_t page_bytes, float k_inv_scale, float v_inv_scale) {
+    __shared__ __align__(16) __nv_bfloat16 ktile[kF8Tile * kF8D];      // the bf16 keys, for the index entry
+    __shared__ __align__(16) uint8_t sv[kF8Tile * kF8Pitch];
+    const int i = blockIdx.x, lg = blockIdx.y, LG = L * G;
+    const int page = table_sess[b_first + i];
+    if (page < 0 || page >= max_blocks) {
+        if (threadIdx.x == 0) atomicExch(status, (int)KVMEM_E_DEVICE_RANGE);
+        return;
+    }
+    const size_t row_stride = (size_t)LG * kF8D;                       // elements between consecutive tokens of the input
+    const __nv_bfloat16* ksrc = k_in + (size_t)i * kF8Tile * row_stride + (size_t)lg * kF8D;
+    const __nv_bfloat16* vsrc = v_in + (size_t)i * kF8Tile * row_stride + (size_t)lg * kF8D;
+    uint8_t* kdst = pages8 + (size_t)page * page_bytes + (size_t)lg * (kF8Tile * kF8D);
+    uint8_t* vdst = kdst + (size_t)LG * (kF8Tile * kF8D);
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int e = threadIdx.x + 256 * it;                          // token e / 16, dims 8 * (e % 16) ..
+        const int t = e >> 4, j = e & 15;
+        const uint4 kk = *reinterpret_cast<const uint4*>(ksrc + (size_t)t * row_stride + j * 8);
+        const uint4 vv = *reinterpret_cast<const uint4*>(vsrc + (size_t)t * row_stride + j * 8);
+        *reinterpret_cast<uint4*>(ktile + (size_t)e * 8) = kk;
+        *reinterpret_cast<uint2*>(kdst + (size_t)e * 8) = quant8(kk, k_inv_scale);
+        const uint2 q = quant8(vv, v_inv_scale);
+        uint32_t* row = reinterpret_cast<uint32_t*>(sv + t * kF8Pitch + j * 8);
+        row[0] = q.x; row[1] = q.y;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {                                    // transposed store: 16 tokens of one dimension per piece
+        const int pce = threadIdx.x + 256 * it;
+        const int dim = pce >> 2, tg = pce & 3;
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            uint32_t x = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) x |= (uint32_t)sv[(tg * 16 + k * 4 + b) * kF8Pitch + dim] << (8 * b);
+            w[k] = x;
+        }
+        *reinterpret_cast<uint4*>(vdst + (size_t)dim * kF8Tile + tg * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    const float inv = 1.0f / (float)kF8Tile;
+    __nv_bfloat16* idx_row = index_sess + ((size_t)lg * max_bps + (size_t)(b_first + i)) * kF8D;
+    if (threadIdx.x < kF8D) {
+        const int c = threadIdx.x;
+        float acc = 0.0f;
+        for (int t = 0; t < kF8Tile; ++t) acc = __fadd_rn(acc, __bfloat162float(ktile[(size_t)t * kF8D + c]));
+        idx_row[c] = __float2bfloat16_rn(__fmul_rn(acc, inv));
+    }
+}
+
+cudaError_t launch_append_fp8(const kvmem_pool& p, int session, int b_first, int n_blocks, const __nv_bfloat16* k,
+                              const __nv_bfloat16* v, cudaStream_t st) {
+    const Geometry& g = p.geo;
+    const int32_t* table = p.tables + (size_t)session * g.max_bps;
+    __nv_bfloat16* index = p.index + (size_t)session * p.lay.index_elems_per_session;
+    dim3 grid((unsigned)n_blocks, (unsigned)(g.L * g.G));
+    append_fp8_kernel<<<grid, 256, 0, st>>>(k, v, reinterpret_cast<uint8_t*>(p.pages), index, table, p.status_dev, b_first, g.L, g.G,
+                                            g.max_blocks, g.max_bps, p.lay.page_elems, 1.0f / p.cfg.fp8_k_scale,
+                                            1.0f / p.cfg.fp8_v_scale);
+    return cudaGetLastError();
+}
+
+// materialize_fp8 over an FP8 repository: the tiles are copied as they are (one 8 KiB K tile and one 8 KiB V tile
+// per selected block, layer and KV head: 4 x 128-bit loads per thread in flight for each)
+__global__ void __launch_bounds__(256)
+gather_fp8_pages_kernel(GatherF8Args a) {
+    pdl_wait();
+    const int s = blockIdx.y;
+    const int NB = a.nblocks_dev[a.session_first + s];
+    int n_blk = a.n_sel[s];
+    const int cap_blocks = a.cap_tokens / kF8Tile;
+    if (n_blk > a.sel_stride || n_blk > cap_blocks) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE);
+        n_blk = min(min(n_blk, a.sel_stride), cap_blocks);
+    }
+    n_blk = max(n_blk, 0);
+    const long long n_items = (long long)n_blk * a.LG;
+    const int tile_bytes = kF8Tile * kF8D;
+    const uint8_t* pages8 = reinterpret_cast<const uint8_t*>(a.pages);
+    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int j = (int)(item / a.LG), lg = (int)(item % a.LG);
+        const int id = a.sel_ids[(size_t)s * a.sel_stride + j];
+        int page = -1;
+        if (id >= 0 && id < NB) page = a.tables[(size_t)(a.session_first + s) * a.max_bps + id];
+        if (page < 0 || page >= a.max_blocks) { if (threadIdx.x == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); continue; }
+        const uint4* ksrc = reinterpret_cast<const uint4*>(pages8 + (size_t)page * a.page_elems + (size_t)lg * tile_bytes);
+        const uint4* vsrc = reinterpret_cast<const uint4*>(pages8 + (size_t)page * a.page_elems + (size_t)(a.LG + lg) * tile_bytes);
+        const size_t head = (size_t)s * a.LG + lg;
+        uint4* kdst = reinterpret_cast<uint4*>(a.view_k + (head * a.cap_tokens + (size_t)j * kF8Tile) * kF8D);
+        uint4* vdst = reinterpret_cast<uint4*>(a.view_v + (head * cap_blocks + (size_t)j) * (size_t)tile_bytes);
+        uint4 kv[2], vv[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) { kv[i] = __ldg(ksrc + threadIdx.x + 256 * i); vv[i] = __ldg(vsrc + threadIdx.x + 256 * i); }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) { kdst[threadIdx.x + 256 * i] = kv[i]; vdst[threadIdx.x + 256 * i] = vv[i]; }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
 // Split-K decode attention over the FP8 view.  Same structure as the bf16 kernel (producer warp with
 // TMA, two groups of four consumer warps, one partial per split, merge kernel), with 16 KiB stages
 // (an 8 KiB K tile and an 8 KiB transposed V tile) and f16 tensor-core MMAs on converted fragments.
@@ -143,8 +250,15 @@ struct AttendF8Args {
     int M, L, H, G, r, rows, n_splits, cap_tokens;
     float scale_log2e;  // softmax scale * k_scale * log2(e)
     float v_scale;
+    // copy-free view over an FP8 repository (attend_fp8_split_kernel<true>): tiles come from the pages through the block table
+    const int32_t* sel_ids;      // [n_sessions][sel_stride]
+    const int32_t* tables;       // [max_sessions][max_bps]
+    const int32_t* nblocks_dev;  // [max_sessions]
+    int session_first, sel_stride, max_bps, max_blocks;
 };
 
+// PAGED: map_k covers the page pool ([pages * 2 * L*G * 64 rows][128 bytes]); map_v is unused.
+template <bool PAGED>
 __global__ void __launch_bounds__(kF8Threads, 1)
 attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, AttendF8Args a) {
     pdl_wait();
@@ -159,7 +273,7 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int z = s * LG + lg;
     const int l = lg / a.G, g = lg % a.G;
 
-    const int n_blk = max(0, min(a.n_sel[s], a.cap_tokens / kF8Tile));
+    const int n_blk = max(0, min(a.n_sel[s], PAGED ? a.sel_stride : a.cap_tokens / kF8Tile));
     const int t0 = (int)((long long)n_blk * split / a.n_splits);
     const int t1 = (int)((long long)n_blk * (split + 1) / a.n_splits);
     const int n_tiles = t1 - t0;
@@ -176,7 +290,40 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
 #pragma unroll
     for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f; }
 
-    if (warp == kF8Consumers) {
+    if (PAGED && warp == kF8Consumers) {
+        // ---------------- producer over pages: the whole warp looks pages up, 32 tiles at a time; lane 0 issues the loads
+        if (n_tiles > 0) {
+            if (lane == 0) ptx::prefetch_tensormap(&map_k);
+            const int NB = a.nblocks_dev[a.session_first + s];
+            auto lookup = [&](int it) -> int {
+                if (it >= n_tiles) return 0;
+                const int id = a.sel_ids[(size_t)s * a.sel_stride + t0 + it];
+                int pg = -1;
+                if (id >= 0 && id < NB) pg = a.tables[(size_t)(a.session_first + s) * a.max_bps + id];
+                if (pg < 0 || pg >= a.max_blocks) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); pg = 0; }
+                return pg;           // a flagged id reads page 0 instead of faulting; the status word reports it
+            };
+            int base_it = 0, my_page = lookup(lane);
+            bool ok = true;
+            for (int it = 0; it < n_tiles; ++it) {
+                if (it >= base_it + 32) { base_it = it; my_page = lookup(base_it + lane); }
+                const int page = __shfl_sync(0xffffffffu, my_page, it - base_it);
+                if (lane == 0) {
+                    const int st = it % kF8Stages;
+                    if (it >= kF8Stages) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kF8Stages) & 1) ^ 1));
+                    if (ok) {
+                        unsigned char* dst = stages + (size_t)st * kF8StageBytes;
+                        // page layout [K|V][L*G][64 rows][128 bytes]
+                        ptx::mbar_expect_tx(&full_bar[st], kF8StageBytes);
+                        ptx::tma_load_2d(dst, &map_k, 0, ((page * 2 + 0) * LG + lg) * kF8Tile, &full_bar[st]);
+                        ptx::tma_load_2d(dst + kF8TileBytes, &map_k, 0, ((page * 2 + 1) * LG + lg) * kF8Tile, &full_bar[st]);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
+            }
+        }
+    } else if (warp == kF8Consumers) {
         // ---------------- producer ----------------
         if (lane == 0 && n_tiles > 0) {
             ptx::prefetch_tensormap(&map_k);
@@ -389,7 +536,10 @@ cudaError_t launch_gather_fp8(const kvmem_pool& p, int session_first, int n_sess
     a.LG = g.L * g.G; a.cap_tokens = view_cap_tokens; a.k_inv_scale = 1.0f / k_scale; a.v_inv_scale = 1.0f / v_scale;
     a.page_elems = p.lay.page_elems;
     const int ctas = std::max(1, p.sm_count * 8 / n_sessions);
-    launch_pdl(gather_fp8_kernel, dim3((unsigned)ctas, (unsigned)n_sessions), dim3(256), 0, st, a);
+    if (p.cfg.fp8_pages)
+        launch_pdl(gather_fp8_pages_kernel, dim3((unsigned)ctas, (unsigned)n_sessions), dim3(256), 0, st, a);
+    else
+        launch_pdl(gather_fp8_kernel, dim3((unsigned)ctas, (unsigned)n_sessions), dim3(256), 0, st, a);
     return cudaGetLastError();
 }
 
@@ -407,15 +557,22 @@ static int f8_choose_splits(int heads, int max_tiles, int sms) {
 
 cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M, const uint8_t* view_k,
                               const uint8_t* view_v, int view_cap_tokens, const int32_t* n_sel, float scale, float k_scale,
-                              float v_scale, float* out, float* lse, void* workspace, cudaStream_t st) {
+                              float v_scale, float* out, float* lse, void* workspace, cudaStream_t st, const int32_t* sel_ids,
+                              int sel_stride, int session_first) {
     const Geometry& g = p.geo;
     const int LG = g.L * g.G, heads = n_sessions * LG;
+    const bool paged = sel_ids != nullptr;                  // copy-free: straight over the pages of an FP8 repository
     CUtensorMap map_k, map_v;
-    if (!make_f8_map(&map_k, view_k, (long long)heads * view_cap_tokens) || !make_f8_map(&map_v, view_v, (long long)heads * view_cap_tokens))
+    if (paged) {
+        if (!make_f8_map(&map_k, reinterpret_cast<const uint8_t*>(p.pages), (long long)g.max_blocks * 2 * LG * kF8Tile)) return cudaErrorInvalidValue;
+        map_v = map_k;
+    } else if (!make_f8_map(&map_k, view_k, (long long)heads * view_cap_tokens) || !make_f8_map(&map_v, view_v, (long long)heads * view_cap_tokens)) {
         return cudaErrorInvalidValue;
+    }
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attend_fp8_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
+        cudaError_t e = cudaFuncSetAttribute(attend_fp8_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -431,8 +588,13 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
     const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
     a.scale_log2e = sc * k_scale * 1.4426950408889634f;
     a.v_scale = v_scale;
+    a.sel_ids = sel_ids; a.tables = p.tables; a.nblocks_dev = p.nblocks_dev;
+    a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
-    launch_pdl(attend_fp8_split_kernel, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, a);
+    if (paged)
+        launch_pdl(attend_fp8_split_kernel<true>, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, a);
+    else
+        launch_pdl(attend_fp8_split_kernel<false>, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     launch_pdl(attend_merge_kernel, dim3((unsigned)a.rows, (unsigned)heads), dim3(kF8D), 0, st, a.part_o, a.part_ml, out, lse, M, g.L,

@@ -30,7 +30,8 @@ class PoolConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "block_tokens",
                                           "max_sessions", "max_blocks", "max_blocks_per_session", "device",
                                           "rope_max_positions")] + [("rope_theta", C.c_float),
-                                                                   ("rope_in_block_keys", C.c_int32)]
+                                                                   ("rope_in_block_keys", C.c_int32), ("fp8_pages", C.c_int32),
+                                                                   ("fp8_k_scale", C.c_float), ("fp8_v_scale", C.c_float)]
 
 
 class SelectParams(C.Structure):
@@ -92,6 +93,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_paged_attend_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_materialize_attend_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, i32, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_materialize_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, f32, f32, vp]),
+        "kvmem_paged_attend_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_fp8": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, f32, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
         "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
@@ -116,7 +118,7 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_working_set_delta", "kvmem_score", "kvmem_view_cache_bytes", "kvmem_view_cache_layout",
             "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend", "kvmem_paged_attend_rope", "kvmem_topk", "kvmem_score_host_workspace_bytes",
             "kvmem_score_host_staging_bytes", "kvmem_score_host_index", "kvmem_materialize_fp8", "kvmem_view_attend_fp8",
-            "kvmem_materialize_attend_rope")
+            "kvmem_materialize_attend_rope", "kvmem_paged_attend_fp8")
 
 
 def _check(status: int) -> None:
@@ -157,10 +159,12 @@ class Pool:
 
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, block_tokens: int,
                  max_sessions: int, max_blocks: int, max_blocks_per_session: int, device: int = 0,
-                 rope_max_positions: int = 0, rope_theta: float = 0.0, rope_in_block_keys: bool = False):
+                 rope_max_positions: int = 0, rope_theta: float = 0.0, rope_in_block_keys: bool = False,
+                 fp8_pages: bool = False, fp8_k_scale: float = 1.0, fp8_v_scale: float = 1.0):
         self.lib = load_library()
         self.cfg = PoolConfig(n_layers, n_q_heads, n_kv_heads, head_dim, block_tokens, max_sessions, max_blocks,
-                              max_blocks_per_session, device, rope_max_positions, rope_theta, int(rope_in_block_keys))
+                              max_blocks_per_session, device, rope_max_positions, rope_theta, int(rope_in_block_keys),
+                              int(fp8_pages), fp8_k_scale, fp8_v_scale)
         nbytes = self.lib.kvmem_pool_bytes(C.byref(self.cfg))
         if nbytes == 0:
             raise KvmemError(E_INVALID, self.lib.kvmem_last_error().decode())
@@ -412,6 +416,16 @@ class Pool:
                                               _dev(v8t, torch.uint8), k8.shape[3], _dev(n_sel, torch.int32), scale, k_scale,
                                               v_scale, _dev(out, torch.float32), _dev(lse, torch.float32), ws.data_ptr(),
                                               ws.numel(), _stream()))
+
+    def paged_attend_fp8(self, q: torch.Tensor, sel_ids: torch.Tensor, n_sel: torch.Tensor, out: torch.Tensor,
+                         lse: torch.Tensor, scale: float = 0.0, session_first: int = 0) -> None:
+        """Copy-free view over an FP8 repository (pool created with fp8_pages): attention straight over the pages."""
+        ns, M = q.shape[0], q.shape[1]
+        ws = self.attend_workspace(ns, M)
+        _check(self.lib.kvmem_paged_attend_fp8(self.handle, session_first, ns, _dev(q, torch.bfloat16), M,
+                                               _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
+                                               scale, _dev(out, torch.float32), _dev(lse, torch.float32),
+                                               ws.data_ptr(), ws.numel(), _stream()))
 
     def view_attend_static(self, q: torch.Tensor, view: View, n_sel: torch.Tensor, out: torch.Tensor,
                            lse: torch.Tensor, scale: float = 0.0) -> None:

@@ -91,3 +91,99 @@ def test_fp8_empty_view_and_argument_errors():
     with pytest.raises(KvmemError):
         pool.view_attend_fp8(q.to(dev), k8, v8t, n_sel, out, lse, v_scale=-1.0)
     assert pool.device_status() == 0
+
+
+# ---- FP8 repository: the pages themselves hold the E4M3 tiles ---------------------------------------
+
+def _fp8_pool(spec, k_scale, v_scale):
+    from kvmem_workloads import kv_blocks, page_table
+    from paper_2609_04852_b200 import Pool
+    dev = torch.device("cuda", 0)
+    pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.block_tokens, spec.n_sessions,
+                spec.n_sessions * spec.n_blocks, spec.n_blocks, 0, fp8_pages=True, fp8_k_scale=k_scale, fp8_v_scale=v_scale)
+    tables = page_table(spec)
+    for b0 in range(0, spec.n_blocks, 64):
+        b1 = min(spec.n_blocks, b0 + 64)
+        K, V = kv_blocks(spec, 0, b0, b1, dev)
+        pool.append_blocks(0, K, V, tables[0, b0:b1].tolist())
+    torch.cuda.synchronize()
+    return pool
+
+
+@pytest.mark.parametrize("n_blocks,k,M,k_scale,v_scale", [(150, 20, 4, 1.0, 1.0), (700, 333, 4, 0.5, 0.25), (90, 1, 1, 2.0, 1.0),
+                                                         (64, 64, 2, 1.0, 0.0625)])
+def test_fp8_repository_pages_view_and_copy_free_attention(n_blocks, k, M, k_scale, v_scale):
+    """Quantised once at append: the gathered view must hold the codes the oracle gets by quantising its bf16 gather,
+    the index must be the bf16 Mean-K of the keys that were appended, and attention straight over the pages must equal
+    attention over the gathered view bit for bit and the oracle's attention over the codes within tolerance."""
+    from kvmem_harness import bits
+    from paper_2609_04852_b200 import SelectParams
+    spec = SPEC.with_(n_blocks=n_blocks, n_planted=min(8, n_blocks // 4), budget_blocks=k, n_q_tokens=M)
+    dev = torch.device("cuda", 0)
+    pool = _fp8_pool(spec, k_scale, v_scale)
+    osess = fill_oracle(spec)[0]
+    assert np.array_equal(bits(pool.index(0)), osess.idx), "the index comes from the bf16 keys"
+    ids = _ids(np.random.default_rng(n_blocks), n_blocks, k)
+    cap = k * 64
+    sel = torch.from_numpy(ids).view(1, -1).to(dev)
+    n_sel = torch.tensor([k], dtype=torch.int32, device=dev)
+    k8, v8t = pool.new_view_fp8(1, cap)
+    pool.materialize_fp8(sel, n_sel, k8, v8t, k_scale, v_scale)
+    q, qb = queries(spec)
+    out, lse = pool.new_outputs(1, M)
+    pool.view_attend_fp8(q.to(dev), k8, v8t, n_sel, out, lse, k_scale, v_scale)
+    out2, lse2 = pool.new_outputs(1, M)
+    pool.paged_attend_fp8(q.to(dev), sel, n_sel, out2, lse2)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    k_inv, v_inv = np.float32(1.0) / np.float32(k_scale), np.float32(1.0) / np.float32(v_scale)
+    rK, rV = orc.gather_fp8(osess.repo, osess.table, ids, cap, float(k_inv), float(v_inv))
+    assert np.array_equal(k8.cpu().numpy()[0], rK), "FP8 key codes differ"
+    assert np.array_equal(v8t.cpu().numpy()[0], rV), "FP8 value codes differ"
+    ref_out, ref_lse = orc.attend_fp8(qb[0], rK, rV, cap, k_scale, v_scale)
+    for o, l in ((out, lse), (out2, lse2)):
+        err_o = np.abs(o.cpu().numpy()[0] - ref_out).max()
+        err_l = np.abs(l.cpu().numpy()[0] - ref_lse).max()
+        assert err_o <= ATTN_ATOL * max(1.0, v_scale) and err_l <= ATTN_ATOL, (err_o, err_l)
+    assert torch.equal(out2, out) and torch.equal(lse2, lse), "copy-free and gathered attention must be the same bits"
+    # selection works off the bf16 index as on any pool: the planted blocks win
+    R, _ = orc.block_scores(qb[0], osess.idx, n_blocks)
+    n_pl = spec.n_planted
+    ref_sel = orc.select(R, 64, n_pl, 1 << 30)
+    sel2 = torch.zeros(1, n_pl, dtype=torch.int32, device=dev)
+    n_sel2 = torch.zeros(1, dtype=torch.int32, device=dev)
+    pool.select(q.to(dev), SelectParams(n_pl, 1 << 30, 0, 0, 0), sel2, n_sel2)
+    assert np.array_equal(sel2.cpu().numpy()[0, : int(n_sel2.item())], ref_sel)
+
+
+def test_page_formats_are_not_mixed_up():
+    from paper_2609_04852_b200 import KvmemError, Pool
+    from paper_2609_04852_b200.kvmem import E_INVALID, E_STATE
+    spec = SPEC.with_(n_blocks=16, n_planted=2)
+    dev = torch.device("cuda", 0)
+    f8 = _fp8_pool(spec, 1.0, 0.5)
+    bf = fill_pool(spec)
+    sel = torch.arange(4, dtype=torch.int32, device=dev).view(1, -1)
+    n_sel = torch.tensor([4], dtype=torch.int32, device=dev)
+    q, _ = queries(spec)
+    qd = q.to(dev)
+    out, lse = f8.new_outputs(1, spec.n_q_tokens)
+    view = f8.new_view(1, 4 * 64)
+    for call in (lambda: f8.materialize(sel, n_sel, view), lambda: f8.materialize_attend(qd, sel, n_sel, view, out, lse),
+                 lambda: f8.paged_attend(qd, sel, n_sel, out, lse), lambda: bf.paged_attend_fp8(qd, sel, n_sel, out, lse)):
+        with pytest.raises(KvmemError) as e:
+            call()
+        assert e.value.status == E_STATE
+    k8, v8t = f8.new_view_fp8(1, 4 * 64)
+    with pytest.raises(KvmemError) as e:
+        f8.materialize_fp8(sel, n_sel, k8, v8t, 1.0, 1.0)            # not the scales the pages were written with
+    assert e.value.status == E_INVALID
+    with pytest.raises(KvmemError):
+        Pool(1, 32, 8, 128, 32, 1, 8, 8, 0, fp8_pages=True)          # 32-token blocks
+    with pytest.raises(KvmemError):
+        Pool(1, 32, 8, 128, 64, 1, 8, 8, 0, 4096, 1.0e6, fp8_pages=True)      # rotary support
+    with pytest.raises(KvmemError):
+        Pool(1, 32, 8, 128, 64, 1, 8, 8, 0, fp8_pages=True, fp8_k_scale=0.0)
+    assert f8.device_status() == 0 and bf.device_status() == 0
+    # half the memory: pages of 1 byte per element
+    assert f8.storage.numel() < 0.6 * bf.storage.numel()

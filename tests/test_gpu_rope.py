@@ -172,4 +172,10 @@ def test_rotary_errors():
     with pytest.raises(KvmemError) as e:
         plain.paged_attend_rope(q, sel, n_sel, out, lse, 0)
     assert e.value.status == E_STATE
+    with pytest.raises(KvmemError) as e:
+        pool.materialize_attend_rope(q, sel, n_sel, view, out, lse, WINDOW - 64)
+    assert e.value.status == E_INVALID
+    with pytest.raises(KvmemError) as e:
+        plain.materialize_attend_rope(q, sel, n_sel, plain.new_view(1, 2 * spec.block_tokens), out, lse, 0)
+    assert e.value.status == E_STATE
     assert pool.device_status() == 0
