@@ -254,6 +254,12 @@ def run_native(args):
                 ev[1].record(stream)
                 ev[2].record(stream)
             return
+        if args.fp8_pages and not args.unfused:  # FP8 repository: tiles stored to the view while attended over, one pass
+            pool.materialize_attend_fp8(q, sel, n_sel, k8, v8t, out, lse)
+            if ev is not None:
+                ev[1].record(stream)
+                ev[2].record(stream)
+            return
         if args.fp8:           # FP8 (E4M3) view: quantise while gathering (or copy the tiles of an FP8 repository), attend over half the bytes
             pool.materialize_fp8(sel, n_sel, k8, v8t)
             if ev is not None:
@@ -362,6 +368,8 @@ def run_native(args):
             pool.select(q_stage, prm, sel, n_sel)
             if args.fp8_pages and args.paged:
                 pool.paged_attend_fp8(q_stage, sel, n_sel, out, lse)
+            elif args.fp8_pages and not args.unfused:
+                pool.materialize_attend_fp8(q_stage, sel, n_sel, k8, v8t, out, lse)
             else:
                 pool.materialize_fp8(sel, n_sel, k8, v8t)
                 pool.view_attend_fp8(q_stage, k8, v8t, n_sel, out, lse)
@@ -524,7 +532,11 @@ def run_native(args):
                                            "kvmem_select + kvmem_materialize_fp8 + kvmem_view_attend_fp8 over an FP8 repository")
                 if args.paged:
                     g_bytes, a_bytes, a_s = a_bytes, 0, 1.0
+                elif not args.unfused:
+                    a_bytes, a_s = 0, 1.0
+                    line["config"]["calls"] = "kvmem_select + kvmem_materialize_attend_fp8 (FP8 repository: view written while attended)"
             line["roofline"] = {"bound": "hbm", "kernel": "attend_fp8_split_kernel<paged> + merge (kvmem_paged_attend_fp8)" if args.fp8_pages and args.paged else
+                                                           "attend_fp8_split_kernel<2> + merge (kvmem_materialize_attend_fp8)" if args.fp8_pages and not args.unfused else
                                                            "gather_fp8_pages_kernel (kvmem_materialize_fp8)" if args.fp8_pages else
                                                            "gather_fp8_kernel (kvmem_materialize_fp8)", "achieved": g_bytes / g_s / 1e9,
                                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": g_bytes / g_s / 1e9 / peaks["hbm_gbs"],
@@ -533,10 +545,11 @@ def run_native(args):
             line["attend_roofline"] = {"kernel": "attend_fp8_split_kernel + merge (kvmem_view_attend_fp8)", "achieved_gbs": a_bytes / a_s / 1e9,
                                        "frac": a_bytes / a_s / 1e9 / peaks["hbm_gbs"], "algorithmic_bytes_per_launch": a_bytes,
                                        "avg_ms": a_s * 1e3}
-            if args.fp8_pages and args.paged:
+            if args.fp8_pages and (args.paged or not args.unfused):
                 line.pop("attend_roofline")
             fp8_step = ns * ab["index"] + g_bytes + a_bytes
             line["step_hbm"] = {"algorithmic_bytes_per_step": fp8_step, "accounting": "index + one read of the selected FP8 pages" if args.fp8_pages and args.paged else
+                                "index + FP8 page read + FP8 view write (fused pass)" if args.fp8_pages and not args.unfused else
                                 "index + FP8 page read + FP8 view write + FP8 view read" if args.fp8_pages else "index + bf16 page read + FP8 view write + FP8 view read",
                                 "achieved_gbs": K * fp8_step / (total_ms * 1e-3) / 1e9,
                                 "frac_of_peak": K * fp8_step / (total_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],

@@ -367,6 +367,16 @@ int kvmem_paged_attend_fp8(kvmem_pool_t* pool, int32_t session_first, int32_t n_
                            const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
                            void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
+/* kvmem_materialize_fp8 followed by kvmem_view_attend_fp8 as ONE pass over an FP8 repository: every selected tile is
+ * read once from the pages, stored to its place in the FP8 view and attended over while it sits in shared memory
+ * (1 byte read + 1 byte written per element).  The view and out/lse are those of the two separate calls with the
+ * pool's scales.  Arguments as kvmem_materialize_attend with the FP8 view buffers.  KVMEM_E_STATE on bf16 pages. */
+int kvmem_materialize_attend_fp8(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
+                                 int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
+                                 const int32_t* n_sel /*DEVICE*/, void* view_k8 /*DEVICE*/, void* view_v8t /*DEVICE*/,
+                                 int32_t view_cap_tokens, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
+                                 void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
 /* Execution cache: the execution view kept across steps, with working-set reuse and bounded delta
  * re-RoPE (Sec. 4.4: the two views; "Retrieval-Aware Hierarchical Reuse"; Eq. "kvmem-working-set-delta").
  *

@@ -854,6 +854,35 @@ int kvmem_paged_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_ses
     return KVMEM_OK;
 }
 
+int kvmem_materialize_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                                 const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k8, void* view_v8t,
+                                 int32_t view_cap_tokens, float scale, float* out, float* lse, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p) || !pages_are(p, true, "kvmem_materialize_attend_fp8")) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!q || !sel_ids || !n_sel || !view_k8 || !view_v8t || !out || !lse || !workspace || !aligned(q, 16) || !aligned(view_k8, 128) ||
+        !aligned(view_v8t, 128) || !aligned(workspace, 256) || !aligned(out, 16)) {
+        set_error("kvmem_materialize_attend_fp8: null or misaligned pointer (views need 128-byte alignment)");
+        return KVMEM_E_INVALID;
+    }
+    if (n_q_tokens < 1 || sel_stride < 1) { set_error("n_q_tokens and sel_stride must be positive"); return KVMEM_E_INVALID; }
+    if (view_cap_tokens < 64 || view_cap_tokens % 64 != 0) { set_error("view_cap_tokens must be a positive multiple of 64"); return KVMEM_E_INVALID; }
+    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
+    if ((int64_t)p->cfg.max_blocks * 2 * p->cfg.n_layers * p->cfg.n_kv_heads * 64 > 0x7fffffffll ||
+        (int64_t)n_sessions * p->cfg.n_layers * p->cfg.n_kv_heads * view_cap_tokens > 0x7fffffffll) {
+        set_error("page pool or view too large for 32-bit TMA row coordinates");
+        return KVMEM_E_UNSUPPORTED;
+    }
+    AttendPlan plan = plan_attend(p->cfg, n_sessions, n_q_tokens, p->sm_count);
+    if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
+    cudaError_t e = launch_attend_fp8(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, (const uint8_t*)view_k8,
+                                      (const uint8_t*)view_v8t, view_cap_tokens, n_sel, scale, p->cfg.fp8_k_scale, p->cfg.fp8_v_scale,
+                                      out, lse, workspace, (cudaStream_t)stream, sel_ids, sel_stride, session_first);
+    if (e != cudaSuccess) return cuda_fail("fused FP8 materialize+attend kernel launch", e);
+    return KVMEM_OK;
+}
+
 // ---- execution cache: working-set reuse with bounded delta re-RoPE ----
 
 static int cache_ok(kvmem_pool_t* p, const void* cache, size_t cache_bytes, int32_t cap_blocks, const char* who) {

@@ -255,12 +255,19 @@ struct AttendF8Args {
     const int32_t* tables;       // [max_sessions][max_bps]
     const int32_t* nblocks_dev;  // [max_sessions]
     int session_first, sel_stride, max_bps, max_blocks;
+    int lookahead;               // MODE 2: tiles the producer may have in flight that have not landed (0: every stage)
 };
 
-// PAGED: map_k covers the page pool ([pages * 2 * L*G * 64 rows][128 bytes]); map_v is unused.
-template <bool PAGED>
-__global__ void __launch_bounds__(kF8Threads, 1)
-attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, AttendF8Args a) {
+// MODE 0: tiles come from the FP8 view (map_k, map_v).
+// MODE 1: copy-free view over an FP8 repository: tiles come from the page pool (map_pages: [pages * 2 * L*G * 64 rows][128
+//         bytes]) through the block table; nothing is written.
+// MODE 2: MODE 1 plus a view-writer warp that stores every landed tile to the FP8 view (map_k, map_v) while the consumers
+//         attend over it: materialize_fp8 + view_attend_fp8 in one pass, 1 byte read + 1 byte written per element.
+template <int MODE>
+__global__ void __launch_bounds__(kF8Threads + (MODE == 2 ? 32 : 0), 1)
+attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                        const __grid_constant__ CUtensorMap map_pages, AttendF8Args a) {
+    constexpr bool PAGED = MODE != 0, FUSED = MODE == 2;
     pdl_wait();
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint64_t full_bar[kF8Stages], empty_bar[kF8Stages];
@@ -273,14 +280,14 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int z = s * LG + lg;
     const int l = lg / a.G, g = lg % a.G;
 
-    const int n_blk = max(0, min(a.n_sel[s], PAGED ? a.sel_stride : a.cap_tokens / kF8Tile));
+    const int n_blk = max(0, min(a.n_sel[s], MODE == 1 ? a.sel_stride : MODE == 2 ? min(a.sel_stride, a.cap_tokens / kF8Tile) : a.cap_tokens / kF8Tile));
     const int t0 = (int)((long long)n_blk * split / a.n_splits);
     const int t1 = (int)((long long)n_blk * (split + 1) / a.n_splits);
     const int n_tiles = t1 - t0;
     const int cap_tiles = a.cap_tokens / kF8Tile;
 
     if (tid == 0) {
-        for (int i = 0; i < kF8Stages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kF8Consumers / kF8Groups); }
+        for (int i = 0; i < kF8Stages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kF8Consumers / kF8Groups + (FUSED ? 1 : 0)); }
         ptx::fence_mbar_init();
     }
     __syncthreads();
@@ -293,8 +300,9 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     if (PAGED && warp == kF8Consumers) {
         // ---------------- producer over pages: the whole warp looks pages up, 32 tiles at a time; lane 0 issues the loads
         if (n_tiles > 0) {
-            if (lane == 0) ptx::prefetch_tensormap(&map_k);
+            if (lane == 0) ptx::prefetch_tensormap(&map_pages);
             const int NB = a.nblocks_dev[a.session_first + s];
+            const int ahead = FUSED && a.lookahead > 0 ? min(a.lookahead, kF8Stages) : kF8Stages;
             auto lookup = [&](int it) -> int {
                 if (it >= n_tiles) return 0;
                 const int id = a.sel_ids[(size_t)s * a.sel_stride + t0 + it];
@@ -310,18 +318,47 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 const int page = __shfl_sync(0xffffffffu, my_page, it - base_it);
                 if (lane == 0) {
                     const int st = it % kF8Stages;
-                    if (it >= kF8Stages) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kF8Stages) & 1) ^ 1));
+                    if (ahead < kF8Stages && it >= ahead) {       // at most `ahead` tiles that have not landed yet
+                        const int jt = it - ahead;
+                        ok = ptx::mbar_wait(&full_bar[jt % kF8Stages], (uint32_t)((jt / kF8Stages) & 1));
+                    }
+                    if (ok && it >= kF8Stages) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kF8Stages) & 1) ^ 1));
                     if (ok) {
                         unsigned char* dst = stages + (size_t)st * kF8StageBytes;
                         // page layout [K|V][L*G][64 rows][128 bytes]
                         ptx::mbar_expect_tx(&full_bar[st], kF8StageBytes);
-                        ptx::tma_load_2d(dst, &map_k, 0, ((page * 2 + 0) * LG + lg) * kF8Tile, &full_bar[st]);
-                        ptx::tma_load_2d(dst + kF8TileBytes, &map_k, 0, ((page * 2 + 1) * LG + lg) * kF8Tile, &full_bar[st]);
+                        ptx::tma_load_2d(dst, &map_pages, 0, ((page * 2 + 0) * LG + lg) * kF8Tile, &full_bar[st]);
+                        ptx::tma_load_2d(dst + kF8TileBytes, &map_pages, 0, ((page * 2 + 1) * LG + lg) * kF8Tile, &full_bar[st]);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
             }
+        }
+    } else if (FUSED && warp == kF8Consumers + 1) {
+        // ---------------- view writer: every tile that lands in shared memory is stored to the FP8 view ----------------
+        if (lane == 0 && n_tiles > 0) {
+            ptx::prefetch_tensormap(&map_k);
+            ptx::prefetch_tensormap(&map_v);
+            bool ok = true;
+            for (int it = 0; it < n_tiles; ++it) {
+                const int st = it % kF8Stages;
+                ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kF8Stages) & 1));
+                if (!ok) break;
+                unsigned char* src = stages + (size_t)st * kF8StageBytes;
+                const int y = (z * cap_tiles + t0 + it) * kF8Tile;
+                ptx::tma_store_2d(&map_k, src, 0, y);
+                ptx::tma_store_2d(&map_v, src + kF8TileBytes, 0, y);
+                ptx::bulk_commit();
+                if (it > 0) {                              // all but the newest store have left shared memory
+                    ptx::bulk_wait_read<1>();
+                    ptx::mbar_arrive(&empty_bar[(it - 1) % kF8Stages]);
+                }
+            }
+            ptx::bulk_wait_read<0>();
+            if (ok) ptx::mbar_arrive(&empty_bar[(n_tiles - 1) % kF8Stages]);
+            else atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+            ptx::bulk_wait<0>();                           // the view is complete before the kernel ends
         }
     } else if (warp == kF8Consumers) {
         // ---------------- producer ----------------
@@ -561,18 +598,22 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
                               int sel_stride, int session_first) {
     const Geometry& g = p.geo;
     const int LG = g.L * g.G, heads = n_sessions * LG;
-    const bool paged = sel_ids != nullptr;                  // copy-free: straight over the pages of an FP8 repository
-    CUtensorMap map_k, map_v;
-    if (paged) {
-        if (!make_f8_map(&map_k, reinterpret_cast<const uint8_t*>(p.pages), (long long)g.max_blocks * 2 * LG * kF8Tile)) return cudaErrorInvalidValue;
-        map_v = map_k;
+    const bool paged = sel_ids != nullptr;                  // straight over the pages of an FP8 repository ...
+    const bool fused = paged && view_k != nullptr;          // ... and, with view buffers, storing the view on the way
+    CUtensorMap map_k, map_v, map_pages;
+    if (paged && !make_f8_map(&map_pages, reinterpret_cast<const uint8_t*>(p.pages), (long long)g.max_blocks * 2 * LG * kF8Tile))
+        return cudaErrorInvalidValue;
+    if (paged && !fused) {
+        map_k = map_pages; map_v = map_pages;               // unused by this mode
     } else if (!make_f8_map(&map_k, view_k, (long long)heads * view_cap_tokens) || !make_f8_map(&map_v, view_v, (long long)heads * view_cap_tokens)) {
         return cudaErrorInvalidValue;
     }
+    if (!paged) map_pages = map_k;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attend_fp8_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
+        cudaError_t e = cudaFuncSetAttribute(attend_fp8_split_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -591,10 +632,20 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
     a.sel_ids = sel_ids; a.tables = p.tables; a.nblocks_dev = p.nblocks_dev;
     a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
-    if (paged)
-        launch_pdl(attend_fp8_split_kernel<true>, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, a);
+    // the view-writing pass is fastest with about 9.5 MiB of tiles that have not landed yet over all SMs (as its bf16 counterpart)
+    a.lookahead = g_attend_lookahead;
+    if (fused && a.lookahead == 0) {
+        const long long ctas = (long long)a.n_splits * heads;
+        const int tiles_per_cta = (view_cap_tokens / kF8Tile + a.n_splits - 1) / a.n_splits;
+        if (ctas <= p.sm_count && tiles_per_cta >= 64)
+            a.lookahead = std::max(2, std::min(kF8Stages, (int)(9.5 * 1024.0 * 1024.0 / ((double)ctas * kF8StageBytes) + 0.5)));
+    }
+    if (fused)
+        launch_pdl(attend_fp8_split_kernel<2>, dim3(grid), dim3(kF8Threads + 32), kF8Smem, st, map_k, map_v, map_pages, a);
+    else if (paged)
+        launch_pdl(attend_fp8_split_kernel<1>, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, map_pages, a);
     else
-        launch_pdl(attend_fp8_split_kernel<false>, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, a);
+        launch_pdl(attend_fp8_split_kernel<0>, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, map_pages, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     launch_pdl(attend_merge_kernel, dim3((unsigned)a.rows, (unsigned)heads), dim3(kF8D), 0, st, a.part_o, a.part_ml, out, lse, M, g.L,

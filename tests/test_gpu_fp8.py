@@ -146,6 +146,13 @@ def test_fp8_repository_pages_view_and_copy_free_attention(n_blocks, k, M, k_sca
         err_l = np.abs(l.cpu().numpy()[0] - ref_lse).max()
         assert err_o <= ATTN_ATOL * max(1.0, v_scale) and err_l <= ATTN_ATOL, (err_o, err_l)
     assert torch.equal(out2, out) and torch.equal(lse2, lse), "copy-free and gathered attention must be the same bits"
+    # one pass: tiles stored to the view while attended over
+    k8f, v8f = pool.new_view_fp8(1, cap)
+    out3, lse3 = pool.new_outputs(1, M)
+    pool.materialize_attend_fp8(q.to(dev), sel, n_sel, k8f, v8f, out3, lse3)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    assert torch.equal(k8f, k8) and torch.equal(v8f, v8t) and torch.equal(out3, out) and torch.equal(lse3, lse)
     # selection works off the bf16 index as on any pool: the planted blocks win
     R, _ = orc.block_scores(qb[0], osess.idx, n_blocks)
     n_pl = spec.n_planted
@@ -170,7 +177,8 @@ def test_page_formats_are_not_mixed_up():
     out, lse = f8.new_outputs(1, spec.n_q_tokens)
     view = f8.new_view(1, 4 * 64)
     for call in (lambda: f8.materialize(sel, n_sel, view), lambda: f8.materialize_attend(qd, sel, n_sel, view, out, lse),
-                 lambda: f8.paged_attend(qd, sel, n_sel, out, lse), lambda: bf.paged_attend_fp8(qd, sel, n_sel, out, lse)):
+                 lambda: f8.paged_attend(qd, sel, n_sel, out, lse), lambda: bf.paged_attend_fp8(qd, sel, n_sel, out, lse),
+                 lambda: bf.materialize_attend_fp8(qd, sel, n_sel, *bf.new_view_fp8(1, 4 * 64), out, lse)):
         with pytest.raises(KvmemError) as e:
             call()
         assert e.value.status == E_STATE
