@@ -389,21 +389,19 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                 t5::fence_after();
                 const int col0 = t * kCkBN + half * kCkHalfCols;
                 const bool ragged = col0 + kCkHalfCols > NB;
-                uint32_t buf[kCkChunks][32];
 #pragma unroll
-                for (int c = 0; c < kCkChunks; ++c) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf[c]);
-                t5::ld_wait();
-                // the accumulator now lives in registers: hand it back before doing the arithmetic
-                t5::fence_before();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
-                if (!ragged) {
-#pragma unroll
-                    for (int c = 0; c < kCkChunks; ++c) rowstat_chunk<false, POLY>(buf[c], 0, a.scale_log2e, run_m, run_z);
-                } else {
-#pragma unroll
-                    for (int c = 0; c < kCkChunks; ++c)
-                        rowstat_chunk<true, POLY>(buf[c], NB - (col0 + c * 32), a.scale_log2e, run_m, run_z);
+                for (int c = 0; c < kCkChunks; ++c) {
+                    // 32 columns at a time: fewer live registers leave the compiler room to overlap the exponentials
+                    uint32_t buf[32];
+                    t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf);
+                    t5::ld_wait();
+                    if (c == kCkChunks - 1) {           // the whole slice has been read: hand the accumulator back
+                        t5::fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
+                    }
+                    if (!ragged) rowstat_chunk<false, POLY>(buf, 0, a.scale_log2e, run_m, run_z);
+                    else rowstat_chunk<true, POLY>(buf, NB - (col0 + c * 32), a.scale_log2e, run_m, run_z);
                 }
             }
             if (!failed && row < a.rows)
@@ -607,23 +605,24 @@ score_chunk_colsum_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 }
                 t5::fence_after();
                 const float4* sh4 = reinterpret_cast<const float4*>(shift + qt * kCkBN + half * kCkHalfCols);
-                uint32_t buf[kCkChunks][32];
-#pragma unroll
-                for (int c = 0; c < kCkChunks; ++c) t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf[c]);
-                t5::ld_wait();
-                // the accumulator now lives in registers: hand it back before doing the arithmetic
-                t5::fence_before();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
                 const uint64_t sc2 = f2::pk(a.scale_log2e, a.scale_log2e);
                 uint64_t acc0 = f2::pk(0.0f, 0.0f), acc1 = acc0;
 #pragma unroll
                 for (int c = 0; c < kCkChunks; ++c) {
+                    // 32 columns at a time: fewer live registers leave the compiler room to overlap the exponentials
+                    uint32_t buf[32];
+                    t5::ld32_issue(lane_addr + (uint32_t)(acc * kCkBN + c * 32), buf);
+                    t5::ld_wait();
+                    if (c == kCkChunks - 1) {           // the whole slice has been read: hand the accumulator back
+                        t5::fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
+                    }
 #pragma unroll
                     for (int i = 0; i < 32; i += 4) {
                         const float4 sh = sh4[c * 8 + (i >> 2)];            // same address in every lane: broadcast
-                        acc0 = f2::add(acc0, ex2_pair<POLY>(f2::fma(f2::pk(buf[c][i], buf[c][i + 1]), sc2, f2::pk(sh.x, sh.y)), i >> 1));
-                        acc1 = f2::add(acc1, ex2_pair<POLY>(f2::fma(f2::pk(buf[c][i + 2], buf[c][i + 3]), sc2, f2::pk(sh.z, sh.w)), (i >> 1) + 1));
+                        acc0 = f2::add(acc0, ex2_pair<POLY>(f2::fma(f2::pk(buf[i], buf[i + 1]), sc2, f2::pk(sh.x, sh.y)), i >> 1));
+                        acc1 = f2::add(acc1, ex2_pair<POLY>(f2::fma(f2::pk(buf[i + 2], buf[i + 3]), sc2, f2::pk(sh.z, sh.w)), (i >> 1) + 1));
                     }
                 }
                 float s0, s1, s2, s3;
