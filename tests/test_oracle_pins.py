@@ -68,13 +68,22 @@ def test_index_incremental_append_equals_one_shot():
 
 
 def test_index_footprint_matches_paper_growth():
-    # Sec. 6.5: ~0.25 GiB at 256K tokens and ~9.5 GiB at 10M tokens with 32-token blocks:
-    # one vector per (block, layer, KV head) means bytes grow linearly in blocks; both
-    # figures give the same per-block size.
-    per_block_256k = 0.25 * 2 ** 30 / (256 * 1024 / 32)
-    per_block_10m = 9.5 * 2 ** 30 / (10_000_000 / 32)
-    assert abs(per_block_256k - 32 * 1024) < 1
-    assert abs(per_block_10m / per_block_256k - 1) < 0.03
+    # Sec. 6.5 (values in tests/golden/index_footprint.txt): ~0.25 GiB at 256K tokens and ~9.5 GiB at 10M tokens with
+    # 32-token blocks.  One vector per (block, layer, KV head) means bytes grow linearly in blocks: both figures give
+    # the same per-block size, and that size is what the oracle's index layout occupies for a model whose scored
+    # layers x KV heads x head_dim x 2 bytes come to 32 KiB per block.
+    import os
+    rows = [ln.split() for ln in open(os.path.join(os.path.dirname(__file__), "golden", "index_footprint.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    (t0, b0, g0), (t1, b1, g1) = [(int(r[0]), int(r[1]), float(r[2])) for r in rows]
+    per_block_small = g0 * 2 ** 30 / (t0 / b0)
+    per_block_large = g1 * 2 ** 30 / (t1 / b1)
+    assert abs(per_block_small - 32 * 1024) < 1
+    assert abs(per_block_large / per_block_small - 1) < 0.03
+    # the oracle's index of a geometry with 32 KiB per block (e.g. 16 scored layers x 8 KV heads x 128 dims, bf16)
+    L, G, d, NB, B = 16, 8, 128, 3, b0
+    idx = orc.mean_k_index(rand_bits(NB * B, L, G, d), B)
+    assert idx.nbytes == NB * int(per_block_small) and idx.shape == (L, G, NB, d)
 
 
 # ------------------------------------------------------------------ block scores (Eq. kvmem-block-score)
