@@ -134,3 +134,38 @@ def test_1m_fp8_repository_passes():
     assert np.array_equal(k8.cpu().numpy()[0], rK) and np.array_equal(v8t.cpu().numpy()[0], rV)
     ref_out, ref_lse = orc.attend_fp8(qb[0], rK, rV, T, 0.5, 0.25)
     assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+
+
+def test_1m_position_consistent_passes_on_raw_keys():
+    """Raw keys in the pages (the paper's layout, Sec. 4.3/4.4): the rotating gather against the oracle at full size,
+    attention over it, and the copy-free pass that rotates key fragments in registers, which must give the same bits."""
+    from paper_2609_04852_b200 import Pool
+    spec = SPEC
+    dev = torch.device("cuda", 0)
+    theta, B = 1.0e6, spec.block_tokens
+    window = spec.max_view_tokens + 64
+    pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, B, 1, spec.n_blocks, spec.n_blocks, 0,
+                window, theta)
+    tab = orc.rope_table(window, spec.head_dim, theta)
+    table = page_table(spec)[0]
+    for b0 in range(0, spec.n_blocks, 1024):
+        b1 = min(spec.n_blocks, b0 + 1024)
+        K, V = kv_blocks(spec, 0, b0, b1, dev)
+        pool.append_blocks(0, K, V, table[b0:b1].tolist())
+    q, qb = queries(spec)
+    qd = q.to(dev)
+    osess = fill_oracle(spec, gen_device=dev)[0]
+    sel, n_sel, ids, k = _oracle_selection(spec, osess, qb, dev)
+    M, T, first = spec.n_q_tokens, k * B, 37
+    view = pool.new_view(1, T)
+    out, lse = pool.new_outputs(1, M)
+    pool.materialize_attend_rope(qd, sel, n_sel, view, out, lse, first)      # two kernels on a raw-key pool
+    out2, lse2 = pool.new_outputs(1, M)
+    pool.paged_attend_rope(qd, sel, n_sel, out2, lse2, first)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    vK, vV = orc.gather_rope(osess.repo, osess.table, ids, T, first, tab)
+    assert np.array_equal(bits(view.k[0]), vK) and np.array_equal(bits(view.v[0]), vV)
+    ref_out, ref_lse = orc.attend(qb[0], vK, vV, T)
+    assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+    assert torch.equal(out2, out) and torch.equal(lse2, lse)
