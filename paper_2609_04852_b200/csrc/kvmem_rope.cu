@@ -127,7 +127,10 @@ cudaError_t launch_gather_rope(const kvmem_pool& p, int session_first, int n_ses
     a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
     a.LG = g.L * g.G; a.B = g.B; a.d = g.d; a.cap_tokens = view_cap_tokens; a.first_position = first_position;
     a.rope_positions = p.cfg.rope_max_positions; a.page_elems = p.lay.page_elems; a.in_block = p.cfg.rope_in_block_keys;
-    const int ctas = std::max(1, p.sm_count * 8 / n_sessions);
+    // many short-lived CTAs (about 64 per SM over the kernel's life, 8 resident): a CTA rotates a K tile with long
+    // dependent chains (table row, then arithmetic) or copies a V tile; the hardware scheduler overlaps and balances them
+    // better than 8 persistent CTAs per SM do (measured at 1M: 397 us with 8 per SM, 355 us with 64)
+    const int ctas = g_gather_ctas > 0 ? g_gather_ctas : std::max(1, p.sm_count * 64 / n_sessions + 1);
     launch_pdl(gather_rope_kernel, dim3(dim3((unsigned)ctas, (unsigned)n_sessions)), dim3(256), 0, st, a);
     return cudaGetLastError();
 }
