@@ -123,7 +123,6 @@ template <int MODE>
 __global__ void __launch_bounds__(MODE == 3 ? (kAttRopeConsumers + 1) * 32 : kAttThreads + (MODE == 1 ? 32 : MODE == 4 ? 32 * kQrotWarps : MODE == 5 ? 32 + 32 * kKrotWarps : 0), 1)
 attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_pages, AttendArgs a) {
-    pdl_wait();        // everything earlier in the stream is complete and visible from here on
     constexpr bool FUSED = MODE == 1 || MODE == 5;   // a view-writer warp shares every stage with the consumers
     constexpr bool KROT = MODE == 5;       // rotator warps re-encode every K tile in place before anybody else reads it
     constexpr bool PAGED = MODE != 0;      // the producer reads pages through the block table
@@ -145,6 +144,20 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     const int z = s * LG + lg;
     const int l = lg / a.G, g = lg % a.G;
 
+    // what needs no global memory comes first, so that it overlaps the tail of the kernel before this one
+    if (tid == 0) {
+        for (int i = 0; i < STAGES; ++i) {
+            ptx::mbar_init(&full_bar[i], 1);
+            ptx::mbar_init(&empty_bar[i], CONSUMERS / GROUPS + (FUSED ? 1 : 0));
+        }
+        for (int i = 0; i < GROUPS; ++i) { ptx::mbar_init(&tab_full[i], 1); ptx::mbar_init(&tab_empty[i], CONSUMERS / GROUPS); }
+        for (int i = 0; i < kAttStages; ++i) ptx::mbar_init(&q_full[i], 1);
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(PAGED ? &map_pages : &map_k);
+    }
+    __syncthreads();
+    pdl_wait();        // everything earlier in the stream is complete and visible from here on
+
     // view length in tokens; the kernel works in 64-token tiles, whatever the block size of the view (a multiple of
     // 16, so each consumer warp's 16 tokens are all inside or all outside the view)
     const int btok = PAGED ? kTile : a.block_tokens;
@@ -155,17 +168,6 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     const int t1 = (int)((long long)n_blk * (split + 1) / a.n_splits);
     const int n_tiles = t1 - t0;
     const int ahead = a.lookahead > 0 ? min(a.lookahead, STAGES) : STAGES;
-
-    if (tid == 0) {
-        for (int i = 0; i < STAGES; ++i) {
-            ptx::mbar_init(&full_bar[i], 1);
-            ptx::mbar_init(&empty_bar[i], CONSUMERS / GROUPS + (FUSED ? 1 : 0));
-        }
-        for (int i = 0; i < GROUPS; ++i) { ptx::mbar_init(&tab_full[i], 1); ptx::mbar_init(&tab_empty[i], CONSUMERS / GROUPS); }
-        for (int i = 0; i < kAttStages; ++i) ptx::mbar_init(&q_full[i], 1);
-        ptx::fence_mbar_init();
-    }
-    __syncthreads();
 
     float o[16][4];           // O accumulators: 16 n-tiles of 8 dims
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
