@@ -66,3 +66,37 @@ def test_calls_without_a_pool_fail_cleanly():
     cfg = PoolConfig(1, 32, 8, 128, 64, 1, 8, 8, 0)
     assert lib.kvmem_pool_create(C.byref(cfg), None, 0, C.byref(handle)) == kvmem.E_INVALID   # null storage
     assert not handle.value
+
+
+def test_page_format_options_are_validated_and_sized_on_the_host():
+    """The optional page formats (keys rotated by their in-block offset; FP8 repository) are configuration: what is
+    accepted, what is refused and how many bytes the pool takes are decided on the host, before any GPU work."""
+    lib = load_library()
+    base = dict(n_layers=1, n_q_heads=32, n_kv_heads=8, head_dim=128, block_tokens=64, max_sessions=1, max_blocks=1024,
+                max_blocks_per_session=1024, device=0)
+
+    def cfg(**kw):
+        c = PoolConfig()
+        for k, v in {**base, **kw}.items():
+            setattr(c, k, v)
+        return c
+
+    plain = lib.kvmem_pool_bytes(C.byref(cfg()))
+    assert plain > 0
+    # rotary table: 8 bytes x head_dim / 2 per position, plus the per-block original positions
+    rope = lib.kvmem_pool_bytes(C.byref(cfg(rope_max_positions=4096, rope_theta=1.0e6)))
+    assert rope - plain >= 4096 * 64 * 8 and rope - plain <= 4096 * 64 * 8 + 1024 * 4 + 1024
+    in_block = lib.kvmem_pool_bytes(C.byref(cfg(rope_max_positions=4096, rope_theta=1.0e6, rope_in_block_keys=1)))
+    assert in_block == rope                                        # a different content of the same pages
+    assert lib.kvmem_pool_bytes(C.byref(cfg(rope_in_block_keys=1))) == 0 and b"rope_in_block_keys" in lib.kvmem_last_error()
+    assert lib.kvmem_pool_bytes(C.byref(cfg(rope_max_positions=32, rope_theta=1.0e6, rope_in_block_keys=1))) == 0
+    assert lib.kvmem_pool_bytes(C.byref(cfg(rope_max_positions=64, rope_theta=0.5))) == 0
+    # FP8 repository: one byte per page element, the index stays bf16
+    f8 = lib.kvmem_pool_bytes(C.byref(cfg(fp8_pages=1, fp8_k_scale=1.0, fp8_v_scale=0.5)))
+    page_elems = 1024 * 2 * 8 * 64 * 128
+    assert plain - f8 == page_elems                                # 2 bytes -> 1 byte per element
+    for bad in (dict(fp8_pages=1, fp8_k_scale=0.0, fp8_v_scale=1.0), dict(fp8_pages=1, fp8_k_scale=1.0, fp8_v_scale=float("inf")),
+                dict(fp8_pages=1, fp8_k_scale=1.0, fp8_v_scale=1.0, block_tokens=32),
+                dict(fp8_pages=1, fp8_k_scale=1.0, fp8_v_scale=1.0, rope_max_positions=4096, rope_theta=1.0e6),
+                dict(fp8_pages=2, fp8_k_scale=1.0, fp8_v_scale=1.0)):
+        assert lib.kvmem_pool_bytes(C.byref(cfg(**bad))) == 0, bad
