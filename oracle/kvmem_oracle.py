@@ -350,3 +350,26 @@ def attend_fp8(q: np.ndarray, viewK8: np.ndarray, viewV8T: np.ndarray, T: int, k
     lib().kvo_attend_fp8(_ptr(q), _ptr(viewK8), _ptr(viewV8T), T, cap, M, L, H, G, d, float(scale), float(k_scale),
                          float(v_scale), _ptr(out), _ptr(lse))
     return out, lse
+
+
+def attend_fp8_qrot(q: np.ndarray, viewK8: np.ndarray, viewV8T: np.ndarray, T: int, block_tokens: int, first_pos: int,
+                    tab: np.ndarray, k_scale: float = 1.0, v_scale: float = 1.0, scale: Optional[float] = None
+                    ) -> Tuple[np.ndarray, np.ndarray]:
+    """Attention over an FP8 view whose keys are the codes of in-block-rotated keys (RoPE(k, offset in block) / k_scale),
+    with the query rotated back by each block's compact position (Sec. 4.4 position consistency on an FP8 KV cache,
+    Sec. 6.1).  Every E4M3 value is exactly representable in bf16, so this is attend_qrot on the dequantised view:
+    the codes widened (exactly) to bf16, the value tiles transposed back, k_scale folded into the softmax scale and
+    v_scale applied to the output."""
+    _u16(q)
+    L, G, cap, d = viewK8.shape
+    assert viewK8.dtype == np.uint8 and viewV8T.dtype == np.uint8 and viewV8T.shape == (L, G, cap // 64, d, 64)
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    kf = dequantize_e4m3(viewK8)
+    vf = dequantize_e4m3(viewV8T).transpose(0, 1, 2, 4, 3).reshape(L, G, cap, d)
+    kb = np.ascontiguousarray(kf).view(np.uint32) >> 16          # exact: an E4M3 value has 3 mantissa bits
+    vb = np.ascontiguousarray(vf).view(np.uint32) >> 16
+    assert np.array_equal(bf16_bits_to_f32(kb.astype(np.uint16)), kf)
+    out, lse = attend_qrot(q, np.ascontiguousarray(kb.astype(np.uint16)), np.ascontiguousarray(vb.astype(np.uint16)), T,
+                           block_tokens, first_pos, tab, float(scale) * float(k_scale))
+    return out * np.float32(v_scale), lse

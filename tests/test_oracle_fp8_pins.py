@@ -116,3 +116,53 @@ def test_fp8_attention_equals_bf16_attention_over_the_dequantised_view():
     vK, vV = orc.gather(repo, table, sel, cap)
     O4, _ = orc.attend(q, vK, vV, T)
     assert np.abs(O4 - O1).max() < 0.1
+
+
+def test_fp8_attention_with_the_query_rotated_back_reduces_to_the_known_cases():
+    """attend_fp8_qrot (FP8 codes of in-block-rotated keys, query rotated back per block): at compact position 0 the
+    rotation is the identity, so one tile must give attend_fp8 exactly; in general it must agree, within the rounding of
+    the rotated query, with attention over keys rotated FORWARD in fp64 (the formulation it replaces); and the
+    scales must act as in attend_fp8."""
+    B, L, G, d, H, M, NB = 64, 1, 2, 16, 4, 3, 3
+    r = np.random.default_rng(77)
+    tab = orc.rope_table(1024, d, 1.0e4)
+    K = to_bits(r.standard_normal((NB * B, L, G, d)).astype(np.float32))
+    V = to_bits(r.standard_normal((NB * B, L, G, d)).astype(np.float32))
+    q = to_bits(r.standard_normal((M, L, H, d)).astype(np.float32))
+    table = np.arange(NB, dtype=np.int32)
+    # repository of in-block-rotated keys, then its FP8 view
+    t_in = (np.arange(NB * B) % B).astype(np.int32)
+    Kp = orc.rope_rotate(np.ascontiguousarray(K.reshape(NB * B, L * G, d)), t_in, tab).reshape(K.shape)
+    repo = orc.Repository.empty(NB, B, L, G, d)
+    repo.place(Kp, V, table)
+    sel = np.array([0, 2], np.int32)
+    cap, T = 2 * B, 2 * B
+    k8, v8t = orc.gather_fp8(repo, table, sel, cap, 0.5, 2.0)
+    # one tile at position 0: R(0) = identity
+    O1, l1 = orc.attend_fp8_qrot(q, k8, v8t, B, B, 0, tab, 2.0, 0.5)
+    O2, l2 = orc.attend_fp8(q, k8, v8t, B, 2.0, 0.5)
+    assert np.array_equal(O1, O2) and np.array_equal(l1, l2)
+    # two tiles at first position 37: against forward rotation of the dequantised keys in fp64
+    first = 37
+    O3, l3 = orc.attend_fp8_qrot(q, k8, v8t, T, B, first, tab, 2.0, 0.5)
+    kd = orc.dequantize_e4m3(k8, 2.0).astype(np.float64)                     # [L][G][cap][d]
+    vd = orc.dequantize_e4m3(v8t, 0.5).astype(np.float64).transpose(0, 1, 2, 4, 3).reshape(L, G, cap, d)
+    half = d // 2
+    freq = 1.0e4 ** (-np.arange(half, dtype=np.float64) * 2.0 / d)
+    qf = from_bits(q).astype(np.float64)
+    for m in range(M):
+        for h in range(H):
+            g = h // (H // G)
+            p0 = first + (np.arange(T) // B) * B                              # the block's compact position: t is already in the key
+            ang = p0[:, None] * freq[None, :]
+            c, s = np.cos(ang), np.sin(ang)
+            kk = kd[0, g, :T]
+            kr = np.concatenate([kk[:, :half] * c - kk[:, half:] * s, kk[:, half:] * c + kk[:, :half] * s], axis=1)
+            logit = kr @ qf[m, 0, h] / np.sqrt(d)
+            w = np.exp(logit - logit.max())
+            o = (w / w.sum()) @ vd[0, g, :T]
+            assert np.abs(O3[m, 0, h] - o).max() < 2e-2
+            assert abs(l3[m, 0, h] - (logit.max() + np.log(w.sum()))) < 2e-2
+    # a different first position changes the result (the rotation is really applied)
+    O4, _ = orc.attend_fp8_qrot(q, k8, v8t, T, B, first + 300, tab, 2.0, 0.5)
+    assert np.abs(O4 - O3).max() > 1e-3
