@@ -226,6 +226,12 @@ def run_native(args):
             pool.select(q_raw, prm, sel, n_sel)
             if ev is not None:
                 ev[0].record(stream)
+            if args.paged and args.fp8_pages:       # FP8 repository of in-block-rotated keys: query rotated back per block
+                pool.paged_attend_fp8_rope(q, sel, n_sel, out, lse, 0)
+                if ev is not None:
+                    ev[1].record(stream)
+                    ev[2].record(stream)
+                return
             if args.paged:      # copy-free: raw key tiles are RoPE'd in shared memory on their way to the tensor cores
                 pool.paged_attend_rope(q, sel, n_sel, out, lse, 0)
                 if ev is not None:
@@ -356,7 +362,9 @@ def run_native(args):
             q_stage.copy_(q_pin[i % len(q_pin)], non_blocking=True)
             pool.rope_rotate(q_stage.view(M, H, d), q_pos, out=q_raw.view(M, H, d), inverse=True)
             pool.select(q_raw, prm, sel, n_sel)
-            if args.paged:
+            if args.paged and args.fp8_pages:
+                pool.paged_attend_fp8_rope(q_stage, sel, n_sel, out, lse, 0)
+            elif args.paged:
                 pool.paged_attend_rope(q_stage, sel, n_sel, out, lse, 0)
             else:
                 pool.materialize_attend_rope(q_stage, sel, n_sel, view, out, lse, 0)
@@ -555,6 +563,22 @@ def run_native(args):
                                 "frac_of_peak": K * fp8_step / (total_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                 "peak_source": f"of {peaks['source']}", "nominal_peak_gbs": 8000.0}
             line["e2e"]["api"] = "pinned host query in, host O and LSE out, around the three calls of the FP8-view step"
+        if args.rope and args.paged and args.fp8_pages:
+            # FP8 repository of in-block-rotated keys, copy-free: one byte per element of the selected blocks is read
+            a_bytes = ns * ab["attend"] // 2
+            a_s = gather_s
+            line["dtype"] = "E4M3 pages (codes of RoPE(k, offset in block), quantised at append), bf16 query and index, f16 tensor-core products, fp32 accumulation"
+            line["config"]["calls"] = ("kvmem_rope_rotate(q) + kvmem_select + kvmem_paged_attend_fp8_rope (FP8 repository, position-consistent, "
+                                       "copy-free: the query is rotated back once per block)")
+            line["roofline"] = {"bound": "hbm", "kernel": "attend_fp8_split_kernel<3> + merge (kvmem_paged_attend_fp8_rope)", "achieved": a_bytes / a_s / 1e9,
+                                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a_bytes / a_s / 1e9 / peaks["hbm_gbs"],
+                                "peak_source": f"of {peaks['source']}", "algorithmic_bytes_per_launch": a_bytes,
+                                "avg_launch_ms": a_s * 1e3, "traffic": None}
+            f8_step = ns * ab["index"] + a_bytes
+            line["step_hbm"] = {"algorithmic_bytes_per_step": f8_step, "accounting": "index + one read of the selected FP8 pages",
+                                "achieved_gbs": K * f8_step / (total_ms * 1e-3) / 1e9,
+                                "frac_of_peak": K * f8_step / (total_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                "peak_source": f"of {peaks['source']}", "nominal_peak_gbs": 8000.0}
         if args.rope:
             line["e2e"]["api"] = "pinned host query in, host O and LSE out, around the four calls of the position-consistent step"
         if world == 1 and not args.no_cpu_baseline:
@@ -978,7 +1002,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-blocks", type=int, default=256)
     args = ap.parse_args()
-    if args.fp8_pages:
+    if args.fp8_pages and args.rope:
+        if not args.paged:
+            raise SystemExit("--fp8-pages --rope is the copy-free position-consistent step: add --paged")
+        args.in_block = True           # codes cannot be re-encoded: the keys carry their in-block rotation, the query is rotated
+    elif args.fp8_pages:
         args.fp8 = True
     if args.in_block and not args.rope:
         raise SystemExit("--in-block needs --rope")

@@ -72,7 +72,9 @@ typedef struct {
                                        block, and the copy-free attention rotates the QUERY back by p0 once per
                                        block instead of every key forward (q . R(p0 + t) k = (R(-p0) q) . R(t) k).
                                        The Mean-K index is built from the raw keys either way              */
-    int32_t fp8_pages;              /* 0: pages hold bf16.  1 (head_dim 128, 64-token blocks, no rotary support): the
+    int32_t fp8_pages;              /* 0: pages hold bf16.  1 (head_dim 128, 64-token blocks; rotary support only together
+                                       with rope_in_block_keys, in which case the codes are those of RoPE(k, t) and
+                                       kvmem_paged_attend_fp8_rope is the position-consistent reader): the
                                        repository itself is FP8 (Sec. 6.1: the KV cache is kept in FP8): a page holds the
                                        E4M3 codes of k / fp8_k_scale ([64 tokens][128] bytes per layer and KV head) and
                                        of v / fp8_v_scale transposed ([128 dims][64 tokens] bytes), i.e. the tiles of the
@@ -366,6 +368,20 @@ int kvmem_paged_attend_fp8(kvmem_pool_t* pool, int32_t session_first, int32_t n_
                            int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
                            const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
                            void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+
+/* kvmem_paged_attend_fp8 with position-consistent keys, for a pool with fp8_pages AND rope_in_block_keys (the
+ * paper's three mechanisms together: FP8 KV cache, Sec. 6.1; keys encoded at their compact positions, Sec. 4.4;
+ * copy-free view, Sec. 5.3).  The pages hold the codes of RoPE(k, t) / fp8_k_scale, t the offset inside the block;
+ * codes cannot be re-encoded without a second quantisation, so no key is touched: the logit q . R(p0 + t) k equals
+ * (R(-p0) q) . RoPE(k, t), and the 16 query rows are rotated back by the block's compact position p0 =
+ * first_position + j*64 once per block (arithmetic of kvmem_rope_rotate, inverse; the rotated query is rounded to
+ * bf16, then widened to f16 for the tensor cores).  q carries RoPE at its own position.
+ * Extra errors: KVMEM_E_STATE unless the pool has both options; KVMEM_E_INVALID if the compact positions leave the
+ * rotary table. */
+int kvmem_paged_attend_fp8_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
+                                int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
+                                const int32_t* n_sel /*DEVICE*/, int32_t first_position, float scale, float* out /*DEVICE*/,
+                                float* lse /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
 /* kvmem_materialize_fp8 followed by kvmem_view_attend_fp8 as ONE pass over an FP8 repository: every selected tile is
  * read once from the pages, stored to its place in the FP8 view and attended over while it sits in shared memory

@@ -44,7 +44,8 @@ bool config_valid(const kvmem_pool_config_t& c, const char** why) {
     if (c.fp8_pages != 0 && c.fp8_pages != 1) return bad("fp8_pages must be 0 or 1");
     if (c.fp8_pages) {
         if (c.head_dim != 128 || c.block_tokens != 64) return bad("an FP8 repository needs head_dim 128 and 64-token blocks");
-        if (c.rope_max_positions > 0) return bad("an FP8 repository cannot be combined with rotary support");
+        if (c.rope_max_positions > 0 && !c.rope_in_block_keys)
+            return bad("an FP8 repository with rotary support needs rope_in_block_keys (codes cannot be re-encoded; the query is rotated instead)");
         if (!(c.fp8_k_scale > 0.0f) || !(c.fp8_v_scale > 0.0f) || !std::isfinite(c.fp8_k_scale) || !std::isfinite(c.fp8_v_scale))
             return bad("fp8_k_scale and fp8_v_scale must be positive and finite");
     }
@@ -302,7 +303,7 @@ static int append_impl(kvmem_pool_t* p, int32_t session, const void* k, const vo
                             (size_t)n_blocks * 4, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) return cuda_fail("block position upload", e);
     }
-    e = p->cfg.fp8_pages ? launch_append_fp8(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st)
+    e = p->cfg.fp8_pages ? launch_append_fp8(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st, block_pos0 != nullptr)
                          : launch_append(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st, block_pos0 != nullptr);
     if (e != cudaSuccess) return cuda_fail("append kernel launch", e);
     for (int32_t pg : ids) { p->page_used[pg] = 1; p->sess_pages[session].push_back(pg); }
@@ -828,9 +829,9 @@ int kvmem_view_attend_fp8(kvmem_pool_t* p, int32_t n_sessions, const void* q, in
     return KVMEM_OK;
 }
 
-int kvmem_paged_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
-                           const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, float scale, float* out, float* lse,
-                           void* workspace, size_t workspace_bytes, void* stream) {
+static int paged_attend_fp8_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                                 const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, int32_t rope_first_position,
+                                 float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
     if (!pool_ok(p) || !pages_are(p, true, "kvmem_paged_attend_fp8")) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q || !sel_ids || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(workspace, 256) || !aligned(out, 16)) {
@@ -849,9 +850,34 @@ int kvmem_paged_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_ses
     if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
     cudaError_t e = launch_attend_fp8(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, nullptr, nullptr, sel_stride * 64, n_sel,
                                       scale, p->cfg.fp8_k_scale, p->cfg.fp8_v_scale, out, lse, workspace, (cudaStream_t)stream,
-                                      sel_ids, sel_stride, session_first);
+                                      sel_ids, sel_stride, session_first, rope_first_position);
     if (e != cudaSuccess) return cuda_fail("paged FP8 attention kernel launch", e);
     return KVMEM_OK;
+}
+
+int kvmem_paged_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                           const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, float scale, float* out, float* lse,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    return paged_attend_fp8_impl(p, session_first, n_sessions, q, n_q_tokens, sel_ids, sel_stride, n_sel, -1, scale, out, lse,
+                                 workspace, workspace_bytes, stream);
+}
+
+int kvmem_paged_attend_fp8_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
+                                const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, int32_t first_position,
+                                float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!p->cfg.fp8_pages || !p->cfg.rope_in_block_keys) {
+        set_error("kvmem_paged_attend_fp8_rope needs a pool with fp8_pages and rope_in_block_keys");
+        return KVMEM_E_STATE;
+    }
+    const int64_t last = (int64_t)first_position + (int64_t)sel_stride * p->cfg.block_tokens;
+    if (first_position < 0 || sel_stride < 1 || last > p->cfg.rope_max_positions) {
+        set_error("compact positions [%d, %lld) outside the rotary table [0, %d)", first_position, (long long)last,
+                  p->cfg.rope_max_positions);
+        return KVMEM_E_INVALID;
+    }
+    return paged_attend_fp8_impl(p, session_first, n_sessions, q, n_q_tokens, sel_ids, sel_stride, n_sel, first_position, scale,
+                                 out, lse, workspace, workspace_bytes, stream);
 }
 
 int kvmem_materialize_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,

@@ -17,6 +17,7 @@
 
 #include "kvmem_internal.cuh"
 #include "kvmem_ptx.cuh"
+#include "kvmem_rope.cuh"
 
 namespace kvmem {
 
@@ -125,8 +126,9 @@ gather_fp8_kernel(GatherF8Args a) {
 __global__ void __launch_bounds__(256)
 append_fp8_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* __restrict__ v_in, uint8_t* __restrict__ pages8,
                   __nv_bfloat16* __restrict__ index_sess, const int32_t* __restrict__ table_sess, int32_t* __restrict__ status,
-                  int b_first, int L, int G, int max_blocks, int max_bps, size_t page_bytes, float k_inv_scale, float v_inv_scale) {
-    __shared__ __align__(16) __nv_bfloat16 ktile[kF8Tile * kF8D];      // the bf16 keys, for the index entry
+                  int b_first, int L, int G, int max_blocks, int max_bps, size_t page_bytes, float k_inv_scale, float v_inv_scale,
+                  const int32_t* __restrict__ pos0_sess, const float2* __restrict__ rope, int rope_positions, int in_block) {
+    __shared__ __align__(16) __nv_bfloat16 ktile[kF8Tile * kF8D];      // the bf16 keys: index entry, rotary steps, then quantised
     __shared__ __align__(16) uint8_t sv[kF8Tile * kF8Pitch];
     const int i = blockIdx.x, lg = blockIdx.y, LG = L * G;
     const int page = table_sess[b_first + i];
@@ -143,10 +145,8 @@ append_fp8_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* _
     for (int it = 0; it < 4; ++it) {
         const int e = threadIdx.x + 256 * it;                          // token e / 16, dims 8 * (e % 16) ..
         const int t = e >> 4, j = e & 15;
-        const uint4 kk = *reinterpret_cast<const uint4*>(ksrc + (size_t)t * row_stride + j * 8);
+        *reinterpret_cast<uint4*>(ktile + (size_t)e * 8) = *reinterpret_cast<const uint4*>(ksrc + (size_t)t * row_stride + j * 8);
         const uint4 vv = *reinterpret_cast<const uint4*>(vsrc + (size_t)t * row_stride + j * 8);
-        *reinterpret_cast<uint4*>(ktile + (size_t)e * 8) = kk;
-        *reinterpret_cast<uint2*>(kdst + (size_t)e * 8) = quant8(kk, k_inv_scale);
         const uint2 q = quant8(vv, v_inv_scale);
         uint32_t* row = reinterpret_cast<uint32_t*>(sv + t * kF8Pitch + j * 8);
         row[0] = q.x; row[1] = q.y;
@@ -166,6 +166,22 @@ append_fp8_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* _
         }
         *reinterpret_cast<uint4*>(vdst + (size_t)dim * kF8Tile + tg * 16) = make_uint4(w[0], w[1], w[2], w[3]);
     }
+    constexpr int half = kF8D / 2;
+    if (pos0_sess) {
+        // the keys still carry RoPE of positions pos0 + t: rotate back (Sec. 4.3); the arithmetic of a rotated element
+        // (fp32 products and sums without fused multiply-add, one rounding to bf16)
+        const int pos0 = pos0_sess[b_first + i];
+        for (int e = threadIdx.x; e < kF8Tile * half; e += 256) {
+            const int t = e / half, x = e % half, pos = pos0 + t;
+            if (pos < 0 || pos >= rope_positions) { atomicExch(status, (int)KVMEM_E_DEVICE_RANGE); continue; }
+            const float2 cs = rope[(size_t)pos * half + x];
+            const float a = __bfloat162float(ktile[t * kF8D + x]), b = __bfloat162float(ktile[t * kF8D + x + half]);
+            ktile[t * kF8D + x] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(a, cs.x), __fmul_rn(b, cs.y)));
+            ktile[t * kF8D + x + half] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(b, cs.x), __fmul_rn(a, cs.y)));
+        }
+        __syncthreads();
+    }
+    // the index entry comes from the raw bf16 keys (position-independent, Sec. 4.3)
     const float inv = 1.0f / (float)kF8Tile;
     __nv_bfloat16* idx_row = index_sess + ((size_t)lg * max_bps + (size_t)(b_first + i)) * kF8D;
     if (threadIdx.x < kF8D) {
@@ -174,17 +190,35 @@ append_fp8_kernel(const __nv_bfloat16* __restrict__ k_in, const __nv_bfloat16* _
         for (int t = 0; t < kF8Tile; ++t) acc = __fadd_rn(acc, __bfloat162float(ktile[(size_t)t * kF8D + c]));
         idx_row[c] = __float2bfloat16_rn(__fmul_rn(acc, inv));
     }
+    if (in_block) {
+        // in-block layout: the page holds the codes of bf16(RoPE(k, t)), t the offset inside the block
+        __syncthreads();
+        for (int e = threadIdx.x; e < kF8Tile * half; e += 256) {
+            const int t = e / half, x = e % half;
+            const float2 cs = rope[(size_t)t * half + x];
+            const float a = __bfloat162float(ktile[t * kF8D + x]), b = __bfloat162float(ktile[t * kF8D + x + half]);
+            ktile[t * kF8D + x] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(a, cs.x), __fmul_rn(b, cs.y)));
+            ktile[t * kF8D + x + half] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(b, cs.x), __fmul_rn(a, cs.y)));
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int e = threadIdx.x + 256 * it;
+        *reinterpret_cast<uint2*>(kdst + (size_t)e * 8) = quant8(*reinterpret_cast<const uint4*>(ktile + (size_t)e * 8), k_inv_scale);
+    }
 }
 
 cudaError_t launch_append_fp8(const kvmem_pool& p, int session, int b_first, int n_blocks, const __nv_bfloat16* k,
-                              const __nv_bfloat16* v, cudaStream_t st) {
+                              const __nv_bfloat16* v, cudaStream_t st, bool derope) {
     const Geometry& g = p.geo;
     const int32_t* table = p.tables + (size_t)session * g.max_bps;
     __nv_bfloat16* index = p.index + (size_t)session * p.lay.index_elems_per_session;
     dim3 grid((unsigned)n_blocks, (unsigned)(g.L * g.G));
     append_fp8_kernel<<<grid, 256, 0, st>>>(k, v, reinterpret_cast<uint8_t*>(p.pages), index, table, p.status_dev, b_first, g.L, g.G,
                                             g.max_blocks, g.max_bps, p.lay.page_elems, 1.0f / p.cfg.fp8_k_scale,
-                                            1.0f / p.cfg.fp8_v_scale);
+                                            1.0f / p.cfg.fp8_v_scale, derope ? p.pos0_dev + (size_t)session * g.max_bps : nullptr,
+                                            p.rope_dev, p.cfg.rope_max_positions, p.cfg.rope_in_block_keys);
     return cudaGetLastError();
 }
 
@@ -238,6 +272,10 @@ constexpr int kF8StageBytes = 2 * kF8TileBytes;
 constexpr int kF8RowsPad = 16;
 constexpr int kF8MergeStride = 136;
 constexpr size_t kF8Smem = (size_t)kF8Stages * kF8StageBytes + 1024;
+constexpr int kF8QrotPitch = kF8D * 2 + 32;      // bytes per rotated query row (f16): 288, so that the consumers' 64-bit reads of 4 rows cover all banks
+constexpr int kF8QrotBytes = kF8RowsPad * kF8QrotPitch;
+constexpr size_t kF8SmemQrot = kF8Smem + (size_t)kF8Stages * kF8QrotBytes;
+constexpr int kF8QrotWarps = 3;                  // query-rotator warps; they take tiles in turn (12 warps in all: the register budget of 9)
 static_assert((size_t)kF8Consumers * kF8RowsPad * kF8MergeStride * sizeof(float) <= (size_t)kF8Stages * kF8StageBytes,
               "the ring is reused for the merge of the consumer warps");
 
@@ -256,6 +294,9 @@ struct AttendF8Args {
     const int32_t* nblocks_dev;  // [max_sessions]
     int session_first, sel_stride, max_bps, max_blocks;
     int lookahead;               // MODE 2: tiles the producer may have in flight that have not landed (0: every stage)
+    // MODE 3: the pages hold the codes of RoPE(k, offset in block); the query is rotated back per tile
+    const float2* rope;          // [rope_positions][64] (cos, sin)
+    int first_position, rope_positions;
 };
 
 // MODE 0: tiles come from the FP8 view (map_k, map_v).
@@ -263,14 +304,18 @@ struct AttendF8Args {
 //         bytes]) through the block table; nothing is written.
 // MODE 2: MODE 1 plus a view-writer warp that stores every landed tile to the FP8 view (map_k, map_v) while the consumers
 //         attend over it: materialize_fp8 + view_attend_fp8 in one pass, 1 byte read + 1 byte written per element.
+// MODE 3: MODE 1 over pages whose keys are the codes of RoPE(k, t), t the offset inside the block: two extra warps, taking
+//         tiles alternately, rotate the 16 query rows back by the tile's compact position p0 (q . R(p0 + t) k = (R(-p0) q) .
+//         RoPE(k, t)), round them to bf16 as the definition says, widen them to f16 and leave them in a small ring of
+//         shared memory from which the consumers fetch their A fragments; no key is touched.
 template <int MODE>
-__global__ void __launch_bounds__(kF8Threads + (MODE == 2 ? 32 : 0), 1)
+__global__ void __launch_bounds__(kF8Threads + (MODE == 2 ? 32 : MODE == 3 ? 32 * kF8QrotWarps : 0), 1)
 attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                         const __grid_constant__ CUtensorMap map_pages, AttendF8Args a) {
-    constexpr bool PAGED = MODE != 0, FUSED = MODE == 2;
+    constexpr bool PAGED = MODE != 0, FUSED = MODE == 2, QROT = MODE == 3;
     pdl_wait();
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ uint64_t full_bar[kF8Stages], empty_bar[kF8Stages];
+    __shared__ uint64_t full_bar[kF8Stages], empty_bar[kF8Stages], q_full[kF8Stages];
     __shared__ float merge_m[kF8Consumers][kF8RowsPad], merge_l[kF8Consumers][kF8RowsPad];
 
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -280,14 +325,14 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int z = s * LG + lg;
     const int l = lg / a.G, g = lg % a.G;
 
-    const int n_blk = max(0, min(a.n_sel[s], MODE == 1 ? a.sel_stride : MODE == 2 ? min(a.sel_stride, a.cap_tokens / kF8Tile) : a.cap_tokens / kF8Tile));
+    const int n_blk = max(0, min(a.n_sel[s], (MODE == 1 || MODE == 3) ? a.sel_stride : MODE == 2 ? min(a.sel_stride, a.cap_tokens / kF8Tile) : a.cap_tokens / kF8Tile));
     const int t0 = (int)((long long)n_blk * split / a.n_splits);
     const int t1 = (int)((long long)n_blk * (split + 1) / a.n_splits);
     const int n_tiles = t1 - t0;
     const int cap_tiles = a.cap_tokens / kF8Tile;
 
     if (tid == 0) {
-        for (int i = 0; i < kF8Stages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kF8Consumers / kF8Groups + (FUSED ? 1 : 0)); }
+        for (int i = 0; i < kF8Stages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kF8Consumers / kF8Groups + (FUSED ? 1 : 0)); ptx::mbar_init(&q_full[i], 1); }
         ptx::fence_mbar_init();
     }
     __syncthreads();
@@ -333,6 +378,61 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
+            }
+        }
+    } else if (QROT && warp > kF8Consumers) {
+        // ---------------- query rotators: Q'(tile) = RoPE^-1(q, p0(tile)), rounded to bf16, stored as f16 ----------------
+        // lane -> 16-byte chunk c = lane & 7 of the low half (dims 8c..8c+7, paired with 64+8c..) of rows (lane >> 3) + 4 i
+        if (n_tiles > 0) {
+            const int c = lane & 7;
+            uint4 raw_lo[4], raw_hi[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = (lane >> 3) + 4 * i;
+                raw_lo[i] = raw_hi[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (row < a.rows) {
+                    const __nv_bfloat16* qr = a.q + ((((size_t)s * a.M + row / a.r) * a.L + l) * a.H + (size_t)g * a.r + row % a.r) * kF8D;
+                    raw_lo[i] = *reinterpret_cast<const uint4*>(qr + c * 8);
+                    raw_hi[i] = *reinterpret_cast<const uint4*>(qr + kF8D / 2 + c * 8);
+                }
+            }
+            unsigned char* qring = stages + (size_t)kF8Stages * kF8StageBytes;
+            auto fetch_row = [&](int it, float4 (&t4)[4]) {
+                int p0 = a.first_position + (t0 + min(it, n_tiles - 1)) * kF8Tile;
+                if (p0 < 0 || p0 >= a.rope_positions) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); p0 = 0; }
+                const float4* cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)p0 * (kF8D / 2) + c * 8);
+#pragma unroll
+                for (int w = 0; w < 4; ++w) t4[w] = __ldg(cs4 + w);
+            };
+            auto to_f16 = [](const uint4& v) -> uint4 {       // 8 bf16 -> 8 f16 (exact for the values a query takes)
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) o[i] = ptx::pack_f16x2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u));
+                return make_uint4(o[0], o[1], o[2], o[3]);
+            };
+            const int it_first = warp - kF8Consumers - 1;
+            float4 t4[4], t4_next[4];
+            fetch_row(it_first, t4_next);
+            for (int it = it_first; it < n_tiles; it += kF8QrotWarps) {
+                const int st = it % kF8Stages;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) t4[w] = t4_next[w];
+                fetch_row(it + kF8QrotWarps, t4_next);
+                bool ok = true;
+                if (it >= kF8Stages) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kF8Stages) & 1) ^ 1));
+                if (!__all_sync(0xffffffffu, ok)) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
+                unsigned char* qb = qring + (size_t)st * kF8QrotBytes;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = (lane >> 3) + 4 * i;
+                    uint4 lo_o, hi_o;
+                    rotate8_cs(raw_lo[i], raw_hi[i], t4, -1.0f, lo_o, hi_o);
+                    *reinterpret_cast<uint4*>(qb + row * kF8QrotPitch + c * 16) = to_f16(lo_o);
+                    *reinterpret_cast<uint4*>(qb + row * kF8QrotPitch + (kF8D / 2) * 2 + c * 16) = to_f16(hi_o);
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&q_full[st]);
             }
         }
     } else if (FUSED && warp == kF8Consumers + 1) {
@@ -383,7 +483,7 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         // dims 16 ks + 4c + {0, 1}, slots {2c+8, 2c+9} hold dims 16 ks + 4c + {2, 3}: what one ldmatrix register of
         // FP8 keys (four consecutive dims of a token) converts to.
         uint32_t qf[8][4];
-        {
+        if (!QROT) {
             const int row_a = lane >> 2, row_b = row_a + 8;
             const __nv_bfloat16* qa = nullptr;
             const __nv_bfloat16* qb = nullptr;
@@ -410,13 +510,25 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
 
         for (int it = grp; it < n_tiles; it += kF8Groups) {
             const int st = it % kF8Stages;
-            const bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kF8Stages) & 1));
+            bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kF8Stages) & 1));
+            if (QROT) arrived = arrived && ptx::mbar_wait(&q_full[st], (uint32_t)((it / kF8Stages) & 1));
             if (!__all_sync(0xffffffffu, arrived)) {
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
             }
             const uint32_t kbase = stage0 + (uint32_t)st * kF8StageBytes;
             const uint32_t vbase = kbase + kF8TileBytes;
+            if (QROT) {
+                // this tile's rotated query: four consecutive dims (two f16x2 words) per k-step for rows lane / 4 and + 8
+                const unsigned char* qb = stages + (size_t)kF8Stages * kF8StageBytes + (size_t)st * kF8QrotBytes;
+                const unsigned char* pa = qb + (lane >> 2) * kF8QrotPitch + 8 * (lane & 3);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint2 va = *reinterpret_cast<const uint2*>(pa + ks * 32);
+                    const uint2 vb = *reinterpret_cast<const uint2*>(pa + 8 * kF8QrotPitch + ks * 32);
+                    qf[ks][0] = va.x; qf[ks][2] = va.y; qf[ks][1] = vb.x; qf[ks][3] = vb.y;
+                }
+            }
 
             // S = Q K^T for this warp's 16 tokens.  Column n of n-tile nt is token 4 (n / 2) + 2 nt + (n % 2) of the 16,
             // so that a lane ends up with the probabilities of four consecutive tokens: the same four an ldmatrix register
@@ -596,7 +708,7 @@ static int f8_choose_splits(int heads, int max_tiles, int sms) {
 cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M, const uint8_t* view_k,
                               const uint8_t* view_v, int view_cap_tokens, const int32_t* n_sel, float scale, float k_scale,
                               float v_scale, float* out, float* lse, void* workspace, cudaStream_t st, const int32_t* sel_ids,
-                              int sel_stride, int session_first) {
+                              int sel_stride, int session_first, int rope_first_position) {
     const Geometry& g = p.geo;
     const int LG = g.L * g.G, heads = n_sessions * LG;
     const bool paged = sel_ids != nullptr;                  // straight over the pages of an FP8 repository ...
@@ -615,6 +727,7 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
         cudaError_t e = cudaFuncSetAttribute(attend_fp8_split_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8SmemQrot);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -641,7 +754,10 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
         if (ctas <= p.sm_count && tiles_per_cta >= 64)
             a.lookahead = std::max(2, std::min(kF8Stages, (int)(9.5 * 1024.0 * 1024.0 / ((double)ctas * kF8StageBytes) + 0.5)));
     }
-    if (fused)
+    a.rope = p.rope_dev; a.first_position = rope_first_position; a.rope_positions = p.cfg.rope_max_positions;
+    if (paged && !fused && rope_first_position >= 0)
+        launch_pdl(attend_fp8_split_kernel<3>, dim3(grid), dim3(kF8Threads + 32 * kF8QrotWarps), kF8SmemQrot, st, map_k, map_v, map_pages, a);
+    else if (fused)
         launch_pdl(attend_fp8_split_kernel<2>, dim3(grid), dim3(kF8Threads + 32), kF8Smem, st, map_k, map_v, map_pages, a);
     else if (paged)
         launch_pdl(attend_fp8_split_kernel<1>, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, map_pages, a);

@@ -143,10 +143,11 @@ cudaError_t launch_gather_fp8(const kvmem_pool& p, int session_first, int n_sess
 cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M, const uint8_t* view_k,
                               const uint8_t* view_v, int view_cap_tokens, const int32_t* n_sel, float scale, float k_scale,
                               float v_scale, float* out, float* lse, void* workspace, cudaStream_t st,
-                              const int32_t* sel_ids = nullptr, int sel_stride = 0, int session_first = 0);
+                              const int32_t* sel_ids = nullptr, int sel_stride = 0, int session_first = 0,
+                              int rope_first_position = -1);
 // FP8 repository (pool created with fp8_pages): quantising append
 cudaError_t launch_append_fp8(const kvmem_pool& p, int session, int b_first, int n_blocks, const __nv_bfloat16* k,
-                              const __nv_bfloat16* v, cudaStream_t st);
+                              const __nv_bfloat16* v, cudaStream_t st, bool derope = false);
 
 // working-set delta (kvmem_delta.cu)
 cudaError_t launch_working_set_delta(const kvmem_pool& p, int n_sessions, const int32_t* prev_ids, const int32_t* n_prev,

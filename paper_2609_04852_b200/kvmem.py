@@ -94,6 +94,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_materialize_attend_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, i32, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_materialize_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, f32, f32, vp]),
         "kvmem_paged_attend_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
+        "kvmem_paged_attend_fp8_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_materialize_attend_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_fp8": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, f32, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
@@ -119,7 +120,8 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_working_set_delta", "kvmem_score", "kvmem_view_cache_bytes", "kvmem_view_cache_layout",
             "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend", "kvmem_paged_attend_rope", "kvmem_topk", "kvmem_score_host_workspace_bytes",
             "kvmem_score_host_staging_bytes", "kvmem_score_host_index", "kvmem_materialize_fp8", "kvmem_view_attend_fp8",
-            "kvmem_materialize_attend_rope", "kvmem_paged_attend_fp8", "kvmem_materialize_attend_fp8")
+            "kvmem_materialize_attend_rope", "kvmem_paged_attend_fp8", "kvmem_materialize_attend_fp8",
+            "kvmem_paged_attend_fp8_rope")
 
 
 def _check(status: int) -> None:
@@ -427,6 +429,17 @@ class Pool:
                                                _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
                                                scale, _dev(out, torch.float32), _dev(lse, torch.float32),
                                                ws.data_ptr(), ws.numel(), _stream()))
+
+    def paged_attend_fp8_rope(self, q: torch.Tensor, sel_ids: torch.Tensor, n_sel: torch.Tensor, out: torch.Tensor,
+                              lse: torch.Tensor, first_position: int = 0, scale: float = 0.0, session_first: int = 0) -> None:
+        """Copy-free, position-consistent attention over an FP8 repository of in-block-rotated keys: the query is rotated
+        back once per block (pool created with fp8_pages and rope_in_block_keys)."""
+        ns, M = q.shape[0], q.shape[1]
+        ws = self.attend_workspace(ns, M)
+        _check(self.lib.kvmem_paged_attend_fp8_rope(self.handle, session_first, ns, _dev(q, torch.bfloat16), M,
+                                                    _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
+                                                    first_position, scale, _dev(out, torch.float32), _dev(lse, torch.float32),
+                                                    ws.data_ptr(), ws.numel(), _stream()))
 
     def materialize_attend_fp8(self, q: torch.Tensor, sel_ids: torch.Tensor, n_sel: torch.Tensor, k8: torch.Tensor,
                                v8t: torch.Tensor, out: torch.Tensor, lse: torch.Tensor, scale: float = 0.0,

@@ -195,3 +195,84 @@ def test_page_formats_are_not_mixed_up():
     assert f8.device_status() == 0 and bf.device_status() == 0
     # half the memory: pages of 1 byte per element
     assert f8.storage.numel() < 0.6 * bf.storage.numel()
+
+
+# ---- FP8 repository of in-block-rotated keys: position-consistent, copy-free, one byte per element ----
+
+@pytest.mark.parametrize("encoded,n_blocks,k,M,first", [(False, 150, 20, 4, 517), (True, 700, 60, 4, 17), (False, 90, 1, 1, 0),
+                                                       (True, 64, 64, 2, 0)])
+def test_fp8_repository_of_in_block_rotated_keys(encoded, n_blocks, k, M, first):
+    """The paper's three mechanisms together (FP8 KV cache, keys encoded at their compact positions, copy-free view):
+    pages hold the codes of bf16(RoPE(k, offset in block)); attention rotates the query back once per block."""
+    from kvmem_harness import bits
+    from kvmem_workloads import kv_blocks, page_table
+    from paper_2609_04852_b200 import Pool
+    spec = SPEC.with_(n_blocks=n_blocks, n_planted=min(8, n_blocks // 4), budget_blocks=k, n_q_tokens=M)
+    dev = torch.device("cuda", 0)
+    theta, window, B, d = 1.0e6, 4096, 64, spec.head_dim
+    k_scale, v_scale = 0.5, 0.25
+    pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, d, B, 1, n_blocks, n_blocks, 0, window, theta,
+                rope_in_block_keys=True, fp8_pages=True, fp8_k_scale=k_scale, fp8_v_scale=v_scale)
+    tab = orc.rope_table(window, d, theta)
+    table = page_table(spec)[0]
+    pos0 = [(37 * b * B) % (window - B) for b in range(n_blocks)]
+    repo = orc.Repository.empty(n_blocks, B, spec.n_layers, spec.n_kv_heads, d)
+    idx = np.zeros((spec.n_layers, spec.n_kv_heads, n_blocks, d), np.uint16)
+    for b0 in range(0, n_blocks, 64):
+        b1 = min(n_blocks, b0 + 64)
+        K, V = kv_blocks(spec, 0, b0, b1, dev)
+        Kb, Vb = bits(K), bits(V)
+        n_tok = (b1 - b0) * B
+        if encoded:      # the generator's keys taken as RoPE-encoded at pos0[b] + t: the append removes that first
+            pool.append_blocks_rope(0, K, V, pos0[b0:b1], table[b0:b1].tolist())
+            tok_pos = np.concatenate([np.arange(pos0[b], pos0[b] + B) for b in range(b0, b1)]).astype(np.int32)
+            raw = orc.rope_rotate(Kb.reshape(n_tok, -1, d), tok_pos, tab, inverse=True).reshape(Kb.shape)
+        else:
+            pool.append_blocks(0, K, V, table[b0:b1].tolist())
+            raw = Kb
+        t_in = (np.arange(n_tok) % B).astype(np.int32)
+        stored = orc.rope_rotate(np.ascontiguousarray(raw.reshape(n_tok, -1, d)), t_in, tab).reshape(Kb.shape)
+        repo.place(stored, Vb, np.ascontiguousarray(table[b0:b1].numpy()))
+        orc.mean_k_index(raw, B, idx, b0)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(pool.index(0)), idx), "the index comes from the raw bf16 keys"
+    ids = _ids(np.random.default_rng(n_blocks + 3), n_blocks, k)
+    cap = k * B
+    sel = torch.from_numpy(ids).view(1, -1).to(dev)
+    n_sel = torch.tensor([k], dtype=torch.int32, device=dev)
+    k8, v8t = pool.new_view_fp8(1, cap)
+    pool.materialize_fp8(sel, n_sel, k8, v8t, k_scale, v_scale)                 # the stored codes, gathered
+    q, qb = queries(spec)
+    out, lse = pool.new_outputs(1, M)
+    pool.paged_attend_fp8_rope(q.to(dev), sel, n_sel, out, lse, first)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    k_inv, v_inv = np.float32(1.0) / np.float32(k_scale), np.float32(1.0) / np.float32(v_scale)
+    rK, rV = orc.gather_fp8(repo, table.numpy(), ids, cap, float(k_inv), float(v_inv))
+    assert np.array_equal(k8.cpu().numpy()[0], rK), "codes of the in-block-rotated keys differ"
+    assert np.array_equal(v8t.cpu().numpy()[0], rV)
+    ref_out, ref_lse = orc.attend_fp8_qrot(qb[0], rK, rV, cap, B, first, tab, k_scale, v_scale)
+    err_o, err_l = np.abs(out.cpu().numpy()[0] - ref_out).max(), np.abs(lse.cpu().numpy()[0] - ref_lse).max()
+    assert err_o <= ATTN_ATOL and err_l <= ATTN_ATOL, (err_o, err_l)
+    if k > 1 and first + 200 + cap <= window:       # the rotation really follows the compact position
+        out2, lse2 = pool.new_outputs(1, M)
+        pool.paged_attend_fp8_rope(q.to(dev), sel, n_sel, out2, lse2, first + 200)
+        torch.cuda.synchronize()
+        ref2, ref_lse2 = orc.attend_fp8_qrot(qb[0], rK, rV, cap, B, first + 200, tab, k_scale, v_scale)
+        assert np.abs(out2.cpu().numpy()[0] - ref2).max() <= ATTN_ATOL and np.abs(lse2.cpu().numpy()[0] - ref_lse2).max() <= ATTN_ATOL
+        assert (lse2 - lse).abs().max().item() > 10 * ATTN_ATOL
+
+
+def test_fp8_rope_reader_needs_both_options():
+    from paper_2609_04852_b200 import KvmemError
+    from paper_2609_04852_b200.kvmem import E_STATE
+    spec = SPEC.with_(n_blocks=16, n_planted=2)
+    dev = torch.device("cuda", 0)
+    f8 = _fp8_pool(spec, 1.0, 1.0)
+    sel = torch.arange(4, dtype=torch.int32, device=dev).view(1, -1)
+    n_sel = torch.tensor([4], dtype=torch.int32, device=dev)
+    q, _ = queries(spec)
+    out, lse = f8.new_outputs(1, spec.n_q_tokens)
+    with pytest.raises(KvmemError) as e:
+        f8.paged_attend_fp8_rope(q.to(dev), sel, n_sel, out, lse, 0)
+    assert e.value.status == E_STATE
