@@ -1008,8 +1008,8 @@ def main():
         args.in_block = True           # codes cannot be re-encoded: the keys carry their in-block rotation, the query is rotated
     elif args.fp8_pages:
         args.fp8 = True
-    if args.in_block and not args.rope:
-        raise SystemExit("--in-block needs --rope")
+    if args.in_block and not (args.rope or args.cache):
+        raise SystemExit("--in-block needs --rope or --cache")
     if args.impl == "reference":
         run_reference(args)
     else:
