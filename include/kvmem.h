@@ -10,7 +10,8 @@
  *     storage, views, outputs and workspaces, are owned by the caller; the library owns only
  *     the opaque handle and its host-side metadata and never allocates device memory.
  *   - All device work is enqueued on the given stream (a cudaStream_t passed as void*) and is
- *     asynchronous unless a call says otherwise.  A pool is not thread-safe.
+ *     asynchronous unless a call says otherwise.  A pool is not thread-safe.  The pool's device must be the calling
+ *     thread's current device in every call that enqueues work (KVMEM_E_STATE otherwise).
  *   - Every call returns a kvmem_status_t.  Argument, state and capacity errors are detected
  *     on the host before anything is enqueued and leave the pool unchanged; kvmem_last_error()
  *     then describes the failure.  Anomalies seen on the device (a block id out of range, a
@@ -128,8 +129,11 @@ int kvmem_pool_create(const kvmem_pool_config_t* cfg /*HOST*/, void* storage /*D
                       kvmem_pool_t** out /*HOST*/);
 int kvmem_pool_destroy(kvmem_pool_t* pool);
 
-/* Forget a session's blocks and return its pages to the free list (host-side, immediate). */
-int kvmem_session_reset(kvmem_pool_t* pool, int32_t session);
+/* Forget a session's blocks and return its pages to the free list.  The host-side bookkeeping changes at once; the
+ * session's block count on the device is cleared on `stream`, so calls enqueued after it on that stream (select, top-k,
+ * attention over its pages) see an empty session: n_sel = 0, nothing read.  Work enqueued earlier that still reads
+ * the session's pages must have been ordered before any append that reuses them (same stream, or an event). */
+int kvmem_session_reset(kvmem_pool_t* pool, int32_t session, void* stream);
 
 /* Blocks appended to a session so far, or a negative status. */
 int32_t kvmem_session_blocks(const kvmem_pool_t* pool, int32_t session);
@@ -145,7 +149,9 @@ int32_t kvmem_session_blocks(const kvmem_pool_t* pool, int32_t session);
  *   phys_ids   HOST int32 [n_blocks] page ids to use, or NULL to take free pages in ascending order
  * On a pool created with rope_in_block_keys, k holds raw keys, the index is built from them, and the
  * page receives RoPE(k, t), t = the token's offset inside its block.
- * Errors: KVMEM_E_CAPACITY (session or pool full), KVMEM_E_STATE (page in use), KVMEM_E_INVALID. */
+ * Errors: KVMEM_E_CAPACITY (session or pool full), KVMEM_E_STATE (page in use), KVMEM_E_INVALID.  The session's block
+ * count on the device is raised only after the kernel that writes the new pages and index rows has been enqueued, so
+ * a KVMEM_E_CUDA from this call leaves the session as it was, on the host and on the device. */
 int kvmem_append_blocks(kvmem_pool_t* pool, int32_t session, const void* k /*DEVICE*/, const void* v /*DEVICE*/,
                         int32_t n_blocks, const int32_t* phys_ids /*HOST*/, void* stream);
 
@@ -237,7 +243,8 @@ int kvmem_select(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, 
  * [j*B, (j+1)*B) of session s are block sel_ids[s][j]'s K and V, fetched through the block table.
  *   view_k, view_v  DEVICE bf16 [n_sessions][n_layers][n_kv_heads][view_cap_tokens][head_dim], 16-byte aligned
  *   n_sel is read on the device; blocks that would not fit view_cap_tokens are skipped and flagged.
- * Tokens past n_sel * B are left untouched. */
+ * An id outside the session (or a table entry outside the pool) is skipped as well: its view tokens are left
+ * untouched and kvmem_device_status reports KVMEM_E_DEVICE_RANGE.  Tokens past n_sel * B are left untouched. */
 int kvmem_materialize(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids /*DEVICE*/,
                       int32_t sel_stride, const int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/,
                       void* view_v /*DEVICE*/, int32_t view_cap_tokens, void* stream);
@@ -266,7 +273,9 @@ int kvmem_view_attend(kvmem_pool_t* pool, int32_t n_sessions, const void* q /*DE
  * block table, written to its place in the view, and attended over while it sits in shared memory.
  * Same arguments, results, limits and error behaviour as the two separate calls; the view it leaves
  * behind is bit-identical to kvmem_materialize's, and out/lse are those of kvmem_view_attend on it.
- * HBM traffic per view byte drops from 2 reads + 1 write to 1 read + 1 write. */
+ * HBM traffic per view byte drops from 2 reads + 1 write to 1 read + 1 write.  (The one difference: an id outside
+ * the session cannot be skipped by a pass that also attends, so page 0 stands in for it, in the view and in out/lse,
+ * and KVMEM_E_DEVICE_RANGE is reported; the results of such a call are to be discarded.) */
 int kvmem_materialize_attend(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
                              int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
                              const int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/, void* view_v /*DEVICE*/,
@@ -444,7 +453,9 @@ int kvmem_view_cache_attend(kvmem_pool_t* pool, const void* q /*DEVICE*/, int32_
  *     a message, and nothing is enqueued.
  *   - The call allocates nothing: no cudaMalloc, cudaFree or allocating library routine.
  *   - The first call on a device looks up the array's device address (the pool's device must be
- *     the current device); make that first call before starting any stream capture.
+ *     the current device); make that first call before starting any stream capture.  The address
+ *     is remembered for the life of the process: the device's primary context must not be reset
+ *     (cudaDeviceReset) while the library is in use.
  *   - All calls in the process share the array and it keeps the previous call's contents.  Nothing
  *     in it needs clearing (every slot that is read is overwritten first), but two calls whose
  *     kernels overlap on the GPU (different streams, or different pools on one device) race on it:
@@ -487,6 +498,15 @@ int kvmem_get_block_table(kvmem_pool_t* pool, int32_t session, const int32_t** t
 /* Synchronise the stream and fetch (and clear) the sticky device status word: KVMEM_OK,
  * KVMEM_E_TIMEOUT or KVMEM_E_DEVICE_RANGE.  Returns KVMEM_OK if the read itself worked. */
 int kvmem_device_status(kvmem_pool_t* pool, int32_t* status /*HOST*/, void* stream);
+
+/* Self-test of the failure path every kernel of this library shares.  (The paper has no counterpart.)  All waits
+ * inside the kernels (for a TMA copy, for another warp) are bounded: after a time limit the kernel records
+ * KVMEM_E_TIMEOUT in the status word and returns, so that a lost copy cannot hang the GPU.  A healthy run never takes
+ * that path; this call does: one warp waits limit_us microseconds (1 .. 100,000) for a barrier nobody arrives at, with
+ * the same wait routine, then sets KVMEM_E_TIMEOUT and returns.  The kernel ends by itself and the context and the pool
+ * stay usable; kvmem_device_status then reports (and clears) KVMEM_E_TIMEOUT.
+ *   waited_ns  DEVICE uint64, may be NULL: receives the time the wait lasted, in nanoseconds */
+int kvmem_selftest_wait_timeout(kvmem_pool_t* pool, uint32_t limit_us, uint64_t* waited_ns /*DEVICE*/, void* stream);
 
 /* Process-wide implementation switches used to compare kernel variants; "gather_mode" and "score_mode"
  * never change results, "chunk_poly" moves scores by a few 1e-6 relative.  (No counterpart in the paper.)  "gather_mode": 1 = bulk asynchronous copies through shared memory

@@ -84,6 +84,19 @@ static bool pool_ok(const kvmem_pool* p) {
     return true;
 }
 
+// pool_ok plus: the pool's device is the calling thread's current device.  Every call that enqueues work launches on the
+// current device with the pool's pointers, so a mismatch is refused on the host instead of faulting on the wrong GPU.
+static bool pool_live(const kvmem_pool* p) {
+    if (!pool_ok(p)) return false;
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device != p->cfg.device) {
+        (void)cudaGetLastError();
+        set_error("the pool lives on device %d but device %d is current", p->cfg.device, device);
+        return false;
+    }
+    return true;
+}
+
 static bool sessions_ok(const kvmem_pool* p, int first, int n) {
     if (first < 0 || n < 1 || first + n > p->cfg.max_sessions) {
         set_error("sessions [%d, %d) outside [0, %d)", first, first + n, p->cfg.max_sessions);
@@ -235,9 +248,12 @@ int kvmem_pool_destroy(kvmem_pool_t* pool) {
     return KVMEM_OK;
 }
 
-int kvmem_session_reset(kvmem_pool_t* p, int32_t session) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+int kvmem_session_reset(kvmem_pool_t* p, int32_t session, void* stream) {
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;
+    // the device's block count first: kernels that size their work from it see an empty session from here on in stream order
+    cudaError_t e = cudaMemsetAsync(p->nblocks_dev + session, 0, 4, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail("clearing the session's block count", e);
     for (int32_t pg : p->sess_pages[session]) p->page_used[pg] = 0;
     p->sess_pages[session].clear();
     p->sess_blocks[session] = 0;
@@ -253,7 +269,7 @@ int32_t kvmem_session_blocks(const kvmem_pool_t* p, int32_t session) {
 
 static int append_impl(kvmem_pool_t* p, int32_t session, const void* k, const void* v, int32_t n_blocks,
                        const int32_t* phys_ids, const int32_t* block_pos0, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session, 1)) return KVMEM_E_INVALID;
     if (n_blocks < 0) { set_error("n_blocks is negative"); return KVMEM_E_INVALID; }
     if (n_blocks == 0) return KVMEM_OK;
@@ -296,8 +312,6 @@ static int append_impl(kvmem_pool_t* p, int32_t session, const void* k, const vo
     cudaError_t e = cudaMemcpyAsync(table + have, ids.data(), (size_t)n_blocks * 4, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail("block table upload", e);
     const int32_t total = have + n_blocks;
-    e = cudaMemcpyAsync(p->nblocks_dev + session, &total, 4, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) return cuda_fail("block count upload", e);
     if (block_pos0) {
         e = cudaMemcpyAsync(p->pos0_dev + (size_t)session * p->cfg.max_blocks_per_session + have, block_pos0,
                             (size_t)n_blocks * 4, cudaMemcpyHostToDevice, st);
@@ -306,6 +320,9 @@ static int append_impl(kvmem_pool_t* p, int32_t session, const void* k, const vo
     e = p->cfg.fp8_pages ? launch_append_fp8(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st, block_pos0 != nullptr)
                          : launch_append(*p, session, have, n_blocks, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, st, block_pos0 != nullptr);
     if (e != cudaSuccess) return cuda_fail("append kernel launch", e);
+    // the device's block count last: it never covers index rows whose kernel was not enqueued
+    e = cudaMemcpyAsync(p->nblocks_dev + session, &total, 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail("block count upload", e);
     for (int32_t pg : ids) { p->page_used[pg] = 1; p->sess_pages[session].push_back(pg); }
     if (!phys_ids) p->free_hint = ids.back() + 1;
     p->sess_blocks[session] = total;
@@ -325,7 +342,7 @@ int kvmem_append_blocks_rope(kvmem_pool_t* p, int32_t session, const void* k_rop
 
 int kvmem_rope_rotate(kvmem_pool_t* p, const void* x, void* y, int64_t n_rows, int32_t n_vec, const int32_t* positions,
                       int32_t inverse, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
     if (!x || !y || !positions || !aligned(x, 16) || !aligned(y, 16) || n_rows < 0 || n_vec < 1) {
         set_error("kvmem_rope_rotate: null or misaligned pointer, or bad sizes");
@@ -341,7 +358,7 @@ int kvmem_rope_rotate(kvmem_pool_t* p, const void* x, void* y, int64_t n_rows, i
 int kvmem_materialize_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids,
                            int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v, int32_t view_cap_tokens,
                            int32_t first_position, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
     if (!sel_ids || !n_sel || !view_k || !view_v || !aligned(view_k, 16) || !aligned(view_v, 16)) {
@@ -401,7 +418,7 @@ static int score_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions
 
 int kvmem_score(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens, float* scores,
                 void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!scores) { set_error("scores is null"); return KVMEM_E_INVALID; }
     float* sc = nullptr;
@@ -434,7 +451,7 @@ size_t kvmem_score_host_staging_bytes(const kvmem_pool_t* p, int32_t tile_blocks
 int kvmem_score_host_index(kvmem_pool_t* p, const void* index_host, int32_t n_blocks, int32_t index_stride_blocks, const void* q,
                            int32_t n_q_tokens, int32_t tile_blocks, float* scores, void* staging, size_t staging_bytes,
                            void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!host_score_args_ok(p, n_blocks, n_q_tokens, tile_blocks)) return KVMEM_E_INVALID;
     if (!index_host || !q || !scores || !staging || !workspace || !aligned(index_host, 16) || !aligned(q, 16) ||
         !aligned(staging, 256) || !aligned(workspace, 256)) {
@@ -454,7 +471,7 @@ int kvmem_score_host_index(kvmem_pool_t* p, const void* index_host, int32_t n_bl
 
 int kvmem_topk(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const float* scores, int32_t scores_stride,
                const kvmem_select_params_t* prm, int32_t* sel_ids, int32_t sel_stride, int32_t* n_sel, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!scores || !prm || !sel_ids || !n_sel) { set_error("kvmem_topk: null pointer"); return KVMEM_E_INVALID; }
     if (prm->n_sink_blocks < 0 || prm->n_recent_blocks < 0) { set_error("sink/recent counts must be non-negative"); return KVMEM_E_INVALID; }
@@ -474,7 +491,7 @@ int kvmem_topk(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const
 int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
                  const kvmem_select_params_t* prm, int32_t* sel_ids, int32_t sel_stride, int32_t* n_sel, float* scores,
                  void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!prm || !sel_ids || !n_sel) { set_error("kvmem_select: null pointer"); return KVMEM_E_INVALID; }
     if (prm->n_sink_blocks < 0 || prm->n_recent_blocks < 0) { set_error("sink/recent counts must be non-negative"); return KVMEM_E_INVALID; }
@@ -494,7 +511,7 @@ int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, con
 int kvmem_materialize(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids,
                       int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v, int32_t view_cap_tokens,
                       void* stream) {
-    if (!pool_ok(p) || !pages_are(p, false, "kvmem_materialize")) return KVMEM_E_STATE;
+    if (!pool_live(p) || !pages_are(p, false, "kvmem_materialize")) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!sel_ids || !n_sel || !view_k || !view_v || !aligned(view_k, 16) || !aligned(view_v, 16)) {
         set_error("kvmem_materialize: null or misaligned pointer");
@@ -513,7 +530,7 @@ int kvmem_materialize(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions
 int kvmem_view_attend(kvmem_pool_t* p, int32_t n_sessions, const void* q, int32_t n_q_tokens, const void* view_k,
                       const void* view_v, int32_t view_cap_tokens, const int32_t* n_sel, float scale, float* out,
                       float* lse, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (n_sessions < 1) { set_error("n_sessions must be positive"); return KVMEM_E_INVALID; }
     if (!q || !view_k || !view_v || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(view_k, 128) ||
         !aligned(view_v, 128) || !aligned(workspace, 256) || !aligned(out, 16)) {
@@ -571,7 +588,7 @@ int kvmem_recall_step_host(kvmem_pool_t* p, int32_t session_first, int32_t n_ses
                            int32_t* n_sel, void* view_k, void* view_v, int32_t view_cap_tokens, float scale,
                            float* out_host, float* lse_host, void* staging, size_t staging_bytes, void* select_ws,
                            size_t select_ws_bytes, void* attend_ws, size_t attend_ws_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q_host || !out_host || !lse_host || !staging || !aligned(staging, 256) || n_q_tokens < 1) {
         set_error("kvmem_recall_step_host: null or misaligned pointer");
@@ -634,7 +651,7 @@ static int materialize_attend_impl(kvmem_pool_t* p, int32_t session_first, int32
                                    const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v,
                                    int32_t view_cap_tokens, int32_t rope_first_position, float scale, float* out, float* lse,
                                    void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p) || !pages_are(p, false, "kvmem_materialize_attend")) return KVMEM_E_STATE;
+    if (!pool_live(p) || !pages_are(p, false, "kvmem_materialize_attend")) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q || !sel_ids || !n_sel || !view_k || !view_v || !out || !lse || !workspace || !aligned(q, 16) ||
         !aligned(view_k, 128) || !aligned(view_v, 128) || !aligned(workspace, 256) || !aligned(out, 16)) {
@@ -677,7 +694,7 @@ int kvmem_materialize_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_
                                   const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v,
                                   int32_t view_cap_tokens, int32_t first_position, float scale, float* out, float* lse,
                                   void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
     if (sel_stride < 1 || view_cap_tokens < 1) { set_error("sel_stride and view_cap_tokens must be positive"); return KVMEM_E_INVALID; }
     const int64_t last = (int64_t)first_position + std::min<int64_t>((int64_t)sel_stride * p->cfg.block_tokens, view_cap_tokens);
@@ -700,7 +717,7 @@ int kvmem_materialize_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_
 static int paged_attend_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
                              const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, int32_t rope_first_position,
                              float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p) || !pages_are(p, false, "kvmem_paged_attend")) return KVMEM_E_STATE;
+    if (!pool_live(p) || !pages_are(p, false, "kvmem_paged_attend")) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q || !sel_ids || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(workspace, 256) || !aligned(out, 16)) {
         set_error("kvmem_paged_attend: null or misaligned pointer");
@@ -739,7 +756,7 @@ int kvmem_paged_attend(kvmem_pool_t* p, int32_t session_first, int32_t n_session
 int kvmem_paged_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
                             const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, int32_t first_position,
                             float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
     const int64_t last = (int64_t)first_position + (int64_t)sel_stride * p->cfg.block_tokens;
     if (first_position < 0 || sel_stride < 1 || last > p->cfg.rope_max_positions) {
@@ -754,7 +771,7 @@ int kvmem_paged_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_se
 int kvmem_working_set_delta(kvmem_pool_t* p, int32_t n_sessions, const int32_t* prev_ids, const int32_t* n_prev,
                             const int32_t* next_ids, const int32_t* n_next, int32_t stride, int32_t* retained,
                             int32_t* incoming, int32_t* outgoing, int32_t* counts, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (n_sessions < 1 || stride < 1 || !prev_ids || !n_prev || !next_ids || !n_next || !retained || !incoming || !outgoing ||
         !counts) {
         set_error("kvmem_working_set_delta: null pointer or non-positive size");
@@ -769,7 +786,7 @@ int kvmem_working_set_delta(kvmem_pool_t* p, int32_t n_sessions, const int32_t* 
 // ---- FP8 execution view ----
 
 static int fp8_common_ok(kvmem_pool_t* p, int32_t view_cap_tokens, float k_scale, float v_scale, const char* who) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
         set_error("%s: the FP8 view kernels are built for head_dim 128 and 64-token blocks", who);
         return KVMEM_E_UNSUPPORTED;
@@ -832,7 +849,7 @@ int kvmem_view_attend_fp8(kvmem_pool_t* p, int32_t n_sessions, const void* q, in
 static int paged_attend_fp8_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
                                  const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, int32_t rope_first_position,
                                  float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p) || !pages_are(p, true, "kvmem_paged_attend_fp8")) return KVMEM_E_STATE;
+    if (!pool_live(p) || !pages_are(p, true, "kvmem_paged_attend_fp8")) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q || !sel_ids || !n_sel || !out || !lse || !workspace || !aligned(q, 16) || !aligned(workspace, 256) || !aligned(out, 16)) {
         set_error("kvmem_paged_attend_fp8: null or misaligned pointer");
@@ -865,7 +882,7 @@ int kvmem_paged_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_ses
 int kvmem_paged_attend_fp8_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
                                 const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, int32_t first_position,
                                 float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!p->cfg.fp8_pages || !p->cfg.rope_in_block_keys) {
         set_error("kvmem_paged_attend_fp8_rope needs a pool with fp8_pages and rope_in_block_keys");
         return KVMEM_E_STATE;
@@ -884,7 +901,7 @@ int kvmem_materialize_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t
                                  const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k8, void* view_v8t,
                                  int32_t view_cap_tokens, float scale, float* out, float* lse, void* workspace,
                                  size_t workspace_bytes, void* stream) {
-    if (!pool_ok(p) || !pages_are(p, true, "kvmem_materialize_attend_fp8")) return KVMEM_E_STATE;
+    if (!pool_live(p) || !pages_are(p, true, "kvmem_materialize_attend_fp8")) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!q || !sel_ids || !n_sel || !view_k8 || !view_v8t || !out || !lse || !workspace || !aligned(q, 16) || !aligned(view_k8, 128) ||
         !aligned(view_v8t, 128) || !aligned(workspace, 256) || !aligned(out, 16)) {
@@ -912,7 +929,7 @@ int kvmem_materialize_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t
 // ---- execution cache: working-set reuse with bounded delta re-RoPE ----
 
 static int cache_ok(kvmem_pool_t* p, const void* cache, size_t cache_bytes, int32_t cap_blocks, const char* who) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (p->cfg.rope_max_positions <= 0) { set_error("%s: the pool was created without rotary support", who); return KVMEM_E_STATE; }
     if (cap_blocks < 1 || cap_blocks > 32768) { set_error("%s: cap_blocks must be in [1, 32768]", who); return KVMEM_E_INVALID; }
     if (!cache || !aligned(cache, 256)) { set_error("%s: cache is null or not 256-byte aligned", who); return KVMEM_E_INVALID; }
@@ -1009,7 +1026,7 @@ int kvmem_get_block_table(kvmem_pool_t* p, int32_t session, const int32_t** tabl
 }
 
 int kvmem_device_status(kvmem_pool_t* p, int32_t* status, void* stream) {
-    if (!pool_ok(p)) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
     if (!status) { set_error("status is null"); return KVMEM_E_INVALID; }
     cudaStream_t st = (cudaStream_t)stream;
     int32_t word = 0;

@@ -672,8 +672,8 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         return cudaErrorInvalidValue;
     }
     if (!fused) map_pages = map_k;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_done;
+    if (attr_done.pending(p.cfg.device)) {
         cudaError_t e = cudaFuncSetAttribute(attend_split_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
@@ -686,7 +686,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.mark(p.cfg.device);
     }
     AttendPlan plan = plan_attend(p.cfg, n_sessions, M, p.sm_count);
     AttendArgs a{};

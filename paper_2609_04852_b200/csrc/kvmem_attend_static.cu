@@ -24,7 +24,6 @@ constexpr size_t kStaticAttendBytes = (size_t)kStaticAttendMaxHeads * 64 * 16 * 
 
 static __device__ __align__(256) unsigned char g_attend_scratch[kStaticAttendBytes];
 
-constexpr int kMaxDevices = 64;
 static void* g_scratch_ptr[kMaxDevices] = {};
 static std::mutex g_scratch_mutex;
 
@@ -49,8 +48,9 @@ extern "C" int kvmem_view_attend_static(kvmem_pool_t* pool, int32_t n_sessions, 
                                         const void* view_k, const void* view_v, int32_t view_cap_tokens,
                                         const int32_t* n_sel, float scale, float* out, float* lse, void* stream) {
     if (!pool || pool->magic != kMagic) { set_error("pool handle is null or stale"); return KVMEM_E_STATE; }
+    if (n_sessions < 1) { set_error("n_sessions must be positive"); return KVMEM_E_INVALID; }
     const long long heads = (long long)n_sessions * pool->cfg.n_layers * pool->cfg.n_kv_heads;
-    if (n_sessions < 1 || heads > kStaticAttendMaxHeads) {
+    if (heads > kStaticAttendMaxHeads) {
         set_error("kvmem_view_attend_static handles at most %d (session, layer, KV head) triples per call, got %lld; "
                   "use kvmem_view_attend with a caller workspace for more",
                   kStaticAttendMaxHeads, heads);

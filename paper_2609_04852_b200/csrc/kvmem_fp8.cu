@@ -722,14 +722,14 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
         return cudaErrorInvalidValue;
     }
     if (!paged) map_pages = map_k;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_done;
+    if (attr_done.pending(p.cfg.device)) {
         cudaError_t e = cudaFuncSetAttribute(attend_fp8_split_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8SmemQrot);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.mark(p.cfg.device);
     }
     AttendPlan plan = plan_attend(p.cfg, n_sessions, M, p.sm_count);
     AttendF8Args a{};

@@ -103,28 +103,36 @@ gather_bulk_kernel(GatherArgs a) {
     };
 
     bool ok = true;
+    uint32_t skip_mask = 0;                     // lane 0: stages whose tile belongs to a flagged id (nothing loaded, nothing stored)
     auto issue_load = [&](int i) {              // tile i of this CTA into stage i % STAGES
         const long long tile = t_begin + i;
         const int page = page_of((int)(tile / per_block));
         if (lane == 0) {
             const int st = i % STAGES;
-            const __nv_bfloat16* src;
-            __nv_bfloat16* dst;
-            // a flagged lookup copies page 0 instead of faulting; the status word reports it
-            tile_addresses(a, s, tile, page < 0 ? 0 : page, src, dst);
-            ptx::mbar_expect_tx(&full[st], tile_bytes);
-            ptx::bulk_g2s(smem + (size_t)st * tile_bytes, src, tile_bytes, &full[st]);
+            if (page < 0) {                     // flagged lookup: the tile is skipped, the status word reports it
+                skip_mask |= 1u << st;
+            } else {
+                const __nv_bfloat16* src;
+                __nv_bfloat16* dst;
+                tile_addresses(a, s, tile, page, src, dst);
+                ptx::mbar_expect_tx(&full[st], tile_bytes);
+                ptx::bulk_g2s(smem + (size_t)st * tile_bytes, src, tile_bytes, &full[st]);
+            }
         }
     };
 
     const int prologue = min(STAGES - 1, n_mine);
     for (int i = 0; i < prologue; ++i) issue_load(i);
 
+    uint32_t phase_mask = 0;                    // lane 0: parity of the next completion of each stage's barrier
     for (int i = 0; i < n_mine; ++i) {
         const int st = i % STAGES;
         if (lane == 0) {
-            ok = ptx::mbar_wait(&full[st], (uint32_t)((i / STAGES) & 1));
-            if (ok) {
+            if (skip_mask & (1u << st)) {
+                skip_mask &= ~(1u << st);
+                ptx::bulk_commit();             // an empty group keeps the group count of the refill logic in step
+            } else if ((ok = ptx::mbar_wait(&full[st], (phase_mask >> st) & 1u))) {
+                phase_mask ^= 1u << st;
                 const __nv_bfloat16* src;
                 __nv_bfloat16* dst;
                 tile_addresses(a, s, t_begin + i, 0, src, dst);
@@ -198,12 +206,12 @@ cudaError_t launch_gather(const kvmem_pool& p, int session_first, int n_sessions
     if (g_gather_mode == 1 && tile_bytes % 16 == 0 && tile_bytes * 4 <= 200 * 1024) {
         constexpr int STAGES = 4;
         const size_t smem = tile_bytes * STAGES;
-        static bool attr_done = false;
-        if (!attr_done) {
+        static PerDeviceOnce attr_done;
+        if (attr_done.pending(p.cfg.device)) {
             cudaError_t e = cudaFuncSetAttribute(gather_bulk_kernel<STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  200 * 1024);
             if (e != cudaSuccess) return e;
-            attr_done = true;
+            attr_done.mark(p.cfg.device);
         }
         // as many single-warp CTAs as fit the shared memory of every SM, split evenly over the sessions
         const int per_sm = std::max(1, (int)((220 * 1024) / (smem + 1024)));

@@ -37,6 +37,15 @@ struct Geometry {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// A kernel attribute (cudaFuncSetAttribute) belongs to one device: launchers that opt in to large dynamic shared
+// memory do it once per device ordinal, keyed by the pool's device.
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+    bool done[kMaxDevices] = {};
+    bool pending(int device) const { return device < 0 || device >= kMaxDevices || !done[device]; }
+    void mark(int device) { if (device >= 0 && device < kMaxDevices) done[device] = true; }
+};
+
 bool config_valid(const kvmem_pool_config_t& c, const char** why);
 Layout make_layout(const kvmem_pool_config_t& c);
 

@@ -46,18 +46,19 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 }
 // Bounded wait: gives up after about kWaitLimitNs of wall time (checked every 256 attempts) or
 // kSpinLimit attempts, whichever comes first.  false = gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t* bar, uint32_t parity, uint64_t limit_ns) {
     uint64_t t0 = 0;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 255u) == 255u) {
             const uint64_t now = globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) return false;
+            else if (now - t0 > limit_ns) return false;
         }
     }
     return false;
 }
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) { return mbar_wait_limited(bar, parity, kWaitLimitNs); }
 
 // Same bound, for waits that are expected to be long (a control warp waiting for the warps that do the
 // arithmetic): every attempt may stay suspended in hardware for up to kSuspendNs, so the waiting warp

@@ -502,11 +502,11 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     if (g_score_mode == 1 && index_rows <= 0x7fffffffll) {     // TMA row coordinates are 32-bit
         CUtensorMap map_idx;
         if (!make_score_index_map(&map_idx, p.index, index_rows)) return cudaErrorInvalidValue;
-        static bool attr_done = false;
-        if (!attr_done) {
+        static PerDeviceOnce attr_done;
+        if (attr_done.pending(p.cfg.device)) {
             e = cudaFuncSetAttribute(score_logits_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem + 1024));
             if (e != cudaSuccess) return e;
-            attr_done = true;
+            attr_done.mark(p.cfg.device);
         }
         launch_pdl(score_logits_mma_kernel, dim3(grid), dim3(kScoreThreads), smem + 1024, st, 
             map_idx, q, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, ws.logits, ws.partials, ws.rows,
@@ -514,11 +514,11 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     } else {
 #define KVMEM_SCORE_LAUNCH(RP)                                                                                         \
     do {                                                                                                               \
-        static bool attr_done = false;                                                                                 \
-        if (!attr_done) {                                                                                              \
+        static PerDeviceOnce attr_done;                                                                                 \
+        if (attr_done.pending(p.cfg.device)) {                                                                                              \
             e = cudaFuncSetAttribute(score_logits_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
             if (e != cudaSuccess) return e;                                                                            \
-            attr_done = true;                                                                                          \
+            attr_done.mark(p.cfg.device);                                                                                          \
         }                                                                                                              \
         launch_pdl(score_logits_kernel<RP>, dim3(grid), dim3(kScoreThreads), smem, st,                                                     \
             q, p.index, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, p.lay.index_elems_per_session,      \
@@ -609,12 +609,12 @@ cudaError_t launch_score_host_index(kvmem_pool& p, const __nv_bfloat16* index_ho
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p.ev_start, cudaEventDisableTiming);
         if (e != cudaSuccess) return e;
     }
-    static bool attr_done = false;
+    static PerDeviceOnce attr_done;
     const size_t smem = (size_t)kScoreStages * kChunk * 256 + 1024;
-    if (!attr_done) {
+    if (attr_done.pending(p.cfg.device)) {
         e = cudaFuncSetAttribute(score_logits_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.mark(p.cfg.device);
     }
     const size_t buf_bytes = align_up((size_t)LG * tile_blocks * 256, 256);
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)g.d);

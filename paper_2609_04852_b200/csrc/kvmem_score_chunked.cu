@@ -756,13 +756,13 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
     cudaError_t e = cudaSuccess;
 #define KVMEM_CHUNK_PASSES(POLY)                                                                                              \
     do {                                                                                                                      \
-        static bool attr_done = false;                                                                                        \
-        if (!attr_done) {                                                                                                     \
+        static PerDeviceOnce attr_done;                                                                                        \
+        if (attr_done.pending(p.cfg.device)) {                                                                                                     \
             e = cudaFuncSetAttribute(score_chunk_rowstat_kernel<POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCkSmem); \
             if (e == cudaSuccess)                                                                                             \
                 e = cudaFuncSetAttribute(score_chunk_colsum_kernel<POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCkSmem2); \
             if (e != cudaSuccess) return e;                                                                                   \
-            attr_done = true;                                                                                                 \
+            attr_done.mark(p.cfg.device);                                                                                                 \
         }                                                                                                                     \
         launch_pdl(score_chunk_rowstat_kernel<POLY>, dim3(grid1), dim3(kCkThreads), kCkSmem, st, q_panel, idx_tile, a);                           \
         e = cudaGetLastError();                                                                                               \

@@ -662,21 +662,21 @@ cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, 
     for (int s = session_first; s < session_first + n_sessions; ++s) max_nb = std::max(max_nb, p.sess_blocks[s]);
     const size_t smem = (size_t)kTopkThreads * kStagePitch * sizeof(unsigned int);
     static_assert(kTopkThreads * kStagePitch >= kTopkTile, "the staging buffer doubles as the output buffer of one sweep");
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_done;
+    if (attr_done.pending(p.cfg.device)) {
         cudaError_t e = cudaFuncSetAttribute(topk_kernel<true, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_kernel<false, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.mark(p.cfg.device);
     }
     const int max_tiles = (max_nb + kTopkTile - 1) / kTopkTile;
     if (max_nb > kTopkTile && g_topk_cluster && max_tiles <= kTopkCluster * kTopkMaxOwnTiles) {
         // long sessions: one cluster of 8 CTAs per session
-        static bool cattr_done = false;
-        if (!cattr_done) {
+        static PerDeviceOnce cattr_done;
+        if (cattr_done.pending(p.cfg.device)) {
             cudaError_t e = cudaFuncSetAttribute(topk_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            cattr_done = true;
+            cattr_done.mark(p.cfg.device);
         }
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)(kTopkCluster * n_sessions));

@@ -64,7 +64,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_last_error": (C.c_char_p, []),
         "kvmem_pool_create": (C.c_int, [cfgp, vp, sz, C.POINTER(vp)]),
         "kvmem_pool_destroy": (C.c_int, [vp]),
-        "kvmem_session_reset": (C.c_int, [vp, i32]),
+        "kvmem_session_reset": (C.c_int, [vp, i32, vp]),
         "kvmem_session_blocks": (i32, [vp, i32]),
         "kvmem_append_blocks": (C.c_int, [vp, i32, vp, vp, i32, C.POINTER(i32), vp]),
         "kvmem_score": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, sz, vp]),
@@ -98,6 +98,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_materialize_attend_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_fp8": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, f32, f32, vp, vp, vp, sz, vp]),
         "kvmem_view_attend_static": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp]),
+        "kvmem_selftest_wait_timeout": (C.c_int, [vp, C.c_uint32, vp, vp]),
         "kvmem_step_staging_bytes": (sz, [cfgp, i32, i32]),
         "kvmem_recall_step_host": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, i32, f32, vp, vp,
                                              vp, sz, vp, sz, vp, sz, vp]),
@@ -121,7 +122,7 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend", "kvmem_paged_attend_rope", "kvmem_topk", "kvmem_score_host_workspace_bytes",
             "kvmem_score_host_staging_bytes", "kvmem_score_host_index", "kvmem_materialize_fp8", "kvmem_view_attend_fp8",
             "kvmem_materialize_attend_rope", "kvmem_paged_attend_fp8", "kvmem_materialize_attend_fp8",
-            "kvmem_paged_attend_fp8_rope")
+            "kvmem_paged_attend_fp8_rope", "kvmem_selftest_wait_timeout")
 
 
 def _check(status: int) -> None:
@@ -195,7 +196,7 @@ class Pool:
 
     # ---- repository
     def session_reset(self, session: int) -> None:
-        _check(self.lib.kvmem_session_reset(self.handle, session))
+        _check(self.lib.kvmem_session_reset(self.handle, session, _stream()))
 
     def session_blocks(self, session: int) -> int:
         n = self.lib.kvmem_session_blocks(self.handle, session)
@@ -513,6 +514,13 @@ class Pool:
         _check(self.lib.kvmem_get_block_table(self.handle, session, C.byref(ptr), C.byref(n)))
         off = ptr.value - self.storage.data_ptr()
         return self.storage[off:off + 4 * n.value].view(torch.int32).clone()
+
+    def selftest_wait_timeout(self, limit_us: int = 1000) -> int:
+        """Run the kernels' bounded wait to its limit on a barrier nobody arrives at; returns the nanoseconds it lasted.
+        The status word then holds E_TIMEOUT until device_status() reads it."""
+        waited = torch.zeros(1, dtype=torch.int64, device=self.device)
+        _check(self.lib.kvmem_selftest_wait_timeout(self.handle, limit_us, waited.data_ptr(), _stream()))
+        return int(waited.item())
 
     def device_status(self) -> int:
         st = C.c_int32()

@@ -11,7 +11,7 @@ from typing import List, Optional
 import numpy as np
 import torch
 
-from kvmem_workloads import WorkloadSpec, kv_blocks, make_queries, page_table
+from kvmem_workloads import WorkloadSpec, kv_blocks, make_queries, page_table, select_params
 from oracle import kvmem_oracle as orc
 
 
@@ -67,6 +67,47 @@ def fill_pool(spec: WorkloadSpec, n_blocks: Optional[List[int]] = None, extra_pa
     return pool
 
 
+class Guards:
+    """Output buffers with canary bytes in front of and behind them.
+
+    Every buffer a GPU entry point writes (ids, counts, scores, views, outputs) is cut out of a larger allocation
+    whose surroundings hold a byte pattern; ``check()`` after the call fails if any entry point wrote outside
+    what it was given.  The payload starts 256 bytes into a fresh torch allocation, so it keeps the 256-byte
+    alignment the views and workspaces need; the rear canary starts at the payload's last byte + 1."""
+    PAD = 256
+    BYTE = 0xA5
+
+    def __init__(self, device):
+        self.device = device
+        self.items = []
+
+    def empty(self, shape, dtype, fill=0) -> torch.Tensor:
+        n = int(np.prod(shape)) * torch.empty(0, dtype=dtype).element_size()
+        buf = torch.full((self.PAD + n + self.PAD,), self.BYTE, dtype=torch.uint8, device=self.device)
+        t = buf[self.PAD:self.PAD + n].view(dtype).view(*shape)
+        if fill is not None:
+            t.fill_(fill)
+        self.items.append((buf, n))
+        return t
+
+    def view(self, pool, n_sessions: int, cap_tokens: int):
+        from paper_2609_04852_b200.kvmem import View
+        c = pool.cfg
+        shape = (n_sessions, c.n_layers, c.n_kv_heads, cap_tokens, c.head_dim)
+        return View(self.empty(shape, torch.bfloat16), self.empty(shape, torch.bfloat16), cap_tokens)
+
+    def outputs(self, pool, n_sessions: int, n_q_tokens: int):
+        c = pool.cfg
+        return (self.empty((n_sessions, n_q_tokens, c.n_layers, c.n_q_heads, c.head_dim), torch.float32),
+                self.empty((n_sessions, n_q_tokens, c.n_layers, c.n_q_heads), torch.float32))
+
+    def check(self) -> None:
+        for i, (buf, n) in enumerate(self.items):
+            front, back = buf[:self.PAD], buf[self.PAD + n:]
+            assert bool((front == self.BYTE).all()) and bool((back == self.BYTE).all()), \
+                f"guard bytes around output buffer {i} ({n} bytes) were overwritten"
+
+
 def queries(spec: WorkloadSpec, qset: int = 0):
     q = make_queries(spec, qset)
     return q, bits(q)
@@ -115,3 +156,70 @@ def check_selection(sel_gpu: np.ndarray, R_ref: np.ndarray, sel_ref: np.ndarray,
     assert np.all(in_gpu[must]), "a block clearly above the boundary was not selected"
     assert not np.any(in_gpu[must_not]), "a block clearly below the boundary was selected"
     return "band"
+
+
+def full_step(spec: WorkloadSpec, qsets=(0,), gap_forced_budget=None, n_sink=0, n_recent=0):
+    """One whole recall step per query set, every stage against the oracle on the same bytes: index bit-exact,
+    scores within SCORE_RTOL, ids exact or by the band rule, gathered view bit-exact, attention within ATTN_ATOL.
+    The fused pass (what the benchmark times) and the copy-free pass must reproduce the view and the results of
+    the separate calls bit for bit.  Every output buffer sits between guard bytes.  Returns the selection modes."""
+    from paper_2609_04852_b200 import SelectParams, budget_blocks
+    dev = torch.device("cuda", 0)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec, gen_device=dev)
+    prm_d = select_params(spec)
+    prm_d["n_sink_blocks"], prm_d["n_recent_blocks"] = n_sink, n_recent
+    if gap_forced_budget is not None:
+        prm_d["budget_blocks"] = gap_forced_budget
+    prm = SelectParams(**prm_d)
+    ns, B, M = spec.n_sessions, spec.block_tokens, spec.n_q_tokens
+    k = budget_blocks(prm, B, spec.n_blocks)
+    fast = B == 64                      # the passes that read pages through the block table
+    guards = Guards(dev)
+    sel = guards.empty((ns, k), torch.int32)
+    n_sel = guards.empty((ns,), torch.int32)
+    scores = guards.empty((ns, spec.n_blocks), torch.float32)
+    view = guards.view(pool, ns, k * B)
+    out, lse = guards.outputs(pool, ns, M)
+    view2 = guards.view(pool, ns, k * B) if fast else None
+    out2, lse2 = guards.outputs(pool, ns, M)
+    out3, lse3 = guards.outputs(pool, ns, M)
+    for s in range(ns):
+        assert np.array_equal(bits(pool.index(s)), osess[s].idx), "Mean-K index differs"
+    modes = []
+    for qset in qsets:
+        q, qb = queries(spec, qset)
+        qd = q.to(dev)
+        pool.select(qd, prm, sel, n_sel, scores)
+        pool.materialize(sel, n_sel, view)
+        if spec.attend:
+            pool.view_attend(qd, view, n_sel, out, lse)
+            if fast:
+                view2.k.zero_(), view2.v.zero_()
+                pool.materialize_attend(qd, sel, n_sel, view2, out2, lse2)
+                pool.paged_attend(qd, sel, n_sel, out3, lse3)
+        torch.cuda.synchronize()
+        assert pool.device_status() == 0
+        guards.check()
+        if spec.attend and fast:
+            assert torch.equal(view.k, view2.k) and torch.equal(view.v, view2.v), "fused pass left a different view"
+            assert torch.equal(out, out2) and torch.equal(lse, lse2), "fused pass: different results"
+            assert torch.equal(out, out3) and torch.equal(lse, lse3), "copy-free pass: different results"
+        sel_h, n_h, sc_h = sel.cpu().numpy(), n_sel.cpu().numpy(), scores.cpu().numpy()
+        out_h, lse_h = out.cpu().numpy(), lse.cpu().numpy()
+        for s in range(ns):
+            R, _ = orc.block_scores(qb[s], osess[s].idx, spec.n_blocks)
+            ref_sel = orc.select(R, B, prm_d["budget_blocks"], prm_d["max_view_tokens"], 0, n_sink, n_recent)
+            check_scores(sc_h[s], R, M)
+            sel_gpu = sel_h[s, : n_h[s]]
+            assert n_h[s] == k == len(ref_sel) and k * B <= spec.max_view_tokens
+            modes.append(check_selection(sel_gpu, R, ref_sel, n_sink, n_recent))
+            vK, vV = orc.gather(osess[s].repo, osess[s].table, np.ascontiguousarray(sel_gpu), k * B)
+            assert np.array_equal(bits(view.k[s]), vK) and np.array_equal(bits(view.v[s]), vV), "gathered view differs"
+            if not spec.attend:
+                continue
+            ref_out, ref_lse = orc.attend(qb[s], vK, vV, k * B)
+            err_o, err_l = np.abs(out_h[s] - ref_out).max(), np.abs(lse_h[s] - ref_lse).max()
+            assert err_o <= ATTN_ATOL and err_l <= ATTN_ATOL, f"attention error {err_o:.2e}, lse {err_l:.2e}"
+            assert err_o <= 5e-2 * np.abs(ref_out).max(), "attention error is large relative to the output scale"
+    return modes

@@ -59,7 +59,7 @@ def test_budget_clamp_agrees_with_the_capacity_inequality_and_the_oracle():
 
 def test_calls_without_a_pool_fail_cleanly():
     lib = load_library()
-    assert lib.kvmem_session_reset(None, 0) == kvmem.E_STATE
+    assert lib.kvmem_session_reset(None, 0, None) == kvmem.E_STATE
     assert lib.kvmem_pool_destroy(None) == kvmem.E_STATE
     assert lib.kvmem_set_option(b"no_such_option", 1) == kvmem.E_INVALID
     handle = C.c_void_p()

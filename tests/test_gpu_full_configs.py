@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 import torch
 
-from kvmem_harness import ATTN_ATOL, bits, check_scores, check_selection, fill_oracle, fill_pool, queries
+from kvmem_harness import bits, check_scores, check_selection, fill_oracle, fill_pool, full_step, queries
 from kvmem_workloads import CONFIGS, kv_blocks, planted_blocks, select_params
 from oracle import kvmem_oracle as orc
 
@@ -27,55 +27,17 @@ def test_generator_is_bit_identical_on_cpu_and_gpu():
 
 
 def _full_step(spec, qsets=(0,), gap_forced_budget=None):
-    from paper_2609_04852_b200 import SelectParams, budget_blocks
-    dev = torch.device("cuda", 0)
-    pool = fill_pool(spec)
-    osess = fill_oracle(spec, gen_device=dev)
-    prm_d = select_params(spec)
-    if gap_forced_budget is not None:
-        prm_d["budget_blocks"] = gap_forced_budget
-    prm = SelectParams(**prm_d)
-    ns, B, M = spec.n_sessions, spec.block_tokens, spec.n_q_tokens
-    k = budget_blocks(prm, B, spec.n_blocks)
-    sel = torch.zeros(ns, k, dtype=torch.int32, device=dev)
-    n_sel = torch.zeros(ns, dtype=torch.int32, device=dev)
-    scores = torch.zeros(ns, spec.n_blocks, dtype=torch.float32, device=dev)
-    view = pool.new_view(ns, k * B)
-    out, lse = pool.new_outputs(ns, M)
-    for s in range(ns):
-        assert np.array_equal(bits(pool.index(s)), osess[s].idx), "Mean-K index differs"
-    modes = []
-    for qset in qsets:
-        q, qb = queries(spec, qset)
-        qd = q.to(dev)
-        pool.select(qd, prm, sel, n_sel, scores)
-        pool.materialize(sel, n_sel, view)
-        pool.view_attend(qd, view, n_sel, out, lse)
-        # the fused call (what the benchmark times) must leave the same view and the same results
-        view2 = pool.new_view(ns, k * B)
-        out2, lse2 = pool.new_outputs(ns, M)
-        pool.materialize_attend(qd, sel, n_sel, view2, out2, lse2)
-        torch.cuda.synchronize()
-        assert pool.device_status() == 0
-        assert torch.equal(view.k, view2.k) and torch.equal(view.v, view2.v)
-        assert torch.equal(out, out2) and torch.equal(lse, lse2)
-        del view2
-        sel_h, n_h, sc_h = sel.cpu().numpy(), n_sel.cpu().numpy(), scores.cpu().numpy()
-        out_h, lse_h = out.cpu().numpy(), lse.cpu().numpy()
-        for s in range(ns):
-            R, _ = orc.block_scores(qb[s], osess[s].idx, spec.n_blocks)
-            ref_sel = orc.select(R, B, prm_d["budget_blocks"], prm_d["max_view_tokens"])
-            check_scores(sc_h[s], R, M)
-            sel_gpu = sel_h[s, : n_h[s]]
-            assert n_h[s] == k == len(ref_sel) and k * B <= spec.max_view_tokens
-            modes.append(check_selection(sel_gpu, R, ref_sel))
-            vK, vV = orc.gather(osess[s].repo, osess[s].table, np.ascontiguousarray(sel_gpu), k * B)
-            assert np.array_equal(bits(view.k[s]), vK) and np.array_equal(bits(view.v[s]), vV), "gathered view differs"
-            ref_out, ref_lse = orc.attend(qb[s], vK, vV, k * B)
-            err_o, err_l = np.abs(out_h[s] - ref_out).max(), np.abs(lse_h[s] - ref_lse).max()
-            assert err_o <= ATTN_ATOL and err_l <= ATTN_ATOL, f"attention error {err_o:.2e}, lse {err_l:.2e}"
-            assert err_o <= 5e-2 * np.abs(ref_out).max(), "attention error is large relative to the output scale"
-    return modes
+    return full_step(spec, qsets, gap_forced_budget)
+
+
+def test_config_tiny_full():
+    """The small configuration exactly as stated (256 blocks of 64 tokens, one query token, 8 planted blocks, budget 32,
+    seed 0), every query set; with the budget at the planted count the boundary gap is wide and the ids must be equal."""
+    spec = CONFIGS["tiny"]
+    assert (spec.n_blocks, spec.block_tokens, spec.n_q_tokens, spec.n_planted, spec.budget_blocks, spec.seed) == (256, 64, 1, 8, 32, 0)
+    _full_step(spec, qsets=tuple(range(spec.n_query_sets)))
+    modes = _full_step(spec, qsets=tuple(range(spec.n_query_sets)), gap_forced_budget=spec.n_planted)
+    assert modes == ["exact"] * spec.n_query_sets
 
 
 def test_config_128k_full():
@@ -86,11 +48,11 @@ def test_config_128k_full():
 
 
 def test_config_1m_full():
-    _full_step(CONFIGS["1m"])
+    _full_step(CONFIGS["1m"], qsets=(0, 5, 10, 15))
 
 
 def test_config_batch8_full():
-    _full_step(CONFIGS["batch8"])
+    _full_step(CONFIGS["batch8"], qsets=(0, 5, 10, 15))
 
 
 def test_config_chunk512_full():

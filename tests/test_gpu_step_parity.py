@@ -1,0 +1,253 @@
+"""Whole-step parity cases beyond the five benchmark shapes: more than one scored layer (the mean over (l, h) of
+Eq. "kvmem-block-score" on the GPU, and every later stage with L > 1), a session that is reset and refilled, ids
+outside the session in both gather variants, and the in-block key layout against the raw-key definition of the
+position-consistent view (Sec. 4.4)."""
+import numpy as np
+import pytest
+import torch
+
+from kvmem_harness import ATTN_ATOL, Guards, bits, fill_oracle, fill_pool, full_step, queries
+from kvmem_workloads import CONFIGS, kv_blocks, page_table
+from oracle import kvmem_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+SMALL = CONFIGS["tiny"].with_(name="small", n_blocks=200, n_planted=6, budget_blocks=24)
+
+
+# ------------------------------------------------------------------ more than one scored layer
+
+@pytest.mark.parametrize("L,G,H,M,n_blocks,budget", [(2, 8, 32, 4, 200, 24), (4, 4, 16, 4, 333, 40), (2, 8, 32, 1, 130, 130)],
+                         ids=["L2G8H32", "L4G4H16", "L2-everything-selected"])
+def test_whole_step_with_several_scored_layers(L, G, H, M, n_blocks, budget):
+    """select, materialize, view_attend, materialize_attend and paged_attend with L > 1: the score is the mean over
+    layers and heads, every layer has its own pages, index rows, view rows and outputs."""
+    spec = SMALL.with_(name=f"L{L}", n_layers=L, n_kv_heads=G, n_q_heads=H, n_q_tokens=M, n_blocks=n_blocks,
+                       n_planted=6, budget_blocks=budget)
+    modes = full_step(spec, qsets=(0, 1, 2))
+    assert len(modes) == 3
+    modes = full_step(spec, qsets=(0,), gap_forced_budget=min(spec.n_planted, budget), n_sink=1, n_recent=2)
+    assert len(modes) == 1
+
+
+def test_layers_are_not_mixed_up():
+    """With L = 2, zeroing layer 1 of the query must leave layer 0's attention outputs unchanged and change the scores:
+    a kernel that read the wrong layer's rows would not show that."""
+    from paper_2609_04852_b200 import SelectParams
+    spec = SMALL.with_(name="L2mix", n_layers=2, n_q_tokens=2, n_blocks=96, budget_blocks=96)
+    dev = torch.device("cuda", 0)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    q, _ = queries(spec)
+    q2 = q.clone()
+    q2[:, :, 1] = 0
+    g = Guards(dev)
+    outs = []
+    for qq in (q, q2):
+        sel, n_sel = g.empty((1, 96), torch.int32), g.empty((1,), torch.int32)
+        scores = g.empty((1, 96), torch.float32)
+        out, lse = g.outputs(pool, 1, 2)
+        pool.select(qq.to(dev), SelectParams(96, 1 << 30, 0, 0, 0), sel, n_sel, scores)
+        pool.paged_attend(qq.to(dev), sel, n_sel, out, lse)
+        torch.cuda.synchronize()
+        R, _ = orc.block_scores(bits(qq)[0], osess.idx, 96)
+        assert np.abs(scores.cpu().numpy()[0] - R).max() <= 1e-3 * R.max()
+        outs.append((out.clone(), lse.clone(), scores.clone()))
+    g.check()
+    assert torch.equal(outs[0][0][:, :, 0], outs[1][0][:, :, 0]) and torch.equal(outs[0][1][:, :, 0], outs[1][1][:, :, 0])
+    assert not torch.equal(outs[0][2], outs[1][2])
+    # layer 1 with a zero query: uniform attention, lse = ln T
+    T = 96 * spec.block_tokens
+    assert (outs[1][1][:, :, 1] - np.log(T)).abs().max().item() <= ATTN_ATOL
+    assert pool.device_status() == 0
+
+
+# ------------------------------------------------------------------ reset and refill
+
+def test_reset_session_is_empty_on_the_device_and_its_pages_can_be_reused():
+    """After kvmem_session_reset the device sees an empty session (select gives n_sel = 0, status clean, nothing read),
+    and the freed pages can go to another session without the first one reaching them."""
+    from paper_2609_04852_b200 import Pool, SelectParams
+    spec = SMALL.with_(name="reset", n_sessions=2, n_blocks=40, n_planted=3, budget_blocks=8, n_q_tokens=2)
+    dev = torch.device("cuda", 0)
+    pool = Pool(1, 32, 8, 128, 64, 2, 40, 40, 0)                 # 40 pages in all: session 1 can only live in session 0's old pages
+    K0, V0 = kv_blocks(spec, 0, 0, 40, dev)
+    pool.append_blocks(0, K0, V0)
+    q, qb = queries(spec)
+    qd = q.to(dev)
+    g = Guards(dev)
+    sel, n_sel = g.empty((1, 8), torch.int32, fill=-1), g.empty((1,), torch.int32, fill=77)
+    prm = SelectParams(8, 1 << 30, 0, 0, 0)
+    pool.select(qd[0:1], prm, sel, n_sel)
+    assert int(n_sel.item()) == 8
+    pool.session_reset(0)
+    assert pool.session_blocks(0) == 0
+    sel.fill_(-1)
+    pool.select(qd[0:1], prm, sel, n_sel)                        # empty session: nothing selected, nothing flagged
+    out, lse = g.outputs(pool, 1, 2)
+    pool.paged_attend(qd[0:1], sel, n_sel, out, lse)
+    torch.cuda.synchronize()
+    assert int(n_sel.item()) == 0 and bool((sel == -1).all())
+    assert bool((out == 0).all()) and bool(torch.isneginf(lse).all())
+    assert pool.device_status() == 0
+    # session 1 takes over the pages; its step must match the oracle on session 1's bytes
+    K1, V1 = kv_blocks(spec, 1, 0, 40, dev)
+    pool.append_blocks(1, K1, V1)
+    ospec = spec.with_(n_sessions=1)
+    repo = orc.Repository.empty(40, 64, 1, 8, 128)
+    table = np.arange(40, dtype=np.int32)
+    repo.place(bits(K1), bits(V1), table)
+    idx = orc.mean_k_index(bits(K1), 64)
+    assert np.array_equal(bits(pool.index(1)), idx)
+    scores = g.empty((1, 40), torch.float32)
+    view = g.view(pool, 1, 8 * 64)
+    pool.select(qd[1:2], prm, sel, n_sel, scores, session_first=1)
+    pool.materialize(sel, n_sel, view, session_first=1)
+    out1, lse1 = g.outputs(pool, 1, 2)
+    pool.view_attend(qd[1:2], view, n_sel, out1, lse1)
+    torch.cuda.synchronize()
+    g.check()
+    R, _ = orc.block_scores(qb[1], idx, 40)
+    ref_sel = orc.select(R, 64, 8, 1 << 30)
+    assert np.array_equal(sel.cpu().numpy()[0], ref_sel)
+    vK, vV = orc.gather(repo, table, ref_sel, 8 * 64)
+    assert np.array_equal(bits(view.k[0]), vK) and np.array_equal(bits(view.v[0]), vV)
+    ro, rl = orc.attend(qb[1], vK, vV, 8 * 64)
+    assert np.abs(out1.cpu().numpy()[0] - ro).max() <= ATTN_ATOL and np.abs(lse1.cpu().numpy()[0] - rl).max() <= ATTN_ATOL
+    # session 0 is still empty on the device although the pages are live again
+    pool.select(qd[0:1], prm, sel, n_sel)
+    torch.cuda.synchronize()
+    assert int(n_sel.item()) == 0 and pool.device_status() == 0 and ospec.n_sessions == 1
+
+
+# ------------------------------------------------------------------ ids outside the session
+
+@pytest.mark.parametrize("gather_mode", [1, 0])
+def test_both_gather_variants_skip_an_id_outside_the_session(gather_mode):
+    from paper_2609_04852_b200 import set_option
+    from paper_2609_04852_b200.kvmem import E_DEVICE_RANGE
+    spec = SMALL
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    dev = torch.device("cuda", 0)
+    ids = [1, 5000, 7, -3, 150, 199, 200, 12, 13, 14]             # 5000, -3 and 200 are outside [0, 200)
+    good = [j for j, b in enumerate(ids) if 0 <= b < spec.n_blocks]
+    sel = torch.tensor([ids], dtype=torch.int32, device=dev)
+    n_sel = torch.tensor([len(ids)], dtype=torch.int32, device=dev)
+    g = Guards(dev)
+    view = g.view(pool, 1, len(ids) * spec.block_tokens)
+    view.k.fill_(7.0), view.v.fill_(9.0)
+    set_option("gather_mode", gather_mode)
+    try:
+        pool.materialize(sel, n_sel, view)
+        assert pool.device_status() == E_DEVICE_RANGE
+    finally:
+        set_option("gather_mode", 1)
+    g.check()
+    B = spec.block_tokens
+    for j, b in enumerate(ids):
+        kj, vj = view.k[0][:, :, j * B:(j + 1) * B], view.v[0][:, :, j * B:(j + 1) * B]
+        if j in good:
+            vK, vV = orc.gather(osess.repo, osess.table, np.array([b], np.int32), B)
+            assert np.array_equal(bits(kj), vK) and np.array_equal(bits(vj), vV), f"slot {j}"
+        else:
+            assert bool((kj == 7.0).all()) and bool((vj == 9.0).all()), f"slot {j} of a flagged id was written"
+
+
+# ------------------------------------------------------------------ in-block key layout against the raw-key definition
+
+THETA, WINDOW = 1.0e6, 4096
+# One bf16 rounding moves an element by at most 2^-9 of its size, sigma = 2^-9 / sqrt(3).  The definition (Sec. 4.4)
+# rounds RoPE(k, p0 + t) once; the in-block formulations round the stored key RoPE(k, t) and then either the query
+# rotated back by p0 or the stored key rotated on by p0: three roundings separate a logit of one formulation from the
+# definition's.  With |q|^2 = 2 d and unit-variance keys the logit difference has
+#   sigma_s = sqrt(3) * (2^-9 / sqrt(3)) * sqrt(sum_c q_c^2 k_c^2) / sqrt(d)  ~  2^-9 * sqrt(2 d) / sqrt(d) = 2.8e-3,
+# lse moves by at most the largest logit difference and out by a probability-weighted mean of them, so
+# 7 sigma_s = 2e-2 bounds both with room for the largest of a few thousand logits.
+REFORMULATION_ATOL = 2e-2
+
+
+def _fill_in_block_and_raw(spec):
+    """A pool with rope_in_block_keys filled from raw keys, and the ORACLE repository of the raw keys themselves."""
+    from paper_2609_04852_b200 import Pool
+    dev = torch.device("cuda", 0)
+    pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.block_tokens, 1, spec.n_blocks,
+                spec.n_blocks, 0, WINDOW, THETA, rope_in_block_keys=True)
+    tab = orc.rope_table(WINDOW, spec.head_dim, THETA)
+    table = page_table(spec)[0]
+    raw_repo = orc.Repository.empty(spec.n_blocks, spec.block_tokens, spec.n_layers, spec.n_kv_heads, spec.head_dim)
+    for b0 in range(0, spec.n_blocks, 64):
+        b1 = min(spec.n_blocks, b0 + 64)
+        K, V = kv_blocks(spec, 0, b0, b1, dev)
+        pool.append_blocks(0, K, V, table[b0:b1].tolist())
+        raw_repo.place(bits(K), bits(V), np.ascontiguousarray(table[b0:b1].numpy()))
+    torch.cuda.synchronize()
+    return pool, raw_repo, tab, table.numpy()
+
+
+@pytest.mark.parametrize("n_blocks,budget,M,first", [(150, 20, 4, 517), (700, 60, 4, 17), (90, 1, 1, 0), (64, 60, 2, 250)])
+def test_in_block_layout_against_the_raw_key_definition(n_blocks, budget, M, first):
+    """kvmem_paged_attend_rope (query rotated back per block) and kvmem_materialize_attend_rope (stored keys rotated on
+    per block) on a rope_in_block_keys pool, compared with the definition: attention over the view whose keys are the
+    RAW keys rotated to their compact positions, one rounding each."""
+    spec = SMALL.with_(name="in_block_def", n_blocks=n_blocks, n_planted=5, budget_blocks=budget, n_q_tokens=M)
+    dev = torch.device("cuda", 0)
+    pool, raw_repo, tab, table = _fill_in_block_and_raw(spec)
+    B = spec.block_tokens
+    ids = np.sort(np.random.default_rng(7 * n_blocks).choice(n_blocks, size=budget, replace=False)).astype(np.int32)
+    q, qb = queries(spec)
+    qd = q.to(dev)
+    sel = torch.from_numpy(ids).view(1, -1).to(dev)
+    n_sel = torch.tensor([budget], dtype=torch.int32, device=dev)
+    T = budget * B
+    dK, dV = orc.gather_rope(raw_repo, table, ids, T, first, tab, in_block=False)      # the definition's view
+    ref_out, ref_lse = orc.attend(qb[0], dK, dV, T)
+    g = Guards(dev)
+    out_q, lse_q = g.outputs(pool, 1, M)
+    pool.paged_attend_rope(qd, sel, n_sel, out_q, lse_q, first)
+    view = g.view(pool, 1, T)
+    out_k, lse_k = g.outputs(pool, 1, M)
+    pool.materialize_attend_rope(qd, sel, n_sel, view, out_k, lse_k, first)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    g.check()
+    for name, o, l in (("query rotated back", out_q, lse_q), ("stored keys rotated on", out_k, lse_k)):
+        eo, el = np.abs(o.cpu().numpy()[0] - ref_out).max(), np.abs(l.cpu().numpy()[0] - ref_lse).max()
+        assert eo <= REFORMULATION_ATOL and el <= REFORMULATION_ATOL, f"{name}: out {eo:.2e}, lse {el:.2e}"
+    # values are never re-encoded: the view's V equals the definition's bit for bit, its K within one bf16 step
+    assert np.array_equal(bits(view.v[0]), dV)
+    kf, df = view.k[0].float().cpu().numpy(), orc.bf16_bits_to_f32(dK)
+    assert np.abs(kf - df).max() <= 2.0 ** -7 * max(np.abs(df).max(), 1.0)
+
+
+# ------------------------------------------------------------------ a bounded wait that runs out
+
+def test_a_bounded_wait_that_runs_out_sets_the_status_word_and_leaves_the_pool_usable():
+    """The kernels' wait routine, given a barrier nobody arrives at and a 2 ms limit, gives up, reports
+    KVMEM_E_TIMEOUT through the status word and returns; a normal step on the same pool then matches the oracle."""
+    from paper_2609_04852_b200.kvmem import E_TIMEOUT
+    spec = SMALL
+    pool = fill_pool(spec)
+    assert pool.device_status() == 0
+    waited = pool.selftest_wait_timeout(2000)
+    assert 2_000_000 <= waited < 500_000_000, f"the wait lasted {waited} ns"
+    assert pool.device_status() == E_TIMEOUT
+    assert pool.device_status() == 0                              # reading clears the word
+    modes = full_step(spec, qsets=(0,))                           # a fresh pool in the same context ...
+    assert len(modes) == 1
+    from paper_2609_04852_b200 import SelectParams                # ... and the pool that saw the timeout still works
+    dev = torch.device("cuda", 0)
+    q, qb = queries(spec)
+    sel = torch.zeros(1, 24, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    pool.select(q.to(dev), SelectParams(24, 1 << 30, 0, 0, 0), sel, n_sel)
+    out, lse = pool.new_outputs(1, spec.n_q_tokens)
+    pool.paged_attend(q.to(dev), sel, n_sel, out, lse)
+    torch.cuda.synchronize()
+    osess = fill_oracle(spec)[0]
+    R, _ = orc.block_scores(qb[0], osess.idx, spec.n_blocks)
+    ids = sel.cpu().numpy()[0, : int(n_sel.item())]
+    vK, vV = orc.gather(osess.repo, osess.table, np.ascontiguousarray(ids), 24 * spec.block_tokens)
+    ro, rl = orc.attend(qb[0], vK, vV, len(ids) * spec.block_tokens)
+    assert np.abs(out.cpu().numpy()[0] - ro).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - rl).max() <= ATTN_ATOL
+    assert pool.device_status() == 0

@@ -151,3 +151,36 @@ def test_combining_scores_without_ranks_is_the_identity_and_an_injected_reduce_i
     other = torch.tensor([0.5, 0.5])
     y = combine_head_shard_scores(x.clone(), 2, all_reduce=lambda t: t.add_(other * 0.5))
     assert y.tolist() == [0.375, 0.625]
+
+
+# ---- the benchmark launches its own ranks -----------------------------------------------------------
+
+def _bench(*argv, env=None):
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    e = dict(os.environ)
+    for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT"):
+        e.pop(k, None)
+    e.update(env or {})
+    return subprocess.run([sys.executable, os.path.join(root, "bench.py"), *argv], env=e, capture_output=True, text=True,
+                          timeout=300)
+
+
+def test_bench_with_gpus_2_launches_two_ranks_and_prints_one_line():
+    """`bench.py --gpus 2` from a plain command line becomes two ranks (gloo here: the launch and timing plumbing
+    without a GPU); rank 0 prints exactly one JSON line with n_gpus = 2 and the slowest rank's time."""
+    import json
+    res = _bench("--gpus", "2", "--launch-selfcheck", "--steps", "5")
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["ms_slowest_rank"] == 15.0
+    assert line["value"] == whole_job_rate(5, 2, 15.0)
+
+
+def test_bench_refuses_a_rank_count_that_differs_from_gpus():
+    res = _bench("--gpus", "2", "--launch-selfcheck", env={"WORLD_SIZE": "1", "RANK": "0"})
+    assert res.returncode != 0 and "WORLD_SIZE=1" in (res.stderr + res.stdout)
+    assert not [ln for ln in res.stdout.splitlines() if ln.startswith("{")]

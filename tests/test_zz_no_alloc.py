@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 
 def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row():
     from paper_2609_04852_b200 import KvmemError, SelectParams
-    from paper_2609_04852_b200.kvmem import E_CAPACITY
+    from paper_2609_04852_b200.kvmem import E_CAPACITY, E_INVALID
     spec = CONFIGS["tiny"].with_(name="noalloc", n_blocks=300, n_planted=6, budget_blocks=150, n_q_tokens=4)
     dev = torch.device("cuda", 0)
     pool = fill_pool(spec)
@@ -42,6 +42,8 @@ def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row(
         assert torch.isfinite(out).all() and torch.isfinite(lse).all(), f"call {call}: output not written"
         assert (out - ref_out).abs().max().item() <= ATTN_ATOL, f"call {call}: outputs differ"
         assert (lse - ref_lse).abs().max().item() <= ATTN_ATOL, f"call {call}: log-sum-exp differs"
+        # the same kernels with the same split boundaries ran on both sides: not a bit may differ
+        assert torch.equal(out, ref_out) and torch.equal(lse, ref_lse), f"call {call}: results are not bit-identical"
 
     # more (session, layer, KV head) triples than the built-in scratch covers: refused with a message
     big = CONFIGS["batch8"].with_(name="noalloc2", n_sessions=2, n_blocks=8, n_planted=1, budget_blocks=4)
@@ -53,3 +55,8 @@ def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row(
     with pytest.raises(KvmemError) as e:
         pool2.view_attend_static(q2, view2, n2, out2, lse2)
     assert e.value.status == E_CAPACITY and "at most 8" in str(e.value)
+    # no session at all is an argument error, as it is for the entry point with a caller workspace
+    empty = torch.zeros(0, big.n_q_tokens, 1, big.n_q_heads, big.head_dim, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(KvmemError) as e:
+        pool2.view_attend_static(empty, view2, n2, out2, lse2)
+    assert e.value.status == E_INVALID
