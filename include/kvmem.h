@@ -10,7 +10,8 @@
  *     storage, views, outputs and workspaces, are owned by the caller; the library owns only
  *     the opaque handle and its host-side metadata and never allocates device memory.
  *   - All device work is enqueued on the given stream (a cudaStream_t passed as void*) and is
- *     asynchronous unless a call says otherwise.  A pool is not thread-safe.  The pool's device must be the calling
+ *     asynchronous unless a call says otherwise.  A pool is not thread-safe, and calls on one pool must not overlap on
+ *     the GPU (one stream, or ordered by events): kernels of one pool share its status and barrier words.  The pool's device must be the calling
  *     thread's current device in every call that enqueues work (KVMEM_E_STATE otherwise).
  *   - Every call returns a kvmem_status_t.  Argument, state and capacity errors are detected
  *     on the host before anything is enqueued and leave the pool unchanged; kvmem_last_error()
@@ -189,9 +190,11 @@ int kvmem_materialize_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_
 /* ---- the recall step ----------------------------------------------------------------------- */
 
 /* Scores only (Eq. "kvmem-block-score", Sec. 4.3): the first half of kvmem_select, same arguments and
- * definitions; scores (required) receives R for every session. */
+ * definitions; scores (required) receives score_scale * R for every session.  score_scale (0 selects 1) lets a rank
+ * that holds 1/N of the heads of a session write its share of the head mean directly (score_scale = 1/N): the sum of
+ * the ranks' outputs is then R, with no arithmetic outside the library. */
 int kvmem_score(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/, int32_t n_q_tokens,
-                float* scores /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
+                float* scores /*DEVICE*/, float score_scale, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
 /* Selection alone (Sec. 4.3: reserve sink and recent blocks, fill the budget with the largest R_b, ties to the
  * lower id, chronological output): the second half of kvmem_select, for scores the caller already has (for
@@ -523,6 +526,9 @@ int kvmem_selftest_wait_timeout(kvmem_pool_t* pool, uint32_t limit_us, uint64_t*
  * number of copy CTAs), "attend_landed" (-1 = chosen by the library, 1 / 0 = the lookahead counts tiles that have not
  * landed in shared memory yet / that have not been consumed yet): the knobs of the bytes-in-flight sweeps; only
  * "attend_splits" can move a result, by the rounding of a different split-K merge order.
+ * "score_fused" (decode-sized queries): 1 = block scores from one kernel that keeps the logits in shared memory and
+ * meets at one grid-wide barrier, where the shape fits (at most 16 query rows per KV head, 16 (layer, KV head) pairs,
+ * one CTA's logits in shared memory; default), 0 = logits kernel + finish kernel; moves scores by rounding only.
  * "pdl": 1 = the kernels of a step are launched with programmatic stream serialization, so that the
  * launch latency of each overlaps the tail of the one before (default), 0 = plain launches. */
 int kvmem_set_option(const char* name /*HOST*/, int32_t value);

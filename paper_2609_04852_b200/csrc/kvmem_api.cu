@@ -383,7 +383,7 @@ int kvmem_materialize_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_ses
 
 // scoring stage shared by kvmem_score and kvmem_select; *sc_out receives where the scores were written
 static int score_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
-                      float* scores, void* workspace, size_t workspace_bytes, cudaStream_t st, float** sc_out) {
+                      float* scores, float score_scale, void* workspace, size_t workspace_bytes, cudaStream_t st, float** sc_out) {
     if (!q || !aligned(q, 16) || !workspace || !aligned(workspace, 256)) {
         set_error("scoring: null or misaligned pointer");
         return KVMEM_E_INVALID;
@@ -403,13 +403,13 @@ static int score_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions
         if (workspace_bytes < cw.total) { set_error("select workspace holds %zu bytes, %zu needed", workspace_bytes, cw.total); return KVMEM_E_CAPACITY; }
         sc = scores ? scores : cw.scores;
         e = launch_score_chunked(*p, session_first, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, cw, sc,
-                                 p->cfg.max_blocks_per_session, st);
+                                 p->cfg.max_blocks_per_session, score_scale, st);
     } else {
         ScoreWorkspace ws = plan_score_workspace(p->cfg, n_sessions, n_q_tokens, (char*)workspace);
         if (workspace_bytes < ws.total) { set_error("select workspace holds %zu bytes, %zu needed", workspace_bytes, ws.total); return KVMEM_E_CAPACITY; }
         sc = scores ? scores : ws.scores;
         e = launch_score_decode(*p, session_first, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, ws, sc,
-                                p->cfg.max_blocks_per_session, st);
+                                p->cfg.max_blocks_per_session, score_scale, st);
     }
     if (e != cudaSuccess) return cuda_fail("score kernel launch", e);
     *sc_out = sc;
@@ -417,12 +417,14 @@ static int score_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions
 }
 
 int kvmem_score(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens, float* scores,
-                void* workspace, size_t workspace_bytes, void* stream) {
+                float score_scale, void* workspace, size_t workspace_bytes, void* stream) {
     if (!pool_live(p)) return KVMEM_E_STATE;
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
     if (!scores) { set_error("scores is null"); return KVMEM_E_INVALID; }
+    if (!(score_scale >= 0.0f) || !std::isfinite(score_scale)) { set_error("score_scale must be non-negative and finite (0 selects 1)"); return KVMEM_E_INVALID; }
     float* sc = nullptr;
-    return score_impl(p, session_first, n_sessions, q, n_q_tokens, scores, workspace, workspace_bytes, (cudaStream_t)stream, &sc);
+    return score_impl(p, session_first, n_sessions, q, n_q_tokens, scores, score_scale > 0.0f ? score_scale : 1.0f, workspace,
+                      workspace_bytes, (cudaStream_t)stream, &sc);
 }
 
 // ---- index in host memory, streamed in tiles
@@ -501,7 +503,7 @@ int kvmem_select(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, con
     if (sel_stride < max_k) { set_error("sel_stride %d is below the clamped budget %d", sel_stride, max_k); return KVMEM_E_CAPACITY; }
     cudaStream_t st = (cudaStream_t)stream;
     float* sc = nullptr;
-    int rc = score_impl(p, session_first, n_sessions, q, n_q_tokens, scores, workspace, workspace_bytes, st, &sc);
+    int rc = score_impl(p, session_first, n_sessions, q, n_q_tokens, scores, 1.0f, workspace, workspace_bytes, st, &sc);
     if (rc != KVMEM_OK) return rc;
     cudaError_t e = launch_topk(*p, session_first, n_sessions, sc, p->cfg.max_blocks_per_session, *prm, sel_ids, sel_stride, n_sel, st);
     if (e != cudaSuccess) return cuda_fail("top-k kernel launch", e);
@@ -642,6 +644,7 @@ int kvmem_set_option(const char* name, int32_t value) {
     if (strcmp(name, "attend_splits") == 0 && value >= 0 && value <= 64) { g_attend_splits = value; return KVMEM_OK; }
     if (strcmp(name, "pdl") == 0 && (value == 0 || value == 1)) { g_pdl = value; return KVMEM_OK; }
     if (strcmp(name, "score_mode") == 0 && (value == 0 || value == 1)) { g_score_mode = value; return KVMEM_OK; }
+    if (strcmp(name, "score_fused") == 0 && (value == 0 || value == 1)) { g_score_fused = value; return KVMEM_OK; }
     set_error("unknown option or value: %s = %d", name, value);
     return KVMEM_E_INVALID;
 }
@@ -1033,6 +1036,11 @@ int kvmem_device_status(kvmem_pool_t* p, int32_t* status, void* stream) {
     cudaError_t e = cudaMemcpyAsync(&word, p->status_dev, 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->status_dev, 0, 4, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    // a kernel that gave up at the grid barrier of the one-kernel scorer leaves the barrier's counter behind: re-arm it
+    if (e == cudaSuccess && word == KVMEM_E_TIMEOUT) {
+        e = cudaMemsetAsync(p->status_dev + 16, 0, 192, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    }
     if (e != cudaSuccess) return cuda_fail("reading the device status word", e);
     *status = word;
     return KVMEM_OK;

@@ -727,7 +727,7 @@ static bool make_index_map(PFN_cuTensorMapEncodeTiled_v12000 enc, CUtensorMap* m
 int g_chunk_poly = 4;   // every n-th exponential of the chunked passes on the FMA pipe; 0: none
 
 cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q, int M,
-                                 const ChunkWorkspace& ws, float* scores, int scores_stride, cudaStream_t st) {
+                                 const ChunkWorkspace& ws, float* scores, int scores_stride, float score_scale, cudaStream_t st) {
     const Geometry& g = p.geo;
     PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode_fn();
     if (!enc) return cudaErrorNotSupported;
@@ -784,7 +784,7 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
 #undef KVMEM_CHUNK_PASSES
     dim3 fgrid((unsigned)((max_nb + 255) / 256), (unsigned)n_sessions);
     launch_pdl(score_chunk_finish_kernel, dim3(fgrid), dim3(256), 0, st, ws.colsum, p.nblocks_dev, session_first, kCkSplit * LG, ws.nb_pad,
-                                                     1.0f / (float)(g.L * g.H), scores, scores_stride);
+                                                     score_scale / (float)(g.L * g.H), scores, scores_stride);
     return cudaGetLastError();
 }
 

@@ -67,7 +67,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_session_reset": (C.c_int, [vp, i32, vp]),
         "kvmem_session_blocks": (i32, [vp, i32]),
         "kvmem_append_blocks": (C.c_int, [vp, i32, vp, vp, i32, C.POINTER(i32), vp]),
-        "kvmem_score": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, sz, vp]),
+        "kvmem_score": (C.c_int, [vp, i32, i32, vp, i32, vp, f32, vp, sz, vp]),
         "kvmem_topk": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp]),
         "kvmem_score_host_workspace_bytes": (sz, [vp, i32, i32, i32]),
         "kvmem_score_host_staging_bytes": (sz, [vp, i32]),
@@ -292,12 +292,13 @@ class Pool:
             self._attend_ws = torch.empty(need, dtype=torch.uint8, device=self.device)
         return self._attend_ws
 
-    def score(self, q: torch.Tensor, scores: torch.Tensor, session_first: int = 0) -> None:
-        """Block relevance only: q bf16 [n_sessions][M][L][H][d] -> scores fp32 [n_sessions][max_blocks_per_session]."""
+    def score(self, q: torch.Tensor, scores: torch.Tensor, session_first: int = 0, score_scale: float = 1.0) -> None:
+        """Block relevance only: q bf16 [n_sessions][M][L][H][d] -> scores fp32 [n_sessions][max_blocks_per_session]
+        (times score_scale: a rank holding 1/N of a session's heads passes 1/N, so that the ranks' outputs sum to R)."""
         ns, M = q.shape[0], q.shape[1]
         ws = self.select_workspace(ns, M)
         _check(self.lib.kvmem_score(self.handle, session_first, ns, _dev(q, torch.bfloat16), M,
-                                    _dev(scores, torch.float32), ws.data_ptr(), ws.numel(), _stream()))
+                                    _dev(scores, torch.float32), score_scale, ws.data_ptr(), ws.numel(), _stream()))
 
     def topk(self, scores: torch.Tensor, params: SelectParams, sel_ids: torch.Tensor, n_sel: torch.Tensor,
              session_first: int = 0) -> None:

@@ -9,7 +9,7 @@ By KV head inside one session (strong scaling): the softmax of the block score (
 Sec. 4.3) is taken per (layer, query token, query head), so a GPU that holds the pages and index rows of
 KV heads [g0, g1) and the query heads that map to them computes its heads' share of R_b without seeing
 the others.  R_b is a mean over heads: one all-reduce (sum) of the NB fp32 partial scores, each scaled by
-its share of the heads, gives every rank the same R bit for bit; every rank then runs the same
+its share of the heads inside the scoring kernel (kvmem_score's score_scale), gives every rank the same R bit for bit; every rank then runs the same
 deterministic top-k and gathers and attends over its own heads.  Outputs are head-disjoint: no second
 exchange.
 """
@@ -70,17 +70,18 @@ def query_heads_of(kv_range: Tuple[int, int], q_per_kv: int) -> Tuple[int, int]:
     return kv_range[0] * q_per_kv, kv_range[1] * q_per_kv
 
 
-def combine_head_shard_scores(r_local: torch.Tensor, world: int, group=None,
+def combine_head_shard_scores(r_share: torch.Tensor, world: int, group=None,
                               all_reduce: Optional[Callable[[torch.Tensor], None]] = None) -> torch.Tensor:
-    """In place: r_local (this rank's mean over ITS heads) -> R (mean over all heads), identical on every rank.
+    """In place: r_share (this rank's mean over ITS heads times 1/world, as kvmem_score writes it when given
+    score_scale = 1/world) -> R (mean over all heads), identical on every rank.
 
-    R = sum over ranks of r_local / world: the scale is applied before the sum (exact for a power-of-two
-    world), the sum is one all-reduce.  all_reduce overrides the collective (tests without a process group)."""
+    R = sum over ranks of r_share: one all-reduce and nothing else; the 1/world factor is applied by the scoring
+    kernel (exact for a power-of-two world).  all_reduce overrides the collective (tests without a process group)."""
     if world < 1:
         raise ValueError("world must be positive")
     if world == 1:
-        return r_local
-    r_local.mul_(1.0 / world)
+        return r_share
+    r_local = r_share
     if all_reduce is not None:
         all_reduce(r_local)
     else:
@@ -97,7 +98,7 @@ def head_sharded_step(pool, q_local: torch.Tensor, params, scores: torch.Tensor,
     matching slice of the query heads.  score (own heads) -> all-reduce of R -> top-k (same ids on every rank)
     -> view assembly and attention over the own heads.  Every step runs in the library's kernels; the only
     exchange is the all-reduce of scores ([n_sessions][max_blocks_per_session] fp32)."""
-    pool.score(q_local, scores)
+    pool.score(q_local, scores, score_scale=1.0 / world)
     combine_head_shard_scores(scores, world, group, all_reduce)
     pool.topk(scores, params, sel_ids, n_sel)
     pool.materialize_attend(q_local, sel_ids, n_sel, view, out, lse)

@@ -43,8 +43,8 @@ def test_head_sharded_step_matches_the_oracle_on_the_whole_session(world, n_bloc
         pool = _shard_pool(spec, g0, g1)
         q_local = q[:, :, :, h0:h1].contiguous().to(dev)
         scores = torch.zeros(1, n_blocks, dtype=torch.float32, device=dev)
-        pool.score(q_local, scores)
-        ranks.append(dict(pool=pool, q=q_local, h=(h0, h1), own=scores.clone() / world))
+        pool.score(q_local, scores, score_scale=1.0 / world)         # the rank's share of the head mean, scaled in the kernel
+        ranks.append(dict(pool=pool, q=q_local, h=(h0, h1), own=scores.clone()))
     torch.cuda.synchronize()
     # the oracle on the unsharded session
     osess = fill_oracle(spec)[0]

@@ -251,3 +251,47 @@ def test_a_bounded_wait_that_runs_out_sets_the_status_word_and_leaves_the_pool_u
     ro, rl = orc.attend(qb[0], vK, vV, len(ids) * spec.block_tokens)
     assert np.abs(out.cpu().numpy()[0] - ro).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - rl).max() <= ATTN_ATOL
     assert pool.device_status() == 0
+
+
+# ------------------------------------------------------------------ one-kernel scorer against the three-kernel form and the oracle
+
+@pytest.mark.parametrize("ns,L,G,H,M,n_blocks", [(1, 1, 8, 32, 4, 2048), (1, 1, 8, 32, 4, 5000), (1, 1, 8, 32, 1, 16384),
+                                               (3, 1, 8, 32, 2, 700), (1, 2, 8, 32, 4, 333), (1, 4, 4, 16, 4, 150),
+                                               (1, 1, 4, 32, 2, 97), (8, 1, 8, 32, 1, 4096), (1, 1, 8, 32, 4, 1)],
+                         ids=["128k-shape", "ragged-5000", "1m-shape", "3-sessions", "L2", "L4G4", "GQA8", "batch8-shape", "one-block"])
+def test_one_kernel_scorer_equals_the_three_kernel_form_and_the_oracle(ns, L, G, H, M, n_blocks):
+    """kvmem_score through the kernel that keeps its logits in shared memory and meets at a grid barrier, for every
+    chunk size it chooses (16 to 128 blocks), several sessions of different length, several layers: against the oracle
+    within the score tolerance and against the logits + finish kernels within rounding; twice in a row (the barrier
+    re-arms itself) with identical bits."""
+    from paper_2609_04852_b200 import Pool, set_option
+    from kvmem_harness import check_scores
+    spec = SMALL.with_(name="fused_score", n_sessions=ns, n_layers=L, n_kv_heads=G, n_q_heads=H, n_q_tokens=M, n_blocks=n_blocks,
+                       n_planted=min(6, n_blocks), budget_blocks=1)
+    dev = torch.device("cuda", 0)
+    lens = [n_blocks if s == 0 else max(1, n_blocks - 37 * s) for s in range(ns)]        # ragged session lengths
+    pool = fill_pool(spec, lens)
+    osess = fill_oracle(spec, lens, gen_device=dev)
+    q, qb = queries(spec)
+    qd = q.to(dev)
+    g = Guards(dev)
+    runs = []
+    for fused in (1, 1, 0):
+        set_option("score_fused", fused)
+        try:
+            sc = g.empty((ns, n_blocks), torch.float32, fill=-1.0)
+            pool.score(qd, sc)
+            torch.cuda.synchronize()
+            assert pool.device_status() == 0
+        finally:
+            set_option("score_fused", 1)
+        runs.append(sc)
+    g.check()
+    assert torch.equal(runs[0], runs[1]), "two runs of the one-kernel scorer differ"
+    for s in range(ns):
+        R, _ = orc.block_scores(qb[s], osess[s].idx, lens[s])
+        for sc in runs:
+            check_scores(sc.cpu().numpy()[s, : lens[s]], R, M)
+            assert bool((sc[s, lens[s]:] == -1.0).all()), "scores past the session's blocks were written"
+        a, b = runs[0][s, : lens[s]], runs[2][s, : lens[s]]
+        assert ((a - b).abs() <= 2e-5 * b.abs() + 1e-12).all(), "one-kernel and three-kernel scores differ by more than rounding"

@@ -105,7 +105,8 @@ def _head_worker(rank, world, port, ret):
         idx_local = orc.mean_k_index(np.ascontiguousarray(Kb[:, :, g0:g1]), spec.block_tokens)
         q_local = np.ascontiguousarray(qb[:, :, h0:h1])
         R_local, _ = orc.block_scores(q_local, idx_local, spec.n_blocks)
-        R = combine_head_shard_scores(torch.from_numpy(R_local.astype(np.float32)), world).numpy()
+        # the library's scoring kernel applies the 1/world share itself (score_scale); the oracle's R_local is scaled here
+        R = combine_head_shard_scores(torch.from_numpy(R_local.astype(np.float32)) * (1.0 / world), world).numpy()
         sel = orc.select(R, spec.block_tokens, spec.budget_blocks, spec.max_view_tokens)
         # attention over the own heads only
         table = np.arange(spec.n_blocks, dtype=np.int32)
@@ -149,7 +150,7 @@ def test_combining_scores_without_ranks_is_the_identity_and_an_injected_reduce_i
     x = torch.tensor([0.25, 0.75])
     assert combine_head_shard_scores(x.clone(), 1).tolist() == [0.25, 0.75]
     other = torch.tensor([0.5, 0.5])
-    y = combine_head_shard_scores(x.clone(), 2, all_reduce=lambda t: t.add_(other * 0.5))
+    y = combine_head_shard_scores(x.clone() * 0.5, 2, all_reduce=lambda t: t.add_(other * 0.5))
     assert y.tolist() == [0.375, 0.625]
 
 
