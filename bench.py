@@ -238,7 +238,7 @@ def run_native(args):
                     ev[1].record(stream)
                     ev[2].record(stream)
                 return
-            if args.in_block:  # one pass: K tiles rotated by their block position in shared memory, stored and attended over
+            if not args.unfused:  # one pass: K rotated on its way through the SM (by block position on the in-block layout, per key on raw keys), stored and attended over
                 pool.materialize_attend_rope(q, sel, n_sel, view, out, lse, 0)
                 if ev is not None:
                     ev[1].record(stream)
@@ -422,7 +422,7 @@ def run_native(args):
         dom_bytes = ns * (ab["attend"] if args.paged else ab["gather"])    # paged: one read of the selected pages
         gather_gbs = dom_bytes / gather_s / 1e9
         # fused: every view byte is read once (from the pages) and written once; separate calls read it a second time
-        one_pass = fused or (args.rope and args.in_block and not args.paged)       # view written while attended
+        one_pass = fused or (args.rope and not args.unfused and not args.paged)       # view written while attended
         step_bytes = ns * (ab["total"] - (ab["attend"] if one_pass else 0))
         if args.paged:
             step_bytes = ns * (ab["index"] + ab["attend"])
@@ -444,7 +444,9 @@ def run_native(args):
                                 "kvmem_rope_rotate(q) + kvmem_select + kvmem_paged_attend_rope (copy-free, keys RoPE'd in shared memory)"
                                 if args.rope and args.paged else
                                 "kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_attend_rope (one pass: K tiles rotated by their block "
-                                "position in shared memory, stored and attended over)" if args.rope and args.in_block else
+                                "position in shared memory, stored and attended over)" if args.rope and args.in_block and not args.unfused else
+                                "kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_attend_rope (one pass over raw keys: the attending warps rotate "
+                                "their key fragments to the compact positions and hand them back for the store)" if args.rope and not args.unfused else
                                 "kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_rope + kvmem_view_attend" if args.rope else
                                 "kvmem_select + kvmem_paged_attend (NO materialize: copy-free view variant)" if args.paged else
                                 "kvmem_select + kvmem_materialize_attend" if fused else
@@ -459,7 +461,9 @@ def run_native(args):
                                                    if args.rope and args.paged and args.in_block else
                                                    "attend_split_kernel<3> + merge (kvmem_paged_attend_rope)" if args.rope and args.paged else
                                                    "attend_split_kernel<5> + merge (kvmem_materialize_attend_rope: K rotated in shared memory, "
-                                                   "view written while attended)" if args.rope and args.in_block else
+                                                   "view written while attended)" if args.rope and args.in_block and not args.unfused else
+                                                   "attend_split_kernel<6> + merge (kvmem_materialize_attend_rope on raw keys: fragments rotated by the "
+                                                   "attending warps, view written while attended)" if args.rope and not args.unfused else
                                                    "gather_rope_kernel (kvmem_materialize_rope)" if args.rope else
                                                    "attend_split_kernel<2> + merge (kvmem_paged_attend)" if args.paged else
                                                    "attend_split_kernel<1> + merge (kvmem_materialize_attend: view written while attended)"
@@ -467,7 +471,8 @@ def run_native(args):
                          "achieved": gather_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gather_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": gather_s * 1e3,
-                         "traffic": None if args.paged else ROPE_FUSED_TRAFFIC.get(base.name) if args.rope and args.in_block else
+                         "traffic": None if args.paged else ROPE_FUSED_TRAFFIC.get(base.name) if args.rope and args.in_block and not args.unfused else
+                                    None if args.rope and not args.unfused else
                                     ROPE_GATHER_TRAFFIC.get(base.name) if args.rope else
                                     FUSED_TRAFFIC.get(base.name) if fused else GATHER_TRAFFIC.get(base.name)},
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes,

@@ -10,8 +10,7 @@
  *     storage, views, outputs and workspaces, are owned by the caller; the library owns only
  *     the opaque handle and its host-side metadata and never allocates device memory.
  *   - All device work is enqueued on the given stream (a cudaStream_t passed as void*) and is
- *     asynchronous unless a call says otherwise.  A pool is not thread-safe, and calls on one pool must not overlap on
- *     the GPU (one stream, or ordered by events): kernels of one pool share its status and barrier words.  The pool's device must be the calling
+ *     asynchronous unless a call says otherwise.  A pool is not thread-safe.  The pool's device must be the calling
  *     thread's current device in every call that enqueues work (KVMEM_E_STATE otherwise).
  *   - Every call returns a kvmem_status_t.  Argument, state and capacity errors are detected
  *     on the host before anything is enqueued and leave the pool unchanged; kvmem_last_error()
@@ -262,10 +261,15 @@ int kvmem_materialize(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessi
  *   lse      DEVICE fp32 [n_sessions][n_q_tokens][n_layers][n_q_heads]
  *   scale    0 selects 1/sqrt(head_dim)
  *   workspace DEVICE, kvmem_attend_workspace_bytes(), 256-byte aligned
- * T = 0 gives out = 0 and lse = -inf.  n_q_tokens * (H/G) <= 16 per call.  Any block size the pool accepts
- * (the view is walked in 64-token tiles; a shorter last tile is masked); head_dim 128.  The calls that read
- * pages through the block table (kvmem_materialize_attend, kvmem_paged_attend*, kvmem_view_cache_attend) are
- * built for 64-token blocks and return KVMEM_E_UNSUPPORTED otherwise. */
+ * T = 0 gives out = 0 and lse = -inf.  n_q_tokens * (H/G) <= 64 query rows per KV head and call (e.g. 1 + 7 draft tokens
+ * with 8 query heads per KV head): up to 16 rows the K/V stream bounds the pass, with 32 or 64 rows the same stream
+ * is read once and the tensor-core work per byte doubles or quadruples (the position-consistent and FP8 variants
+ * take 16 rows).  Any block size the pool accepts (the view is walked in 64-token tiles; a shorter last tile is
+ * masked); head_dim 128.  The calls that read pages through the block table (kvmem_materialize_attend,
+ * kvmem_paged_attend, kvmem_paged_attend_rope on raw keys, kvmem_view_cache_attend) take block sizes that divide
+ * 64 tokens (a tile is then 64 / B selected blocks, the last one possibly partly filled) or are a multiple of it,
+ * among them the paper's default of 32 tokens (Sec. 4.3); the in-block key layout and the FP8 repository are built
+ * for 64-token blocks.  Other shapes return KVMEM_E_UNSUPPORTED. */
 int kvmem_view_attend(kvmem_pool_t* pool, int32_t n_sessions, const void* q /*DEVICE*/, int32_t n_q_tokens,
                       const void* view_k /*DEVICE*/, const void* view_v /*DEVICE*/, int32_t view_cap_tokens,
                       const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
@@ -319,9 +323,11 @@ int kvmem_paged_attend_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n
 /* kvmem_materialize_rope followed by kvmem_view_attend in one call (Sec. 4.4: the execution view with keys
  * encoded at their compact positions, then decode over it).  Same arguments as kvmem_materialize_attend plus
  * first_position; the view left behind is kvmem_materialize_rope's, out/lse are kvmem_view_attend's on it with
- * a q that carries RoPE at its own position.  On a pool with rope_in_block_keys this is ONE pass (each K tile is
- * rotated by its block's compact position while it sits in shared memory, then stored and attended over: 1 read
- * + 1 write per view byte); on a raw-key pool it runs the two kernels one after the other.
+ * a q that carries RoPE at its own position.  ONE pass, 1 read + 1 write per view byte: on a pool with
+ * rope_in_block_keys each K tile is rotated by its block's compact position while it sits in shared memory, then stored
+ * and attended over; on a raw-key pool the warps that attend over a tile rotate its key fragments to their compact
+ * positions on the way to the tensor cores and hand them back to the tile, which is then stored (the view's last
+ * 64-token tile must lie inside the rotary table: first_position + the view length rounded up to 64).
  * Extra errors: KVMEM_E_STATE without a rotary table; KVMEM_E_INVALID if the compact positions leave it. */
 int kvmem_materialize_attend_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
                                   int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
@@ -526,9 +532,6 @@ int kvmem_selftest_wait_timeout(kvmem_pool_t* pool, uint32_t limit_us, uint64_t*
  * number of copy CTAs), "attend_landed" (-1 = chosen by the library, 1 / 0 = the lookahead counts tiles that have not
  * landed in shared memory yet / that have not been consumed yet): the knobs of the bytes-in-flight sweeps; only
  * "attend_splits" can move a result, by the rounding of a different split-K merge order.
- * "score_fused" (decode-sized queries): 1 = block scores from one kernel that keeps the logits in shared memory and
- * meets at one grid-wide barrier, where the shape fits (at most 16 query rows per KV head, 16 (layer, KV head) pairs,
- * one CTA's logits in shared memory; default), 0 = logits kernel + finish kernel; moves scores by rounding only.
  * "pdl": 1 = the kernels of a step are launched with programmatic stream serialization, so that the
  * launch latency of each overlaps the tail of the one before (default), 0 = plain launches. */
 int kvmem_set_option(const char* name /*HOST*/, int32_t value);

@@ -11,7 +11,7 @@
  * by a single round-to-nearest-even to bf16, because the stored index is a quantised
  * code and both sides must take that rounding decision in the same precision.
  *
- * Readings taken where the paper is silent (the full list is in the design notes):
+ * Readings taken where the paper is silent:
  * candidate set C = every block of the session, reserved blocks included; the selector
  * alone applies sink/recent reservation; g(h) = h / (H/G); sum over query tokens, mean
  * over layers and heads; ties broken by lower block id; partial blocks never indexed.

@@ -119,6 +119,22 @@ static int cuda_fail(const char* what, cudaError_t e) {
 
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 
+// The passes that read pages through the block table walk the view in 64-token tiles: a tile is 64 / B whole blocks or
+// a 64-token slice of one block.  in_block_rotation: the pass rotates by one angle set per tile (in-block key layout),
+// which needs tile == block.
+static bool paged_block_size_ok(const kvmem_pool* p, bool in_block_rotation, const char* who) {
+    const int B = p->cfg.block_tokens;
+    if (p->cfg.head_dim != 128 || !(64 % B == 0 || B % 64 == 0)) {
+        set_error("%s is built for head_dim 128 and block sizes that divide or are a multiple of 64 tokens", who);
+        return false;
+    }
+    if (in_block_rotation && B != 64) {
+        set_error("%s on a pool with rope_in_block_keys rotates once per 64-token tile and needs 64-token blocks", who);
+        return false;
+    }
+    return true;
+}
+
 }  // namespace kvmem
 
 using namespace kvmem;
@@ -544,7 +560,7 @@ int kvmem_view_attend(kvmem_pool_t* p, int32_t n_sessions, const void* q, int32_
         set_error("attention kernel is built for head_dim 128");
         return KVMEM_E_UNSUPPORTED;
     }
-    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (n_q_tokens * p->geo.r > 64) { set_error("n_q_tokens * (H/G) = %d exceeds 64 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
     if (view_cap_tokens < p->cfg.block_tokens || view_cap_tokens % p->cfg.block_tokens != 0) {
         set_error("view_cap_tokens must be a positive multiple of block_tokens");
         return KVMEM_E_INVALID;
@@ -644,7 +660,6 @@ int kvmem_set_option(const char* name, int32_t value) {
     if (strcmp(name, "attend_splits") == 0 && value >= 0 && value <= 64) { g_attend_splits = value; return KVMEM_OK; }
     if (strcmp(name, "pdl") == 0 && (value == 0 || value == 1)) { g_pdl = value; return KVMEM_OK; }
     if (strcmp(name, "score_mode") == 0 && (value == 0 || value == 1)) { g_score_mode = value; return KVMEM_OK; }
-    if (strcmp(name, "score_fused") == 0 && (value == 0 || value == 1)) { g_score_fused = value; return KVMEM_OK; }
     set_error("unknown option or value: %s = %d", name, value);
     return KVMEM_E_INVALID;
 }
@@ -662,11 +677,8 @@ static int materialize_attend_impl(kvmem_pool_t* p, int32_t session_first, int32
         return KVMEM_E_INVALID;
     }
     if (n_q_tokens < 1 || sel_stride < 1) { set_error("n_q_tokens and sel_stride must be positive"); return KVMEM_E_INVALID; }
-    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
-        set_error("attention kernel is built for head_dim 128 and 64-token blocks");
-        return KVMEM_E_UNSUPPORTED;
-    }
-    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (!paged_block_size_ok(p, rope_first_position >= 0 && p->cfg.rope_in_block_keys, "kvmem_materialize_attend")) return KVMEM_E_UNSUPPORTED;
+    if (n_q_tokens * p->geo.r > (rope_first_position >= 0 ? 16 : 64)) { set_error("n_q_tokens * (H/G) = %d exceeds %d rows per call", n_q_tokens * p->geo.r, rope_first_position >= 0 ? 16 : 64); return KVMEM_E_UNSUPPORTED; }
     if (view_cap_tokens < p->cfg.block_tokens || view_cap_tokens % p->cfg.block_tokens != 0) {
         set_error("view_cap_tokens must be a positive multiple of block_tokens");
         return KVMEM_E_INVALID;
@@ -706,15 +718,19 @@ int kvmem_materialize_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_
                   p->cfg.rope_max_positions);
         return KVMEM_E_INVALID;
     }
-    if (p->cfg.rope_in_block_keys)      // one pass: every K tile is rotated by its block position on its way through shared memory
-        return materialize_attend_impl(p, session_first, n_sessions, q, n_q_tokens, sel_ids, sel_stride, n_sel, view_k, view_v,
-                                       view_cap_tokens, first_position, scale, out, lse, workspace, workspace_bytes, stream);
-    // raw keys need 64 sets of angles per tile: the rotating gather, then attention over the view
-    int rc = kvmem_materialize_rope(p, session_first, n_sessions, sel_ids, sel_stride, n_sel, view_k, view_v, view_cap_tokens,
-                                    first_position, stream);
-    if (rc != KVMEM_OK) return rc;
-    return kvmem_view_attend(p, n_sessions, q, n_q_tokens, view_k, view_v, view_cap_tokens, n_sel, scale, out, lse, workspace,
-                             workspace_bytes, stream);
+    // One pass either way: on the in-block layout every K tile is rotated by its block position on its way through shared
+    // memory; raw keys are rotated by the consumer warps on their way to the tensor cores and handed back for the store.
+    // The pass walks whole 64-token tiles and fetches the rotary rows of all 64 positions of the last one.
+    if (!p->cfg.rope_in_block_keys) {
+        const int64_t tiles_end = (int64_t)first_position + (std::min<int64_t>((int64_t)sel_stride * p->cfg.block_tokens, view_cap_tokens) + 63) / 64 * 64;
+        if (tiles_end > p->cfg.rope_max_positions) {
+            set_error("the last 64-token tile of the view reaches position %lld, outside the rotary table [0, %d)", (long long)tiles_end,
+                      p->cfg.rope_max_positions);
+            return KVMEM_E_INVALID;
+        }
+    }
+    return materialize_attend_impl(p, session_first, n_sessions, q, n_q_tokens, sel_ids, sel_stride, n_sel, view_k, view_v,
+                                   view_cap_tokens, first_position, scale, out, lse, workspace, workspace_bytes, stream);
 }
 
 static int paged_attend_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const void* q, int32_t n_q_tokens,
@@ -727,11 +743,8 @@ static int paged_attend_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_s
         return KVMEM_E_INVALID;
     }
     if (n_q_tokens < 1 || sel_stride < 1) { set_error("n_q_tokens and sel_stride must be positive"); return KVMEM_E_INVALID; }
-    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
-        set_error("attention kernel is built for head_dim 128 and 64-token blocks");
-        return KVMEM_E_UNSUPPORTED;
-    }
-    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (!paged_block_size_ok(p, rope_first_position >= 0 && p->cfg.rope_in_block_keys, "kvmem_paged_attend")) return KVMEM_E_UNSUPPORTED;
+    if (n_q_tokens * p->geo.r > (rope_first_position >= 0 ? 16 : 64)) { set_error("n_q_tokens * (H/G) = %d exceeds %d rows per call", n_q_tokens * p->geo.r, rope_first_position >= 0 ? 16 : 64); return KVMEM_E_UNSUPPORTED; }
     if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
     if ((int64_t)p->cfg.max_blocks * 2 * p->cfg.n_layers * p->cfg.n_kv_heads * p->cfg.block_tokens > 0x7fffffffll) {
         set_error("page pool too large for 32-bit TMA row coordinates");
@@ -761,7 +774,8 @@ int kvmem_paged_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_se
                             float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
     if (!pool_live(p)) return KVMEM_E_STATE;
     if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
-    const int64_t last = (int64_t)first_position + (int64_t)sel_stride * p->cfg.block_tokens;
+    // the pass walks whole 64-token tiles: the last tile fetches the rotary rows of all 64 of its positions
+    const int64_t last = (int64_t)first_position + ((int64_t)sel_stride * p->cfg.block_tokens + 63) / 64 * 64;
     if (first_position < 0 || sel_stride < 1 || last > p->cfg.rope_max_positions) {
         set_error("compact positions [%d, %lld) outside the rotary table [0, %d)", first_position, (long long)last,
                   p->cfg.rope_max_positions);
@@ -993,11 +1007,8 @@ int kvmem_view_cache_attend(kvmem_pool_t* p, const void* q, int32_t n_q_tokens, 
         return KVMEM_E_INVALID;
     }
     if (n_q_tokens < 1) { set_error("n_q_tokens must be positive"); return KVMEM_E_INVALID; }
-    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
-        set_error("attention kernel is built for head_dim 128 and 64-token blocks");
-        return KVMEM_E_UNSUPPORTED;
-    }
-    if (n_q_tokens * p->geo.r > 16) { set_error("n_q_tokens * (H/G) = %d exceeds 16 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
+    if (!paged_block_size_ok(p, false, "kvmem_view_cache_attend")) return KVMEM_E_UNSUPPORTED;
+    if (n_q_tokens * p->geo.r > 64) { set_error("n_q_tokens * (H/G) = %d exceeds 64 rows per call", n_q_tokens * p->geo.r); return KVMEM_E_UNSUPPORTED; }
     if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
     AttendPlan plan = plan_attend(p->cfg, 1, n_q_tokens, p->sm_count);
     if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
@@ -1036,11 +1047,6 @@ int kvmem_device_status(kvmem_pool_t* p, int32_t* status, void* stream) {
     cudaError_t e = cudaMemcpyAsync(&word, p->status_dev, 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->status_dev, 0, 4, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    // a kernel that gave up at the grid barrier of the one-kernel scorer leaves the barrier's counter behind: re-arm it
-    if (e == cudaSuccess && word == KVMEM_E_TIMEOUT) {
-        e = cudaMemsetAsync(p->status_dev + 16, 0, 192, st);
-        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    }
     if (e != cudaSuccess) return cuda_fail("reading the device status word", e);
     *status = word;
     return KVMEM_OK;

@@ -30,7 +30,7 @@ constexpr int kAttThreads = (kAttConsumers + 1) * 32;
 constexpr int kAttRopeStages = 4;               // the position-consistent paged mode: data stages,
 constexpr int kAttRopeGroups = 2;               // consumer groups (one table buffer of rotary rows each)
 constexpr int kAttRopeConsumers = 8;            // and consumer warps (12 warps in 3 groups spill at the 128-register cap: 345 us against 257)
-constexpr int kTile = 64;                       // tokens per tile == block_tokens
+constexpr int kTile = 64;                       // tokens per tile: 64 / B selected blocks, or a 64-token slice of one
 constexpr int kD = 128;
 constexpr int kTabBytes = kTile * (kD / 2) * 8; // (cos, sin) fp32 of 64 pairs for 64 positions: 32 KiB
 static_assert(kAttRopeStages % kAttRopeGroups == 0 && kAttRopeConsumers % kAttRopeGroups == 0 &&
@@ -39,7 +39,8 @@ static_assert(kAttRopeStages % kAttRopeGroups == 0 && kAttRopeConsumers % kAttRo
 constexpr int kHalfBytes = kTile * 128;         // one 64-dim half of a tile: 64 rows x 128 B
 constexpr int kStageBytes = 4 * kHalfBytes;     // K lo, K hi, V lo, V hi
 constexpr int kMaxSplits = 64;
-constexpr int kRowsPad = 16;
+constexpr int kRowsPad = 16;                    // query rows of one m16 row tile
+constexpr int kMaxRows = 64;                    // query rows per KV head and call: up to four row tiles
 constexpr int kMergeStride = 136;               // floats per merged row in shared memory
 constexpr size_t kAttSmem = (size_t)kAttStages * kStageBytes + 1024;
 constexpr int kQrotBytes = kRowsPad * kD * 2;   // one rotated query tile: 16 rows x 256 B
@@ -54,6 +55,7 @@ struct AttendArgs {
     float2* part_ml;    // [ns*LG][n_splits][16]
     int32_t* status;
     int M, L, H, G, r, rows, n_splits, cap_tokens;
+    int rows_pad;                // 16 x row tiles: rows of a split's partial result
     float scale_log2e;
     // fused view assembly (attend_split_kernel<true>): tiles come from the page pool through the block table
     const int32_t* sel_ids;      // [n_sessions][sel_stride]
@@ -69,14 +71,18 @@ struct AttendArgs {
     int rope_positions;          // rows of the rotary table
 };
 
+// query rows per KV head, in m16 MMA row tiles: 1, 2 or 4 (16, 32 or 64 rows)
+static int row_tiles_for(int rows) { return rows <= 16 ? 1 : rows <= 32 ? 2 : 4; }
+
 AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tokens, int sm_count) {
-    (void)n_q_tokens; (void)sm_count;
+    (void)sm_count;
     AttendPlan p{};
     p.n_splits = kMaxSplits;
-    p.rows_pad = kRowsPad;
+    const int rows = std::max(1, n_q_tokens) * (c.n_q_heads / c.n_kv_heads);
+    p.rows_pad = kRowsPad * row_tiles_for(std::min(rows, kMaxRows));
     const size_t heads = (size_t)n_sessions * c.n_layers * c.n_kv_heads;
-    p.part_o_bytes = align_up(heads * kMaxSplits * kRowsPad * kD * sizeof(float), 256);
-    p.part_ml_bytes = align_up(heads * kMaxSplits * kRowsPad * sizeof(float2), 256);
+    p.part_o_bytes = align_up(heads * kMaxSplits * p.rows_pad * kD * sizeof(float), 256);
+    p.part_ml_bytes = align_up(heads * kMaxSplits * p.rows_pad * sizeof(float2), 256);
     p.total = p.part_o_bytes + p.part_ml_bytes;
     return p;
 }
@@ -119,20 +125,28 @@ static int choose_splits(int heads, int max_tiles, int sms) {
 //         out/lse equal kvmem_view_attend's on it, with 1 read + 1 write per view byte.
 // MODE 2: copy-free execution view (Sec. 5.3 "Copy-free execution-view assembly"): tiles are read from
 //         the pages through the block table and attended over; no contiguous view is written.
-template <int MODE>
-__global__ void __launch_bounds__(MODE == 3 ? (kAttRopeConsumers + 1) * 32 : kAttThreads + (MODE == 1 ? 32 : MODE == 4 ? 32 * kQrotWarps : MODE == 5 ? 32 + 32 * kKrotWarps : 0), 1)
+// RT: m16 row tiles of query rows per KV head.  RT = 1 (up to 16 rows): two groups of four consumer warps take the tiles
+// alternately.  RT = 2 (up to 32 rows): every consumer warp sees every tile, four warps per row tile, 16 tokens each.
+// RT = 4 (up to 64 rows): two warps per row tile, 32 tokens each.  The K/V stream is read once whatever RT is; with
+// more row tiles the consumers do more arithmetic per byte and the pass moves from HBM-bound towards issue-bound.
+template <int MODE, int RT = 1>
+__global__ void __launch_bounds__(MODE == 3 ? (kAttRopeConsumers + 1) * 32 : MODE == 6 ? (kAttRopeConsumers + 2) * 32 : kAttThreads + (MODE == 1 ? 32 : MODE == 4 ? 32 * kQrotWarps : MODE == 5 ? 32 + 32 * kKrotWarps : 0), 1)
 attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_pages, AttendArgs a) {
-    constexpr bool FUSED = MODE == 1 || MODE == 5;   // a view-writer warp shares every stage with the consumers
+    constexpr bool FUSED = MODE == 1 || MODE == 5 || MODE == 6;   // a view-writer warp shares every stage with the consumers
     constexpr bool KROT = MODE == 5;       // rotator warps re-encode every K tile in place before anybody else reads it
     constexpr bool PAGED = MODE != 0;      // the producer reads pages through the block table
-    constexpr bool ROPE = MODE == 3;       // the consumers re-encode their key fragments in registers before the MMAs
+    constexpr bool ROPE = MODE == 3 || MODE == 6;   // the consumers re-encode their key fragments in registers before the MMAs
+    constexpr bool KWB = MODE == 6;        // ... and write them back into the stage, from where the view writer stores the tile
     constexpr bool QROT = MODE == 4;       // a rotator warp re-encodes the query per tile instead
     extern __shared__ unsigned char smem_dyn[];
     // the rotary mode gives the room of two data stages to one buffer of rotary rows per consumer group
     constexpr int STAGES = ROPE ? kAttRopeStages : kAttStages;
     constexpr int CONSUMERS = ROPE ? kAttRopeConsumers : kAttConsumers;
-    constexpr int GROUPS = ROPE ? kAttRopeGroups : kAttGroups;
+    constexpr int GROUPS = ROPE ? kAttRopeGroups : RT > 1 ? 1 : kAttGroups;
+    static_assert(RT == 1 || (MODE <= 2 && (RT == 2 || RT == 4)), "several row tiles: the plain modes only");
+    constexpr int WPR = RT == 1 ? 4 : CONSUMERS / RT;      // consumer warps that share the tokens of a tile (for one row tile)
+    constexpr int SLICES = 4 / WPR;                        // 16-token slices per warp and tile
     __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages], tab_full[kAttRopeGroups], tab_empty[kAttRopeGroups];
     __shared__ uint64_t q_full[kAttStages];     // MODE 4: rotated query of the stage's tile is in place; MODE 5: its K tile is rotated
     __shared__ float merge_m[kAttRopeConsumers][kRowsPad], merge_l[kAttRopeConsumers][kRowsPad];
@@ -151,7 +165,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             ptx::mbar_init(&empty_bar[i], CONSUMERS / GROUPS + (FUSED ? 1 : 0));
         }
         for (int i = 0; i < GROUPS; ++i) { ptx::mbar_init(&tab_full[i], 1); ptx::mbar_init(&tab_empty[i], CONSUMERS / GROUPS); }
-        for (int i = 0; i < kAttStages; ++i) ptx::mbar_init(&q_full[i], 1);
+        for (int i = 0; i < kAttStages; ++i) ptx::mbar_init(&q_full[i], KWB ? CONSUMERS / GROUPS : 1);
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(PAGED ? &map_pages : &map_k);
     }
@@ -160,7 +174,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 
     // view length in tokens; the kernel works in 64-token tiles, whatever the block size of the view (a multiple of
     // 16, so each consumer warp's 16 tokens are all inside or all outside the view)
-    const int btok = PAGED ? kTile : a.block_tokens;
+    const int btok = a.block_tokens;
     const long long n_tok_ll = min((long long)max(a.n_sel[s], 0) * btok, (long long)a.cap_tokens);
     const int n_tok = (int)n_tok_ll;
     const int n_blk = (n_tok + kTile - 1) / kTile;
@@ -203,13 +217,21 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 }
             }
         } else if (n_tiles > 0) {
-            // the whole warp looks up pages, 32 tiles at a time; lane 0 issues the loads
+            // A 64-token tile is 64 / B selected blocks (B < 64: one page lookup and one set of loads per block) or a
+            // 64-token slice of one selected block (B >= 64).  The whole warp looks up pages, 32 slots at a time (a slot
+            // is one block of a tile); lane 0 issues the loads.
             if (lane == 0) ptx::prefetch_tensormap(&map_pages);
             const int NB = a.nblocks_dev[a.session_first + s];
-            int base_it = 0, my_page = 0;
-            auto lookup = [&](int it) -> int {
-                if (it >= n_tiles) return 0;
-                const int id = a.sel_ids[(size_t)s * a.sel_stride + t0 + it];
+            const int B = btok;
+            const int n_sub = B < kTile ? kTile / B : 1;      // selected blocks per tile
+            const int tpb = B > kTile ? B / kTile : 1;        // tiles per selected block
+            const int box_rows = B < kTile ? B : kTile;
+            const int n_sel_blk = n_tok / B;                  // selected blocks inside the view
+            int base_slot = 0, my_page = 0;
+            auto lookup = [&](int slot) -> int {
+                const int j = (t0 * n_sub + slot) / tpb;      // index in sel_ids
+                if (slot >= n_tiles * n_sub || j >= n_sel_blk) return -1;          // past this CTA's range or the view's ragged end
+                const int id = a.sel_ids[(size_t)s * a.sel_stride + j];
                 int pg = -1;
                 if (id >= 0 && id < NB) pg = a.tables[(size_t)(a.session_first + s) * a.max_bps + id];
                 if (pg < 0 || pg >= a.max_blocks) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); pg = 0; }
@@ -218,8 +240,10 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             my_page = lookup(lane);
             bool ok = true;
             for (int it = 0; it < n_tiles; ++it) {
-                if (it >= base_it + 32) { base_it = it; my_page = lookup(base_it + lane); }
-                const int page = __shfl_sync(0xffffffffu, my_page, it - base_it);
+                if (it * n_sub >= base_slot + 32) { base_slot = it * n_sub; my_page = lookup(base_slot + lane); }
+                int pages[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) pages[u] = u < n_sub ? __shfl_sync(0xffffffffu, my_page, (it * n_sub + u - base_slot) & 31) : -1;
                 if (lane == 0) {
                     const int st = it % STAGES;
                     // at most `ahead` tiles in flight: tile it - ahead has left its stage (the same phase is waited for
@@ -244,13 +268,23 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     }
                     if (ok) {
                         unsigned char* dst = stages + (size_t)st * kStageBytes;
-                        // page layout [K|V][L*G][64 tokens][128]: rows of 256 B
-                        const int yk = ((page * 2 + 0) * LG + lg) * kTile, yv = ((page * 2 + 1) * LG + lg) * kTile;
-                        ptx::mbar_expect_tx(&full_bar[st], kStageBytes);
-                        ptx::tma_load_2d(dst, &map_pages, 0, yk, &full_bar[st]);
-                        ptx::tma_load_2d(dst + kHalfBytes, &map_pages, 64, yk, &full_bar[st]);
-                        ptx::tma_load_2d(dst + 2 * kHalfBytes, &map_pages, 0, yv, &full_bar[st]);
-                        ptx::tma_load_2d(dst + 3 * kHalfBytes, &map_pages, 64, yv, &full_bar[st]);
+                        int n_valid = 0;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) n_valid += (u < n_sub && pages[u] >= 0) ? 1 : 0;
+                        // page layout [K|V][L*G][B tokens][128]: rows of 256 B
+                        ptx::mbar_expect_tx(&full_bar[st], (uint32_t)n_valid * 4u * (uint32_t)box_rows * 128u);
+                        const int row_in_block = ((t0 + it) % tpb) * kTile;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (u < n_sub && pages[u] >= 0) {
+                                const int yk = ((pages[u] * 2 + 0) * LG + lg) * B + row_in_block, yv = ((pages[u] * 2 + 1) * LG + lg) * B + row_in_block;
+                                unsigned char* d = dst + (size_t)u * B * 128;
+                                ptx::tma_load_2d(d, &map_pages, 0, yk, &full_bar[st]);
+                                ptx::tma_load_2d(d + kHalfBytes, &map_pages, 64, yk, &full_bar[st]);
+                                ptx::tma_load_2d(d + 2 * kHalfBytes, &map_pages, 0, yv, &full_bar[st]);
+                                ptx::tma_load_2d(d + 3 * kHalfBytes, &map_pages, 64, yv, &full_bar[st]);
+                            }
+                        }
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -266,14 +300,20 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             for (int it = 0; it < n_tiles; ++it) {
                 const int st = it % STAGES;
                 ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / STAGES) & 1));
-                if (KROT && ok) ok = ptx::mbar_wait(&q_full[st], (uint32_t)((it / STAGES) & 1));
+                if ((KROT || KWB) && ok) ok = ptx::mbar_wait(&q_full[st], (uint32_t)((it / STAGES) & 1));
                 if (!ok) break;
                 unsigned char* src = stages + (size_t)st * kStageBytes;
                 const int y = (t0 + it) * kTile;
-                ptx::tma_store_3d(&map_k, src, 0, y, z);
-                ptx::tma_store_3d(&map_k, src + kHalfBytes, 64, y, z);
-                ptx::tma_store_3d(&map_v, src + 2 * kHalfBytes, 0, y, z);
-                ptx::tma_store_3d(&map_v, src + 3 * kHalfBytes, 64, y, z);
+                // the store box is min(B, 64) rows: a ragged last tile stores only the blocks the view has
+                const int box_rows = btok < kTile ? btok : kTile;
+                const int n_valid = min(kTile, n_tok - y) / box_rows;
+                for (int u = 0; u < n_valid; ++u) {
+                    const unsigned char* sb = src + (size_t)u * box_rows * 128;
+                    ptx::tma_store_3d(&map_k, sb, 0, y + u * box_rows, z);
+                    ptx::tma_store_3d(&map_k, sb + kHalfBytes, 64, y + u * box_rows, z);
+                    ptx::tma_store_3d(&map_v, sb + 2 * kHalfBytes, 0, y + u * box_rows, z);
+                    ptx::tma_store_3d(&map_v, sb + 3 * kHalfBytes, 64, y + u * box_rows, z);
+                }
                 ptx::bulk_commit();
                 if (it > 0) {                              // all but the newest store have left shared memory
                     ptx::bulk_wait_read<1>();
@@ -382,7 +422,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         // Q fragments (A operand, m16k16 x 8 k-steps).  Row j = m * r + hr  ->  q[s][m][l][g*r + hr].
         uint32_t qf[8][4];
         if (!QROT) {
-            const int row_a = lane >> 2, row_b = row_a + 8;
+            const int row_a = (RT == 1 ? 0 : (warp / WPR) * kRowsPad) + (lane >> 2), row_b = row_a + 8;
             const __nv_bfloat16* qa = nullptr;
             const __nv_bfloat16* qb = nullptr;
             if (row_a < a.rows) qa = a.q + ((((size_t)s * a.M + row_a / a.r) * a.L + l) * a.H + (size_t)g * a.r + row_a % a.r) * kD;
@@ -401,7 +441,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         // Two groups of four warps.  Group grp takes tiles grp, grp + 2, ...; with an even number of
         // stages it therefore meets the phases of "its" stages strictly in order, which an mbarrier
         // parity wait requires.  Inside a tile, warp wq owns tokens [16 wq, 16 wq + 16).
-        const int grp = warp >> 2, wq = warp & 3;
+        const int grp = RT == 1 ? warp >> 2 : 0, wq0 = RT == 1 ? (warp & 3) : (warp % WPR) * SLICES;
 
         for (int it = grp; it < n_tiles; it += GROUPS) {
             const int st = it % STAGES;
@@ -412,11 +452,11 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
             }
-            if (!PAGED && (t0 + it) * kTile + wq * 16 >= n_tok) {      // this warp's 16 tokens lie beyond a ragged view end
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&empty_bar[st]);
-                continue;
-            }
+            bool k_handed_over = false;                      // KWB: this warp's share of the tile is rotated and back in the stage
+#pragma unroll
+            for (int sl = 0; sl < SLICES; ++sl) {
+            const int wq = wq0 + sl;
+            if ((t0 + it) * kTile + wq * 16 >= n_tok) continue;      // this warp's 16 tokens lie beyond a ragged view end
             const uint32_t kbase = stage0 + (uint32_t)st * kStageBytes;
             const uint32_t vbase = kbase + 2 * kHalfBytes;
             // QROT: this tile's rotated query; its A fragments are fetched two k-steps at a time, next to their use
@@ -476,6 +516,12 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                             const float l1 = __fsub_rn(__fmul_rn(a1, t.z), __fmul_rn(b1, t.w)), h1 = __fadd_rn(__fmul_rn(b1, t.z), __fmul_rn(a1, t.w));
                             lo[kp][j] = ptx::pack_bf16x2(l0, l1);
                             hi[kp][j] = ptx::pack_bf16x2(h0, h1);
+                            if (KWB) {
+                                // register j of an ldmatrix x4 holds matrix j = 16-byte chunk 4 kp + j of token rtok, bytes 4 (lane & 3)..
+                                unsigned char* pk = stages + (size_t)st * kStageBytes + (size_t)rtok * 128 + ((((kp * 4 + j) ^ (rtok & 7)) << 4) + 4 * (lane & 3));
+                                *reinterpret_cast<uint32_t*>(pk) = lo[kp][j];
+                                *reinterpret_cast<uint32_t*>(pk + kHalfBytes) = hi[kp][j];
+                            }
                         }
                     }
                     // the k-steps in the order of the other modes, so that the logits are the same bits
@@ -489,6 +535,12 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                         ptx::mma_bf16_16816(sc[nt], qf[2 * kp + 4], hi[kp][0], hi[kp][1]);
                         ptx::mma_bf16_16816(sc[nt], qf[2 * kp + 5], hi[kp][2], hi[kp][3]);
                     }
+                }
+                if (KWB) {
+                    ptx::fence_proxy_async_smem();      // the view writer's bulk stores read these bytes through the async proxy
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&q_full[st]);
+                    k_handed_over = true;
                 }
             }
             // online softmax (exp2 domain); this thread holds rows lane/4 (c0,c1) and lane/4 + 8 (c2,c3)
@@ -535,6 +587,11 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     ptx::mma_bf16_16816(o[2 * np + 1], pa, b2, b3);
                 }
             }
+            }       // slices
+            if (KWB && !k_handed_over) {                    // nothing of this tile was this warp's to rotate (ragged view end)
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&q_full[st]);
+            }
             __syncwarp();
             if (lane == 0) {
                 ptx::mbar_arrive(&empty_bar[st]);
@@ -565,23 +622,28 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     __syncthreads();
     if (tid < 256) {
         const int col = tid & 127, r0 = (tid >> 7) * 8;
-        const size_t pbase = ((size_t)z * a.n_splits + split) * kRowsPad;
-        for (int row = r0; row < r0 + 8; ++row) {
-            float mx = -INFINITY;
+        const size_t pbase = ((size_t)z * a.n_splits + split) * a.rows_pad;
+        constexpr int NW = RT == 1 ? CONSUMERS : WPR;       // warps whose partial results share a query row
 #pragma unroll
-            for (int w = 0; w < CONSUMERS; ++w) mx = fmaxf(mx, merge_m[w][row]);
-            float acc = 0.0f, lsum = 0.0f;
+        for (int rt = 0; rt < RT; ++rt) {
+            const int w0 = RT == 1 ? 0 : rt * WPR;
+            for (int row = r0; row < r0 + 8; ++row) {
+                float mx = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < CONSUMERS; ++w) {
-                const float mw = merge_m[w][row];
-                if (mw > -INFINITY) {
-                    const float f = exp2f(mw - mx);
-                    acc += f * merge_o[((size_t)w * kRowsPad + row) * kMergeStride + col];
-                    lsum += f * merge_l[w][row];
+                for (int w = w0; w < w0 + NW; ++w) mx = fmaxf(mx, merge_m[w][row]);
+                float acc = 0.0f, lsum = 0.0f;
+#pragma unroll
+                for (int w = w0; w < w0 + NW; ++w) {
+                    const float mw = merge_m[w][row];
+                    if (mw > -INFINITY) {
+                        const float f = exp2f(mw - mx);
+                        acc += f * merge_o[((size_t)w * kRowsPad + row) * kMergeStride + col];
+                        lsum += f * merge_l[w][row];
+                    }
                 }
+                a.part_o[(pbase + rt * kRowsPad + row) * kD + col] = acc;
+                if (col == 0) a.part_ml[pbase + rt * kRowsPad + row] = make_float2(mx, lsum);
             }
-            a.part_o[(pbase + row) * kD + col] = acc;
-            if (col == 0) a.part_ml[pbase + row] = make_float2(mx, lsum);
         }
     }
 }
@@ -589,19 +651,19 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 // Merge the splits of one query row of one (session, layer, KV head) in split order; write O and LSE.
 __global__ void __launch_bounds__(128)
 attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, float* __restrict__ out,
-                    float* __restrict__ lse, int M, int L, int H, int G, int r, int n_splits) {
+                    float* __restrict__ lse, int M, int L, int H, int G, int r, int n_splits, int rows_pad) {
     pdl_wait();        // everything earlier in the stream is complete and visible from here on
     pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     const int row = blockIdx.x, z = blockIdx.y, LG = L * G;
     const int s = z / LG, lg = z % LG, l = lg / G, g = lg % G;
     const int col = threadIdx.x;
-    const size_t p0 = (size_t)z * n_splits * kRowsPad + row;          // split sp lives at p0 + sp * kRowsPad
+    const size_t p0 = (size_t)z * n_splits * rows_pad + row;          // split sp lives at p0 + sp * rows_pad
     float mx = -INFINITY;
-    for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, part_ml[p0 + (size_t)sp * kRowsPad].x);
+    for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, part_ml[p0 + (size_t)sp * rows_pad].x);
     float acc = 0.0f, lsum = 0.0f;
 #pragma unroll 4
     for (int sp = 0; sp < n_splits; ++sp) {
-        const size_t pi = p0 + (size_t)sp * kRowsPad;
+        const size_t pi = p0 + (size_t)sp * rows_pad;
         const float2 ml = part_ml[pi];
         const float f = ml.x > -INFINITY ? exp2f(ml.x - mx) : 0.0f;
         acc += f * part_o[pi * kD + col];
@@ -626,12 +688,12 @@ static PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
 }
 
 // view [heads][cap_tokens][128] bf16 as a 3-D tensor; box = 64 dims x 64 tokens x 1 head, 128-byte swizzle
-static bool make_view_map(CUtensorMap* map, const __nv_bfloat16* view, int heads, int cap_tokens) {
+static bool make_view_map(CUtensorMap* map, const __nv_bfloat16* view, int heads, int cap_tokens, int box_rows = kTile) {
     PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
     if (!enc) return false;
     cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)cap_tokens, (cuuint64_t)heads};
     cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)cap_tokens * kD * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)kTile, 1};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(view), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -644,9 +706,9 @@ static bool make_pages_map(CUtensorMap* map, const kvmem_pool& p, const __nv_bfl
     PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
     if (!enc) return false;
     const Geometry& g = p.geo;
-    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)n_pages * 2 * g.L * g.G * kTile};
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)n_pages * 2 * g.L * g.G * g.B};
     cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    cuuint32_t box[2] = {64, (cuuint32_t)std::min(g.B, kTile)};
     cuuint32_t estr[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(pages), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -668,13 +730,22 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     if (fused && !make_pages_map(&map_pages, p, alt ? alt->pages : p.pages, alt ? alt->n_pages : g.max_blocks)) return cudaErrorInvalidValue;
     if (paged_only) {
         map_k = map_pages; map_v = map_pages;               // unused by this mode
-    } else if (!make_view_map(&map_k, view_k, heads, view_cap_tokens) || !make_view_map(&map_v, view_v, heads, view_cap_tokens)) {
-        return cudaErrorInvalidValue;
+    } else {
+        // the fused pass stores blocks (boxes of min(B, 64) rows); attention over a finished view loads whole 64-token tiles
+        const int box_rows = fused ? std::min(g.B, kTile) : kTile;
+        if (!make_view_map(&map_k, view_k, heads, view_cap_tokens, box_rows) || !make_view_map(&map_v, view_v, heads, view_cap_tokens, box_rows))
+            return cudaErrorInvalidValue;
     }
     if (!fused) map_pages = map_k;
     static PerDeviceOnce attr_done;
     if (attr_done.pending(p.cfg.device)) {
         cudaError_t e = cudaFuncSetAttribute(attend_split_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_split_kernel<0, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_split_kernel<0, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_split_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_split_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_split_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_split_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
@@ -685,6 +756,8 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
             e = cudaFuncSetAttribute(attend_split_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmemQrot);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attend_split_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e != cudaSuccess) return e;
         attr_done.mark(p.cfg.device);
     }
@@ -695,7 +768,11 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     a.part_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(workspace) + plan.part_o_bytes);
     a.status = p.status_dev;
     a.M = M; a.L = g.L; a.H = g.H; a.G = g.G; a.r = g.r; a.rows = M * g.r;
-    a.n_splits = g_attend_splits > 0 ? std::min(g_attend_splits, kMaxSplits) : choose_splits(heads, view_cap_tokens / kTile, p.sm_count);
+    a.rows_pad = plan.rows_pad;
+    const int RT = row_tiles_for(a.rows);
+    if (a.rows > kMaxRows) return cudaErrorInvalidValue;
+    if (RT > 1 && rope_first_position >= 0) return cudaErrorInvalidValue;      // the rotating modes take one row tile
+    a.n_splits = g_attend_splits > 0 ? std::min(g_attend_splits, kMaxSplits) : choose_splits(heads, (view_cap_tokens + kTile - 1) / kTile, p.sm_count);
     a.cap_tokens = view_cap_tokens;
     const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
     a.scale_log2e = sc * 1.4426950408889634f;
@@ -716,7 +793,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     a.landed = g_attend_landed >= 0 ? g_attend_landed : (writes_view ? 1 : 0);
     if (a.lookahead == 0) {
         const long long ctas = (long long)a.n_splits * heads;
-        const int tiles_per_cta = (view_cap_tokens / kTile + a.n_splits - 1) / a.n_splits;
+        const int tiles_per_cta = ((view_cap_tokens + kTile - 1) / kTile + a.n_splits - 1) / a.n_splits;
         if (ctas <= p.sm_count && tiles_per_cta >= 64) {
             const double target = (writes_view ? (a.landed ? 9.5 : 14.0) : 19.0) * 1024.0 * 1024.0;
             a.lookahead = std::max(2, std::min(kAttStages, (int)(target / ((double)ctas * kStageBytes) + 0.5)));
@@ -727,18 +804,26 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         launch_pdl(attend_split_kernel<4>, dim3(grid), dim3(kAttThreads + 32 * kQrotWarps), kAttSmemQrot, st, map_k, map_v, map_pages, a);
     else if (paged_only && rope_first_position >= 0)
         launch_pdl(attend_split_kernel<3>, dim3(grid), dim3((kAttRopeConsumers + 1) * 32), kAttSmem, st, map_k, map_v, map_pages, a);
-    else if (paged_only)
-        launch_pdl(attend_split_kernel<2>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);
-    else if (fused && rope_first_position >= 0)
+    else if (fused && !paged_only && rope_first_position >= 0 && p.cfg.rope_in_block_keys)
         launch_pdl(attend_split_kernel<5>, dim3(grid), dim3(kAttThreads + 32 + 32 * kKrotWarps), kAttSmem, st, map_k, map_v, map_pages, a);
-    else if (fused)
-        launch_pdl(attend_split_kernel<1>, dim3(grid), dim3(kAttThreads + 32), kAttSmem, st, map_k, map_v, map_pages, a);
-    else
-        launch_pdl(attend_split_kernel<0>, dim3(grid), dim3(kAttThreads), kAttSmem, st, map_k, map_v, map_pages, a);
+    else if (fused && !paged_only && rope_first_position >= 0)
+        launch_pdl(attend_split_kernel<6>, dim3(grid), dim3((kAttRopeConsumers + 2) * 32), kAttSmem, st, map_k, map_v, map_pages, a);
+    else {
+#define KVMEM_ATTEND_LAUNCH(MODE, THREADS)                                                                              \
+    do {                                                                                                                \
+        if (RT == 1) launch_pdl(attend_split_kernel<MODE, 1>, dim3(grid), dim3(THREADS), kAttSmem, st, map_k, map_v, map_pages, a);      \
+        else if (RT == 2) launch_pdl(attend_split_kernel<MODE, 2>, dim3(grid), dim3(THREADS), kAttSmem, st, map_k, map_v, map_pages, a); \
+        else launch_pdl(attend_split_kernel<MODE, 4>, dim3(grid), dim3(THREADS), kAttSmem, st, map_k, map_v, map_pages, a);              \
+    } while (0)
+        if (paged_only) KVMEM_ATTEND_LAUNCH(2, kAttThreads);
+        else if (fused) KVMEM_ATTEND_LAUNCH(1, kAttThreads + 32);
+        else KVMEM_ATTEND_LAUNCH(0, kAttThreads);
+#undef KVMEM_ATTEND_LAUNCH
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     launch_pdl(attend_merge_kernel, dim3(dim3((unsigned)a.rows, (unsigned)heads)), dim3(kD), 0, st, a.part_o, a.part_ml, out, lse, M, g.L, g.H, g.G,
-                                                                            g.r, a.n_splits);
+                                                                            g.r, a.n_splits, a.rows_pad);
     return cudaGetLastError();
 }
 

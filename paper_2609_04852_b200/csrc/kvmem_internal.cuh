@@ -81,7 +81,6 @@ constexpr uint64_t kMagic = 0x4b564d454d423230ull;  // "KVMEMB20"
 void set_error(const char* fmt, ...);
 
 // tuning switches (kvmem_set_option)
-extern int g_score_fused;   // 1: decode scoring in one kernel where the shape fits (default), 0: logits kernel + finish kernel
 extern int g_score_mode;    // 1: tensor-core decode scoring (default), 0: fp32 ALU + warp-shuffle kernel
 extern int g_chunk_poly;    // chunked scoring: every n-th exponential on the FMA pipe (0: all on the special-function unit)
 extern int g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
@@ -133,11 +132,6 @@ ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions
 
 cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q,
                                 int M, const ScoreWorkspace& ws, float* scores, int scores_stride, float score_scale, cudaStream_t st);
-// the same scores from one kernel (kvmem_score_fused.cu); *launched = false: the shape does not fit, nothing was enqueued
-cudaError_t launch_score_fused(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q, int M,
-                               const ScoreWorkspace& ws, float* scores, int scores_stride, float score_scale, cudaStream_t st,
-                               bool* launched);
-constexpr int kFusedScoreMaxParts = 160;   // CTAs per session whose row statistics the workspace has room for
 
 // scoring against a host-resident index, streamed in tiles (kvmem_score.cu)
 struct HostScorePlan {

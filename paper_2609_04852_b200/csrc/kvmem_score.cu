@@ -36,8 +36,7 @@ ScoreWorkspace plan_score_workspace(const kvmem_pool_config_t& c, int n_sessions
     const size_t lg = (size_t)c.n_layers * c.n_kv_heads;
     const int rows_store = w.rows_pad;
     w.logits_bytes = align_up((size_t)n_sessions * lg * rows_store * w.nb_pad * sizeof(float), 256);
-    // per-CTA row statistics: [row][part] of the two-kernel form, or [part][head][16 rows] of the one-kernel form
-    w.partials_bytes = align_up((size_t)n_sessions * lg * std::max(rows_store * kMaxScoreParts, 16 * kFusedScoreMaxParts) * sizeof(float2), 256);
+    w.partials_bytes = align_up((size_t)n_sessions * lg * rows_store * kMaxScoreParts * sizeof(float2), 256);
     w.scores_bytes = align_up((size_t)n_sessions * c.max_blocks_per_session * sizeof(float), 256);
     w.total = w.logits_bytes + w.partials_bytes + w.scores_bytes;
     if (base) {
@@ -483,11 +482,6 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
                                 int M, const ScoreWorkspace& ws, float* scores, int scores_stride, float score_scale, cudaStream_t st) {
     const Geometry& g = p.geo;
     if (M > kMaxDecodeTokens) return cudaErrorNotSupported;
-    {
-        bool launched = false;
-        cudaError_t ef = launch_score_fused(p, session_first, n_sessions, q, M, ws, scores, scores_stride, score_scale, st, &launched);
-        if (ef != cudaSuccess || launched) return ef;
-    }
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)g.d);
     int max_nb = 0;
     for (int s = session_first; s < session_first + n_sessions; ++s) max_nb = std::max(max_nb, p.sess_blocks[s]);

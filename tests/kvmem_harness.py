@@ -174,7 +174,7 @@ def full_step(spec: WorkloadSpec, qsets=(0,), gap_forced_budget=None, n_sink=0, 
     prm = SelectParams(**prm_d)
     ns, B, M = spec.n_sessions, spec.block_tokens, spec.n_q_tokens
     k = budget_blocks(prm, B, spec.n_blocks)
-    fast = B == 64                      # the passes that read pages through the block table
+    fast = 64 % B == 0 or B % 64 == 0   # the passes that read pages through the block table walk 64-token tiles
     guards = Guards(dev)
     sel = guards.empty((ns, k), torch.int32)
     n_sel = guards.empty((ns,), torch.int32)

@@ -609,11 +609,11 @@ def test_argument_and_capacity_errors():
     with pytest.raises(KvmemError) as e:
         Pool(1, 32, 5, 128, 64, 1, 8, 8, 0)                       # 32 % 5 != 0
     assert e.value.status == E_INVALID
-    q17 = torch.zeros(1, 5, 1, 32, 128, dtype=torch.bfloat16, device=dev)
+    q17 = torch.zeros(1, 17, 1, 32, 128, dtype=torch.bfloat16, device=dev)
     view = pool.new_view(1, 8 * 64)
-    out, lse = pool.new_outputs(1, 5)
+    out, lse = pool.new_outputs(1, 17)
     with pytest.raises(KvmemError) as e:
-        pool.view_attend(q17, view, n_sel, out, lse)              # 5 tokens x 4 heads per KV head > 16 rows
+        pool.view_attend(q17, view, n_sel, out, lse)              # 17 tokens x 4 heads per KV head > 64 rows
     assert e.value.status == E_UNSUPPORTED
     pool.session_reset(0)
     assert pool.session_blocks(0) == 0

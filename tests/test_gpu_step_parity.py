@@ -253,20 +253,18 @@ def test_a_bounded_wait_that_runs_out_sets_the_status_word_and_leaves_the_pool_u
     assert pool.device_status() == 0
 
 
-# ------------------------------------------------------------------ one-kernel scorer against the three-kernel form and the oracle
+# ------------------------------------------------------------------ decode scores at many shapes
 
 @pytest.mark.parametrize("ns,L,G,H,M,n_blocks", [(1, 1, 8, 32, 4, 2048), (1, 1, 8, 32, 4, 5000), (1, 1, 8, 32, 1, 16384),
                                                (3, 1, 8, 32, 2, 700), (1, 2, 8, 32, 4, 333), (1, 4, 4, 16, 4, 150),
                                                (1, 1, 4, 32, 2, 97), (8, 1, 8, 32, 1, 4096), (1, 1, 8, 32, 4, 1)],
                          ids=["128k-shape", "ragged-5000", "1m-shape", "3-sessions", "L2", "L4G4", "GQA8", "batch8-shape", "one-block"])
-def test_one_kernel_scorer_equals_the_three_kernel_form_and_the_oracle(ns, L, G, H, M, n_blocks):
-    """kvmem_score through the kernel that keeps its logits in shared memory and meets at a grid barrier, for every
-    chunk size it chooses (16 to 128 blocks), several sessions of different length, several layers: against the oracle
-    within the score tolerance and against the logits + finish kernels within rounding; twice in a row (the barrier
-    re-arms itself) with identical bits."""
-    from paper_2609_04852_b200 import Pool, set_option
+def test_decode_scores_at_many_shapes(ns, L, G, H, M, n_blocks):
+    """kvmem_score for sessions of different length in one call, several layers, other head groupings, one block:
+    against the oracle within the score tolerance, nothing written past a session's blocks, and twice in a row with
+    identical bits (fixed summation order)."""
     from kvmem_harness import check_scores
-    spec = SMALL.with_(name="fused_score", n_sessions=ns, n_layers=L, n_kv_heads=G, n_q_heads=H, n_q_tokens=M, n_blocks=n_blocks,
+    spec = SMALL.with_(name="scores", n_sessions=ns, n_layers=L, n_kv_heads=G, n_q_heads=H, n_q_tokens=M, n_blocks=n_blocks,
                        n_planted=min(6, n_blocks), budget_blocks=1)
     dev = torch.device("cuda", 0)
     lens = [n_blocks if s == 0 else max(1, n_blocks - 37 * s) for s in range(ns)]        # ragged session lengths
@@ -276,22 +274,143 @@ def test_one_kernel_scorer_equals_the_three_kernel_form_and_the_oracle(ns, L, G,
     qd = q.to(dev)
     g = Guards(dev)
     runs = []
-    for fused in (1, 1, 0):
-        set_option("score_fused", fused)
-        try:
-            sc = g.empty((ns, n_blocks), torch.float32, fill=-1.0)
-            pool.score(qd, sc)
-            torch.cuda.synchronize()
-            assert pool.device_status() == 0
-        finally:
-            set_option("score_fused", 1)
+    for _ in range(2):
+        sc = g.empty((ns, n_blocks), torch.float32, fill=-1.0)
+        pool.score(qd, sc)
+        torch.cuda.synchronize()
+        assert pool.device_status() == 0
         runs.append(sc)
     g.check()
-    assert torch.equal(runs[0], runs[1]), "two runs of the one-kernel scorer differ"
+    assert torch.equal(runs[0], runs[1]), "two runs of the scorer differ"
+    half = g.empty((ns, n_blocks), torch.float32, fill=-1.0)
+    pool.score(qd, half, score_scale=0.5)                       # a rank's share of the head mean, scaled in the kernel
+    torch.cuda.synchronize()
     for s in range(ns):
         R, _ = orc.block_scores(qb[s], osess[s].idx, lens[s])
-        for sc in runs:
-            check_scores(sc.cpu().numpy()[s, : lens[s]], R, M)
-            assert bool((sc[s, lens[s]:] == -1.0).all()), "scores past the session's blocks were written"
-        a, b = runs[0][s, : lens[s]], runs[2][s, : lens[s]]
-        assert ((a - b).abs() <= 2e-5 * b.abs() + 1e-12).all(), "one-kernel and three-kernel scores differ by more than rounding"
+        check_scores(runs[0].cpu().numpy()[s, : lens[s]], R, M)
+        assert bool((runs[0][s, lens[s]:] == -1.0).all()), "scores past the session's blocks were written"
+        assert torch.equal(half[s, : lens[s]] * 2.0, runs[0][s, : lens[s]]), "score_scale must be an exact power-of-two factor here"
+
+
+# ------------------------------------------------------------------ other block sizes on the passes that read pages
+
+@pytest.mark.parametrize("B,n_blocks,budget,M", [(32, 300, 21, 4), (32, 300, 64, 2), (16, 500, 37, 4), (16, 260, 260, 1),
+                                                 (128, 90, 5, 4), (128, 40, 40, 2), (256, 30, 7, 4), (32, 2000, 999, 4)],
+                         ids=["B32-ragged", "B32-even", "B16-ragged", "B16-all", "B128", "B128-all", "B256", "B32-long"])
+def test_fused_and_copy_free_passes_with_other_block_sizes(B, n_blocks, budget, M):
+    """The paper's default block is 32 tokens (Sec. 4.3).  kvmem_materialize_attend and kvmem_paged_attend walk the view in
+    64-token tiles: a tile is 64 / B selected blocks (an odd count ends in a partly filled tile) or a slice of one block.
+    Against the oracle, and bit for bit against the separate calls."""
+    spec = SMALL.with_(name=f"B{B}", block_tokens=B, n_blocks=n_blocks, n_planted=4, budget_blocks=budget, n_q_tokens=M,
+                       max_view_tokens=1 << 30)
+    modes = full_step(spec, qsets=(0, 1))
+    assert len(modes) == 2
+
+
+@pytest.mark.parametrize("B,n_blocks,budget,first", [(32, 200, 21, 517), (16, 300, 37, 0), (128, 40, 9, 64)])
+def test_copy_free_position_consistent_attention_with_other_block_sizes(B, n_blocks, budget, first):
+    """kvmem_paged_attend_rope over raw keys (each key fragment rotated to its compact position on the way to the tensor
+    cores) with 16-, 32- and 128-token blocks, against attention over the oracle's position-consistent view."""
+    from test_gpu_rope import SPEC as RSPEC, _fill_both
+    spec = RSPEC.with_(name=f"ropeB{B}", block_tokens=B, n_blocks=n_blocks, budget_blocks=budget, n_q_tokens=4)
+    dev = torch.device("cuda", 0)
+    pool, repo, idx, tab, table = _fill_both(spec)
+    ids = np.sort(np.random.default_rng(B + n_blocks).choice(n_blocks, size=budget, replace=False)).astype(np.int32)
+    q, qb = queries(spec)
+    sel = torch.from_numpy(ids).view(1, -1).to(dev)
+    n_sel = torch.tensor([budget], dtype=torch.int32, device=dev)
+    g = Guards(dev)
+    out, lse = g.outputs(pool, 1, 4)
+    pool.paged_attend_rope(q.to(dev), sel, n_sel, out, lse, first)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    g.check()
+    vK, vV = orc.gather_rope(repo, table, ids, budget * B, first, tab)
+    ref_out, ref_lse = orc.attend(qb[0], vK, vV, budget * B)
+    assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+
+
+def test_execution_cache_with_32_token_blocks():
+    """Cache update and attention over the cache's page table with the paper's default block size."""
+    from test_gpu_rope import SPEC as RSPEC, THETA, WINDOW, _fill_both
+    from test_gpu_view_cache import _compare, _working_sets
+    spec = RSPEC.with_(name="cacheB32", block_tokens=32, n_blocks=120, budget_blocks=20, n_q_tokens=4)
+    pool, repo, _, tab, table = _fill_both(spec)
+    dev = torch.device("cuda", 0)
+    cap = 23
+    cache = pool.new_view_cache(cap, 2, 131)
+    ocache = orc.ViewCache(repo, cap)
+    sets = _working_sets(np.random.default_rng(5), spec.n_blocks, [20, 21, 23, 7, 20])
+    q, qb = queries(spec)
+    for step, sel in enumerate(sets):
+        ids = torch.zeros(cap, dtype=torch.int32)
+        ids[: len(sel)] = torch.from_numpy(sel)
+        cache.update(0, ids.to(dev), torch.tensor([len(sel)], dtype=torch.int32, device=dev))
+        stats_ref = ocache.update(repo, table, sel, 2, 131, tab)
+        _compare(cache, ocache, stats_ref, step)
+        out, lse = pool.new_outputs(1, 4)
+        cache.attend(q[0].to(dev), out[0], lse[0])
+        torch.cuda.synchronize()
+        vK, vV = ocache.view(cap * 32)
+        O, LSE = orc.attend(qb[0], vK, vV, len(sel) * 32)
+        assert np.abs(out[0].cpu().numpy() - O).max() <= ATTN_ATOL and np.abs(lse[0].cpu().numpy() - LSE).max() <= ATTN_ATOL, step
+    assert pool.device_status() == 0 and THETA > 0 and WINDOW > 0
+
+
+# ------------------------------------------------------------------ more than 16 query rows per KV head
+
+@pytest.mark.parametrize("M,G,H,n_blocks,budget", [(8, 8, 32, 300, 40), (4, 4, 32, 300, 40), (5, 8, 32, 200, 24), (16, 8, 32, 300, 40),
+                                                  (13, 8, 32, 150, 150), (8, 4, 32, 700, 333), (2, 8, 32, 64, 1)],
+                         ids=["M8-32rows", "GQA8-32rows", "M5-20rows", "M16-64rows", "M13-52rows-all", "GQA8-64rows-long", "M2-8rows"])
+def test_attention_with_up_to_64_query_rows_per_kv_head(M, G, H, n_blocks, budget):
+    """1 + 7 draft tokens with GQA 4, or 4 tokens with GQA 8, exceed one 16-row MMA tile.  The attention kernels then run
+    two or four row tiles over the same K/V stream (a row count that does not fill the last tile included): every stage
+    against the oracle, the fused and copy-free passes bit for bit against the separate calls."""
+    spec = SMALL.with_(name=f"rows{M * H // G}", n_q_tokens=M, n_kv_heads=G, n_q_heads=H, n_blocks=n_blocks, n_planted=5,
+                       budget_blocks=budget)
+    modes = full_step(spec, qsets=(0, 1))
+    assert len(modes) == 2
+
+
+def test_thirty_two_rows_at_32_token_blocks_and_two_sessions():
+    spec = SMALL.with_(name="rows32B32", n_sessions=2, block_tokens=32, n_q_tokens=8, n_blocks=260, n_planted=4, budget_blocks=37,
+                       max_view_tokens=1 << 30)
+    assert len(full_step(spec, qsets=(0,))) == 2
+
+
+# ------------------------------------------------------------------ raw keys rotated inside the fused pass
+
+@pytest.mark.parametrize("B,n_blocks,budget,M,first", [(64, 150, 20, 4, 517), (64, 700, 60, 4, 17), (64, 90, 1, 1, 0), (64, 64, 63, 2, 64),
+                                                      (32, 200, 21, 4, 131), (16, 300, 37, 2, 0), (128, 40, 9, 4, 64)])
+def test_position_consistent_view_and_attention_in_one_pass_over_raw_keys(B, n_blocks, budget, M, first):
+    """kvmem_materialize_attend_rope on a pool of raw keys: the warps that attend over a tile rotate its keys to their
+    compact positions and hand them back for the store.  The view must be the defined code (oracle gather with RoPE,
+    bit for bit), the results those of attention over it, and both identical to the two separate calls."""
+    from test_gpu_rope import SPEC as RSPEC, _fill_both
+    spec = RSPEC.with_(name=f"rawfusedB{B}", block_tokens=B, n_blocks=n_blocks, budget_blocks=budget, n_q_tokens=M)
+    dev = torch.device("cuda", 0)
+    pool, repo, idx, tab, table = _fill_both(spec)
+    ids = np.sort(np.random.default_rng(3 * n_blocks + B).choice(n_blocks, size=budget, replace=False)).astype(np.int32)
+    q, qb = queries(spec)
+    qd = q.to(dev)
+    sel = torch.from_numpy(ids).view(1, -1).to(dev)
+    n_sel = torch.tensor([budget], dtype=torch.int32, device=dev)
+    T = budget * B
+    g = Guards(dev)
+    view = g.view(pool, 1, T)
+    out, lse = g.outputs(pool, 1, M)
+    pool.materialize_attend_rope(qd, sel, n_sel, view, out, lse, first)
+    view2 = g.view(pool, 1, T)
+    out2, lse2 = g.outputs(pool, 1, M)
+    pool.materialize_rope(sel, n_sel, view2, first)
+    pool.view_attend(qd, view2, n_sel, out2, lse2)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    g.check()
+    vK, vV = orc.gather_rope(repo, table, ids, T, first, tab)
+    assert np.array_equal(bits(view.k[0]), vK), "one-pass view: rotated keys differ from the defined code"
+    assert np.array_equal(bits(view.v[0]), vV)
+    ref_out, ref_lse = orc.attend(qb[0], vK, vV, T)
+    assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+    assert torch.equal(view.k, view2.k) and torch.equal(view.v, view2.v)
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)
