@@ -264,6 +264,46 @@ def working_set_delta(prev: np.ndarray, nxt: np.ndarray):
     return ret[: cnt[0]].copy(), inc[: cnt[1]].copy(), out[: cnt[2]].copy()
 
 
+# ---- incremental contiguous view (Eq. "kvmem-working-set-delta", Sec. 4.4) ----------------------------
+
+def view_delta_plan(prev: np.ndarray, nxt: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """What has to happen to every slot of a contiguous view that held the blocks `prev` (ascending ids, block prev[j] at
+    tokens [j*B, (j+1)*B)) so that it holds `nxt`: action[j] = 0 the slot already holds nxt[j] (nothing moves),
+    1 nxt[j] is a retained block (in W_next and W_prev) that sat in another slot, 2 nxt[j] is incoming (in W_next only).
+    Returns (action int32 [len(nxt)], counts int32 [3] = slots unchanged, retained and moved, incoming)."""
+    prev, nxt = np.ascontiguousarray(prev, np.int32), np.ascontiguousarray(nxt, np.int32)
+    held = set(int(b) for b in prev)
+    action = np.zeros(len(nxt), np.int32)
+    for j, b in enumerate(nxt):
+        if j < len(prev) and int(prev[j]) == int(b):
+            action[j] = 0
+        elif int(b) in held:
+            action[j] = 1
+        else:
+            action[j] = 2
+    counts = np.array([(action == 0).sum(), (action == 1).sum(), (action == 2).sum()], np.int32)
+    return action, counts
+
+
+def view_update(repo: Repository, table: np.ndarray, viewK: np.ndarray, viewV: np.ndarray, prev: np.ndarray,
+                nxt: np.ndarray) -> np.ndarray:
+    """Move a contiguous view (uint16 [L][G][cap][d] keys and values, in place) from the working set `prev` to `nxt`: a
+    slot whose block stays is not touched; every other slot of `nxt` receives its block from the repository (with the
+    whole history in one memory a moved retained block costs the same read and write whether it is shifted inside the
+    view or fetched again, and fetching has no ordering hazard).  Tokens past len(nxt) * B are left as they were.
+    Returns the counts of view_delta_plan."""
+    _, B, L, G, d = repo.pagesK.shape
+    action, counts = view_delta_plan(prev, nxt)
+    assert len(nxt) * B <= viewK.shape[2]
+    for j, b in enumerate(np.ascontiguousarray(nxt, np.int32)):
+        if action[j] == 0:
+            continue
+        page = int(table[int(b)])
+        viewK[:, :, j * B:(j + 1) * B, :] = repo.pagesK[page].transpose(1, 2, 0, 3)      # [B][L][G][d] -> [L][G][B][d]
+        viewV[:, :, j * B:(j + 1) * B, :] = repo.pagesV[page].transpose(1, 2, 0, 3)
+    return counts
+
+
 # ---- execution cache: working-set reuse with bounded delta re-RoPE -----------------------------------
 
 class ViewCache:
