@@ -315,14 +315,19 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     ptx::tma_store_3d(&map_v, sb + 3 * kHalfBytes, 64, y + u * box_rows, z);
                 }
                 ptx::bulk_commit();
-                if (it > 0) {                              // all but the newest store have left shared memory
+                if (KWB) {
+                    // four stages and a tile that is held until its consumers have rotated it: the stage goes back as soon
+                    // as this store has read it, not one tile later
+                    ptx::bulk_wait_read<0>();
+                    ptx::mbar_arrive(&empty_bar[st]);
+                } else if (it > 0) {                       // all but the newest store have left shared memory
                     ptx::bulk_wait_read<1>();
                     ptx::mbar_arrive(&empty_bar[(it - 1) % STAGES]);
                 }
             }
             ptx::bulk_wait_read<0>();
-            if (ok) ptx::mbar_arrive(&empty_bar[(n_tiles - 1) % STAGES]);
-            else atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
+            if (ok && !KWB) ptx::mbar_arrive(&empty_bar[(n_tiles - 1) % STAGES]);
+            else if (!ok) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
             ptx::bulk_wait<0>();                           // the view is complete before the kernel ends
         }
     } else if (KROT && warp > CONSUMERS + 1) {
