@@ -251,6 +251,21 @@ int kvmem_materialize(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessi
                       int32_t sel_stride, const int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/,
                       void* view_v /*DEVICE*/, int32_t view_cap_tokens, void* stream);
 
+/* Incremental execution view (Eq. "kvmem-working-set-delta", Sec. 4.4: only what changed between two consecutive
+ * working sets moves).  view_k / view_v hold the view kvmem_materialize (or this call) built from prev_ids; afterwards
+ * they hold the view of sel_ids, bit-identical to kvmem_materialize's.  A slot j whose block stays (prev_ids[s][j] ==
+ * sel_ids[s][j], j < n_prev[s]) is neither read nor written; every other slot receives its block from the pages
+ * through the block table.  (A retained block that changes its slot is fetched from the repository rather than
+ * shifted inside the view: with the whole history in HBM both cost one read and one write, and fetching has no
+ * ordering hazard.)  HBM traffic: 2 bytes per byte of the slots that change.
+ *   prev_ids  DEVICE int32 [n_sessions][sel_stride], n_prev DEVICE int32 [n_sessions]: the selection the view holds
+ *   stats     DEVICE int32 [n_sessions][3] or NULL: slots unchanged, retained blocks that moved, incoming blocks
+ * Other arguments and errors as kvmem_materialize.  prev_ids and sel_ids must be different buffers. */
+int kvmem_materialize_delta(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const int32_t* prev_ids /*DEVICE*/,
+                            const int32_t* n_prev /*DEVICE*/, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
+                            const int32_t* n_sel /*DEVICE*/, void* view_k /*DEVICE*/, void* view_v /*DEVICE*/,
+                            int32_t view_cap_tokens, int32_t* stats /*DEVICE, may be NULL*/, void* stream);
+
 /* GQA decode attention over the view (QW3 attention kernels, Sec. 5.1; decode over the fixed
  * working set, Sec. 5.2).  For every query token m, layer l and head h, over the first
  * T = n_sel[s] * B view tokens of KV head g(h), without mask:

@@ -545,6 +545,25 @@ int kvmem_materialize(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions
     return KVMEM_OK;
 }
 
+int kvmem_materialize_delta(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const int32_t* prev_ids, const int32_t* n_prev,
+                            const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k, void* view_v,
+                            int32_t view_cap_tokens, int32_t* stats, void* stream) {
+    if (!pool_live(p) || !pages_are(p, false, "kvmem_materialize_delta")) return KVMEM_E_STATE;
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!prev_ids || !n_prev || !sel_ids || !n_sel || !view_k || !view_v || !aligned(view_k, 16) || !aligned(view_v, 16)) {
+        set_error("kvmem_materialize_delta: null or misaligned pointer");
+        return KVMEM_E_INVALID;
+    }
+    if (sel_stride < 1 || view_cap_tokens < p->cfg.block_tokens || view_cap_tokens % p->cfg.block_tokens != 0) {
+        set_error("view_cap_tokens must be a positive multiple of block_tokens and sel_stride positive");
+        return KVMEM_E_INVALID;
+    }
+    cudaError_t e = launch_gather(*p, session_first, n_sessions, sel_ids, sel_stride, n_sel, (__nv_bfloat16*)view_k,
+                                  (__nv_bfloat16*)view_v, view_cap_tokens, (cudaStream_t)stream, prev_ids, n_prev, stats);
+    if (e != cudaSuccess) return cuda_fail("incremental gather kernel launch", e);
+    return KVMEM_OK;
+}
+
 int kvmem_view_attend(kvmem_pool_t* p, int32_t n_sessions, const void* q, int32_t n_q_tokens, const void* view_k,
                       const void* view_v, int32_t view_cap_tokens, const int32_t* n_sel, float scale, float* out,
                       float* lse, void* workspace, size_t workspace_bytes, void* stream) {

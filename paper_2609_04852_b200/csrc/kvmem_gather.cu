@@ -35,11 +35,15 @@ struct GatherArgs {
     int cap_tokens;              // view capacity in tokens
     int d;
     size_t page_elems;
+    // incremental view (Eq. "kvmem-working-set-delta"): the ids the view holds now; a slot whose block stays is skipped
+    const int32_t* prev_ids;     // [n_sessions][sel_stride] or null
+    const int32_t* n_prev;       // [n_sessions]
 };
 
-// page of selected block j of session s, or -1 (flagged) if anything is out of range
+// page of selected block j of session s; -1 (flagged) if anything is out of range, -2 if the view's slot j holds the block already
 __device__ __forceinline__ int lookup_page(const GatherArgs& a, int s, int j, int NB) {
     const int id = a.sel_ids[(size_t)s * a.sel_stride + j];
+    if (a.prev_ids && j < a.n_prev[s] && a.prev_ids[(size_t)s * a.sel_stride + j] == id) return -2;   // the slot already holds this block
     if (id < 0 || id >= NB) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); return -1; }
     const int pg = a.tables[(size_t)(a.session_first + s) * a.max_bps + id];
     if (pg < 0 || pg >= a.max_blocks) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); return -1; }
@@ -192,11 +196,52 @@ int g_pdl = 1;           // programmatic dependent launch of the step's kernels
 int g_gather_ctas = 0;    // 0: as many single-warp CTAs as fit; > 0: at most this many (kernel-variant switch)
 int g_gather_mode = 1;   // 1: TMA bulk ring, 0: ld/st
 
+// Per session: how many slots of the new view keep their block, receive a retained block that sat elsewhere, receive an
+// incoming block (the counts of the working-set delta, Eq. "kvmem-working-set-delta").  One CTA per session.
+__global__ void __launch_bounds__(256)
+view_delta_stats_kernel(const int32_t* __restrict__ prev_ids, const int32_t* __restrict__ n_prev, const int32_t* __restrict__ sel_ids,
+                        const int32_t* __restrict__ n_sel, int sel_stride, int32_t* __restrict__ stats) {
+    pdl_wait();
+    __shared__ int cnt[3];
+    const int s = blockIdx.x;
+    if (threadIdx.x < 3) cnt[threadIdx.x] = 0;
+    __syncthreads();
+    const int np = min(max(n_prev[s], 0), sel_stride), nn = min(max(n_sel[s], 0), sel_stride);
+    const int32_t* prev = prev_ids + (size_t)s * sel_stride;
+    const int32_t* next = sel_ids + (size_t)s * sel_stride;
+    int mine[3] = {0, 0, 0};
+    for (int j = threadIdx.x; j < nn; j += blockDim.x) {
+        const int id = next[j];
+        int act = 2;
+        if (j < np && prev[j] == id) act = 0;
+        else {
+            int lo = 0, hi = np - 1;                         // prev is ascending: binary search
+            while (lo <= hi) {
+                const int mid = (lo + hi) >> 1, v = prev[mid];
+                if (v == id) { act = 1; break; }
+                if (v < id) lo = mid + 1; else hi = mid - 1;
+            }
+        }
+        mine[act] += 1;
+    }
+#pragma unroll
+    for (int i = 0; i < 3; ++i)
+        if (mine[i]) atomicAdd(&cnt[i], mine[i]);
+    __syncthreads();
+    if (threadIdx.x < 3) stats[(size_t)s * 3 + threadIdx.x] = cnt[threadIdx.x];
+}
+
 cudaError_t launch_gather(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids,
                           int sel_stride, const int32_t* n_sel, __nv_bfloat16* view_k, __nv_bfloat16* view_v,
-                          int view_cap_tokens, cudaStream_t st) {
+                          int view_cap_tokens, cudaStream_t st, const int32_t* prev_ids, const int32_t* n_prev, int32_t* delta_stats) {
     const Geometry& g = p.geo;
+    if (prev_ids && delta_stats) {
+        launch_pdl(view_delta_stats_kernel, dim3((unsigned)n_sessions), dim3(256), 0, st, prev_ids, n_prev, sel_ids, n_sel, sel_stride, delta_stats);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     GatherArgs a{};
+    a.prev_ids = prev_ids; a.n_prev = n_prev;
     a.pages = p.pages; a.tables = p.tables; a.nblocks_dev = p.nblocks_dev;
     a.sel_ids = sel_ids; a.n_sel = n_sel; a.view_k = view_k; a.view_v = view_v; a.status = p.status_dev;
     a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;

@@ -210,9 +210,11 @@ cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, 
                         int scores_stride, const kvmem_select_params_t& prm, int32_t* sel_ids, int sel_stride,
                         int32_t* n_sel, cudaStream_t st);
 
+// prev_ids != null: incremental view, slots whose block stays are skipped; delta_stats (may be null) receives the counts
 cudaError_t launch_gather(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids,
                           int sel_stride, const int32_t* n_sel, __nv_bfloat16* view_k, __nv_bfloat16* view_v,
-                          int view_cap_tokens, cudaStream_t st);
+                          int view_cap_tokens, cudaStream_t st, const int32_t* prev_ids = nullptr, const int32_t* n_prev = nullptr,
+                          int32_t* delta_stats = nullptr);
 
 struct AttendPlan {
     int n_splits;

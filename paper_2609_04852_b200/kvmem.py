@@ -74,6 +74,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_score_host_index": (C.c_int, [vp, vp, i32, i32, vp, i32, i32, vp, vp, sz, vp, sz, vp]),
         "kvmem_select": (C.c_int, [vp, i32, i32, vp, i32, prmp, vp, i32, vp, vp, vp, sz, vp]),
         "kvmem_materialize": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, vp]),
+        "kvmem_materialize_delta": (C.c_int, [vp, i32, i32, vp, vp, vp, i32, vp, vp, vp, i32, vp, vp]),
         "kvmem_view_attend": (C.c_int, [vp, i32, vp, i32, vp, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
         "kvmem_get_index": (C.c_int, [vp, i32, C.POINTER(vp), C.POINTER(i32)]),
         "kvmem_get_block_table": (C.c_int, [vp, i32, C.POINTER(vp), C.POINTER(i32)]),
@@ -122,7 +123,7 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend", "kvmem_paged_attend_rope", "kvmem_topk", "kvmem_score_host_workspace_bytes",
             "kvmem_score_host_staging_bytes", "kvmem_score_host_index", "kvmem_materialize_fp8", "kvmem_view_attend_fp8",
             "kvmem_materialize_attend_rope", "kvmem_paged_attend_fp8", "kvmem_materialize_attend_fp8",
-            "kvmem_paged_attend_fp8_rope", "kvmem_selftest_wait_timeout")
+            "kvmem_paged_attend_fp8_rope", "kvmem_selftest_wait_timeout", "kvmem_materialize_delta")
 
 
 def _check(status: int) -> None:
@@ -343,6 +344,18 @@ class Pool:
         _check(self.lib.kvmem_materialize(self.handle, session_first, ns, _dev(sel_ids, torch.int32),
                                           sel_ids.shape[-1], _dev(n_sel, torch.int32), _dev(view.k, torch.bfloat16),
                                           _dev(view.v, torch.bfloat16), view.cap_tokens, _stream()))
+
+    def materialize_delta(self, prev_ids: torch.Tensor, n_prev: torch.Tensor, sel_ids: torch.Tensor, n_sel: torch.Tensor,
+                          view: View, stats: Optional[torch.Tensor] = None, session_first: int = 0) -> None:
+        """Move a view built from prev_ids to sel_ids: slots whose block stays are not touched, the others are fetched.
+        stats int32 [n_sessions][3] (optional) receives (unchanged, retained and moved, incoming) per session."""
+        ns = n_sel.shape[0]
+        if prev_ids.shape != sel_ids.shape:
+            raise ValueError("both id lists must have the same [n_sessions][stride] shape")
+        _check(self.lib.kvmem_materialize_delta(self.handle, session_first, ns, _dev(prev_ids, torch.int32), _dev(n_prev, torch.int32),
+                                                _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
+                                                _dev(view.k, torch.bfloat16), _dev(view.v, torch.bfloat16), view.cap_tokens,
+                                                None if stats is None else _dev(stats, torch.int32), _stream()))
 
     def view_attend(self, q: torch.Tensor, view: View, n_sel: torch.Tensor, out: torch.Tensor, lse: torch.Tensor,
                     scale: float = 0.0) -> None:

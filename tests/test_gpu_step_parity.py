@@ -414,3 +414,59 @@ def test_position_consistent_view_and_attention_in_one_pass_over_raw_keys(B, n_b
     assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
     assert torch.equal(view.k, view2.k) and torch.equal(view.v, view2.v)
     assert torch.equal(out, out2) and torch.equal(lse, lse2)
+
+
+# ------------------------------------------------------------------ incremental contiguous view
+
+@pytest.mark.parametrize("gather_mode,B", [(1, 64), (0, 64), (1, 32)])
+def test_incremental_view_over_a_sequence_of_working_sets(gather_mode, B):
+    """kvmem_materialize_delta against the oracle's view_update over overlapping working sets: the view equals the plain
+    gather of the newest set after every step, the counts are the oracle's, and a slot whose block stays is provably not
+    written (it is overwritten with a marker before the call and keeps it)."""
+    from paper_2609_04852_b200 import set_option
+    spec = SMALL.with_(name="delta_view", block_tokens=B, n_blocks=150, n_planted=4, budget_blocks=24, max_view_tokens=1 << 30)
+    dev = torch.device("cuda", 0)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)[0]
+    cap = 24
+    g = Guards(dev)
+    view = g.view(pool, 1, cap * B)
+    stats = g.empty((1, 3), torch.int32)
+    oK = np.zeros((1, spec.n_kv_heads, cap * B, spec.head_dim), np.uint16)
+    oV = np.zeros_like(oK)
+    rng = np.random.default_rng(21)
+    from test_gpu_view_cache import _working_sets
+    sets = _working_sets(rng, spec.n_blocks, [20, 20, 24, 7, 20, 24, 24, 1])
+    sets.insert(3, sets[2].copy())                        # an unchanged working set
+    sets.append(np.concatenate([sets[-1], np.array([140, 141], np.int32)]))      # pure append behind an unchanged prefix
+    prev = np.zeros(0, np.int32)
+    set_option("gather_mode", gather_mode)
+    try:
+        for step, sel in enumerate(sets):
+            def dev_ids(a):
+                t = torch.zeros(1, cap, dtype=torch.int32)
+                t[0, : len(a)] = torch.from_numpy(np.ascontiguousarray(a, np.int32))
+                return t.to(dev), torch.tensor([len(a)], dtype=torch.int32, device=dev)
+            p_ids, p_n = dev_ids(prev)
+            s_ids, s_n = dev_ids(sel)
+            action, _ = orc.view_delta_plan(prev, sel)
+            stay = [j for j in range(len(sel)) if action[j] == 0]
+            marker = torch.tensor(-7.0, dtype=torch.bfloat16)
+            for j in stay[:2]:                             # a slot that stays must not be written: it keeps a marker
+                view.k[0, :, :, j * B:(j + 1) * B] = marker
+            pool.materialize_delta(p_ids, p_n, s_ids, s_n, view, stats)
+            torch.cuda.synchronize()
+            assert pool.device_status() == 0
+            g.check()
+            counts = orc.view_update(osess.repo, osess.table, oK, oV, prev, sel)
+            assert stats.cpu().numpy()[0].tolist() == counts.tolist(), step
+            T = len(sel) * B
+            for j in stay[:2]:
+                assert bool((view.k[0, :, :, j * B:(j + 1) * B] == marker).all()), f"step {step}: slot {j} stays but was written"
+                view.k[0, :, :, j * B:(j + 1) * B] = torch.from_numpy(oK[:, :, j * B:(j + 1) * B].view(np.int16)).view(torch.bfloat16).to(dev)
+            gK, gV = orc.gather(osess.repo, osess.table, sel, cap * B)
+            assert np.array_equal(bits(view.k[0])[:, :, :T], gK[:, :, :T]) and np.array_equal(bits(view.v[0])[:, :, :T], gV[:, :, :T]), step
+            assert np.array_equal(oK[:, :, :T], gK[:, :, :T])
+            prev = sel
+    finally:
+        set_option("gather_mode", 1)
