@@ -59,8 +59,9 @@ def measured_tensor_peak():
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant kernel on the 1M workload.
 # These are constants taken from earlier ncu captures of the same kernels, not measured in the run that prints them
 # (a bench run is never made under a profiler); the line says so in "traffic_source".
-GATHER_TRAFFIC = {"1m": 2099369984}       # gather_bulk_kernel
-FUSED_TRAFFIC = {"1m": 2099557205}        # attend_split_kernel<1>, mean of six launches
+GATHER_TRAFFIC = {"1m": 2099369984, "chunk512": 2098579520}       # gather_bulk_kernel
+# attend_split_kernel<1>, mean of six launches (128k: 134 MB read + 79 MB written; the rest of the view is still in L2 when the kernel ends)
+FUSED_TRAFFIC = {"1m": 2099538346, "128k": 213239722, "batch8": 4253410560}
 ROPE_FUSED_TRAFFIC = {"1m": 2098100000}   # attend_split_kernel<5> (in-block key layout)
 ROPE_GATHER_TRAFFIC = {"1m": 2298386176}  # gather_rope_kernel
 TRAFFIC_SOURCE = ("constant from an earlier ncu capture of this kernel on this workload (one launch, "
@@ -518,6 +519,30 @@ def run_native(args):
                                 "counted once (frac_algorithmic) the target is not met",
                                 "executed_flop_per_launch_pair": 2 * flop_alg, "algorithmic_flop": flop_alg,
                                 "executed_tflops": exe_tf, "algorithmic_tflops": alg_tf, "avg_score_ms": sel_s * 1e3, "traffic": None}
+        if not spec.attend and B != 64 and ns == 1:
+            # The scaling workload has the paper's 32-token blocks.  Decode over the view it selects (4 query tokens:
+            # 1 + 3 drafts) through the passes that read pages through the block table, each timed alone over 50 calls.
+            spec4 = spec.with_(n_q_tokens=4)
+            q4 = [make_queries(spec4, i).to(device) for i in range(4)]
+            out4, lse4 = pool.new_outputs(ns, 4)
+            view_bytes = ns * ab["gather"] // 2
+            dec = {}
+            for name, fn, nbytes in (("kvmem_materialize_attend", lambda qq: pool.materialize_attend(qq, sel, n_sel, view, out4, lse4), 2 * view_bytes),
+                                     ("kvmem_paged_attend", lambda qq: pool.paged_attend(qq, sel, n_sel, out4, lse4), view_bytes)):
+                for i in range(3):
+                    fn(q4[i % 4])
+                d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize(device)
+                d0.record(stream)
+                for i in range(50):
+                    fn(q4[i % 4])
+                d1.record(stream)
+                torch.cuda.synchronize(device)
+                us = d0.elapsed_time(d1) / 50 * 1e3
+                dec[name] = {"us": us, "algorithmic_bytes": nbytes, "gbs": nbytes / (us * 1e-6) / 1e9,
+                             "frac_of_peak": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+            assert pool.device_status() == 0
+            line["decode_over_view"] = {"query_tokens": 4, "block_tokens": B, "view_tokens": cap, **dec}
         if args.host_index and spec.attend and ns == 1:
             # the memory-bounded variant: the index stays in pinned host memory and is streamed over PCIe in tiles
             idx_host = pool.index(0).cpu().contiguous().pin_memory()
