@@ -179,6 +179,10 @@ def run_native(args):
         name, _, value = opt.partition("=")
         set_option(name, int(value))
     if world > 1 and not dist.is_initialized():
+        # NCCL's own log stays on (on stderr: stdout carries rank 0's one JSON line): a multi-GPU run then shows its ranks,
+        # transports and whether in-switch reduction was used
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
         dist.init_process_group("nccl", device_id=device)
 
     base = CONFIGS[args.workload]
@@ -786,6 +790,8 @@ def run_head_sharded(args):
         name, _, value = opt.partition("=")
         set_option(name, int(value))
     if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
         dist.init_process_group("nccl", device_id=device)
     spec = CONFIGS[args.workload]
     if not spec.attend or spec.n_sessions != 1:
@@ -1013,7 +1019,8 @@ def launch_ranks(n, argv, script=None, extra_env=None):
     cmd = [sys.executable, "-m", "torch.distributed.run", "--standalone", "--nnodes=1", f"--nproc-per-node={n}",
            "--local-addr", "127.0.0.1", script or os.path.abspath(__file__), *argv]
     env = dict(os.environ)
-    env.setdefault("NCCL_DEBUG", "WARN")          # NCCL's own log stays on: a transport problem is then visible in the run's output
+    env.setdefault("NCCL_DEBUG", "INFO")          # NCCL's own log stays on (stderr): ranks, transports and NVLS use are visible in the run's output
+    env.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
     env.update(extra_env or {})
     return subprocess.call(cmd, env=env)
 
@@ -1069,6 +1076,14 @@ def other_workloads(args):
         rec = {k: line[k] for k in keep if k in line}
         rec["config"] = {k: line["config"][k] for k in ("workload", "l2", "calls")}
         rec["step_hbm"] = {k: line["step_hbm"][k] for k in ("algorithmic_bytes_per_step", "accounting", "achieved_gbs", "frac_of_peak", "peak_source")}
+        if flush:
+            # the headline figures of this workload flush L2 between steps (its view fits, or nearly fits, the 126 MB L2);
+            # the same steps back to back, as a decode loop would issue them, for comparison
+            a.flush_l2 = False
+            warm = run_native(a)
+            rec["without_l2_flush"] = {"value": warm["value"], "ms_per_step": warm["ms_per_step"],
+                                       "step_hbm_frac_of_peak": warm["step_hbm"]["frac_of_peak"],
+                                       "note": "partly L2-resident: not a DRAM-roofline figure"}
         out[name] = rec
     gc.collect()
     torch.cuda.empty_cache()

@@ -239,11 +239,53 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             };
             my_page = lookup(lane);
             bool ok = true;
+            if (B == kTile) {
+                // One block per tile, the common case, kept as lean as the tile needs (one shuffle, four loads): the
+                // producer's own instructions sit on the critical path of a read-only stream.
+                for (int it = 0; it < n_tiles; ++it) {
+                    if (it >= base_slot + 32) { base_slot = it; my_page = lookup(base_slot + lane); }
+                    const int page = __shfl_sync(0xffffffffu, my_page, it - base_slot);
+                    if (lane == 0) {
+                        const int st = it % STAGES;
+                        if (ok && ahead < STAGES && it >= ahead) {
+                            const int jt = it - ahead;
+                            ok = (KROT || a.landed) ? ptx::mbar_wait(&full_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1))
+                                                    : ptx::mbar_wait(&empty_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1));
+                        }
+                        if (ok && it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
+                        if (ROPE && ok) {
+                            const int tb = it % GROUPS;
+                            if (it >= GROUPS) ok = ptx::mbar_wait(&tab_empty[tb], (uint32_t)(((it / GROUPS) & 1) ^ 1));
+                            if (ok) {
+                                const float2* rows = a.rope + (size_t)(a.first_position + (t0 + it) * kTile) * (kD / 2);
+                                ptx::mbar_expect_tx(&tab_full[tb], kTabBytes);
+                                ptx::bulk_g2s(stages + (size_t)STAGES * kStageBytes + (size_t)tb * kTabBytes, rows, kTabBytes, &tab_full[tb]);
+                            }
+                        }
+                        if (ok) {
+                            unsigned char* dst = stages + (size_t)st * kStageBytes;
+                            // page layout [K|V][L*G][64 tokens][128]: rows of 256 B
+                            const int yk = ((page * 2 + 0) * LG + lg) * kTile, yv = ((page * 2 + 1) * LG + lg) * kTile;
+                            ptx::mbar_expect_tx(&full_bar[st], kStageBytes);
+                            ptx::tma_load_2d(dst, &map_pages, 0, yk, &full_bar[st]);
+                            ptx::tma_load_2d(dst + kHalfBytes, &map_pages, 64, yk, &full_bar[st]);
+                            ptx::tma_load_2d(dst + 2 * kHalfBytes, &map_pages, 0, yv, &full_bar[st]);
+                            ptx::tma_load_2d(dst + 3 * kHalfBytes, &map_pages, 64, yv, &full_bar[st]);
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
+                }
+            } else
             for (int it = 0; it < n_tiles; ++it) {
                 if (it * n_sub >= base_slot + 32) { base_slot = it * n_sub; my_page = lookup(base_slot + lane); }
-                int pages[4];
+                int pages[4] = {-1, -1, -1, -1};
+                if (n_sub == 1) {
+                    pages[0] = __shfl_sync(0xffffffffu, my_page, (it - base_slot) & 31);
+                } else {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) pages[u] = u < n_sub ? __shfl_sync(0xffffffffu, my_page, (it * n_sub + u - base_slot) & 31) : -1;
+                    for (int u = 0; u < 4; ++u) pages[u] = u < n_sub ? __shfl_sync(0xffffffffu, my_page, (it * n_sub + u - base_slot) & 31) : -1;
+                }
                 if (lane == 0) {
                     const int st = it % STAGES;
                     // at most `ahead` tiles in flight: tile it - ahead has left its stage (the same phase is waited for
@@ -663,16 +705,30 @@ attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__
     const int s = z / LG, lg = z % LG, l = lg / G, g = lg % G;
     const int col = threadIdx.x;
     const size_t p0 = (size_t)z * n_splits * rows_pad + row;          // split sp lives at p0 + sp * rows_pad
+    // eight splits at a time: the statistics and the partial outputs of a batch are loaded before any of them is used,
+    // so that a merge costs a few memory round trips instead of one per split (same split order, same arithmetic)
     float mx = -INFINITY;
     for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, part_ml[p0 + (size_t)sp * rows_pad].x);
     float acc = 0.0f, lsum = 0.0f;
-#pragma unroll 4
-    for (int sp = 0; sp < n_splits; ++sp) {
-        const size_t pi = p0 + (size_t)sp * rows_pad;
-        const float2 ml = part_ml[pi];
-        const float f = ml.x > -INFINITY ? exp2f(ml.x - mx) : 0.0f;
-        acc += f * part_o[pi * kD + col];
-        lsum += f * ml.y;
+    constexpr int U = 8;
+    for (int sp0 = 0; sp0 < n_splits; sp0 += U) {
+        float2 ml[U];
+        float po[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int sp = min(sp0 + u, n_splits - 1);
+            const size_t pi = p0 + (size_t)sp * rows_pad;
+            ml[u] = part_ml[pi];
+            po[u] = part_o[pi * kD + col];
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (sp0 + u < n_splits) {
+                const float f = ml[u].x > -INFINITY ? exp2f(ml[u].x - mx) : 0.0f;
+                acc += f * po[u];
+                lsum += f * ml[u].y;
+            }
+        }
     }
     const int m = row / r, hr = row % r;
     const size_t orow = (((size_t)s * M + m) * L + l) * H + (size_t)g * r + hr;
