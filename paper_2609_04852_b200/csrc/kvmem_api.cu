@@ -762,7 +762,7 @@ static int paged_attend_impl(kvmem_pool_t* p, int32_t session_first, int32_t n_s
         return KVMEM_E_INVALID;
     }
     if (n_q_tokens < 1 || sel_stride < 1) { set_error("n_q_tokens and sel_stride must be positive"); return KVMEM_E_INVALID; }
-    if (!paged_block_size_ok(p, rope_first_position >= 0 && p->cfg.rope_in_block_keys, "kvmem_paged_attend")) return KVMEM_E_UNSUPPORTED;
+    if (!paged_block_size_ok(p, false, "kvmem_paged_attend")) return KVMEM_E_UNSUPPORTED;     // the query-rotating mode handles every block size too
     if (n_q_tokens * p->geo.r > (rope_first_position >= 0 ? 16 : 64)) { set_error("n_q_tokens * (H/G) = %d exceeds %d rows per call", n_q_tokens * p->geo.r, rope_first_position >= 0 ? 16 : 64); return KVMEM_E_UNSUPPORTED; }
     if (!(scale >= 0.0f)) { set_error("scale must be non-negative (0 selects 1/sqrt(d))"); return KVMEM_E_INVALID; }
     if ((int64_t)p->cfg.max_blocks * 2 * p->cfg.n_layers * p->cfg.n_kv_heads * p->cfg.block_tokens > 0x7fffffffll) {

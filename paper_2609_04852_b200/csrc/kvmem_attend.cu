@@ -129,7 +129,9 @@ static int choose_splits(int heads, int max_tiles, int sms) {
 // alternately.  RT = 2 (up to 32 rows): every consumer warp sees every tile, four warps per row tile, 16 tokens each.
 // RT = 4 (up to 64 rows): two warps per row tile, 32 tokens each.  The K/V stream is read once whatever RT is; with
 // more row tiles the consumers do more arithmetic per byte and the pass moves from HBM-bound towards issue-bound.
-template <int MODE, int RT = 1>
+// SUB (MODE 4 only): selected blocks per 64-token tile (64 / B for B < 64); every block of a tile has its own compact
+// position, hence its own rotated copy of the query (four data stages then, to make room for the copies).
+template <int MODE, int RT = 1, int SUB = 1>
 __global__ void __launch_bounds__(MODE == 3 ? (kAttRopeConsumers + 1) * 32 : MODE == 6 ? (kAttRopeConsumers + 2) * 32 : kAttThreads + (MODE == 1 ? 32 : MODE == 4 ? 32 * kQrotWarps : MODE == 5 ? 32 + 32 * kKrotWarps : 0), 1)
 attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_pages, AttendArgs a) {
@@ -141,7 +143,8 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     constexpr bool QROT = MODE == 4;       // a rotator warp re-encodes the query per tile instead
     extern __shared__ unsigned char smem_dyn[];
     // the rotary mode gives the room of two data stages to one buffer of rotary rows per consumer group
-    constexpr int STAGES = ROPE ? kAttRopeStages : kAttStages;
+    static_assert(SUB == 1 || (MODE == 4 && (SUB == 2 || SUB == 4)), "several blocks per tile with their own rotation: the query-rotating mode only");
+    constexpr int STAGES = ROPE ? kAttRopeStages : (QROT && SUB > 1) ? 4 : kAttStages;
     constexpr int CONSUMERS = ROPE ? kAttRopeConsumers : kAttConsumers;
     constexpr int GROUPS = ROPE ? kAttRopeGroups : RT > 1 ? 1 : kAttGroups;
     static_assert(RT == 1 || (MODE <= 2 && (RT == 2 || RT == 4)), "several row tiles: the plain modes only");
@@ -430,35 +433,50 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     raw_hi[i] = *reinterpret_cast<const uint4*>(qr + kD / 2 + c * 8);
                 }
             }
-            unsigned char* qring = stages + (size_t)kAttStages * kStageBytes;
-            // the rotary row of a tile is fetched one of this warp's tiles ahead: an L2 round trip per tile would
-            // otherwise sit on the critical path of every tile
-            auto fetch_row = [&](int it, float4 (&t4)[4]) {
-                int p0 = a.first_position + (t0 + min(it, n_tiles - 1)) * kTile;
+            unsigned char* qring = stages + (size_t)STAGES * kStageBytes;
+            const int tpb = btok > kTile ? btok / kTile : 1;       // tiles per block (blocks larger than a tile)
+            // position of the block that holds sub-block u of tile it: the query is rotated back by it
+            auto block_pos = [&](int it, int u) -> int { return a.first_position + (((t0 + it) * SUB + u) / tpb) * btok; };
+            auto fetch_row = [&](int p0, float4 (&t4)[4]) {
                 if (p0 < 0 || p0 >= a.rope_positions) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); p0 = 0; }
                 const float4* cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)p0 * (kD / 2) + c * 8);
 #pragma unroll
                 for (int w = 0; w < 4; ++w) t4[w] = __ldg(cs4 + w);
             };
             const int it_first = warp - CONSUMERS - 1;
-            float4 t4[4], t4_next[4];
-            fetch_row(it_first, t4_next);
+            // SUB == 1: the rotary row of a tile is fetched one of this warp's tiles ahead (an L2 round trip per tile would
+            // otherwise sit on the critical path of every tile); SUB > 1: the rows of a tile's blocks are fetched when
+            // the tile comes up, before the wait for its stage
+            float4 t4[SUB][4], t4_next[4];
+            if (SUB == 1) fetch_row(block_pos(min(it_first, n_tiles - 1), 0), t4_next);
             for (int it = it_first; it < n_tiles; it += kQrotWarps) {
                 const int st = it % STAGES;
+                int n_valid = 1;
+                if (SUB == 1) {
 #pragma unroll
-                for (int w = 0; w < 4; ++w) t4[w] = t4_next[w];
-                fetch_row(it + kQrotWarps, t4_next);
+                    for (int w = 0; w < 4; ++w) t4[0][w] = t4_next[w];
+                    fetch_row(block_pos(min(it + kQrotWarps, n_tiles - 1), 0), t4_next);
+                } else {
+                    n_valid = min(kTile, n_tok - (t0 + it) * kTile) / btok;       // blocks the (possibly ragged) tile holds
+#pragma unroll
+                    for (int u = 0; u < SUB; ++u)
+                        if (u < n_valid) fetch_row(block_pos(it, u), t4[u]);
+                }
                 bool ok = true;
                 if (it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
                 if (!__all_sync(0xffffffffu, ok)) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
-                unsigned char* qb = qring + (size_t)st * kQrotBytes;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = (lane >> 3) + 4 * i;
-                    uint4 lo_o, hi_o;
-                    rotate8_cs(raw_lo[i], raw_hi[i], t4, -1.0f, lo_o, hi_o);
-                    *reinterpret_cast<uint4*>(qb + row * 256 + ((c ^ (row & 7)) << 4)) = lo_o;
-                    *reinterpret_cast<uint4*>(qb + row * 256 + (((c + 8) ^ (row & 7)) << 4)) = hi_o;
+                for (int u = 0; u < SUB; ++u) {
+                    if (u >= n_valid) continue;
+                    unsigned char* qb = qring + ((size_t)st * SUB + u) * kQrotBytes;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int row = (lane >> 3) + 4 * i;
+                        uint4 lo_o, hi_o;
+                        rotate8_cs(raw_lo[i], raw_hi[i], t4[u], -1.0f, lo_o, hi_o);
+                        *reinterpret_cast<uint4*>(qb + row * 256 + ((c ^ (row & 7)) << 4)) = lo_o;
+                        *reinterpret_cast<uint4*>(qb + row * 256 + (((c + 8) ^ (row & 7)) << 4)) = hi_o;
+                    }
                 }
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&q_full[st]);
@@ -500,6 +518,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 break;
             }
             bool k_handed_over = false;                      // KWB: this warp's share of the tile is rotated and back in the stage
+            bool tab_released = false;                       // ROPE: this warp has given the group's table buffer back
 #pragma unroll
             for (int sl = 0; sl < SLICES; ++sl) {
             const int wq = wq0 + sl;
@@ -508,7 +527,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             const uint32_t vbase = kbase + 2 * kHalfBytes;
             // QROT: this tile's rotated query; its A fragments are fetched two k-steps at a time, next to their use
             const int qrow = mr + 8 * (mj & 1);
-            const uint32_t qaddr = stage0 + (uint32_t)kAttStages * kStageBytes + (uint32_t)st * kQrotBytes + (uint32_t)qrow * 256u;
+            const uint32_t qaddr = stage0 + (uint32_t)STAGES * kStageBytes + (uint32_t)(st * SUB + (SUB > 1 ? (wq * 16) / btok : 0)) * kQrotBytes + (uint32_t)qrow * 256u;
 
             // S = Q K^T for this warp's 16 tokens: 2 n-tiles (8 tokens each) x 8 k-steps
             float sc[2][4];
@@ -589,6 +608,11 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     if (lane == 0) ptx::mbar_arrive(&q_full[st]);
                     k_handed_over = true;
                 }
+                // the rotary rows are done with: the group's table buffer goes back now, so that the rows of its next
+                // tile load during the softmax and the P V products instead of after them
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&tab_empty[grp]);
+                tab_released = true;
             }
             // online softmax (exp2 domain); this thread holds rows lane/4 (c0,c1) and lane/4 + 8 (c2,c3)
             float mx0 = -INFINITY, mx1 = -INFINITY;
@@ -642,7 +666,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             __syncwarp();
             if (lane == 0) {
                 ptx::mbar_arrive(&empty_bar[st]);
-                if (ROPE) ptx::mbar_arrive(&tab_empty[grp]);
+                if (ROPE && !tab_released) ptx::mbar_arrive(&tab_empty[grp]);
             }
         }
         // row sums live spread over the 4 lanes of a quad
@@ -816,6 +840,10 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmemQrot);
         if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attend_split_kernel<4, 1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmemQrot);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attend_split_kernel<4, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmemQrot);
+        if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
@@ -861,7 +889,11 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         }
     }
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
-    if (paged_only && rope_first_position >= 0 && p.cfg.rope_in_block_keys)
+    if (paged_only && rope_first_position >= 0 && p.cfg.rope_in_block_keys && g.B == 32)
+        launch_pdl(attend_split_kernel<4, 1, 2>, dim3(grid), dim3(kAttThreads + 32 * kQrotWarps), kAttSmemQrot, st, map_k, map_v, map_pages, a);
+    else if (paged_only && rope_first_position >= 0 && p.cfg.rope_in_block_keys && g.B == 16)
+        launch_pdl(attend_split_kernel<4, 1, 4>, dim3(grid), dim3(kAttThreads + 32 * kQrotWarps), kAttSmemQrot, st, map_k, map_v, map_pages, a);
+    else if (paged_only && rope_first_position >= 0 && p.cfg.rope_in_block_keys)
         launch_pdl(attend_split_kernel<4>, dim3(grid), dim3(kAttThreads + 32 * kQrotWarps), kAttSmemQrot, st, map_k, map_v, map_pages, a);
     else if (paged_only && rope_first_position >= 0)
         launch_pdl(attend_split_kernel<3>, dim3(grid), dim3((kAttRopeConsumers + 1) * 32), kAttSmem, st, map_k, map_v, map_pages, a);

@@ -470,3 +470,36 @@ def test_incremental_view_over_a_sequence_of_working_sets(gather_mode, B):
             prev = sel
     finally:
         set_option("gather_mode", 1)
+
+
+# ------------------------------------------------------------------ in-block key layout with other block sizes (copy-free pass)
+
+@pytest.mark.parametrize("B,n_blocks,budget,M,first", [(32, 200, 21, 4, 131), (32, 300, 128, 2, 0), (16, 300, 37, 4, 17), (128, 40, 9, 4, 64),
+                                                      (32, 64, 1, 1, 5)])
+def test_query_rotating_copy_free_attention_with_other_block_sizes(B, n_blocks, budget, M, first):
+    """kvmem_paged_attend_rope on a pool whose pages hold RoPE(k, offset in block), with 16-, 32- and 128-token blocks: every
+    block of a 64-token tile has its own compact position, so the query is rotated back once per block.  Against the
+    oracle's statement of the same formulation at the attention tolerance."""
+    from test_gpu_rope_in_block import SPEC as ISPEC, _fill_both as fill_in_block
+    spec = ISPEC.with_(name=f"inblockB{B}", block_tokens=B, n_blocks=n_blocks, budget_blocks=budget, n_q_tokens=M)
+    dev = torch.device("cuda", 0)
+    pool, repo, idx, tab, table = fill_in_block(spec, encoded=False)
+    ids = np.sort(np.random.default_rng(11 * n_blocks + B).choice(n_blocks, size=budget, replace=False)).astype(np.int32)
+    q, qb = queries(spec)
+    sel = torch.from_numpy(ids).view(1, -1).to(dev)
+    n_sel = torch.tensor([budget], dtype=torch.int32, device=dev)
+    T = budget * B
+    g = Guards(dev)
+    out, lse = g.outputs(pool, 1, M)
+    pool.paged_attend_rope(q.to(dev), sel, n_sel, out, lse, first)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    g.check()
+    pK, pV = orc.gather(repo, table, ids, T)
+    ro, rl = orc.attend_qrot(qb[0], pK, pV, T, B, first, tab)
+    assert np.abs(out.cpu().numpy()[0] - ro).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - rl).max() <= ATTN_ATOL
+    # and the position-consistent view of the same blocks (one rotation per block) gives the same attention within the
+    # rounding that separates the two formulations
+    vK, vV = orc.gather_rope(repo, table, ids, T, first, tab, in_block=True)
+    do, dl = orc.attend(qb[0], vK, vV, T)
+    assert np.abs(out.cpu().numpy()[0] - do).max() <= REFORMULATION_ATOL and np.abs(lse.cpu().numpy()[0] - dl).max() <= REFORMULATION_ATOL
