@@ -66,8 +66,8 @@ typedef struct {
                                        head_dim / 2 per position)                                      */
     float rope_theta;               /* rotary base (e.g. 1e6); used when rope_max_positions > 0        */
     int32_t rope_in_block_keys;     /* 0: the pages hold raw (position-free) keys.  1 (needs rotary support with
-                                       rope_max_positions >= block_tokens and 64-token blocks for the copy-free
-                                       attention): a page holds k' = RoPE(k, t), t the token's offset inside its
+                                       rope_max_positions >= block_tokens; the fused materialise+attend pass on this
+                                       layout needs 64-token blocks): a page holds k' = RoPE(k, t), t the token's offset inside its
                                        block, so that a block placed at compact position p0 needs the rotation
                                        of p0 alone: the position-consistent view rotates by one angle set per
                                        block, and the copy-free attention rotates the QUERY back by p0 once per
@@ -283,8 +283,9 @@ int kvmem_materialize_delta(kvmem_pool_t* pool, int32_t session_first, int32_t n
  * masked); head_dim 128.  The calls that read pages through the block table (kvmem_materialize_attend,
  * kvmem_paged_attend, kvmem_paged_attend_rope on raw keys, kvmem_view_cache_attend) take block sizes that divide
  * 64 tokens (a tile is then 64 / B selected blocks, the last one possibly partly filled) or are a multiple of it,
- * among them the paper's default of 32 tokens (Sec. 4.3); the in-block key layout and the FP8 repository are built
- * for 64-token blocks.  Other shapes return KVMEM_E_UNSUPPORTED. */
+ * among them the paper's default of 32 tokens (Sec. 4.3), also on the in-block key layout (kvmem_paged_attend_rope
+ * then rotates the query back once per block of a tile); kvmem_materialize_attend_rope on the in-block layout and the
+ * FP8 repository are built for 64-token blocks.  Other shapes return KVMEM_E_UNSUPPORTED. */
 int kvmem_view_attend(kvmem_pool_t* pool, int32_t n_sessions, const void* q /*DEVICE*/, int32_t n_q_tokens,
                       const void* view_k /*DEVICE*/, const void* view_v /*DEVICE*/, int32_t view_cap_tokens,
                       const int32_t* n_sel /*DEVICE*/, float scale, float* out /*DEVICE*/, float* lse /*DEVICE*/,
