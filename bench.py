@@ -237,6 +237,14 @@ def run_native(args):
                     ev[1].record(stream)
                     ev[2].record(stream)
                 return
+            if args.fp8:        # position-consistent FP8 view from bf16 pages: rotate, quantise, then FP8 attention
+                pool.materialize_fp8_rope(sel, n_sel, k8, v8t, 0)
+                if ev is not None:
+                    ev[1].record(stream)
+                pool.view_attend_fp8(q, k8, v8t, n_sel, out, lse)
+                if ev is not None:
+                    ev[2].record(stream)
+                return
             if args.paged:      # copy-free: raw key tiles are RoPE'd in shared memory on their way to the tensor cores
                 pool.paged_attend_rope(q, sel, n_sel, out, lse, 0)
                 if ev is not None:
@@ -369,6 +377,9 @@ def run_native(args):
             pool.select(q_raw, prm, sel, n_sel)
             if args.paged and args.fp8_pages:
                 pool.paged_attend_fp8_rope(q_stage, sel, n_sel, out, lse, 0)
+            elif args.fp8:
+                pool.materialize_fp8_rope(sel, n_sel, k8, v8t, 0)
+                pool.view_attend_fp8(q_stage, k8, v8t, n_sel, out, lse)
             elif args.paged:
                 pool.paged_attend_rope(q_stage, sel, n_sel, out, lse, 0)
             else:
@@ -571,7 +582,8 @@ def run_native(args):
             g_bytes = ns * ab["gather"] * 3 // 4
             a_bytes = ns * ab["attend"] // 2
             g_s, a_s = med(gat_ms) * 1e-3, med(att_ms) * 1e-3
-            line["config"]["calls"] = "kvmem_select + kvmem_materialize_fp8 + kvmem_view_attend_fp8 (E4M3 view, static scales 1.0)"
+            line["config"]["calls"] = ("kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_fp8_rope + kvmem_view_attend_fp8 (position-consistent E4M3 view)"
+                                       if args.rope else "kvmem_select + kvmem_materialize_fp8 + kvmem_view_attend_fp8 (E4M3 view, static scales 1.0)")
             line["dtype"] = "bf16 pages and query, E4M3 view, f16 tensor-core products, fp32 accumulation"
             if args.fp8_pages:      # FP8 repository: the gather copies 1-byte tiles; --paged reads them in place
                 g_bytes = ns * ab["gather"] // 2

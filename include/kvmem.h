@@ -391,6 +391,18 @@ int kvmem_view_attend_fp8(kvmem_pool_t* pool, int32_t n_sessions, const void* q 
                           const int32_t* n_sel /*DEVICE*/, float scale, float k_scale, float v_scale, float* out /*DEVICE*/,
                           float* lse /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
+/* Position-consistent FP8 execution view (Sec. 4.4 + Sec. 6.1) from a pool of bf16 pages with a rotary table: as
+ * kvmem_materialize_fp8, but the key of view token j*64 + t is first rotated to compact position first_position + j*64 + t
+ * (arithmetic of kvmem_rope_rotate, one rounding to bf16; with rope_in_block_keys the stored key is rotated by
+ * first_position + j*64) and then quantised: element = E4M3 code of RoPE(k, position)_bf16 / k_scale.  Values as in
+ * kvmem_materialize_fp8.  kvmem_view_attend_fp8 then attends over it with a q that carries RoPE at its own position.
+ * Extra errors: KVMEM_E_STATE without a rotary table or on an FP8 repository; KVMEM_E_INVALID if the compact positions
+ * leave the table. */
+int kvmem_materialize_fp8_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids /*DEVICE*/,
+                               int32_t sel_stride, const int32_t* n_sel /*DEVICE*/, void* view_k8 /*DEVICE*/,
+                               void* view_v8t /*DEVICE*/, int32_t view_cap_tokens, int32_t first_position, float k_scale,
+                               float v_scale, void* stream);
+
 /* On a pool created with fp8_pages: kvmem_materialize_fp8 copies the selected blocks' 8 KiB tiles as they are (1 byte
  * read + 1 byte written per element; k_scale and v_scale must be the pool's, KVMEM_E_INVALID otherwise), and
  * kvmem_paged_attend_fp8 is the copy-free execution view over such a repository (Sec. 5.3): attention straight

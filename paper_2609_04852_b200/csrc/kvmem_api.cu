@@ -856,6 +856,29 @@ int kvmem_materialize_fp8(kvmem_pool_t* p, int32_t session_first, int32_t n_sess
     return KVMEM_OK;
 }
 
+int kvmem_materialize_fp8_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_sessions, const int32_t* sel_ids, int32_t sel_stride,
+                               const int32_t* n_sel, void* view_k8, void* view_v8t, int32_t view_cap_tokens, int32_t first_position,
+                               float k_scale, float v_scale, void* stream) {
+    const int rc = fp8_common_ok(p, view_cap_tokens, k_scale, v_scale, "kvmem_materialize_fp8_rope");
+    if (rc != KVMEM_OK) return rc;
+    if (!pages_are(p, false, "kvmem_materialize_fp8_rope")) return KVMEM_E_STATE;
+    if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
+    if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    if (!sel_ids || !n_sel || !view_k8 || !view_v8t || !aligned(view_k8, 128) || !aligned(view_v8t, 128) || sel_stride < 1) {
+        set_error("kvmem_materialize_fp8_rope: null or misaligned pointer (views need 128-byte alignment), or sel_stride < 1");
+        return KVMEM_E_INVALID;
+    }
+    const int64_t last = (int64_t)first_position + std::min<int64_t>((int64_t)sel_stride * 64, view_cap_tokens);
+    if (first_position < 0 || last > p->cfg.rope_max_positions) {
+        set_error("compact positions [%d, %lld) outside the rotary table [0, %d)", first_position, (long long)last, p->cfg.rope_max_positions);
+        return KVMEM_E_INVALID;
+    }
+    cudaError_t e = launch_gather_fp8(*p, session_first, n_sessions, sel_ids, sel_stride, n_sel, (uint8_t*)view_k8,
+                                      (uint8_t*)view_v8t, view_cap_tokens, k_scale, v_scale, (cudaStream_t)stream, first_position);
+    if (e != cudaSuccess) return cuda_fail("rotating FP8 gather kernel launch", e);
+    return KVMEM_OK;
+}
+
 int kvmem_view_attend_fp8(kvmem_pool_t* p, int32_t n_sessions, const void* q, int32_t n_q_tokens, const void* view_k8,
                           const void* view_v8t, int32_t view_cap_tokens, const int32_t* n_sel, float scale, float k_scale,
                           float v_scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {

@@ -51,11 +51,15 @@ struct GatherF8Args {
     int session_first, sel_stride, max_bps, max_blocks, LG, cap_tokens;
     float k_inv_scale, v_inv_scale;
     size_t page_elems;
+    // position-consistent view: keys are rotated to compact position first_position + j*64 + t before they are quantised
+    const float2* rope;          // null: keys quantised as stored
+    int first_position, rope_positions, in_block;
 };
 
 // One CTA pass = one (selected block, layer x KV head): the K tile is quantised straight through, the V
 // tile goes through shared memory to come out transposed.  HBM: 2 bytes read + 1 byte written per element.
 constexpr int kF8Pitch = kF8D + 4;               // bytes per token row of the staging buffer (33 words: conflict-free columns)
+template <bool ROPE>
 __global__ void __launch_bounds__(256)
 gather_fp8_kernel(GatherF8Args a) {
     pdl_wait();
@@ -87,13 +91,30 @@ gather_fp8_kernel(GatherF8Args a) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int e = threadIdx.x + 256 * i;
-            kv[i] = __ldg(reinterpret_cast<const uint4*>(ksrc) + e);
+            // ROPE: a thread takes the low-half group (token, c) and its partner (token, c + 8) of the high half, which
+            // rotate together: groups 2 i and 2 i + 1 of the four are one such pair
+            const int ek = ROPE ? ((threadIdx.x + 256 * (i >> 1)) >> 3) * 16 + ((threadIdx.x + 256 * (i >> 1)) & 7) + 8 * (i & 1) : e;
+            kv[i] = __ldg(reinterpret_cast<const uint4*>(ksrc) + ek);
             vv[i] = __ldg(reinterpret_cast<const uint4*>(vsrc) + e);
+        }
+        if (ROPE) {
+            // RoPE at the compact position (arithmetic of kvmem_rope_rotate: fp32 products and sums, one rounding to bf16),
+            // then the quantisation of the rotated bf16 key: the code of the position-consistent view's element
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int item = threadIdx.x + 256 * h, tok = item >> 3, c = item & 7;
+                int pos = a.first_position + j * kF8Tile + (a.in_block ? 0 : tok);
+                if (pos < 0 || pos >= a.rope_positions) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); pos = 0; }
+                uint4 lo_o, hi_o;
+                rotate8(kv[2 * h], kv[2 * h + 1], a.rope + (size_t)pos * (kF8D / 2) + c * 8, 1.0f, lo_o, hi_o);
+                kv[2 * h] = lo_o; kv[2 * h + 1] = hi_o;
+            }
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int e = threadIdx.x + 256 * i;                  // token e / 16, dims 8 * (e % 16) ..
-            *reinterpret_cast<uint2*>(kdst + (size_t)e * 8) = quant8(kv[i], a.k_inv_scale);
+            const int ek = ROPE ? ((threadIdx.x + 256 * (i >> 1)) >> 3) * 16 + ((threadIdx.x + 256 * (i >> 1)) & 7) + 8 * (i & 1) : e;
+            *reinterpret_cast<uint2*>(kdst + (size_t)ek * 8) = quant8(kv[i], a.k_inv_scale);
             const uint2 q = quant8(vv[i], a.v_inv_scale);
             uint32_t* row = reinterpret_cast<uint32_t*>(sv + (e >> 4) * kF8Pitch + (e & 15) * 8);
             row[0] = q.x; row[1] = q.y;
@@ -676,7 +697,7 @@ static bool make_f8_map(CUtensorMap* map, const uint8_t* base, long long rows) {
 
 cudaError_t launch_gather_fp8(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids, int sel_stride,
                               const int32_t* n_sel, uint8_t* view_k, uint8_t* view_v, int view_cap_tokens, float k_scale,
-                              float v_scale, cudaStream_t st) {
+                              float v_scale, cudaStream_t st, int rope_first_position) {
     const Geometry& g = p.geo;
     GatherF8Args a{};
     a.pages = p.pages; a.tables = p.tables; a.nblocks_dev = p.nblocks_dev; a.sel_ids = sel_ids; a.n_sel = n_sel;
@@ -686,10 +707,14 @@ cudaError_t launch_gather_fp8(const kvmem_pool& p, int session_first, int n_sess
     a.page_elems = p.lay.page_elems;
     // about 64 short-lived CTAs per SM over the kernel's life (8 resident): 250 -> 240 us (quantising) and 176 -> 164 us (tile copy) at 1M
     const int ctas = g_gather_ctas > 0 ? g_gather_ctas : std::max(1, p.sm_count * 64 / n_sessions + 1);
+    a.rope = rope_first_position >= 0 ? p.rope_dev : nullptr;
+    a.first_position = rope_first_position; a.rope_positions = p.cfg.rope_max_positions; a.in_block = p.cfg.rope_in_block_keys;
     if (p.cfg.fp8_pages)
         launch_pdl(gather_fp8_pages_kernel, dim3((unsigned)ctas, (unsigned)n_sessions), dim3(256), 0, st, a);
+    else if (rope_first_position >= 0)
+        launch_pdl(gather_fp8_kernel<true>, dim3((unsigned)ctas, (unsigned)n_sessions), dim3(256), 0, st, a);
     else
-        launch_pdl(gather_fp8_kernel, dim3((unsigned)ctas, (unsigned)n_sessions), dim3(256), 0, st, a);
+        launch_pdl(gather_fp8_kernel<false>, dim3((unsigned)ctas, (unsigned)n_sessions), dim3(256), 0, st, a);
     return cudaGetLastError();
 }
 

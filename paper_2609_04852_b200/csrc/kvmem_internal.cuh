@@ -148,7 +148,7 @@ cudaError_t launch_score_host_index(kvmem_pool& p, const __nv_bfloat16* index_ho
 // FP8 (E4M3) execution view (kvmem_fp8.cu)
 cudaError_t launch_gather_fp8(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids, int sel_stride,
                               const int32_t* n_sel, uint8_t* view_k, uint8_t* view_v, int view_cap_tokens, float k_scale,
-                              float v_scale, cudaStream_t st);
+                              float v_scale, cudaStream_t st, int rope_first_position = -1);
 cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bfloat16* q, int M, const uint8_t* view_k,
                               const uint8_t* view_v, int view_cap_tokens, const int32_t* n_sel, float scale, float k_scale,
                               float v_scale, float* out, float* lse, void* workspace, cudaStream_t st,

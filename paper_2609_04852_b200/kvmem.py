@@ -94,6 +94,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
         "kvmem_paged_attend_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_materialize_attend_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, i32, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_materialize_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, f32, f32, vp]),
+        "kvmem_materialize_fp8_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, vp, vp, i32, i32, f32, f32, vp]),
         "kvmem_paged_attend_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp, vp, vp, sz, vp]),
         "kvmem_paged_attend_fp8_rope": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, i32, f32, vp, vp, vp, sz, vp]),
         "kvmem_materialize_attend_fp8": (C.c_int, [vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, i32, f32, vp, vp, vp, sz, vp]),
@@ -123,7 +124,8 @@ EXPORTED = ("kvmem_pool_bytes", "kvmem_budget_blocks", "kvmem_select_workspace_b
             "kvmem_view_cache_reset", "kvmem_view_cache_update", "kvmem_view_cache_attend", "kvmem_paged_attend_rope", "kvmem_topk", "kvmem_score_host_workspace_bytes",
             "kvmem_score_host_staging_bytes", "kvmem_score_host_index", "kvmem_materialize_fp8", "kvmem_view_attend_fp8",
             "kvmem_materialize_attend_rope", "kvmem_paged_attend_fp8", "kvmem_materialize_attend_fp8",
-            "kvmem_paged_attend_fp8_rope", "kvmem_selftest_wait_timeout", "kvmem_materialize_delta")
+            "kvmem_paged_attend_fp8_rope", "kvmem_selftest_wait_timeout", "kvmem_materialize_delta",
+            "kvmem_materialize_fp8_rope")
 
 
 def _check(status: int) -> None:
@@ -425,6 +427,14 @@ class Pool:
         _check(self.lib.kvmem_materialize_fp8(self.handle, session_first, ns, _dev(sel_ids, torch.int32), sel_ids.shape[-1],
                                               _dev(n_sel, torch.int32), _dev(k8, torch.uint8), _dev(v8t, torch.uint8),
                                               k8.shape[3], k_scale, v_scale, _stream()))
+
+    def materialize_fp8_rope(self, sel_ids: torch.Tensor, n_sel: torch.Tensor, k8: torch.Tensor, v8t: torch.Tensor,
+                             first_position: int = 0, k_scale: float = 1.0, v_scale: float = 1.0, session_first: int = 0) -> None:
+        """Position-consistent FP8 view: keys rotated to their compact positions, then quantised; values as materialize_fp8."""
+        ns = sel_ids.shape[0]
+        _check(self.lib.kvmem_materialize_fp8_rope(self.handle, session_first, ns, _dev(sel_ids, torch.int32), sel_ids.shape[-1],
+                                                   _dev(n_sel, torch.int32), _dev(k8, torch.uint8), _dev(v8t, torch.uint8),
+                                                   k8.shape[3], first_position, k_scale, v_scale, _stream()))
 
     def view_attend_fp8(self, q: torch.Tensor, k8: torch.Tensor, v8t: torch.Tensor, n_sel: torch.Tensor, out: torch.Tensor,
                         lse: torch.Tensor, k_scale: float = 1.0, v_scale: float = 1.0, scale: float = 0.0) -> None:

@@ -503,3 +503,46 @@ def test_query_rotating_copy_free_attention_with_other_block_sizes(B, n_blocks, 
     vK, vV = orc.gather_rope(repo, table, ids, T, first, tab, in_block=True)
     do, dl = orc.attend(qb[0], vK, vV, T)
     assert np.abs(out.cpu().numpy()[0] - do).max() <= REFORMULATION_ATOL and np.abs(lse.cpu().numpy()[0] - dl).max() <= REFORMULATION_ATOL
+
+
+# ------------------------------------------------------------------ position-consistent FP8 view
+
+@pytest.mark.parametrize("in_block,k,M,first,k_scale,v_scale", [(False, 20, 4, 517, 1.0, 1.0), (False, 33, 1, 0, 0.5, 0.25),
+                                                                (True, 20, 4, 131, 1.0, 1.0), (False, 1, 2, 64, 2.0, 1.0)])
+def test_position_consistent_fp8_view(in_block, k, M, first, k_scale, v_scale):
+    """kvmem_materialize_fp8_rope: the code of a key is the E4M3 code of the key rotated to its compact position (the
+    oracle's position-consistent gather, then its quantiser: both pinned); values as in the plain FP8 view.  Codes byte
+    for byte, then FP8 attention over the view against the oracle's."""
+    if in_block:
+        from test_gpu_rope_in_block import SPEC as RSPEC, _fill_both as fill
+        spec = RSPEC.with_(name="fp8rope_ib", n_q_tokens=M)
+        pool, repo, idx, tab, table = fill(spec, encoded=False)
+    else:
+        from test_gpu_rope import SPEC as RSPEC, _fill_both as fill
+        spec = RSPEC.with_(name="fp8rope", n_q_tokens=M)
+        pool, repo, idx, tab, table = fill(spec)
+    dev = torch.device("cuda", 0)
+    B = spec.block_tokens
+    ids = np.sort(np.random.default_rng(5 + k).choice(spec.n_blocks, size=k, replace=False)).astype(np.int32)
+    sel = torch.from_numpy(ids).view(1, -1).to(dev)
+    n_sel = torch.tensor([k], dtype=torch.int32, device=dev)
+    cap = k * B
+    g = Guards(dev)
+    k8 = g.empty((1, spec.n_layers, spec.n_kv_heads, cap, spec.head_dim), torch.uint8)
+    v8t = g.empty((1, spec.n_layers, spec.n_kv_heads, cap // 64, spec.head_dim, 64), torch.uint8)
+    pool.materialize_fp8_rope(sel, n_sel, k8, v8t, first, k_scale, v_scale)
+    q, qb = queries(spec)
+    out, lse = g.outputs(pool, 1, M)
+    pool.view_attend_fp8(q.to(dev), k8, v8t, n_sel, out, lse, k_scale, v_scale)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    g.check()
+    k_inv, v_inv = float(np.float32(1.0) / np.float32(k_scale)), float(np.float32(1.0) / np.float32(v_scale))
+    vK, _ = orc.gather_rope(repo, table, ids, cap, first, tab, in_block=in_block)       # the position-consistent bf16 keys
+    rK = orc.quantize_e4m3(vK, k_inv)
+    _, rV = orc.gather_fp8(repo, table, ids, cap, k_inv, v_inv)                         # values: quantised and transposed per tile
+    assert np.array_equal(k8.cpu().numpy()[0], rK), "FP8 codes of the rotated keys differ"
+    assert np.array_equal(v8t.cpu().numpy()[0], rV), "FP8 value codes differ"
+    ref_out, ref_lse = orc.attend_fp8(qb[0], rK, rV, cap, k_scale, v_scale)
+    err_o, err_l = np.abs(out.cpu().numpy()[0] - ref_out).max(), np.abs(lse.cpu().numpy()[0] - ref_lse).max()
+    assert err_o <= ATTN_ATOL * max(1.0, v_scale) and err_l <= ATTN_ATOL, (err_o, err_l)
