@@ -73,14 +73,31 @@ gather_fp8_kernel(GatherF8Args a) {
         n_blk = min(min(n_blk, a.sel_stride), cap_blocks);
     }
     n_blk = max(n_blk, 0);
-    const long long n_items = (long long)n_blk * a.LG;
+    // ROPE: an item is a whole selected block and the (layer, KV head) tiles are walked inside it, so that the rotary rows
+    // of the block's 64 positions are fetched once and serve every head
+    const int inner = ROPE ? a.LG : 1;
+    const long long n_items = ROPE ? (long long)n_blk : (long long)n_blk * a.LG;
     const int tile_elems = kF8Tile * kF8D;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const int j = (int)(item / a.LG), lg = (int)(item % a.LG);
+        const int j = ROPE ? (int)item : (int)(item / a.LG);
+        float4 cs[2][4];
+        if (ROPE) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int it2 = threadIdx.x + 256 * h, tok = it2 >> 3, c = it2 & 7;
+                int pos = a.first_position + j * kF8Tile + (a.in_block ? 0 : tok);
+                if (pos < 0 || pos >= a.rope_positions) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); pos = 0; }
+                const float4* cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)pos * (kF8D / 2) + c * 8);
+#pragma unroll
+                for (int w = 0; w < 4; ++w) cs[h][w] = __ldg(cs4 + w);
+            }
+        }
+        for (int in = 0; in < inner; ++in) {
+        const int lg = ROPE ? in : (int)(item % a.LG);
         const int id = a.sel_ids[(size_t)s * a.sel_stride + j];
         int page = -1;
         if (id >= 0 && id < NB) page = a.tables[(size_t)(a.session_first + s) * a.max_bps + id];
-        if (page < 0 || page >= a.max_blocks) { if (threadIdx.x == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); continue; }
+        if (page < 0 || page >= a.max_blocks) { if (threadIdx.x == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); break; }
         const __nv_bfloat16* ksrc = a.pages + (size_t)page * a.page_elems + (size_t)lg * tile_elems;
         const __nv_bfloat16* vsrc = ksrc + (size_t)a.LG * tile_elems;
         const size_t head = (size_t)s * a.LG + lg;
@@ -102,11 +119,8 @@ gather_fp8_kernel(GatherF8Args a) {
             // then the quantisation of the rotated bf16 key: the code of the position-consistent view's element
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const int item = threadIdx.x + 256 * h, tok = item >> 3, c = item & 7;
-                int pos = a.first_position + j * kF8Tile + (a.in_block ? 0 : tok);
-                if (pos < 0 || pos >= a.rope_positions) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); pos = 0; }
                 uint4 lo_o, hi_o;
-                rotate8(kv[2 * h], kv[2 * h + 1], a.rope + (size_t)pos * (kF8D / 2) + c * 8, 1.0f, lo_o, hi_o);
+                rotate8_cs(kv[2 * h], kv[2 * h + 1], cs[h], 1.0f, lo_o, hi_o);
                 kv[2 * h] = lo_o; kv[2 * h + 1] = hi_o;
             }
         }
@@ -136,6 +150,7 @@ gather_fp8_kernel(GatherF8Args a) {
             *reinterpret_cast<uint4*>(vdst + (size_t)dim * kF8Tile + tg * 16) = make_uint4(w[0], w[1], w[2], w[3]);
         }
         __syncthreads();
+        }       // tiles of the item
     }
 }
 
