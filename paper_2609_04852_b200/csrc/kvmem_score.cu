@@ -395,6 +395,17 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
     if ((int)(blockIdx.x * kFinishBlocks) >= NB) return;
     const int n_slots = LG * rows_pad;                        // rows incl. padding: slot = lg * rows_pad + j
     const float2* sess_parts = partials + (size_t)s * n_slots * n_parts;
+    // the logits of this thread's first head are requested before the statistics are merged: their round trip then
+    // overlaps the merge instead of following it
+    const int bl = threadIdx.x & 31, lgs = threadIdx.x >> 5;
+    const int b0 = blockIdx.x * kFinishBlocks + bl;
+    float pre[16];
+    const bool have_pre = rows <= 16 && b0 < NB && lgs < LG;
+    if (have_pre) {
+        const float* base = logits + (((size_t)s * LG + lgs) * rows_pad) * (size_t)nb_pad + b0;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) pre[j] = j < rows ? base[(size_t)j * nb_pad] : 0.0f;
+    }
     if (stage_parts) {
         const int n16 = n_slots * n_parts / 2;                // rows_pad is a multiple of 16: an even number of pairs
         const uint4* src = reinterpret_cast<const uint4*>(sess_parts);
@@ -429,17 +440,25 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
         if (live && sub == 0) rowstat[slot] = make_float2(mx, 1.0f / z);
     }
     __syncthreads();
-    const int bl = threadIdx.x & 31, lgs = threadIdx.x >> 5;
-    const int b0 = blockIdx.x * kFinishBlocks + bl;
     float part = 0.0f;
     if (b0 < NB) {
         for (int lg = lgs; lg < LG; lg += 8) {
             const float* base = logits + (((size_t)s * LG + lg) * rows_pad) * (size_t)nb_pad + b0;
             float sub = 0.0f;
+            if (have_pre && lg == lgs) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    if (j < rows) {
+                        const float2 st = rowstat[lg * rows_pad + j];
+                        sub += exp2f(pre[j] - st.x) * st.y;
+                    }
+                }
+            } else {
 #pragma unroll 16
-            for (int j = 0; j < rows; ++j) {
-                const float2 st = rowstat[lg * rows_pad + j];
-                sub += exp2f(base[(size_t)j * nb_pad] - st.x) * st.y;
+                for (int j = 0; j < rows; ++j) {
+                    const float2 st = rowstat[lg * rows_pad + j];
+                    sub += exp2f(base[(size_t)j * nb_pad] - st.x) * st.y;
+                }
             }
             part += sub;
         }
