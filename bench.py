@@ -453,7 +453,9 @@ def run_native(args):
                                    f"d={spec.head_dim}, budget {k} blocks ({cap} view tokens)",
                        "history_tokens": spec.tokens, "view_tokens": cap, "query_sets": len(qsets),
                        "l2": "flushed between steps (256 MiB write)" if flush is not None else
-                             "no flush: every step streams far more than the 126 MB L2",
+                             "no flush: every step streams far more than the 126 MB L2" if step_bytes > 8 * (126 << 20) else
+                             f"NO flush and {step_bytes / 1e6:.0f} MB per step against the 126 MB L2: partly L2-resident, "
+                             "a warm-cache figure (--flush-l2 for the cold one)",
                        "parallelism": f"{world} independent session replica(s), one per GPU",
                        "calls": "kvmem_rope_rotate(q) + kvmem_select + kvmem_paged_attend_rope (copy-free, pages hold RoPE(k, in-block offset), "
                                 "the query rotated back once per block)" if args.rope and args.paged and args.in_block else

@@ -729,21 +729,31 @@ attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__
     const int s = z / LG, lg = z % LG, l = lg / G, g = lg % G;
     const int col = threadIdx.x;
     const size_t p0 = (size_t)z * n_splits * rows_pad + row;          // split sp lives at p0 + sp * rows_pad
-    // eight splits at a time: the statistics and the partial outputs of a batch are loaded before any of them is used,
-    // so that a merge costs a few memory round trips instead of one per split (same split order, same arithmetic)
-    float mx = -INFINITY;
-    for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, part_ml[p0 + (size_t)sp * rows_pad].x);
-    float acc = 0.0f, lsum = 0.0f;
+    // eight splits at a time: the statistics and the partial outputs of a batch are loaded before any of them is used, and
+    // the first batch is requested together with the statistics the maximum needs, so that a merge costs a few memory
+    // round trips instead of one per split (same split order, same arithmetic)
     constexpr int U = 8;
-    for (int sp0 = 0; sp0 < n_splits; sp0 += U) {
-        float2 ml[U];
-        float po[U];
+    float2 ml[U];
+    float po[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int sp = min(sp0 + u, n_splits - 1);
-            const size_t pi = p0 + (size_t)sp * rows_pad;
-            ml[u] = part_ml[pi];
-            po[u] = part_o[pi * kD + col];
+    for (int u = 0; u < U; ++u) {
+        const size_t pi = p0 + (size_t)min(u, n_splits - 1) * rows_pad;
+        ml[u] = part_ml[pi];
+        po[u] = part_o[pi * kD + col];
+    }
+    float mx = -INFINITY;
+#pragma unroll
+    for (int u = 0; u < U; ++u) mx = fmaxf(mx, ml[u].x);
+    for (int sp = U; sp < n_splits; ++sp) mx = fmaxf(mx, part_ml[p0 + (size_t)sp * rows_pad].x);
+    float acc = 0.0f, lsum = 0.0f;
+    for (int sp0 = 0; sp0 < n_splits; sp0 += U) {
+        if (sp0 > 0) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const size_t pi = p0 + (size_t)min(sp0 + u, n_splits - 1) * rows_pad;
+                ml[u] = part_ml[pi];
+                po[u] = part_o[pi * kD + col];
+            }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {

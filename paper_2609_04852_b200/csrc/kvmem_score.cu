@@ -391,21 +391,22 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
     float2* staged = fin_smem + LG * rows_pad;
     __shared__ float red[8][kFinishBlocks];
     const int s = blockIdx.y;
-    const int NB = nb_override >= 0 ? nb_override : nblocks_dev[session_first + s];
-    if ((int)(blockIdx.x * kFinishBlocks) >= NB) return;
     const int n_slots = LG * rows_pad;                        // rows incl. padding: slot = lg * rows_pad + j
     const float2* sess_parts = partials + (size_t)s * n_slots * n_parts;
-    // the logits of this thread's first head are requested before the statistics are merged: their round trip then
-    // overlaps the merge instead of following it
+    // The kernel is a chain of memory round trips with little data behind them, so the first loads of every kind are
+    // requested together: the session's block count, the logits of this thread's first head (the logit rows are
+    // nb_pad long, so a column below nb_pad is readable whatever the count turns out to be) and the statistics.
     const int bl = threadIdx.x & 31, lgs = threadIdx.x >> 5;
     const int b0 = blockIdx.x * kFinishBlocks + bl;
     float pre[16];
-    const bool have_pre = rows <= 16 && b0 < NB && lgs < LG;
+    const bool have_pre = rows <= 16 && b0 < nb_pad && lgs < LG;
     if (have_pre) {
         const float* base = logits + (((size_t)s * LG + lgs) * rows_pad) * (size_t)nb_pad + b0;
 #pragma unroll
         for (int j = 0; j < 16; ++j) pre[j] = j < rows ? base[(size_t)j * nb_pad] : 0.0f;
     }
+    const int NB = nb_override >= 0 ? nb_override : nblocks_dev[session_first + s];
+    if ((int)(blockIdx.x * kFinishBlocks) >= NB) return;
     if (stage_parts) {
         const int n16 = n_slots * n_parts / 2;                // rows_pad is a multiple of 16: an even number of pairs
         const uint4* src = reinterpret_cast<const uint4*>(sess_parts);
@@ -506,6 +507,9 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     for (int s = session_first; s < session_first + n_sessions; ++s) max_nb = std::max(max_nb, p.sess_blocks[s]);
     if (max_nb == 0) return cudaSuccess;
     const int LG = g.L * g.G;
+    // One session: its block count is known here (the host's copy, which sized the grid anyway) and is handed to the
+    // kernels as an argument, which spares each of them a dependent read of the device copy before its first load.
+    const int nb_known = n_sessions == 1 ? max_nb : -1;
     const int chunks = (max_nb + kChunk - 1) / kChunk;
     // persistent CTAs: about one per SM, each streaming a contiguous range of chunks of one (session, l, g)
     // Two CTAs of the tensor-core kernel fit on an SM.  The second one is used only while the row statistics stay
@@ -529,7 +533,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
         }
         launch_pdl(score_logits_mma_kernel, dim3(grid), dim3(kScoreThreads), smem + 1024, st, 
             map_idx, q, p.nblocks_dev, session_first, M, g.L, g.H, g.G, g.max_bps, ws.logits, ws.partials, ws.rows,
-            ws.rows_pad, ws.nb_pad, n_parts, scale_log2e, p.status_dev, -1, 0, n_parts, 0);
+            ws.rows_pad, ws.nb_pad, n_parts, scale_log2e, p.status_dev, nb_known, 0, n_parts, 0);
     } else {
 #define KVMEM_SCORE_LAUNCH(RP)                                                                                         \
     do {                                                                                                               \
@@ -561,7 +565,7 @@ cudaError_t launch_score_decode(const kvmem_pool& p, int session_first, int n_se
     dim3 fgrid((unsigned)((max_nb + kFinishBlocks - 1) / kFinishBlocks), (unsigned)n_sessions);
     launch_pdl(score_finish_kernel, dim3(fgrid), dim3(256), fsmem, st, ws.logits, ws.partials, p.nblocks_dev, session_first, LG, ws.rows,
                                                    ws.rows_pad, ws.nb_pad, n_parts, score_scale / (float)(g.L * g.H),
-                                                   scores, scores_stride, stage_parts, -1);
+                                                   scores, scores_stride, stage_parts, nb_known);
     return cudaGetLastError();
 }
 

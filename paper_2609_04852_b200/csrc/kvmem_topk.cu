@@ -75,7 +75,10 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
     __shared__ TopkShared sh;
     extern __shared__ __align__(16) unsigned int stage[];   // [kTopkThreads][kStagePitch] score staging (REG), then kTopkTile output ids
     const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+    // The session's block count and its scores are requested together: the vector reads below are bounded by the row
+    // length (readable whatever the count is) and masked by the count afterwards, one memory round trip instead of two.
     const int NB = nblocks_dev[session_first + s];
+    const int row_len = scores_stride;
     const unsigned int* bits = reinterpret_cast<const unsigned int*>(scores + (size_t)s * scores_stride);
     int32_t* out = sel_ids + (size_t)s * sel_stride;
     constexpr int kItems = ITEMS, kTopkTile = kTopkThreads * ITEMS;      // shadow the file-scope values of the 16-item layout
@@ -86,15 +89,17 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
             for (int j = 0; j < ITEMS / 4; ++j) {
                 const int g4 = tid * (ITEMS / 4) + j;                      // ids 4*g4 .. 4*g4 + 3
                 uint4 u = make_uint4(0u, 0u, 0u, 0u);
-                if (4 * g4 + 3 < NB) {
+                if (4 * g4 + 3 < row_len) {
                     u = *reinterpret_cast<const uint4*>(bits + 4 * g4);
-                } else if (4 * g4 < NB) {
+                } else if (4 * g4 < row_len) {
                     u.x = bits[4 * g4];
-                    if (4 * g4 + 1 < NB) u.y = bits[4 * g4 + 1];
-                    if (4 * g4 + 2 < NB) u.z = bits[4 * g4 + 2];
+                    if (4 * g4 + 1 < row_len) u.y = bits[4 * g4 + 1];
+                    if (4 * g4 + 2 < row_len) u.z = bits[4 * g4 + 2];
                 }
                 vreg[(4 * j) % ITEMS] = u.x; vreg[(4 * j + 1) % ITEMS] = u.y; vreg[(4 * j + 2) % ITEMS] = u.z; vreg[(4 * j + 3) % ITEMS] = u.w;
             }
+#pragma unroll
+            for (int i = 0; i < ITEMS; ++i) vreg[i] = tid * ITEMS + i < NB ? vreg[i] : 0u;
         } else {
 #pragma unroll
             for (int i = 0; i < ITEMS; ++i) {
@@ -110,17 +115,21 @@ topk_kernel(const float* __restrict__ scores, int scores_stride, const int32_t* 
             for (int j = 0; j < kItems / 4; ++j) {
                 const int g4 = j * kTopkThreads + tid;                     // group of ids 4*g4 .. 4*g4 + 3
                 u[j] = make_uint4(0u, 0u, 0u, 0u);
-                if (4 * g4 + 3 < NB) {
+                if (4 * g4 + 3 < row_len) {
                     u[j] = *reinterpret_cast<const uint4*>(bits + 4 * g4);
-                } else if (4 * g4 < NB) {
+                } else if (4 * g4 < row_len) {
                     u[j].x = bits[4 * g4];
-                    if (4 * g4 + 1 < NB) u[j].y = bits[4 * g4 + 1];
-                    if (4 * g4 + 2 < NB) u[j].z = bits[4 * g4 + 2];
+                    if (4 * g4 + 1 < row_len) u[j].y = bits[4 * g4 + 1];
+                    if (4 * g4 + 2 < row_len) u[j].z = bits[4 * g4 + 2];
                 }
             }
 #pragma unroll
             for (int j = 0; j < kItems / 4; ++j) {
                 const int g4 = j * kTopkThreads + tid;
+                u[j].x = 4 * g4 < NB ? u[j].x : 0u;
+                u[j].y = 4 * g4 + 1 < NB ? u[j].y : 0u;
+                u[j].z = 4 * g4 + 2 < NB ? u[j].z : 0u;
+                u[j].w = 4 * g4 + 3 < NB ? u[j].w : 0u;
                 *reinterpret_cast<uint4*>(&stage[(g4 / (kItems / 4)) * kStagePitch + (g4 % (kItems / 4)) * 4]) = u[j];
             }
         } else {
