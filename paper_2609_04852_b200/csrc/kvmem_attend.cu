@@ -178,6 +178,19 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     // view length in tokens; the kernel works in 64-token tiles, whatever the block size of the view (a multiple of
     // 16, so each consumer warp's 16 tokens are all inside or all outside the view)
     const int btok = a.block_tokens;
+    // The producer's first page lookup is a chain of dependent reads (count of selected blocks, ids, block table) ahead of
+    // the first tile.  When the selection fills its row (the budget binds, the usual case) the ids this CTA starts at are
+    // known without the count, so they are requested together with it and used if the count confirms them.
+    int spec_j = -1, spec_id = -1;
+    if (PAGED && warp == CONSUMERS) {
+        const int n_sub = btok < kTile ? kTile / btok : 1, tpb = btok > kTile ? btok / kTile : 1;
+        const long long tok_h = min((long long)a.sel_stride * btok, (long long)a.cap_tokens);
+        const int blk_h = (int)((tok_h + kTile - 1) / kTile);
+        const int t0_h = (int)((long long)blk_h * split / a.n_splits);
+        spec_j = (t0_h * n_sub + lane) / tpb;
+        if (spec_j < a.sel_stride) spec_id = a.sel_ids[(size_t)s * a.sel_stride + spec_j];
+        else spec_j = -1;
+    }
     const long long n_tok_ll = min((long long)max(a.n_sel[s], 0) * btok, (long long)a.cap_tokens);
     const int n_tok = (int)n_tok_ll;
     const int n_blk = (n_tok + kTile - 1) / kTile;
@@ -234,7 +247,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             auto lookup = [&](int slot) -> int {
                 const int j = (t0 * n_sub + slot) / tpb;      // index in sel_ids
                 if (slot >= n_tiles * n_sub || j >= n_sel_blk) return -1;          // past this CTA's range or the view's ragged end
-                const int id = a.sel_ids[(size_t)s * a.sel_stride + j];
+                const int id = (slot == lane && j == spec_j) ? spec_id : a.sel_ids[(size_t)s * a.sel_stride + j];
                 int pg = -1;
                 if (id >= 0 && id < NB) pg = a.tables[(size_t)(a.session_first + s) * a.max_bps + id];
                 if (pg < 0 || pg >= a.max_blocks) { atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); pg = 0; }
@@ -720,6 +733,8 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 }
 
 // Merge the splits of one query row of one (session, layer, KV head) in split order; write O and LSE.
+// U splits are in flight at a time (8, or 24 when there are more than 8 splits: the usual 18 then take one round trip).
+template <int U>
 __global__ void __launch_bounds__(128)
 attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, float* __restrict__ out,
                     float* __restrict__ lse, int M, int L, int H, int G, int r, int n_splits, int rows_pad) {
@@ -729,10 +744,9 @@ attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__
     const int s = z / LG, lg = z % LG, l = lg / G, g = lg % G;
     const int col = threadIdx.x;
     const size_t p0 = (size_t)z * n_splits * rows_pad + row;          // split sp lives at p0 + sp * rows_pad
-    // eight splits at a time: the statistics and the partial outputs of a batch are loaded before any of them is used, and
+    // U splits at a time: the statistics and the partial outputs of a batch are loaded before any of them is used, and
     // the first batch is requested together with the statistics the maximum needs, so that a merge costs a few memory
     // round trips instead of one per split (same split order, same arithmetic)
-    constexpr int U = 8;
     float2 ml[U];
     float po[U];
 #pragma unroll
@@ -768,6 +782,17 @@ attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__
     const size_t orow = (((size_t)s * M + m) * L + l) * H + (size_t)g * r + hr;
     out[orow * kD + col] = lsum > 0.0f ? acc / lsum : 0.0f;
     if (col == 0) lse[orow] = lsum > 0.0f ? (mx + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
+}
+
+cudaError_t launch_attend_merge(const float* part_o, const float2* part_ml, float* out, float* lse, int rows, int heads, int M, int L,
+                                int H, int G, int r, int n_splits, int rows_pad, cudaStream_t st) {
+    if (n_splits <= 8)
+        launch_pdl(attend_merge_kernel<8>, dim3((unsigned)rows, (unsigned)heads), dim3(kD), 0, st, part_o, part_ml, out, lse, M, L, H, G, r,
+                   n_splits, rows_pad);
+    else
+        launch_pdl(attend_merge_kernel<24>, dim3((unsigned)rows, (unsigned)heads), dim3(kD), 0, st, part_o, part_ml, out, lse, M, L, H, G, r,
+                   n_splits, rows_pad);
+    return cudaGetLastError();
 }
 
 static PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
@@ -925,9 +950,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    launch_pdl(attend_merge_kernel, dim3(dim3((unsigned)a.rows, (unsigned)heads)), dim3(kD), 0, st, a.part_o, a.part_ml, out, lse, M, g.L, g.H, g.G,
-                                                                            g.r, a.n_splits, a.rows_pad);
-    return cudaGetLastError();
+    return launch_attend_merge(a.part_o, a.part_ml, out, lse, a.rows, heads, M, g.L, g.H, g.G, g.r, a.n_splits, a.rows_pad, st);
 }
 
 }  // namespace kvmem

@@ -681,9 +681,6 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     }
 }
 
-// defined with the bf16 kernel: merges the splits of a head in split order
-__global__ void attend_merge_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, float* __restrict__ out,
-                                    float* __restrict__ lse, int M, int L, int H, int G, int r, int n_splits, int rows_pad);
 
 static PFN_cuTensorMapEncodeTiled_v12000 f8_encode() {
     static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
@@ -805,9 +802,7 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
         launch_pdl(attend_fp8_split_kernel<0>, dim3(grid), dim3(kF8Threads), kF8Smem, st, map_k, map_v, map_pages, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    launch_pdl(attend_merge_kernel, dim3((unsigned)a.rows, (unsigned)heads), dim3(kF8D), 0, st, a.part_o, a.part_ml, out, lse, M, g.L,
-               g.H, g.G, g.r, a.n_splits, plan.rows_pad);
-    return cudaGetLastError();
+    return launch_attend_merge(a.part_o, a.part_ml, out, lse, a.rows, heads, M, g.L, g.H, g.G, g.r, a.n_splits, plan.rows_pad, st);
 }
 
 }  // namespace kvmem

@@ -211,6 +211,10 @@ cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, 
                         int32_t* n_sel, cudaStream_t st);
 
 // prev_ids != null: incremental view, slots whose block stays are skipped; delta_stats (may be null) receives the counts
+// merges the splits of every (session, layer, KV head) row in split order (defined with the bf16 attention kernel; the FP8
+// attention kernels write partials of the same layout and share it)
+cudaError_t launch_attend_merge(const float* part_o, const float2* part_ml, float* out, float* lse, int rows, int heads, int M, int L,
+                                int H, int G, int r, int n_splits, int rows_pad, cudaStream_t st);
 cudaError_t launch_gather(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids,
                           int sel_stride, const int32_t* n_sel, __nv_bfloat16* view_k, __nv_bfloat16* view_v,
                           int view_cap_tokens, cudaStream_t st, const int32_t* prev_ids = nullptr, const int32_t* n_prev = nullptr,
