@@ -27,15 +27,24 @@ constexpr int kAttConsumers = 8;
 constexpr int kAttGroups = 2;                   // consumer groups; kAttStages % kAttGroups == 0
 static_assert(kAttStages % kAttGroups == 0, "each group must own whole stages");
 constexpr int kAttThreads = (kAttConsumers + 1) * 32;
-constexpr int kAttRopeStages = 4;               // the position-consistent paged mode: data stages,
-constexpr int kAttRopeGroups = 2;               // consumer groups (one table buffer of rotary rows each)
+constexpr int kAttRopeStages = 6;               // the position-consistent raw-key modes: data stages,
+constexpr int kAttRopeGroups = 2;               // consumer groups
 constexpr int kAttRopeConsumers = 8;            // and consumer warps (12 warps in 3 groups spill at the 128-register cap: 345 us against 257)
 constexpr int kTile = 64;                       // tokens per tile: 64 / B selected blocks, or a 64-token slice of one
 constexpr int kD = 128;
-constexpr int kTabBytes = kTile * (kD / 2) * 8; // (cos, sin) fp32 of 64 pairs for 64 positions: 32 KiB
-static_assert(kAttRopeStages % kAttRopeGroups == 0 && kAttRopeConsumers % kAttRopeGroups == 0 &&
-                  kAttRopeStages * 4 * kTile * 128 + kAttRopeGroups * kTabBytes <= kAttStages * 4 * kTile * 128,
-              "the rotary mode's data stages and table buffers must fit the ring of the other modes");
+// Rotary angles of the raw-key modes.  A consumer warp owns 16 consecutive compact positions p1 .. p1 + 15 of a tile
+// (p1 = the tile's first position + 16 x the warp's index in its group).  The angle of pair i at p1 + b is the sum of its
+// angles at p1 and at b, so (cos, sin)(p1 + b) = (cos, sin)(p1) composed with (cos, sin)(b): the rows of offsets
+// b = 0 .. 15 are loaded once per CTA (8 KiB) and a tile brings only the four rows of its warps' p1 (2 KiB) instead of
+// the rows of all its 64 positions (32 KiB per tile and KV head, which made shared memory per tile in flight the bound
+// of these modes).  The composed values differ from the table's own row of p1 + b by fp32 rounding (a few units in the
+// last place of cos and sin), hence the rotated key by at most one bf16 rounding step on rare elements.
+constexpr int kRotRowBytes = (kD / 2) * 8;      // one table row: (cos, sin) fp32 of 64 pairs
+constexpr int kRopeShare = 16;                  // compact positions per consumer warp and tile
+constexpr int kOffsPitch = kRotRowBytes + 64;   // offset rows 576 B apart: the 128-bit reads of a quarter-warp (two rows) hit 32 different banks
+constexpr int kOffsBytes = kRopeShare * kOffsPitch;
+constexpr int kBaseBytes = (kTile / kRopeShare) * kRotRowBytes;        // per stage: the rows of p0, p0 + 16, p0 + 32, p0 + 48
+static_assert(kAttRopeStages % kAttRopeGroups == 0 && kAttRopeConsumers % kAttRopeGroups == 0, "each group must own whole stages");
 constexpr int kHalfBytes = kTile * 128;         // one 64-dim half of a tile: 64 rows x 128 B
 constexpr int kStageBytes = 4 * kHalfBytes;     // K lo, K hi, V lo, V hi
 constexpr int kMaxSplits = 64;
@@ -43,6 +52,7 @@ constexpr int kRowsPad = 16;                    // query rows of one m16 row til
 constexpr int kMaxRows = 64;                    // query rows per KV head and call: up to four row tiles
 constexpr int kMergeStride = 136;               // floats per merged row in shared memory
 constexpr size_t kAttSmem = (size_t)kAttStages * kStageBytes + 1024;
+constexpr size_t kAttSmemRope = (size_t)kAttRopeStages * (kStageBytes + kBaseBytes) + kOffsBytes + 1024;
 constexpr int kQrotBytes = kRowsPad * kD * 2;   // one rotated query tile: 16 rows x 256 B
 constexpr size_t kAttSmemQrot = kAttSmem + (size_t)kAttStages * kQrotBytes;
 constexpr int kQrotWarps = 2;                   // query-rotator warps; they take tiles alternately
@@ -142,7 +152,6 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     constexpr bool KWB = MODE == 6;        // ... and write them back into the stage, from where the view writer stores the tile
     constexpr bool QROT = MODE == 4;       // a rotator warp re-encodes the query per tile instead
     extern __shared__ unsigned char smem_dyn[];
-    // the rotary mode gives the room of two data stages to one buffer of rotary rows per consumer group
     static_assert(SUB == 1 || (MODE == 4 && (SUB == 2 || SUB == 4)), "several blocks per tile with their own rotation: the query-rotating mode only");
     constexpr int STAGES = ROPE ? kAttRopeStages : (QROT && SUB > 1) ? 4 : kAttStages;
     constexpr int CONSUMERS = ROPE ? kAttRopeConsumers : kAttConsumers;
@@ -150,7 +159,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     static_assert(RT == 1 || (MODE <= 2 && (RT == 2 || RT == 4)), "several row tiles: the plain modes only");
     constexpr int WPR = RT == 1 ? 4 : CONSUMERS / RT;      // consumer warps that share the tokens of a tile (for one row tile)
     constexpr int SLICES = 4 / WPR;                        // 16-token slices per warp and tile
-    __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages], tab_full[kAttRopeGroups], tab_empty[kAttRopeGroups];
+    __shared__ uint64_t full_bar[kAttStages], empty_bar[kAttStages], tab_full;      // tab_full: the raw-key modes' offset rows are in place
     __shared__ uint64_t q_full[kAttStages];     // MODE 4: rotated query of the stage's tile is in place; MODE 5: its K tile is rotated
     __shared__ float merge_m[kAttRopeConsumers][kRowsPad], merge_l[kAttRopeConsumers][kRowsPad];
 
@@ -167,7 +176,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             ptx::mbar_init(&full_bar[i], 1);
             ptx::mbar_init(&empty_bar[i], CONSUMERS / GROUPS + (FUSED ? 1 : 0));
         }
-        for (int i = 0; i < GROUPS; ++i) { ptx::mbar_init(&tab_full[i], 1); ptx::mbar_init(&tab_empty[i], CONSUMERS / GROUPS); }
+        ptx::mbar_init(&tab_full, 1);
         for (int i = 0; i < kAttStages; ++i) ptx::mbar_init(&q_full[i], KWB ? CONSUMERS / GROUPS : 1);
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(PAGED ? &map_pages : &map_k);
@@ -237,6 +246,14 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             // 64-token slice of one selected block (B >= 64).  The whole warp looks up pages, 32 slots at a time (a slot
             // is one block of a tile); lane 0 issues the loads.
             if (lane == 0) ptx::prefetch_tensormap(&map_pages);
+            unsigned char* const rot_offs = stages + (size_t)STAGES * kStageBytes;       // [16 offsets][64 pairs], rows kOffsPitch apart
+            unsigned char* const rot_base = rot_offs + kOffsBytes;                       // [STAGES][4 rows of 64 pairs]
+            if (ROPE && lane == 0) {
+                // rows of positions 0 .. 15, once per CTA and ahead of the page lookups
+                ptx::mbar_expect_tx(&tab_full, (uint32_t)kRopeShare * kRotRowBytes);
+                for (int b = 0; b < kRopeShare; ++b)
+                    ptx::bulk_g2s(rot_offs + (size_t)b * kOffsPitch, a.rope + (size_t)b * (kD / 2), kRotRowBytes, &tab_full);
+            }
             const int NB = a.nblocks_dev[a.session_first + s];
             const int B = btok;
             const int n_sub = B < kTile ? kTile / B : 1;      // selected blocks per tile
@@ -269,20 +286,19 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                                                     : ptx::mbar_wait(&empty_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1));
                         }
                         if (ok && it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
-                        if (ROPE && ok) {
-                            const int tb = it % GROUPS;
-                            if (it >= GROUPS) ok = ptx::mbar_wait(&tab_empty[tb], (uint32_t)(((it / GROUPS) & 1) ^ 1));
-                            if (ok) {
-                                const float2* rows = a.rope + (size_t)(a.first_position + (t0 + it) * kTile) * (kD / 2);
-                                ptx::mbar_expect_tx(&tab_full[tb], kTabBytes);
-                                ptx::bulk_g2s(stages + (size_t)STAGES * kStageBytes + (size_t)tb * kTabBytes, rows, kTabBytes, &tab_full[tb]);
-                            }
-                        }
                         if (ok) {
                             unsigned char* dst = stages + (size_t)st * kStageBytes;
                             // page layout [K|V][L*G][64 tokens][128]: rows of 256 B
                             const int yk = ((page * 2 + 0) * LG + lg) * kTile, yv = ((page * 2 + 1) * LG + lg) * kTile;
-                            ptx::mbar_expect_tx(&full_bar[st], kStageBytes);
+                            ptx::mbar_expect_tx(&full_bar[st], kStageBytes + (ROPE ? kBaseBytes : 0));
+                            if (ROPE) {
+                                // the rotary rows of the four warps' first positions travel with the tile
+                                const float2* rows = a.rope + (size_t)(a.first_position + (t0 + it) * kTile) * (kD / 2);
+#pragma unroll
+                                for (int w = 0; w < kTile / kRopeShare; ++w)
+                                    ptx::bulk_g2s(rot_base + (size_t)st * kBaseBytes + (size_t)w * kRotRowBytes,
+                                                  rows + (size_t)w * kRopeShare * (kD / 2), kRotRowBytes, &full_bar[st]);
+                            }
                             ptx::tma_load_2d(dst, &map_pages, 0, yk, &full_bar[st]);
                             ptx::tma_load_2d(dst + kHalfBytes, &map_pages, 64, yk, &full_bar[st]);
                             ptx::tma_load_2d(dst + 2 * kHalfBytes, &map_pages, 0, yv, &full_bar[st]);
@@ -314,23 +330,20 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                                                 : ptx::mbar_wait(&empty_bar[jt % STAGES], (uint32_t)((jt / STAGES) & 1));
                     }
                     if (ok && it >= STAGES) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / STAGES) & 1) ^ 1));
-                    if (ROPE && ok) {
-                        // the (cos, sin) rows of the tile's 64 compact positions are contiguous: one 32 KiB bulk copy
-                        const int tb = it % GROUPS;              // group tb consumes tile it: one table buffer per group
-                        if (it >= GROUPS) ok = ptx::mbar_wait(&tab_empty[tb], (uint32_t)(((it / GROUPS) & 1) ^ 1));
-                        if (ok) {
-                            const float2* rows = a.rope + (size_t)(a.first_position + (t0 + it) * kTile) * (kD / 2);
-                            ptx::mbar_expect_tx(&tab_full[tb], kTabBytes);
-                            ptx::bulk_g2s(stages + (size_t)STAGES * kStageBytes + (size_t)tb * kTabBytes, rows, kTabBytes, &tab_full[tb]);
-                        }
-                    }
                     if (ok) {
                         unsigned char* dst = stages + (size_t)st * kStageBytes;
                         int n_valid = 0;
 #pragma unroll
                         for (int u = 0; u < 4; ++u) n_valid += (u < n_sub && pages[u] >= 0) ? 1 : 0;
                         // page layout [K|V][L*G][B tokens][128]: rows of 256 B
-                        ptx::mbar_expect_tx(&full_bar[st], (uint32_t)n_valid * 4u * (uint32_t)box_rows * 128u);
+                        ptx::mbar_expect_tx(&full_bar[st], (uint32_t)n_valid * 4u * (uint32_t)box_rows * 128u + (ROPE ? (uint32_t)kBaseBytes : 0u));
+                        if (ROPE) {
+                            const float2* rows = a.rope + (size_t)(a.first_position + (t0 + it) * kTile) * (kD / 2);
+#pragma unroll
+                            for (int w = 0; w < kTile / kRopeShare; ++w)
+                                ptx::bulk_g2s(rot_base + (size_t)st * kBaseBytes + (size_t)w * kRotRowBytes,
+                                              rows + (size_t)w * kRopeShare * (kD / 2), kRotRowBytes, &full_bar[st]);
+                        }
                         const int row_in_block = ((t0 + it) % tpb) * kTile;
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
@@ -524,14 +537,13 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         for (int it = grp; it < n_tiles; it += GROUPS) {
             const int st = it % STAGES;
             bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / STAGES) & 1));
-            if (ROPE) arrived = arrived && ptx::mbar_wait(&tab_full[grp], (uint32_t)((it / GROUPS) & 1));
+            if (ROPE && it == grp) arrived = arrived && ptx::mbar_wait(&tab_full, 0u);       // the offset rows, once
             if (QROT || KROT) arrived = arrived && ptx::mbar_wait(&q_full[st], (uint32_t)((it / STAGES) & 1));
             if (!__all_sync(0xffffffffu, arrived)) {          // warp-uniform decision
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
             }
             bool k_handed_over = false;                      // KWB: this warp's share of the tile is rotated and back in the stage
-            bool tab_released = false;                       // ROPE: this warp has given the group's table buffer back
 #pragma unroll
             for (int sl = 0; sl < SLICES; ++sl) {
             const int wq = wq0 + sl;
@@ -573,7 +585,10 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 // Dimension i pairs with i + 64: the fragment of chunk cg (low half) and the one of chunk cg + 8
                 // (high half) sit in the same lane, so a lane rotates what it holds: registers lo[j], hi[j] carry
                 // dims 8 (4 kp + j) + 2 (lane & 3) + {0, 1} (+ 64) of token wq*16 + nt*8 + lane/4.
-                const unsigned char* tab = stages + (size_t)STAGES * kStageBytes + (size_t)grp * kTabBytes;   // [64 positions][64 pairs] (cos, sin)
+                // (cos, sin) of this lane's pairs at the warp's first position p1 (the row that came with the tile) and at
+                // the offsets b of its tokens inside the warp's share (the rows loaded once)
+                const unsigned char* rot_offs = stages + (size_t)STAGES * kStageBytes;
+                const unsigned char* base_row = rot_offs + kOffsBytes + (size_t)st * kBaseBytes + (size_t)wq * kRotRowBytes;
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt) {
                     const int tok = wq * 16 + nt * 8 + mr;
@@ -585,14 +600,18 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                         const uint32_t addr = kbase + (uint32_t)tok * 128u + (uint32_t)((c ^ (tok & 7)) << 4);
                         ptx::ldmatrix_x4(addr, lo[kp][0], lo[kp][1], lo[kp][2], lo[kp][3]);
                         ptx::ldmatrix_x4(addr + kHalfBytes, hi[kp][0], hi[kp][1], hi[kp][2], hi[kp][3]);
-                        const float4* row = reinterpret_cast<const float4*>(tab + (size_t)rtok * (kD * 4)) + (kp * 16 + (lane & 3));
+                        const float4* orow = reinterpret_cast<const float4*>(rot_offs + (size_t)(nt * 8 + (lane >> 2)) * kOffsPitch) + (kp * 16 + (lane & 3));
+                        const float4* brow = reinterpret_cast<const float4*>(base_row) + (kp * 16 + (lane & 3));
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const float4 t = row[j * 4];                          // pairs 8 (4 kp + j) + 2 (lane & 3) + {0, 1}
+                            const float4 o4 = orow[j * 4], b4 = brow[j * 4];      // pairs 8 (4 kp + j) + 2 (lane & 3) + {0, 1}
+                            float4 t;                                             // (cos, sin)(p1 + b) = (cos, sin)(p1) o (cos, sin)(b)
+                            t.x = fmaf(b4.x, o4.x, -(b4.y * o4.y)); t.y = fmaf(b4.y, o4.x, b4.x * o4.y);
+                            t.z = fmaf(b4.z, o4.z, -(b4.w * o4.w)); t.w = fmaf(b4.w, o4.z, b4.z * o4.w);
                             const float a0 = __uint_as_float(lo[kp][j] << 16), a1 = __uint_as_float(lo[kp][j] & 0xffff0000u);
                             const float b0 = __uint_as_float(hi[kp][j] << 16), b1 = __uint_as_float(hi[kp][j] & 0xffff0000u);
-                            const float l0 = __fsub_rn(__fmul_rn(a0, t.x), __fmul_rn(b0, t.y)), h0 = __fadd_rn(__fmul_rn(b0, t.x), __fmul_rn(a0, t.y));
-                            const float l1 = __fsub_rn(__fmul_rn(a1, t.z), __fmul_rn(b1, t.w)), h1 = __fadd_rn(__fmul_rn(b1, t.z), __fmul_rn(a1, t.w));
+                            const float l0 = fmaf(a0, t.x, -(b0 * t.y)), h0 = fmaf(b0, t.x, a0 * t.y);
+                            const float l1 = fmaf(a1, t.z, -(b1 * t.w)), h1 = fmaf(b1, t.z, a1 * t.w);
                             lo[kp][j] = ptx::pack_bf16x2(l0, l1);
                             hi[kp][j] = ptx::pack_bf16x2(h0, h1);
                             if (KWB) {
@@ -621,11 +640,6 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     if (lane == 0) ptx::mbar_arrive(&q_full[st]);
                     k_handed_over = true;
                 }
-                // the rotary rows are done with: the group's table buffer goes back now, so that the rows of its next
-                // tile load during the softmax and the P V products instead of after them
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&tab_empty[grp]);
-                tab_released = true;
             }
             // online softmax (exp2 domain); this thread holds rows lane/4 (c0,c1) and lane/4 + 8 (c2,c3)
             float mx0 = -INFINITY, mx1 = -INFINITY;
@@ -677,10 +691,7 @@ attend_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (lane == 0) ptx::mbar_arrive(&q_full[st]);
             }
             __syncwarp();
-            if (lane == 0) {
-                ptx::mbar_arrive(&empty_bar[st]);
-                if (ROPE && !tab_released) ptx::mbar_arrive(&tab_empty[grp]);
-            }
+            if (lane == 0) ptx::mbar_arrive(&empty_bar[st]);
         }
         // row sums live spread over the 4 lanes of a quad
         l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1); l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
@@ -871,7 +882,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attend_split_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+            e = cudaFuncSetAttribute(attend_split_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmemRope);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmemQrot);
         if (e == cudaSuccess)
@@ -881,7 +892,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attend_split_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attend_split_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmem);
+            e = cudaFuncSetAttribute(attend_split_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttSmemRope);
         if (e != cudaSuccess) return e;
         attr_done.mark(p.cfg.device);
     }
@@ -923,6 +934,9 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
             a.lookahead = std::max(2, std::min(kAttStages, (int)(target / ((double)ctas * kStageBytes) + 0.5)));
         }
     }
+    // the copy-free raw-key pass is bound by what its consumer warps issue per tile, not by HBM: every stage in flight
+    // (233 us per step at a 1M-token history against 249 with five and 305 with four)
+    if (paged_only && rope_first_position >= 0 && !p.cfg.rope_in_block_keys && g_attend_lookahead == 0) a.lookahead = kAttRopeStages;
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
     if (paged_only && rope_first_position >= 0 && p.cfg.rope_in_block_keys && g.B == 32)
         launch_pdl(attend_split_kernel<4, 1, 2>, dim3(grid), dim3(kAttThreads + 32 * kQrotWarps), kAttSmemQrot, st, map_k, map_v, map_pages, a);
@@ -931,11 +945,11 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     else if (paged_only && rope_first_position >= 0 && p.cfg.rope_in_block_keys)
         launch_pdl(attend_split_kernel<4>, dim3(grid), dim3(kAttThreads + 32 * kQrotWarps), kAttSmemQrot, st, map_k, map_v, map_pages, a);
     else if (paged_only && rope_first_position >= 0)
-        launch_pdl(attend_split_kernel<3>, dim3(grid), dim3((kAttRopeConsumers + 1) * 32), kAttSmem, st, map_k, map_v, map_pages, a);
+        launch_pdl(attend_split_kernel<3>, dim3(grid), dim3((kAttRopeConsumers + 1) * 32), kAttSmemRope, st, map_k, map_v, map_pages, a);
     else if (fused && !paged_only && rope_first_position >= 0 && p.cfg.rope_in_block_keys)
         launch_pdl(attend_split_kernel<5>, dim3(grid), dim3(kAttThreads + 32 + 32 * kKrotWarps), kAttSmem, st, map_k, map_v, map_pages, a);
     else if (fused && !paged_only && rope_first_position >= 0)
-        launch_pdl(attend_split_kernel<6>, dim3(grid), dim3((kAttRopeConsumers + 2) * 32), kAttSmem, st, map_k, map_v, map_pages, a);
+        launch_pdl(attend_split_kernel<6>, dim3(grid), dim3((kAttRopeConsumers + 2) * 32), kAttSmemRope, st, map_k, map_v, map_pages, a);
     else {
 #define KVMEM_ATTEND_LAUNCH(MODE, THREADS)                                                                              \
     do {                                                                                                                \

@@ -119,6 +119,32 @@ ATTN_ATOL = 2e-3           # max-abs on unit-scale values, outputs and log-sum-e
 GAP_RTOL = 1e-3            # ids must be identical where the relative gap at the k-th boundary exceeds this
 
 
+# Keys rotated by COMPOSED angles (the raw-key one-pass and copy-free modes): the kernel forms (cos, sin)(p1 + b) from the
+# table rows of p1 and of b, four fp32 operations whose result is within 3 units in the last place (3 * 2^-24 relative to
+# 1) of the table's own row of p1 + b.  A rotated key a*cos - b*sin therefore moves by at most 3 * 2^-24 * (|a| + |b|)
+# < 4e-6 for keys below 10 in magnitude before its rounding to bf16, which shifts the stored code by at most one bf16 step
+# (2^-8 relative) unless the rotated value is itself tiny next to its inputs.  An element sits that close to a rounding
+# boundary with probability about (4e-6 * 2) / (2^-9 |k|), far below one in a hundred.
+ROTATED_KEY_ABS = 4e-6
+ROTATED_KEY_MAX_DIFFERING = 1e-2
+
+
+def check_rotated_keys(view_bits: np.ndarray, ref_bits: np.ndarray) -> None:
+    """view_bits, ref_bits: bf16 codes (uint16) of rotated keys; equal up to one bf16 rounding step (plus the absolute
+    slack above) on a small fraction of the elements."""
+    assert view_bits.shape == ref_bits.shape and view_bits.dtype == np.uint16 and ref_bits.dtype == np.uint16
+    differing = view_bits != ref_bits
+    if not differing.any():
+        return
+    frac = differing.mean()
+    assert frac <= ROTATED_KEY_MAX_DIFFERING, f"{frac:.2e} of the rotated keys differ from the defined code"
+    got = (view_bits[differing].astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    ref = (ref_bits[differing].astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    bound = np.abs(ref) * 2.0 ** -7 + ROTATED_KEY_ABS     # one step of the binade above (a step doubles across a power of two)
+    worst = np.abs(got - ref) - bound
+    assert worst.max() <= 0, f"a rotated key is off by more than one bf16 step: {got[worst.argmax()]} against {ref[worst.argmax()]}"
+
+
 def check_scores(R_gpu: np.ndarray, R_ref: np.ndarray, M: int) -> None:
     floor = 1e-6 * M / max(len(R_ref), 1)      # a millionth of the mean score: only matters near underflow
     err = np.abs(R_gpu - R_ref)

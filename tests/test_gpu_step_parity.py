@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 import torch
 
-from kvmem_harness import ATTN_ATOL, Guards, bits, fill_oracle, fill_pool, full_step, queries
+from kvmem_harness import ATTN_ATOL, Guards, bits, check_rotated_keys, fill_oracle, fill_pool, full_step, queries
 from kvmem_workloads import CONFIGS, kv_blocks, page_table
 from oracle import kvmem_oracle as orc
 
@@ -384,8 +384,10 @@ def test_thirty_two_rows_at_32_token_blocks_and_two_sessions():
                                                       (32, 200, 21, 4, 131), (16, 300, 37, 2, 0), (128, 40, 9, 4, 64)])
 def test_position_consistent_view_and_attention_in_one_pass_over_raw_keys(B, n_blocks, budget, M, first):
     """kvmem_materialize_attend_rope on a pool of raw keys: the warps that attend over a tile rotate its keys to their
-    compact positions and hand them back for the store.  The view must be the defined code (oracle gather with RoPE,
-    bit for bit), the results those of attention over it, and both identical to the two separate calls."""
+    compact positions (angles composed from the table rows of the warp's first position and of the offset inside its
+    share) and hand them back for the store.  Values are copied bit for bit; a rotated key may differ from the defined code
+    (oracle gather with RoPE) by one bf16 rounding step on a small fraction of the elements; the results are those of
+    attention over the defined view within the attention tolerance, and they are the copy-free pass's bit for bit."""
     from test_gpu_rope import SPEC as RSPEC, _fill_both
     spec = RSPEC.with_(name=f"rawfusedB{B}", block_tokens=B, n_blocks=n_blocks, budget_blocks=budget, n_q_tokens=M)
     dev = torch.device("cuda", 0)
@@ -408,12 +410,18 @@ def test_position_consistent_view_and_attention_in_one_pass_over_raw_keys(B, n_b
     assert pool.device_status() == 0
     g.check()
     vK, vV = orc.gather_rope(repo, table, ids, T, first, tab)
-    assert np.array_equal(bits(view.k[0]), vK), "one-pass view: rotated keys differ from the defined code"
+    check_rotated_keys(bits(view.k[0]), vK)
     assert np.array_equal(bits(view.v[0]), vV)
     ref_out, ref_lse = orc.attend(qb[0], vK, vV, T)
     assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
-    assert torch.equal(view.k, view2.k) and torch.equal(view.v, view2.v)
-    assert torch.equal(out, out2) and torch.equal(lse, lse2)
+    # the separate calls rotate by the table's own rows: their view IS the defined code
+    assert np.array_equal(bits(view2.k[0]), vK) and torch.equal(view.v, view2.v)
+    assert np.abs(out2.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse2.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+    out3, lse3 = g.outputs(pool, 1, M)
+    pool.paged_attend_rope(qd, sel, n_sel, out3, lse3, first)
+    torch.cuda.synchronize()
+    g.check()
+    assert torch.equal(out3, out) and torch.equal(lse3, lse), "copy-free and one-pass rotate the same fragments the same way"
 
 
 # ------------------------------------------------------------------ incremental contiguous view
