@@ -318,12 +318,15 @@ int kvmem_paged_attend(kvmem_pool_t* pool, int32_t session_first, int32_t n_sess
 
 /* Copy-free execution view with position-consistent keys (Sec. 4.4: the view is a page table over the
  * physical pages, and RoPE is applied to raw K at the block's assigned compact position): as
- * kvmem_paged_attend, but every key tile is rotated in shared memory, between its arrival from the
- * pages and its use, to compact position first_position + j*block_tokens + t (j = index in sel_ids),
- * with the arithmetic of kvmem_rope_rotate.  out and lse equal kvmem_view_attend's on the view
- * kvmem_materialize_rope would build from the same ids; nothing is written besides out and lse.  The
- * pool's pages must hold raw keys and q must carry RoPE at its own position.  HBM traffic: one read per
- * view byte plus the rotary table rows of the view's positions.
+ * kvmem_paged_attend, but the warps that attend over a tile rotate their key fragments, between the tile's
+ * arrival from the pages and their use, to compact position first_position + j*block_tokens + t (j = index in
+ * sel_ids).  The angle of a position p1 + b (p1 the first of a warp's 16 positions, b < 16) is composed from the
+ * table rows of p1 and of b: cos and sin within a few fp32 units in the last place of the table's own row, so a
+ * rotated key is within one bf16 rounding step of kvmem_rope_rotate's, and out and lse are those of
+ * kvmem_view_attend on the view kvmem_materialize_rope would build from the same ids within the attention
+ * tolerance (not bit for bit); they equal kvmem_materialize_attend_rope's on a raw-key pool bit for bit.  Nothing is
+ * written besides out and lse.  The pool's pages must hold raw keys and q must carry RoPE at its own position.
+ * HBM traffic: one read per view byte (the rotary rows are 2 KiB per 64-token tile).
  * On a pool created with rope_in_block_keys (pages hold k' = RoPE(k, t)) no key is rotated: the logit
  * q . R(p0 + t) k equals (R(-p0) q) . k', p0 = first_position + j*block_tokens, so the 16 query rows are rotated
  * back by p0 once per block (arithmetic of kvmem_rope_rotate, inverse; the rotated query is a bf16 vector)
@@ -338,12 +341,17 @@ int kvmem_paged_attend_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n
 
 /* kvmem_materialize_rope followed by kvmem_view_attend in one call (Sec. 4.4: the execution view with keys
  * encoded at their compact positions, then decode over it).  Same arguments as kvmem_materialize_attend plus
- * first_position; the view left behind is kvmem_materialize_rope's, out/lse are kvmem_view_attend's on it with
- * a q that carries RoPE at its own position.  ONE pass, 1 read + 1 write per view byte: on a pool with
- * rope_in_block_keys each K tile is rotated by its block's compact position while it sits in shared memory, then stored
- * and attended over; on a raw-key pool the warps that attend over a tile rotate its key fragments to their compact
- * positions on the way to the tensor cores and hand them back to the tile, which is then stored (the view's last
- * 64-token tile must lie inside the rotary table: first_position + the view length rounded up to 64).
+ * first_position and a q that carries RoPE at its own position.  ONE pass, 1 read + 1 write per view byte.
+ * On a pool with rope_in_block_keys each K tile is rotated by its block's compact position while it sits in shared
+ * memory, then stored and attended over: the view left behind is kvmem_materialize_rope's and out/lse are
+ * kvmem_view_attend's on it, bit for bit.
+ * On a raw-key pool the warps that attend over a tile rotate its key fragments to their compact positions on the way
+ * to the tensor cores and hand them back to the tile, which is then stored.  Their angles are composed from two
+ * table rows as in kvmem_paged_attend_rope, so the view's VALUES are kvmem_materialize_rope's bit for bit and its KEYS
+ * are within one bf16 rounding step of them (a small fraction of the elements differs at all); out/lse are the
+ * attention over the view this call writes.  Callers that need the key bytes of kvmem_materialize_rope exactly use
+ * that call and kvmem_view_attend.  (The view's last 64-token tile must lie inside the rotary table: first_position +
+ * the view length rounded up to 64.)
  * Extra errors: KVMEM_E_STATE without a rotary table; KVMEM_E_INVALID if the compact positions leave it. */
 int kvmem_materialize_attend_rope(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
                                   int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
