@@ -186,3 +186,21 @@ def test_query_rotation_at_position_zero_is_plain_attention_over_the_stored_keys
     _, l0 = orc.attend(q, sK2[:, :, :B].copy(), sV2[:, :, :B].copy(), B)
     _, l1 = orc.attend(q_rot, sK2[:, :, B:].copy(), sV2[:, :, B:].copy(), B)
     assert np.allclose(l_both, np.logaddexp(l0, l1), atol=1e-5)
+
+
+def test_composed_angles_stay_within_three_fp32_steps_of_the_table():
+    """The bound behind the tolerance on keys rotated with composed angles: (cos, sin)(p1 + b) formed in fp32 from the
+    table rows of p1 and b (two products, two fused multiply-adds) is within 3 * 2^-24 of the table's own row of p1 + b,
+    for every warp share (b < 16) of a long window."""
+    d, n = 128, 1 << 15
+    tab = orc.rope_table(n, d, THETA)
+    p1 = np.arange(0, n - 16, 16, dtype=np.int64)
+    worst = 0.0
+    for b in range(16):
+        cb, sb = tab[p1, :, 0], tab[p1, :, 1]
+        co, so = tab[b, :, 0][None, :], tab[b, :, 1][None, :]
+        # fp32 products rounded once, then a fused multiply-add (exact product, one rounding): emulated in fp64
+        c = (cb.astype(np.float64) * co.astype(np.float64) - (sb * so).astype(np.float64)).astype(np.float32)
+        s = (sb.astype(np.float64) * co.astype(np.float64) + (cb * so).astype(np.float64)).astype(np.float32)
+        worst = max(worst, float(np.abs(c - tab[p1 + b, :, 0]).max()), float(np.abs(s - tab[p1 + b, :, 1]).max()))
+    assert worst <= 3 * 2.0 ** -24, worst
