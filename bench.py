@@ -273,7 +273,7 @@ def run_native(args):
                 ev[1].record(stream)
                 ev[2].record(stream)
             return
-        if args.fp8_pages and not args.unfused:  # FP8 repository: tiles stored to the view while attended over, one pass
+        if args.fp8 and not args.unfused:  # tiles (quantised on the way from bf16 pages) stored to the FP8 view while attended over, one pass
             pool.materialize_attend_fp8(q, sel, n_sel, k8, v8t, out, lse)
             if ev is not None:
                 ev[1].record(stream)
@@ -392,7 +392,7 @@ def run_native(args):
             pool.select(q_stage, prm, sel, n_sel)
             if args.fp8_pages and args.paged:
                 pool.paged_attend_fp8(q_stage, sel, n_sel, out, lse)
-            elif args.fp8_pages and not args.unfused:
+            elif not args.unfused:
                 pool.materialize_attend_fp8(q_stage, sel, n_sel, k8, v8t, out, lse)
             else:
                 pool.materialize_fp8(sel, n_sel, k8, v8t)
@@ -587,6 +587,11 @@ def run_native(args):
             line["config"]["calls"] = ("kvmem_rope_rotate(q) + kvmem_select + kvmem_materialize_fp8_rope + kvmem_view_attend_fp8 (position-consistent E4M3 view)"
                                        if args.rope else "kvmem_select + kvmem_materialize_fp8 + kvmem_view_attend_fp8 (E4M3 view, static scales 1.0)")
             line["dtype"] = "bf16 pages and query, E4M3 view, f16 tensor-core products, fp32 accumulation"
+            one_pass_bf16 = not args.fp8_pages and not args.rope and not args.unfused
+            if one_pass_bf16:       # bf16 pages quantised on their way to the view and to the tensor cores: no second read of the view
+                a_bytes, a_s = 0, 1.0
+                line["config"]["calls"] = ("kvmem_select + kvmem_materialize_attend_fp8 (bf16 repository: tiles quantised on the way, "
+                                           "E4M3 view written while attended, static scales 1.0)")
             if args.fp8_pages:      # FP8 repository: the gather copies 1-byte tiles; --paged reads them in place
                 g_bytes = ns * ab["gather"] // 2
                 line["dtype"] = "E4M3 pages (quantised at append), bf16 query and index, f16 tensor-core products, fp32 accumulation"
@@ -600,6 +605,7 @@ def run_native(args):
             line["roofline"] = {"bound": "hbm", "kernel": "attend_fp8_split_kernel<paged> + merge (kvmem_paged_attend_fp8)" if args.fp8_pages and args.paged else
                                                            "attend_fp8_split_kernel<2> + merge (kvmem_materialize_attend_fp8)" if args.fp8_pages and not args.unfused else
                                                            "gather_fp8_pages_kernel (kvmem_materialize_fp8)" if args.fp8_pages else
+                                                           "attend_fp8_split_kernel<4> + merge (kvmem_materialize_attend_fp8 over bf16 pages)" if one_pass_bf16 else
                                                            "gather_fp8_kernel (kvmem_materialize_fp8)", "achieved": g_bytes / g_s / 1e9,
                                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": g_bytes / g_s / 1e9 / peaks["hbm_gbs"],
                                 "peak_source": f"of {peaks['source']}", "algorithmic_bytes_per_launch": g_bytes,
@@ -607,12 +613,13 @@ def run_native(args):
             line["attend_roofline"] = {"kernel": "attend_fp8_split_kernel + merge (kvmem_view_attend_fp8)", "achieved_gbs": a_bytes / a_s / 1e9,
                                        "frac": a_bytes / a_s / 1e9 / peaks["hbm_gbs"], "algorithmic_bytes_per_launch": a_bytes,
                                        "avg_ms": a_s * 1e3}
-            if args.fp8_pages and (args.paged or not args.unfused):
+            if (args.fp8_pages and (args.paged or not args.unfused)) or one_pass_bf16:
                 line.pop("attend_roofline")
             fp8_step = ns * ab["index"] + g_bytes + a_bytes
             line["step_hbm"] = {"algorithmic_bytes_per_step": fp8_step, "accounting": "index + one read of the selected FP8 pages" if args.fp8_pages and args.paged else
                                 "index + FP8 page read + FP8 view write (fused pass)" if args.fp8_pages and not args.unfused else
-                                "index + FP8 page read + FP8 view write + FP8 view read" if args.fp8_pages else "index + bf16 page read + FP8 view write + FP8 view read",
+                                "index + FP8 page read + FP8 view write + FP8 view read" if args.fp8_pages else
+                                "index + bf16 page read + FP8 view write (fused pass)" if one_pass_bf16 else "index + bf16 page read + FP8 view write + FP8 view read",
                                 "achieved_gbs": K * fp8_step / (total_ms * 1e-3) / 1e9,
                                 "frac_of_peak": K * fp8_step / (total_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                 "peak_source": f"of {peaks['source']}", "nominal_peak_gbs": 8000.0}

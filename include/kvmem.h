@@ -437,10 +437,12 @@ int kvmem_paged_attend_fp8_rope(kvmem_pool_t* pool, int32_t session_first, int32
                                 const int32_t* n_sel /*DEVICE*/, int32_t first_position, float scale, float* out /*DEVICE*/,
                                 float* lse /*DEVICE*/, void* workspace /*DEVICE*/, size_t workspace_bytes, void* stream);
 
-/* kvmem_materialize_fp8 followed by kvmem_view_attend_fp8 as ONE pass over an FP8 repository: every selected tile is
- * read once from the pages, stored to its place in the FP8 view and attended over while it sits in shared memory
- * (1 byte read + 1 byte written per element).  The view and out/lse are those of the two separate calls with the
- * pool's scales.  Arguments as kvmem_materialize_attend with the FP8 view buffers.  KVMEM_E_STATE on bf16 pages. */
+/* kvmem_materialize_fp8 followed by kvmem_view_attend_fp8 as ONE pass: every selected tile is read once from the pages,
+ * stored to its place in the FP8 view and attended over while it sits in shared memory.  Over an FP8 repository that is
+ * 1 byte read + 1 byte written per element; over a bf16 repository (64-token blocks) the tile is quantised on the way
+ * (2 bytes read + 1 byte written per element; arithmetic of kvmem_materialize_fp8) with the pool's fp8_k_scale and
+ * fp8_v_scale, 1 where the configuration leaves them at 0.  The view and out/lse are those of the two separate calls
+ * with the same scales, bit for bit.  Arguments as kvmem_materialize_attend with the FP8 view buffers. */
 int kvmem_materialize_attend_fp8(kvmem_pool_t* pool, int32_t session_first, int32_t n_sessions, const void* q /*DEVICE*/,
                                  int32_t n_q_tokens, const int32_t* sel_ids /*DEVICE*/, int32_t sel_stride,
                                  const int32_t* n_sel /*DEVICE*/, void* view_k8 /*DEVICE*/, void* view_v8t /*DEVICE*/,

@@ -960,8 +960,15 @@ int kvmem_materialize_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t
                                  const int32_t* sel_ids, int32_t sel_stride, const int32_t* n_sel, void* view_k8, void* view_v8t,
                                  int32_t view_cap_tokens, float scale, float* out, float* lse, void* workspace,
                                  size_t workspace_bytes, void* stream) {
-    if (!pool_live(p) || !pages_are(p, true, "kvmem_materialize_attend_fp8")) return KVMEM_E_STATE;
+    if (!pool_live(p)) return KVMEM_E_STATE;
+    if (p->cfg.head_dim != 128 || p->cfg.block_tokens != 64) {
+        set_error("kvmem_materialize_attend_fp8: the FP8 view kernels are built for head_dim 128 and 64-token blocks");
+        return KVMEM_E_UNSUPPORTED;
+    }
     if (!sessions_ok(p, session_first, n_sessions)) return KVMEM_E_INVALID;
+    // a bf16 repository is quantised on the way with the pool's scales, 1 where the configuration leaves them unset
+    const float k_scale = p->cfg.fp8_k_scale > 0.0f && std::isfinite(p->cfg.fp8_k_scale) ? p->cfg.fp8_k_scale : 1.0f;
+    const float v_scale = p->cfg.fp8_v_scale > 0.0f && std::isfinite(p->cfg.fp8_v_scale) ? p->cfg.fp8_v_scale : 1.0f;
     if (!q || !sel_ids || !n_sel || !view_k8 || !view_v8t || !out || !lse || !workspace || !aligned(q, 16) || !aligned(view_k8, 128) ||
         !aligned(view_v8t, 128) || !aligned(workspace, 256) || !aligned(out, 16)) {
         set_error("kvmem_materialize_attend_fp8: null or misaligned pointer (views need 128-byte alignment)");
@@ -979,7 +986,7 @@ int kvmem_materialize_attend_fp8(kvmem_pool_t* p, int32_t session_first, int32_t
     AttendPlan plan = plan_attend(p->cfg, n_sessions, n_q_tokens, p->sm_count);
     if (workspace_bytes < plan.total) { set_error("attend workspace holds %zu bytes, %zu needed", workspace_bytes, plan.total); return KVMEM_E_CAPACITY; }
     cudaError_t e = launch_attend_fp8(*p, n_sessions, (const __nv_bfloat16*)q, n_q_tokens, (const uint8_t*)view_k8,
-                                      (const uint8_t*)view_v8t, view_cap_tokens, n_sel, scale, p->cfg.fp8_k_scale, p->cfg.fp8_v_scale,
+                                      (const uint8_t*)view_v8t, view_cap_tokens, n_sel, scale, k_scale, v_scale,
                                       out, lse, workspace, (cudaStream_t)stream, sel_ids, sel_stride, session_first);
     if (e != cudaSuccess) return cuda_fail("fused FP8 materialize+attend kernel launch", e);
     return KVMEM_OK;

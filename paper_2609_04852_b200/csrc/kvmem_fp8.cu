@@ -24,19 +24,23 @@ namespace kvmem {
 constexpr int kF8Tile = 64;                      // tokens per tile == block_tokens on this path
 constexpr int kF8D = 128;
 
+// UNIT: the scale is 1 and the multiplication by its inverse is left out (x * 1 is x: the same codes)
+template <bool UNIT = false>
 __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d, float inv) {
-    const __nv_fp8x2_storage_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(a, inv), __fmul_rn(b, inv)), __NV_SATFINITE, __NV_E4M3);
-    const __nv_fp8x2_storage_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(c, inv), __fmul_rn(d, inv)), __NV_SATFINITE, __NV_E4M3);
+    if (!UNIT) { a = __fmul_rn(a, inv); b = __fmul_rn(b, inv); c = __fmul_rn(c, inv); d = __fmul_rn(d, inv); }
+    const __nv_fp8x2_storage_t lo = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
+    const __nv_fp8x2_storage_t hi = __nv_cvt_float2_to_fp8x2(make_float2(c, d), __NV_SATFINITE, __NV_E4M3);
     return (uint32_t)lo | ((uint32_t)hi << 16);
 }
 
 // 8 bf16 (one 128-bit load) -> 8 E4M3 bytes
+template <bool UNIT = false>
 __device__ __forceinline__ uint2 quant8(const uint4& v, float inv) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     float f[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
-    return make_uint2(quant4(f[0], f[1], f[2], f[3], inv), quant4(f[4], f[5], f[6], f[7], inv));
+    return make_uint2(quant4<UNIT>(f[0], f[1], f[2], f[3], inv), quant4<UNIT>(f[4], f[5], f[6], f[7], inv));
 }
 
 struct GatherF8Args {
@@ -312,8 +316,66 @@ constexpr int kF8QrotPitch = kF8D * 2 + 32;      // bytes per rotated query row 
 constexpr int kF8QrotBytes = kF8RowsPad * kF8QrotPitch;
 constexpr size_t kF8SmemQrot = kF8Smem + (size_t)kF8Stages * kF8QrotBytes;
 constexpr int kF8QrotWarps = 3;                  // query-rotator warps; they take tiles in turn (12 warps in all: the register budget of 9)
+constexpr int kF8QuantWarps = 4;                 // MODE 4: warps that turn a landed bf16 tile into the FP8 tiles of the view
+constexpr int kF8BfStages = 5;                   // MODE 4: ring of bf16 tiles (K lo, K hi, V lo, V hi halves of 8 KiB) in front of
+constexpr int kF8QuantStages = 4;                //         a shorter FP8 ring: what is in flight from HBM is the bf16 tiles
+constexpr int kF8BfStageBytes = 4 * kF8Tile * 128;
+constexpr size_t kF8SmemQuant = (size_t)kF8QuantStages * kF8StageBytes + (size_t)kF8BfStages * kF8BfStageBytes + 1024;
+static_assert(kF8QuantStages % kF8Groups == 0, "each group must own whole stages");
 static_assert((size_t)kF8Consumers * kF8RowsPad * kF8MergeStride * sizeof(float) <= (size_t)kF8Stages * kF8StageBytes,
               "the ring is reused for the merge of the consumer warps");
+
+// One quantiser warp's share of a landed bf16 tile (MODE 4 of the attention kernel below): srcK / srcV are the tile's K and V
+// halves in the bf16 ring, dstK / dstV the FP8 tiles of the view in the FP8 ring.
+template <bool UNIT>
+__device__ __forceinline__ void quantise_tile_share(const unsigned char* srcK, const unsigned char* srcV, unsigned char* dstK,
+                                                    unsigned char* dstV, int qw, int lane, float k_inv, float v_inv) {
+    // Both tiles carry the 128-byte swizzle of their TMA maps: the 16-byte chunk c of row r sits at chunk c ^ (r & 7).
+    // K: a lane takes chunk c = lane & 7 (8 dims) of half h = (lane >> 3) & 1 of one token per step; half a warp reads
+    // and writes one token's row, conflict-free.
+    {
+        const int c = lane & 7, h = (lane >> 3) & 1;
+#pragma unroll 4
+        for (int i = 0; i < kF8Tile / (2 * kF8QuantWarps); ++i) {
+            const int t = i * 2 * kF8QuantWarps + qw * 2 + (lane >> 4);
+            const uint4 u = *reinterpret_cast<const uint4*>(srcK + h * kF8TileBytes + t * 128 + ((c ^ (t & 7)) << 4));
+            const int cc = 4 * h + (c >> 1);                                 // dims 64 h + 8 c .. are bytes 64 h + 8 c .. of the row
+            *reinterpret_cast<uint2*>(dstK + t * 128 + ((cc ^ (t & 7)) << 4) + 8 * (c & 1)) = quant8<UNIT>(u, k_inv);
+        }
+    }
+    // V: a lane takes 8 dims (chunk c of half h) of 8 consecutive tokens (group tg) and leaves, for each of the 8 dims, the
+    // 8 bytes of its tokens in the transposed tile: row = dim / 2, bytes (dim & 1) * 64 + token.  The items are dealt so
+    // that both sides of the transposition are conflict-free: a quarter-warp reads eight different chunks (one 128-bit
+    // load each), and the sixteen 64-bit stores of half a warp fall on sixteen different bank pairs (the chunk a store
+    // lands in depends on tg and on the parity of c only).
+    {
+        static_assert(kF8QuantWarps == 4, "the item assignment below is for four quantiser warps: 16 chunks x 8 token groups = 128 lanes");
+        const int c = lane & 7, u = (lane >> 3) & 1, h = lane >> 4, tg = ((c >> 1) + 4 * u + qw) & 7;
+        uint4 v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int t = tg * 8 + k;
+            v[k] = *reinterpret_cast<const uint4*>(srcV + h * kF8TileBytes + t * 128 + ((c ^ (t & 7)) << 4));
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int dim = 64 * h + 8 * c + e, vr = dim >> 1, col = (dim & 1) * 64 + tg * 8;
+            uint32_t w[2];
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) {
+                float fv[4];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const uint4& x = v[4 * kk + b];
+                    const uint32_t word = (e >> 1) == 0 ? x.x : (e >> 1) == 1 ? x.y : (e >> 1) == 2 ? x.z : x.w;
+                    fv[b] = (e & 1) ? __uint_as_float(word & 0xffff0000u) : __uint_as_float(word << 16);
+                }
+                w[kk] = quant4<UNIT>(fv[0], fv[1], fv[2], fv[3], v_inv);
+            }
+            *reinterpret_cast<uint2*>(dstV + vr * 128 + ((((col >> 4) ^ (vr & 7)) << 4) | (col & 15))) = make_uint2(w[0], w[1]);
+        }
+    }
+}
 
 struct AttendF8Args {
     const __nv_bfloat16* q;
@@ -330,6 +392,7 @@ struct AttendF8Args {
     const int32_t* nblocks_dev;  // [max_sessions]
     int session_first, sel_stride, max_bps, max_blocks;
     int lookahead;               // MODE 2: tiles the producer may have in flight that have not landed (0: every stage)
+    float k_inv_scale, v_inv_scale;      // MODE 4: what the bf16 keys and values are multiplied by before their conversion to E4M3
     // MODE 3: the pages hold the codes of RoPE(k, offset in block); the query is rotated back per tile
     const float2* rope;          // [rope_positions][64] (cos, sin)
     int first_position, rope_positions;
@@ -344,14 +407,21 @@ struct AttendF8Args {
 //         tiles alternately, rotate the 16 query rows back by the tile's compact position p0 (q . R(p0 + t) k = (R(-p0) q) .
 //         RoPE(k, t)), round them to bf16 as the definition says, widen them to f16 and leave them in a small ring of
 //         shared memory from which the consumers fetch their A fragments; no key is touched.
+// MODE 4: MODE 2 over a bf16 repository (kvmem_materialize_fp8 + kvmem_view_attend_fp8 in one pass, 2 bytes read + 1 byte
+//         written per element): the producer brings bf16 tiles (map_pages: [pages * 2 * L*G * 64 rows][128 bf16], 64-dim
+//         halves) into a ring of their own; two quantiser warps turn each landed tile into the view's FP8 tiles (K straight,
+//         V transposed; arithmetic of the quantising gather) in the FP8 ring, from where the consumers attend over it and
+//         the view writer stores it, exactly as in MODE 2.
 template <int MODE>
-__global__ void __launch_bounds__(kF8Threads + (MODE == 2 ? 32 : MODE == 3 ? 32 * kF8QrotWarps : 0), 1)
+__global__ void __launch_bounds__(kF8Threads + (MODE == 2 ? 32 : MODE == 3 ? 32 * kF8QrotWarps : MODE == 4 ? 32 + 32 * kF8QuantWarps : 0), 1)
 attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                         const __grid_constant__ CUtensorMap map_pages, AttendF8Args a) {
-    constexpr bool PAGED = MODE != 0, FUSED = MODE == 2, QROT = MODE == 3;
+    constexpr bool PAGED = MODE != 0, QUANT = MODE == 4, FUSED = MODE == 2 || QUANT, QROT = MODE == 3;
     pdl_wait();
     extern __shared__ unsigned char smem_dyn[];
+    constexpr int NST = QUANT ? kF8QuantStages : kF8Stages;      // stages of the FP8 ring
     __shared__ uint64_t full_bar[kF8Stages], empty_bar[kF8Stages], q_full[kF8Stages];
+    __shared__ uint64_t bf_full[kF8BfStages], bf_empty[kF8BfStages];       // MODE 4: the ring of bf16 tiles
     __shared__ float merge_m[kF8Consumers][kF8RowsPad], merge_l[kF8Consumers][kF8RowsPad];
 
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -361,14 +431,16 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int z = s * LG + lg;
     const int l = lg / a.G, g = lg % a.G;
 
-    const int n_blk = max(0, min(a.n_sel[s], (MODE == 1 || MODE == 3) ? a.sel_stride : MODE == 2 ? min(a.sel_stride, a.cap_tokens / kF8Tile) : a.cap_tokens / kF8Tile));
+    const int n_blk = max(0, min(a.n_sel[s], (MODE == 1 || MODE == 3) ? a.sel_stride : FUSED ? min(a.sel_stride, a.cap_tokens / kF8Tile) : a.cap_tokens / kF8Tile));
     const int t0 = (int)((long long)n_blk * split / a.n_splits);
     const int t1 = (int)((long long)n_blk * (split + 1) / a.n_splits);
     const int n_tiles = t1 - t0;
     const int cap_tiles = a.cap_tokens / kF8Tile;
 
     if (tid == 0) {
-        for (int i = 0; i < kF8Stages; ++i) { ptx::mbar_init(&full_bar[i], 1); ptx::mbar_init(&empty_bar[i], kF8Consumers / kF8Groups + (FUSED ? 1 : 0)); ptx::mbar_init(&q_full[i], 1); }
+        // MODE 4: a stage of the FP8 ring is full when both quantiser warps have written their share of it
+        for (int i = 0; i < NST; ++i) { ptx::mbar_init(&full_bar[i], QUANT ? kF8QuantWarps : 1); ptx::mbar_init(&empty_bar[i], kF8Consumers / kF8Groups + (FUSED ? 1 : 0)); ptx::mbar_init(&q_full[i], 1); }
+        for (int i = 0; i < kF8BfStages; ++i) { ptx::mbar_init(&bf_full[i], 1); ptx::mbar_init(&bf_empty[i], kF8QuantWarps); }
         ptx::fence_mbar_init();
     }
     __syncthreads();
@@ -383,7 +455,7 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         if (n_tiles > 0) {
             if (lane == 0) ptx::prefetch_tensormap(&map_pages);
             const int NB = a.nblocks_dev[a.session_first + s];
-            const int ahead = FUSED && a.lookahead > 0 ? min(a.lookahead, kF8Stages) : kF8Stages;
+            const int ahead = MODE == 2 && a.lookahead > 0 ? min(a.lookahead, NST) : NST;
             auto lookup = [&](int it) -> int {
                 if (it >= n_tiles) return 0;
                 const int id = a.sel_ids[(size_t)s * a.sel_stride + t0 + it];
@@ -397,13 +469,29 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             for (int it = 0; it < n_tiles; ++it) {
                 if (it >= base_it + 32) { base_it = it; my_page = lookup(base_it + lane); }
                 const int page = __shfl_sync(0xffffffffu, my_page, it - base_it);
-                if (lane == 0) {
-                    const int st = it % kF8Stages;
-                    if (ahead < kF8Stages && it >= ahead) {       // at most `ahead` tiles that have not landed yet
-                        const int jt = it - ahead;
-                        ok = ptx::mbar_wait(&full_bar[jt % kF8Stages], (uint32_t)((jt / kF8Stages) & 1));
+                if (QUANT) {
+                    if (lane == 0) {
+                        // bf16 tile into its own ring; the ring's depth bounds the tiles in flight
+                        const int sb = it % kF8BfStages;
+                        if (it >= kF8BfStages) ok = ptx::mbar_wait(&bf_empty[sb], (uint32_t)(((it / kF8BfStages) & 1) ^ 1));
+                        if (ok) {
+                            unsigned char* dst = stages + (size_t)NST * kF8StageBytes + (size_t)sb * kF8BfStageBytes;
+                            // page layout [K|V][L*G][64 tokens][128 bf16]: rows of 256 B, fetched as two 64-dim halves
+                            const int yk = ((page * 2 + 0) * LG + lg) * kF8Tile, yv = ((page * 2 + 1) * LG + lg) * kF8Tile;
+                            ptx::mbar_expect_tx(&bf_full[sb], kF8BfStageBytes);
+                            ptx::tma_load_2d(dst, &map_pages, 0, yk, &bf_full[sb]);
+                            ptx::tma_load_2d(dst + kF8TileBytes, &map_pages, 64, yk, &bf_full[sb]);
+                            ptx::tma_load_2d(dst + 2 * kF8TileBytes, &map_pages, 0, yv, &bf_full[sb]);
+                            ptx::tma_load_2d(dst + 3 * kF8TileBytes, &map_pages, 64, yv, &bf_full[sb]);
+                        }
                     }
-                    if (ok && it >= kF8Stages) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kF8Stages) & 1) ^ 1));
+                } else if (lane == 0) {
+                    const int st = it % NST;
+                    if (ahead < NST && it >= ahead) {       // at most `ahead` tiles that have not landed yet
+                        const int jt = it - ahead;
+                        ok = ptx::mbar_wait(&full_bar[jt % NST], (uint32_t)((jt / NST) & 1));
+                    }
+                    if (ok && it >= NST) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / NST) & 1) ^ 1));
                     if (ok) {
                         unsigned char* dst = stages + (size_t)st * kF8StageBytes;
                         // page layout [K|V][L*G][64 rows][128 bytes]
@@ -432,7 +520,7 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                     raw_hi[i] = *reinterpret_cast<const uint4*>(qr + kF8D / 2 + c * 8);
                 }
             }
-            unsigned char* qring = stages + (size_t)kF8Stages * kF8StageBytes;
+            unsigned char* qring = stages + (size_t)NST * kF8StageBytes;
             auto fetch_row = [&](int it, float4 (&t4)[4]) {
                 int p0 = a.first_position + (t0 + min(it, n_tiles - 1)) * kF8Tile;
                 if (p0 < 0 || p0 >= a.rope_positions) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_DEVICE_RANGE); p0 = 0; }
@@ -451,12 +539,12 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             float4 t4[4], t4_next[4];
             fetch_row(it_first, t4_next);
             for (int it = it_first; it < n_tiles; it += kF8QrotWarps) {
-                const int st = it % kF8Stages;
+                const int st = it % NST;
 #pragma unroll
                 for (int w = 0; w < 4; ++w) t4[w] = t4_next[w];
                 fetch_row(it + kF8QrotWarps, t4_next);
                 bool ok = true;
-                if (it >= kF8Stages) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kF8Stages) & 1) ^ 1));
+                if (it >= NST) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / NST) & 1) ^ 1));
                 if (!__all_sync(0xffffffffu, ok)) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
                 unsigned char* qb = qring + (size_t)st * kF8QrotBytes;
 #pragma unroll
@@ -471,6 +559,27 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 if (lane == 0) ptx::mbar_arrive(&q_full[st]);
             }
         }
+    } else if (QUANT && warp > kF8Consumers + 1) {
+        // ---------------- quantisers: landed bf16 tile -> the view's FP8 tiles (K [token][128 B], V^T [dim / 2][128 B]) ----------------
+        const int qw = warp - kF8Consumers - 2;
+        for (int it = 0; it < n_tiles; ++it) {
+            const int sb = it % kF8BfStages, st = it % NST;
+            bool ok = ptx::mbar_wait(&bf_full[sb], (uint32_t)((it / kF8BfStages) & 1));
+            if (ok && it >= NST) ok = ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / NST) & 1) ^ 1));
+            if (!__all_sync(0xffffffffu, ok)) { if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT); break; }
+            const unsigned char* srcK = stages + (size_t)NST * kF8StageBytes + (size_t)sb * kF8BfStageBytes;
+            const unsigned char* srcV = srcK + 2 * kF8TileBytes;
+            unsigned char* dstK = stages + (size_t)st * kF8StageBytes;
+            unsigned char* dstV = dstK + kF8TileBytes;
+            if (a.k_inv_scale == 1.0f && a.v_inv_scale == 1.0f) quantise_tile_share<true>(srcK, srcV, dstK, dstV, qw, lane, 1.0f, 1.0f);
+            else quantise_tile_share<false>(srcK, srcV, dstK, dstV, qw, lane, a.k_inv_scale, a.v_inv_scale);
+            ptx::fence_proxy_async_smem();      // the view writer's bulk stores read these bytes through the async proxy
+            __syncwarp();
+            if (lane == 0) {
+                ptx::mbar_arrive(&full_bar[st]);
+                ptx::mbar_arrive(&bf_empty[sb]);
+            }
+        }
     } else if (FUSED && warp == kF8Consumers + 1) {
         // ---------------- view writer: every tile that lands in shared memory is stored to the FP8 view ----------------
         if (lane == 0 && n_tiles > 0) {
@@ -478,8 +587,8 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             ptx::prefetch_tensormap(&map_v);
             bool ok = true;
             for (int it = 0; it < n_tiles; ++it) {
-                const int st = it % kF8Stages;
-                ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kF8Stages) & 1));
+                const int st = it % NST;
+                ok = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / NST) & 1));
                 if (!ok) break;
                 unsigned char* src = stages + (size_t)st * kF8StageBytes;
                 const int y = (z * cap_tiles + t0 + it) * kF8Tile;
@@ -488,11 +597,11 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 ptx::bulk_commit();
                 if (it > 0) {                              // all but the newest store have left shared memory
                     ptx::bulk_wait_read<1>();
-                    ptx::mbar_arrive(&empty_bar[(it - 1) % kF8Stages]);
+                    ptx::mbar_arrive(&empty_bar[(it - 1) % NST]);
                 }
             }
             ptx::bulk_wait_read<0>();
-            if (ok) ptx::mbar_arrive(&empty_bar[(n_tiles - 1) % kF8Stages]);
+            if (ok) ptx::mbar_arrive(&empty_bar[(n_tiles - 1) % NST]);
             else atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
             ptx::bulk_wait<0>();                           // the view is complete before the kernel ends
         }
@@ -502,8 +611,8 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             ptx::prefetch_tensormap(&map_k);
             ptx::prefetch_tensormap(&map_v);
             for (int it = 0; it < n_tiles; ++it) {
-                const int st = it % kF8Stages;
-                if (it >= kF8Stages && !ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / kF8Stages) & 1) ^ 1))) {
+                const int st = it % NST;
+                if (it >= NST && !ptx::mbar_wait(&empty_bar[st], (uint32_t)(((it / NST) & 1) ^ 1))) {
                     atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                     break;
                 }
@@ -545,9 +654,9 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         const int grp = warp >> 2, wq = warp & 3;       // group grp takes tiles grp, grp + 2, ...; warp wq tokens [16 wq, 16 wq + 16)
 
         for (int it = grp; it < n_tiles; it += kF8Groups) {
-            const int st = it % kF8Stages;
-            bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / kF8Stages) & 1));
-            if (QROT) arrived = arrived && ptx::mbar_wait(&q_full[st], (uint32_t)((it / kF8Stages) & 1));
+            const int st = it % NST;
+            bool arrived = ptx::mbar_wait(&full_bar[st], (uint32_t)((it / NST) & 1));
+            if (QROT) arrived = arrived && ptx::mbar_wait(&q_full[st], (uint32_t)((it / NST) & 1));
             if (!__all_sync(0xffffffffu, arrived)) {
                 if (lane == 0) atomicExch(a.status, (int)KVMEM_E_TIMEOUT);
                 break;
@@ -556,7 +665,7 @@ attend_fp8_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             const uint32_t vbase = kbase + kF8TileBytes;
             if (QROT) {
                 // this tile's rotated query: four consecutive dims (two f16x2 words) per k-step for rows lane / 4 and + 8
-                const unsigned char* qb = stages + (size_t)kF8Stages * kF8StageBytes + (size_t)st * kF8QrotBytes;
+                const unsigned char* qb = stages + (size_t)NST * kF8StageBytes + (size_t)st * kF8QrotBytes;
                 const unsigned char* pa = qb + (lane >> 2) * kF8QrotPitch + 8 * (lane & 3);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -707,6 +816,19 @@ static bool make_f8_map(CUtensorMap* map, const uint8_t* base, long long rows) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 page pool as [rows][128 bf16]; box = one 64-dim half (128 bytes) x 64 rows, 128-byte swizzle
+static bool make_bf16_pages_map(CUtensorMap* map, const __nv_bfloat16* base, long long rows) {
+    PFN_cuTensorMapEncodeTiled_v12000 enc = f8_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)kF8D, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)kF8D * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kF8Tile};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 cudaError_t launch_gather_fp8(const kvmem_pool& p, int session_first, int n_sessions, const int32_t* sel_ids, int sel_stride,
                               const int32_t* n_sel, uint8_t* view_k, uint8_t* view_v, int view_cap_tokens, float k_scale,
                               float v_scale, cudaStream_t st, int rope_first_position) {
@@ -750,8 +872,11 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
     const int LG = g.L * g.G, heads = n_sessions * LG;
     const bool paged = sel_ids != nullptr;                  // straight over the pages of an FP8 repository ...
     const bool fused = paged && view_k != nullptr;          // ... and, with view buffers, storing the view on the way
+    const bool quant = fused && !p.cfg.fp8_pages;           // bf16 repository: tiles are quantised on their way through
     CUtensorMap map_k, map_v, map_pages;
-    if (paged && !make_f8_map(&map_pages, reinterpret_cast<const uint8_t*>(p.pages), (long long)g.max_blocks * 2 * LG * kF8Tile))
+    if (quant) {
+        if (!make_bf16_pages_map(&map_pages, p.pages, (long long)g.max_blocks * 2 * LG * kF8Tile)) return cudaErrorInvalidValue;
+    } else if (paged && !make_f8_map(&map_pages, reinterpret_cast<const uint8_t*>(p.pages), (long long)g.max_blocks * 2 * LG * kF8Tile))
         return cudaErrorInvalidValue;
     if (paged && !fused) {
         map_k = map_pages; map_v = map_pages;               // unused by this mode
@@ -765,6 +890,7 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8Smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8SmemQrot);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attend_fp8_split_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF8SmemQuant);
         if (e != cudaSuccess) return e;
         attr_done.mark(p.cfg.device);
     }
@@ -780,6 +906,7 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
     const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
     a.scale_log2e = sc * k_scale * 1.4426950408889634f;
     a.v_scale = v_scale;
+    a.k_inv_scale = 1.0f / k_scale; a.v_inv_scale = 1.0f / v_scale;
     a.sel_ids = sel_ids; a.tables = p.tables; a.nblocks_dev = p.nblocks_dev;
     a.session_first = session_first; a.sel_stride = sel_stride; a.max_bps = g.max_bps; a.max_blocks = g.max_blocks;
     dim3 grid((unsigned)a.n_splits, (unsigned)LG, (unsigned)n_sessions);
@@ -794,6 +921,8 @@ cudaError_t launch_attend_fp8(const kvmem_pool& p, int n_sessions, const __nv_bf
     a.rope = p.rope_dev; a.first_position = rope_first_position; a.rope_positions = p.cfg.rope_max_positions;
     if (paged && !fused && rope_first_position >= 0)
         launch_pdl(attend_fp8_split_kernel<3>, dim3(grid), dim3(kF8Threads + 32 * kF8QrotWarps), kF8SmemQrot, st, map_k, map_v, map_pages, a);
+    else if (quant)
+        launch_pdl(attend_fp8_split_kernel<4>, dim3(grid), dim3(kF8Threads + 32 + 32 * kF8QuantWarps), kF8SmemQuant, st, map_k, map_v, map_pages, a);
     else if (fused)
         launch_pdl(attend_fp8_split_kernel<2>, dim3(grid), dim3(kF8Threads + 32), kF8Smem, st, map_k, map_v, map_pages, a);
     else if (paged)

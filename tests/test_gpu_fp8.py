@@ -93,6 +93,61 @@ def test_fp8_empty_view_and_argument_errors():
     assert pool.device_status() == 0
 
 
+# ---- one pass over a bf16 repository: tiles quantised on the way to the view and to the tensor cores ----
+
+@pytest.mark.parametrize("n_blocks,k,cap_blocks,M,k_scale,v_scale", [(150, 20, 20, 4, 1.0, 1.0), (700, 333, 340, 4, 0.5, 0.25),
+                                                                    (90, 1, 1, 1, 2.0, 1.0), (64, 64, 64, 2, 1.0, 0.0625),
+                                                                    (300, 7, 7, 3, 1.0, 1.0)])
+def test_fp8_view_written_while_attended_over_bf16_pages(n_blocks, k, cap_blocks, M, k_scale, v_scale):
+    """kvmem_materialize_attend_fp8 on a bf16 repository: the view must hold the oracle's codes byte for byte, the results
+    must be the oracle's attention over those codes within tolerance, and both must equal the two separate calls bit
+    for bit; nothing outside the view and the outputs is written."""
+    from kvmem_harness import Guards
+    from kvmem_workloads import kv_blocks, page_table
+    from paper_2609_04852_b200 import Pool
+    spec = SPEC.with_(n_blocks=n_blocks, n_planted=min(8, n_blocks // 4), budget_blocks=k, n_q_tokens=M)
+    dev = torch.device("cuda", 0)
+    pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.block_tokens, 1, n_blocks, n_blocks, 0,
+                fp8_k_scale=k_scale, fp8_v_scale=v_scale)
+    table = page_table(spec)[0]
+    for b0 in range(0, n_blocks, 256):
+        b1 = min(n_blocks, b0 + 256)
+        K, V = kv_blocks(spec, 0, b0, b1, dev)
+        pool.append_blocks(0, K, V, table[b0:b1].tolist())
+    osess = fill_oracle(spec)[0]
+    ids = _ids(np.random.default_rng(n_blocks + k), n_blocks, k)
+    cap = cap_blocks * 64
+    sel = torch.full((1, cap_blocks), -1, dtype=torch.int32)
+    sel[0, :k] = torch.from_numpy(ids)
+    sel = sel.to(dev)
+    n_sel = torch.tensor([k], dtype=torch.int32, device=dev)
+    q, qb = queries(spec)
+    qd = q.to(dev)
+    g = Guards(dev)
+    k8 = g.empty((1, spec.n_layers, spec.n_kv_heads, cap, 128), torch.uint8)
+    v8t = g.empty((1, spec.n_layers, spec.n_kv_heads, cap_blocks, 128, 64), torch.uint8)
+    out, lse = g.outputs(pool, 1, M)
+    pool.materialize_attend_fp8(qd, sel, n_sel, k8, v8t, out, lse)
+    k8s, v8s = pool.new_view_fp8(1, cap)
+    out2, lse2 = pool.new_outputs(1, M)
+    pool.materialize_fp8(sel, n_sel, k8s, v8s, k_scale, v_scale)
+    pool.view_attend_fp8(qd, k8s, v8s, n_sel, out2, lse2, k_scale, v_scale)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    g.check()
+    k_inv, v_inv = np.float32(1.0) / np.float32(k_scale), np.float32(1.0) / np.float32(v_scale)
+    rK, rV = orc.gather_fp8(osess.repo, osess.table, ids, cap, float(k_inv), float(v_inv))
+    T = k * 64
+    assert np.array_equal(k8.cpu().numpy()[0][:, :, :T], rK[:, :, :T]), "FP8 key codes differ"
+    assert np.array_equal(v8t.cpu().numpy()[0][:, :, :k], rV[:, :, :k]), "FP8 value codes differ"
+    ref_out, ref_lse = orc.attend_fp8(qb[0], rK, rV, T, k_scale, v_scale)
+    err_o = np.abs(out.cpu().numpy()[0] - ref_out).max()
+    err_l = np.abs(lse.cpu().numpy()[0] - ref_lse).max()
+    assert err_o <= ATTN_ATOL * max(1.0, v_scale) and err_l <= ATTN_ATOL, (err_o, err_l)
+    assert torch.equal(k8[0, :, :, :T], k8s[0, :, :, :T]) and torch.equal(v8t[0, :, :, :k], v8s[0, :, :, :k])
+    assert torch.equal(out, out2) and torch.equal(lse, lse2), "one pass and separate calls must be the same bits"
+
+
 # ---- FP8 repository: the pages themselves hold the E4M3 tiles ---------------------------------------
 
 def _fp8_pool(spec, k_scale, v_scale):
@@ -177,8 +232,7 @@ def test_page_formats_are_not_mixed_up():
     out, lse = f8.new_outputs(1, spec.n_q_tokens)
     view = f8.new_view(1, 4 * 64)
     for call in (lambda: f8.materialize(sel, n_sel, view), lambda: f8.materialize_attend(qd, sel, n_sel, view, out, lse),
-                 lambda: f8.paged_attend(qd, sel, n_sel, out, lse), lambda: bf.paged_attend_fp8(qd, sel, n_sel, out, lse),
-                 lambda: bf.materialize_attend_fp8(qd, sel, n_sel, *bf.new_view_fp8(1, 4 * 64), out, lse)):
+                 lambda: f8.paged_attend(qd, sel, n_sel, out, lse), lambda: bf.paged_attend_fp8(qd, sel, n_sel, out, lse)):
         with pytest.raises(KvmemError) as e:
             call()
         assert e.value.status == E_STATE
