@@ -148,6 +148,42 @@ def test_fp8_view_written_while_attended_over_bf16_pages(n_blocks, k, cap_blocks
     assert torch.equal(out, out2) and torch.equal(lse, lse2), "one pass and separate calls must be the same bits"
 
 
+def test_fp8_one_pass_over_bf16_pages_with_two_sessions_of_different_lengths():
+    """Sessions are independent: each gets its own selection length (one of them shorter than the row, one empty in a
+    second call) and its own slice of the view; what lies beyond a session's selection is not written."""
+    spec = SPEC.with_(name="fp8two", n_sessions=2, n_blocks=96, n_planted=4, n_q_tokens=2)
+    dev = torch.device("cuda", 0)
+    pool = fill_pool(spec)
+    osess = fill_oracle(spec)
+    M, cap_blocks = 2, 24
+    cap = cap_blocks * 64
+    rng = np.random.default_rng(5)
+    for ks in ((24, 7), (0, 13)):
+        ids = [_ids(rng, spec.n_blocks, k) for k in ks]
+        sel = torch.full((2, cap_blocks), -1, dtype=torch.int32)
+        for s_, idv in enumerate(ids):
+            sel[s_, :len(idv)] = torch.from_numpy(idv)
+        sel = sel.to(dev)
+        n_sel = torch.tensor(list(ks), dtype=torch.int32, device=dev)
+        q, qb = queries(spec)
+        k8, v8t = pool.new_view_fp8(2, cap)
+        k8.fill_(0x5A); v8t.fill_(0x5A)
+        out, lse = pool.new_outputs(2, M)
+        pool.materialize_attend_fp8(q.to(dev), sel, n_sel, k8, v8t, out, lse)
+        torch.cuda.synchronize()
+        assert pool.device_status() == 0
+        for s_, k in enumerate(ks):
+            rK, rV = orc.gather_fp8(osess[s_].repo, osess[s_].table, ids[s_], cap, 1.0, 1.0)
+            T = k * 64
+            assert np.array_equal(k8.cpu().numpy()[s_][:, :, :T], rK[:, :, :T]) and np.array_equal(v8t.cpu().numpy()[s_][:, :, :k], rV[:, :, :k])
+            assert bool((k8[s_][:, :, T:] == 0x5A).all()) and bool((v8t[s_][:, :, k:] == 0x5A).all()), "wrote past the selection"
+            if k == 0:
+                assert bool((out[s_] == 0).all()) and bool(torch.isinf(lse[s_]).all())
+                continue
+            ref_out, ref_lse = orc.attend_fp8(qb[s_], rK, rV, T, 1.0, 1.0)
+            assert np.abs(out.cpu().numpy()[s_] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[s_] - ref_lse).max() <= ATTN_ATOL
+
+
 # ---- FP8 repository: the pages themselves hold the E4M3 tiles ---------------------------------------
 
 def _fp8_pool(spec, k_scale, v_scale):
