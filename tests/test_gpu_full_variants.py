@@ -136,6 +136,35 @@ def test_1m_fp8_repository_passes():
     assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
 
 
+def test_1m_fp8_view_written_while_attended_over_bf16_pages():
+    """kvmem_materialize_attend_fp8 on the bf16 repository at full size, in the launch configuration bench.py --fp8 times:
+    codes byte for byte against the oracle's quantising gather, results within tolerance of the oracle's FP8 attention and
+    equal to the two separate calls bit for bit."""
+    spec = SPEC
+    dev = torch.device("cuda", 0)
+    B = spec.block_tokens
+    pool = fill_pool(spec)
+    q, qb = queries(spec)
+    qd = q.to(dev)
+    osess = fill_oracle(spec, gen_device=dev)[0]
+    sel, n_sel, ids, k = _oracle_selection(spec, osess, qb, dev)
+    M, T = spec.n_q_tokens, k * B
+    k8, v8t = pool.new_view_fp8(1, T)
+    out, lse = pool.new_outputs(1, M)
+    pool.materialize_attend_fp8(qd, sel, n_sel, k8, v8t, out, lse)
+    k8s, v8s = pool.new_view_fp8(1, T)
+    out2, lse2 = pool.new_outputs(1, M)
+    pool.materialize_fp8(sel, n_sel, k8s, v8s)
+    pool.view_attend_fp8(qd, k8s, v8s, n_sel, out2, lse2)
+    torch.cuda.synchronize()
+    assert pool.device_status() == 0
+    assert torch.equal(k8, k8s) and torch.equal(v8t, v8s) and torch.equal(out, out2) and torch.equal(lse, lse2)
+    rK, rV = orc.gather_fp8(osess.repo, osess.table, np.ascontiguousarray(ids), T, 1.0, 1.0)
+    assert np.array_equal(k8.cpu().numpy()[0], rK) and np.array_equal(v8t.cpu().numpy()[0], rV)
+    ref_out, ref_lse = orc.attend_fp8(qb[0], rK, rV, T, 1.0, 1.0)
+    assert np.abs(out.cpu().numpy()[0] - ref_out).max() <= ATTN_ATOL and np.abs(lse.cpu().numpy()[0] - ref_lse).max() <= ATTN_ATOL
+
+
 def test_1m_position_consistent_passes_on_raw_keys():
     """Raw keys in the pages (the paper's layout, Sec. 4.3/4.4): the rotating gather against the oracle at full size,
     attention over it, and the copy-free pass that rotates key fragments in registers, which must give the same bits."""
