@@ -95,17 +95,17 @@ def test_fp8_empty_view_and_argument_errors():
 
 # ---- one pass over a bf16 repository: tiles quantised on the way to the view and to the tensor cores ----
 
-@pytest.mark.parametrize("n_blocks,k,cap_blocks,M,k_scale,v_scale", [(150, 20, 20, 4, 1.0, 1.0), (700, 333, 340, 4, 0.5, 0.25),
-                                                                    (90, 1, 1, 1, 2.0, 1.0), (64, 64, 64, 2, 1.0, 0.0625),
-                                                                    (300, 7, 7, 3, 1.0, 1.0)])
-def test_fp8_view_written_while_attended_over_bf16_pages(n_blocks, k, cap_blocks, M, k_scale, v_scale):
+@pytest.mark.parametrize("n_blocks,k,cap_blocks,M,k_scale,v_scale,L", [(150, 20, 20, 4, 1.0, 1.0, 1), (700, 333, 340, 4, 0.5, 0.25, 1),
+                                                                      (90, 1, 1, 1, 2.0, 1.0, 1), (64, 64, 64, 2, 1.0, 0.0625, 1),
+                                                                      (300, 7, 7, 3, 1.0, 1.0, 1), (120, 37, 40, 2, 1.0, 0.5, 2)])
+def test_fp8_view_written_while_attended_over_bf16_pages(n_blocks, k, cap_blocks, M, k_scale, v_scale, L):
     """kvmem_materialize_attend_fp8 on a bf16 repository: the view must hold the oracle's codes byte for byte, the results
     must be the oracle's attention over those codes within tolerance, and both must equal the two separate calls bit
     for bit; nothing outside the view and the outputs is written."""
     from kvmem_harness import Guards
     from kvmem_workloads import kv_blocks, page_table
     from paper_2609_04852_b200 import Pool
-    spec = SPEC.with_(n_blocks=n_blocks, n_planted=min(8, n_blocks // 4), budget_blocks=k, n_q_tokens=M)
+    spec = SPEC.with_(n_blocks=n_blocks, n_planted=min(8, n_blocks // 4), budget_blocks=k, n_q_tokens=M, n_layers=L)
     dev = torch.device("cuda", 0)
     pool = Pool(spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.block_tokens, 1, n_blocks, n_blocks, 0,
                 fp8_k_scale=k_scale, fp8_v_scale=v_scale)

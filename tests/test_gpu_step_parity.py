@@ -380,16 +380,17 @@ def test_thirty_two_rows_at_32_token_blocks_and_two_sessions():
 
 # ------------------------------------------------------------------ raw keys rotated inside the fused pass
 
-@pytest.mark.parametrize("B,n_blocks,budget,M,first", [(64, 150, 20, 4, 517), (64, 700, 60, 4, 17), (64, 90, 1, 1, 0), (64, 64, 63, 2, 64),
-                                                      (32, 200, 21, 4, 131), (16, 300, 37, 2, 0), (128, 40, 9, 4, 64)])
-def test_position_consistent_view_and_attention_in_one_pass_over_raw_keys(B, n_blocks, budget, M, first):
+@pytest.mark.parametrize("B,n_blocks,budget,M,first,L", [(64, 150, 20, 4, 517, 1), (64, 700, 60, 4, 17, 1), (64, 90, 1, 1, 0, 1), (64, 64, 63, 2, 64, 1),
+                                                        (32, 200, 21, 4, 131, 1), (16, 300, 37, 2, 0, 1), (128, 40, 9, 4, 64, 1),
+                                                        (64, 120, 33, 3, 200, 2), (32, 90, 50, 4, 7, 2)])
+def test_position_consistent_view_and_attention_in_one_pass_over_raw_keys(B, n_blocks, budget, M, first, L):
     """kvmem_materialize_attend_rope on a pool of raw keys: the warps that attend over a tile rotate its keys to their
     compact positions (angles composed from the table rows of the warp's first position and of the offset inside its
     share) and hand them back for the store.  Values are copied bit for bit; a rotated key may differ from the defined code
     (oracle gather with RoPE) by one bf16 rounding step on a small fraction of the elements; the results are those of
     attention over the defined view within the attention tolerance, and they are the copy-free pass's bit for bit."""
     from test_gpu_rope import SPEC as RSPEC, _fill_both
-    spec = RSPEC.with_(name=f"rawfusedB{B}", block_tokens=B, n_blocks=n_blocks, budget_blocks=budget, n_q_tokens=M)
+    spec = RSPEC.with_(name=f"rawfusedB{B}L{L}", block_tokens=B, n_blocks=n_blocks, budget_blocks=budget, n_q_tokens=M, n_layers=L)
     dev = torch.device("cuda", 0)
     pool, repo, idx, tab, table = _fill_both(spec)
     ids = np.sort(np.random.default_rng(3 * n_blocks + B).choice(n_blocks, size=budget, replace=False)).astype(np.int32)
