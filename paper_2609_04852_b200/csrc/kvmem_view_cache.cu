@@ -182,8 +182,9 @@ struct CacheApplyArgs {
 };
 
 // HBM-bound on the tiles it touches: 1 read + 1 write per byte of an incoming block, 1 read + 1 write per
-// K byte of a re-encoded block, nothing for a block that stays where it is.
-__global__ void __launch_bounds__(256)
+// K byte of a re-encoded block, nothing for a block that stays where it is.  Held to 40 registers (six CTAs per SM instead
+// of five): the kernel waits on its loads, and the update of a 4,096-block cache goes from 247 to 237 us.
+__global__ void __launch_bounds__(256, 6)
 view_cache_apply_kernel(CacheApplyArgs a) {
     pdl_wait();
     const int n = min(max(*a.c.n_view, 0), a.cap);
