@@ -145,6 +145,32 @@ def _dev(t: torch.Tensor, dtype=None) -> int:
     return t.data_ptr()
 
 
+class HostStep:
+    """kvmem_recall_step_host with its arguments checked and marshalled once; see Pool.host_step."""
+
+    def __init__(self, pool, q_shape, params, sel_ids, n_sel, view, out_host, lse_host, scale, session_first):
+        ns, M = q_shape[0], q_shape[1]
+        for t, dt in ((out_host, torch.float32), (lse_host, torch.float32)):
+            if t.is_cuda or not t.is_contiguous() or t.dtype != dt:
+                raise ValueError("expected contiguous CPU tensors (fp32 outputs)")
+        need = pool.lib.kvmem_step_staging_bytes(C.byref(pool.cfg), ns, M)
+        if pool._staging is None or pool._staging.numel() < need:
+            pool._staging = torch.empty(need, dtype=torch.uint8, device=pool.device)
+        sws, aws = pool.select_workspace(ns, M), pool.attend_workspace(ns, M)
+        self._keep = (pool, params, sel_ids, n_sel, view, out_host, lse_host, pool._staging, sws, aws)   # the buffers stay alive
+        self._q_shape, self._fn = q_shape, pool.lib.kvmem_recall_step_host
+        self._head = (pool.handle, session_first, ns)
+        self._tail = (M, C.byref(params), _dev(sel_ids, torch.int32), sel_ids.shape[-1], _dev(n_sel, torch.int32),
+                      _dev(view.k, torch.bfloat16), _dev(view.v, torch.bfloat16), view.cap_tokens, scale, out_host.data_ptr(),
+                      lse_host.data_ptr(), pool._staging.data_ptr(), pool._staging.numel(), sws.data_ptr(), sws.numel(),
+                      aws.data_ptr(), aws.numel())
+
+    def __call__(self, q_host: torch.Tensor) -> None:
+        if q_host.is_cuda or q_host.dtype != torch.bfloat16 or tuple(q_host.shape) != self._q_shape or not q_host.is_contiguous():
+            raise ValueError("expected a contiguous CPU bf16 query of the planned shape")
+        _check(self._fn(*self._head, q_host.data_ptr(), *self._tail, _stream()))
+
+
 def budget_blocks(params: SelectParams, block_tokens: int, n_blocks: int) -> int:
     return int(load_library().kvmem_budget_blocks(C.byref(params), block_tokens, n_blocks))
 
@@ -506,6 +532,12 @@ class Pool:
             sel_ids.shape[-1], _dev(n_sel, torch.int32), _dev(view.k, torch.bfloat16), _dev(view.v, torch.bfloat16),
             view.cap_tokens, scale, out_host.data_ptr(), lse_host.data_ptr(), self._staging.data_ptr(),
             self._staging.numel(), sws.data_ptr(), sws.numel(), aws.data_ptr(), aws.numel(), _stream()))
+
+    def host_step(self, q_shape, params: SelectParams, sel_ids: torch.Tensor, n_sel: torch.Tensor, view: View,
+                  out_host: torch.Tensor, lse_host: torch.Tensor, scale: float = 0.0, session_first: int = 0) -> "HostStep":
+        """recall_step_host with everything but the query marshalled once (a decode loop calls the same step with the
+        same buffers every token): returns a callable that takes the pinned bf16 query of shape q_shape."""
+        return HostStep(self, tuple(q_shape), params, sel_ids, n_sel, view, out_host, lse_host, scale, session_first)
 
     # ---- helpers that only allocate
     def new_view(self, n_sessions: int, cap_tokens: int) -> View:

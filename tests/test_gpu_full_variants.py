@@ -59,6 +59,14 @@ def test_1m_copy_free_and_host_buffer_steps_equal_the_materialised_path():
     pool.recall_step_host(q.pin_memory(), prm, sel3, n_sel3, view3, out_h, lse_h)
     assert torch.equal(sel3, sel) and torch.equal(view3.k, view.k) and torch.equal(view3.v, view.v)
     assert torch.equal(out_h, out.cpu()) and torch.equal(lse_h, lse.cpu())
+    # the same step with its arguments marshalled once
+    sel4, n_sel4 = torch.zeros_like(sel), torch.zeros_like(n_sel)
+    out_h2, lse_h2 = torch.zeros_like(out_h).pin_memory(), torch.zeros_like(lse_h).pin_memory()
+    step = pool.host_step(q.shape, prm, sel4, n_sel4, view3, out_h2, lse_h2)
+    step(q.pin_memory())
+    assert torch.equal(sel4, sel) and torch.equal(out_h2, out_h) and torch.equal(lse_h2, lse_h)
+    with pytest.raises(ValueError):
+        step(q[:, :1].contiguous())
     assert pool.device_status() == 0
 
 
