@@ -97,9 +97,9 @@ AttendPlan plan_attend(const kvmem_pool_config_t& c, int n_sessions, int n_q_tok
     return p;
 }
 
-int g_attend_landed = -1;     // -1: chosen in launch_attend; 0 / 1: the lookahead counts tiles not yet consumed / not yet landed
-int g_attend_lookahead = 0;   // 0: chosen in launch_attend; > 0: forced number of tiles in flight per CTA
-int g_attend_splits = 0;   // 0: chosen by the cost model below; > 0: forced (kernel-variant switch)
+Option g_attend_landed{-1};     // -1: chosen in launch_attend; 0 / 1: the lookahead counts tiles not yet consumed / not yet landed
+Option g_attend_lookahead{0};   // 0: chosen in launch_attend; > 0: forced number of tiles in flight per CTA
+Option g_attend_splits{0};   // 0: chosen by the cost model below; > 0: forced (kernel-variant switch)
 
 // splits per head: fewest waves of CTAs over the SMs, counting a fixed per-CTA cost in tiles
 static int choose_splits(int heads, int max_tiles, int sms) {
@@ -907,7 +907,7 @@ cudaError_t launch_attend(const kvmem_pool& p, int n_sessions, const __nv_bfloat
     const int RT = row_tiles_for(a.rows);
     if (a.rows > kMaxRows) return cudaErrorInvalidValue;
     if (RT > 1 && rope_first_position >= 0) return cudaErrorInvalidValue;      // the rotating modes take one row tile
-    a.n_splits = g_attend_splits > 0 ? std::min(g_attend_splits, kMaxSplits) : choose_splits(heads, (view_cap_tokens + kTile - 1) / kTile, p.sm_count);
+    a.n_splits = g_attend_splits > 0 ? std::min((int)g_attend_splits, kMaxSplits) : choose_splits(heads, (view_cap_tokens + kTile - 1) / kTile, p.sm_count);
     a.cap_tokens = view_cap_tokens;
     const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
     a.scale_log2e = sc * 1.4426950408889634f;

@@ -192,9 +192,9 @@ gather_ldst_kernel(GatherArgs a) {
     }
 }
 
-int g_pdl = 1;           // programmatic dependent launch of the step's kernels
-int g_gather_ctas = 0;    // 0: as many single-warp CTAs as fit; > 0: at most this many (kernel-variant switch)
-int g_gather_mode = 1;   // 1: TMA bulk ring, 0: ld/st
+Option g_pdl{1};           // programmatic dependent launch of the step's kernels
+Option g_gather_ctas{0};    // 0: as many single-warp CTAs as fit; > 0: at most this many (kernel-variant switch)
+Option g_gather_mode{1};   // 1: TMA bulk ring, 0: ld/st
 
 // Per session: how many slots of the new view keep their block, receive a retained block that sat elsewhere, receive an
 // incoming block (the counts of the working-set delta, Eq. "kvmem-working-set-delta").  One CTA per session.

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <atomic>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -81,16 +82,24 @@ constexpr uint64_t kMagic = 0x4b564d454d423230ull;  // "KVMEMB20"
 void set_error(const char* fmt, ...);
 
 // tuning switches (kvmem_set_option)
-extern int g_score_mode;    // 1: tensor-core decode scoring (default), 0: fp32 ALU + warp-shuffle kernel
-extern int g_chunk_poly;    // chunked scoring: every n-th exponential on the FMA pipe (0: all on the special-function unit)
-extern int g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
-extern int g_attend_landed;
-extern int g_topk_items;    // 0: the top-k kernel holds the fewest scores per thread that cover the session; 1..16: at least this many
-extern int g_topk_cluster;  // 1: sessions above 16,384 blocks are selected by a cluster of 8 CTAs (default), 0: by one CTA
-extern int g_gather_ctas;
-extern int g_attend_lookahead;
-extern int g_attend_splits; // 0: split count from the cost model (default); > 0: forced
-extern int g_pdl;           // 1: the kernels of a step are launched with programmatic stream serialization (default), 0: plain launches
+// Kernel-variant switches set by kvmem_set_option and read by every launch: process-wide, so they are atomics (relaxed:
+// a switch is an independent integer, nothing is published through it).
+struct Option {
+    std::atomic<int> v;
+    explicit constexpr Option(int x) : v(x) {}
+    operator int() const { return v.load(std::memory_order_relaxed); }
+    Option& operator=(int x) { v.store(x, std::memory_order_relaxed); return *this; }
+};
+extern Option g_score_mode;    // 1: tensor-core decode scoring (default), 0: fp32 ALU + warp-shuffle kernel
+extern Option g_chunk_poly;    // chunked scoring: every n-th exponential on the FMA pipe (0: all on the special-function unit)
+extern Option g_gather_mode;   // 1: TMA bulk ring (default), 0: 128-bit ld/st copy
+extern Option g_attend_landed;
+extern Option g_topk_items;    // 0: the top-k kernel holds the fewest scores per thread that cover the session; 1..16: at least this many
+extern Option g_topk_cluster;  // 1: sessions above 16,384 blocks are selected by a cluster of 8 CTAs (default), 0: by one CTA
+extern Option g_gather_ctas;
+extern Option g_attend_lookahead;
+extern Option g_attend_splits; // 0: split count from the cost model (default); > 0: forced
+extern Option g_pdl;           // 1: the kernels of a step are launched with programmatic stream serialization (default), 0: plain launches
 
 // Programmatic dependent launch.  A kernel launched through launch_pdl may be scheduled while the previous
 // kernel of the stream is still running; its first statement is pdl_wait(), which returns once that

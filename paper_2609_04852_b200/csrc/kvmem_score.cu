@@ -477,7 +477,7 @@ score_finish_kernel(const float* __restrict__ logits, const float2* __restrict__
     }
 }
 
-int g_score_mode = 1;   // 1: tensor-core dot products (default), 0: fp32 ALU + warp-shuffle kernel
+Option g_score_mode{1};   // 1: tensor-core dot products (default), 0: fp32 ALU + warp-shuffle kernel
 
 // index [max_sessions * L * G * max_bps rows][128] bf16 as a 2-D tensor; box = 64 dims x 128 rows, 128-byte swizzle
 static bool make_score_index_map(CUtensorMap* map, const __nv_bfloat16* index, long long index_rows) {

@@ -724,7 +724,7 @@ static bool make_index_map(PFN_cuTensorMapEncodeTiled_v12000 enc, CUtensorMap* m
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int g_chunk_poly = 4;   // every n-th exponential of the chunked passes on the FMA pipe; 0: none
+Option g_chunk_poly{4};   // every n-th exponential of the chunked passes on the FMA pipe; 0: none
 
 cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_sessions, const __nv_bfloat16* q, int M,
                                  const ChunkWorkspace& ws, float* scores, int scores_stride, float score_scale, cudaStream_t st) {

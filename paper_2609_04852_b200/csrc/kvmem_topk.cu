@@ -661,8 +661,8 @@ topk_cluster_kernel(const float* __restrict__ scores, int scores_stride, const i
     cluster.sync();                                          // nobody leaves while its shared memory may still be read
 }
 
-int g_topk_items = 0;     // 0: fewest items per thread that cover the session; 2..16: at least this many (kernel-variant switch)
-int g_topk_cluster = 1;   // sessions above 16,384 blocks: 1 = cluster of 8 CTAs, 0 = one CTA re-reading the scores
+Option g_topk_items{0};     // 0: fewest items per thread that cover the session; 2..16: at least this many (kernel-variant switch)
+Option g_topk_cluster{1};   // sessions above 16,384 blocks: 1 = cluster of 8 CTAs, 0 = one CTA re-reading the scores
 
 cudaError_t launch_topk(const kvmem_pool& p, int session_first, int n_sessions, const float* scores,
                         int scores_stride, const kvmem_select_params_t& prm, int32_t* sel_ids, int sel_stride,
