@@ -571,7 +571,9 @@ int kvmem_selftest_wait_timeout(kvmem_pool_t* pool, uint32_t limit_us, uint64_t*
  * landed in shared memory yet / that have not been consumed yet): the knobs of the bytes-in-flight sweeps; only
  * "attend_splits" can move a result, by the rounding of a different split-K merge order.
  * "pdl": 1 = the kernels of a step are launched with programmatic stream serialization, so that the
- * launch latency of each overlaps the tail of the one before (default), 0 = plain launches. */
+ * launch latency of each overlaps the tail of the one before (default), 0 = plain launches.
+ * The switches are process-wide (every pool, every thread) and atomic: a call that runs while another thread changes a
+ * switch sees either value. */
 int kvmem_set_option(const char* name /*HOST*/, int32_t value);
 
 #ifdef __cplusplus
