@@ -66,7 +66,7 @@ constexpr int kF8Pitch = kF8D + 4;               // bytes per token row of the s
 // (The rotating form is held to 64 registers: four CTAs per SM instead of three.  It is bound by the latency of its loads,
 // not by its arithmetic: 322 -> 289 us at a 1M-token history; five CTAs at 48 registers spill and take 311 us.)
 template <bool ROPE>
-__global__ void __launch_bounds__(256, ROPE ? 4 : 1)
+__global__ void __launch_bounds__(256, ROPE ? 4 : 8)
 gather_fp8_kernel(GatherF8Args a) {
     pdl_wait();
     __shared__ __align__(16) uint8_t sv[kF8Tile * kF8Pitch];
