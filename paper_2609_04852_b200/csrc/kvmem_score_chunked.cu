@@ -418,17 +418,16 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 }
 
 // Between the passes: shift = -(max + log2 Z) of every query row, merging the row statistics of all
-// tile runs and column slices; -inf switches a padding row off in pass 2.  One warp per row (a long
-// history has hundreds of partials per row): every lane folds a strided share, then a butterfly whose
-// operand order is fixed, so the result is the same bits in every lane and from run to run.
-__global__ void __launch_bounds__(256)
+// tile runs and column slices; -inf switches a padding row off in pass 2.  One THREAD per row: the partials of
+// neighbouring rows are neighbours in memory, so a warp's loads are coalesced (a warp per row read one 32-byte sector
+// per 8-byte pair), and a thread's loads are independent of one another and all in flight before the fixed-order merge.
+__global__ void __launch_bounds__(128)
 score_chunk_shift_kernel(ChunkArgs a) {
     pdl_wait();
     pdl_trigger();
     const int LG = a.L * a.G;
     const long long total = (long long)a.n_sessions * LG * a.shift_stride;
-    const long long e = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;      // one warp per row
-    const int lane = threadIdx.x & 31;
+    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;      // one thread per row
     if (e >= total) return;
     const int j = (int)(e % a.shift_stride);
     const int head = (int)(e / a.shift_stride);
@@ -440,25 +439,22 @@ score_chunk_shift_kernel(ChunkArgs a) {
         const float2* rs = a.rowstat + ((size_t)head * a.n_chunks * kCkSplit) * a.rows_pad + j;
         const int n_part = live_chunks * kCkSplit;
         float mx = -INFINITY, z = 0.0f;
-        for (int h = lane; h < n_part; h += 32) {
-            const float2 pp = rs[(size_t)h * a.rows_pad];
-            if (pp.x > -INFINITY) {
-                const float nm = fmaxf(mx, pp.x);
-                z = z * exp2f(mx - nm) + pp.y * exp2f(pp.x - nm);
-                mx = nm;
-            }
-        }
+        for (int h0 = 0; h0 < n_part; h0 += 16) {
+            float2 pp[16];
 #pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) {
-            const float om = __shfl_xor_sync(0xffffffffu, mx, o), oz = __shfl_xor_sync(0xffffffffu, z, o);
-            const float nm = fmaxf(mx, om);
-            const float za = mx > -INFINITY ? z * exp2f(mx - nm) : 0.0f, zb = om > -INFINITY ? oz * exp2f(om - nm) : 0.0f;
-            z = (lane & o) ? zb + za : za + zb;         // same operand order on both partners: identical bits in every lane
-            mx = nm;
+            for (int u = 0; u < 16; ++u) pp[u] = h0 + u < n_part ? rs[(size_t)(h0 + u) * a.rows_pad] : make_float2(-INFINITY, 0.0f);
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                if (pp[u].x > -INFINITY) {
+                    const float nm = fmaxf(mx, pp[u].x);
+                    z = z * exp2f(mx - nm) + pp[u].y * exp2f(pp[u].x - nm);
+                    mx = nm;
+                }
+            }
         }
         sh = -(mx + log2f(z));
     }
-    if (lane == 0) a.shift[e] = sh;
+    a.shift[e] = sh;
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -651,13 +647,21 @@ score_chunk_finish_kernel(const float* __restrict__ headsum, const int32_t* __re
     pdl_wait();        // everything earlier in the stream is complete and visible from here on
     pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     const int s = blockIdx.y;
-    const int NB = nblocks_dev[session_first + s];
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= NB) return;
+    if (b >= nb_pad) return;
+    // the head sums (rows of nb_pad columns: readable whatever the session's length is) are requested together with the
+    // block count
     const float* p = headsum + (size_t)s * LG * nb_pad + b;
     float total = 0.0f;
-    for (int i = 0; i < LG; ++i) total += p[(size_t)i * nb_pad];
-    scores[(size_t)s * scores_stride + b] = total * inv_LH;
+    for (int i0 = 0; i0 < LG; i0 += 8) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = i0 + u < LG ? p[(size_t)(i0 + u) * nb_pad] : 0.0f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) total += v[u];
+    }
+    const int NB = nblocks_dev[session_first + s];
+    if (b < NB) scores[(size_t)s * scores_stride + b] = total * inv_LH;
 }
 
 static PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
@@ -752,7 +756,7 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
     const int n_items2 = n_sessions * LG * a.n_bpanels;
     const int grid1 = std::min(n_items1, p.sm_count), grid2 = std::min(n_items2, p.sm_count);
     const long long n_shift = (long long)n_sessions * LG * a.shift_stride;
-    const int sgrid = (int)((n_shift * 32 + 255) / 256);             // one warp per row
+    const int sgrid = (int)((n_shift + 127) / 128);                  // one thread per row
     cudaError_t e = cudaSuccess;
 #define KVMEM_CHUNK_PASSES(POLY)                                                                                              \
     do {                                                                                                                      \
@@ -767,7 +771,7 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
         launch_pdl(score_chunk_rowstat_kernel<POLY>, dim3(grid1), dim3(kCkThreads), kCkSmem, st, q_panel, idx_tile, a);                           \
         e = cudaGetLastError();                                                                                               \
         if (e != cudaSuccess) return e;                                                                                       \
-        launch_pdl(score_chunk_shift_kernel, dim3(sgrid), dim3(256), 0, st, a);                                                                   \
+        launch_pdl(score_chunk_shift_kernel, dim3(sgrid), dim3(128), 0, st, a);                                                                   \
         e = cudaGetLastError();                                                                                               \
         if (e != cudaSuccess) return e;                                                                                       \
         launch_pdl(score_chunk_colsum_kernel<POLY>, dim3(grid2), dim3(kCkThreads), kCkSmem2, st, q_tile, idx_panel, a);                           \
