@@ -647,21 +647,13 @@ score_chunk_finish_kernel(const float* __restrict__ headsum, const int32_t* __re
     pdl_wait();        // everything earlier in the stream is complete and visible from here on
     pdl_trigger();     // the next kernel's CTAs may take their places; they wait in the same way
     const int s = blockIdx.y;
+    const int NB = nblocks_dev[session_first + s];
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= nb_pad) return;
-    // the head sums (rows of nb_pad columns: readable whatever the session's length is) are requested together with the
-    // block count
+    if (b >= NB) return;
     const float* p = headsum + (size_t)s * LG * nb_pad + b;
     float total = 0.0f;
-    for (int i0 = 0; i0 < LG; i0 += 8) {
-        float v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = i0 + u < LG ? p[(size_t)(i0 + u) * nb_pad] : 0.0f;
-#pragma unroll
-        for (int u = 0; u < 8; ++u) total += v[u];
-    }
-    const int NB = nblocks_dev[session_first + s];
-    if (b < NB) scores[(size_t)s * scores_stride + b] = total * inv_LH;
+    for (int i = 0; i < LG; ++i) total += p[(size_t)i * nb_pad];
+    scores[(size_t)s * scores_stride + b] = total * inv_LH;
 }
 
 static PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
