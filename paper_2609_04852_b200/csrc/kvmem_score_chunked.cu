@@ -418,33 +418,39 @@ score_chunk_rowstat_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 }
 
 // Between the passes: shift = -(max + log2 Z) of every query row, merging the row statistics of all
-// tile runs and column slices; -inf switches a padding row off in pass 2.  One THREAD per row: the partials of
-// neighbouring rows are neighbours in memory, so a warp's loads are coalesced (a warp per row read one 32-byte sector
-// per 8-byte pair), and a thread's loads are independent of one another and all in flight before the fixed-order merge.
-__global__ void __launch_bounds__(128)
+// tile runs and column slices; -inf switches a padding row off in pass 2.  A CTA takes 32 consecutive rows: a lane is a
+// row (the partials of neighbouring rows are neighbours in memory, so every load of a warp is one coalesced 256 bytes; a
+// warp per row read one 32-byte sector per 8-byte pair), the eight warps share out the partials (a long history has
+// hundreds per row), eight of a warp's loads are in flight at a time, and the eight partial results are merged in warp
+// order: fixed order throughout, so the same bits from run to run.
+constexpr int kCkShiftWarps = 8;
+__global__ void __launch_bounds__(32 * kCkShiftWarps)
 score_chunk_shift_kernel(ChunkArgs a) {
     pdl_wait();
     pdl_trigger();
+    __shared__ float2 part[kCkShiftWarps][32];
     const int LG = a.L * a.G;
-    const long long total = (long long)a.n_sessions * LG * a.shift_stride;
-    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;      // one thread per row
-    if (e >= total) return;
+    const long long total = (long long)a.n_sessions * LG * a.shift_stride;      // shift_stride is a multiple of 32
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long e = (long long)blockIdx.x * 32 + lane;
+    if ((long long)blockIdx.x * 32 >= total) return;
     const int j = (int)(e % a.shift_stride);
     const int head = (int)(e / a.shift_stride);
     const int NB = a.nblocks_dev[a.session_first + head / LG];
     const int n_tiles = (NB + kCkBN - 1) / kCkBN;
     const int live_chunks = (n_tiles + kCkChunkTiles - 1) / kCkChunkTiles;
-    float sh = -INFINITY;
-    if (j < a.rows && live_chunks > 0) {
+    const bool live = e < total && j < a.rows && live_chunks > 0;
+    float mx = -INFINITY, z = 0.0f;
+    if (live) {
         const float2* rs = a.rowstat + ((size_t)head * a.n_chunks * kCkSplit) * a.rows_pad + j;
         const int n_part = live_chunks * kCkSplit;
-        float mx = -INFINITY, z = 0.0f;
-        for (int h0 = 0; h0 < n_part; h0 += 16) {
-            float2 pp[16];
+        const int h_begin = (int)((long long)n_part * warp / kCkShiftWarps), h_end = (int)((long long)n_part * (warp + 1) / kCkShiftWarps);
+        for (int h0 = h_begin; h0 < h_end; h0 += 8) {
+            float2 pp[8];
 #pragma unroll
-            for (int u = 0; u < 16; ++u) pp[u] = h0 + u < n_part ? rs[(size_t)(h0 + u) * a.rows_pad] : make_float2(-INFINITY, 0.0f);
+            for (int u = 0; u < 8; ++u) pp[u] = h0 + u < h_end ? rs[(size_t)(h0 + u) * a.rows_pad] : make_float2(-INFINITY, 0.0f);
 #pragma unroll
-            for (int u = 0; u < 16; ++u) {
+            for (int u = 0; u < 8; ++u) {
                 if (pp[u].x > -INFINITY) {
                     const float nm = fmaxf(mx, pp[u].x);
                     z = z * exp2f(mx - nm) + pp[u].y * exp2f(pp[u].x - nm);
@@ -452,9 +458,22 @@ score_chunk_shift_kernel(ChunkArgs a) {
                 }
             }
         }
-        sh = -(mx + log2f(z));
     }
-    a.shift[e] = sh;
+    part[warp][lane] = make_float2(mx, z);
+    __syncthreads();
+    if (warp == 0 && e < total) {
+        float m = -INFINITY, zz = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kCkShiftWarps; ++w) {
+            const float2 p = part[w][lane];
+            if (p.x > -INFINITY) {
+                const float nm = fmaxf(m, p.x);
+                zz = zz * exp2f(m - nm) + p.y * exp2f(p.x - nm);
+                m = nm;
+            }
+        }
+        a.shift[e] = live ? -(m + log2f(zz)) : -INFINITY;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -748,7 +767,7 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
     const int n_items2 = n_sessions * LG * a.n_bpanels;
     const int grid1 = std::min(n_items1, p.sm_count), grid2 = std::min(n_items2, p.sm_count);
     const long long n_shift = (long long)n_sessions * LG * a.shift_stride;
-    const int sgrid = (int)((n_shift + 127) / 128);                  // one thread per row
+    const int sgrid = (int)((n_shift + 31) / 32);                    // 32 rows per CTA
     cudaError_t e = cudaSuccess;
 #define KVMEM_CHUNK_PASSES(POLY)                                                                                              \
     do {                                                                                                                      \
@@ -763,7 +782,7 @@ cudaError_t launch_score_chunked(const kvmem_pool& p, int session_first, int n_s
         launch_pdl(score_chunk_rowstat_kernel<POLY>, dim3(grid1), dim3(kCkThreads), kCkSmem, st, q_panel, idx_tile, a);                           \
         e = cudaGetLastError();                                                                                               \
         if (e != cudaSuccess) return e;                                                                                       \
-        launch_pdl(score_chunk_shift_kernel, dim3(sgrid), dim3(128), 0, st, a);                                                                   \
+        launch_pdl(score_chunk_shift_kernel, dim3(sgrid), dim3(32 * kCkShiftWarps), 0, st, a);                                                                   \
         e = cudaGetLastError();                                                                                               \
         if (e != cudaSuccess) return e;                                                                                       \
         launch_pdl(score_chunk_colsum_kernel<POLY>, dim3(grid2), dim3(kCkThreads), kCkSmem2, st, q_tile, idx_panel, a);                           \
