@@ -739,7 +739,8 @@ int kvmem_materialize_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_
     }
     // One pass either way: on the in-block layout every K tile is rotated by its block position on its way through shared
     // memory; raw keys are rotated by the consumer warps on their way to the tensor cores and handed back for the store.
-    // The pass walks whole 64-token tiles and fetches the rotary rows of all 64 positions of the last one.
+    // The pass walks whole 64-token tiles and fetches rotary rows up to the 49th position of the last one (the bound is
+    // kept at the whole tile).
     if (!p->cfg.rope_in_block_keys) {
         const int64_t tiles_end = (int64_t)first_position + (std::min<int64_t>((int64_t)sel_stride * p->cfg.block_tokens, view_cap_tokens) + 63) / 64 * 64;
         if (tiles_end > p->cfg.rope_max_positions) {
@@ -793,7 +794,7 @@ int kvmem_paged_attend_rope(kvmem_pool_t* p, int32_t session_first, int32_t n_se
                             float scale, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
     if (!pool_live(p)) return KVMEM_E_STATE;
     if (p->cfg.rope_max_positions <= 0) { set_error("the pool was created without rotary support"); return KVMEM_E_STATE; }
-    // the pass walks whole 64-token tiles: the last tile fetches the rotary rows of all 64 of its positions
+    // the pass walks whole 64-token tiles: the last tile fetches rotary rows up to its 49th position (bound kept at the whole tile)
     const int64_t last = (int64_t)first_position + ((int64_t)sel_stride * p->cfg.block_tokens + 63) / 64 * 64;
     if (first_position < 0 || sel_stride < 1 || last > p->cfg.rope_max_positions) {
         set_error("compact positions [%d, %lld) outside the rotary table [0, %d)", first_position, (long long)last,

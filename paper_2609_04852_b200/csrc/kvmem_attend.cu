@@ -120,10 +120,11 @@ static int choose_splits(int heads, int max_tiles, int sms) {
 //         so the view is assembled and attended in one pass: 1 read + 1 write per view byte
 //         instead of 2 reads + 1 write.
 // MODE 3: MODE 2 with position-consistent keys (Sec. 4.4: RoPE is applied to raw K at the block's compact
-//         position): the rotary rows of a tile's 64 positions ride along in a small ring of their own,
-//         and each consumer warp rotates its key fragments in registers between ldmatrix and the MMAs, with
-//         the arithmetic of kvmem_rope_rotate (fp32 products and sums, no fused multiply-add, one rounding
-//         to bf16).  The result equals attention over kvmem_materialize_rope's view and no byte is written.
+//         position): each consumer warp rotates its key fragments in registers between ldmatrix and the MMAs (one
+//         rounding to bf16), with angles composed from two table rows (the warp's first position, which comes with
+//         the tile, and the offset inside its 16 positions, loaded once per CTA: see kRopeShare above).  The result
+//         is attention over kvmem_materialize_rope's view up to that composition (a key within one bf16 step on rare
+//         elements) and no byte is written.
 // MODE 4: position-consistent keys over pages that hold k' = RoPE(k, t), t the offset inside the block: the logit
 //         q . R(p0 + t) k equals (R(-p0) q) . k', so two extra warps, taking tiles alternately, rotate the 16 query rows back by the tile's
 //         compact position p0 (one rotary row per tile instead of 64) into a small shared-memory ring, the
@@ -133,6 +134,10 @@ static int choose_splits(int heads, int max_tiles, int sms) {
 //         position p0 (one set of angles per tile, arithmetic of kvmem_rope_rotate) as soon as it has landed; the
 //         consumers and the view writer wait for the rotated tile.  The view equals kvmem_materialize_rope's and
 //         out/lse equal kvmem_view_attend's on it, with 1 read + 1 write per view byte.
+// MODE 6: MODE 1 with the keys of MODE 3 (raw keys, position-consistent view in one pass): the consumer warps rotate
+//         their key fragments as in MODE 3, write each register back to the four bytes of the swizzled tile it came from,
+//         and the view writer stores the tile once the four warps that share it have done so.  Values are copied bit for
+//         bit; keys are kvmem_materialize_rope's up to the composition of the angles.
 // MODE 2: copy-free execution view (Sec. 5.3 "Copy-free execution-view assembly"): tiles are read from
 //         the pages through the block table and attended over; no contiguous view is written.
 // RT: m16 row tiles of query rows per KV head.  RT = 1 (up to 16 rows): two groups of four consumer warps take the tiles
