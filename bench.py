@@ -61,9 +61,10 @@ def measured_tensor_peak():
 # (a bench run is never made under a profiler); the line says so in "traffic_source".
 GATHER_TRAFFIC = {"1m": 2099369984, "chunk512": 2098579520}       # gather_bulk_kernel
 # attend_split_kernel<1>, mean of six launches (128k: 134 MB read + 79 MB written; the rest of the view is still in L2 when the kernel ends)
-FUSED_TRAFFIC = {"1m": 2099538346, "128k": 213239722, "batch8": 4253410560}
+FUSED_TRAFFIC = {"1m": 2099720917, "128k": 212966016, "batch8": 4250897493}
 ROPE_FUSED_TRAFFIC = {"1m": 2098100000}   # attend_split_kernel<5> (in-block key layout)
-ROPE_GATHER_TRAFFIC = {"1m": 2298386176}  # gather_rope_kernel
+ROPE_RAW_FUSED_TRAFFIC = {"1m": 2105828736}   # attend_split_kernel<6> (raw keys, one pass), mean of two launches
+ROPE_GATHER_TRAFFIC = {"1m": 2270831360}  # gather_rope_kernel, mean of two launches
 TRAFFIC_SOURCE = ("constant from an earlier ncu capture of this kernel on this workload (one launch, "
                   "dram__bytes_read.sum + dram__bytes_write.sum); not measured in this run")
 
@@ -492,7 +493,7 @@ def run_native(args):
                          "frac": gather_gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                          "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": gather_s * 1e3,
                          "traffic": None if args.paged else ROPE_FUSED_TRAFFIC.get(base.name) if args.rope and args.in_block and not args.unfused else
-                                    None if args.rope and not args.unfused else
+                                    ROPE_RAW_FUSED_TRAFFIC.get(base.name) if args.rope and not args.unfused else
                                     ROPE_GATHER_TRAFFIC.get(base.name) if args.rope else
                                     FUSED_TRAFFIC.get(base.name) if fused else GATHER_TRAFFIC.get(base.name)},
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes,
